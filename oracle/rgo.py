@@ -1,0 +1,225 @@
+"""ctypes front end of the CPU oracle (``oracle/rgo.cpp``).
+
+TEST INFRASTRUCTURE ONLY: tests, the smoke check and the benchmark's
+cpu_baseline / reference legs may import this module; the product package never
+does.  Arrays are numpy; bf16 values travel as ``uint16`` bit patterns.
+
+The functions mirror the C interface one to one; every arithmetic step happens
+in the C++ file, which cites the paper passage it follows.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rgo.cpp")
+_LIB = os.path.join(_HERE, "librgo.so")
+
+BF16, F32 = 0, 1
+TREE_LEFT, TREE_BALANCED = 0, 1
+OP_SUM, OP_RMSNORM, OP_SOFTMAX_DENOM = 0, 1, 2
+ATOM_EXACT_RN, ATOM_SEQ, ATOM_ALIGN_TRUNC = 0, 1, 2
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no fast-math, no contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
+               "-fPIC", "-shared", "-o", _LIB, _SRC]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+class _AtomStruct(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "model", "atom_k", "fma", "group", "window_bits", "exp_mode", "acc_in_window",
+        "addend_round", "final_round")]
+
+
+@dataclass(frozen=True)
+class AtomModel:
+    """The matrix-instruction step (Sec. 3.2.1).  ``EXACT_RN`` is the semantics the
+    paper assumes; ``SEQ`` the scalar path; ``ALIGN_TRUNC`` the probe-fitted family."""
+    model: int = ATOM_EXACT_RN
+    atom_k: int = 16
+    fma: int = 1
+    group: int = 16
+    window_bits: int = 90
+    exp_mode: int = 0
+    acc_in_window: int = 1
+    addend_round: int = 0
+    final_round: int = 1
+
+    def c(self) -> _AtomStruct:
+        return _AtomStruct(self.model, self.atom_k, self.fma, self.group, self.window_bits,
+                           self.exp_mode, self.acc_in_window, self.addend_round, self.final_round)
+
+
+EXACT_RN = AtomModel(model=ATOM_EXACT_RN)
+SEQ_FMA = AtomModel(model=ATOM_SEQ, atom_k=1, fma=1)
+SEQ_NOFMA = AtomModel(model=ATOM_SEQ, atom_k=1, fma=0)
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        f32, i32, i64, vp = C.c_float, C.c_int32, C.c_int64, C.c_void_p
+        L.rgo_num_threads.restype = i32
+        L.rgo_bf16_to_f32.restype = f32; L.rgo_bf16_to_f32.argtypes = [C.c_uint16]
+        L.rgo_f32_to_bf16.restype = C.c_uint16; L.rgo_f32_to_bf16.argtypes = [f32]
+        for n in ("rgo_add_f32", "rgo_mul_f32"):
+            getattr(L, n).restype = f32; getattr(L, n).argtypes = [f32, f32]
+        for n in ("rgo_expf", "rgo_silu"):
+            getattr(L, n).restype = f32; getattr(L, n).argtypes = [f32]
+        L.rgo_tree_sum.restype = f32; L.rgo_tree_sum.argtypes = [vp, i64, i32]
+        L.rgo_atom.restype = f32; L.rgo_atom.argtypes = [C.POINTER(_AtomStruct), f32, vp, vp, i32]
+        L.rgo_gemm.restype = None
+        L.rgo_gemm.argtypes = [C.POINTER(_AtomStruct), i32, i32, vp, i64, i64, i64, vp, i64, vp, i64,
+                               vp, i32, i64, vp, i32, i32, vp, i32, i64]
+        L.rgo_gemm_samples.restype = None
+        L.rgo_gemm_samples.argtypes = [C.POINTER(_AtomStruct), i32, i32, vp, i64, vp, i64, vp, i64,
+                                       i32, vp, i32, i32, vp, i32, i64, i64, vp, vp, vp]
+        L.rgo_gemm_partials.restype = None
+        L.rgo_gemm_partials.argtypes = [C.POINTER(_AtomStruct), i32, vp, i64, i64, i64, vp, i64, vp, i64, vp]
+        L.rgo_reduce_rows.restype = None
+        L.rgo_reduce_rows.argtypes = [i32, i32, i32, vp, i32, i64, i64, i64, vp, i32, i64, vp, i32, f32, vp]
+        _lib = L
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().rgo_num_threads())
+
+
+# ----------------------------------------------------------------- primitives
+def bf16_to_f32(h: int) -> float:
+    return float(lib().rgo_bf16_to_f32(int(h)))
+
+
+def f32_to_bf16(f) -> int:
+    return int(lib().rgo_f32_to_bf16(np.float32(f)))
+
+
+def add_f32(a, b) -> np.float32:
+    return np.float32(lib().rgo_add_f32(np.float32(a), np.float32(b)))
+
+
+def mul_f32(a, b) -> np.float32:
+    return np.float32(lib().rgo_mul_f32(np.float32(a), np.float32(b)))
+
+
+def expf(x) -> np.float32:
+    return np.float32(lib().rgo_expf(np.float32(x)))
+
+
+def silu(x) -> np.float32:
+    return np.float32(lib().rgo_silu(np.float32(x)))
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _dtype_code(a: np.ndarray) -> int:
+    if a.dtype == np.uint16:
+        return BF16
+    if a.dtype == np.float32:
+        return F32
+    raise TypeError(f"oracle arrays are uint16 (bf16 bits) or float32, got {a.dtype}")
+
+
+def tree_sum(v, tree: int = TREE_BALANCED) -> np.float32:
+    v = np.ascontiguousarray(v, dtype=np.float32)
+    return np.float32(lib().rgo_tree_sum(_ptr(v), v.size, tree))
+
+
+def atom(model: AtomModel, acc, a_bits, b_bits) -> np.float32:
+    a = np.ascontiguousarray(a_bits, dtype=np.uint16)
+    b = np.ascontiguousarray(b_bits, dtype=np.uint16)
+    assert a.size == b.size <= 64
+    m = model.c()
+    return np.float32(lib().rgo_atom(C.byref(m), np.float32(acc), _ptr(a), _ptr(b), a.size))
+
+
+def _cuts(cuts):
+    c = np.ascontiguousarray(list(cuts) if cuts is not None else [], dtype=np.int64)
+    return c
+
+
+def _epi(bias, residual):
+    b = None if bias is None else np.ascontiguousarray(bias)
+    r = None if residual is None else np.ascontiguousarray(residual)
+    return (b, _dtype_code(b) if b is not None else 0,
+            r, _dtype_code(r) if r is not None else 0, r.shape[1] if r is not None else 0)
+
+
+def gemm(A, B, *, cuts=(), tree=TREE_BALANCED, atom_model: AtomModel = EXACT_RN, out_dtype=BF16,
+         bias=None, act=0, residual=None) -> np.ndarray:
+    """C = epilogue(A @ B.T) per the descriptor semantics (Sec. 3.2.2).
+    A [M,K], B [N,K] are uint16 bf16 bit patterns.  Returns uint16 (bf16) or float32."""
+    A = np.ascontiguousarray(A, dtype=np.uint16); B = np.ascontiguousarray(B, dtype=np.uint16)
+    M, K = A.shape; N, K2 = B.shape
+    assert K == K2
+    c = _cuts(cuts)
+    out = np.empty((M, N), dtype=np.uint16 if out_dtype == BF16 else np.float32)
+    b, bd, r, rd, ldr = _epi(bias, residual)
+    m = atom_model.c()
+    lib().rgo_gemm(C.byref(m), tree, c.size, _ptr(c), M, N, K, _ptr(A), K, _ptr(B), K,
+                   _ptr(out), out_dtype, N, _ptr(b), bd, act, _ptr(r), rd, ldr)
+    return out
+
+
+def gemm_samples(A, B, si, sj, *, cuts=(), tree=TREE_BALANCED, atom_model: AtomModel = EXACT_RN,
+                 out_dtype=BF16, bias=None, act=0, residual=None) -> np.ndarray:
+    """Output elements (si[t], sj[t]) only; returned as float32 after the output rounding."""
+    A = np.ascontiguousarray(A, dtype=np.uint16); B = np.ascontiguousarray(B, dtype=np.uint16)
+    K = A.shape[1]
+    si = np.ascontiguousarray(si, dtype=np.int64); sj = np.ascontiguousarray(sj, dtype=np.int64)
+    c = _cuts(cuts)
+    out = np.empty(si.size, dtype=np.float32)
+    b, bd, r, rd, ldr = _epi(bias, residual)
+    m = atom_model.c()
+    lib().rgo_gemm_samples(C.byref(m), tree, c.size, _ptr(c), K, _ptr(A), K, _ptr(B), K, out_dtype,
+                           _ptr(b), bd, act, _ptr(r), rd, ldr, si.size, _ptr(si), _ptr(sj), _ptr(out))
+    return out
+
+
+def gemm_partials(A, B, *, cuts=(), atom_model: AtomModel = EXACT_RN) -> np.ndarray:
+    """fp32 partial of every part, shape [S, M, N] (Sec. 3.2.2, split-K)."""
+    A = np.ascontiguousarray(A, dtype=np.uint16); B = np.ascontiguousarray(B, dtype=np.uint16)
+    M, K = A.shape; N = B.shape[0]
+    c = _cuts(cuts)
+    P = np.empty((c.size + 1, M, N), dtype=np.float32)
+    m = atom_model.c()
+    lib().rgo_gemm_partials(C.byref(m), c.size, _ptr(c), M, N, K, _ptr(A), K, _ptr(B), K, _ptr(P))
+    return P
+
+
+def reduce_rows(op: int, x, *, tree=TREE_BALANCED, fma=0, weight=None, eps=0.0, out_dtype=None):
+    """Row reductions.  Returns (out, aux): sum -> ([R] f32, None); rmsnorm -> ([R,C] y, rinv[R]);
+    softmax normaliser -> (Z[R] f32, rowmax[R])."""
+    x = np.ascontiguousarray(x)
+    R, Cc = x.shape
+    xd = _dtype_code(x)
+    aux = np.empty(R, dtype=np.float32)
+    w = None if weight is None else np.ascontiguousarray(weight)
+    wd = _dtype_code(w) if w is not None else 0
+    if op == OP_RMSNORM:
+        od = xd if out_dtype is None else out_dtype
+        out = np.empty((R, Cc), dtype=np.uint16 if od == BF16 else np.float32)
+        ldo = Cc
+    else:
+        od = F32
+        out = np.empty(R, dtype=np.float32)
+        ldo = 1
+    lib().rgo_reduce_rows(op, tree, fma, _ptr(x), xd, R, Cc, Cc, _ptr(out), od, ldo,
+                          _ptr(w), wd, np.float32(eps), _ptr(aux))
+    return out, (None if op == OP_SUM else aux)

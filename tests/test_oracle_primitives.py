@@ -1,0 +1,98 @@
+"""Pins for the oracle's primitives: conversions, single fp32 operations, the specified exp."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import rgo
+
+
+def test_bf16_widening_exhaustive():
+    # every one of the 65,536 patterns: bf16 is the top half of binary32
+    for h in range(0, 65536, 1):
+        f = np.float32(rgo.lib().rgo_bf16_to_f32(h))
+        assert f.view(np.uint32) == np.uint32(h << 16) or (math.isnan(f) and (h & 0x7fff) > 0x7f80)
+
+
+def test_bf16_round_trip_exhaustive():
+    for h in range(65536):
+        if (h & 0x7fff) > 0x7f80:
+            continue
+        f = np.uint32(h << 16).view(np.float32)
+        assert rgo.f32_to_bf16(f) == h
+
+
+def test_bf16_narrowing_matches_library_rne():
+    # independent route: torch's CPU conversion is round-to-nearest-even
+    g = np.random.default_rng(0)
+    x = g.standard_normal(200000).astype(np.float32) * np.exp2(g.integers(-60, 60, 200000)).astype(np.float32)
+    # exact ties and their neighbours
+    base = (g.integers(0, 0x7f7f, 20000).astype(np.uint32) << 16)
+    ties = np.concatenate([base | 0x8000, (base | 0x8000) + 1, (base | 0x8000) - 1]).astype(np.uint32).view(np.float32)
+    x = np.concatenate([x, ties, -ties])
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    got = np.array([rgo.f32_to_bf16(v) for v in x], dtype=np.uint16)
+    assert np.array_equal(got, want)
+
+
+def test_tie_goes_to_even():
+    # 1 + 2^-8 is exactly between bf16(1) and bf16(1 + 2^-7): even mantissa wins
+    assert rgo.f32_to_bf16(np.float32(1 + 2.0 ** -8)) == 0x3F80
+    assert rgo.f32_to_bf16(np.float32(1 + 2.0 ** -7 + 2.0 ** -8)) == 0x3F82
+
+
+def test_add_mul_single_rounding():
+    # double arithmetic then one rounding equals a correctly rounded fp32 add / mul
+    g = np.random.default_rng(1)
+    a = (g.standard_normal(50000) * np.exp2(g.integers(-30, 30, 50000))).astype(np.float32)
+    b = (g.standard_normal(50000) * np.exp2(g.integers(-30, 30, 50000))).astype(np.float32)
+    for x, y in zip(a[:20000], b[:20000]):
+        assert rgo.add_f32(x, y) == np.float32(np.float64(x) + np.float64(y))
+        assert rgo.mul_f32(x, y) == np.float32(np.float64(x) * np.float64(y))
+    assert (np.float32(1.0) + np.float32(2.0 ** -24)) == np.float32(1.0)  # tie to even
+    assert rgo.add_f32(1.0, 2.0 ** -24) == np.float32(1.0)
+    assert rgo.add_f32(1.0 + 2.0 ** -23, 2.0 ** -24) == np.float32(1.0 + 2.0 ** -22)
+    # -0 is the additive identity, +0 is not
+    assert np.signbit(rgo.add_f32(-0.0, -0.0)) and not np.signbit(rgo.add_f32(-0.0, 0.0))
+
+
+def _ulp_err(got: float, exact: float) -> float:
+    if exact == 0:
+        return abs(got)
+    e = math.floor(math.log2(abs(exact)))
+    ulp = 2.0 ** (max(e, -126) - 23)
+    return abs(float(got) - exact) / ulp
+
+
+def test_expf_accuracy_monotone_and_clamps():
+    xs = np.linspace(-87.3, 88.7, 200001).astype(np.float32)
+    prev = -1.0
+    worst = 0.0
+    for x in xs:
+        y = float(rgo.expf(x))
+        worst = max(worst, _ulp_err(y, math.exp(float(x))))
+        assert y >= prev
+        prev = y
+    assert worst <= 2.0, worst
+    assert rgo.expf(0.0) == np.float32(1.0)
+    assert rgo.expf(-0.0) == np.float32(1.0)
+    assert rgo.expf(89.0) == np.float32(np.inf)
+    assert rgo.expf(-88.0) == np.float32(0.0)
+    assert rgo.expf(-1e30) == np.float32(0.0)
+    assert math.isnan(float(rgo.expf(np.float32(np.nan))))
+    # dense around zero and around the reduction boundaries n*ln2/2
+    for k in range(-60, 61):
+        for d in (-3e-7, 0.0, 3e-7):
+            x = np.float32(k * 0.34657359 + d)
+            assert _ulp_err(float(rgo.expf(x)), math.exp(float(x))) <= 2.0
+
+
+def test_silu():
+    assert rgo.silu(0.0) == np.float32(0.0)
+    xs = np.linspace(-30, 30, 20001).astype(np.float32)
+    for x in xs:
+        want = float(x) / (1.0 + math.exp(-float(x)))
+        assert _ulp_err(float(rgo.silu(x)), want) <= 4.0
+    assert rgo.silu(-200.0) == np.float32(-0.0)  # x / inf
+    assert rgo.silu(200.0) == np.float32(200.0)
