@@ -1,0 +1,187 @@
+/* rg — reduction-order-fixed GEMM and row reductions for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every result's bits are decided by a reduction-order descriptor and by nothing
+ * else: not by the tile shape, the batch size M, the launch, or the run.  The descriptor is
+ * the frozen record of every order-deciding factor (paper Sec. 3.2.2 "GEMM computation
+ * descriptor", Sec. 4: "two equal records owe each other the same bits"); tile sizes,
+ * pipeline depth and warp roles are speed knobs that leave the dependence tree alone
+ * (Sec. 3.1 "Pipeline depth leaves the tree alone", "Warp specialization leaves it alone";
+ * Sec. 3.2.2 "What tiles the output stays out of all three").
+ *
+ * Conventions
+ *   - Pointers named in rg_tensor_t / rg_epilogue_t / rg_reduce_args_t are DEVICE pointers
+ *     unless a function says "host".  The caller owns every buffer.  No function here
+ *     allocates or frees device memory, and none synchronises the device or the stream,
+ *     except rg_device_status (which reads a word back) and entry points that say otherwise.
+ *   - Matrices are row-major; `ld` is the distance between rows in ELEMENTS.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Every call validates all of its arguments before launching anything; a call that
+ *     returns an error has launched nothing.  A well-formed request the kernels cannot honour
+ *     returns RG_ERR_UNSUPPORTED rather than silently computing in a different order.
+ *   - No exceptions cross this boundary and there is no global state that changes arithmetic.
+ */
+#ifndef RG_H_
+#define RG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RG_OK = 0,
+  RG_ERR_NULL = 1,          /* a required pointer is NULL */
+  RG_ERR_INVALID_DESC = 2,  /* descriptor malformed (size, enum range, cuts not increasing, ...) */
+  RG_ERR_UNSUPPORTED = 3,   /* well-formed, but no kernel here realises it */
+  RG_ERR_SHAPE = 4,         /* tensor shapes disagree or are out of range */
+  RG_ERR_ALIGNMENT = 5,     /* pointer or leading dimension breaks a 16-byte rule */
+  RG_ERR_WORKSPACE = 6,     /* workspace missing or too small */
+  RG_ERR_CUDA = 7,          /* the CUDA runtime or driver reported an error */
+  RG_ERR_TIMEOUT = 8        /* a bounded device-side wait gave up (see rg_device_status) */
+} rg_status_t;
+
+typedef enum { RG_BF16 = 0, RG_F32 = 1 } rg_dtype_t;
+
+/* The tree that combines values (split-K partials in rg_gemm, the leaves of a row in
+ * rg_reduce_rows).  Sec. 3.1: a reduction order is a binary tree up to swapping an addition's
+ * inputs.  LEFT = ((v0+v1)+v2)+...; BALANCED = neighbours pair first, level by level, an
+ * unpaired last value moves up unchanged: the tree a count-up butterfly builds over the logical
+ * element order (Sec. 5.1, Fig. 3), height ceil(log2 n). */
+typedef enum { RG_TREE_LEFT = 0, RG_TREE_BALANCED = 1 } rg_tree_t;
+
+/* Which instruction folds products into the accumulator and how many per rounding step
+ * (`instruction_k`, Sec. 3.2.1/3.2.2).  TC_BF16_K16: one tcgen05.mma kind::f16 step of 16
+ * bf16 products, accumulator fp32 in tensor memory, steps chained in ascending k (App. E).
+ * SCALAR names the fma-chain path; no kernel here implements it. */
+typedef enum { RG_ATOM_TC_BF16_K16 = 0, RG_ATOM_SCALAR = 1 } rg_atom_t;
+
+#define RG_MAX_CUTS 63
+
+typedef struct {
+  uint32_t size;          /* = sizeof(rg_desc_t) */
+  /* ---- speed knobs: validated, NOT part of the class key (Sec. 3.2.2) ---- */
+  uint16_t BM, BN, BK;    /* output tile and K step per pipeline stage; 0 = library default */
+  uint8_t stages;         /* shared-memory ring depth; 0 = as many as fit */
+  uint8_t cta_group;      /* 1, or 2 (pair of SMs on one 256-row tile); 0 = default */
+  uint8_t raster;         /* tile walk: 0 = default grouped-M swizzle, 1 = row-major */
+  uint8_t _pad0;
+  /* ---- order-deciding fields: these ARE the class key ---- */
+  uint8_t in_dtype;       /* rg_dtype_t of A and B: RG_BF16 */
+  uint8_t acc_dtype;      /* accumulator: RG_F32 */
+  uint8_t partial_dtype;  /* type a finished split-K part is written at: RG_F32 (Sec. 3.2.2) */
+  uint8_t merge_dtype;    /* type the parts are summed at: RG_F32 */
+  uint8_t atom;           /* rg_atom_t */
+  uint8_t k_tail;         /* 0 = the short K turn runs last, missing products are absent */
+  uint8_t fma;            /* multiply-add fusion on scalar leaves (reductions: x*x feeding an add) */
+  uint8_t tree;           /* rg_tree_t */
+  uint32_t n_cuts;        /* split-K: number of interior cut points (0 = plain GEMM) */
+  uint32_t cuts[RG_MAX_CUTS]; /* 0 < cuts[0] < ... < cuts[n_cuts-1] < K; part s = [cuts[s-1], cuts[s]) */
+} rg_desc_t;
+
+/* A row-major matrix in device memory. */
+typedef struct {
+  void* ptr;
+  int32_t dtype;          /* rg_dtype_t */
+  int64_t rows, cols;
+  int64_t ld;             /* elements between consecutive rows, >= cols */
+} rg_tensor_t;
+
+/* Fused epilogue, applied in this fixed order in fp32 with one rounding at the very end
+ * (where the rounding to the output type falls is part of the order, Sec. 2):
+ *   v = merged accumulator;  v += bias[j];  v = silu(v);  v += residual[i, j];  C = round(v). */
+typedef struct {
+  const void* bias;       /* [N], nullable */
+  int32_t bias_dtype;
+  int32_t act;            /* 0 none, 1 SiLU: v / (1 + rg_exp(-v)) */
+  const void* residual;   /* [M, N], nullable */
+  int32_t residual_dtype;
+  int64_t ldr;
+} rg_epilogue_t;
+
+typedef enum { RG_OP_SUM = 0, RG_OP_RMSNORM = 1, RG_OP_SOFTMAX_DENOM = 2 } rg_reduce_op_t;
+
+typedef struct {
+  const void* weight;     /* RMSNorm: [cols], nullable (= all ones) */
+  int32_t weight_dtype;
+  float eps;              /* RMSNorm: added to the mean square inside the square root */
+  void* aux_out;          /* SOFTMAX_DENOM: row maxima [rows] fp32; RMSNorm: 1/rms [rows] fp32; nullable */
+} rg_reduce_args_t;
+
+/* Fill *d with the library defaults: bf16 in, fp32 accumulate/partial/merge, tensor-core atom,
+ * balanced tree, no cuts, all speed knobs 0. */
+void rg_desc_init(rg_desc_t* d);
+
+/* Check a descriptor against a GEMM shape (Sec. 3.2.2: cuts are contiguous parts of the
+ * contracted axis).  Host only.  Cuts must be strictly increasing multiples of 16 inside (0, K). */
+rg_status_t rg_desc_validate(const rg_desc_t* d, int64_t M, int64_t N, int64_t K);
+
+/* Equivalence-class key (Sec. 4: a descriptor holds every order-deciding factor "and nothing
+ * else"; Sec. 6: configs that differ only in tiling form one class).  A 64-bit hash of the
+ * canonical serialisation of the order-deciding fields; BM/BN/BK/stages/cta_group/raster and
+ * the epilogue are excluded.  Returns 0 for a malformed descriptor.  Host only. */
+uint64_t rg_desc_class(const rg_desc_t* d);
+
+/* Bytes of fp32 workspace rg_gemm needs: 0 without cuts, else (n_cuts+1) * M * roundup(N,4) * 4. */
+size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N);
+
+/* C[M,N] = epilogue( merge_s( sum_{k in part s} A[i,k] * B[j,k] ) )   (C = A * B^T).
+ *
+ * Sec. 3.2.2 "Plain GEMM" and "Split-K"; Sec. 3.2.1 for the step; App. E for the chaining:
+ * per output element and per part, the accumulator starts at zero and takes one tensor-core
+ * step per 16 consecutive k, in ascending k; a finished part is an fp32 value; the parts are
+ * added in the descriptor's tree; then the epilogue.  Without cuts one kernel does everything;
+ * with cuts the parts go to `ws` as fp32 [part][M][roundup(N,4)] and a second kernel merges
+ * them (no atomics anywhere).
+ *
+ *   A: [M,K] bf16, B: [N,K] bf16 (both K-contiguous), C: [M,N] bf16 or fp32.
+ *   A.ptr, B.ptr 16-byte aligned; A.ld, B.ld multiples of 8.  C, bias, residual: any alignment.
+ *   epi: nullable.  ws: device, 16-byte aligned, >= rg_gemm_workspace_bytes; contents undefined
+ *   afterwards; may be NULL when there are no cuts.
+ *   M == 0 or N == 0: returns RG_OK and launches nothing.  K == 0: RG_ERR_SHAPE.
+ * Asynchronous on `cuda_stream`. */
+rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
+                    const rg_epilogue_t* epi, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Row reductions with a fixed tree over the columns (Sec. 3.1, Sec. 5.1; kernels named in
+ * Sec. 7: row sums, softmax, rmsnorm).  `d->tree` (BALANCED only on the GPU), `d->acc_dtype`
+ * (fp32) and `d->fma` apply; the leaves are the `x.cols` columns in index order.
+ *   RG_OP_SUM:           out[r] = TREE(f32(x[r,:]));            out: rows x 1 fp32
+ *   RG_OP_RMSNORM:       ss = TREE(x*x); rinv = 1/sqrt(ss/cols + eps);
+ *                        y[r,c] = round((x*rinv)*w[c]);           out: rows x cols, bf16 or fp32
+ *   RG_OP_SOFTMAX_DENOM: m = max_c x; out[r] = TREE(rg_exp(x - m)); out: rows x 1 fp32;
+ *                        args->aux_out (nullable) receives m.
+ * x: bf16 or fp32.  rows == 0: RG_OK, nothing launched.  cols == 0: RG_ERR_SHAPE.
+ * Asynchronous on `cuda_stream`. */
+rg_status_t rg_reduce_rows(const rg_desc_t* d, rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out,
+                           const rg_reduce_args_t* args, void* cuda_stream);
+
+/* Host-buffer forms of the two calls above, for callers whose data lives in host memory.
+ * Every tensor / epilogue / args pointer is a HOST pointer (pinned memory makes the copies
+ * asynchronous).  `dev_scratch` is a caller-owned DEVICE buffer of at least
+ * rg_*_host_scratch_bytes(...) bytes, 256-byte aligned, that the call uses for the device
+ * copies of its operands, its result and the split-K workspace.  Each call enqueues the
+ * host-to-device copies, the kernels and the device-to-host copy of the result on
+ * `cuda_stream` and returns without synchronising. */
+size_t rg_gemm_host_scratch_bytes(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, int32_t c_dtype,
+                                  const rg_epilogue_t* epi);
+rg_status_t rg_gemm_host(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
+                         const rg_epilogue_t* epi, void* dev_scratch, size_t dev_scratch_bytes, void* cuda_stream);
+size_t rg_reduce_rows_host_scratch_bytes(rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out);
+rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out,
+                                const rg_reduce_args_t* args, void* dev_scratch, size_t dev_scratch_bytes,
+                                void* cuda_stream);
+
+/* Device-side health word of the current device.  Every wait inside the kernels is bounded; a
+ * wait that gives up records a code here, lets the kernel drain and return, and leaves the
+ * context usable.  Copies the word to *code (0 = healthy) and clears it.  Synchronises the
+ * device.  Returns RG_ERR_TIMEOUT if the word was non-zero. */
+rg_status_t rg_device_status(uint32_t* code);
+
+const char* rg_status_string(rg_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RG_H_ */

@@ -1,0 +1,79 @@
+"""ctypes mirror of include/rg.h: structures, prototypes and the loader.
+
+Argument marshalling only.  If the CUDA library has not been built the loader raises; there is
+no fallback path of any kind.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librg.so")
+
+RG_OK = 0
+STATUS_NAMES = {0: "RG_OK", 1: "RG_ERR_NULL", 2: "RG_ERR_INVALID_DESC", 3: "RG_ERR_UNSUPPORTED", 4: "RG_ERR_SHAPE",
+                5: "RG_ERR_ALIGNMENT", 6: "RG_ERR_WORKSPACE", 7: "RG_ERR_CUDA", 8: "RG_ERR_TIMEOUT"}
+RG_BF16, RG_F32 = 0, 1
+RG_TREE_LEFT, RG_TREE_BALANCED = 0, 1
+RG_ATOM_TC_BF16_K16, RG_ATOM_SCALAR = 0, 1
+RG_OP_SUM, RG_OP_RMSNORM, RG_OP_SOFTMAX_DENOM = 0, 1, 2
+RG_MAX_CUTS = 63
+
+# every symbol include/rg.h declares
+EXPORTS = ["rg_desc_init", "rg_desc_validate", "rg_desc_class", "rg_gemm_workspace_bytes", "rg_gemm",
+           "rg_reduce_rows", "rg_gemm_host_scratch_bytes", "rg_gemm_host", "rg_reduce_rows_host_scratch_bytes",
+           "rg_reduce_rows_host", "rg_device_status", "rg_status_string"]
+
+
+class rg_desc_t(C.Structure):
+    _fields_ = [("size", C.c_uint32),
+                ("BM", C.c_uint16), ("BN", C.c_uint16), ("BK", C.c_uint16),
+                ("stages", C.c_uint8), ("cta_group", C.c_uint8), ("raster", C.c_uint8), ("_pad0", C.c_uint8),
+                ("in_dtype", C.c_uint8), ("acc_dtype", C.c_uint8), ("partial_dtype", C.c_uint8), ("merge_dtype", C.c_uint8),
+                ("atom", C.c_uint8), ("k_tail", C.c_uint8), ("fma", C.c_uint8), ("tree", C.c_uint8),
+                ("n_cuts", C.c_uint32), ("cuts", C.c_uint32 * RG_MAX_CUTS)]
+
+
+class rg_tensor_t(C.Structure):
+    _fields_ = [("ptr", C.c_void_p), ("dtype", C.c_int32), ("rows", C.c_int64), ("cols", C.c_int64), ("ld", C.c_int64)]
+
+
+class rg_epilogue_t(C.Structure):
+    _fields_ = [("bias", C.c_void_p), ("bias_dtype", C.c_int32), ("act", C.c_int32),
+                ("residual", C.c_void_p), ("residual_dtype", C.c_int32), ("ldr", C.c_int64)]
+
+
+class rg_reduce_args_t(C.Structure):
+    _fields_ = [("weight", C.c_void_p), ("weight_dtype", C.c_int32), ("eps", C.c_float), ("aux_out", C.c_void_p)]
+
+
+_lib = None
+
+
+def load():
+    """Load librg.so.  Raises if it is missing: the product has no other path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build the CUDA library first "
+            "(python -m paper_2609_11356_b200.build, or __graft_entry__.build()).")
+    L = C.CDLL(LIB_PATH)
+    D, T, E, A = C.POINTER(rg_desc_t), C.POINTER(rg_tensor_t), C.POINTER(rg_epilogue_t), C.POINTER(rg_reduce_args_t)
+    i64, vp, sz = C.c_int64, C.c_void_p, C.c_size_t
+    L.rg_desc_init.restype = None; L.rg_desc_init.argtypes = [D]
+    L.rg_desc_validate.restype = C.c_int; L.rg_desc_validate.argtypes = [D, i64, i64, i64]
+    L.rg_desc_class.restype = C.c_uint64; L.rg_desc_class.argtypes = [D]
+    L.rg_gemm_workspace_bytes.restype = sz; L.rg_gemm_workspace_bytes.argtypes = [D, i64, i64]
+    L.rg_gemm.restype = C.c_int; L.rg_gemm.argtypes = [D, T, T, T, E, vp, sz, vp]
+    L.rg_reduce_rows.restype = C.c_int; L.rg_reduce_rows.argtypes = [D, C.c_int, T, T, A, vp]
+    L.rg_gemm_host_scratch_bytes.restype = sz; L.rg_gemm_host_scratch_bytes.argtypes = [D, i64, i64, i64, C.c_int32, E]
+    L.rg_gemm_host.restype = C.c_int; L.rg_gemm_host.argtypes = [D, T, T, T, E, vp, sz, vp]
+    L.rg_reduce_rows_host_scratch_bytes.restype = sz; L.rg_reduce_rows_host_scratch_bytes.argtypes = [C.c_int, T, T]
+    L.rg_reduce_rows_host.restype = C.c_int; L.rg_reduce_rows_host.argtypes = [D, C.c_int, T, T, A, vp, sz, vp]
+    L.rg_device_status.restype = C.c_int; L.rg_device_status.argtypes = [C.POINTER(C.c_uint32)]
+    L.rg_status_string.restype = C.c_char_p; L.rg_status_string.argtypes = [C.c_int]
+    _lib = L
+    return L

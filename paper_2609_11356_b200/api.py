@@ -1,0 +1,162 @@
+"""Python names for the C entry points (same names, argument marshalling only)."""
+from __future__ import annotations
+
+import ctypes as C
+from typing import Optional, Sequence
+
+from . import _cabi as K
+
+
+class RgError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = K.load().rg_status_string(status).decode()
+        super().__init__(f"{where}: {K.STATUS_NAMES.get(status, status)} ({msg})")
+
+
+def _check(status: int, where: str):
+    if status != K.RG_OK:
+        raise RgError(status, where)
+
+
+def rg_desc(*, cuts: Sequence[int] = (), tree: int = K.RG_TREE_BALANCED, fma: int = 0, BM: int = 0, BN: int = 0,
+            BK: int = 0, stages: int = 0, cta_group: int = 0, raster: int = 0, **order_fields) -> K.rg_desc_t:
+    """A descriptor with the library defaults (rg_desc_init), then the given fields."""
+    d = K.rg_desc_t()
+    K.load().rg_desc_init(C.byref(d))
+    d.BM, d.BN, d.BK, d.stages, d.cta_group, d.raster = BM, BN, BK, stages, cta_group, raster
+    d.tree, d.fma = tree, fma
+    for k, v in order_fields.items():
+        setattr(d, k, v)
+    cuts = list(cuts)
+    if len(cuts) > K.RG_MAX_CUTS:
+        raise RgError(2, "rg_desc")
+    d.n_cuts = len(cuts)
+    for i, c in enumerate(cuts):
+        d.cuts[i] = int(c)
+    return d
+
+
+def rg_desc_validate(d: K.rg_desc_t, M: int, N: int, Kdim: int) -> int:
+    return int(K.load().rg_desc_validate(C.byref(d), M, N, Kdim))
+
+
+def rg_desc_class(d: K.rg_desc_t) -> int:
+    return int(K.load().rg_desc_class(C.byref(d)))
+
+
+def rg_gemm_workspace_bytes(d: K.rg_desc_t, M: int, N: int) -> int:
+    return int(K.load().rg_gemm_workspace_bytes(C.byref(d), M, N))
+
+
+def rg_status_string(status: int) -> str:
+    return K.load().rg_status_string(status).decode()
+
+
+def rg_device_status() -> int:
+    """Read and clear the device health word (synchronises).  0 = healthy."""
+    code = C.c_uint32(0)
+    K.load().rg_device_status(C.byref(code))
+    return int(code.value)
+
+
+# ---------------------------------------------------------------- marshalling
+def _dtype_code(t) -> int:
+    import torch
+    if t.dtype == torch.bfloat16:
+        return K.RG_BF16
+    if t.dtype == torch.float32:
+        return K.RG_F32
+    raise TypeError(f"rg tensors are bfloat16 or float32, got {t.dtype}")
+
+
+def _tensor(t) -> K.rg_tensor_t:
+    if t.dim() == 1:
+        return K.rg_tensor_t(t.data_ptr(), _dtype_code(t), t.shape[0], 1, max(int(t.stride(0)), 1))
+    assert t.dim() == 2 and (t.shape[1] <= 1 or t.stride(1) == 1), "rows must be contiguous"
+    ld = int(t.stride(0)) if t.shape[0] > 1 else max(int(t.stride(0)), int(t.shape[1]))
+    return K.rg_tensor_t(t.data_ptr(), _dtype_code(t), t.shape[0], t.shape[1], max(ld, int(t.shape[1])))
+
+
+def _epilogue(bias, act, residual) -> Optional[K.rg_epilogue_t]:
+    if bias is None and residual is None and not act:
+        return None
+    e = K.rg_epilogue_t()
+    e.act = int(act)
+    if bias is not None:
+        e.bias, e.bias_dtype = bias.data_ptr(), _dtype_code(bias)
+    if residual is not None:
+        e.residual, e.residual_dtype, e.ldr = residual.data_ptr(), _dtype_code(residual), int(residual.stride(0))
+    return e
+
+
+def _stream(t) -> int:
+    import torch
+    return torch.cuda.current_stream(t.device).cuda_stream if t.is_cuda else 0
+
+
+def rg_gemm(d: K.rg_desc_t, A, B, C_out, *, bias=None, act: int = 0, residual=None, ws=None):
+    """C_out[M,N] = epilogue(A[M,K] @ B[N,K]^T) with the bits the descriptor fixes.
+    All tensors are CUDA tensors; `ws` is a CUDA byte/float tensor of at least
+    rg_gemm_workspace_bytes(d, M, N) bytes when the descriptor has cuts."""
+    L = K.load()
+    a, b, c = _tensor(A), _tensor(B), _tensor(C_out)
+    e = _epilogue(bias, act, residual)
+    ws_ptr = ws.data_ptr() if ws is not None else None
+    ws_bytes = ws.numel() * ws.element_size() if ws is not None else 0
+    st = L.rg_gemm(C.byref(d), C.byref(a), C.byref(b), C.byref(c), C.byref(e) if e is not None else None,
+                   ws_ptr, ws_bytes, _stream(A))
+    _check(st, "rg_gemm")
+    return C_out
+
+
+def rg_reduce_rows(d: K.rg_desc_t, op: int, x, out, *, weight=None, eps: float = 0.0, aux_out=None):
+    """Row reduction with the descriptor's tree (see include/rg.h for the three operations)."""
+    L = K.load()
+    xt, ot = _tensor(x), _tensor(out)
+    args = K.rg_reduce_args_t()
+    if weight is not None:
+        args.weight, args.weight_dtype = weight.data_ptr(), _dtype_code(weight)
+    args.eps = float(eps)
+    if aux_out is not None:
+        args.aux_out = aux_out.data_ptr()
+    st = L.rg_reduce_rows(C.byref(d), int(op), C.byref(xt), C.byref(ot), C.byref(args), _stream(x))
+    _check(st, "rg_reduce_rows")
+    return out
+
+
+def rg_gemm_host(d: K.rg_desc_t, A, B, C_out, dev_scratch, *, bias=None, act: int = 0, residual=None):
+    """Host-buffer form: A, B, C_out, bias, residual are CPU tensors (pinned for async copies);
+    `dev_scratch` is a CUDA tensor.  Enqueues copies + kernels on the current stream."""
+    L = K.load()
+    a, b, c = _tensor(A), _tensor(B), _tensor(C_out)
+    e = _epilogue(bias, act, residual)
+    st = L.rg_gemm_host(C.byref(d), C.byref(a), C.byref(b), C.byref(c), C.byref(e) if e is not None else None,
+                        dev_scratch.data_ptr(), dev_scratch.numel() * dev_scratch.element_size(), _stream(dev_scratch))
+    _check(st, "rg_gemm_host")
+    return C_out
+
+
+def rg_gemm_host_scratch_bytes(d, M, N, Kdim, c_dtype, bias=None, act=0, residual=None) -> int:
+    e = _epilogue(bias, act, residual)
+    return int(K.load().rg_gemm_host_scratch_bytes(C.byref(d), M, N, Kdim, c_dtype, C.byref(e) if e is not None else None))
+
+
+def rg_reduce_rows_host(d: K.rg_desc_t, op: int, x, out, dev_scratch, *, weight=None, eps: float = 0.0, aux_out=None):
+    L = K.load()
+    xt, ot = _tensor(x), _tensor(out)
+    args = K.rg_reduce_args_t()
+    if weight is not None:
+        args.weight, args.weight_dtype = weight.data_ptr(), _dtype_code(weight)
+    args.eps = float(eps)
+    if aux_out is not None:
+        args.aux_out = aux_out.data_ptr()
+    st = L.rg_reduce_rows_host(C.byref(d), int(op), C.byref(xt), C.byref(ot), C.byref(args), dev_scratch.data_ptr(),
+                               dev_scratch.numel() * dev_scratch.element_size(), _stream(dev_scratch))
+    _check(st, "rg_reduce_rows_host")
+    return out
+
+
+def rg_reduce_rows_host_scratch_bytes(op, x, out) -> int:
+    xt, ot = _tensor(x), _tensor(out)
+    return int(K.load().rg_reduce_rows_host_scratch_bytes(int(op), C.byref(xt), C.byref(ot)))

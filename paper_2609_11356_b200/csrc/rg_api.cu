@@ -1,0 +1,313 @@
+// The C boundary: argument validation, descriptor canonicalisation and class key, plan
+// selection, and the host-buffer forms.  Nothing here does arithmetic on data.
+#include <string.h>
+
+#include "rg_internal.h"
+
+namespace {
+
+constexpr int64_t DIM_LIMIT = (int64_t(1) << 31) - 1024;
+
+bool dtype_ok(int32_t t) { return t == RG_BF16 || t == RG_F32; }
+size_t esize(int32_t t) { return t == RG_BF16 ? 2 : 4; }
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Structural checks that do not depend on a shape.
+rg_status_t check_desc_fields(const rg_desc_t* d) {
+  if (!d) return RG_ERR_NULL;
+  if (d->size != sizeof(rg_desc_t)) return RG_ERR_INVALID_DESC;
+  if (d->in_dtype > RG_F32 || d->acc_dtype > RG_F32 || d->partial_dtype > RG_F32 || d->merge_dtype > RG_F32)
+    return RG_ERR_INVALID_DESC;
+  if (d->atom > RG_ATOM_SCALAR || d->tree > RG_TREE_BALANCED || d->fma > 1 || d->k_tail > 1) return RG_ERR_INVALID_DESC;
+  if (d->n_cuts > RG_MAX_CUTS) return RG_ERR_INVALID_DESC;
+  for (uint32_t i = 0; i < d->n_cuts; ++i) {
+    if (d->cuts[i] == 0) return RG_ERR_INVALID_DESC;
+    if (i > 0 && d->cuts[i] <= d->cuts[i - 1]) return RG_ERR_INVALID_DESC;
+  }
+  return RG_OK;
+}
+
+// What the kernels of this library can honour.
+rg_status_t check_desc_supported(const rg_desc_t* d) {
+  if (d->in_dtype != RG_BF16 || d->acc_dtype != RG_F32 || d->partial_dtype != RG_F32 || d->merge_dtype != RG_F32)
+    return RG_ERR_UNSUPPORTED;
+  if (d->atom != RG_ATOM_TC_BF16_K16 || d->k_tail != 0) return RG_ERR_UNSUPPORTED;
+  if (d->BM != 0 && d->BM != 128) return RG_ERR_UNSUPPORTED;
+  if (d->BN != 0 && d->BN != 64 && d->BN != 128 && d->BN != 256) return RG_ERR_UNSUPPORTED;
+  if (d->BK != 0 && d->BK != 64 && d->BK != 128) return RG_ERR_UNSUPPORTED;
+  if (d->cta_group > 1) return RG_ERR_UNSUPPORTED;
+  if (d->raster > 1) return RG_ERR_INVALID_DESC;
+  for (uint32_t i = 0; i < d->n_cuts; ++i)
+    if (d->cuts[i] % 16 != 0) return RG_ERR_UNSUPPORTED;   // a cut may not split a 16-wide step
+  return RG_OK;
+}
+
+rg_status_t check_tensor(const rg_tensor_t* t) {
+  if (!t) return RG_ERR_NULL;
+  if (!dtype_ok(t->dtype)) return RG_ERR_SHAPE;
+  if (t->rows < 0 || t->cols < 0 || t->rows > DIM_LIMIT || t->cols > DIM_LIMIT) return RG_ERR_SHAPE;
+  if (t->ld < t->cols) return RG_ERR_SHAPE;
+  if (t->rows > 0 && t->cols > 0 && !t->ptr) return RG_ERR_NULL;
+  return RG_OK;
+}
+
+rg_status_t check_epilogue(const rg_epilogue_t* e, int64_t N) {
+  if (!e) return RG_OK;
+  if (e->act != 0 && e->act != 1) return RG_ERR_UNSUPPORTED;
+  if (e->bias && !dtype_ok(e->bias_dtype)) return RG_ERR_SHAPE;
+  if (e->residual && (!dtype_ok(e->residual_dtype) || e->ldr < N)) return RG_ERR_SHAPE;
+  return RG_OK;
+}
+
+rg_status_t check_gemm_shapes(const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C) {
+  rg_status_t s;
+  if ((s = check_tensor(A)) != RG_OK || (s = check_tensor(B)) != RG_OK || (s = check_tensor(C)) != RG_OK) return s;
+  if (A->dtype != RG_BF16 || B->dtype != RG_BF16) return RG_ERR_UNSUPPORTED;
+  if (A->cols != B->cols || C->rows != A->rows || C->cols != B->rows) return RG_ERR_SHAPE;
+  return RG_OK;
+}
+
+int device_sms() {
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  return sms > 0 ? sms : 148;
+}
+
+rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::GemmPlan* plan) {
+  plan->n_parts = (int)d->n_cuts + 1;
+  plan->tree = d->tree;
+  for (int s = 0; s < plan->n_parts; ++s) {
+    plan->part_begin[s] = s == 0 ? 0 : (int32_t)d->cuts[s - 1];
+    plan->part_end[s] = s == plan->n_parts - 1 ? (int32_t)K : (int32_t)d->cuts[s];
+  }
+  plan->BK = d->BK ? d->BK : 64;
+  if (d->BN) plan->BN = d->BN;
+  else {
+    // largest tile that still gives every SM a work item
+    const int64_t tiles_m = (M + 127) / 128;
+    const int sms = device_sms();
+    plan->BN = 64;
+    for (int bn : {256, 128}) {
+      if (tiles_m * ((N + bn - 1) / bn) * plan->n_parts >= sms) { plan->BN = bn; break; }
+    }
+  }
+  const int smax = rg::max_stages_for(plan->BN, plan->BK);
+  plan->stages = d->stages ? d->stages : smax;
+  if (plan->stages > smax) return RG_ERR_UNSUPPORTED;
+  plan->raster = d->raster;
+  return RG_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+void rg_desc_init(rg_desc_t* d) {
+  if (!d) return;
+  memset(d, 0, sizeof(*d));
+  d->size = sizeof(rg_desc_t);
+  d->in_dtype = RG_BF16; d->acc_dtype = RG_F32; d->partial_dtype = RG_F32; d->merge_dtype = RG_F32;
+  d->atom = RG_ATOM_TC_BF16_K16; d->k_tail = 0; d->fma = 0; d->tree = RG_TREE_BALANCED;
+}
+
+rg_status_t rg_desc_validate(const rg_desc_t* d, int64_t M, int64_t N, int64_t K) {
+  rg_status_t s = check_desc_fields(d);
+  if (s != RG_OK) return s;
+  if (M < 0 || N < 0 || K < 1 || M > DIM_LIMIT || N > DIM_LIMIT || K > DIM_LIMIT) return RG_ERR_SHAPE;
+  if (d->n_cuts && (int64_t)d->cuts[d->n_cuts - 1] >= K) return RG_ERR_INVALID_DESC;
+  return check_desc_supported(d);
+}
+
+uint64_t rg_desc_class(const rg_desc_t* d) {
+  if (check_desc_fields(d) != RG_OK) return 0;
+  // canonical serialisation of the order-deciding fields only; "no cuts" has one spelling
+  uint8_t buf[12 + 4 * RG_MAX_CUTS];
+  size_t n = 0;
+  const uint8_t head[8] = {d->in_dtype, d->acc_dtype, d->partial_dtype, d->merge_dtype, d->atom, d->k_tail, d->fma, d->tree};
+  memcpy(buf, head, 8); n = 8;
+  const uint32_t nc = d->n_cuts;
+  for (int b = 0; b < 4; ++b) buf[n++] = (uint8_t)(nc >> (8 * b));
+  for (uint32_t i = 0; i < nc; ++i)
+    for (int b = 0; b < 4; ++b) buf[n++] = (uint8_t)(d->cuts[i] >> (8 * b));
+  uint64_t h = 0xcbf29ce484222325ull;                  // FNV-1a, 64 bit
+  for (size_t i = 0; i < n; ++i) { h ^= buf[i]; h *= 0x100000001b3ull; }
+  return h ? h : 1;
+}
+
+size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N) {
+  if (!d || d->n_cuts == 0 || d->n_cuts > RG_MAX_CUTS || M <= 0 || N <= 0) return 0;
+  return (size_t)(d->n_cuts + 1) * (size_t)M * (size_t)((N + 3) / 4 * 4) * sizeof(float);
+}
+
+rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
+                    const rg_epilogue_t* epi, void* ws, size_t ws_bytes, void* cuda_stream) {
+  rg_status_t s = check_desc_fields(d);
+  if (s != RG_OK) return s;
+  if ((s = check_gemm_shapes(A, B, C)) != RG_OK) return s;
+  const int64_t M = A->rows, K = A->cols, N = B->rows;
+  if (K < 1) return RG_ERR_SHAPE;
+  if ((s = rg_desc_validate(d, M, N, K)) != RG_OK) return s;
+  if ((s = check_epilogue(epi, N)) != RG_OK) return s;
+  if (M == 0 || N == 0) return RG_OK;
+  if ((reinterpret_cast<uintptr_t>(A->ptr) & 15) || (reinterpret_cast<uintptr_t>(B->ptr) & 15) ||
+      (A->ld % 8) || (B->ld % 8))
+    return RG_ERR_ALIGNMENT;
+  if (d->n_cuts) {
+    if (!ws || ws_bytes < rg_gemm_workspace_bytes(d, M, N)) return RG_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(ws) & 15) return RG_ERR_ALIGNMENT;
+  }
+  rg::GemmPlan plan;
+  if ((s = make_plan(d, M, N, K, &plan)) != RG_OK) return s;
+  return rg::launch_gemm(plan, A, B, C, epi, ws, static_cast<cudaStream_t>(cuda_stream));
+}
+
+static rg_status_t check_reduce(const rg_desc_t* d, rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out) {
+  rg_status_t s = check_desc_fields(d);
+  if (s != RG_OK) return s;
+  if ((s = check_tensor(x)) != RG_OK || (s = check_tensor(out)) != RG_OK) return s;
+  if (op != RG_OP_SUM && op != RG_OP_RMSNORM && op != RG_OP_SOFTMAX_DENOM) return RG_ERR_UNSUPPORTED;
+  if (d->acc_dtype != RG_F32 || d->tree != RG_TREE_BALANCED) return RG_ERR_UNSUPPORTED;
+  if (x->cols < 1) return RG_ERR_SHAPE;
+  if (out->rows != x->rows) return RG_ERR_SHAPE;
+  if (op == RG_OP_RMSNORM) { if (out->cols != x->cols) return RG_ERR_SHAPE; }
+  else if (out->cols != 1 || out->dtype != RG_F32) return RG_ERR_SHAPE;
+  return RG_OK;
+}
+
+rg_status_t rg_reduce_rows(const rg_desc_t* d, rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out,
+                           const rg_reduce_args_t* args, void* cuda_stream) {
+  rg_status_t s = check_reduce(d, op, x, out);
+  if (s != RG_OK) return s;
+  if (args && args->weight && !dtype_ok(args->weight_dtype)) return RG_ERR_SHAPE;
+  if (x->rows == 0) return RG_OK;
+  // speed knobs reused for reductions: BN = threads per row, stages = warp-blocks per step
+  return rg::launch_reduce_rows((int)op, d->fma, x, out, args, d->BN, d->stages, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ------------------------------------------------------------ host-buffer forms
+size_t rg_gemm_host_scratch_bytes(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, int32_t c_dtype,
+                                  const rg_epilogue_t* epi) {
+  if (M <= 0 || N <= 0 || K <= 0) return 0;
+  const int64_t ldk = (K + 7) / 8 * 8;
+  size_t b = 0;
+  b += align_up((size_t)M * ldk * 2, 256);
+  b += align_up((size_t)N * ldk * 2, 256);
+  b += align_up((size_t)M * N * esize(c_dtype), 256);
+  if (epi && epi->bias) b += align_up((size_t)N * esize(epi->bias_dtype), 256);
+  if (epi && epi->residual) b += align_up((size_t)M * N * esize(epi->residual_dtype), 256);
+  b += align_up(rg_gemm_workspace_bytes(d, M, N), 256);
+  return b;
+}
+
+rg_status_t rg_gemm_host(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
+                         const rg_epilogue_t* epi, void* dev_scratch, size_t dev_scratch_bytes, void* cuda_stream) {
+  rg_status_t s = check_desc_fields(d);
+  if (s != RG_OK) return s;
+  if ((s = check_gemm_shapes(A, B, C)) != RG_OK) return s;
+  const int64_t M = A->rows, K = A->cols, N = B->rows;
+  if (K < 1) return RG_ERR_SHAPE;
+  if ((s = rg_desc_validate(d, M, N, K)) != RG_OK) return s;
+  if ((s = check_epilogue(epi, N)) != RG_OK) return s;
+  if (M == 0 || N == 0) return RG_OK;
+  if (!dev_scratch || dev_scratch_bytes < rg_gemm_host_scratch_bytes(d, M, N, K, C->dtype, epi)) return RG_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(dev_scratch) & 255) return RG_ERR_ALIGNMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t ldk = (K + 7) / 8 * 8;
+  uint8_t* cur = static_cast<uint8_t*>(dev_scratch);
+  auto take = [&](size_t bytes) { uint8_t* p = cur; cur += align_up(bytes, 256); return p; };
+  rg_tensor_t dA{take((size_t)M * ldk * 2), RG_BF16, M, K, ldk};
+  rg_tensor_t dB{take((size_t)N * ldk * 2), RG_BF16, N, K, ldk};
+  rg_tensor_t dC{take((size_t)M * N * esize(C->dtype)), C->dtype, M, N, N};
+  rg_epilogue_t de{};
+  if (epi) de = *epi;
+  bool ok = true;
+  ok &= cudaMemcpy2DAsync(dA.ptr, ldk * 2, A->ptr, A->ld * 2, K * 2, M, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpy2DAsync(dB.ptr, ldk * 2, B->ptr, B->ld * 2, K * 2, N, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (epi && epi->bias) {
+    void* p = take((size_t)N * esize(epi->bias_dtype));
+    ok &= cudaMemcpyAsync(p, epi->bias, (size_t)N * esize(epi->bias_dtype), cudaMemcpyHostToDevice, st) == cudaSuccess;
+    de.bias = p;
+  }
+  if (epi && epi->residual) {
+    const size_t es = esize(epi->residual_dtype);
+    void* p = take((size_t)M * N * es);
+    ok &= cudaMemcpy2DAsync(p, N * es, epi->residual, epi->ldr * es, N * es, M, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    de.residual = p; de.ldr = N;
+  }
+  if (!ok) return RG_ERR_CUDA;
+  const size_t wsb = rg_gemm_workspace_bytes(d, M, N);
+  void* ws = wsb ? take(wsb) : nullptr;
+  if ((s = rg_gemm(d, &dA, &dB, &dC, epi ? &de : nullptr, ws, wsb, cuda_stream)) != RG_OK) return s;
+  const size_t ces = esize(C->dtype);
+  if (cudaMemcpy2DAsync(C->ptr, C->ld * ces, dC.ptr, N * ces, N * ces, M, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return RG_ERR_CUDA;
+  return RG_OK;
+}
+
+size_t rg_reduce_rows_host_scratch_bytes(rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out) {
+  if (!x || !out || x->rows <= 0 || x->cols <= 0) return 0;
+  const int64_t ldx = (x->cols + 7) / 8 * 8;
+  size_t b = align_up((size_t)x->rows * ldx * esize(x->dtype), 256);
+  if (op == RG_OP_RMSNORM) b += align_up((size_t)x->rows * ldx * esize(out->dtype), 256) + align_up((size_t)x->cols * 4, 256);
+  else b += align_up((size_t)x->rows * 4, 256);
+  b += align_up((size_t)x->rows * 4, 256);   // aux
+  return b;
+}
+
+rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out,
+                                const rg_reduce_args_t* args, void* dev_scratch, size_t dev_scratch_bytes,
+                                void* cuda_stream) {
+  rg_status_t s = check_reduce(d, op, x, out);
+  if (s != RG_OK) return s;
+  if (args && args->weight && !dtype_ok(args->weight_dtype)) return RG_ERR_SHAPE;
+  if (x->rows == 0) return RG_OK;
+  if (!dev_scratch || dev_scratch_bytes < rg_reduce_rows_host_scratch_bytes(op, x, out)) return RG_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(dev_scratch) & 255) return RG_ERR_ALIGNMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t R = x->rows, Cc = x->cols, ldx = (Cc + 7) / 8 * 8;
+  const size_t xes = esize(x->dtype), oes = esize(out->dtype);
+  uint8_t* cur = static_cast<uint8_t*>(dev_scratch);
+  auto take = [&](size_t bytes) { uint8_t* p = cur; cur += align_up(bytes, 256); return p; };
+  rg_tensor_t dx{take((size_t)R * ldx * xes), x->dtype, R, Cc, ldx};
+  rg_tensor_t dout;
+  if (op == RG_OP_RMSNORM) dout = rg_tensor_t{take((size_t)R * ldx * oes), out->dtype, R, Cc, ldx};
+  else dout = rg_tensor_t{take((size_t)R * 4), RG_F32, R, 1, 1};
+  rg_reduce_args_t da{};
+  if (args) da = *args;
+  bool ok = cudaMemcpy2DAsync(dx.ptr, ldx * xes, x->ptr, x->ld * xes, Cc * xes, R, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (args && args->weight) {
+    const size_t wes = esize(args->weight_dtype);
+    void* p = take((size_t)Cc * 4);
+    ok &= cudaMemcpyAsync(p, args->weight, (size_t)Cc * wes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    da.weight = p;
+  }
+  void* daux = (args && args->aux_out) ? take((size_t)R * 4) : nullptr;
+  da.aux_out = daux;
+  if (!ok) return RG_ERR_CUDA;
+  if ((s = rg_reduce_rows(d, op, &dx, &dout, &da, cuda_stream)) != RG_OK) return s;
+  if (op == RG_OP_RMSNORM)
+    ok = cudaMemcpy2DAsync(out->ptr, out->ld * oes, dout.ptr, ldx * oes, Cc * oes, R, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  else
+    ok = cudaMemcpy2DAsync(out->ptr, out->ld * 4, dout.ptr, 4, 4, R, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (daux) ok &= cudaMemcpyAsync(args->aux_out, daux, (size_t)R * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  return ok ? RG_OK : RG_ERR_CUDA;
+}
+
+rg_status_t rg_device_status(uint32_t* code) { return rg::read_and_clear_status(code); }
+
+const char* rg_status_string(rg_status_t s) {
+  switch (s) {
+    case RG_OK: return "ok";
+    case RG_ERR_NULL: return "a required pointer is null";
+    case RG_ERR_INVALID_DESC: return "malformed descriptor";
+    case RG_ERR_UNSUPPORTED: return "well-formed request that no kernel here realises";
+    case RG_ERR_SHAPE: return "tensor shapes disagree or are out of range";
+    case RG_ERR_ALIGNMENT: return "pointer or leading dimension breaks a 16-byte rule";
+    case RG_ERR_WORKSPACE: return "workspace missing or too small";
+    case RG_ERR_CUDA: return "CUDA runtime or driver error";
+    case RG_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

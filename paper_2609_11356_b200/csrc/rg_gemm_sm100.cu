@@ -1,0 +1,566 @@
+// Descriptor-fixed bf16 GEMM for sm_100a: TMA-fed tcgen05.mma with the fp32 accumulator in
+// tensor memory, a fixed in-CTA K order, and a fused epilogue.
+//
+// What fixes the bits (Sec. 3.2.1, 3.2.2, App. E): for every output element and every
+// split-K part, one accumulator starts at zero and receives one tcgen05.mma kind::f16 step per
+// 16 consecutive k, in ascending k.  Everything else in this file is schedule and may change
+// without moving a bit (Sec. 3.1): the tile shape, the shared-memory ring depth, which warp
+// loads and which issues, the persistent tile walk, the double-buffered accumulator.
+//
+// CTA roles (192 threads):
+//   warp 0, lane 0   TMA producer: A[BM x 64] and B[BN x 64] boxes (128-byte swizzle) per stage
+//   warp 1, lane 0   MMA issuer: 4 steps of K=16 per 64-wide box, ascending; tcgen05.commit
+//                    frees the stage; a final commit publishes the accumulator
+//   warps 2..5       epilogue: tcgen05.ld of their 32 TMEM lanes, epilogue math, global stores
+// Two accumulators of BN columns each live in TMEM, so the epilogue of tile t overlaps the
+// mainloop of tile t+1.
+//
+// Every wait is bounded: after ~2 s a waiter raises an abort flag, records a code in the
+// device status word, and all roles drain and return; tensor memory is always released.
+#include <cuda.h>
+
+#include "rg_common.cuh"
+#include "rg_internal.h"
+
+namespace rg {
+
+__device__ unsigned int g_status_word = 0;
+
+namespace {
+
+constexpr int BM = 128;           // rows per tile = TMEM lanes = UMMA M
+constexpr int KBOX = 64;          // bf16 per 128-byte swizzle row
+constexpr int UMMA_K = 16;        // instruction_k for 16-bit inputs
+constexpr int NUM_THREADS = 192;
+constexpr int EPI_WARP0 = 2;
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Bounded wait.  Returns false if the wait was abandoned (own timeout or another role's abort).
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t code) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 255u) {
+      if (*abort_flag) return false;
+      const uint64_t now = globaltimer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        atomicCAS(&g_status_word, 0u, code);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, one K=16 step.  accumulate = 0 overwrites D.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor for a K-major bf16 tile whose rows are 128 bytes, stored
+// with the 128-byte swizzle TMA produced: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);   // start address, 16-byte units
+  d |= static_cast<uint64_t>(1) << 16;                         // leading byte offset: unused with swizzle
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;                 // stride byte offset between 8-row groups
+  d |= static_cast<uint64_t>(1) << 46;                         // descriptor version for this architecture
+  d |= static_cast<uint64_t>(2) << 61;                         // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t make_idesc(int bn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(bn >> 3) << 17) |
+         (static_cast<uint32_t>(BM >> 4) << 24);
+}
+
+struct GemmParams {
+  int32_t M, N, K;
+  int32_t tiles_m, tiles_n, n_parts;
+  int32_t num_stages, raster;
+  void* C;
+  int64_t ldc;
+  int32_t c_dtype;
+  float* ws;            // split-K partials [part][M][ldw], fp32; null without cuts
+  int64_t ldw;
+  EpilogueArgs epi;
+  int32_t part_begin[RG_MAX_CUTS + 1];
+  int32_t part_end[RG_MAX_CUTS + 1];
+};
+
+__device__ __forceinline__ void decode_work(const GemmParams& p, int w, int& part, int& tm, int& tn) {
+  const int tiles = p.tiles_m * p.tiles_n;
+  part = w / tiles;
+  const int t = w - part * tiles;
+  if (p.raster == 1) {
+    tm = t / p.tiles_n;
+    tn = t - tm * p.tiles_n;
+  } else {
+    // grouped walk: 8 tile-rows share their B columns while they are hot in L2
+    constexpr int GROUP_M = 8;
+    const int per_group = GROUP_M * p.tiles_n;
+    const int g = t / per_group;
+    const int first_m = g * GROUP_M;
+    const int gsize = min(p.tiles_m - first_m, GROUP_M);
+    const int r = t - g * per_group;
+    tm = first_m + r % gsize;
+    tn = r / gsize;
+  }
+}
+
+// Store up to 32 consecutive columns of one output row.
+__device__ __forceinline__ void store_row_segment(const GemmParams& p, int64_t row, int col0, int ncols, const float (&v)[32]) {
+  if (p.c_dtype == RG_BF16) {
+    __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.C) + row * p.ldc + col0;
+    if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint4 o = make_uint4(pack_bf16x2(v[8 * q], v[8 * q + 1]), pack_bf16x2(v[8 * q + 2], v[8 * q + 3]),
+                             pack_bf16x2(v[8 * q + 4], v[8 * q + 5]), pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
+        reinterpret_cast<uint4*>(dst)[q] = o;
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __float2bfloat16_rn(v[c]);
+    }
+  } else {
+    float* dst = static_cast<float*>(p.C) + row * p.ldc + col0;
+    if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        reinterpret_cast<float4*>(dst)[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+    } else {
+#pragma unroll
+      for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = v[c];
+    }
+  }
+}
+
+// BN: tile columns (UMMA N).  KSUB: 64-wide boxes per pipeline stage (BK = 64 * KSUB).
+template <int BN, int KSUB>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                    const GemmParams p) {
+  constexpr uint32_t A_BOX_BYTES = BM * KBOX * 2;
+  constexpr uint32_t B_BOX_BYTES = BN * KBOX * 2;
+  constexpr uint32_t STAGE_BYTES = KSUB * (A_BOX_BYTES + B_BOX_BYTES);
+  constexpr uint32_t TMEM_COLS = (2 * BN <= 32) ? 32 : 2 * BN;   // two accumulators; power of two for BN in {64,128,256}
+  constexpr uint32_t IDESC = make_idesc(BN);
+
+  extern __shared__ uint8_t smem_raw[];
+  // the swizzle pattern is a function of the absolute address: tiles sit on 1024-byte boundaries
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const int S = p.num_stages;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + (size_t)S * STAGE_BYTES);
+  // layout: full[S], empty[S], tmem_full[2], tmem_empty[2], then tmem base slot and abort flag
+  const uint32_t bar_full = smem_u32(bars);
+  const uint32_t bar_empty = bar_full + 8u * S;
+  const uint32_t bar_tfull = bar_empty + 8u * S;
+  const uint32_t bar_tempty = bar_tfull + 16u;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_work = p.tiles_m * p.tiles_n * p.n_parts;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8u * s, 1); mbar_init(bar_empty + 8u * s, 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8u * b, 1); mbar_init(bar_tempty + 8u * b, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      bool alive = true;
+      for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
+        int part, tm, tn;
+        decode_work(p, w, part, tm, tn);
+        const int k_begin = p.part_begin[part], k_end = p.part_end[part];
+        for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
+          if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, 0x100u | stage)) { alive = false; break; }
+          const uint32_t full = bar_full + 8u * stage;
+          mbar_expect_tx(full, STAGE_BYTES);
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+#pragma unroll
+          for (int sub = 0; sub < KSUB; ++sub) {
+            tma_load_2d(sa + sub * A_BOX_BYTES, &tmap_a, k0 + sub * KBOX, tm * BM, full);
+            tma_load_2d(sa + KSUB * A_BOX_BYTES + sub * B_BOX_BYTES, &tmap_b, k0 + sub * KBOX, tn * BN, full);
+          }
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      bool alive = true;
+      int it = 0;
+      for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x, ++it) {
+        int part, tm, tn;
+        decode_work(p, w, part, tm, tn);
+        const int k_begin = p.part_begin[part], k_end = p.part_end[part];
+        const int buf = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1;
+        if (!mbar_wait(bar_tempty + 8u * buf, acc_phase ^ 1u, abort_flag, 0x200u | buf)) { alive = false; break; }
+        tcgen05_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        uint32_t accumulate = 0;                        // every part starts from a zero accumulator
+        for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
+          if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, 0x300u | stage)) { alive = false; break; }
+          tcgen05_fence_after();
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+#pragma unroll
+          for (int sub = 0; sub < KSUB; ++sub) {
+            const uint64_t adesc = make_kmajor_sw128_desc(sa + sub * A_BOX_BYTES);
+            const uint64_t bdesc = make_kmajor_sw128_desc(sa + KSUB * A_BOX_BYTES + sub * B_BOX_BYTES);
+#pragma unroll
+            for (int a = 0; a < KBOX / UMMA_K; ++a) {
+              // ascending k; steps at or past the end of the part are not issued
+              if (k0 + sub * KBOX + a * UMMA_K < k_end) {
+                umma_bf16(d_tmem, adesc + 2u * a, bdesc + 2u * a, IDESC, accumulate);
+                accumulate = 1;
+              }
+            }
+          }
+          umma_commit(bar_empty + 8u * stage);           // stage reusable once these steps have read it
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+        if (alive) umma_commit(bar_tfull + 8u * buf);     // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps
+    const int quarter = warp & 3;                         // TMEM lanes [32*quarter, 32*quarter+32)
+    bool alive = true;
+    int it = 0;
+    for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x, ++it) {
+      int part, tm, tn;
+      decode_work(p, w, part, tm, tn);
+      const int buf = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1;
+      if (!mbar_wait(bar_tfull + 8u * buf, acc_phase, abort_flag, 0x400u | buf)) { alive = false; break; }
+      tcgen05_fence_after();
+      const int64_t row = (int64_t)tm * BM + quarter * 32 + lane;
+      const bool row_ok = row < p.M;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        const int col0 = tn * BN + c0;
+        if (col0 >= p.N) break;                           // uniform across the warp
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(taddr + c0, r);
+        tmem_ld_wait();
+        const int ncols = min(32, p.N - col0);
+        if (row_ok) {
+          if (p.ws) {
+            // split-K: the finished part is written at fp32, untouched (Sec. 3.2.2)
+            float* dst = p.ws + ((int64_t)part * p.M + row) * p.ldw + col0;
+            if (ncols == 32) {
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                reinterpret_cast<uint4*>(dst)[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __uint_as_float(r[c]);
+            }
+          } else {
+            float v[32];
+#pragma unroll
+            for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(r[c]);
+            if (p.epi.bias || p.epi.act || p.epi.residual) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (c < ncols) v[c] = apply_epilogue(v[c], p.epi, row, col0 + c);
+            }
+            store_row_segment(p, row, col0, ncols, v);
+          }
+        }
+      }
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  __syncthreads();
+  if (*abort_flag) {
+    // let copies and steps already in flight land before shared and tensor memory go away
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tcgen05_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// -------------------------------------------------------------- split-K merge
+struct FixupParams {
+  const float* ws;
+  int64_t ldw;
+  int32_t M, N, S, tree;
+  void* C;
+  int64_t ldc;
+  int32_t c_dtype;
+  EpilogueArgs epi;
+};
+
+// One thread per (row, 4 consecutive columns).  The parts are combined in the descriptor's
+// tree with plain fp32 adds; BALANCED is evaluated with a binary-counter stack, which visits
+// exactly the aligned pairs of the level-by-level definition.
+__global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) {
+  const int64_t ncol4 = (p.N + 3) / 4;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)p.M * ncol4) return;
+  const int64_t row = idx / ncol4;
+  const int col0 = (int)(idx - row * ncol4) * 4;
+  const float* src = p.ws + row * p.ldw + col0;
+  const int64_t part_stride = (int64_t)p.M * p.ldw;
+  float4 acc;
+  if (p.tree == RG_TREE_LEFT) {
+    acc = *reinterpret_cast<const float4*>(src);
+    for (int s = 1; s < p.S; ++s) {
+      const float4 v = *reinterpret_cast<const float4*>(src + s * part_stride);
+      acc.x = f_add(acc.x, v.x); acc.y = f_add(acc.y, v.y); acc.z = f_add(acc.z, v.z); acc.w = f_add(acc.w, v.w);
+    }
+  } else {
+    float4 stack[7];
+    for (int s = 0; s < p.S; ++s) {
+      float4 v = *reinterpret_cast<const float4*>(src + s * part_stride);
+      int b = 0;
+      for (; (s >> b) & 1; ++b) {
+        const float4 l = stack[b];
+        v.x = f_add(l.x, v.x); v.y = f_add(l.y, v.y); v.z = f_add(l.z, v.z); v.w = f_add(l.w, v.w);
+      }
+      stack[b] = v;
+    }
+    // leftovers: the lowest pending level moves up unchanged until it meets a sibling
+    bool have = false;
+    for (int b = 0; b < 7; ++b) {
+      if (!((p.S >> b) & 1)) continue;
+      if (!have) { acc = stack[b]; have = true; }
+      else {
+        const float4 l = stack[b];
+        acc.x = f_add(l.x, acc.x); acc.y = f_add(l.y, acc.y); acc.z = f_add(l.z, acc.z); acc.w = f_add(l.w, acc.w);
+      }
+    }
+  }
+  float v[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    if (col0 + c < p.N) {
+      const float o = apply_epilogue(v[c], p.epi, row, col0 + c);
+      if (p.c_dtype == RG_BF16) static_cast<__nv_bfloat16*>(p.C)[row * p.ldc + col0 + c] = __float2bfloat16_rn(o);
+      else static_cast<float*>(p.C)[row * p.ldc + col0 + c] = o;
+    }
+  }
+}
+
+// ------------------------------------------------------------ host: tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor map over a row-major [rows, cols] matrix: box = 64 columns x box_rows rows,
+// 128-byte swizzle, zero fill outside the matrix (missing products are then exact zeros).
+bool make_tmap(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)KBOX, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr size_t SMEM_LIMIT = 232448;   // 227 KiB of dynamic shared memory per CTA
+
+size_t smem_bytes_for(int bn, int ksub, int stages) {
+  const size_t stage = (size_t)ksub * (BM * KBOX * 2 + (size_t)bn * KBOX * 2);
+  return 1024 + stages * stage + (2 * stages + 4) * 8 + 16;
+}
+
+template <int BN, int KSUB>
+cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
+  const size_t smem = smem_bytes_for(BN, KSUB, p.num_stages);
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, KSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    if (e != cudaSuccess) return e;
+    configured = SMEM_LIMIT;
+  }
+  gemm_tcgen05_kernel<BN, KSUB><<<grid, NUM_THREADS, smem, st>>>(ta, tb, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int max_stages_for(int bn, int bk) {
+  const int ksub = bk / KBOX;
+  int s = 1;
+  while (s < 8 && smem_bytes_for(bn, ksub, s + 1) <= SMEM_LIMIT) ++s;
+  return s;
+}
+
+rg_status_t read_and_clear_status(uint32_t* code) {
+  unsigned int v = 0, zero = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return RG_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(&v, g_status_word, sizeof(v)) != cudaSuccess) return RG_ERR_CUDA;
+  if (v != 0 && cudaMemcpyToSymbol(g_status_word, &zero, sizeof(zero)) != cudaSuccess) return RG_ERR_CUDA;
+  if (code) *code = v;
+  return v ? RG_ERR_TIMEOUT : RG_OK;
+}
+
+// Launch the GEMM (and the merge when there are cuts).  All arguments were validated by the caller.
+rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
+                        const rg_epilogue_t* epi, void* ws, cudaStream_t st) {
+  const int64_t M = A->rows, K = A->cols, N = B->rows;
+  CUtensorMap ta, tb;
+  if (!make_tmap(&ta, A->ptr, M, K, A->ld, BM) || !make_tmap(&tb, B->ptr, N, K, B->ld, plan.BN)) return RG_ERR_CUDA;
+
+  GemmParams p;
+  p.M = (int32_t)M; p.N = (int32_t)N; p.K = (int32_t)K;
+  p.tiles_m = (int32_t)((M + BM - 1) / BM);
+  p.tiles_n = (int32_t)((N + plan.BN - 1) / plan.BN);
+  p.n_parts = plan.n_parts;
+  p.num_stages = plan.stages;
+  p.raster = plan.raster;
+  for (int s = 0; s < plan.n_parts; ++s) { p.part_begin[s] = plan.part_begin[s]; p.part_end[s] = plan.part_end[s]; }
+  EpilogueArgs e{};
+  if (epi) {
+    e.bias = epi->bias; e.bias_dtype = epi->bias_dtype; e.act = epi->act;
+    e.residual = epi->residual; e.residual_dtype = epi->residual_dtype; e.ldr = epi->ldr;
+  }
+  const bool split = plan.n_parts > 1;
+  p.C = C->ptr; p.ldc = C->ld; p.c_dtype = C->dtype;
+  p.ws = split ? static_cast<float*>(ws) : nullptr;
+  p.ldw = (N + 3) / 4 * 4;
+  p.epi = split ? EpilogueArgs{} : e;
+
+  const int64_t total = (int64_t)p.tiles_m * p.tiles_n * p.n_parts;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int grid = (int)(total < sms ? total : sms);
+  cudaError_t err;
+  const int ksub = plan.BK / KBOX;
+  if (plan.BN == 256 && ksub == 1) err = launch_one<256, 1>(ta, tb, p, grid, st);
+  else if (plan.BN == 256 && ksub == 2) err = launch_one<256, 2>(ta, tb, p, grid, st);
+  else if (plan.BN == 128 && ksub == 1) err = launch_one<128, 1>(ta, tb, p, grid, st);
+  else if (plan.BN == 128 && ksub == 2) err = launch_one<128, 2>(ta, tb, p, grid, st);
+  else if (plan.BN == 64 && ksub == 1) err = launch_one<64, 1>(ta, tb, p, grid, st);
+  else if (plan.BN == 64 && ksub == 2) err = launch_one<64, 2>(ta, tb, p, grid, st);
+  else return RG_ERR_UNSUPPORTED;
+  if (err != cudaSuccess) return RG_ERR_CUDA;
+
+  if (split) {
+    FixupParams f;
+    f.ws = static_cast<const float*>(ws); f.ldw = p.ldw;
+    f.M = p.M; f.N = p.N; f.S = plan.n_parts; f.tree = plan.tree;
+    f.C = C->ptr; f.ldc = C->ld; f.c_dtype = C->dtype; f.epi = e;
+    const int64_t items = M * ((N + 3) / 4);
+    splitk_fixup_kernel<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(f);
+    if (cudaGetLastError() != cudaSuccess) return RG_ERR_CUDA;
+  }
+  return RG_OK;
+}
+
+}  // namespace rg

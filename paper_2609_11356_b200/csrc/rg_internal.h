@@ -1,0 +1,25 @@
+// Internal host-side declarations shared by the translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/rg.h"
+
+namespace rg {
+
+// A validated launch plan: speed knobs resolved, parts laid out.
+struct GemmPlan {
+  int BN, BK, stages, raster;
+  int n_parts, tree;
+  int32_t part_begin[RG_MAX_CUTS + 1];
+  int32_t part_end[RG_MAX_CUTS + 1];
+};
+
+int max_stages_for(int bn, int bk);
+rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
+                        const rg_epilogue_t* epi, void* ws, cudaStream_t st);
+rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* out,
+                               const rg_reduce_args_t* args, int threads_hint, int unroll_hint, cudaStream_t st);
+rg_status_t read_and_clear_status(uint32_t* code);
+
+}  // namespace rg
