@@ -94,7 +94,7 @@ typedef struct {
 typedef struct {
   const void* bias;       /* [N], nullable */
   int32_t bias_dtype;
-  int32_t act;            /* 0 none, 1 SiLU: v / (1 + rg_exp(-v)) */
+  int32_t act;            /* 0 none, 1 SiLU: v / (1 + exp(-v)), exp as fixed by this library */
   const void* residual;   /* [M, N], nullable */
   int32_t residual_dtype;
   int64_t ldr;
@@ -150,7 +150,7 @@ rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t*
  *   RG_OP_SUM:           out[r] = TREE(f32(x[r,:]));            out: rows x 1 fp32
  *   RG_OP_RMSNORM:       ss = TREE(x*x); rinv = 1/sqrt(ss/cols + eps);
  *                        y[r,c] = round((x*rinv)*w[c]);           out: rows x cols, bf16 or fp32
- *   RG_OP_SOFTMAX_DENOM: m = max_c x; out[r] = TREE(rg_exp(x - m)); out: rows x 1 fp32;
+ *   RG_OP_SOFTMAX_DENOM: m = max_c x; out[r] = TREE(exp(x - m)); out: rows x 1 fp32;
  *                        args->aux_out (nullable) receives m.
  * x: bf16 or fp32.  rows == 0: RG_OK, nothing launched.  cols == 0: RG_ERR_SHAPE.
  * Asynchronous on `cuda_stream`. */

@@ -101,3 +101,46 @@ def from_torch(t) -> np.ndarray:
     if t.dtype == torch.bfloat16:
         return t.view(torch.uint16).numpy() if hasattr(torch, "uint16") else t.view(torch.int16).numpy().view(np.uint16)
     return t.numpy()
+
+
+# ---------------------------------------------------------------- device-side draws
+# Full-size tensors (up to 8 GiB) are drawn on the GPU with torch's counter-based generator;
+# the oracle then reads back the rows it checks, so both sides still see the same bytes.
+def device_normal(shape, std: float, seed: int, dtype, device="cuda", mean: float = 0.0, chunk_rows: int = 4096):
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    out = torch.empty(shape, dtype=dtype, device=device)
+    rows = shape[0]
+    for r0 in range(0, rows, chunk_rows):
+        r1 = min(rows, r0 + chunk_rows)
+        blk = torch.randn((r1 - r0,) + tuple(shape[1:]), generator=g, device=device, dtype=torch.float32)
+        out[r0:r1] = (blk * std + mean).to(dtype)
+    return out
+
+
+def device_uniform(shape, lo: float, hi: float, seed: int, dtype, device="cuda"):
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    u = torch.rand(shape, generator=g, device=device, dtype=torch.float32)
+    return (u * (hi - lo) + lo).to(dtype)
+
+
+def device_add_cancellation_pairs(x, seed: int, pairs: int = 64, mag: float = 1e8):
+    """In place: on even rows, `pairs` disjoint positions get +mag and `pairs` others -mag.
+    Positions are (base + stride * t) mod C with an odd stride, a bijection when C is a power
+    of two, so the 2*pairs positions of a row are distinct."""
+    import torch
+    R, Cc = x.shape
+    assert Cc & (Cc - 1) == 0 and 2 * pairs <= Cc
+    g = torch.Generator(device="cpu")
+    g.manual_seed(int(seed))
+    rows = torch.arange(0, R, 2)
+    base = torch.randint(0, Cc, (rows.numel(), 1), generator=g)
+    stride = torch.randint(0, Cc // 2, (rows.numel(), 1), generator=g) * 2 + 1
+    t = torch.arange(2 * pairs).unsqueeze(0)
+    pos = ((base + stride * t) % Cc).to(x.device)
+    vals = torch.cat([torch.full((pairs,), mag), torch.full((pairs,), -mag)]).to(x.dtype).to(x.device)
+    x[rows.to(x.device).unsqueeze(1), pos] = vals.unsqueeze(0).expand(rows.numel(), -1)
+    return x

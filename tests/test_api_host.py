@@ -1,0 +1,116 @@
+"""Host-side logic of the C boundary: the library loads without a GPU, exports every declared
+symbol, validates descriptors and arguments before anything could launch, and hashes classes."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import paper_2609_11356_b200 as rg
+from paper_2609_11356_b200 import _cabi as K
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    L = K.load()
+    header = open(os.path.join(ROOT, "include", "rg.h")).read()
+    declared = set(re.findall(r"\b(rg_[a-z_]+)\s*\(", header))
+    assert declared == set(K.EXPORTS)
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_struct_layout_matches_c():
+    d = rg.rg_desc()
+    assert d.size == C.sizeof(K.rg_desc_t)
+    assert (d.in_dtype, d.acc_dtype, d.partial_dtype, d.merge_dtype) == (K.RG_BF16, K.RG_F32, K.RG_F32, K.RG_F32)
+    assert d.tree == K.RG_TREE_BALANCED and d.n_cuts == 0 and d.BN == 0
+
+
+def test_validate_rules():
+    ok = rg.rg_desc(cuts=(256,))
+    assert rg.rg_desc_validate(ok, 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(cuts=(256, 128)), 64, 256, 512) == 2      # not increasing
+    assert rg.rg_desc_validate(rg.rg_desc(cuts=(512,)), 64, 256, 512) == 2          # cut at K
+    assert rg.rg_desc_validate(rg.rg_desc(cuts=(0,)), 64, 256, 512) == 2
+    assert rg.rg_desc_validate(rg.rg_desc(cuts=(40,)), 64, 256, 512) == 3           # splits a 16-wide step
+    assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_SCALAR), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(BN=96), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(cta_group=2), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(tree=7), 64, 256, 512) == 2
+    assert rg.rg_desc_validate(ok, 64, 256, 0) == 4
+    bad = rg.rg_desc(); bad.size = 12
+    assert rg.rg_desc_validate(bad, 1, 1, 16) == 2
+    assert rg.rg_desc_validate(rg.rg_desc(cuts=tuple(16 * i for i in range(1, 64))), 4, 4, 2048) == 0
+
+
+def test_class_key_holds_order_fields_only():
+    base = rg.rg_desc(cuts=(1792, 3584))
+    k = rg.rg_desc_class(base)
+    assert k != 0
+    # speed knobs do not move the class (Sec. 3.2.2)
+    for kw in (dict(BN=64), dict(BN=256, BK=128), dict(stages=2), dict(raster=1), dict(BM=128)):
+        assert rg.rg_desc_class(rg.rg_desc(cuts=(1792, 3584), **kw)) == k
+    # every order-deciding field does
+    others = [rg.rg_desc(cuts=(1792,)), rg.rg_desc(cuts=(1792, 3600)), rg.rg_desc(),
+              rg.rg_desc(cuts=(1792, 3584), tree=K.RG_TREE_LEFT), rg.rg_desc(cuts=(1792, 3584), fma=1),
+              rg.rg_desc(cuts=(1792, 3584), partial_dtype=K.RG_BF16), rg.rg_desc(cuts=(1792, 3584), merge_dtype=K.RG_BF16),
+              rg.rg_desc(cuts=(1792, 3584), atom=K.RG_ATOM_SCALAR), rg.rg_desc(cuts=(1792, 3584), k_tail=1)]
+    keys = [rg.rg_desc_class(o) for o in others]
+    assert len(set(keys + [k])) == len(keys) + 1
+    # stale entries beyond n_cuts are not part of the record
+    d = rg.rg_desc(cuts=(1792, 3584)); d.cuts[5] = 999
+    assert rg.rg_desc_class(d) == k
+    assert rg.rg_desc_class(rg.rg_desc(cuts=(256, 128))) == 0
+
+
+def test_workspace_bytes():
+    assert rg.rg_gemm_workspace_bytes(rg.rg_desc(), 64, 256) == 0
+    assert rg.rg_gemm_workspace_bytes(rg.rg_desc(cuts=(256,)), 64, 256) == 2 * 64 * 256 * 4
+    assert rg.rg_gemm_workspace_bytes(rg.rg_desc(cuts=(16, 32, 48)), 3, 5) == 4 * 3 * 8 * 4
+
+
+def _t(ptr, dtype, rows, cols, ld=None):
+    return K.rg_tensor_t(ptr, dtype, rows, cols, cols if ld is None else ld)
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    L = K.load()
+    d = rg.rg_desc()
+    A = _t(0x1000, K.RG_BF16, 4, 64); B = _t(0x2000, K.RG_BF16, 8, 64); Cm = _t(0x3000, K.RG_BF16, 4, 8)
+    call = lambda d_, a, b, c, e=None, ws=None, wsb=0: L.rg_gemm(
+        C.byref(d_) if d_ is not None else None, C.byref(a) if a is not None else None,
+        C.byref(b) if b is not None else None, C.byref(c) if c is not None else None, e, ws, wsb, None)
+    assert call(None, A, B, Cm) == 1
+    assert call(d, None, B, Cm) == 1
+    assert call(d, _t(None, K.RG_BF16, 4, 64), B, Cm) == 1
+    assert call(d, A, _t(0x2000, K.RG_BF16, 8, 32), Cm) == 4                       # K disagrees
+    assert call(d, A, B, _t(0x3000, K.RG_BF16, 4, 9)) == 4
+    assert call(d, _t(0x1000, K.RG_F32, 4, 64), B, Cm) == 3                        # fp32 operands
+    assert call(d, _t(0x1008, K.RG_BF16, 4, 64), B, Cm) == 5                       # 16-byte rule
+    assert call(d, _t(0x1000, K.RG_BF16, 4, 60, 60), _t(0x2000, K.RG_BF16, 8, 60, 60), Cm) == 5   # ld % 8
+    assert call(d, _t(0x1000, K.RG_BF16, 4, 0), _t(0x2000, K.RG_BF16, 8, 0), Cm) == 4            # K = 0
+    ds = rg.rg_desc(cuts=(32,))
+    assert call(ds, A, B, Cm) == 6                                                  # workspace missing
+    assert call(ds, A, B, Cm, None, 0x4000, 16) == 6                                # too small
+    e = K.rg_epilogue_t(); e.act = 5
+    assert call(d, A, B, Cm, C.byref(e)) == 3
+    # empty problems are a no-op
+    assert call(d, _t(None, K.RG_BF16, 0, 64), B, _t(None, K.RG_BF16, 0, 8)) == 0
+    x = _t(0x1000, K.RG_F32, 4, 64); o = _t(0x2000, K.RG_F32, 4, 1)
+    red = lambda d_, op, x_, o_: L.rg_reduce_rows(C.byref(d_), op, C.byref(x_), C.byref(o_), None, None)
+    assert red(rg.rg_desc(tree=K.RG_TREE_LEFT), K.RG_OP_SUM, x, o) == 3
+    assert red(d, K.RG_OP_SUM, _t(0x1000, K.RG_F32, 4, 0), o) == 4
+    assert red(d, K.RG_OP_SUM, x, _t(0x2000, K.RG_F32, 5, 1)) == 4
+    assert red(d, K.RG_OP_RMSNORM, x, o) == 4
+    assert red(d, 9, x, o) == 3
+    assert red(d, K.RG_OP_SUM, _t(None, K.RG_F32, 0, 64), _t(None, K.RG_F32, 0, 1)) == 0
+
+
+def test_status_strings():
+    for s in range(9):
+        assert len(rg.rg_status_string(s)) > 1
+    with pytest.raises(rg.RgError):
+        raise rg.RgError(3, "x")
