@@ -1,0 +1,410 @@
+#!/usr/bin/env python
+"""Benchmark of the descriptor-fixed hot path on B200.
+
+One "step" runs every step of the hot path once over synthetic LLM-shaped inputs:
+  G  plain GEMM 8192^3 (bf16 out)                               [large square]
+  G  GEMM 8192 x 14336 x 4096 with bias + SiLU                  [fused-epilogue prefill]
+  G  decode GEMM M=32, N=4096, K=14336, split-K 8, residual     [partials + tree merge]
+  R  fp32 tree row-sum over 65536 x 32768                        [reduction stress]
+  R  RMSNorm over 8192 x 4096 bf16
+  R  softmax normaliser over 65536 x 32768
+`value` is the GEMM throughput (flops of the three GEMMs / device time of the GEMM section);
+the reduction bandwidth, per-kernel rooflines and the bit-match rate ride along in the same line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "deterministic bf16 GEMM TFLOP/s"
+UNIT = "TFLOP/s"
+WORKLOAD = ("configs[4] large square 8192^3 + reduction stress 65536x32768 fp32, plus configs[2] decode split-K "
+            "(M=32) and configs[3] fused-epilogue prefill + RMSNorm 8192x4096, so every hot-path step runs")
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/; None until a capture exists for that kernel.
+NCU_TRAFFIC_BYTES = {"gemm_8192": None, "row_sum_65536x32768": None}
+
+GEMMS = {  # name: (M, N, K)
+    "square": (8192, 8192, 8192),
+    "prefill": (8192, 14336, 4096),
+    "decode": (32, 4096, 14336),
+}
+RED_R, RED_C = 65536, 32768
+RMS_R, RMS_C = 8192, 4096
+
+
+def gemm_flops():
+    return sum(2.0 * m * n * k for m, n, k in GEMMS.values())
+
+
+def reduce_bytes():
+    return 2 * (4.0 * RED_R * RED_C + 4.0 * RED_R) + (2.0 * RMS_R * RMS_C * 2 + 2.0 * RMS_C)
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+                 "hw_power_brake_slowdown": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for n, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+# ------------------------------------------------------------------ our arm
+def run_ours(args):
+    import numpy as np
+    import torch
+
+    import paper_2609_11356_b200 as rg
+    from paper_2609_11356_b200 import dist, synth
+    from paper_2609_11356_b200.api import rg_gemm_host, rg_gemm_host_scratch_bytes, rg_reduce_rows_host, \
+        rg_reduce_rows_host_scratch_bytes
+
+    rank, local_rank, world = dist.init("nccl")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    peaks = load_peaks()
+    bf, f32 = torch.bfloat16, torch.float32
+
+    # ---- inputs (seeded, synthetic; every rank holds its own replica of the batch: weak scaling)
+    seed0 = 1000 * rank
+    T = {}
+    T["sq_A"] = synth.device_normal((8192, 8192), 1.0, seed0 + 11, bf, dev)
+    T["sq_B"] = synth.device_normal((8192, 8192), 1.0, seed0 + 12, bf, dev)
+    T["sq_C"] = torch.empty((8192, 8192), dtype=bf, device=dev)
+    T["pf_X"] = synth.device_normal((8192, 4096), 1.0, seed0 + 6, bf, dev)
+    T["pf_W"] = synth.device_normal((14336, 4096), 0.02, seed0 + 7, bf, dev)
+    T["pf_b"] = synth.device_uniform((14336,), -0.1, 0.1, seed0 + 8, bf, dev)
+    T["pf_C"] = torch.empty((8192, 14336), dtype=bf, device=dev)
+    T["dc_X"] = synth.device_normal((32, 14336), 1.0, seed0 + 4, bf, dev)
+    T["dc_W"] = synth.device_normal((4096, 14336), 0.02, seed0 + 3, bf, dev)
+    T["dc_R"] = synth.device_normal((32, 4096), 1.0, seed0 + 5, bf, dev)
+    T["dc_C"] = torch.empty((32, 4096), dtype=bf, device=dev)
+    T["red_X"] = synth.device_normal((RED_R, RED_C), 100.0, seed0 + 13, f32, dev)
+    synth.device_add_cancellation_pairs(T["red_X"], seed0 + 14, pairs=64)
+    T["red_sum"] = torch.empty(RED_R, dtype=f32, device=dev)
+    T["red_Z"] = torch.empty(RED_R, dtype=f32, device=dev)
+    T["red_m"] = torch.empty(RED_R, dtype=f32, device=dev)
+    T["rms_X"] = synth.device_normal((RMS_R, RMS_C), 1.0, seed0 + 9, bf, dev)
+    T["rms_w"] = synth.device_normal((RMS_C,), 0.05, seed0 + 10, bf, dev, mean=1.0)
+    T["rms_Y"] = torch.empty((RMS_R, RMS_C), dtype=bf, device=dev)
+
+    d_plain = rg.rg_desc()
+    dc_cuts = tuple(1792 * t for t in range(1, 8))
+    d_split = rg.rg_desc(cuts=dc_cuts)
+    ws = torch.empty(rg.rg_gemm_workspace_bytes(d_split, 32, 4096), dtype=torch.uint8, device=dev)
+
+    def step(ev=None):
+        if ev: ev[0].record()
+        rg.rg_gemm(d_plain, T["sq_A"], T["sq_B"], T["sq_C"])
+        if ev: ev[1].record()
+        rg.rg_gemm(d_plain, T["pf_X"], T["pf_W"], T["pf_C"], bias=T["pf_b"], act=1)
+        if ev: ev[2].record()
+        rg.rg_gemm(d_split, T["dc_X"], T["dc_W"], T["dc_C"], residual=T["dc_R"], ws=ws)
+        if ev: ev[3].record()
+        rg.rg_reduce_rows(d_plain, rg.RG_OP_SUM, T["red_X"], T["red_sum"])
+        if ev: ev[4].record()
+        rg.rg_reduce_rows(d_plain, rg.RG_OP_RMSNORM, T["rms_X"], T["rms_Y"], weight=T["rms_w"], eps=1e-5)
+        if ev: ev[5].record()
+        rg.rg_reduce_rows(d_plain, rg.RG_OP_SOFTMAX_DENOM, T["red_X"], T["red_Z"], aux_out=T["red_m"])
+        if ev: ev[6].record()
+
+    launches_per_step = 7   # 3 GEMM kernels + 1 split-K merge + 3 reduction kernels
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    dist.barrier(); torch.cuda.synchronize()
+    sampler.start()
+    t_begin.record()
+    for i in range(args.steps):
+        step(events[i])
+    t_end.record()
+    torch.cuda.synchronize(); dist.barrier()
+    clocks = sampler.stop()
+    total_ms = dist.max_over_ranks(t_begin.elapsed_time(t_end), dev)
+    sec = np.array([[e[j].elapsed_time(e[j + 1]) for j in range(6)] for e in events])   # ms, [steps, 6]
+    mean = sec.mean(0)
+    gemm_ms = dist.max_over_ranks(float(mean[0] + mean[1] + mean[2]), dev)
+    red_ms = dist.max_over_ranks(float(mean[3] + mean[4] + mean[5]), dev)
+    status = rg.rg_device_status()
+
+    line = None
+    if rank == 0:
+        value = world * gemm_flops() / (gemm_ms * 1e-3) / 1e12
+        red_gbs = world * reduce_bytes() / (red_ms * 1e-3) / 1e9
+        sq_tflops = 2.0 * 8192 ** 3 / (mean[0] * 1e-3) / 1e12
+        sum_gbs = (4.0 * RED_R * RED_C + 4.0 * RED_R) / (mean[3] * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": round(total_ms / args.steps, 4), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 inputs, f32 accumulate", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: each step streams two 8 GiB passes",
+                       "gemm_shapes": GEMMS, "reduce_shape": [RED_R, RED_C], "rmsnorm_shape": [RMS_R, RMS_C]},
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks,
+            "sections_ms": {"gemm_square": round(float(mean[0]), 4), "gemm_prefill_bias_silu": round(float(mean[1]), 4),
+                            "gemm_decode_splitk8_residual": round(float(mean[2]), 4), "row_sum": round(float(mean[3]), 4),
+                            "rmsnorm": round(float(mean[4]), 4), "softmax_normaliser": round(float(mean[5]), 4)},
+            "gemm_tflops": {"square": round(sq_tflops, 1),
+                            "prefill": round(2.0 * 8192 * 14336 * 4096 / (mean[1] * 1e-3) / 1e12, 1),
+                            "decode_weight_gbs": round((2.0 * 4096 * 14336) / (mean[2] * 1e-3) / 1e9, 1)},
+            "reduce": {"value": round(red_gbs, 1), "unit": "GB/s", "frac_of_hbm": round(red_gbs / world / peaks["hbm_gbs"], 4),
+                       "row_sum_gbs": round(sum_gbs, 1),
+                       "softmax_gbs": round((4.0 * RED_R * RED_C + 8.0 * RED_R) / (mean[5] * 1e-3) / 1e9, 1),
+                       "rmsnorm_gbs": round((4.0 * RMS_R * RMS_C) / (mean[4] * 1e-3) / 1e9, 1)},
+            "roofline": {"bound": "tensor", "kernel": "gemm_tcgen05_kernel<256,1> on 8192^3",
+                         "achieved": round(sq_tflops, 1), "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                         "frac": round(sq_tflops / peaks["bf16_tflops_sustained"], 4),
+                         "frac_of_burst_peak": round(sq_tflops / peaks["bf16_tflops"], 4),
+                         "frac_of_nominal_2250": round(sq_tflops / 2250.0, 4),
+                         "peak_source": peaks["source"] + " (sustained: the kernel is timed inside a long step)",
+                         "traffic": NCU_TRAFFIC_BYTES["gemm_8192"]},
+            "roofline_reduce": {"bound": "hbm", "kernel": "reduce_rows_kernel<float,SUM> on 65536x32768",
+                                "achieved": round(sum_gbs, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                "frac": round(sum_gbs / peaks["hbm_gbs"], 4), "frac_of_nominal_8000": round(sum_gbs / 8000.0, 4),
+                                "peak_source": peaks["source"], "traffic": NCU_TRAFFIC_BYTES["row_sum_65536x32768"]},
+            "device_status": status,
+        }
+
+    # ---- torch default (cuBLAS) bf16 matmul on the same tensors: a speed reference, order-free
+    if rank == 0:
+        ref = torch.empty_like(T["sq_C"])
+        for _ in range(3): torch.matmul(T["sq_A"], T["sq_B"].T, out=ref)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(); e0.record()
+        for _ in range(10): torch.matmul(T["sq_A"], T["sq_B"].T, out=ref)
+        e1.record(); torch.cuda.synchronize()
+        line["torch_cublas_square_tflops"] = round(2.0 * 8192 ** 3 / (e0.elapsed_time(e1) / 10 * 1e-3) / 1e12, 1)
+        line["bitwise_equal_to_torch_cublas_square"] = bool(torch.equal(ref, T["sq_C"]))
+        del ref
+
+    # ---- bit-match against the oracle on sampled outputs of this very run, and GPU-vs-GPU identity
+    if rank == 0:
+        from oracle import rgo
+        HW = rgo.TCGEN05_BF16_B200
+        g = np.random.default_rng(0)
+        cases, elems_ok, elems_n = [], 0, 0
+
+        def tally(got_f32, want_f32):
+            nonlocal elems_ok, elems_n
+            eq = got_f32.view(np.uint32) == want_f32.view(np.uint32)
+            elems_ok += int(eq.sum()); elems_n += eq.size
+            cases.append(bool(eq.all()))
+
+        si, sj = g.integers(0, 8192, 256), g.integers(0, 8192, 256)
+        tally(T["sq_C"][si, sj].float().cpu().numpy(),
+              rgo.gemm_samples(synth.from_torch(T["sq_A"]), synth.from_torch(T["sq_B"]), si, sj, atom_model=HW))
+        si, sj = g.integers(0, 8192, 256), g.integers(0, 14336, 256)
+        tally(T["pf_C"][si, sj].float().cpu().numpy(),
+              rgo.gemm_samples(synth.from_torch(T["pf_X"]), synth.from_torch(T["pf_W"]), si, sj, atom_model=HW,
+                               bias=synth.from_torch(T["pf_b"]), act=1))
+        si, sj = g.integers(0, 32, 512), g.integers(0, 4096, 512)
+        tally(T["dc_C"][si, sj].float().cpu().numpy(),
+              rgo.gemm_samples(synth.from_torch(T["dc_X"]), synth.from_torch(T["dc_W"]), si, sj, cuts=dc_cuts, atom_model=HW,
+                               residual=synth.from_torch(T["dc_R"])))
+        rows = np.unique(g.integers(0, RED_R, 64))
+        xs = T["red_X"][torch.from_numpy(rows).to(dev)].cpu().numpy()
+        tally(T["red_sum"].cpu().numpy()[rows], rgo.reduce_rows(rgo.OP_SUM, xs)[0])
+        tally(T["red_Z"].cpu().numpy()[rows], rgo.reduce_rows(rgo.OP_SOFTMAX_DENOM, xs)[0])
+        rr = np.unique(g.integers(0, RMS_R, 64))
+        wy, _ = rgo.reduce_rows(rgo.OP_RMSNORM, synth.from_torch(T["rms_X"])[rr], weight=synth.from_torch(T["rms_w"]), eps=1e-5)
+        tally(synth.bf16_bits_to_f32(synth.from_torch(T["rms_Y"])[rr]), synth.bf16_bits_to_f32(wy))
+        # GPU vs GPU: another tile configuration of the same class, and a second run
+        alt = torch.empty_like(T["sq_C"])
+        rg.rg_gemm(rg.rg_desc(BN=128, BK=128, raster=1), T["sq_A"], T["sq_B"], alt)
+        same_class = bool(torch.equal(alt, T["sq_C"]))
+        rg.rg_gemm(d_plain, T["sq_A"], T["sq_B"], alt)
+        same_run = bool(torch.equal(alt, T["sq_C"]))
+        del alt
+        line["bit_match"] = {"vs_oracle_elements_pct": round(100.0 * elems_ok / elems_n, 4),
+                             "vs_oracle_cases_pct": round(100.0 * sum(cases) / len(cases), 2), "sampled_elements": elems_n,
+                             "gpu_tile_configs_identical": same_class, "gpu_runs_identical": same_run,
+                             "atom_model": "probe-fitted tcgen05 bf16 step (25-bit window, truncation)"}
+
+    # ---- end to end through the host-buffer C entry points (GEMM metric): pinned host tensors,
+    # H2D of the operands and D2H of the result inside the timed region, every step
+    e2e = None
+    if True:
+        host = {}
+        for k in ("sq_A", "sq_B", "pf_X", "pf_W", "pf_b", "dc_X", "dc_W", "dc_R"):
+            host[k] = T[k].cpu().pin_memory()
+        for k in ("sq_C", "pf_C", "dc_C"):
+            host[k] = torch.empty(T[k].shape, dtype=bf).pin_memory()
+        del T["red_X"]
+        torch.cuda.empty_cache()
+        nb = max(rg_gemm_host_scratch_bytes(d_plain, 8192, 8192, 8192, rg.RG_BF16),
+                 rg_gemm_host_scratch_bytes(d_plain, 8192, 14336, 4096, rg.RG_BF16, bias=host["pf_b"], act=1),
+                 rg_gemm_host_scratch_bytes(d_split, 32, 4096, 14336, rg.RG_BF16, residual=host["dc_R"]))
+        scratch = torch.empty(nb, dtype=torch.uint8, device=dev)
+
+        def e2e_step():
+            rg_gemm_host(d_plain, host["sq_A"], host["sq_B"], host["sq_C"], scratch)
+            rg_gemm_host(d_plain, host["pf_X"], host["pf_W"], host["pf_C"], scratch, bias=host["pf_b"], act=1)
+            rg_gemm_host(d_split, host["dc_X"], host["dc_W"], host["dc_C"], scratch, residual=host["dc_R"])
+
+        h2d = sum(host[k].numel() * 2 for k in ("sq_A", "sq_B", "pf_X", "pf_W", "pf_b", "dc_X", "dc_W", "dc_R"))
+        d2h = sum(host[k].numel() * 2 for k in ("sq_C", "pf_C", "dc_C"))
+        n_e2e = max(3, min(args.steps, 10))
+        for _ in range(2): e2e_step()
+        torch.cuda.synchronize(); dist.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_e2e): e2e_step()
+        e1.record(); torch.cuda.synchronize(); dist.barrier()
+        ms = dist.max_over_ranks(e0.elapsed_time(e1) / n_e2e, dev)
+        e2e = {"value": round(world * gemm_flops() / (ms * 1e-3) / 1e12, 2), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": round(ms, 3), "steps": n_e2e,
+               "api": "rg_gemm_host (pinned host operands and result)"}
+        if rank == 0:
+            line["e2e"] = e2e
+            line["e2e_matches_device_path"] = bool(torch.equal(host["sq_C"], T["sq_C"].cpu()))
+
+    if rank == 0:
+        line["cpu_baseline"] = cpu_baseline(budget_s=12.0)
+        print(json.dumps(line), flush=True)
+    dist.finalize()
+
+
+# ------------------------------------------------------------------ oracle timing
+def _oracle_gemm_sample(rows: int, cols: int, K: int = 8192, seed: int = 0):
+    import numpy as np
+    from oracle import rgo
+    from paper_2609_11356_b200 import synth
+    A = synth.normal_bf16((rows, K), 1.0, seed + 11); B = synth.normal_bf16((cols, K), 1.0, seed + 12)
+    t0 = time.perf_counter()
+    rgo.gemm(A, B, atom_model=rgo.TCGEN05_BF16_B200, out_dtype=rgo.BF16)
+    return time.perf_counter() - t0, 2.0 * rows * cols * K
+
+
+def cpu_baseline(budget_s: float):
+    """The oracle as it stands, on the host cores: a rows x cols block of the 8192^3 GEMM sized to
+    about `budget_s` seconds, and a band of rows of the 65536 x 32768 row-sum."""
+    import numpy as np
+    from oracle import rgo
+    from paper_2609_11356_b200 import synth
+    cores = rgo.num_threads()
+    t, fl = _oracle_gemm_sample(8, 256)                       # calibration
+    rate = fl / t
+    cols = 2048
+    rows = int(max(8, min(256, budget_s * 0.7 * rate / (2.0 * cols * 8192))))
+    t, fl = _oracle_gemm_sample(rows, cols)
+    x = synth.normal_f32((2048, RED_C), 100.0, 13)
+    t0 = time.perf_counter()
+    rgo.reduce_rows(rgo.OP_SUM, x)
+    tr = time.perf_counter() - t0
+    return {"value": round(fl / t / 1e12, 6), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{rows} rows x {cols} cols of the 8192^3 GEMM ({t:.1f} s); row-sum of 2048 x {RED_C} fp32 rows "
+                      f"({tr:.2f} s)",
+            "reduce_gbs": round(x.nbytes / tr / 1e9, 3)}
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle, unmodified, on bounded samples of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import rgo
+    n_total = args.steps + args.warmup
+    per_step = max(0.2, min(3.0, 150.0 / max(n_total, 1)))
+    t, fl = _oracle_gemm_sample(8, 256)
+    rate = fl / t
+    cols = 1024
+    rows = int(max(2, min(256, per_step * rate / (2.0 * cols * 8192))))
+    for _ in range(args.warmup):
+        _oracle_gemm_sample(rows, cols)
+    t0 = time.perf_counter(); flops = 0.0
+    for _ in range(args.steps):
+        _, f = _oracle_gemm_sample(rows, cols)
+        flops += f
+    dt = time.perf_counter() - t0
+    v = round(flops / dt / 1e12, 6)
+    sample = f"per step: {rows} rows x {cols} cols of the 8192^3 GEMM, probe-fitted tcgen05 step model"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(dt / args.steps * 1e3, 3), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 inputs, f32 accumulate", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": rgo.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
