@@ -173,6 +173,27 @@ rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_
                                 const rg_reduce_args_t* args, void* dev_scratch, size_t dev_scratch_bytes,
                                 void* cuda_stream);
 
+/* Split-K GEMM for callers that cannot allocate device memory (the paper has no counterpart:
+ * this entry point exists for deployment, not for the method).  A serving loop whose memory
+ * pool is frozen after start-up, a plugin whose host framework owns the allocator, or a decode
+ * path that cannot afford the device-wide synchronisation of cudaMalloc still needs somewhere
+ * to put the fp32 parts of a split-K GEMM.  This variant of rg_gemm keeps that workspace in a
+ * fixed array of RG_NOALLOC_WS_BYTES inside the library image (each GPU that loads the library
+ * holds it until the process exits), so the caller passes only inputs and the output.
+ *   - Same arguments, results and bits as rg_gemm with the same descriptor.
+ *   - It calls no cudaMalloc, cudaFree or allocating library routine.
+ *   - A shape whose workspace, rg_gemm_workspace_bytes(d, M, N), exceeds RG_NOALLOC_WS_BYTES is
+ *     refused with RG_ERR_WORKSPACE; nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left.
+ *     Nothing needs clearing (every part that is read was written by the same call), but two
+ *     calls that overlap on the GPU (different streams, no dependency) race on it: serialise
+ *     them. */
+#define RG_NOALLOC_WS_BYTES (8u << 20)
+rg_status_t rg_gemm_noalloc(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
+                            const rg_epilogue_t* epi, void* cuda_stream);
+
 /* Device-side health word of the current device.  Every wait inside the kernels is bounded; a
  * wait that gives up records a code here, lets the kernel drain and return, and leaves the
  * context usable.  Copies the word to *code (0 = healthy) and clears it.  Synchronises the

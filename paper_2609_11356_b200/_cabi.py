@@ -19,11 +19,12 @@ RG_TREE_LEFT, RG_TREE_BALANCED = 0, 1
 RG_ATOM_TC_BF16_K16, RG_ATOM_SCALAR = 0, 1
 RG_OP_SUM, RG_OP_RMSNORM, RG_OP_SOFTMAX_DENOM = 0, 1, 2
 RG_MAX_CUTS = 63
+RG_NOALLOC_WS_BYTES = 8 << 20
 
 # every symbol include/rg.h declares
 EXPORTS = ["rg_desc_init", "rg_desc_validate", "rg_desc_class", "rg_gemm_workspace_bytes", "rg_gemm",
            "rg_reduce_rows", "rg_gemm_host_scratch_bytes", "rg_gemm_host", "rg_reduce_rows_host_scratch_bytes",
-           "rg_reduce_rows_host", "rg_device_status", "rg_status_string"]
+           "rg_reduce_rows_host", "rg_device_status", "rg_status_string", "rg_gemm_noalloc"]
 
 
 class rg_desc_t(C.Structure):
@@ -73,6 +74,7 @@ def load():
     L.rg_gemm_host.restype = C.c_int; L.rg_gemm_host.argtypes = [D, T, T, T, E, vp, sz, vp]
     L.rg_reduce_rows_host_scratch_bytes.restype = sz; L.rg_reduce_rows_host_scratch_bytes.argtypes = [C.c_int, T, T]
     L.rg_reduce_rows_host.restype = C.c_int; L.rg_reduce_rows_host.argtypes = [D, C.c_int, T, T, A, vp, sz, vp]
+    L.rg_gemm_noalloc.restype = C.c_int; L.rg_gemm_noalloc.argtypes = [D, T, T, T, E, vp]
     L.rg_device_status.restype = C.c_int; L.rg_device_status.argtypes = [C.POINTER(C.c_uint32)]
     L.rg_status_string.restype = C.c_char_p; L.rg_status_string.argtypes = [C.c_int]
     _lib = L

@@ -110,6 +110,19 @@ def rg_gemm(d: K.rg_desc_t, A, B, C_out, *, bias=None, act: int = 0, residual=No
     return C_out
 
 
+def rg_gemm_noalloc(d: K.rg_desc_t, A, B, C_out, *, bias=None, act: int = 0, residual=None):
+    """rg_gemm for callers that cannot allocate device memory: the split-K workspace is a fixed
+    array inside the library (at most RG_NOALLOC_WS_BYTES; larger shapes raise RG_ERR_WORKSPACE).
+    Calls on one device share that array, so do not let two of them overlap on the GPU."""
+    L = K.load()
+    a, b, c = _tensor(A), _tensor(B), _tensor(C_out)
+    e = _epilogue(bias, act, residual)
+    st = L.rg_gemm_noalloc(C.byref(d), C.byref(a), C.byref(b), C.byref(c), C.byref(e) if e is not None else None,
+                           _stream(A))
+    _check(st, "rg_gemm_noalloc")
+    return C_out
+
+
 def rg_reduce_rows(d: K.rg_desc_t, op: int, x, out, *, weight=None, eps: float = 0.0, aux_out=None):
     """Row reduction with the descriptor's tree (see include/rg.h for the three operations)."""
     L = K.load()
