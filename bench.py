@@ -393,14 +393,75 @@ def run_reference(args):
     }), flush=True)
 
 
+def run_only(args):
+    """One kernel on a small case (inputs above L2, a couple of GB at most): the command the ncu
+    captures under profiles/ were taken with.  Prints the device time per launch."""
+    import torch
+
+    import paper_2609_11356_b200 as rg
+    from paper_2609_11356_b200 import synth
+    dev = torch.device("cuda", 0)
+    bf, f32 = torch.bfloat16, torch.float32
+    name = args.only
+    d = rg.rg_desc()
+    if name in ("gemm_square", "gemm_prefill"):
+        M, N, K = GEMMS["square"] if name == "gemm_square" else GEMMS["prefill"]
+        A = synth.device_normal((M, K), 1.0, 11, bf, dev); B = synth.device_normal((N, K), 0.02, 12, bf, dev)
+        Cm = torch.empty((M, N), dtype=bf, device=dev)
+        bias = synth.device_uniform((N,), -0.1, 0.1, 8, bf, dev) if name == "gemm_prefill" else None
+        fn = lambda: rg.rg_gemm(d, A, B, Cm, bias=bias, act=1 if bias is not None else 0)
+        work, unit = 2.0 * M * N * K / 1e12, "TFLOP/s"
+    elif name == "gemm_decode":
+        M, N, K = GEMMS["decode"]
+        d = rg.rg_desc(cuts=tuple(1792 * t for t in range(1, 8)))
+        A = synth.device_normal((M, K), 1.0, 4, bf, dev)
+        Ws = [synth.device_normal((N, K), 0.02, 3 + i, bf, dev) for i in range(4)]    # rotate: weights leave L2
+        R = synth.device_normal((M, N), 1.0, 5, bf, dev); Cm = torch.empty((M, N), dtype=bf, device=dev)
+        ws = torch.empty(rg.rg_gemm_workspace_bytes(d, M, N), dtype=torch.uint8, device=dev)
+        it = [0]
+        def fn():
+            it[0] += 1
+            rg.rg_gemm(d, A, Ws[it[0] % 4], Cm, residual=R, ws=ws)
+        work, unit = 2.0 * N * K / 1e9, "GB/s (weights)"
+    else:
+        R_, C_ = (16384, RED_C) if name in ("row_sum", "softmax") else (RMS_R * 4, RMS_C)
+        if name == "rmsnorm":
+            x = synth.device_normal((R_, C_), 1.0, 9, bf, dev); w = synth.device_normal((C_,), 0.05, 10, bf, dev, mean=1.0)
+            y = torch.empty_like(x)
+            fn = lambda: rg.rg_reduce_rows(d, rg.RG_OP_RMSNORM, x, y, weight=w, eps=1e-5)
+            work = 4.0 * R_ * C_ / 1e9
+        else:
+            x = synth.device_normal((R_, C_), 100.0, 13, f32, dev)
+            out = torch.empty(R_, dtype=f32, device=dev)
+            op = rg.RG_OP_SUM if name == "row_sum" else rg.RG_OP_SOFTMAX_DENOM
+            fn = lambda: rg.rg_reduce_rows(d, op, x, out)
+            work = 4.0 * R_ * C_ / 1e9
+        unit = "GB/s"
+    for _ in range(max(args.warmup, 1)):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        fn()
+    e1.record(); torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    print(json.dumps({"only": name, "ms_per_launch": round(ms, 4), "rate": round(work / (ms * 1e-3), 1), "unit": unit,
+                      "device_status": rg.rg_device_status()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_prefill", "gemm_decode", "row_sum", "softmax", "rmsnorm"],
+                    help="run one kernel on a small case (used for the ncu captures)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.only:
+        run_only(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

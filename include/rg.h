@@ -65,7 +65,7 @@ typedef struct {
   uint16_t BM, BN, BK;    /* output tile and K step per pipeline stage; 0 = library default */
   uint8_t stages;         /* shared-memory ring depth; 0 = as many as fit */
   uint8_t cta_group;      /* 1, or 2 (pair of SMs on one 256-row tile); 0 = default */
-  uint8_t raster;         /* tile walk: 0 = default grouped-M swizzle, 1 = row-major */
+  uint8_t raster;         /* tile walk: 0 = default grouped walk, 1 = row-major, n in 2..64 = groups of n tile rows */
   uint8_t _pad0;
   /* ---- order-deciding fields: these ARE the class key ---- */
   uint8_t in_dtype;       /* rg_dtype_t of A and B: RG_BF16 */

@@ -36,7 +36,7 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
   if (d->BN != 0 && d->BN != 64 && d->BN != 128 && d->BN != 256) return RG_ERR_UNSUPPORTED;
   if (d->BK != 0 && d->BK != 64 && d->BK != 128) return RG_ERR_UNSUPPORTED;
   if (d->cta_group > 1) return RG_ERR_UNSUPPORTED;
-  if (d->raster > 1) return RG_ERR_INVALID_DESC;
+  if (d->raster > 64) return RG_ERR_INVALID_DESC;
   for (uint32_t i = 0; i < d->n_cuts; ++i)
     if (d->cuts[i] % 16 != 0) return RG_ERR_UNSUPPORTED;   // a cut may not split a 16-wide step
   return RG_OK;
@@ -94,7 +94,8 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   const int smax = rg::max_stages_for(plan->BN, plan->BK);
   plan->stages = d->stages ? d->stages : smax;
   if (plan->stages > smax) return RG_ERR_UNSUPPORTED;
-  plan->raster = d->raster;
+  plan->raster = d->raster == 1 ? 1 : 0;
+  plan->group_m = d->raster >= 2 ? d->raster : 8;
   return RG_OK;
 }
 

@@ -22,10 +22,10 @@ __device__ __forceinline__ float bf16_bits_to_f32(uint32_t h) { return __uint_as
 // two-term Cody-Waite reduction with fused multiply-adds, degree-7 Taylor polynomial in
 // Horner form, and an exact two-factor scaling by 2^n.
 __device__ __forceinline__ float rg_exp(float x) {
-  if (x != x) return x;
-  if (x > 88.72284f) return __int_as_float(0x7f800000);
-  if (x < -87.33655f) return 0.0f;
-  const float n = rintf(f_mul(x, 0x1.715476p+0f));
+  // straight-line code: the range checks are selects at the end, so independent calls overlap
+  const float y = f_mul(x, 0x1.715476p+0f);
+  const float t = f_add(y, 12582912.0f);                // round to nearest-even integer: same value as rint(y)
+  const float n = f_add(t, -12582912.0f);               //   for |y| < 2^22, which the range checks guarantee
   float r = f_fma(n, -0x1.62e400p-1f, x);
   r = f_fma(n, -0x1.7f7d1cp-20f, r);
   float p = 0x1.a01a02p-13f;
@@ -36,11 +36,14 @@ __device__ __forceinline__ float rg_exp(float x) {
   p = f_fma(p, r, 0.5f);
   p = f_fma(p, r, 1.0f);
   p = f_fma(p, r, 1.0f);
-  const int ni = (int)n;
+  const int ni = __float_as_int(t) - 0x4B400000;        // the integer n, read from t's mantissa
   const int h = ni >> 1;
   const float s1 = __int_as_float((ni - h + 127) << 23);
   const float s2 = __int_as_float((h + 127) << 23);
-  return f_mul(f_mul(p, s1), s2);
+  float e = f_mul(f_mul(p, s1), s2);
+  e = x < -87.33655f ? 0.0f : e;
+  e = x > 88.72284f ? __int_as_float(0x7f800000) : e;
+  return x != x ? x : e;
 }
 
 __device__ __forceinline__ float rg_silu(float v) { return __fdiv_rn(v, f_add(1.0f, rg_exp(-v))); }
@@ -58,6 +61,41 @@ struct EpilogueArgs {
 __device__ __forceinline__ float load_scalar(const void* p, int dtype, int64_t idx) {
   if (dtype == RG_BF16) return bf16_bits_to_f32(static_cast<const uint16_t*>(p)[idx]);
   return static_cast<const float*>(p)[idx];
+}
+
+// `n` (<= 32) consecutive elements starting at element index `idx` of a bf16 or fp32 array, widened
+// to fp32; entries past n are zero.  Uses 16-byte loads when the segment is full and aligned.
+__device__ __forceinline__ void load_row_segment(const void* base, int dtype, int64_t idx, int n, float (&out)[32]) {
+  if (dtype == RG_BF16) {
+    const uint16_t* p = static_cast<const uint16_t*>(base) + idx;
+    if (n == 32 && (reinterpret_cast<uintptr_t>(p) & 15) == 0) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 w = __ldg(reinterpret_cast<const uint4*>(p) + q);
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          out[8 * q + 2 * t] = bf16_bits_to_f32(ww[t] & 0xffffu);
+          out[8 * q + 2 * t + 1] = bf16_bits_to_f32(ww[t] >> 16);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < 32; ++c) out[c] = c < n ? bf16_bits_to_f32(p[c]) : 0.0f;
+    }
+  } else {
+    const float* p = static_cast<const float*>(base) + idx;
+    if (n == 32 && (reinterpret_cast<uintptr_t>(p) & 15) == 0) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const float4 w = __ldg(reinterpret_cast<const float4*>(p) + q);
+        out[4 * q] = w.x; out[4 * q + 1] = w.y; out[4 * q + 2] = w.z; out[4 * q + 3] = w.w;
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < 32; ++c) out[c] = c < n ? p[c] : 0.0f;
+    }
+  }
 }
 
 // bias -> activation -> residual, in that order, on one fp32 value (Sec. 2: the position of

@@ -7,11 +7,13 @@
 // without moving a bit (Sec. 3.1): the tile shape, the shared-memory ring depth, which warp
 // loads and which issues, the persistent tile walk, the double-buffered accumulator.
 //
-// CTA roles (192 threads):
+// CTA roles (320 threads):
 //   warp 0, lane 0   TMA producer: A[BM x 64] and B[BN x 64] boxes (128-byte swizzle) per stage
 //   warp 1, lane 0   MMA issuer: 4 steps of K=16 per 64-wide box, ascending; tcgen05.commit
 //                    frees the stage; a final commit publishes the accumulator
-//   warps 2..5       epilogue: tcgen05.ld of their 32 TMEM lanes, epilogue math, global stores
+//   warps 2..9       epilogue: tcgen05.ld of their 32 TMEM lanes (warp % 4 picks the lane
+//                    quarter; the two warps of a quarter take alternate 32-column chunks),
+//                    epilogue math, global stores
 // Two accumulators of BN columns each live in TMEM, so the epilogue of tile t overlaps the
 // mainloop of tile t+1.
 //
@@ -31,8 +33,8 @@ namespace {
 constexpr int BM = 128;           // rows per tile = TMEM lanes = UMMA M
 constexpr int KBOX = 64;          // bf16 per 128-byte swizzle row
 constexpr int UMMA_K = 16;        // instruction_k for 16-bit inputs
-constexpr int NUM_THREADS = 192;
-constexpr int EPI_WARP0 = 2;
+constexpr int NUM_THREADS = 320;
+constexpr int NUM_EPI_WARPS = 8;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -144,7 +146,7 @@ __host__ __device__ constexpr uint32_t make_idesc(int bn) {
 struct GemmParams {
   int32_t M, N, K;
   int32_t tiles_m, tiles_n, n_parts;
-  int32_t num_stages, raster;
+  int32_t num_stages, raster, group_m;
   void* C;
   int64_t ldc;
   int32_t c_dtype;
@@ -163,15 +165,38 @@ __device__ __forceinline__ void decode_work(const GemmParams& p, int w, int& par
     tm = t / p.tiles_n;
     tn = t - tm * p.tiles_n;
   } else {
-    // grouped walk: 8 tile-rows share their B columns while they are hot in L2
-    constexpr int GROUP_M = 8;
-    const int per_group = GROUP_M * p.tiles_n;
+    // grouped walk: group_m tile-rows share their B columns while they are hot in L2
+    const int per_group = p.group_m * p.tiles_n;
     const int g = t / per_group;
-    const int first_m = g * GROUP_M;
-    const int gsize = min(p.tiles_m - first_m, GROUP_M);
+    const int first_m = g * p.group_m;
+    const int gsize = min(p.tiles_m - first_m, p.group_m);
     const int r = t - g * per_group;
     tm = first_m + r % gsize;
     tn = r / gsize;
+  }
+}
+
+// bias -> SiLU -> residual on 32 consecutive columns of one row, stage by stage so that the 32
+// independent chains of each stage overlap in the pipeline.
+__device__ __forceinline__ void epilogue_row_segment(float (&v)[32], const EpilogueArgs& e, int64_t row, int col0, int ncols) {
+  if (e.bias) {
+    float b[32];
+    load_row_segment(e.bias, e.bias_dtype, col0, ncols, b);
+#pragma unroll
+    for (int c = 0; c < 32; ++c) v[c] = f_add(v[c], b[c]);
+  }
+  if (e.act == 1) {
+    float ex[32];
+#pragma unroll
+    for (int c = 0; c < 32; ++c) ex[c] = f_add(1.0f, rg_exp(-v[c]));
+#pragma unroll
+    for (int c = 0; c < 32; ++c) v[c] = __fdiv_rn(v[c], ex[c]);
+  }
+  if (e.residual) {
+    float rr[32];
+    load_row_segment(e.residual, e.residual_dtype, row * e.ldr + col0, ncols, rr);
+#pragma unroll
+    for (int c = 0; c < 32; ++c) v[c] = f_add(v[c], rr[c]);
   }
 }
 
@@ -233,7 +258,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8u * s, 1); mbar_init(bar_empty + 8u * s, 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8u * b, 1); mbar_init(bar_tempty + 8u * b, 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8u * b, 1); mbar_init(bar_tempty + 8u * b, NUM_EPI_WARPS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -311,6 +336,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   } else {
     // ------------------------------------------------------------ epilogue warps
     const int quarter = warp & 3;                         // TMEM lanes [32*quarter, 32*quarter+32)
+    const int chunk0 = (warp - 2) >> 2;                   // this warp takes chunks chunk0, chunk0+2, ...
     bool alive = true;
     int it = 0;
     for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x, ++it) {
@@ -324,7 +350,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       const bool row_ok = row < p.M;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
+      for (int c0 = chunk0 * 32; c0 < BN; c0 += 64) {
         const int col0 = tn * BN + c0;
         if (col0 >= p.N) break;                           // uniform across the warp
         uint32_t r[32];
@@ -347,11 +373,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             float v[32];
 #pragma unroll
             for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(r[c]);
-            if (p.epi.bias || p.epi.act || p.epi.residual) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (c < ncols) v[c] = apply_epilogue(v[c], p.epi, row, col0 + c);
-            }
+            epilogue_row_segment(v, p.epi, row, col0, ncols);
             store_row_segment(p, row, col0, ncols, v);
           }
         }
@@ -523,6 +545,7 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   p.n_parts = plan.n_parts;
   p.num_stages = plan.stages;
   p.raster = plan.raster;
+  p.group_m = plan.group_m;
   for (int s = 0; s < plan.n_parts; ++s) { p.part_begin[s] = plan.part_begin[s]; p.part_end[s] = plan.part_end[s]; }
   EpilogueArgs e{};
   if (epi) {

@@ -9,7 +9,7 @@ namespace rg {
 
 // A validated launch plan: speed knobs resolved, parts laid out.
 struct GemmPlan {
-  int BN, BK, stages, raster;
+  int BN, BK, stages, raster, group_m;
   int n_parts, tree;
   int32_t part_begin[RG_MAX_CUTS + 1];
   int32_t part_end[RG_MAX_CUTS + 1];

@@ -1,7 +1,7 @@
 // Row reductions with a pinned balanced tree (Sec. 3.1 three-level tree; Sec. 5.1 count-up
 // butterfly).  The tree is defined over the logical column index: level l combines aligned
 // blocks of 2^l columns, an unpaired block moves up unchanged.  A pinned tree makes the data
-// layout a free speed knob (Sec. 5.2), which is what the kernel spends:
+// layout a free speed knob (Sec. 5.2), which is what the kernels spend:
 //
 //   thread : one 16-byte vector = an aligned block of V columns (V = 4 fp32 / 8 bf16), folded
 //            in registers in index order                                  (levels 0 .. log2 V)
@@ -9,18 +9,29 @@
 //            so neighbours pair first                                     (next 5 levels)
 //   unroll : a warp folds U consecutive warp-blocks (U independent loads in flight), then
 //            combines the U values pairwise in registers                  (next log2 U levels)
-//   CTA    : the remaining values go through shared memory and one last butterfly.
+//   above  : "super-block" values are combined in index order with a binary-counter stack
+//            (warp-per-row kernel) or through shared memory (CTA-per-row kernel); both visit
+//            exactly the aligned pairs of the level-by-level definition.
 //
 // Columns past the end of the row are the additive identity -0.0f: x + (-0) = x for every x,
 // so padding is bit-identical to "moves up unchanged".  (+0.0 would not be: -0 + +0 = +0.)
 // All adds are __fadd_rn; nothing here can be contracted or reassociated by the compiler.
+//
+// Two kernels, same bits:
+//   reduce_rows_warp_kernel  one warp owns a row: no barriers, all warps independent.  Used
+//                            for sums and RMSNorm when there are enough rows to fill the GPU.
+//   reduce_rows_cta_kernel   one CTA owns a row (32..1024 threads).  Used for few rows, and for
+//                            the softmax normaliser, whose second pass re-reads the row: the rows
+//                            in flight (CTAs x row bytes) are kept well inside L2.
 #include "rg_common.cuh"
+#include "rg_internal.h"
 
 namespace rg {
 
 namespace {
 
 constexpr float NEG_ZERO = -0.0f;
+constexpr int MAX_LEVELS = 13;          // super-blocks per row < 2^13
 
 enum : int { OP_SUM = 0, OP_RMS = 1, OP_SOFTMAX = 2 };
 
@@ -31,52 +42,62 @@ template <> struct VecTraits<uint16_t> { static constexpr int V = 8; };
 __device__ __forceinline__ float elem_to_f32(float v) { return v; }
 __device__ __forceinline__ float elem_to_f32(uint16_t v) { return bf16_bits_to_f32(v); }
 
-// Load V consecutive elements starting at column `col` of a row; out-of-range columns are
-// flagged invalid.  VEC: the row start is 16-byte aligned and ld is a multiple of V.
-template <typename T, bool VEC>
-__device__ __forceinline__ void load_block(const T* __restrict__ xr, int64_t col, int64_t C,
-                                           float (&v)[VecTraits<T>::V], bool (&ok)[VecTraits<T>::V]) {
-  constexpr int V = VecTraits<T>::V;
-  if (VEC && col + V <= C) {
-    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(xr + col));
-    if constexpr (sizeof(T) == 4) {
-      v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y);
-      v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
-    } else {
-      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-      for (int t = 0; t < 4; ++t) {
-        v[2 * t] = bf16_bits_to_f32(w[t] & 0xffffu);
-        v[2 * t + 1] = bf16_bits_to_f32(w[t] >> 16);
-      }
-    }
-#pragma unroll
-    for (int t = 0; t < V; ++t) ok[t] = true;
+template <typename T>
+__device__ __forceinline__ void unpack(const uint4& raw, float (&v)[VecTraits<T>::V]) {
+  if constexpr (sizeof(T) == 4) {
+    v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y);
+    v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
   } else {
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-    for (int t = 0; t < V; ++t) {
-      ok[t] = (col + t) < C;
-      v[t] = ok[t] ? elem_to_f32(xr[col + t]) : 0.0f;
+    for (int t = 0; t < 4; ++t) {
+      v[2 * t] = bf16_bits_to_f32(w[t] & 0xffffu);
+      v[2 * t + 1] = bf16_bits_to_f32(w[t] >> 16);
     }
   }
 }
 
+// exp(d) for d <= 0 (the softmax leaf x - max): the library's exponential with the branches
+// that cannot trigger for d <= 0 removed and rint / the 2^n scaling done with bit-exact
+// equivalents (round-to-integer by adding 1.5*2^23; one multiply by 2^n, n in [-126, 0]).
+__device__ __forceinline__ float exp_nonpositive(float d) {
+  const float y = f_mul(d, 0x1.715476p+0f);
+  const float t = f_add(y, 12582912.0f);
+  const float n = f_add(t, -12582912.0f);
+  float r = f_fma(n, -0x1.62e400p-1f, d);
+  r = f_fma(n, -0x1.7f7d1cp-20f, r);
+  float p = 0x1.a01a02p-13f;
+  p = f_fma(p, r, 0x1.6c16c2p-10f);
+  p = f_fma(p, r, 0x1.111112p-7f);
+  p = f_fma(p, r, 0x1.555556p-5f);
+  p = f_fma(p, r, 0x1.555556p-3f);
+  p = f_fma(p, r, 0.5f);
+  p = f_fma(p, r, 1.0f);
+  p = f_fma(p, r, 1.0f);
+  const int ni = __float_as_int(t) - 0x4B400000;        // the integer n, read from t's mantissa
+  const float s = __int_as_float((ni + 127) << 23);
+  const float e = f_mul(p, s);
+  return d < -87.33655f ? 0.0f : e;
+}
+
 // Fold one thread's V leaves in index order: (l0+l1), (l2+l3), ... then pairs of pairs.
-template <int OP, int V>
-__device__ __forceinline__ float fold_block(const float (&x)[V], const bool (&ok)[V], float shift, int fma) {
+// FULL: all V columns exist.  Otherwise `nvalid` leading ones do; the rest are -0.0f.
+template <int OP, int V, bool FULL>
+__device__ __forceinline__ float fold_block(const float (&x)[V], int nvalid, float shift, int fma) {
   float n[V / 2];
 #pragma unroll
   for (int t = 0; t < V / 2; ++t) {
     const float x0 = x[2 * t], x1 = x[2 * t + 1];
+    const bool ok0 = FULL || (2 * t < nvalid), ok1 = FULL || (2 * t + 1 < nvalid);
     if (OP == OP_SUM) {
-      n[t] = f_add(ok[2 * t] ? x0 : NEG_ZERO, ok[2 * t + 1] ? x1 : NEG_ZERO);
+      n[t] = f_add(ok0 ? x0 : NEG_ZERO, ok1 ? x1 : NEG_ZERO);
     } else if (OP == OP_RMS) {
-      const float s0 = ok[2 * t] ? f_mul(x0, x0) : NEG_ZERO;
-      if (fma) n[t] = ok[2 * t + 1] ? f_fma(x1, x1, s0) : s0;   // second square fused into the add
-      else n[t] = f_add(s0, ok[2 * t + 1] ? f_mul(x1, x1) : NEG_ZERO);
+      const float s0 = ok0 ? f_mul(x0, x0) : NEG_ZERO;
+      if (fma) n[t] = ok1 ? f_fma(x1, x1, s0) : s0;      // second square fused into the add
+      else n[t] = f_add(s0, ok1 ? f_mul(x1, x1) : NEG_ZERO);
     } else {
-      const float e0 = ok[2 * t] ? rg_exp(f_add(x0, -shift)) : NEG_ZERO;
-      const float e1 = ok[2 * t + 1] ? rg_exp(f_add(x1, -shift)) : NEG_ZERO;
+      const float e0 = ok0 ? exp_nonpositive(f_add(x0, -shift)) : NEG_ZERO;
+      const float e1 = ok1 ? exp_nonpositive(f_add(x1, -shift)) : NEG_ZERO;
       n[t] = f_add(e0, e1);
     }
   }
@@ -87,58 +108,55 @@ __device__ __forceinline__ float fold_block(const float (&x)[V], const bool (&ok
   return n[0];
 }
 
-__device__ __forceinline__ float warp_tree(float v) {
-  // count-up butterfly: neighbours pair first (Sec. 5.1, Fig. 3)
+// Load the V columns starting at `col` (VEC: 16-byte aligned rows) and fold them.
+template <typename T, int OP, bool VEC>
+__device__ __forceinline__ float load_fold(const T* __restrict__ xr, int64_t col, int64_t C, float shift, int fma) {
+  constexpr int V = VecTraits<T>::V;
+  float x[V];
+  if (VEC && col + V <= C) {
+    unpack<T>(__ldg(reinterpret_cast<const uint4*>(xr + col)), x);
+    return fold_block<OP, V, true>(x, V, shift, fma);
+  }
+  int nvalid = 0;
 #pragma unroll
-  for (int off = 1; off < 32; off <<= 1) v = f_add(v, __shfl_xor_sync(0xffffffffu, v, off));
-  return v;
+  for (int t = 0; t < V; ++t) {
+    const bool ok = (col + t) < C;
+    x[t] = ok ? elem_to_f32(xr[col + t]) : 0.0f;
+    nvalid += ok ? 1 : 0;
+  }
+  return fold_block<OP, V, false>(x, nvalid, shift, fma);
 }
 
-// TREE over the row's leaves; every thread of the CTA returns the root.
-// sb: shared scratch of 2 * cap floats (ping-pong), cap >= number of super-blocks.
+// One super-block (U warp-blocks of 32*V columns) folded by one warp; every lane returns it.
 template <typename T, int OP, bool VEC, int U>
-__device__ float row_tree(const T* __restrict__ xr, int64_t C, float shift, int fma, float* sb, int cap) {
+__device__ __forceinline__ float superblock(const T* __restrict__ xr, int64_t base, int64_t C, float shift, int fma, int lane) {
   constexpr int V = VecTraits<T>::V;
-  constexpr int WB = 32 * V;           // columns per warp-block
-  constexpr int SBW = WB * U;          // columns per super-block
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  const int nsb = (int)((C + SBW - 1) / SBW);
-  for (int sbi = warp; sbi < nsb; sbi += nwarps) {
-    const int64_t base = (int64_t)sbi * SBW + lane * V;
-    float bv[U];
+  constexpr int WB = 32 * V;
+  float bv[U];
+  if (VEC && base + (int64_t)U * WB <= C) {
+    // whole super-block in range: issue all loads first
+    uint4 raw[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) raw[u] = __ldg(reinterpret_cast<const uint4*>(xr + base + (int64_t)u * WB + lane * V));
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      float x[V]; bool ok[V];
-      load_block<T, VEC>(xr, base + (int64_t)u * WB, C, x, ok);
-      bv[u] = fold_block<OP, V>(x, ok, shift, fma);
+      float x[V];
+      unpack<T>(raw[u], x);
+      bv[u] = fold_block<OP, V, true>(x, V, shift, fma);
     }
+  } else {
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1)
-#pragma unroll
-      for (int u = 0; u < U; ++u) bv[u] = f_add(bv[u], __shfl_xor_sync(0xffffffffu, bv[u], off));
-#pragma unroll
-    for (int s = 1; s < U; s <<= 1)
-#pragma unroll
-      for (int u = 0; u < U; u += 2 * s) bv[u] = f_add(bv[u], bv[u + s]);
-    if (lane == 0) sb[sbi] = bv[0];
+    for (int u = 0; u < U; ++u) bv[u] = load_fold<T, OP, VEC>(xr, base + (int64_t)u * WB + lane * V, C, shift, fma);
   }
-  __syncthreads();
-  // remaining levels over nsb values
-  int n = nsb;
-  float* cur = sb;
-  float* nxt = sb + cap;
-  while (n > 32) {
-    const int half = (n + 1) >> 1;
-    for (int t = threadIdx.x; t < half; t += blockDim.x)
-      nxt[t] = (2 * t + 1 < n) ? f_add(cur[2 * t], cur[2 * t + 1]) : cur[2 * t];
-    __syncthreads();
-    float* tmp = cur; cur = nxt; nxt = tmp;
-    n = half;
-  }
-  float v = (lane < n) ? cur[lane] : NEG_ZERO;
-  v = warp_tree(v);
-  __syncthreads();                      // scratch may be reused by the caller's next row
-  return v;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1)      // count-up butterfly: neighbours pair first
+#pragma unroll
+    for (int u = 0; u < U; ++u) bv[u] = f_add(bv[u], __shfl_xor_sync(0xffffffffu, bv[u], off));
+#pragma unroll
+  for (int s = 1; s < U; s <<= 1)
+#pragma unroll
+    for (int u = 0; u < U; u += 2 * s) bv[u] = f_add(bv[u], bv[u + s]);
+  return bv[0];
 }
 
 struct ReduceParams {
@@ -151,25 +169,132 @@ struct ReduceParams {
   int32_t fma, out_dtype, w_dtype, cap;
 };
 
+// y = round((x * rinv) * w) for the V columns at `c` of one row.
+template <typename T, bool VEC>
+__device__ __forceinline__ void rms_scale_store(const ReduceParams& p, const T* __restrict__ xr, int64_t row, int64_t c,
+                                                float rinv, bool out_vec) {
+  constexpr int V = VecTraits<T>::V;
+  float x[V], y[V];
+  const bool full = c + V <= p.C;
+  if (VEC && full) {
+    unpack<T>(__ldg(reinterpret_cast<const uint4*>(xr + c)), x);
+  } else {
+#pragma unroll
+    for (int t = 0; t < V; ++t) x[t] = (c + t) < p.C ? elem_to_f32(xr[c + t]) : 0.0f;
+  }
+  float w[V];
+  const bool w_vec = full && p.weight && ((reinterpret_cast<uintptr_t>(p.weight) & 15) == 0) &&
+                     p.w_dtype == (sizeof(T) == 2 ? RG_BF16 : RG_F32);
+  if (w_vec) {
+    unpack<T>(__ldg(reinterpret_cast<const uint4*>(static_cast<const T*>(p.weight) + c)), w);
+  } else {
+#pragma unroll
+    for (int t = 0; t < V; ++t) w[t] = (p.weight && (c + t) < p.C) ? load_scalar(p.weight, p.w_dtype, c + t) : 1.0f;
+  }
+#pragma unroll
+  for (int t = 0; t < V; ++t) y[t] = f_mul(f_mul(x[t], rinv), w[t]);
+  if (out_vec && full) {
+    if constexpr (sizeof(T) == 4) {
+      *reinterpret_cast<uint4*>(static_cast<float*>(p.out) + row * p.ldo + c) =
+          make_uint4(__float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]), __float_as_uint(y[3]));
+    } else {
+      *reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + row * p.ldo + c) =
+          make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
+    }
+  } else {
+#pragma unroll
+    for (int t = 0; t < V; ++t)
+      if ((c + t) < p.C) {
+        if (p.out_dtype == RG_BF16) static_cast<__nv_bfloat16*>(p.out)[row * p.ldo + c + t] = __float2bfloat16_rn(y[t]);
+        else static_cast<float*>(p.out)[row * p.ldo + c + t] = y[t];
+      }
+  }
+}
+
+template <typename T, bool VEC>
+__device__ __forceinline__ bool rms_out_vec(const ReduceParams& p) {
+  constexpr int V = VecTraits<T>::V;
+  return VEC && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) && (p.ldo % V == 0) &&
+         (p.out_dtype == (sizeof(T) == 2 ? RG_BF16 : RG_F32));
+}
+
+__device__ __forceinline__ float rms_rinv(float ss, int64_t C, float eps) {
+  const float ms = __fdiv_rn(ss, (float)C);
+  return __fdiv_rn(1.0f, __fsqrt_rn(f_add(ms, eps)));
+}
+
+// ------------------------------------------------------------------ warp per row
 template <typename T, int OP, bool VEC, int U>
-__global__ void __launch_bounds__(256) reduce_rows_kernel(const ReduceParams p) {
+__global__ void __launch_bounds__(256) reduce_rows_warp_kernel(const ReduceParams p) {
+  static_assert(OP != OP_SOFTMAX, "the softmax normaliser re-reads its row: CTA kernel");
+  constexpr int V = VecTraits<T>::V;
+  constexpr int SBW = 32 * V * U;
+  const int lane = threadIdx.x & 31;
+  const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int nsb = (int)((p.C + SBW - 1) / SBW);
+  for (int64_t row = warp0; row < p.R; row += nwarps) {
+    const T* xr = static_cast<const T*>(p.x) + row * p.ldx;
+    float stk[MAX_LEVELS];
+#pragma unroll
+    for (int b = 0; b < MAX_LEVELS; ++b) stk[b] = NEG_ZERO;
+    for (int sbi = 0; sbi < nsb; ++sbi) {
+      float v = superblock<T, OP, VEC, U>(xr, (int64_t)sbi * SBW, p.C, 0.0f, p.fma, lane);
+      // binary counter: a finished block of 2^b super-blocks meets its left sibling
+      bool carry = true;
+#pragma unroll
+      for (int b = 0; b < MAX_LEVELS; ++b) {
+        if (carry) {
+          if ((sbi >> b) & 1) v = f_add(stk[b], v);
+          else { stk[b] = v; carry = false; }
+        }
+      }
+    }
+    // leftovers: the lowest pending block moves up unchanged until it meets a sibling
+    float root = NEG_ZERO;
+    bool have = false;
+#pragma unroll
+    for (int b = 0; b < MAX_LEVELS; ++b) {
+      if ((nsb >> b) & 1) {
+        root = have ? f_add(stk[b], root) : stk[b];
+        have = true;
+      }
+    }
+    if (OP == OP_SUM) {
+      if (lane == 0) static_cast<float*>(p.out)[row * p.ldo] = root;
+    } else {
+      const float rinv = rms_rinv(root, p.C, p.eps);
+      if (lane == 0 && p.aux) p.aux[row] = rinv;
+      const bool out_vec = rms_out_vec<T, VEC>(p);
+      for (int64_t c = (int64_t)lane * V; c < p.C; c += 32 * V) rms_scale_store<T, VEC>(p, xr, row, c, rinv, out_vec);
+    }
+  }
+}
+
+// ------------------------------------------------------------------ CTA per row
+template <typename T, int OP, bool VEC, int U>
+__global__ void __launch_bounds__(1024) reduce_rows_cta_kernel(const ReduceParams p) {
   extern __shared__ float smem[];
-  float* sb = smem;                     // 2 * cap floats
+  float* sb = smem;                     // 2 * cap floats (ping-pong)
   float* red = smem + 2 * p.cap;        // 32 floats for the order-free max
   constexpr int V = VecTraits<T>::V;
+  constexpr int SBW = 32 * V * U;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int nsb = (int)((p.C + SBW - 1) / SBW);
   for (int64_t row = blockIdx.x; row < p.R; row += gridDim.x) {
     const T* xr = static_cast<const T*>(p.x) + row * p.ldx;
     float shift = 0.0f;
     if (OP == OP_SOFTMAX) {
       // The row maximum rounds nothing, so its order is free (App. F).
       float m = -INFINITY;
-      for (int64_t c = (int64_t)threadIdx.x * V; c < p.C; c += (int64_t)blockDim.x * V) {
-        float x[V]; bool ok[V];
-        load_block<T, VEC>(xr, c, p.C, x, ok);
+      const int64_t nvec = VEC ? p.C / V : 0;
+      for (int64_t i = threadIdx.x; i < nvec; i += blockDim.x) {
+        float x[V];
+        unpack<T>(__ldg(reinterpret_cast<const uint4*>(xr) + i), x);
 #pragma unroll
-        for (int t = 0; t < V; ++t) if (ok[t]) m = fmaxf(m, x[t]);
+        for (int t = 0; t < V; ++t) m = fmaxf(m, x[t]);
       }
+      for (int64_t c = nvec * V + threadIdx.x; c < p.C; c += blockDim.x) m = fmaxf(m, elem_to_f32(xr[c]));
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
       if (lane == 0) red[warp] = m;
@@ -177,9 +302,28 @@ __global__ void __launch_bounds__(256) reduce_rows_kernel(const ReduceParams p) 
       m = red[0];
       for (int w = 1; w < nwarps; ++w) m = fmaxf(m, red[w]);
       shift = m;
-      __syncthreads();
     }
-    const float root = row_tree<T, OP, VEC, U>(xr, p.C, shift, p.fma, sb, p.cap);
+    for (int sbi = warp; sbi < nsb; sbi += nwarps) {
+      const float v = superblock<T, OP, VEC, U>(xr, (int64_t)sbi * SBW, p.C, shift, p.fma, lane);
+      if (lane == 0) sb[sbi] = v;
+    }
+    __syncthreads();
+    // remaining levels over the nsb super-block values
+    int n = nsb;
+    float* cur = sb;
+    float* nxt = sb + p.cap;
+    while (n > 32) {
+      const int half = (n + 1) >> 1;
+      for (int t = threadIdx.x; t < half; t += blockDim.x)
+        nxt[t] = (2 * t + 1 < n) ? f_add(cur[2 * t], cur[2 * t + 1]) : cur[2 * t];
+      __syncthreads();
+      float* tmp = cur; cur = nxt; nxt = tmp;
+      n = half;
+    }
+    float root = (lane < n) ? cur[lane] : NEG_ZERO;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) root = f_add(root, __shfl_xor_sync(0xffffffffu, root, off));
+    __syncthreads();                    // scratch is reused by the next row
     if (OP == OP_SUM) {
       if (threadIdx.x == 0) static_cast<float*>(p.out)[row * p.ldo] = root;
     } else if (OP == OP_SOFTMAX) {
@@ -188,107 +332,110 @@ __global__ void __launch_bounds__(256) reduce_rows_kernel(const ReduceParams p) 
         if (p.aux) p.aux[row] = shift;
       }
     } else {
-      const float ms = __fdiv_rn(root, (float)p.C);
-      const float rinv = __fdiv_rn(1.0f, __fsqrt_rn(f_add(ms, p.eps)));
+      const float rinv = rms_rinv(root, p.C, p.eps);
       if (threadIdx.x == 0 && p.aux) p.aux[row] = rinv;
-      const bool out_vec = VEC && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) &&
-                           (p.ldo % V == 0) && (p.out_dtype == (sizeof(T) == 2 ? RG_BF16 : RG_F32));
-      for (int64_t c = (int64_t)threadIdx.x * V; c < p.C; c += (int64_t)blockDim.x * V) {
-        float x[V]; bool ok[V];
-        load_block<T, VEC>(xr, c, p.C, x, ok);
-        float y[V];
-#pragma unroll
-        for (int t = 0; t < V; ++t) {
-          const float w = (p.weight && ok[t]) ? load_scalar(p.weight, p.w_dtype, c + t) : 1.0f;
-          y[t] = f_mul(f_mul(x[t], rinv), w);
-        }
-        if (out_vec && c + V <= p.C) {
-          uint4 o;
-          if constexpr (sizeof(T) == 4) {
-            o = make_uint4(__float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]), __float_as_uint(y[3]));
-            *reinterpret_cast<uint4*>(static_cast<float*>(p.out) + row * p.ldo + c) = o;
-          } else {
-            o = make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
-            *reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + row * p.ldo + c) = o;
-          }
-        } else {
-#pragma unroll
-          for (int t = 0; t < V; ++t)
-            if (ok[t]) {
-              if (p.out_dtype == RG_BF16)
-                static_cast<__nv_bfloat16*>(p.out)[row * p.ldo + c + t] = __float2bfloat16_rn(y[t]);
-              else
-                static_cast<float*>(p.out)[row * p.ldo + c + t] = y[t];
-            }
-        }
-      }
+      const bool out_vec = rms_out_vec<T, VEC>(p);
+      for (int64_t c = (int64_t)threadIdx.x * V; c < p.C; c += (int64_t)blockDim.x * V)
+        rms_scale_store<T, VEC>(p, xr, row, c, rinv, out_vec);
     }
   }
 }
 
-template <typename T, int OP, bool VEC>
-cudaError_t launch_u(const ReduceParams& p, int U, int threads, int grid, size_t smem, cudaStream_t st) {
-  switch (U) {
-    case 1: reduce_rows_kernel<T, OP, VEC, 1><<<grid, threads, smem, st>>>(p); break;
-    case 2: reduce_rows_kernel<T, OP, VEC, 2><<<grid, threads, smem, st>>>(p); break;
-    case 4: reduce_rows_kernel<T, OP, VEC, 4><<<grid, threads, smem, st>>>(p); break;
-    default: reduce_rows_kernel<T, OP, VEC, 8><<<grid, threads, smem, st>>>(p); break;
+template <typename T, int OP, bool VEC, int U>
+cudaError_t launch_kernel(const ReduceParams& p, bool warp_rows, int threads, int grid, size_t smem, cudaStream_t st) {
+  if constexpr (OP != OP_SOFTMAX) {
+    if (warp_rows) {
+      reduce_rows_warp_kernel<T, OP, VEC, U><<<grid, threads, 0, st>>>(p);
+      return cudaGetLastError();
+    }
   }
+  reduce_rows_cta_kernel<T, OP, VEC, U><<<grid, threads, smem, st>>>(p);
   return cudaGetLastError();
 }
 
+template <typename T, int OP, bool VEC>
+cudaError_t launch_u(const ReduceParams& p, bool wr, int U, int threads, int grid, size_t smem, cudaStream_t st) {
+  switch (U) {
+    case 1: return launch_kernel<T, OP, VEC, 1>(p, wr, threads, grid, smem, st);
+    case 2: return launch_kernel<T, OP, VEC, 2>(p, wr, threads, grid, smem, st);
+    case 4: return launch_kernel<T, OP, VEC, 4>(p, wr, threads, grid, smem, st);
+    default: return launch_kernel<T, OP, VEC, 8>(p, wr, threads, grid, smem, st);
+  }
+}
+
 template <typename T, int OP>
-cudaError_t launch_vec(const ReduceParams& p, bool vec, int U, int threads, int grid, size_t smem, cudaStream_t st) {
-  return vec ? launch_u<T, OP, true>(p, U, threads, grid, smem, st)
-             : launch_u<T, OP, false>(p, U, threads, grid, smem, st);
+cudaError_t launch_vec(const ReduceParams& p, bool vec, bool wr, int U, int threads, int grid, size_t smem, cudaStream_t st) {
+  return vec ? launch_u<T, OP, true>(p, wr, U, threads, grid, smem, st)
+             : launch_u<T, OP, false>(p, wr, U, threads, grid, smem, st);
 }
 
 template <typename T>
-cudaError_t launch_op(int op, const ReduceParams& p, bool vec, int U, int threads, int grid, size_t smem, cudaStream_t st) {
+cudaError_t launch_op(int op, const ReduceParams& p, bool vec, bool wr, int U, int threads, int grid, size_t smem, cudaStream_t st) {
   switch (op) {
-    case RG_OP_SUM: return launch_vec<T, OP_SUM>(p, vec, U, threads, grid, smem, st);
-    case RG_OP_RMSNORM: return launch_vec<T, OP_RMS>(p, vec, U, threads, grid, smem, st);
-    default: return launch_vec<T, OP_SOFTMAX>(p, vec, U, threads, grid, smem, st);
+    case RG_OP_SUM: return launch_vec<T, OP_SUM>(p, vec, wr, U, threads, grid, smem, st);
+    case RG_OP_RMSNORM: return launch_vec<T, OP_RMS>(p, vec, wr, U, threads, grid, smem, st);
+    default: return launch_vec<T, OP_SOFTMAX>(p, vec, wr, U, threads, grid, smem, st);
   }
 }
 
 }  // namespace
 
-// Host launcher.  threads_hint / unroll_hint: 0 = choose; both are speed knobs only.
+// Host launcher.  Speed knobs only (0 = choose): threads_hint = threads per row, where 32 selects
+// the warp-per-row kernel for sums and RMSNorm; unroll_hint = warp-blocks in flight per warp.
 rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* out,
                                const rg_reduce_args_t* args, int threads_hint, int unroll_hint,
                                cudaStream_t st) {
   const int V = x->dtype == RG_BF16 ? 8 : 4;
-  const int64_t C = x->cols;
+  const int64_t C = x->cols, R = x->rows;
+  const size_t esz = x->dtype == RG_BF16 ? 2 : 4;
   const int64_t nblocks = (C + 32 * V - 1) / (32 * V);          // warp-blocks in a row
   int U = unroll_hint;
-  if (U != 1 && U != 2 && U != 4 && U != 8) {
-    U = nblocks >= 64 ? 8 : nblocks >= 16 ? 4 : nblocks >= 4 ? 2 : 1;
-  }
+  if (U != 1 && U != 2 && U != 4 && U != 8) U = nblocks >= 8 ? 8 : nblocks >= 4 ? 4 : nblocks >= 2 ? 2 : 1;
   const int64_t nsb = (nblocks + U - 1) / U;
-  int threads = threads_hint;
-  if (threads != 32 && threads != 64 && threads != 128 && threads != 256) {
-    threads = nsb >= 8 ? 256 : nsb >= 4 ? 128 : nsb >= 2 ? 64 : 32;
-  }
-  if (nsb > 4096) return RG_ERR_UNSUPPORTED;                   // rows beyond ~4M fp32 columns
-  const int cap = (int)((nsb + 31) / 32 * 32);
-  const size_t smem = (size_t)(2 * cap + 32) * sizeof(float);
-  const size_t esz = x->dtype == RG_BF16 ? 2 : 4;
-  const bool vec = (reinterpret_cast<uintptr_t>(x->ptr) % 16 == 0) && ((x->ld * esz) % 16 == 0);
+  if (nsb >= (1 << (MAX_LEVELS - 1))) return RG_ERR_UNSUPPORTED;   // rows beyond ~4M fp32 columns
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int64_t max_grid = (int64_t)sms * (2048 / threads);
-  const int grid = (int)(x->rows < max_grid ? x->rows : max_grid);
+
+  int threads = threads_hint;
+  const bool valid_hint = threads == 32 || threads == 64 || threads == 128 || threads == 256 || threads == 512 || threads == 1024;
+  bool warp_rows;
+  if (valid_hint) {
+    warp_rows = (threads == 32) && op != RG_OP_SOFTMAX_DENOM;
+  } else if (op == RG_OP_SOFTMAX_DENOM) {
+    // the second pass re-reads the row: keep (rows in flight) x (row bytes) near a quarter of L2
+    warp_rows = false;
+    const int64_t row_bytes = C * (int64_t)esz;
+    threads = 128;
+    while (threads < 1024 && ((int64_t)sms * (2048 / threads)) * row_bytes > (32ll << 20)) threads *= 2;
+    while (threads > 32 && nsb < threads / 32) threads /= 2;
+  } else {
+    // enough rows to give every resident warp its own: no barriers at all
+    warp_rows = R >= (int64_t)sms * 32;
+    threads = nsb >= 8 ? 256 : nsb >= 4 ? 128 : nsb >= 2 ? 64 : 32;
+  }
+  const bool vec = (reinterpret_cast<uintptr_t>(x->ptr) % 16 == 0) && ((x->ld * esz) % 16 == 0);
+  const int cap = (int)((nsb + 31) / 32 * 32);
+  size_t smem = 0;
+  int grid;
+  if (warp_rows) {
+    threads = 256;
+    const int64_t need = (R + 7) / 8, max_grid = (int64_t)sms * 8;
+    grid = (int)(need < max_grid ? need : max_grid);
+  } else {
+    smem = (size_t)(2 * cap + 32) * sizeof(float);
+    const int64_t max_grid = (int64_t)sms * (2048 / threads);
+    grid = (int)(R < max_grid ? R : max_grid);
+  }
   ReduceParams p;
   p.x = x->ptr; p.out = out->ptr;
   p.weight = args ? args->weight : nullptr;
   p.aux = args ? static_cast<float*>(args->aux_out) : nullptr;
-  p.R = x->rows; p.C = C; p.ldx = x->ld; p.ldo = out->ld;
+  p.R = R; p.C = C; p.ldx = x->ld; p.ldo = out->ld;
   p.eps = args ? args->eps : 0.0f;
   p.fma = fma; p.out_dtype = out->dtype; p.w_dtype = args ? args->weight_dtype : RG_F32; p.cap = cap;
-  cudaError_t e = x->dtype == RG_BF16 ? launch_op<uint16_t>(op, p, vec, U, threads, grid, smem, st)
-                                      : launch_op<float>(op, p, vec, U, threads, grid, smem, st);
+  cudaError_t e = x->dtype == RG_BF16 ? launch_op<uint16_t>(op, p, vec, warp_rows, U, threads, grid, smem, st)
+                                      : launch_op<float>(op, p, vec, warp_rows, U, threads, grid, smem, st);
   return e == cudaSuccess ? RG_OK : RG_ERR_CUDA;
 }
 

@@ -86,7 +86,7 @@ def test_layout_knobs_do_not_move_a_bit(op):
     """Sec. 5.2: with the tree pinned, threads per row and loads in flight are free speed knobs."""
     x = synth.spread_exponents_f32(synth.normal_f32((6, 20000), 1.0, 7), 8, -10, 10)
     ref, _ = gpu_reduce(op, x, eps=1e-5)
-    for threads in (32, 64, 128, 256):
+    for threads in (32, 64, 128, 256, 512, 1024):
         for unroll in (1, 2, 4, 8):
             got, _ = gpu_reduce(op, x, eps=1e-5, BN=threads, stages=unroll)
             assert_bits_equal(got, ref, f"threads={threads} unroll={unroll}")
