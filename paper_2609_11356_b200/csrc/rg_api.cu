@@ -294,7 +294,15 @@ rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_
   return ok ? RG_OK : RG_ERR_CUDA;
 }
 
-rg_status_t rg_device_status(uint32_t* code) { return rg::read_and_clear_status(code); }
+rg_status_t rg_device_status(uint32_t* code) {
+  uint32_t a = 0, b = 0;
+  const rg_status_t s1 = rg::read_and_clear_status(&a);          // synchronises the device
+  if (s1 == RG_ERR_CUDA) return s1;
+  const rg_status_t s2 = rg::read_and_clear_reduce_status(&b);
+  if (s2 == RG_ERR_CUDA) return s2;
+  if (code) *code = a ? a : b;
+  return (a || b) ? RG_ERR_TIMEOUT : RG_OK;
+}
 
 const char* rg_status_string(rg_status_t s) {
   switch (s) {

@@ -23,6 +23,7 @@
 
 #include "rg_common.cuh"
 #include "rg_internal.h"
+#include "rg_ptx.cuh"
 
 namespace rg {
 
@@ -35,54 +36,8 @@ constexpr int KBOX = 64;          // bf16 per 128-byte swizzle row
 constexpr int UMMA_K = 16;        // instruction_k for 16-bit inputs
 constexpr int NUM_THREADS = 320;
 constexpr int NUM_EPI_WARPS = 8;
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ uint64_t globaltimer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok;
-}
-// Bounded wait.  Returns false if the wait was abandoned (own timeout or another role's abort).
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t code) {
-  uint64_t t0 = 0;
-  for (uint32_t it = 0;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 255u) {
-      if (*abort_flag) return false;
-      const uint64_t now = globaltimer_ns();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > WAIT_LIMIT_NS) {
-        *abort_flag = 1;
-        atomicCAS(&g_status_word, 0u, code);
-        return false;
-      }
-    }
-  }
-}
+// ------------------------------------------------------------------ PTX wrappers (tensor core side)
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -281,7 +236,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         decode_work(p, w, part, tm, tn);
         const int k_begin = p.part_begin[part], k_end = p.part_end[part];
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
-          if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, 0x100u | stage)) { alive = false; break; }
+          if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, &g_status_word, 0x100u | stage)) { alive = false; break; }
           const uint32_t full = bar_full + 8u * stage;
           mbar_expect_tx(full, STAGE_BYTES);
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
@@ -306,12 +261,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         const int k_begin = p.part_begin[part], k_end = p.part_end[part];
         const int buf = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1;
-        if (!mbar_wait(bar_tempty + 8u * buf, acc_phase ^ 1u, abort_flag, 0x200u | buf)) { alive = false; break; }
+        if (!mbar_wait(bar_tempty + 8u * buf, acc_phase ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
         tcgen05_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN;
         uint32_t accumulate = 0;                        // every part starts from a zero accumulator
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
-          if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, 0x300u | stage)) { alive = false; break; }
+          if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0x300u | stage)) { alive = false; break; }
           tcgen05_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
 #pragma unroll
@@ -344,7 +299,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       decode_work(p, w, part, tm, tn);
       const int buf = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
-      if (!mbar_wait(bar_tfull + 8u * buf, acc_phase, abort_flag, 0x400u | buf)) { alive = false; break; }
+      if (!mbar_wait(bar_tfull + 8u * buf, acc_phase, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
       tcgen05_fence_after();
       const int64_t row = (int64_t)tm * BM + quarter * 32 + lane;
       const bool row_ok = row < p.M;

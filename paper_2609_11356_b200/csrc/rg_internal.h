@@ -21,5 +21,6 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
 rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* out,
                                const rg_reduce_args_t* args, int threads_hint, int unroll_hint, cudaStream_t st);
 rg_status_t read_and_clear_status(uint32_t* code);
+rg_status_t read_and_clear_reduce_status(uint32_t* code);
 
 }  // namespace rg

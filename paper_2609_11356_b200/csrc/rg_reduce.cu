@@ -21,12 +21,14 @@
 //   reduce_rows_warp_kernel  one warp owns a row: no barriers, all warps independent.  Used
 //                            for sums and RMSNorm when there are enough rows to fill the GPU.
 //   reduce_rows_cta_kernel   one CTA owns a row (32..1024 threads).  Used for few rows, and for
-//                            the softmax normaliser, whose second pass re-reads the row: the rows
-//                            in flight (CTAs x row bytes) are kept well inside L2.
+//                            the softmax normaliser, whose second pass re-reads the row (from L2).
 #include "rg_common.cuh"
 #include "rg_internal.h"
+#include "rg_ptx.cuh"
 
 namespace rg {
+
+__device__ unsigned int g_reduce_status_word = 0;
 
 namespace {
 
@@ -341,6 +343,83 @@ __global__ void __launch_bounds__(1024) reduce_rows_cta_kernel(const ReduceParam
   }
 }
 
+// ------------------------------------------------------------------ RMSNorm, row kept in registers
+// One CTA per row; every warp owns at most one super-block of U vectors per lane and keeps the
+// raw vectors, so the row is read from memory exactly once.  Needs 16-byte aligned rows whose
+// length is a multiple of V.
+template <typename T, int U>
+__global__ void __launch_bounds__(256) rmsnorm_keep_kernel(const ReduceParams p) {
+  __shared__ float sb[8];
+  constexpr int V = VecTraits<T>::V;
+  constexpr int WB = 32 * V;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const bool out_vec = rms_out_vec<T, true>(p);
+  for (int64_t row = blockIdx.x; row < p.R; row += gridDim.x) {
+    const T* xr = static_cast<const T*>(p.x) + row * p.ldx;
+    const int64_t base = (int64_t)warp * WB * U + lane * V;
+    uint4 raw[U];
+    float bv[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int64_t c = base + (int64_t)u * WB;
+      raw[u] = c + V <= p.C ? __ldg(reinterpret_cast<const uint4*>(xr + c)) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      float x[V];
+      unpack<T>(raw[u], x);
+      bv[u] = (base + (int64_t)u * WB + V <= p.C) ? fold_block<OP_RMS, V, true>(x, V, 0.0f, p.fma) : NEG_ZERO;
+    }
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1)
+#pragma unroll
+      for (int u = 0; u < U; ++u) bv[u] = f_add(bv[u], __shfl_xor_sync(0xffffffffu, bv[u], off));
+#pragma unroll
+    for (int s2 = 1; s2 < U; s2 <<= 1)
+#pragma unroll
+      for (int u = 0; u < U; u += 2 * s2) bv[u] = f_add(bv[u], bv[u + s2]);
+    if (lane == 0) sb[warp] = bv[0];
+    __syncthreads();
+    float root = (lane < nwarps) ? sb[lane] : NEG_ZERO;   // nwarps <= 8 super-blocks, padded with the identity
+#pragma unroll
+    for (int off = 1; off < 8; off <<= 1) root = f_add(root, __shfl_xor_sync(0xffffffffu, root, off));
+    root = __shfl_sync(0xffffffffu, root, 0);
+    __syncthreads();
+    const float rinv = rms_rinv(root, p.C, p.eps);
+    if (threadIdx.x == 0 && p.aux) p.aux[row] = rinv;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int64_t c = base + (int64_t)u * WB;
+      if (c + V > p.C) continue;
+      float x[V], w[V], y[V];
+      unpack<T>(raw[u], x);
+      const bool w_vec = p.weight && ((reinterpret_cast<uintptr_t>(p.weight) & 15) == 0) &&
+                         p.w_dtype == (sizeof(T) == 2 ? RG_BF16 : RG_F32);
+      if (w_vec) unpack<T>(__ldg(reinterpret_cast<const uint4*>(static_cast<const T*>(p.weight) + c)), w);
+      else {
+#pragma unroll
+        for (int t = 0; t < V; ++t) w[t] = p.weight ? load_scalar(p.weight, p.w_dtype, c + t) : 1.0f;
+      }
+#pragma unroll
+      for (int t = 0; t < V; ++t) y[t] = f_mul(f_mul(x[t], rinv), w[t]);
+      if (out_vec) {
+        if constexpr (sizeof(T) == 4)
+          *reinterpret_cast<uint4*>(static_cast<float*>(p.out) + row * p.ldo + c) =
+              make_uint4(__float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]), __float_as_uint(y[3]));
+        else
+          *reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + row * p.ldo + c) =
+              make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
+      } else {
+#pragma unroll
+        for (int t = 0; t < V; ++t) {
+          if (p.out_dtype == RG_BF16) static_cast<__nv_bfloat16*>(p.out)[row * p.ldo + c + t] = __float2bfloat16_rn(y[t]);
+          else static_cast<float*>(p.out)[row * p.ldo + c + t] = y[t];
+        }
+      }
+    }
+  }
+}
+
 template <typename T, int OP, bool VEC, int U>
 cudaError_t launch_kernel(const ReduceParams& p, bool warp_rows, int threads, int grid, size_t smem, cudaStream_t st) {
   if constexpr (OP != OP_SOFTMAX) {
@@ -403,11 +482,11 @@ rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_t
   if (valid_hint) {
     warp_rows = (threads == 32) && op != RG_OP_SOFTMAX_DENOM;
   } else if (op == RG_OP_SOFTMAX_DENOM) {
-    // the second pass re-reads the row: keep (rows in flight) x (row bytes) near a quarter of L2
+    // The second pass re-reads the row from L2.  Eight CTAs of 256 threads per SM measured best on
+    // 32768-column rows: enough CTAs in different phases to overlap the DRAM-bound maximum pass
+    // with the ALU-bound exp pass.
     warp_rows = false;
-    const int64_t row_bytes = C * (int64_t)esz;
-    threads = 128;
-    while (threads < 1024 && ((int64_t)sms * (2048 / threads)) * row_bytes > (32ll << 20)) threads *= 2;
+    threads = 256;
     while (threads > 32 && nsb < threads / 32) threads /= 2;
   } else {
     // enough rows to give every resident warp its own: no barriers at all
@@ -415,6 +494,31 @@ rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_t
     threads = nsb >= 8 ? 256 : nsb >= 4 ? 128 : nsb >= 2 ? 64 : 32;
   }
   const bool vec = (reinterpret_cast<uintptr_t>(x->ptr) % 16 == 0) && ((x->ld * esz) % 16 == 0);
+  ReduceParams p;
+  p.x = x->ptr; p.out = out->ptr;
+  p.weight = args ? args->weight : nullptr;
+  p.aux = args ? static_cast<float*>(args->aux_out) : nullptr;
+  p.R = R; p.C = C; p.ldx = x->ld; p.ldo = out->ld;
+  p.eps = args ? args->eps : 0.0f;
+  p.fma = fma; p.out_dtype = out->dtype; p.w_dtype = args ? args->weight_dtype : RG_F32; p.cap = 0;
+
+  // RMSNorm of rows short enough to live in registers: each row is read once.
+  if (op == RG_OP_RMSNORM && !valid_hint && vec && C % V == 0 && nblocks <= 32) {
+    const int Uk = nblocks >= 16 ? 4 : nblocks >= 4 ? 2 : 1;
+    const int warps = (int)((nblocks + Uk - 1) / Uk);          // <= 8
+    const int64_t max_grid = (int64_t)sms * (2048 / (warps * 32));
+    const int grid = (int)(R < max_grid ? R : max_grid);
+    if (x->dtype == RG_BF16) {
+      if (Uk == 4) rmsnorm_keep_kernel<uint16_t, 4><<<grid, warps * 32, 0, st>>>(p);
+      else if (Uk == 2) rmsnorm_keep_kernel<uint16_t, 2><<<grid, warps * 32, 0, st>>>(p);
+      else rmsnorm_keep_kernel<uint16_t, 1><<<grid, warps * 32, 0, st>>>(p);
+    } else {
+      if (Uk == 4) rmsnorm_keep_kernel<float, 4><<<grid, warps * 32, 0, st>>>(p);
+      else if (Uk == 2) rmsnorm_keep_kernel<float, 2><<<grid, warps * 32, 0, st>>>(p);
+      else rmsnorm_keep_kernel<float, 1><<<grid, warps * 32, 0, st>>>(p);
+    }
+    return cudaGetLastError() == cudaSuccess ? RG_OK : RG_ERR_CUDA;
+  }
   const int cap = (int)((nsb + 31) / 32 * 32);
   size_t smem = 0;
   int grid;
@@ -427,16 +531,18 @@ rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_t
     const int64_t max_grid = (int64_t)sms * (2048 / threads);
     grid = (int)(R < max_grid ? R : max_grid);
   }
-  ReduceParams p;
-  p.x = x->ptr; p.out = out->ptr;
-  p.weight = args ? args->weight : nullptr;
-  p.aux = args ? static_cast<float*>(args->aux_out) : nullptr;
-  p.R = R; p.C = C; p.ldx = x->ld; p.ldo = out->ld;
-  p.eps = args ? args->eps : 0.0f;
-  p.fma = fma; p.out_dtype = out->dtype; p.w_dtype = args ? args->weight_dtype : RG_F32; p.cap = cap;
+  p.cap = cap;
   cudaError_t e = x->dtype == RG_BF16 ? launch_op<uint16_t>(op, p, vec, warp_rows, U, threads, grid, smem, st)
                                       : launch_op<float>(op, p, vec, warp_rows, U, threads, grid, smem, st);
   return e == cudaSuccess ? RG_OK : RG_ERR_CUDA;
+}
+
+rg_status_t read_and_clear_reduce_status(uint32_t* code) {
+  unsigned int v = 0, zero = 0;
+  if (cudaMemcpyFromSymbol(&v, g_reduce_status_word, sizeof(v)) != cudaSuccess) return RG_ERR_CUDA;
+  if (v != 0 && cudaMemcpyToSymbol(g_reduce_status_word, &zero, sizeof(zero)) != cudaSuccess) return RG_ERR_CUDA;
+  if (code) *code = v;
+  return v ? RG_ERR_TIMEOUT : RG_OK;
 }
 
 }  // namespace rg

@@ -57,6 +57,38 @@ def test_rmsnorm_bit_exact(shape, dtype, fma):
     assert_bits_equal(grinv, wrinv, "1/rms")
 
 
+@pytest.mark.parametrize("shape", [(300, 8192), (200, 20000), (150, 32764), (160, 12292), (149, 32768), (700, 8196), (150, 49152)])
+@pytest.mark.parametrize("spread", [False, True])
+def test_softmax_normaliser_staged_rows_bit_exact(shape, spread):
+    """fp32 rows between 8192 and 32768 columns with at least one row per SM take the kernel that
+    stages whole rows in shared memory; ragged last chunks and exponent-spread draws included."""
+    x = synth.normal_f32(shape, 100.0, 31)
+    if spread:
+        x = synth.spread_exponents_f32(synth.normal_f32(shape, 1.0, 32), 33, -6, 6)
+    got, gmax = gpu_reduce(rg.RG_OP_SOFTMAX_DENOM, x)
+    want, wmax = rgo.reduce_rows(rgo.OP_SOFTMAX_DENOM, x)
+    assert_bits_equal(got, want, f"staged softmax normaliser {shape}")
+    assert_bits_equal(gmax, wmax, "row max")
+    # the generic kernel gives the same bits
+    other, _ = gpu_reduce(rg.RG_OP_SOFTMAX_DENOM, x, BN=256)
+    assert_bits_equal(other, got, "staged vs CTA-per-row kernel")
+    assert rg.rg_device_status() == 0
+
+
+@pytest.mark.parametrize("shape", [(500, 4096), (77, 8192), (40, 2048), (9, 520), (300, 3000)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_rmsnorm_register_resident_rows_match_generic_kernels(shape, dtype):
+    x = _draw(shape, dtype, 41, True)
+    w = synth.normal_bf16((shape[1],), 0.05, 42, mean=1.0) if dtype == "bf16" else synth.normal_f32((shape[1],), 0.05, 42, mean=1.0)
+    got, gr = gpu_reduce(rg.RG_OP_RMSNORM, x, weight=w, eps=1e-5)
+    want, wr = rgo.reduce_rows(rgo.OP_RMSNORM, x, weight=w, eps=1e-5)
+    assert_bits_equal(got, want, f"rmsnorm {shape} {dtype}")
+    assert_bits_equal(gr, wr, "1/rms")
+    for threads in (32, 128):
+        other, _ = gpu_reduce(rg.RG_OP_RMSNORM, x, weight=w, eps=1e-5, BN=threads)
+        assert_bits_equal(other, got, f"generic kernel, threads={threads}")
+
+
 def test_rmsnorm_mixed_types_and_no_weight():
     x = synth.normal_bf16((17, 520), 1.0, 3)
     got, _ = gpu_reduce(rg.RG_OP_RMSNORM, x, eps=1e-6, out_dtype=torch.float32)
