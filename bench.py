@@ -215,14 +215,14 @@ def run_ours(args):
                        "row_sum_gbs": round(sum_gbs, 1),
                        "softmax_gbs": round((4.0 * RED_R * RED_C + 8.0 * RED_R) / (mean[5] * 1e-3) / 1e9, 1),
                        "rmsnorm_gbs": round((4.0 * RMS_R * RMS_C) / (mean[4] * 1e-3) / 1e9, 1)},
-            "roofline": {"bound": "tensor", "kernel": "gemm_tcgen05_kernel<256,1> on 8192^3",
+            "roofline": {"bound": "tensor", "kernel": "gemm_tcgen05_pair_kernel<256,2> (two-SM tiles 256x256x128) on 8192^3",
                          "achieved": round(sq_tflops, 1), "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                          "frac": round(sq_tflops / peaks["bf16_tflops_sustained"], 4),
                          "frac_of_burst_peak": round(sq_tflops / peaks["bf16_tflops"], 4),
                          "frac_of_nominal_2250": round(sq_tflops / 2250.0, 4),
                          "peak_source": peaks["source"] + " (sustained: the kernel is timed inside a long step)",
                          "traffic": NCU_TRAFFIC_BYTES["gemm_8192"]},
-            "roofline_reduce": {"bound": "hbm", "kernel": "reduce_rows_kernel<float,SUM> on 65536x32768",
+            "roofline_reduce": {"bound": "hbm", "kernel": "reduce_rows_warp_kernel<float,SUM> on 65536x32768",
                                 "achieved": round(sum_gbs, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                 "frac": round(sum_gbs / peaks["hbm_gbs"], 4), "frac_of_nominal_8000": round(sum_gbs / 8000.0, 4),
                                 "peak_source": peaks["source"], "traffic": NCU_TRAFFIC_BYTES["row_sum_65536x32768"]},

@@ -32,10 +32,12 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
   if (d->in_dtype != RG_BF16 || d->acc_dtype != RG_F32 || d->partial_dtype != RG_F32 || d->merge_dtype != RG_F32)
     return RG_ERR_UNSUPPORTED;
   if (d->atom != RG_ATOM_TC_BF16_K16 || d->k_tail != 0) return RG_ERR_UNSUPPORTED;
-  if (d->BM != 0 && d->BM != 128) return RG_ERR_UNSUPPORTED;
+  if (d->BM != 0 && d->BM != 128 && d->BM != 256) return RG_ERR_UNSUPPORTED;
   if (d->BN != 0 && d->BN != 64 && d->BN != 128 && d->BN != 256) return RG_ERR_UNSUPPORTED;
   if (d->BK != 0 && d->BK != 64 && d->BK != 128) return RG_ERR_UNSUPPORTED;
-  if (d->cta_group > 1) return RG_ERR_UNSUPPORTED;
+  if (d->cta_group > 2) return RG_ERR_INVALID_DESC;
+  if (d->cta_group == 2 && (d->BM == 128 || d->BN == 64)) return RG_ERR_UNSUPPORTED;   // a pair works on 256 rows, BN >= 128
+  if (d->cta_group == 1 && d->BM == 256) return RG_ERR_UNSUPPORTED;
   if (d->raster > 64) return RG_ERR_INVALID_DESC;
   for (uint32_t i = 0; i < d->n_cuts; ++i)
     if (d->cuts[i] % 16 != 0) return RG_ERR_UNSUPPORTED;   // a cut may not split a 16-wide step
@@ -80,7 +82,6 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
     plan->part_begin[s] = s == 0 ? 0 : (int32_t)d->cuts[s - 1];
     plan->part_end[s] = s == plan->n_parts - 1 ? (int32_t)K : (int32_t)d->cuts[s];
   }
-  plan->BK = d->BK ? d->BK : 64;
   if (d->BN) plan->BN = d->BN;
   else {
     // largest tile that still gives every SM a work item
@@ -91,7 +92,15 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
       if (tiles_m * ((N + bn - 1) / bn) * plan->n_parts >= sms) { plan->BN = bn; break; }
     }
   }
-  const int smax = rg::max_stages_for(plan->BN, plan->BK);
+  // one CTA per 128-row tile, or a pair of CTAs (two SMs) per 256-row tile
+  if (d->cta_group) plan->cta_group = d->cta_group;
+  else if (d->BM == 256) plan->cta_group = 2;
+  else if (d->BM == 128) plan->cta_group = 1;
+  else plan->cta_group = (plan->BN >= 128 && M > 128 && ((M + 255) / 256) * ((N + plan->BN - 1) / plan->BN) * plan->n_parts >= device_sms() / 2) ? 2 : 1;
+  if (plan->cta_group == 2 && plan->BN < 128) plan->cta_group = 1;
+  // a pair moves half the B bytes per CTA, so a 128-wide K step fits three times: fewer hand-offs per k
+  plan->BK = d->BK ? d->BK : (plan->cta_group == 2 && plan->BN == 256 ? 128 : 64);
+  const int smax = rg::max_stages_for(plan->BN, plan->BK, plan->cta_group);
   plan->stages = d->stages ? d->stages : smax;
   if (plan->stages > smax) return RG_ERR_UNSUPPORTED;
   plan->raster = d->raster == 1 ? 1 : 0;

@@ -81,6 +81,56 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- two-SM (cta_group::2) forms: a pair of CTAs in a cluster works on one 256-row tile
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same variable in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// The box lands in this CTA's shared memory; its bytes are counted on `bar`, which may live in the peer.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// Arrive on the barrier at this offset in both CTAs of the pair once the steps issued so far are done.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 // Shared-memory matrix descriptor for a K-major bf16 tile whose rows are 128 bytes, stored
 // with the 128-byte swizzle TMA produced: 8-row groups are 1024 bytes apart.
 __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
@@ -93,9 +143,9 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
   return d;
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = BN.
-__host__ __device__ constexpr uint32_t make_idesc(int bn) {
+__host__ __device__ constexpr uint32_t make_idesc(int bn, int m = BM) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(bn >> 3) << 17) |
-         (static_cast<uint32_t>(BM >> 4) << 24);
+         (static_cast<uint32_t>(m >> 4) << 24);
 }
 
 struct GemmParams {
@@ -179,6 +229,42 @@ __device__ __forceinline__ void store_row_segment(const GemmParams& p, int64_t r
     } else {
 #pragma unroll
       for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = v[c];
+    }
+  }
+}
+
+// Epilogue of one accumulator tile for one warp: the warp's 32 TMEM lanes (one output row per
+// thread), 32-column chunks chunk0, chunk0+2, ...  Split-K parts go to the workspace at fp32,
+// untouched (Sec. 3.2.2); otherwise bias / SiLU / residual and one rounding to the output type.
+template <int BN>
+__device__ __forceinline__ void epilogue_tile(const GemmParams& p, int part, int64_t row, bool row_ok, int tn,
+                                              uint32_t taddr, int chunk0) {
+#pragma unroll 1
+  for (int c0 = chunk0 * 32; c0 < BN; c0 += 64) {
+    const int col0 = tn * BN + c0;
+    if (col0 >= p.N) break;                               // uniform across the warp
+    uint32_t r[32];
+    tmem_ld_32x32b_x32(taddr + c0, r);
+    tmem_ld_wait();
+    const int ncols = min(32, p.N - col0);
+    if (row_ok) {
+      if (p.ws) {
+        float* dst = p.ws + ((int64_t)part * p.M + row) * p.ldw + col0;
+        if (ncols == 32) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            reinterpret_cast<uint4*>(dst)[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __uint_as_float(r[c]);
+        }
+      } else {
+        float v[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(r[c]);
+        epilogue_row_segment(v, p.epi, row, col0, ncols);
+        store_row_segment(p, row, col0, ncols, v);
+      }
     }
   }
 }
@@ -304,35 +390,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       const int64_t row = (int64_t)tm * BM + quarter * 32 + lane;
       const bool row_ok = row < p.M;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
-#pragma unroll 1
-      for (int c0 = chunk0 * 32; c0 < BN; c0 += 64) {
-        const int col0 = tn * BN + c0;
-        if (col0 >= p.N) break;                           // uniform across the warp
-        uint32_t r[32];
-        tmem_ld_32x32b_x32(taddr + c0, r);
-        tmem_ld_wait();
-        const int ncols = min(32, p.N - col0);
-        if (row_ok) {
-          if (p.ws) {
-            // split-K: the finished part is written at fp32, untouched (Sec. 3.2.2)
-            float* dst = p.ws + ((int64_t)part * p.M + row) * p.ldw + col0;
-            if (ncols == 32) {
-#pragma unroll
-              for (int q = 0; q < 8; ++q)
-                reinterpret_cast<uint4*>(dst)[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
-            } else {
-#pragma unroll
-              for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __uint_as_float(r[c]);
-            }
-          } else {
-            float v[32];
-#pragma unroll
-            for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(r[c]);
-            epilogue_row_segment(v, p.epi, row, col0, ncols);
-            store_row_segment(p, row, col0, ncols, v);
-          }
-        }
-      }
+      epilogue_tile<BN>(p, part, row, row_ok, tn, taddr, chunk0);
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
@@ -350,6 +408,159 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   if (warp == 1) {
     tcgen05_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------ two-SM kernel
+// Same arithmetic, different schedule: two CTAs of a cluster share one 256 x BN output tile.
+// CTA r loads rows [128r, 128r+128) of the A tile and rows [BN/2*r, ...) of the B tile into its own
+// shared memory; the even CTA issues tcgen05.mma.cta_group::2 (M = 256), which reads both CTAs'
+// shared memory and writes each CTA's 128 rows of the accumulator into that CTA's tensor memory.
+// Each CTA moves half the B bytes, so a stage is 16 KiB + BN*64 B and the ring is deeper.
+//   full[s]   lives in the even CTA; both CTAs' boxes count their bytes on it
+//   empty[s]  in each CTA; tcgen05.commit arrives on both
+//   tfull[b]  in each CTA; tcgen05.commit arrives on both
+//   tempty[b] in the even CTA; the epilogue warps of both CTAs arrive on it
+template <int BN, int KSUB>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                         const GemmParams p) {
+  constexpr uint32_t A_BOX_BYTES = BM * KBOX * 2;
+  constexpr uint32_t B_BOX_BYTES = (BN / 2) * KBOX * 2;
+  constexpr uint32_t STAGE_BYTES = KSUB * (A_BOX_BYTES + B_BOX_BYTES);      // per CTA
+  constexpr uint32_t TMEM_COLS = 2 * BN;
+  constexpr uint32_t IDESC = make_idesc(BN, 2 * BM);
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const int S = p.num_stages;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + (size_t)S * STAGE_BYTES);
+  const uint32_t bar_full = smem_u32(bars);
+  const uint32_t bar_empty = bar_full + 8u * S;
+  const uint32_t bar_tfull = bar_empty + 8u * S;
+  const uint32_t bar_tempty = bar_tfull + 16u;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();                 // 0 = the CTA that issues the steps
+  const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  const int total_work = p.tiles_m * p.tiles_n * p.n_parts;   // tiles_m counts 256-row tiles here
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8u * s, 1); mbar_init(bar_empty + 8u * s, 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8u * b, 1); mbar_init(bar_tempty + 8u * b, 2 * NUM_EPI_WARPS); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
+    tmem_relinquish_pair();
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                      // both CTAs' barriers exist before any remote arrive
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      bool alive = true;
+      for (int w = pair_id; w < total_work && alive; w += num_pairs) {
+        int part, tm, tn;
+        decode_work(p, w, part, tm, tn);
+        const int k_begin = p.part_begin[part], k_end = p.part_end[part];
+        for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
+          if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, &g_status_word, 0x900u | stage)) { alive = false; break; }
+          const uint32_t full_local = bar_full + 8u * stage;
+          if (rank == 0) mbar_expect_tx(full_local, 2u * STAGE_BYTES);      // bytes of both CTAs
+          const uint32_t full = map_to_cta(full_local, 0);
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+#pragma unroll
+          for (int sub = 0; sub < KSUB; ++sub) {
+            tma_load_2d_pair(sa + sub * A_BOX_BYTES, &tmap_a, k0 + sub * KBOX, tm * 2 * BM + (int)rank * BM, full);
+            tma_load_2d_pair(sa + KSUB * A_BOX_BYTES + sub * B_BOX_BYTES, &tmap_b, k0 + sub * KBOX,
+                             tn * BN + (int)rank * (BN / 2), full);
+          }
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (even CTA only)
+    if (lane == 0 && rank == 0) {
+      int stage = 0; uint32_t phase = 0;
+      bool alive = true;
+      int it = 0;
+      for (int w = pair_id; w < total_work && alive; w += num_pairs, ++it) {
+        int part, tm, tn;
+        decode_work(p, w, part, tm, tn);
+        const int k_begin = p.part_begin[part], k_end = p.part_end[part];
+        const int buf = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1;
+        if (!mbar_wait(bar_tempty + 8u * buf, acc_phase ^ 1u, abort_flag, &g_status_word, 0xa00u | buf)) { alive = false; break; }
+        tcgen05_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        uint32_t accumulate = 0;                        // every part starts from a zero accumulator
+        for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
+          if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0xb00u | stage)) { alive = false; break; }
+          tcgen05_fence_after();
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+#pragma unroll
+          for (int sub = 0; sub < KSUB; ++sub) {
+            const uint64_t adesc = make_kmajor_sw128_desc(sa + sub * A_BOX_BYTES);
+            const uint64_t bdesc = make_kmajor_sw128_desc(sa + KSUB * A_BOX_BYTES + sub * B_BOX_BYTES);
+#pragma unroll
+            for (int a = 0; a < KBOX / UMMA_K; ++a) {
+              if (k0 + sub * KBOX + a * UMMA_K < k_end) {   // ascending k; nothing past the end of the part
+                umma_bf16_pair(d_tmem, adesc + 2u * a, bdesc + 2u * a, IDESC, accumulate);
+                accumulate = 1;
+              }
+            }
+          }
+          umma_commit_pair(bar_empty + 8u * stage);      // frees the stage in both CTAs
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+        if (alive) umma_commit_pair(bar_tfull + 8u * buf);   // accumulator complete, in both CTAs
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps (both CTAs)
+    const int quarter = warp & 3;
+    const int chunk0 = (warp - 2) >> 2;
+    const uint32_t tempty_leader = map_to_cta(bar_tempty, 0);
+    bool alive = true;
+    int it = 0;
+    for (int w = pair_id; w < total_work && alive; w += num_pairs, ++it) {
+      int part, tm, tn;
+      decode_work(p, w, part, tm, tn);
+      const int buf = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1;
+      if (!mbar_wait(bar_tfull + 8u * buf, acc_phase, abort_flag, &g_status_word, 0xc00u | buf)) { alive = false; break; }
+      tcgen05_fence_after();
+      const int64_t row = (int64_t)tm * 2 * BM + (int64_t)rank * BM + quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
+      epilogue_tile<BN>(p, part, row, row < p.M, tn, taddr, chunk0);
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(tempty_leader + 8u * buf);
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  __syncthreads();
+  if (*abort_flag) {
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  cluster_sync_all();          // the peer may still be reading this CTA's shared memory or arriving on its barriers
+  if (warp == 1) {
+    tcgen05_fence_after();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
   }
 }
 
@@ -455,6 +666,33 @@ size_t smem_bytes_for(int bn, int ksub, int stages) {
   return 1024 + stages * stage + (2 * stages + 4) * 8 + 16;
 }
 
+size_t smem_bytes_for_pair(int bn, int ksub, int stages) {
+  const size_t stage = (size_t)ksub * (BM * KBOX * 2 + (size_t)(bn / 2) * KBOX * 2);
+  return 1024 + stages * stage + (2 * stages + 4) * 8 + 16;
+}
+
+template <int BN, int KSUB>
+cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
+  const size_t smem = smem_bytes_for_pair(BN, KSUB, p.num_stages);
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_pair_kernel<BN, KSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_pair_kernel<BN, KSUB>, ta, tb, p);
+}
+
 template <int BN, int KSUB>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   const size_t smem = smem_bytes_for(BN, KSUB, p.num_stages);
@@ -470,10 +708,11 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmP
 
 }  // namespace
 
-int max_stages_for(int bn, int bk) {
+int max_stages_for(int bn, int bk, int cta_group) {
   const int ksub = bk / KBOX;
   int s = 1;
-  while (s < 8 && smem_bytes_for(bn, ksub, s + 1) <= SMEM_LIMIT) ++s;
+  if (cta_group == 2) { while (s < 8 && smem_bytes_for_pair(bn, ksub, s + 1) <= SMEM_LIMIT) ++s; }
+  else { while (s < 8 && smem_bytes_for(bn, ksub, s + 1) <= SMEM_LIMIT) ++s; }
   return s;
 }
 
@@ -490,12 +729,15 @@ rg_status_t read_and_clear_status(uint32_t* code) {
 rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
                         const rg_epilogue_t* epi, void* ws, cudaStream_t st) {
   const int64_t M = A->rows, K = A->cols, N = B->rows;
+  const bool pair = plan.cta_group == 2;
+  const int tile_m = pair ? 2 * BM : BM;
   CUtensorMap ta, tb;
-  if (!make_tmap(&ta, A->ptr, M, K, A->ld, BM) || !make_tmap(&tb, B->ptr, N, K, B->ld, plan.BN)) return RG_ERR_CUDA;
+  if (!make_tmap(&ta, A->ptr, M, K, A->ld, BM) || !make_tmap(&tb, B->ptr, N, K, B->ld, pair ? plan.BN / 2 : plan.BN))
+    return RG_ERR_CUDA;
 
   GemmParams p;
   p.M = (int32_t)M; p.N = (int32_t)N; p.K = (int32_t)K;
-  p.tiles_m = (int32_t)((M + BM - 1) / BM);
+  p.tiles_m = (int32_t)((M + tile_m - 1) / tile_m);
   p.tiles_n = (int32_t)((N + plan.BN - 1) / plan.BN);
   p.n_parts = plan.n_parts;
   p.num_stages = plan.stages;
@@ -517,16 +759,26 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int grid = (int)(total < sms ? total : sms);
   cudaError_t err;
   const int ksub = plan.BK / KBOX;
-  if (plan.BN == 256 && ksub == 1) err = launch_one<256, 1>(ta, tb, p, grid, st);
-  else if (plan.BN == 256 && ksub == 2) err = launch_one<256, 2>(ta, tb, p, grid, st);
-  else if (plan.BN == 128 && ksub == 1) err = launch_one<128, 1>(ta, tb, p, grid, st);
-  else if (plan.BN == 128 && ksub == 2) err = launch_one<128, 2>(ta, tb, p, grid, st);
-  else if (plan.BN == 64 && ksub == 1) err = launch_one<64, 1>(ta, tb, p, grid, st);
-  else if (plan.BN == 64 && ksub == 2) err = launch_one<64, 2>(ta, tb, p, grid, st);
-  else return RG_ERR_UNSUPPORTED;
+  if (pair) {
+    const int64_t pairs = sms / 2;
+    const int grid = 2 * (int)(total < pairs ? total : pairs);
+    if (plan.BN == 256 && ksub == 1) err = launch_pair<256, 1>(ta, tb, p, grid, st);
+    else if (plan.BN == 256 && ksub == 2) err = launch_pair<256, 2>(ta, tb, p, grid, st);
+    else if (plan.BN == 128 && ksub == 1) err = launch_pair<128, 1>(ta, tb, p, grid, st);
+    else if (plan.BN == 128 && ksub == 2) err = launch_pair<128, 2>(ta, tb, p, grid, st);
+    else return RG_ERR_UNSUPPORTED;
+  } else {
+    const int grid = (int)(total < sms ? total : sms);
+    if (plan.BN == 256 && ksub == 1) err = launch_one<256, 1>(ta, tb, p, grid, st);
+    else if (plan.BN == 256 && ksub == 2) err = launch_one<256, 2>(ta, tb, p, grid, st);
+    else if (plan.BN == 128 && ksub == 1) err = launch_one<128, 1>(ta, tb, p, grid, st);
+    else if (plan.BN == 128 && ksub == 2) err = launch_one<128, 2>(ta, tb, p, grid, st);
+    else if (plan.BN == 64 && ksub == 1) err = launch_one<64, 1>(ta, tb, p, grid, st);
+    else if (plan.BN == 64 && ksub == 2) err = launch_one<64, 2>(ta, tb, p, grid, st);
+    else return RG_ERR_UNSUPPORTED;
+  }
   if (err != cudaSuccess) return RG_ERR_CUDA;
 
   if (split) {

@@ -9,13 +9,13 @@ namespace rg {
 
 // A validated launch plan: speed knobs resolved, parts laid out.
 struct GemmPlan {
-  int BN, BK, stages, raster, group_m;
+  int BN, BK, stages, raster, group_m, cta_group;
   int n_parts, tree;
   int32_t part_begin[RG_MAX_CUTS + 1];
   int32_t part_end[RG_MAX_CUTS + 1];
 };
 
-int max_stages_for(int bn, int bk);
+int max_stages_for(int bn, int bk, int cta_group);
 rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
                         const rg_epilogue_t* epi, void* ws, cudaStream_t st);
 rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* out,

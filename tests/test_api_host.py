@@ -38,7 +38,10 @@ def test_validate_rules():
     assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_SCALAR), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(BN=96), 64, 256, 512) == 3
-    assert rg.rg_desc_validate(rg.rg_desc(cta_group=2), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(cta_group=2), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(cta_group=3), 64, 256, 512) == 2
+    assert rg.rg_desc_validate(rg.rg_desc(cta_group=2, BN=64), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(cta_group=1, BM=256), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(tree=7), 64, 256, 512) == 2
     assert rg.rg_desc_validate(ok, 64, 256, 0) == 4
     bad = rg.rg_desc(); bad.size = 12
@@ -51,7 +54,7 @@ def test_class_key_holds_order_fields_only():
     k = rg.rg_desc_class(base)
     assert k != 0
     # speed knobs do not move the class (Sec. 3.2.2)
-    for kw in (dict(BN=64), dict(BN=256, BK=128), dict(stages=2), dict(raster=1), dict(BM=128)):
+    for kw in (dict(BN=64), dict(BN=256, BK=128), dict(stages=2), dict(raster=1), dict(BM=128), dict(BM=256), dict(cta_group=2)):
         assert rg.rg_desc_class(rg.rg_desc(cuts=(1792, 3584), **kw)) == k
     # every order-deciding field does
     others = [rg.rg_desc(cuts=(1792,)), rg.rg_desc(cuts=(1792, 3600)), rg.rg_desc(),

@@ -41,7 +41,8 @@ def test_tiny_descriptor_check_full_oracle_compare():
 # ------------------------------------------------------------------ exactness
 @pytest.mark.parametrize("M,N,K", [(1, 1, 16), (1, 8, 8), (3, 5, 24), (128, 64, 64), (129, 65, 80), (300, 520, 1000),
                                    (7, 4096, 1024), (2000, 3000, 2048), (64, 100, 72)])
-@pytest.mark.parametrize("knobs", [dict(), dict(BN=64), dict(BN=128, BK=128), dict(BN=256, stages=2, raster=1)])
+@pytest.mark.parametrize("knobs", [dict(), dict(BN=64), dict(BN=128, BK=128), dict(BN=256, stages=2, raster=1),
+                                   dict(cta_group=1, BN=256), dict(cta_group=2, BN=256, BK=64), dict(BM=256, BN=128, BK=128, raster=4)])
 def test_integer_inputs_exact(M, N, K, knobs):
     A = synth.int_valued_bf16((M, K), -8, 8, K + M); B = synth.int_valued_bf16((N, K), -8, 8, K + N + 1)
     assert_bits_equal(gpu_gemm(A, B, out_dtype=rgo.F32, **knobs), _exact_int(A, B), f"ints {M}x{N}x{K} {knobs}")
@@ -64,6 +65,9 @@ def test_integer_split_k_exact(cuts, tree):
     K = max(cuts) + 40
     A = synth.int_valued_bf16((70, K), -8, 8, 1); B = synth.int_valued_bf16((90, K), -8, 8, 2)
     assert_bits_equal(gpu_gemm(A, B, cuts=cuts, tree=tree, out_dtype=rgo.F32), _exact_int(A, B), f"cuts {cuts[:4]}")
+    A = synth.int_valued_bf16((300, K), -8, 8, 3); B = synth.int_valued_bf16((260, K), -8, 8, 4)
+    assert_bits_equal(gpu_gemm(A, B, cuts=cuts, tree=tree, out_dtype=rgo.F32, cta_group=2, BN=128), _exact_int(A, B),
+                      f"two-SM tiles, cuts {cuts[:4]}")
 
 
 # ------------------------------------------------------------------ atom model
@@ -71,9 +75,10 @@ def test_integer_split_k_exact(cuts, tree):
                                         (40, 72, 2048, (512, 1024, 1536)), (16, 64, 576, (192, 384))])
 def test_random_inputs_bit_exact_under_fitted_atom_model(M, N, K, cuts):
     for name, A, B in _draws(M, N, K, 40 + K):
-        got = gpu_gemm(A, B, cuts=cuts, out_dtype=rgo.F32)
         want = rgo.gemm(A, B, cuts=cuts, atom_model=HW, out_dtype=rgo.F32)
-        assert_bits_equal(got, want, f"{M}x{N}x{K} {name}")
+        for knobs in (dict(), dict(cta_group=2, BN=128), dict(cta_group=2, BN=256)):
+            got = gpu_gemm(A, B, cuts=cuts, out_dtype=rgo.F32, **knobs)
+            assert_bits_equal(got, want, f"{M}x{N}x{K} {name} {knobs}")
 
 
 @pytest.mark.parametrize("K", [512, 4096, 14336])
@@ -115,7 +120,7 @@ def test_position_independence_of_one_k_vector():
     b = synth.spread_exponents_bf16(synth.normal_bf16((1, K), 1.0, 72), 73, -8, 8)
     A = np.repeat(a, 300, 0); B = np.repeat(b, 600, 0)
     vals = set()
-    for knobs in (dict(BN=64), dict(BN=128), dict(BN=256), dict(BN=256, BK=128)):
+    for knobs in (dict(BN=64), dict(BN=128), dict(BN=256), dict(BN=256, BK=128), dict(cta_group=2, BN=256), dict(cta_group=2, BN=128)):
         got = gpu_gemm(A, B, out_dtype=rgo.F32, **knobs)
         vals |= set(np.unique(got.view(np.uint32)).tolist())
     vals |= set(np.unique(gpu_gemm(A[:1], B[:5], out_dtype=rgo.F32).view(np.uint32)).tolist())
@@ -152,6 +157,8 @@ def test_batch_invariance_sweep():
         assert_bits_equal(got, ref[:M], f"row bits at M={M}")
         got = gpu_gemm(X[:M], W)                               # tile chosen per M, same class
         assert_bits_equal(got, ref[:M], f"row bits at M={M}, tuned tiles")
+        got = gpu_gemm(X[:M], W, cta_group=2, BN=256)          # a pair of SMs per 256-row tile, same class
+        assert_bits_equal(got, ref[:M], f"row bits at M={M}, two-SM tiles")
     # a permutation of the rows permutes the output rows
     perm = torch.randperm(4096, generator=torch.Generator().manual_seed(0)).to(DEV)
     assert_bits_equal(gpu_gemm(X[perm], W), ref[perm.cpu().numpy()], "row permutation")
@@ -216,8 +223,10 @@ def test_large_square_all_tile_configs_agree_bitwise():
     n = 8192
     A = synth.device_normal((n, n), 1.0, 11, torch.bfloat16, DEV)
     B = synth.device_normal((n, n), 1.0, 12, torch.bfloat16, DEV)
-    configs = [dict(BN=bn, BK=bk, stages=st, raster=ra) for bn in (64, 128, 256) for bk in (64, 128)
+    configs = [dict(cta_group=1, BN=bn, BK=bk, stages=st, raster=ra) for bn in (64, 128, 256) for bk in (64, 128)
                for st in (0, 2) for ra in (0, 1)]
+    configs += [dict(cta_group=2, BN=bn, BK=bk, stages=st, raster=ra) for bn in (128, 256) for bk in (64, 128)
+                for st in (0, 2) for ra in (0, 1, 16)]
     keys = {rg.rg_desc_class(rg.rg_desc(**c)) for c in configs}
     assert len(keys) == 1
     ref = gpu_gemm(A, B, **configs[0])
