@@ -33,10 +33,11 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
     return RG_ERR_UNSUPPORTED;
   if (d->atom != RG_ATOM_TC_BF16_K16 || d->k_tail != 0) return RG_ERR_UNSUPPORTED;
   if (d->BM != 0 && d->BM != 128 && d->BM != 256) return RG_ERR_UNSUPPORTED;
-  if (d->BN != 0 && d->BN != 64 && d->BN != 128 && d->BN != 256) return RG_ERR_UNSUPPORTED;
-  if (d->BK != 0 && d->BK != 64 && d->BK != 128) return RG_ERR_UNSUPPORTED;
+  if (d->BN != 0 && (d->BN % 16 != 0 || d->BN < 16 || d->BN > 256)) return RG_ERR_UNSUPPORTED;
+  if (d->BK != 0 && d->BK != 64 && d->BK != 128 && d->BK != 256) return RG_ERR_UNSUPPORTED;
+
   if (d->cta_group > 2) return RG_ERR_INVALID_DESC;
-  if (d->cta_group == 2 && (d->BM == 128 || d->BN == 64)) return RG_ERR_UNSUPPORTED;   // a pair works on 256 rows, BN >= 128
+  if (d->cta_group == 2 && (d->BM == 128 || (d->BN != 0 && d->BN != 128 && d->BN != 256) || d->BK == 256)) return RG_ERR_UNSUPPORTED;   // a pair works on 256 rows, BN >= 128
   if (d->cta_group == 1 && d->BM == 256) return RG_ERR_UNSUPPORTED;
   if (d->raster > 64) return RG_ERR_INVALID_DESC;
   for (uint32_t i = 0; i < d->n_cuts; ++i)
@@ -82,11 +83,22 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
     plan->part_begin[s] = s == 0 ? 0 : (int32_t)d->cuts[s - 1];
     plan->part_end[s] = s == plan->n_parts - 1 ? (int32_t)K : (int32_t)d->cuts[s];
   }
+  const int sms = device_sms();
+  const int64_t tiles_m = (M + 127) / 128;
+  const bool skinny = M <= 64;     // weight-streaming regime: HBM bound, one partial tile row
   if (d->BN) plan->BN = d->BN;
-  else {
+  else if (skinny) {
+    // Weight streaming: time ~ (rounds of work items per SM) x (tile width).  Any multiple of 16 is a
+    // legal tile width, so pick the one that wastes the least of the last round.
+    int best = 128; int64_t best_cost = -1;
+    for (int bn = 64; bn <= 256; bn += 16) {
+      const int64_t items = ((N + bn - 1) / bn) * plan->n_parts;
+      const int64_t cost = ((items + sms - 1) / sms) * bn;
+      if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
+    }
+    plan->BN = best;
+  } else {
     // largest tile that still gives every SM a work item
-    const int64_t tiles_m = (M + 127) / 128;
-    const int sms = device_sms();
     plan->BN = 64;
     for (int bn : {256, 128}) {
       if (tiles_m * ((N + bn - 1) / bn) * plan->n_parts >= sms) { plan->BN = bn; break; }
@@ -96,11 +108,13 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   if (d->cta_group) plan->cta_group = d->cta_group;
   else if (d->BM == 256) plan->cta_group = 2;
   else if (d->BM == 128) plan->cta_group = 1;
-  else plan->cta_group = (plan->BN >= 128 && M > 128 && ((M + 255) / 256) * ((N + plan->BN - 1) / plan->BN) * plan->n_parts >= device_sms() / 2) ? 2 : 1;
+  else plan->cta_group = (plan->BN >= 128 && M > 128 && ((M + 255) / 256) * ((N + plan->BN - 1) / plan->BN) * plan->n_parts >= sms / 2) ? 2 : 1;
   if (plan->cta_group == 2 && plan->BN < 128) plan->cta_group = 1;
   // a pair moves half the B bytes per CTA, so a 128-wide K step fits three times: fewer hand-offs per k
-  plan->BK = d->BK ? d->BK : (plan->cta_group == 2 && plan->BN == 256 ? 128 : 64);
-  const int smax = rg::max_stages_for(plan->BN, plan->BK, plan->cta_group);
+  // skinny problems read long runs of each weight row per stage (DRAM likes 512-byte bursts)
+  plan->BK = d->BK ? d->BK : ((plan->cta_group == 2 && plan->BN == 256) || skinny ? 128 : 64);
+  if (plan->cta_group == 2 && plan->BN != 128 && plan->BN != 256) return RG_ERR_UNSUPPORTED;
+  const int smax = rg::max_stages_for(plan->BN, plan->BK, plan->cta_group, M);
   plan->stages = d->stages ? d->stages : smax;
   if (plan->stages > smax) return RG_ERR_UNSUPPORTED;
   plan->raster = d->raster == 1 ? 1 : 0;

@@ -108,9 +108,9 @@ __device__ __forceinline__ float apply_epilogue(float v, const EpilogueArgs& e, 
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  const uint32_t l = __bfloat16_as_ushort(__float2bfloat16_rn(lo));
-  const uint32_t h = __bfloat16_as_ushort(__float2bfloat16_rn(hi));
-  return l | (h << 16);
+  // one cvt.rn.bf16x2.f32: each half is rounded to nearest even exactly as a single conversion is
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
 }
 
 }  // namespace rg

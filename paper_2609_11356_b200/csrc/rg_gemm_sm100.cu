@@ -152,6 +152,10 @@ struct GemmParams {
   int32_t M, N, K;
   int32_t tiles_m, tiles_n, n_parts;
   int32_t num_stages, raster, group_m;
+  int32_t bn;             // tile columns of the one-CTA kernel (any multiple of 16 up to 256)
+  uint32_t idesc;         // instruction descriptor for N = bn
+  uint32_t tmem_cols;     // tensor-memory columns allocated: two accumulators of tmem_cols / 2
+  uint32_t a_box_bytes;   // bytes of one A box: 128 B per row actually loaded (rows past M are never fetched)
   void* C;
   int64_t ldc;
   int32_t c_dtype;
@@ -236,17 +240,17 @@ __device__ __forceinline__ void store_row_segment(const GemmParams& p, int64_t r
 // Epilogue of one accumulator tile for one warp: the warp's 32 TMEM lanes (one output row per
 // thread), 32-column chunks chunk0, chunk0+2, ...  Split-K parts go to the workspace at fp32,
 // untouched (Sec. 3.2.2); otherwise bias / SiLU / residual and one rounding to the output type.
-template <int BN>
-__device__ __forceinline__ void epilogue_tile(const GemmParams& p, int part, int64_t row, bool row_ok, int tn,
+__device__ __forceinline__ void epilogue_tile(const GemmParams& p, const int BN, int part, int64_t row, bool row_ok, int tn,
                                               uint32_t taddr, int chunk0) {
+  const int col_end = min(p.N, (tn + 1) * BN);            // this tile's columns end here
 #pragma unroll 1
   for (int c0 = chunk0 * 32; c0 < BN; c0 += 64) {
     const int col0 = tn * BN + c0;
-    if (col0 >= p.N) break;                               // uniform across the warp
+    if (col0 >= col_end) break;                           // uniform across the warp
     uint32_t r[32];
     tmem_ld_32x32b_x32(taddr + c0, r);
     tmem_ld_wait();
-    const int ncols = min(32, p.N - col0);
+    const int ncols = min(32, col_end - col0);
     if (row_ok) {
       if (p.ws) {
         float* dst = p.ws + ((int64_t)part * p.M + row) * p.ldw + col0;
@@ -269,23 +273,31 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, int part, int
   }
 }
 
-// BN: tile columns (UMMA N).  KSUB: 64-wide boxes per pipeline stage (BK = 64 * KSUB).
-template <int BN, int KSUB>
+// KSUB: 64-wide boxes per pipeline stage (BK = 64 * KSUB).  The tile width p.bn is a run-time value:
+// any multiple of 16 up to 256 is a legal step width, which lets the host size tiles so that the
+// work items fill whole waves.
+template <int KSUB>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const GemmParams p) {
-  constexpr uint32_t A_BOX_BYTES = BM * KBOX * 2;
-  constexpr uint32_t B_BOX_BYTES = BN * KBOX * 2;
-  constexpr uint32_t STAGE_BYTES = KSUB * (A_BOX_BYTES + B_BOX_BYTES);
-  constexpr uint32_t TMEM_COLS = (2 * BN <= 32) ? 32 : 2 * BN;   // two accumulators; power of two for BN in {64,128,256}
-  constexpr uint32_t IDESC = make_idesc(BN);
+  // The A box holds only the rows that exist (a multiple of 8, so 1024-byte swizzle groups stay whole);
+  // the tensor-core step still reads 128 rows, and whatever lies past the box only reaches
+  // accumulator rows that are never stored.
+  const uint32_t A_BOX_BYTES = p.a_box_bytes;
+  const int BN = p.bn;
+  const uint32_t B_BOX_BYTES = (uint32_t)BN * KBOX * 2;
+  const uint32_t STAGE_BYTES = KSUB * (A_BOX_BYTES + B_BOX_BYTES);
+  const uint32_t TMEM_COLS = p.tmem_cols;                // a power of two >= 32; accumulator b starts at column b * TMEM_COLS / 2
+  const uint32_t ACC_STRIDE = TMEM_COLS >> 1;
+  const uint32_t IDESC = p.idesc;
 
   extern __shared__ uint8_t smem_raw[];
   // the swizzle pattern is a function of the absolute address: tiles sit on 1024-byte boundaries
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const int S = p.num_stages;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + (size_t)S * STAGE_BYTES);
+  // barriers sit behind the ring and behind the span a short A box leaves readable (see smem_bytes_for)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + (size_t)S * STAGE_BYTES + (BM * KBOX * 2 - A_BOX_BYTES));
   // layout: full[S], empty[S], tmem_full[2], tmem_empty[2], then tmem base slot and abort flag
   const uint32_t bar_full = smem_u32(bars);
   const uint32_t bar_empty = bar_full + 8u * S;
@@ -311,6 +323,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // a split-K merge launched behind this kernel may be scheduled now; it still waits for this grid to finish
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -349,7 +363,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         const uint32_t acc_phase = (it >> 1) & 1;
         if (!mbar_wait(bar_tempty + 8u * buf, acc_phase ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
         tcgen05_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * BN;
+        const uint32_t d_tmem = tmem_base + buf * ACC_STRIDE;
         uint32_t accumulate = 0;                        // every part starts from a zero accumulator
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
           if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0x300u | stage)) { alive = false; break; }
@@ -389,8 +403,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       tcgen05_fence_after();
       const int64_t row = (int64_t)tm * BM + quarter * 32 + lane;
       const bool row_ok = row < p.M;
-      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
-      epilogue_tile<BN>(p, part, row, row_ok, tn, taddr, chunk0);
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
+      epilogue_tile(p, BN, part, row, row_ok, tn, taddr, chunk0);
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
@@ -463,6 +477,8 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   cluster_sync_all();                                      // both CTAs' barriers exist before any remote arrive
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // a split-K merge launched behind this kernel may be scheduled now; it still waits for this grid to finish
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -543,7 +559,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       tcgen05_fence_after();
       const int64_t row = (int64_t)tm * 2 * BM + (int64_t)rank * BM + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
-      epilogue_tile<BN>(p, part, row, row < p.M, tn, taddr, chunk0);
+      epilogue_tile(p, BN, part, row, row < p.M, tn, taddr, chunk0);
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(tempty_leader + 8u * buf);
@@ -581,6 +597,9 @@ struct FixupParams {
 __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) {
   const int64_t ncol4 = (p.N + 3) / 4;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  // launched with programmatic stream serialisation: the grid may start while the GEMM kernel is
+  // still draining; nothing is read before that kernel has completed and flushed its stores
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (idx >= (int64_t)p.M * ncol4) return;
   const int64_t row = idx / ncol4;
   const int col0 = (int)(idx - row * ncol4) * 4;
@@ -661,9 +680,12 @@ bool make_tmap(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, in
 
 constexpr size_t SMEM_LIMIT = 232448;   // 227 KiB of dynamic shared memory per CTA
 
-size_t smem_bytes_for(int bn, int ksub, int stages) {
-  const size_t stage = (size_t)ksub * (BM * KBOX * 2 + (size_t)bn * KBOX * 2);
-  return 1024 + stages * stage + (2 * stages + 4) * 8 + 16;
+size_t smem_bytes_for(int bn, int ksub, int stages, int a_rows) {
+  const size_t stage = (size_t)ksub * ((size_t)a_rows * KBOX * 2 + (size_t)bn * KBOX * 2);
+  // The tensor-core step reads 128 rows from the start of an A box even when the box holds fewer:
+  // keep that whole span inside the allocation (the extra rows feed accumulator rows nobody stores).
+  const size_t slack = (size_t)(BM - a_rows) * KBOX * 2;
+  return 1024 + stages * stage + slack + (2 * stages + 4) * 8 + 16;
 }
 
 size_t smem_bytes_for_pair(int bn, int ksub, int stages) {
@@ -693,26 +715,28 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const Gemm
   return cudaLaunchKernelEx(&cfg, gemm_tcgen05_pair_kernel<BN, KSUB>, ta, tb, p);
 }
 
-template <int BN, int KSUB>
+template <int KSUB>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
-  const size_t smem = smem_bytes_for(BN, KSUB, p.num_stages);
+  const size_t smem = smem_bytes_for(p.bn, KSUB, p.num_stages, (int)(p.a_box_bytes / (KBOX * 2)));
   static size_t configured = 0;
   if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, KSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<KSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
     if (e != cudaSuccess) return e;
     configured = SMEM_LIMIT;
   }
-  gemm_tcgen05_kernel<BN, KSUB><<<grid, NUM_THREADS, smem, st>>>(ta, tb, p);
+  gemm_tcgen05_kernel<KSUB><<<grid, NUM_THREADS, smem, st>>>(ta, tb, p);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-int max_stages_for(int bn, int bk, int cta_group) {
+int a_box_rows_for(int64_t M) { return M >= BM ? BM : (int)((M + 7) / 8 * 8); }
+
+int max_stages_for(int bn, int bk, int cta_group, int64_t M) {
   const int ksub = bk / KBOX;
   int s = 1;
   if (cta_group == 2) { while (s < 8 && smem_bytes_for_pair(bn, ksub, s + 1) <= SMEM_LIMIT) ++s; }
-  else { while (s < 8 && smem_bytes_for(bn, ksub, s + 1) <= SMEM_LIMIT) ++s; }
+  else { while (s < 8 && smem_bytes_for(bn, ksub, s + 1, a_box_rows_for(M)) <= SMEM_LIMIT) ++s; }
   return s;
 }
 
@@ -732,7 +756,8 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   const bool pair = plan.cta_group == 2;
   const int tile_m = pair ? 2 * BM : BM;
   CUtensorMap ta, tb;
-  if (!make_tmap(&ta, A->ptr, M, K, A->ld, BM) || !make_tmap(&tb, B->ptr, N, K, B->ld, pair ? plan.BN / 2 : plan.BN))
+  const int a_rows = pair ? BM : a_box_rows_for(M);
+  if (!make_tmap(&ta, A->ptr, M, K, A->ld, a_rows) || !make_tmap(&tb, B->ptr, N, K, B->ld, pair ? plan.BN / 2 : plan.BN))
     return RG_ERR_CUDA;
 
   GemmParams p;
@@ -743,6 +768,10 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   p.num_stages = plan.stages;
   p.raster = plan.raster;
   p.group_m = plan.group_m;
+  p.a_box_bytes = (uint32_t)a_rows * KBOX * 2;
+  p.bn = plan.BN;
+  p.idesc = make_idesc(plan.BN);
+  { uint32_t c = 32; while (c < 2u * (uint32_t)((plan.BN + 31) / 32 * 32)) c <<= 1; p.tmem_cols = c; }
   for (int s = 0; s < plan.n_parts; ++s) { p.part_begin[s] = plan.part_begin[s]; p.part_end[s] = plan.part_end[s]; }
   EpilogueArgs e{};
   if (epi) {
@@ -771,12 +800,9 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     else return RG_ERR_UNSUPPORTED;
   } else {
     const int grid = (int)(total < sms ? total : sms);
-    if (plan.BN == 256 && ksub == 1) err = launch_one<256, 1>(ta, tb, p, grid, st);
-    else if (plan.BN == 256 && ksub == 2) err = launch_one<256, 2>(ta, tb, p, grid, st);
-    else if (plan.BN == 128 && ksub == 1) err = launch_one<128, 1>(ta, tb, p, grid, st);
-    else if (plan.BN == 128 && ksub == 2) err = launch_one<128, 2>(ta, tb, p, grid, st);
-    else if (plan.BN == 64 && ksub == 1) err = launch_one<64, 1>(ta, tb, p, grid, st);
-    else if (plan.BN == 64 && ksub == 2) err = launch_one<64, 2>(ta, tb, p, grid, st);
+    if (ksub == 1) err = launch_one<1>(ta, tb, p, grid, st);
+    else if (ksub == 2) err = launch_one<2>(ta, tb, p, grid, st);
+    else if (ksub == 4) err = launch_one<4>(ta, tb, p, grid, st);
     else return RG_ERR_UNSUPPORTED;
   }
   if (err != cudaSuccess) return RG_ERR_CUDA;
@@ -787,8 +813,17 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     f.M = p.M; f.N = p.N; f.S = plan.n_parts; f.tree = plan.tree;
     f.C = C->ptr; f.ldc = C->ld; f.c_dtype = C->dtype; f.epi = e;
     const int64_t items = M * ((N + 3) / 4);
-    splitk_fixup_kernel<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(f);
-    if (cudaGetLastError() != cudaSuccess) return RG_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((items + 255) / 256), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, splitk_fixup_kernel, f) != cudaSuccess) return RG_ERR_CUDA;
   }
   return RG_OK;
 }

@@ -98,6 +98,7 @@ __device__ __forceinline__ float fold_block(const float (&x)[V], int nvalid, flo
       if (fma) n[t] = ok1 ? f_fma(x1, x1, s0) : s0;      // second square fused into the add
       else n[t] = f_add(s0, ok1 ? f_mul(x1, x1) : NEG_ZERO);
     } else {
+      // scalar on purpose: the packed f32x2 form measured slower here (the fp32 pipe, not issue, is the limit)
       const float e0 = ok0 ? exp_nonpositive(f_add(x0, -shift)) : NEG_ZERO;
       const float e1 = ok1 ? exp_nonpositive(f_add(x1, -shift)) : NEG_ZERO;
       n[t] = f_add(e0, e1);
@@ -401,7 +402,10 @@ __global__ void __launch_bounds__(256) rmsnorm_keep_kernel(const ReduceParams p)
         for (int t = 0; t < V; ++t) w[t] = p.weight ? load_scalar(p.weight, p.w_dtype, c + t) : 1.0f;
       }
 #pragma unroll
-      for (int t = 0; t < V; ++t) y[t] = f_mul(f_mul(x[t], rinv), w[t]);
+      for (int t = 0; t < V; t += 2) {
+        const float2 q = __fmul2_rn(__fmul2_rn(make_float2(x[t], x[t + 1]), make_float2(rinv, rinv)), make_float2(w[t], w[t + 1]));
+        y[t] = q.x; y[t + 1] = q.y;
+      }
       if (out_vec) {
         if constexpr (sizeof(T) == 4)
           *reinterpret_cast<uint4*>(static_cast<float*>(p.out) + row * p.ldo + c) =

@@ -37,7 +37,9 @@ def test_validate_rules():
     assert rg.rg_desc_validate(rg.rg_desc(cuts=(40,)), 64, 256, 512) == 3           # splits a 16-wide step
     assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_SCALAR), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16), 64, 256, 512) == 3
-    assert rg.rg_desc_validate(rg.rg_desc(BN=96), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(BN=100), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(BN=112, BK=256), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(BN=112, cta_group=2), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(cta_group=2), 64, 256, 512) == 0
     assert rg.rg_desc_validate(rg.rg_desc(cta_group=3), 64, 256, 512) == 2
     assert rg.rg_desc_validate(rg.rg_desc(cta_group=2, BN=64), 64, 256, 512) == 3

@@ -42,7 +42,8 @@ def test_tiny_descriptor_check_full_oracle_compare():
 @pytest.mark.parametrize("M,N,K", [(1, 1, 16), (1, 8, 8), (3, 5, 24), (128, 64, 64), (129, 65, 80), (300, 520, 1000),
                                    (7, 4096, 1024), (2000, 3000, 2048), (64, 100, 72)])
 @pytest.mark.parametrize("knobs", [dict(), dict(BN=64), dict(BN=128, BK=128), dict(BN=256, stages=2, raster=1),
-                                   dict(cta_group=1, BN=256), dict(cta_group=2, BN=256, BK=64), dict(BM=256, BN=128, BK=128, raster=4)])
+                                   dict(cta_group=1, BN=256), dict(cta_group=2, BN=256, BK=64), dict(BM=256, BN=128, BK=128, raster=4),
+                                   dict(BN=112, BK=128), dict(BN=48, BK=256, cta_group=1), dict(BN=240, cta_group=1), dict(BN=16, cta_group=1)])
 def test_integer_inputs_exact(M, N, K, knobs):
     A = synth.int_valued_bf16((M, K), -8, 8, K + M); B = synth.int_valued_bf16((N, K), -8, 8, K + N + 1)
     assert_bits_equal(gpu_gemm(A, B, out_dtype=rgo.F32, **knobs), _exact_int(A, B), f"ints {M}x{N}x{K} {knobs}")
@@ -120,7 +121,8 @@ def test_position_independence_of_one_k_vector():
     b = synth.spread_exponents_bf16(synth.normal_bf16((1, K), 1.0, 72), 73, -8, 8)
     A = np.repeat(a, 300, 0); B = np.repeat(b, 600, 0)
     vals = set()
-    for knobs in (dict(BN=64), dict(BN=128), dict(BN=256), dict(BN=256, BK=128), dict(cta_group=2, BN=256), dict(cta_group=2, BN=128)):
+    for knobs in (dict(BN=64), dict(BN=128), dict(BN=256), dict(BN=256, BK=128), dict(cta_group=2, BN=256), dict(cta_group=2, BN=128),
+                  dict(cta_group=1, BN=112, BK=256), dict(cta_group=1, BN=208)):
         got = gpu_gemm(A, B, out_dtype=rgo.F32, **knobs)
         vals |= set(np.unique(got.view(np.uint32)).tolist())
     vals |= set(np.unique(gpu_gemm(A[:1], B[:5], out_dtype=rgo.F32).view(np.uint32)).tolist())
@@ -187,6 +189,8 @@ def test_decode_split_k_with_residual(M):
         assert_bits_equal(synth.bf16_bits_to_f32(got[si, sj]), want, "config 3 M=32 sampled")
     full = gpu_gemm(synth.normal_bf16((32, K), 1.0, 4), W, cuts=cuts, residual=synth.normal_bf16((32, N), 1.0, 5))
     assert_bits_equal(got, full[:M], "rows do not depend on M")
+    for knobs in (dict(BN=128, BK=64), dict(BN=64, BK=256), dict(BN=32, BK=128), dict(BN=256, BK=128)):
+        assert_bits_equal(gpu_gemm(X, W, cuts=cuts, residual=res, **knobs), got, f"tile knobs {knobs}")
 
 
 # ------------------------------------------------------------------ config 4: fused epilogue
@@ -227,6 +231,7 @@ def test_large_square_all_tile_configs_agree_bitwise():
                for st in (0, 2) for ra in (0, 1)]
     configs += [dict(cta_group=2, BN=bn, BK=bk, stages=st, raster=ra) for bn in (128, 256) for bk in (64, 128)
                 for st in (0, 2) for ra in (0, 1, 16)]
+    configs += [dict(cta_group=1, BN=bn, BK=bk) for bn in (112, 176, 240) for bk in (64, 256)]
     keys = {rg.rg_desc_class(rg.rg_desc(**c)) for c in configs}
     assert len(keys) == 1
     ref = gpu_gemm(A, B, **configs[0])
