@@ -8,7 +8,7 @@
 // loads and which issues, the persistent tile walk, the double-buffered accumulator.
 //
 // CTA roles (320 threads):
-//   warp 0, lane 0   TMA producer: A[BM x 64] and B[BN x 64] boxes (128-byte swizzle) per stage
+//   warp 0           TMA producer: A[BM x 64] and B[BN x 64] boxes (128-byte swizzle), one lane per box
 //   warp 1, lane 0   MMA issuer: 4 steps of K=16 per 64-wide box, ascending; tcgen05.commit
 //                    frees the stage; a final commit publishes the accumulator
 //   warps 2..9       epilogue: tcgen05.ld of their 32 TMEM lanes (warp % 4 picks the lane
@@ -328,23 +328,25 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // 2*KSUB lanes, one box each (lane < KSUB: A sub-box `lane`; otherwise B sub-box lane - KSUB):
+    // the lanes run converged, so one instruction issue starts all of a stage's copies.
+    if (lane < 2 * KSUB) {
+      const bool is_b = lane >= KSUB;
+      const int sub = is_b ? lane - KSUB : lane;
+      const CUtensorMap* map = is_b ? &tmap_b : &tmap_a;
+      const uint32_t box_off = is_b ? KSUB * A_BOX_BYTES + sub * B_BOX_BYTES : sub * A_BOX_BYTES;
       int stage = 0; uint32_t phase = 0;
       bool alive = true;
       for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);
         const int k_begin = p.part_begin[part], k_end = p.part_end[part];
+        const int y = is_b ? tn * BN : tm * BM;
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
           if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, &g_status_word, 0x100u | stage)) { alive = false; break; }
           const uint32_t full = bar_full + 8u * stage;
-          mbar_expect_tx(full, STAGE_BYTES);
-          const uint32_t sa = smem_base + stage * STAGE_BYTES;
-#pragma unroll
-          for (int sub = 0; sub < KSUB; ++sub) {
-            tma_load_2d(sa + sub * A_BOX_BYTES, &tmap_a, k0 + sub * KBOX, tm * BM, full);
-            tma_load_2d(sa + KSUB * A_BOX_BYTES + sub * B_BOX_BYTES, &tmap_b, k0 + sub * KBOX, tn * BN, full);
-          }
+          if (lane == 0) mbar_expect_tx(full, STAGE_BYTES);
+          tma_load_2d(smem_base + stage * STAGE_BYTES + box_off, map, k0 + sub * KBOX, y, full);
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
       }
@@ -482,25 +484,25 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (both CTAs)
-    if (lane == 0) {
+    // 2*KSUB lanes, one box each, converged: one instruction issue starts all of a stage's copies.
+    if (lane < 2 * KSUB) {
+      const bool is_b = lane >= KSUB;
+      const int sub = is_b ? lane - KSUB : lane;
+      const CUtensorMap* map = is_b ? &tmap_b : &tmap_a;
+      const uint32_t box_off = is_b ? KSUB * A_BOX_BYTES + sub * B_BOX_BYTES : sub * A_BOX_BYTES;
       int stage = 0; uint32_t phase = 0;
       bool alive = true;
       for (int w = pair_id; w < total_work && alive; w += num_pairs) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);
         const int k_begin = p.part_begin[part], k_end = p.part_end[part];
+        const int y = is_b ? tn * BN + (int)rank * (BN / 2) : tm * 2 * BM + (int)rank * BM;
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
           if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, &g_status_word, 0x900u | stage)) { alive = false; break; }
           const uint32_t full_local = bar_full + 8u * stage;
-          if (rank == 0) mbar_expect_tx(full_local, 2u * STAGE_BYTES);      // bytes of both CTAs
+          if (lane == 0 && rank == 0) mbar_expect_tx(full_local, 2u * STAGE_BYTES);      // bytes of both CTAs
           const uint32_t full = map_to_cta(full_local, 0);
-          const uint32_t sa = smem_base + stage * STAGE_BYTES;
-#pragma unroll
-          for (int sub = 0; sub < KSUB; ++sub) {
-            tma_load_2d_pair(sa + sub * A_BOX_BYTES, &tmap_a, k0 + sub * KBOX, tm * 2 * BM + (int)rank * BM, full);
-            tma_load_2d_pair(sa + KSUB * A_BOX_BYTES + sub * B_BOX_BYTES, &tmap_b, k0 + sub * KBOX,
-                             tn * BN + (int)rank * (BN / 2), full);
-          }
+          tma_load_2d_pair(smem_base + stage * STAGE_BYTES + box_off, map, k0 + sub * KBOX, y, full);
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
       }
