@@ -70,8 +70,8 @@ typedef struct {
   /* ---- order-deciding fields: these ARE the class key ---- */
   uint8_t in_dtype;       /* rg_dtype_t of A and B: RG_BF16 */
   uint8_t acc_dtype;      /* accumulator: RG_F32 */
-  uint8_t partial_dtype;  /* type a finished split-K part is written at: RG_F32 (Sec. 3.2.2) */
-  uint8_t merge_dtype;    /* type the parts are summed at: RG_F32 */
+  uint8_t partial_dtype;  /* type a finished split-K part is written at: RG_F32 or RG_BF16 (Sec. 3.2.2) */
+  uint8_t merge_dtype;    /* type the running sum of the parts is kept at: RG_F32, or RG_BF16 with bf16 parts */
   uint8_t atom;           /* rg_atom_t */
   uint8_t k_tail;         /* 0 = the short K turn runs last, missing products are absent */
   uint8_t fma;            /* multiply-add fusion on scalar leaves (reductions: x*x feeding an add) */
@@ -123,7 +123,7 @@ rg_status_t rg_desc_validate(const rg_desc_t* d, int64_t M, int64_t N, int64_t K
  * the epilogue are excluded.  Returns 0 for a malformed descriptor.  Host only. */
 uint64_t rg_desc_class(const rg_desc_t* d);
 
-/* Bytes of fp32 workspace rg_gemm needs: 0 without cuts, else (n_cuts+1) * M * roundup(N,4) * 4. */
+/* Bytes of workspace rg_gemm needs: 0 without cuts, else (n_cuts+1) * M * roundup(N,4) * sizeof(partial_dtype). */
 size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N);
 
 /* C[M,N] = epilogue( merge_s( sum_{k in part s} A[i,k] * B[j,k] ) )   (C = A * B^T).
@@ -132,8 +132,8 @@ size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N);
  * per output element and per part, the accumulator starts at zero and takes one tensor-core
  * step per 16 consecutive k, in ascending k; a finished part is an fp32 value; the parts are
  * added in the descriptor's tree; then the epilogue.  Without cuts one kernel does everything;
- * with cuts the parts go to `ws` as fp32 [part][M][roundup(N,4)] and a second kernel merges
- * them (no atomics anywhere).
+ * with cuts the parts go to `ws` as [part][M][roundup(N,4)] at partial_dtype and a second kernel
+ * merges them, the running sum kept at merge_dtype (no atomics anywhere).
  *
  *   A: [M,K] bf16, B: [N,K] bf16 (both K-contiguous), C: [M,N] bf16 or fp32.
  *   A.ptr, B.ptr 16-byte aligned; A.ld, B.ld multiples of 8.  C, bias, residual: any alignment.

@@ -95,6 +95,30 @@ float tree_reduce(std::vector<float>& v, int tree) {
   return v[0];
 }
 
+// The same trees with the running sum kept at `merge_dtype` (Sec. 3.2.2, split-K: "a finished part
+// is written at one type and the running sum kept at another"): every add is an fp32 add whose
+// result is then rounded to the merge type (for bf16 operands this equals the correctly rounded
+// bf16 sum: the fp32 add is exact or its error lies far below half a bf16 ulp).
+inline float round_to(float v, int dtype) { return dtype == DT_BF16 ? bf16_to_f32(f32_to_bf16(v)) : v; }
+
+float tree_reduce_at(std::vector<float>& v, int tree, int merge_dtype) {
+  if (merge_dtype == DT_F32) return tree_reduce(v, tree);
+  size_t n = v.size();
+  if (n == 0) return 0.0f;
+  if (tree == TREE_LEFT) {
+    float acc = v[0];
+    for (size_t t = 1; t < n; ++t) acc = round_to(acc + v[t], merge_dtype);
+    return acc;
+  }
+  while (n > 1) {
+    size_t m = 0;
+    for (size_t t = 0; 2 * t + 1 < n; ++t) v[m++] = round_to(v[2 * t] + v[2 * t + 1], merge_dtype);
+    if (n & 1) v[m++] = v[n - 1];
+    n = m;
+  }
+  return v[0];
+}
+
 // --------------------------------------------------- exact long accumulator
 // Fixed-point accumulator wide enough for any sum of bf16*bf16 products and
 // binary32 values: bit i of the accumulator has weight 2^(i - BIAS).
@@ -355,6 +379,8 @@ struct GemmDesc {
   int32_t act;             // 0 none, 1 SiLU
   const void* residual; int32_t residual_dtype; int64_t ldr;
   int32_t out_dtype;
+  int32_t partial_dtype;   // type a finished part is written at (fp32 or bf16)
+  int32_t merge_dtype;     // type the running sum of the parts is kept at
 };
 
 // One output element, Sec. 3.2.2.  `partials_out` (nullable) receives the
@@ -372,10 +398,10 @@ float gemm_element(const GemmDesc& d, const uint16_t* arow, const uint16_t* brow
       int n = int(std::min<int64_t>(ak, k_hi - k0));
       acc = atom_step(acc, arow + k0, brow + k0, n, d.atom);
     }
-    part[s] = acc;                                      // fp32 partial, no rounding
-    if (partials_out) partials_out[s] = acc;
+    part[s] = round_to(acc, d.partial_dtype);           // the finished part, at partial_dtype
+    if (partials_out) partials_out[s] = part[s];
   }
-  float v = tree_reduce(part, d.tree);                  // merge: fp32 adds in tree order
+  float v = tree_reduce_at(part, d.tree, d.merge_dtype);  // merge in tree order, sum kept at merge_dtype
   if (d.bias) v = v + load_elem(d.bias, d.bias_dtype, j);
   if (d.act == 1) v = silu(v);
   if (d.residual) v = v + load_elem(d.residual, d.residual_dtype, i * d.ldr + j);
@@ -420,8 +446,8 @@ void rgo_gemm(const AtomModel* atom, int tree, int n_cuts, const int64_t* cuts,
               const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
               void* C, int out_dtype, int64_t ldc,
               const void* bias, int bias_dtype, int act,
-              const void* residual, int residual_dtype, int64_t ldr) {
-  GemmDesc d{*atom, tree, n_cuts, cuts, bias, bias_dtype, act, residual, residual_dtype, ldr, out_dtype};
+              const void* residual, int residual_dtype, int64_t ldr, int partial_dtype, int merge_dtype) {
+  GemmDesc d{*atom, tree, n_cuts, cuts, bias, bias_dtype, act, residual, residual_dtype, ldr, out_dtype, partial_dtype, merge_dtype};
 #pragma omp parallel for collapse(2) schedule(static)
   for (int64_t i = 0; i < M; ++i)
     for (int64_t j = 0; j < N; ++j) {
@@ -437,8 +463,9 @@ void rgo_gemm_samples(const AtomModel* atom, int tree, int n_cuts, const int64_t
                       int out_dtype,
                       const void* bias, int bias_dtype, int act,
                       const void* residual, int residual_dtype, int64_t ldr,
-                      int64_t n_samples, const int64_t* si, const int64_t* sj, float* out) {
-  GemmDesc d{*atom, tree, n_cuts, cuts, bias, bias_dtype, act, residual, residual_dtype, ldr, out_dtype};
+                      int64_t n_samples, const int64_t* si, const int64_t* sj, float* out,
+                      int partial_dtype, int merge_dtype) {
+  GemmDesc d{*atom, tree, n_cuts, cuts, bias, bias_dtype, act, residual, residual_dtype, ldr, out_dtype, partial_dtype, merge_dtype};
 #pragma omp parallel for schedule(static)
   for (int64_t t = 0; t < n_samples; ++t) {
     float v = gemm_element(d, A + si[t] * lda, B + sj[t] * ldb, K, si[t], sj[t], nullptr);
@@ -446,11 +473,11 @@ void rgo_gemm_samples(const AtomModel* atom, int tree, int n_cuts, const int64_t
   }
 }
 
-// fp32 partials of every part, [S][M][N], before the merge.
+// Partials of every part, [S][M][N], before the merge (fp32 holding the value at partial_dtype).
 void rgo_gemm_partials(const AtomModel* atom, int n_cuts, const int64_t* cuts,
                        int64_t M, int64_t N, int64_t K,
-                       const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb, float* P) {
-  GemmDesc d{*atom, TREE_LEFT, n_cuts, cuts, nullptr, 0, 0, nullptr, 0, 0, DT_F32};
+                       const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb, float* P, int partial_dtype) {
+  GemmDesc d{*atom, TREE_LEFT, n_cuts, cuts, nullptr, 0, 0, nullptr, 0, 0, DT_F32, partial_dtype, DT_F32};
   int S = n_cuts + 1;
 #pragma omp parallel for collapse(2) schedule(static)
   for (int64_t i = 0; i < M; ++i)

@@ -29,8 +29,9 @@ rg_status_t check_desc_fields(const rg_desc_t* d) {
 
 // What the kernels of this library can honour.
 rg_status_t check_desc_supported(const rg_desc_t* d) {
-  if (d->in_dtype != RG_BF16 || d->acc_dtype != RG_F32 || d->partial_dtype != RG_F32 || d->merge_dtype != RG_F32)
-    return RG_ERR_UNSUPPORTED;
+  if (d->in_dtype != RG_BF16 || d->acc_dtype != RG_F32) return RG_ERR_UNSUPPORTED;
+  // parts at fp32 summed at fp32, parts at bf16 summed at fp32, or both at bf16 (Sec. 3.2.2)
+  if (d->partial_dtype == RG_F32 && d->merge_dtype != RG_F32) return RG_ERR_UNSUPPORTED;
   if (d->atom != RG_ATOM_TC_BF16_K16 || d->k_tail != 0) return RG_ERR_UNSUPPORTED;
   if (d->BM != 0 && d->BM != 128 && d->BM != 256) return RG_ERR_UNSUPPORTED;
   if (d->BN != 0 && (d->BN % 16 != 0 || d->BN < 16 || d->BN > 256)) return RG_ERR_UNSUPPORTED;
@@ -79,6 +80,8 @@ int device_sms() {
 rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::GemmPlan* plan) {
   plan->n_parts = (int)d->n_cuts + 1;
   plan->tree = d->tree;
+  plan->partial_dtype = d->partial_dtype;
+  plan->merge_dtype = d->merge_dtype;
   for (int s = 0; s < plan->n_parts; ++s) {
     plan->part_begin[s] = s == 0 ? 0 : (int32_t)d->cuts[s - 1];
     plan->part_end[s] = s == plan->n_parts - 1 ? (int32_t)K : (int32_t)d->cuts[s];
@@ -160,7 +163,7 @@ uint64_t rg_desc_class(const rg_desc_t* d) {
 
 size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N) {
   if (!d || d->n_cuts == 0 || d->n_cuts > RG_MAX_CUTS || M <= 0 || N <= 0) return 0;
-  return (size_t)(d->n_cuts + 1) * (size_t)M * (size_t)((N + 3) / 4 * 4) * sizeof(float);
+  return (size_t)(d->n_cuts + 1) * (size_t)M * (size_t)((N + 3) / 4 * 4) * (d->partial_dtype == RG_BF16 ? 2 : 4);
 }
 
 rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,

@@ -159,8 +159,9 @@ struct GemmParams {
   void* C;
   int64_t ldc;
   int32_t c_dtype;
-  float* ws;            // split-K partials [part][M][ldw], fp32; null without cuts
+  void* ws;             // split-K partials [part][M][ldw] at ws_dtype; null without cuts
   int64_t ldw;
+  int32_t ws_dtype;
   EpilogueArgs epi;
   int32_t part_begin[RG_MAX_CUTS + 1];
   int32_t part_end[RG_MAX_CUTS + 1];
@@ -252,8 +253,8 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, const int BN,
     tmem_ld_wait();
     const int ncols = min(32, col_end - col0);
     if (row_ok) {
-      if (p.ws) {
-        float* dst = p.ws + ((int64_t)part * p.M + row) * p.ldw + col0;
+      if (p.ws && p.ws_dtype == RG_F32) {
+        float* dst = static_cast<float*>(p.ws) + ((int64_t)part * p.M + row) * p.ldw + col0;
         if (ncols == 32) {
 #pragma unroll
           for (int q = 0; q < 8; ++q)
@@ -261,6 +262,21 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, const int BN,
         } else {
 #pragma unroll
           for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __uint_as_float(r[c]);
+        }
+      } else if (p.ws) {
+        // the finished part written at bf16: one rounding of the fp32 accumulator
+        __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.ws) + ((int64_t)part * p.M + row) * p.ldw + col0;
+        if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            reinterpret_cast<uint4*>(dst)[q] = make_uint4(
+                pack_bf16x2(__uint_as_float(r[8 * q]), __uint_as_float(r[8 * q + 1])),
+                pack_bf16x2(__uint_as_float(r[8 * q + 2]), __uint_as_float(r[8 * q + 3])),
+                pack_bf16x2(__uint_as_float(r[8 * q + 4]), __uint_as_float(r[8 * q + 5])),
+                pack_bf16x2(__uint_as_float(r[8 * q + 6]), __uint_as_float(r[8 * q + 7])));
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __float2bfloat16_rn(__uint_as_float(r[c]));
         }
       } else {
         float v[32];
@@ -584,18 +600,21 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 
 // -------------------------------------------------------------- split-K merge
 struct FixupParams {
-  const float* ws;
+  const void* ws;
   int64_t ldw;
   int32_t M, N, S, tree;
+  int32_t partial_dtype, merge_dtype;
   void* C;
   int64_t ldc;
   int32_t c_dtype;
   EpilogueArgs epi;
 };
 
-// One thread per (row, 4 consecutive columns).  The parts are combined in the descriptor's
-// tree with plain fp32 adds; BALANCED is evaluated with a binary-counter stack, which visits
+// One thread per (row, 4 consecutive columns).  The parts are combined in the descriptor's tree
+// with fp32 adds, the running sum kept at merge_dtype (an add whose result is rounded to bf16 when
+// the sum is kept at bf16); BALANCED is evaluated with a binary-counter stack, which visits
 // exactly the aligned pairs of the level-by-level definition.
+template <bool PART_BF16, bool MERGE_BF16>
 __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) {
   const int64_t ncol4 = (p.N + 3) / 4;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -605,24 +624,33 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
   if (idx >= (int64_t)p.M * ncol4) return;
   const int64_t row = idx / ncol4;
   const int col0 = (int)(idx - row * ncol4) * 4;
-  const float* src = p.ws + row * p.ldw + col0;
   const int64_t part_stride = (int64_t)p.M * p.ldw;
+  const int64_t off = row * p.ldw + col0;
+  auto load = [&](int s) -> float4 {
+    if (PART_BF16) {
+      const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.ws) + s * part_stride + off);
+      return make_float4(bf16_bits_to_f32(w.x & 0xffffu), bf16_bits_to_f32(w.x >> 16),
+                         bf16_bits_to_f32(w.y & 0xffffu), bf16_bits_to_f32(w.y >> 16));
+    }
+    return *reinterpret_cast<const float4*>(static_cast<const float*>(p.ws) + s * part_stride + off);
+  };
+  auto add1 = [](float a, float b) -> float {
+    const float v = f_add(a, b);
+    return MERGE_BF16 ? __bfloat162float(__float2bfloat16_rn(v)) : v;
+  };
+  auto add4 = [&](const float4& a, const float4& b) -> float4 {
+    return make_float4(add1(a.x, b.x), add1(a.y, b.y), add1(a.z, b.z), add1(a.w, b.w));
+  };
   float4 acc;
   if (p.tree == RG_TREE_LEFT) {
-    acc = *reinterpret_cast<const float4*>(src);
-    for (int s = 1; s < p.S; ++s) {
-      const float4 v = *reinterpret_cast<const float4*>(src + s * part_stride);
-      acc.x = f_add(acc.x, v.x); acc.y = f_add(acc.y, v.y); acc.z = f_add(acc.z, v.z); acc.w = f_add(acc.w, v.w);
-    }
+    acc = load(0);
+    for (int s = 1; s < p.S; ++s) acc = add4(acc, load(s));
   } else {
     float4 stack[7];
     for (int s = 0; s < p.S; ++s) {
-      float4 v = *reinterpret_cast<const float4*>(src + s * part_stride);
+      float4 v = load(s);
       int b = 0;
-      for (; (s >> b) & 1; ++b) {
-        const float4 l = stack[b];
-        v.x = f_add(l.x, v.x); v.y = f_add(l.y, v.y); v.z = f_add(l.z, v.z); v.w = f_add(l.w, v.w);
-      }
+      for (; (s >> b) & 1; ++b) v = add4(stack[b], v);
       stack[b] = v;
     }
     // leftovers: the lowest pending level moves up unchanged until it meets a sibling
@@ -630,10 +658,7 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
     for (int b = 0; b < 7; ++b) {
       if (!((p.S >> b) & 1)) continue;
       if (!have) { acc = stack[b]; have = true; }
-      else {
-        const float4 l = stack[b];
-        acc.x = f_add(l.x, acc.x); acc.y = f_add(l.y, acc.y); acc.z = f_add(l.z, acc.z); acc.w = f_add(l.w, acc.w);
-      }
+      else acc = add4(stack[b], acc);
     }
   }
   float v[4] = {acc.x, acc.y, acc.z, acc.w};
@@ -782,7 +807,8 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   }
   const bool split = plan.n_parts > 1;
   p.C = C->ptr; p.ldc = C->ld; p.c_dtype = C->dtype;
-  p.ws = split ? static_cast<float*>(ws) : nullptr;
+  p.ws = split ? ws : nullptr;
+  p.ws_dtype = plan.partial_dtype;
   p.ldw = (N + 3) / 4 * 4;
   p.epi = split ? EpilogueArgs{} : e;
 
@@ -811,7 +837,7 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
 
   if (split) {
     FixupParams f;
-    f.ws = static_cast<const float*>(ws); f.ldw = p.ldw;
+    f.ws = ws; f.ldw = p.ldw; f.partial_dtype = plan.partial_dtype; f.merge_dtype = plan.merge_dtype;
     f.M = p.M; f.N = p.N; f.S = plan.n_parts; f.tree = plan.tree;
     f.C = C->ptr; f.ldc = C->ld; f.c_dtype = C->dtype; f.epi = e;
     const int64_t items = M * ((N + 3) / 4);
@@ -825,7 +851,11 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, splitk_fixup_kernel, f) != cudaSuccess) return RG_ERR_CUDA;
+    cudaError_t fe;
+    if (plan.partial_dtype == RG_F32) fe = cudaLaunchKernelEx(&cfg, splitk_fixup_kernel<false, false>, f);
+    else if (plan.merge_dtype == RG_F32) fe = cudaLaunchKernelEx(&cfg, splitk_fixup_kernel<true, false>, f);
+    else fe = cudaLaunchKernelEx(&cfg, splitk_fixup_kernel<true, true>, f);
+    if (fe != cudaSuccess) return RG_ERR_CUDA;
   }
   return RG_OK;
 }

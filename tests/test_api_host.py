@@ -36,7 +36,9 @@ def test_validate_rules():
     assert rg.rg_desc_validate(rg.rg_desc(cuts=(0,)), 64, 256, 512) == 2
     assert rg.rg_desc_validate(rg.rg_desc(cuts=(40,)), 64, 256, 512) == 3           # splits a 16-wide step
     assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_SCALAR), 64, 256, 512) == 3
-    assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16, merge_dtype=K.RG_BF16), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(merge_dtype=K.RG_BF16), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(BN=100), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(BN=112, BK=256), 64, 256, 512) == 0
     assert rg.rg_desc_validate(rg.rg_desc(BN=112, cta_group=2), 64, 256, 512) == 3
@@ -75,6 +77,7 @@ def test_workspace_bytes():
     assert rg.rg_gemm_workspace_bytes(rg.rg_desc(), 64, 256) == 0
     assert rg.rg_gemm_workspace_bytes(rg.rg_desc(cuts=(256,)), 64, 256) == 2 * 64 * 256 * 4
     assert rg.rg_gemm_workspace_bytes(rg.rg_desc(cuts=(16, 32, 48)), 3, 5) == 4 * 3 * 8 * 4
+    assert rg.rg_gemm_workspace_bytes(rg.rg_desc(cuts=(16, 32, 48), partial_dtype=K.RG_BF16), 3, 5) == 4 * 3 * 8 * 2
 
 
 def _t(ptr, dtype, rows, cols, ld=None):

@@ -283,3 +283,19 @@ def test_host_buffer_form_matches_device_form():
     rg_gemm_host(d, Ah, Bh, Ch, scratch, bias=bh, act=1)
     torch.cuda.synchronize()
     assert_bits_equal(synth.from_torch(Ch), gpu_gemm(A, B, cuts=(256,), bias=bias, act=1), "host-buffer GEMM")
+
+
+# ------------------------------------------------------------------ parts at bf16 (Sec. 3.2.2)
+@pytest.mark.parametrize("pd,md", [(rgo.BF16, rgo.F32), (rgo.BF16, rgo.BF16)])
+@pytest.mark.parametrize("tree", [rg.RG_TREE_LEFT, rg.RG_TREE_BALANCED])
+def test_partial_and_merge_dtypes_bit_exact(pd, md, tree):
+    for M, N, K, cuts in ((70, 200, 1024, (256, 512, 768)), (33, 130, 576, (192, 384)), (300, 260, 2048, tuple(256 * t for t in range(1, 8)))):
+        for name, A, B in _draws(M, N, K, 60 + K):
+            res = synth.normal_bf16((M, N), 1.0, 61)
+            for knobs in (dict(), dict(cta_group=2, BN=128), dict(BN=48)):
+                got = gpu_gemm(A, B, cuts=cuts, tree=tree, partial_dtype=pd, merge_dtype=md, residual=res, out_dtype=rgo.F32, **knobs)
+                want = rgo.gemm(A, B, cuts=cuts, tree=tree, atom_model=HW, partial_dtype=pd, merge_dtype=md, residual=res, out_dtype=rgo.F32)
+                assert_bits_equal(got, want, f"{M}x{N}x{K} {name} partial={pd} merge={md} {knobs}")
+    # the three combinations are three classes
+    keys = {rg.rg_desc_class(rg.rg_desc(cuts=(256,), partial_dtype=p_, merge_dtype=m_)) for p_, m_ in ((1, 1), (0, 1), (0, 0))}
+    assert len(keys) == 3

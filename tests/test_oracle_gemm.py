@@ -261,3 +261,36 @@ def test_epilogue_indexing_and_order():
     # bf16 output: exactly one rounding of the fp32 value
     got16 = rgo.gemm(Z, B, bias=bias, act=1, residual=res, out_dtype=rgo.BF16)
     assert np.array_equal(got16, synth.f32_to_bf16_bits(got))
+
+
+# ---- parts written at bf16, sum kept at fp32 or bf16 (Sec. 3.2.2: partial_dtype / merge_dtype)
+def test_partial_and_merge_dtypes():
+    A = synth.normal_bf16((6, 512), 1.0, 50); B = synth.normal_bf16((7, 512), 1.0, 51)
+    cuts = (128, 256, 384)
+    P32 = rgo.gemm_partials(A, B, cuts=cuts, atom_model=rgo.EXACT_RN)
+    P16 = rgo.gemm_partials(A, B, cuts=cuts, atom_model=rgo.EXACT_RN, partial_dtype=rgo.BF16)
+    # a bf16 part is the fp32 part rounded once (library conversion as the independent route)
+    import torch
+    want = torch.from_numpy(P32).to(torch.bfloat16).to(torch.float32).numpy()
+    assert np.array_equal(P16, want)
+    # parts at bf16, sum at fp32: the fp32 tree over the rounded parts
+    c_16_32 = rgo.gemm(A, B, cuts=cuts, atom_model=rgo.EXACT_RN, out_dtype=rgo.F32, partial_dtype=rgo.BF16)
+    assert np.array_equal(c_16_32, (P16[0] + P16[1]) + (P16[2] + P16[3]))
+    # both at bf16: every add rounded to bf16, checked with torch's bf16 adds (correctly rounded)
+    t = torch.from_numpy(P16).to(torch.bfloat16)
+    want = ((t[0] + t[1]) + (t[2] + t[3])).to(torch.float32).numpy()
+    c_16_16 = rgo.gemm(A, B, cuts=cuts, atom_model=rgo.EXACT_RN, out_dtype=rgo.F32, partial_dtype=rgo.BF16, merge_dtype=rgo.BF16)
+    assert np.array_equal(c_16_16, want)
+    want_left = (((t[0] + t[1]) + t[2]) + t[3]).to(torch.float32).numpy()
+    c_left = rgo.gemm(A, B, cuts=cuts, tree=rgo.TREE_LEFT, atom_model=rgo.EXACT_RN, out_dtype=rgo.F32,
+                      partial_dtype=rgo.BF16, merge_dtype=rgo.BF16)
+    assert np.array_equal(c_left, want_left)
+    # the three recorded combinations are three different classes of bits on ordinary inputs
+    c_32_32 = rgo.gemm(A, B, cuts=cuts, atom_model=rgo.EXACT_RN, out_dtype=rgo.F32)
+    assert not np.array_equal(c_32_32, c_16_32) and not np.array_equal(c_16_32, c_16_16)
+    # small integers are exact at every type, so all combinations agree with the integer product
+    Ai = synth.int_valued_bf16((5, 64), -2, 2, 1); Bi = synth.int_valued_bf16((4, 64), -2, 2, 2)
+    exact = (synth.bf16_bits_to_f32(Ai).astype(np.int64) @ synth.bf16_bits_to_f32(Bi).astype(np.int64).T).astype(np.float32)
+    for pd, md in ((rgo.F32, rgo.F32), (rgo.BF16, rgo.F32), (rgo.BF16, rgo.BF16)):
+        got = rgo.gemm(Ai, Bi, cuts=(16, 32, 48), out_dtype=rgo.F32, partial_dtype=pd, merge_dtype=md)
+        assert np.array_equal(got, exact)
