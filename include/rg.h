@@ -42,7 +42,7 @@ typedef enum {
   RG_ERR_TIMEOUT = 8        /* a bounded device-side wait gave up (see rg_device_status) */
 } rg_status_t;
 
-typedef enum { RG_BF16 = 0, RG_F32 = 1 } rg_dtype_t;
+typedef enum { RG_BF16 = 0, RG_F32 = 1, RG_F16 = 2 } rg_dtype_t;   /* RG_F16 = IEEE binary16 */
 
 /* The tree that combines values (split-K partials in rg_gemm, the leaves of a row in
  * rg_reduce_rows).  Sec. 3.1: a reduction order is a binary tree up to swapping an addition's
@@ -54,7 +54,8 @@ typedef enum { RG_TREE_LEFT = 0, RG_TREE_BALANCED = 1 } rg_tree_t;
 /* Which instruction folds products into the accumulator and how many per rounding step
  * (`instruction_k`, Sec. 3.2.1/3.2.2).  TC_BF16_K16: one tcgen05.mma kind::f16 step of 16
  * bf16 products, accumulator fp32 in tensor memory, steps chained in ascending k (App. E).
- * SCALAR names the fma-chain path; no kernel here implements it. */
+ * With RG_F16 operands the same step runs on fp16 products.  SCALAR names the fma-chain path; no kernel
+ * here implements it. */
 typedef enum { RG_ATOM_TC_BF16_K16 = 0, RG_ATOM_SCALAR = 1 } rg_atom_t;
 
 #define RG_MAX_CUTS 63
@@ -68,10 +69,10 @@ typedef struct {
   uint8_t raster;         /* tile walk: 0 = default grouped walk, 1 = row-major, n in 2..64 = groups of n tile rows */
   uint8_t _pad0;
   /* ---- order-deciding fields: these ARE the class key ---- */
-  uint8_t in_dtype;       /* rg_dtype_t of A and B: RG_BF16 */
+  uint8_t in_dtype;       /* rg_dtype_t of A and B: RG_BF16 or RG_F16 */
   uint8_t acc_dtype;      /* accumulator: RG_F32 */
-  uint8_t partial_dtype;  /* type a finished split-K part is written at: RG_F32 or RG_BF16 (Sec. 3.2.2) */
-  uint8_t merge_dtype;    /* type the running sum of the parts is kept at: RG_F32, or RG_BF16 with bf16 parts */
+  uint8_t partial_dtype;  /* type a finished split-K part is written at: RG_F32, RG_BF16 or RG_F16 (Sec. 3.2.2) */
+  uint8_t merge_dtype;    /* type the running sum of the parts is kept at: RG_F32, or the 16-bit type of the parts */
   uint8_t atom;           /* rg_atom_t */
   uint8_t k_tail;         /* 0 = the short K turn runs last, missing products are absent */
   uint8_t fma;            /* multiply-add fusion on scalar leaves (reductions: x*x feeding an add) */
@@ -135,7 +136,8 @@ size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N);
  * with cuts the parts go to `ws` as [part][M][roundup(N,4)] at partial_dtype and a second kernel
  * merges them, the running sum kept at merge_dtype (no atomics anywhere).
  *
- *   A: [M,K] bf16, B: [N,K] bf16 (both K-contiguous), C: [M,N] bf16 or fp32.
+ *   A: [M,K], B: [N,K] (both K-contiguous) at d->in_dtype (bf16 or fp16); C: [M,N] bf16, fp16 or fp32;
+ *   bias and residual likewise bf16, fp16 or fp32.
  *   A.ptr, B.ptr 16-byte aligned; A.ld, B.ld multiples of 8.  C, bias, residual: any alignment.
  *   epi: nullable.  ws: device, 16-byte aligned, >= rg_gemm_workspace_bytes; contents undefined
  *   afterwards; may be NULL when there are no cuts.

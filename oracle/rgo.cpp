@@ -55,14 +55,54 @@ inline uint16_t f32_to_bf16(float f) {
   return uint16_t(u >> 16);
 }
 
-enum { DT_BF16 = 0, DT_F32 = 1 };
+enum { DT_BF16 = 0, DT_F32 = 1, DT_F16 = 2 };
+
+// IEEE binary16 (1-5-10): widening is exact.
+inline float f16_to_f32(uint16_t h) {
+  const uint32_t sign = uint32_t(h >> 15) << 31;
+  const int e = (h >> 10) & 0x1f;
+  const uint32_t m = h & 0x3ffu;
+  if (e == 0x1f) return bits_f32(sign | 0x7f800000u | (m << 13));
+  if (e == 0) {                                   // zero or subnormal: m * 2^-24
+    const float v = float(m) * 0x1p-24f;          // exact
+    return sign ? -v : v;
+  }
+  return bits_f32(sign | (uint32_t(e + 112) << 23) | (m << 13));
+}
+
+// Round-to-nearest-even narrowing binary32 -> binary16, subnormals kept, overflow to infinity.
+inline uint16_t f32_to_f16(float f) {
+  const uint32_t u = f32_bits(f);
+  const uint16_t sign = uint16_t((u >> 16) & 0x8000u);
+  const uint32_t a = u & 0x7fffffffu;
+  if (a > 0x7f800000u) return uint16_t(sign | 0x7e00u);          // NaN
+  if (a >= 0x47800000u) return uint16_t(sign | 0x7c00u);         // >= 65536 (or inf): infinity
+  const int e = int(a >> 23) - 127;                               // unbiased exponent
+  uint32_t mant = (a & 0x7fffffu) | 0x800000u;                    // 24-bit significand
+  int shift;                                                      // bits dropped from the significand
+  uint32_t base;
+  if (e >= -14) { shift = 13; base = uint32_t(e + 15) << 10; }    // normal target
+  else { shift = 13 + (-14 - e); base = 0; }                      // subnormal target
+  if (a == 0) return sign;
+  if (shift > 25) return sign;                                    // below half the smallest subnormal
+  const uint32_t kept = mant >> shift;
+  const uint32_t rem = mant & ((1u << shift) - 1u);
+  const uint32_t half = 1u << (shift - 1);
+  uint32_t r = (e >= -14) ? (base + (kept & 0x3ffu)) : kept;      // hidden bit folded into the exponent field
+  if (rem > half || (rem == half && (r & 1u))) r += 1;            // a carry walks into the exponent: still correct
+  return uint16_t(sign | r);                                      // 0x7c00 when it rounds up to infinity
+}
+
+inline float in_to_f32(uint16_t h, int dtype) { return dtype == DT_F16 ? f16_to_f32(h) : bf16_to_f32(h); }
 
 inline float load_elem(const void* p, int dtype, int64_t idx) {
   if (dtype == DT_BF16) return bf16_to_f32(static_cast<const uint16_t*>(p)[idx]);
+  if (dtype == DT_F16) return f16_to_f32(static_cast<const uint16_t*>(p)[idx]);
   return static_cast<const float*>(p)[idx];
 }
 inline void store_elem(void* p, int dtype, int64_t idx, float v) {
   if (dtype == DT_BF16) static_cast<uint16_t*>(p)[idx] = f32_to_bf16(v);
+  else if (dtype == DT_F16) static_cast<uint16_t*>(p)[idx] = f32_to_f16(v);
   else static_cast<float*>(p)[idx] = v;
 }
 
@@ -99,7 +139,9 @@ float tree_reduce(std::vector<float>& v, int tree) {
 // is written at one type and the running sum kept at another"): every add is an fp32 add whose
 // result is then rounded to the merge type (for bf16 operands this equals the correctly rounded
 // bf16 sum: the fp32 add is exact or its error lies far below half a bf16 ulp).
-inline float round_to(float v, int dtype) { return dtype == DT_BF16 ? bf16_to_f32(f32_to_bf16(v)) : v; }
+inline float round_to(float v, int dtype) {
+  return dtype == DT_BF16 ? bf16_to_f32(f32_to_bf16(v)) : dtype == DT_F16 ? f16_to_f32(f32_to_f16(v)) : v;
+}
 
 float tree_reduce_at(std::vector<float>& v, int tree, int merge_dtype) {
   if (merge_dtype == DT_F32) return tree_reduce(v, tree);
@@ -228,6 +270,7 @@ struct AtomModel {
   int32_t acc_in_window;  // 1: the accumulator is aligned/truncated like a product
   int32_t addend_round;   // 0: truncate toward zero; 1: floor (toward -inf)
   int32_t final_round;    // 0: RZ; 1: RN-even
+  int32_t in_dtype;       // operand type of the products: DT_BF16 or DT_F16
 };
 enum { ATOM_EXACT_RN = 0, ATOM_SEQ = 1, ATOM_ALIGN_TRUNC = 2 };
 
@@ -241,39 +284,48 @@ inline void bf16_decode(uint16_t h, int& sign, uint32_t& mag, int& exp, int& e_l
   else { mag = m | 0x80; exp = e - 134; e_lead = e - 127; }
 }
 inline bool bf16_finite(uint16_t h) { return ((h >> 7) & 0xff) != 0xff; }
+inline void f16_decode(uint16_t h, int& sign, uint32_t& mag, int& exp, int& e_lead) {
+  sign = (h >> 15) ? -1 : 1;
+  int e = (h >> 10) & 0x1f;
+  uint32_t m = h & 0x3ff;
+  if (e == 0) { mag = m; exp = -24; e_lead = -14; }
+  else { mag = m | 0x400; exp = e - 25; e_lead = e - 15; }
+}
+inline bool f16_finite(uint16_t h) { return ((h >> 10) & 0x1f) != 0x1f; }
+inline bool in_finite(uint16_t h, int dtype) { return dtype == DT_F16 ? f16_finite(h) : bf16_finite(h); }
 
-inline Prod make_prod(uint16_t a, uint16_t b) {
+inline Prod make_prod(uint16_t a, uint16_t b, int dtype) {
   int sa, sb, ea, eb, la, lb; uint32_t ma, mb;
-  bf16_decode(a, sa, ma, ea, la);
-  bf16_decode(b, sb, mb, eb, lb);
+  if (dtype == DT_F16) { f16_decode(a, sa, ma, ea, la); f16_decode(b, sb, mb, eb, lb); }
+  else { bf16_decode(a, sa, ma, ea, la); bf16_decode(b, sb, mb, eb, lb); }
   Prod p; p.sign = sa * sb; p.mag = ma * mb; p.exp = ea + eb; p.e_op = la + lb;
   return p;
 }
 
 inline int ilog2_u64(uint64_t v) { return 63 - __builtin_clzll(v); }
 
-float atom_seq(float acc, const uint16_t* a, const uint16_t* b, int n, int fma) {
+float atom_seq(float acc, const uint16_t* a, const uint16_t* b, int n, int fma, int dtype) {
   // Sec. 3.2.1, scalar path: acc <- fma(a, b, acc), or two roundings unfused.
   for (int u = 0; u < n; ++u) {
-    float x = bf16_to_f32(a[u]), y = bf16_to_f32(b[u]);
+    float x = in_to_f32(a[u], dtype), y = in_to_f32(b[u], dtype);
     if (fma) acc = std::fmaf(x, y, acc);
     else { float p = x * y; acc = acc + p; }
   }
   return acc;
 }
 
-float atom_exact_rn(float acc, const uint16_t* a, const uint16_t* b, int n) {
+float atom_exact_rn(float acc, const uint16_t* a, const uint16_t* b, int n, int dtype) {
   // Sec. 3.2.1: acc <- RN_fp32(acc + sum_j a_j*b_j), the sum formed exactly.
   LongAcc L;
   L.add_f32(acc);
   for (int u = 0; u < n; ++u) {
-    Prod p = make_prod(a[u], b[u]);
+    Prod p = make_prod(a[u], b[u], dtype);
     L.add(p.sign, p.mag, p.exp);
   }
   // An exactly-zero sum: IEEE gives +0 under RN unless every addend is -0.
   bool all_neg_zero = (f32_bits(acc) == 0x80000000u);
   for (int u = 0; u < n && all_neg_zero; ++u) {
-    Prod p = make_prod(a[u], b[u]);
+    Prod p = make_prod(a[u], b[u], dtype);
     if (!(p.mag == 0 && p.sign < 0)) all_neg_zero = false;
   }
   return round_longacc(L, ROUND_RN, all_neg_zero ? -0.0f : 0.0f);
@@ -285,7 +337,7 @@ float align_trunc_step(float acc, const uint16_t* a, const uint16_t* b, int n, c
   Prod p[64];
   int emax = INT32_MIN;
   for (int u = 0; u < n; ++u) {
-    p[u] = make_prod(a[u], b[u]);
+    p[u] = make_prod(a[u], b[u], m.in_dtype);
     if (p[u].mag) {
       int e = m.exp_mode ? p[u].e_op : (p[u].exp + ilog2_u64(p[u].mag));
       emax = std::max(emax, e);
@@ -324,11 +376,11 @@ float align_trunc_step(float acc, const uint16_t* a, const uint16_t* b, int n, c
 
 float atom_step(float acc, const uint16_t* a, const uint16_t* b, int n, const AtomModel& m) {
   for (int u = 0; u < n; ++u)
-    if (!bf16_finite(a[u]) || !bf16_finite(b[u])) return atom_seq(acc, a, b, n, 1);
-  if (!std::isfinite(acc)) return atom_seq(acc, a, b, n, 1);
+    if (!in_finite(a[u], m.in_dtype) || !in_finite(b[u], m.in_dtype)) return atom_seq(acc, a, b, n, 1, m.in_dtype);
+  if (!std::isfinite(acc)) return atom_seq(acc, a, b, n, 1, m.in_dtype);
   switch (m.model) {
-    case ATOM_SEQ: return atom_seq(acc, a, b, n, m.fma);
-    case ATOM_EXACT_RN: return atom_exact_rn(acc, a, b, n);
+    case ATOM_SEQ: return atom_seq(acc, a, b, n, m.fma, m.in_dtype);
+    case ATOM_EXACT_RN: return atom_exact_rn(acc, a, b, n, m.in_dtype);
     default: {
       int g = m.group > 0 ? m.group : n;
       for (int u0 = 0; u0 < n; u0 += g) acc = align_trunc_step(acc, a + u0, b + u0, std::min(g, n - u0), m);
@@ -423,6 +475,8 @@ int rgo_num_threads() {
 
 float rgo_bf16_to_f32(uint16_t h) { return bf16_to_f32(h); }
 uint16_t rgo_f32_to_bf16(float f) { return f32_to_bf16(f); }
+float rgo_f16_to_f32(uint16_t h) { return f16_to_f32(h); }
+uint16_t rgo_f32_to_f16(float f) { return f32_to_f16(f); }
 float rgo_add_f32(float a, float b) { return a + b; }
 float rgo_mul_f32(float a, float b) { return a * b; }
 float rgo_expf(float x) { return rg_expf(x); }
@@ -469,7 +523,7 @@ void rgo_gemm_samples(const AtomModel* atom, int tree, int n_cuts, const int64_t
 #pragma omp parallel for schedule(static)
   for (int64_t t = 0; t < n_samples; ++t) {
     float v = gemm_element(d, A + si[t] * lda, B + sj[t] * ldb, K, si[t], sj[t], nullptr);
-    out[t] = out_dtype == DT_BF16 ? bf16_to_f32(f32_to_bf16(v)) : v;
+    out[t] = round_to(v, out_dtype);
   }
 }
 

@@ -20,7 +20,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "rgo.cpp")
 _LIB = os.path.join(_HERE, "librgo.so")
 
-BF16, F32 = 0, 1
+BF16, F32, F16 = 0, 1, 2
 TREE_LEFT, TREE_BALANCED = 0, 1
 OP_SUM, OP_RMSNORM, OP_SOFTMAX_DENOM = 0, 1, 2
 ATOM_EXACT_RN, ATOM_SEQ, ATOM_ALIGN_TRUNC = 0, 1, 2
@@ -38,7 +38,7 @@ def build(force: bool = False) -> str:
 class _AtomStruct(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "model", "atom_k", "fma", "group", "window_bits", "exp_mode", "acc_in_window",
-        "addend_round", "final_round")]
+        "addend_round", "final_round", "in_dtype")]
 
 
 @dataclass(frozen=True)
@@ -54,10 +54,16 @@ class AtomModel:
     acc_in_window: int = 1
     addend_round: int = 0
     final_round: int = 1
+    in_dtype: int = BF16
 
     def c(self) -> _AtomStruct:
         return _AtomStruct(self.model, self.atom_k, self.fma, self.group, self.window_bits,
-                           self.exp_mode, self.acc_in_window, self.addend_round, self.final_round)
+                           self.exp_mode, self.acc_in_window, self.addend_round, self.final_round, self.in_dtype)
+
+    def with_inputs(self, in_dtype: int) -> "AtomModel":
+        """The same step model reading operands of another 16-bit type."""
+        import dataclasses
+        return dataclasses.replace(self, in_dtype=in_dtype)
 
 
 EXACT_RN = AtomModel(model=ATOM_EXACT_RN)
@@ -82,6 +88,8 @@ def lib():
         L.rgo_num_threads.restype = i32
         L.rgo_bf16_to_f32.restype = f32; L.rgo_bf16_to_f32.argtypes = [C.c_uint16]
         L.rgo_f32_to_bf16.restype = C.c_uint16; L.rgo_f32_to_bf16.argtypes = [f32]
+        L.rgo_f16_to_f32.restype = f32; L.rgo_f16_to_f32.argtypes = [C.c_uint16]
+        L.rgo_f32_to_f16.restype = C.c_uint16; L.rgo_f32_to_f16.argtypes = [f32]
         for n in ("rgo_add_f32", "rgo_mul_f32"):
             getattr(L, n).restype = f32; getattr(L, n).argtypes = [f32, f32]
         for n in ("rgo_expf", "rgo_silu"):
@@ -115,6 +123,14 @@ def f32_to_bf16(f) -> int:
     return int(lib().rgo_f32_to_bf16(np.float32(f)))
 
 
+def f16_to_f32(h: int) -> float:
+    return float(lib().rgo_f16_to_f32(int(h)))
+
+
+def f32_to_f16(f) -> int:
+    return int(lib().rgo_f32_to_f16(np.float32(f)))
+
+
 def add_f32(a, b) -> np.float32:
     return np.float32(lib().rgo_add_f32(np.float32(a), np.float32(b)))
 
@@ -140,7 +156,21 @@ def _dtype_code(a: np.ndarray) -> int:
         return BF16
     if a.dtype == np.float32:
         return F32
-    raise TypeError(f"oracle arrays are uint16 (bf16 bits) or float32, got {a.dtype}")
+    if a.dtype == np.float16:
+        return F16
+    raise TypeError(f"oracle arrays are uint16 (bf16 bits), float16 or float32, got {a.dtype}")
+
+
+def _operands(A, B, atom_model):
+    """A, B as 16-bit patterns; float16 arrays select fp16 operands in the step model."""
+    A = np.ascontiguousarray(A); B = np.ascontiguousarray(B)
+    if A.dtype == np.float16 or B.dtype == np.float16:
+        assert A.dtype == np.float16 and B.dtype == np.float16
+        return A.view(np.uint16), B.view(np.uint16), atom_model.with_inputs(F16)
+    return np.ascontiguousarray(A, dtype=np.uint16), np.ascontiguousarray(B, dtype=np.uint16), atom_model.with_inputs(BF16)
+
+
+_OUT_NP = {BF16: np.uint16, F32: np.float32, F16: np.float16}
 
 
 def tree_sum(v, tree: int = TREE_BALANCED) -> np.float32:
@@ -149,6 +179,8 @@ def tree_sum(v, tree: int = TREE_BALANCED) -> np.float32:
 
 
 def atom(model: AtomModel, acc, a_bits, b_bits) -> np.float32:
+    if isinstance(a_bits, np.ndarray) and a_bits.dtype == np.float16:
+        a_bits, b_bits, model = a_bits.view(np.uint16), np.ascontiguousarray(b_bits, np.float16).view(np.uint16), model.with_inputs(F16)
     a = np.ascontiguousarray(a_bits, dtype=np.uint16)
     b = np.ascontiguousarray(b_bits, dtype=np.uint16)
     assert a.size == b.size <= 64
@@ -174,11 +206,11 @@ def gemm(A, B, *, cuts=(), tree=TREE_BALANCED, atom_model: AtomModel = EXACT_RN,
     A [M,K], B [N,K] are uint16 bf16 bit patterns.  Returns uint16 (bf16) or float32.
     partial_dtype / merge_dtype: the type a finished split-K part is written at and the type the
     running sum of the parts is kept at."""
-    A = np.ascontiguousarray(A, dtype=np.uint16); B = np.ascontiguousarray(B, dtype=np.uint16)
+    A, B, atom_model = _operands(A, B, atom_model)
     M, K = A.shape; N, K2 = B.shape
     assert K == K2
     c = _cuts(cuts)
-    out = np.empty((M, N), dtype=np.uint16 if out_dtype == BF16 else np.float32)
+    out = np.empty((M, N), dtype=_OUT_NP[out_dtype])
     b, bd, r, rd, ldr = _epi(bias, residual)
     m = atom_model.c()
     lib().rgo_gemm(C.byref(m), tree, c.size, _ptr(c), M, N, K, _ptr(A), K, _ptr(B), K,
@@ -189,7 +221,7 @@ def gemm(A, B, *, cuts=(), tree=TREE_BALANCED, atom_model: AtomModel = EXACT_RN,
 def gemm_samples(A, B, si, sj, *, cuts=(), tree=TREE_BALANCED, atom_model: AtomModel = EXACT_RN,
                  out_dtype=BF16, bias=None, act=0, residual=None, partial_dtype=F32, merge_dtype=F32) -> np.ndarray:
     """Output elements (si[t], sj[t]) only; returned as float32 after the output rounding."""
-    A = np.ascontiguousarray(A, dtype=np.uint16); B = np.ascontiguousarray(B, dtype=np.uint16)
+    A, B, atom_model = _operands(A, B, atom_model)
     K = A.shape[1]
     si = np.ascontiguousarray(si, dtype=np.int64); sj = np.ascontiguousarray(sj, dtype=np.int64)
     c = _cuts(cuts)
@@ -204,7 +236,7 @@ def gemm_samples(A, B, si, sj, *, cuts=(), tree=TREE_BALANCED, atom_model: AtomM
 
 def gemm_partials(A, B, *, cuts=(), atom_model: AtomModel = EXACT_RN, partial_dtype=F32) -> np.ndarray:
     """The partial of every part, shape [S, M, N], as fp32 values at partial_dtype (Sec. 3.2.2, split-K)."""
-    A = np.ascontiguousarray(A, dtype=np.uint16); B = np.ascontiguousarray(B, dtype=np.uint16)
+    A, B, atom_model = _operands(A, B, atom_model)
     M, K = A.shape; N = B.shape[0]
     c = _cuts(cuts)
     P = np.empty((c.size + 1, M, N), dtype=np.float32)

@@ -28,6 +28,8 @@ def rg_desc(*, cuts: Sequence[int] = (), tree: int = K.RG_TREE_BALANCED, fma: in
     d.tree, d.fma = tree, fma
     for k, v in order_fields.items():
         setattr(d, k, v)
+    if "in_dtype" not in order_fields:
+        d.in_dtype = K.RG_BF16
     cuts = list(cuts)
     if len(cuts) > K.RG_MAX_CUTS:
         raise RgError(2, "rg_desc")
@@ -67,7 +69,9 @@ def _dtype_code(t) -> int:
         return K.RG_BF16
     if t.dtype == torch.float32:
         return K.RG_F32
-    raise TypeError(f"rg tensors are bfloat16 or float32, got {t.dtype}")
+    if t.dtype == torch.float16:
+        return K.RG_F16
+    raise TypeError(f"rg tensors are bfloat16, float16 or float32, got {t.dtype}")
 
 
 def _tensor(t) -> K.rg_tensor_t:

@@ -8,15 +8,15 @@ namespace {
 
 constexpr int64_t DIM_LIMIT = (int64_t(1) << 31) - 1024;
 
-bool dtype_ok(int32_t t) { return t == RG_BF16 || t == RG_F32; }
-size_t esize(int32_t t) { return t == RG_BF16 ? 2 : 4; }
+bool dtype_ok(int32_t t) { return t == RG_BF16 || t == RG_F32 || t == RG_F16; }
+size_t esize(int32_t t) { return t == RG_F32 ? 4 : 2; }
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Structural checks that do not depend on a shape.
 rg_status_t check_desc_fields(const rg_desc_t* d) {
   if (!d) return RG_ERR_NULL;
   if (d->size != sizeof(rg_desc_t)) return RG_ERR_INVALID_DESC;
-  if (d->in_dtype > RG_F32 || d->acc_dtype > RG_F32 || d->partial_dtype > RG_F32 || d->merge_dtype > RG_F32)
+  if (d->in_dtype > RG_F16 || d->acc_dtype > RG_F16 || d->partial_dtype > RG_F16 || d->merge_dtype > RG_F16)
     return RG_ERR_INVALID_DESC;
   if (d->atom > RG_ATOM_SCALAR || d->tree > RG_TREE_BALANCED || d->fma > 1 || d->k_tail > 1) return RG_ERR_INVALID_DESC;
   if (d->n_cuts > RG_MAX_CUTS) return RG_ERR_INVALID_DESC;
@@ -29,9 +29,9 @@ rg_status_t check_desc_fields(const rg_desc_t* d) {
 
 // What the kernels of this library can honour.
 rg_status_t check_desc_supported(const rg_desc_t* d) {
-  if (d->in_dtype != RG_BF16 || d->acc_dtype != RG_F32) return RG_ERR_UNSUPPORTED;
-  // parts at fp32 summed at fp32, parts at bf16 summed at fp32, or both at bf16 (Sec. 3.2.2)
-  if (d->partial_dtype == RG_F32 && d->merge_dtype != RG_F32) return RG_ERR_UNSUPPORTED;
+  if ((d->in_dtype != RG_BF16 && d->in_dtype != RG_F16) || d->acc_dtype != RG_F32) return RG_ERR_UNSUPPORTED;
+  // parts at fp32 summed at fp32, parts at a 16-bit type summed at fp32, or both at that type (Sec. 3.2.2)
+  if (d->merge_dtype != RG_F32 && d->merge_dtype != d->partial_dtype) return RG_ERR_UNSUPPORTED;
   if (d->atom != RG_ATOM_TC_BF16_K16 || d->k_tail != 0) return RG_ERR_UNSUPPORTED;
   if (d->BM != 0 && d->BM != 128 && d->BM != 256) return RG_ERR_UNSUPPORTED;
   if (d->BN != 0 && (d->BN % 16 != 0 || d->BN < 16 || d->BN > 256)) return RG_ERR_UNSUPPORTED;
@@ -66,7 +66,7 @@ rg_status_t check_epilogue(const rg_epilogue_t* e, int64_t N) {
 rg_status_t check_gemm_shapes(const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C) {
   rg_status_t s;
   if ((s = check_tensor(A)) != RG_OK || (s = check_tensor(B)) != RG_OK || (s = check_tensor(C)) != RG_OK) return s;
-  if (A->dtype != RG_BF16 || B->dtype != RG_BF16) return RG_ERR_UNSUPPORTED;
+  if ((A->dtype != RG_BF16 && A->dtype != RG_F16) || B->dtype != A->dtype) return RG_ERR_UNSUPPORTED;
   if (A->cols != B->cols || C->rows != A->rows || C->cols != B->rows) return RG_ERR_SHAPE;
   return RG_OK;
 }
@@ -163,7 +163,7 @@ uint64_t rg_desc_class(const rg_desc_t* d) {
 
 size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N) {
   if (!d || d->n_cuts == 0 || d->n_cuts > RG_MAX_CUTS || M <= 0 || N <= 0) return 0;
-  return (size_t)(d->n_cuts + 1) * (size_t)M * (size_t)((N + 3) / 4 * 4) * (d->partial_dtype == RG_BF16 ? 2 : 4);
+  return (size_t)(d->n_cuts + 1) * (size_t)M * (size_t)((N + 3) / 4 * 4) * (d->partial_dtype == RG_F32 ? 4 : 2);
 }
 
 rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
@@ -174,6 +174,7 @@ rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t*
   const int64_t M = A->rows, K = A->cols, N = B->rows;
   if (K < 1) return RG_ERR_SHAPE;
   if ((s = rg_desc_validate(d, M, N, K)) != RG_OK) return s;
+  if (A->dtype != d->in_dtype) return RG_ERR_SHAPE;          // operands must be of the descriptor's input type
   if ((s = check_epilogue(epi, N)) != RG_OK) return s;
   if (M == 0 || N == 0) return RG_OK;
   if ((reinterpret_cast<uintptr_t>(A->ptr) & 15) || (reinterpret_cast<uintptr_t>(B->ptr) & 15) ||
@@ -194,6 +195,7 @@ static rg_status_t check_reduce(const rg_desc_t* d, rg_reduce_op_t op, const rg_
   if ((s = check_tensor(x)) != RG_OK || (s = check_tensor(out)) != RG_OK) return s;
   if (op != RG_OP_SUM && op != RG_OP_RMSNORM && op != RG_OP_SOFTMAX_DENOM) return RG_ERR_UNSUPPORTED;
   if (d->acc_dtype != RG_F32 || d->tree != RG_TREE_BALANCED) return RG_ERR_UNSUPPORTED;
+  if (x->dtype == RG_F16 || out->dtype == RG_F16) return RG_ERR_UNSUPPORTED;   // reductions read bf16 or fp32 rows
   if (x->cols < 1) return RG_ERR_SHAPE;
   if (out->rows != x->rows) return RG_ERR_SHAPE;
   if (op == RG_OP_RMSNORM) { if (out->cols != x->cols) return RG_ERR_SHAPE; }
@@ -242,8 +244,8 @@ rg_status_t rg_gemm_host(const rg_desc_t* d, const rg_tensor_t* A, const rg_tens
   const int64_t ldk = (K + 7) / 8 * 8;
   uint8_t* cur = static_cast<uint8_t*>(dev_scratch);
   auto take = [&](size_t bytes) { uint8_t* p = cur; cur += align_up(bytes, 256); return p; };
-  rg_tensor_t dA{take((size_t)M * ldk * 2), RG_BF16, M, K, ldk};
-  rg_tensor_t dB{take((size_t)N * ldk * 2), RG_BF16, N, K, ldk};
+  rg_tensor_t dA{take((size_t)M * ldk * 2), A->dtype, M, K, ldk};
+  rg_tensor_t dB{take((size_t)N * ldk * 2), B->dtype, N, K, ldk};
   rg_tensor_t dC{take((size_t)M * N * esize(C->dtype)), C->dtype, M, N, N};
   rg_epilogue_t de{};
   if (epi) de = *epi;

@@ -4,6 +4,7 @@
 // written here is the one that runs (Sec. 3.1).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -58,16 +59,33 @@ struct EpilogueArgs {
   int32_t act;
 };
 
+__device__ __forceinline__ float f16_bits_to_f32(uint32_t h) { return __half2float(__ushort_as_half((unsigned short)h)); }
+
 __device__ __forceinline__ float load_scalar(const void* p, int dtype, int64_t idx) {
   if (dtype == RG_BF16) return bf16_bits_to_f32(static_cast<const uint16_t*>(p)[idx]);
+  if (dtype == RG_F16) return f16_bits_to_f32(static_cast<const uint16_t*>(p)[idx]);
   return static_cast<const float*>(p)[idx];
 }
+
+// One rounding of an fp32 value to `dtype` and back (identity for fp32).
+__device__ __forceinline__ float round_through(float v, int dtype) {
+  if (dtype == RG_BF16) return __bfloat162float(__float2bfloat16_rn(v));
+  if (dtype == RG_F16) return __half2float(__float2half_rn(v));
+  return v;
+}
+
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  const __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+__device__ __forceinline__ uint32_t pack_16x2(float lo, float hi, int dtype);
 
 // `n` (<= 32) consecutive elements starting at element index `idx` of a bf16 or fp32 array, widened
 // to fp32; entries past n are zero.  Uses 16-byte loads when the segment is full and aligned.
 __device__ __forceinline__ void load_row_segment(const void* base, int dtype, int64_t idx, int n, float (&out)[32]) {
-  if (dtype == RG_BF16) {
+  if (dtype == RG_BF16 || dtype == RG_F16) {
     const uint16_t* p = static_cast<const uint16_t*>(base) + idx;
+    const bool half = dtype == RG_F16;
     if (n == 32 && (reinterpret_cast<uintptr_t>(p) & 15) == 0) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
@@ -75,13 +93,13 @@ __device__ __forceinline__ void load_row_segment(const void* base, int dtype, in
         const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-          out[8 * q + 2 * t] = bf16_bits_to_f32(ww[t] & 0xffffu);
-          out[8 * q + 2 * t + 1] = bf16_bits_to_f32(ww[t] >> 16);
+          out[8 * q + 2 * t] = half ? f16_bits_to_f32(ww[t] & 0xffffu) : bf16_bits_to_f32(ww[t] & 0xffffu);
+          out[8 * q + 2 * t + 1] = half ? f16_bits_to_f32(ww[t] >> 16) : bf16_bits_to_f32(ww[t] >> 16);
         }
       }
     } else {
 #pragma unroll
-      for (int c = 0; c < 32; ++c) out[c] = c < n ? bf16_bits_to_f32(p[c]) : 0.0f;
+      for (int c = 0; c < 32; ++c) out[c] = c < n ? (half ? f16_bits_to_f32(p[c]) : bf16_bits_to_f32(p[c])) : 0.0f;
     }
   } else {
     const float* p = static_cast<const float*>(base) + idx;
@@ -111,6 +129,17 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   // one cvt.rn.bf16x2.f32: each half is rounded to nearest even exactly as a single conversion is
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+__device__ __forceinline__ uint32_t pack_16x2(float lo, float hi, int dtype) {
+  return dtype == RG_F16 ? pack_f16x2(lo, hi) : pack_bf16x2(lo, hi);
+}
+
+// Store one fp32 value rounded once to a 16-bit or fp32 output element.
+__device__ __forceinline__ void store_scalar(void* p, int dtype, int64_t idx, float v) {
+  if (dtype == RG_BF16) static_cast<__nv_bfloat16*>(p)[idx] = __float2bfloat16_rn(v);
+  else if (dtype == RG_F16) static_cast<__half*>(p)[idx] = __float2half_rn(v);
+  else static_cast<float*>(p)[idx] = v;
 }
 
 }  // namespace rg

@@ -142,9 +142,10 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
   d |= static_cast<uint64_t>(2) << 61;                         // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = BN.
-__host__ __device__ constexpr uint32_t make_idesc(int bn, int m = BM) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(bn >> 3) << 17) |
+// Instruction descriptor: 16-bit x 16-bit -> fp32, both operands K-major.
+// operand format field: 0 = fp16, 1 = bf16
+__host__ __device__ constexpr uint32_t make_idesc(int bn, int m, uint32_t fmt) {
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | (static_cast<uint32_t>(bn >> 3) << 17) |
          (static_cast<uint32_t>(m >> 4) << 24);
 }
 
@@ -210,20 +211,20 @@ __device__ __forceinline__ void epilogue_row_segment(float (&v)[32], const Epilo
   }
 }
 
-// Store up to 32 consecutive columns of one output row.
+// Store up to 32 consecutive columns of one output row, each value rounded once to the output type.
 __device__ __forceinline__ void store_row_segment(const GemmParams& p, int64_t row, int col0, int ncols, const float (&v)[32]) {
-  if (p.c_dtype == RG_BF16) {
-    __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.C) + row * p.ldc + col0;
+  if (p.c_dtype == RG_BF16 || p.c_dtype == RG_F16) {
+    uint16_t* dst = static_cast<uint16_t*>(p.C) + row * p.ldc + col0;
     if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        uint4 o = make_uint4(pack_bf16x2(v[8 * q], v[8 * q + 1]), pack_bf16x2(v[8 * q + 2], v[8 * q + 3]),
-                             pack_bf16x2(v[8 * q + 4], v[8 * q + 5]), pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
+        uint4 o = make_uint4(pack_16x2(v[8 * q], v[8 * q + 1], p.c_dtype), pack_16x2(v[8 * q + 2], v[8 * q + 3], p.c_dtype),
+                             pack_16x2(v[8 * q + 4], v[8 * q + 5], p.c_dtype), pack_16x2(v[8 * q + 6], v[8 * q + 7], p.c_dtype));
         reinterpret_cast<uint4*>(dst)[q] = o;
       }
     } else {
 #pragma unroll
-      for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __float2bfloat16_rn(v[c]);
+      for (int c = 0; c < 32; ++c) if (c < ncols) store_scalar(p.C, p.c_dtype, row * p.ldc + col0 + c, v[c]);
     }
   } else {
     float* dst = static_cast<float*>(p.C) + row * p.ldc + col0;
@@ -264,19 +265,20 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, const int BN,
           for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __uint_as_float(r[c]);
         }
       } else if (p.ws) {
-        // the finished part written at bf16: one rounding of the fp32 accumulator
-        __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.ws) + ((int64_t)part * p.M + row) * p.ldw + col0;
+        // the finished part written at a 16-bit type: one rounding of the fp32 accumulator
+        const int64_t off = ((int64_t)part * p.M + row) * p.ldw + col0;
+        uint16_t* dst = static_cast<uint16_t*>(p.ws) + off;
         if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
 #pragma unroll
           for (int q = 0; q < 4; ++q)
             reinterpret_cast<uint4*>(dst)[q] = make_uint4(
-                pack_bf16x2(__uint_as_float(r[8 * q]), __uint_as_float(r[8 * q + 1])),
-                pack_bf16x2(__uint_as_float(r[8 * q + 2]), __uint_as_float(r[8 * q + 3])),
-                pack_bf16x2(__uint_as_float(r[8 * q + 4]), __uint_as_float(r[8 * q + 5])),
-                pack_bf16x2(__uint_as_float(r[8 * q + 6]), __uint_as_float(r[8 * q + 7])));
+                pack_16x2(__uint_as_float(r[8 * q]), __uint_as_float(r[8 * q + 1]), p.ws_dtype),
+                pack_16x2(__uint_as_float(r[8 * q + 2]), __uint_as_float(r[8 * q + 3]), p.ws_dtype),
+                pack_16x2(__uint_as_float(r[8 * q + 4]), __uint_as_float(r[8 * q + 5]), p.ws_dtype),
+                pack_16x2(__uint_as_float(r[8 * q + 6]), __uint_as_float(r[8 * q + 7]), p.ws_dtype));
         } else {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __float2bfloat16_rn(__uint_as_float(r[c]));
+          for (int c = 0; c < 32; ++c) if (c < ncols) store_scalar(p.ws, p.ws_dtype, off + c, __uint_as_float(r[c]));
         }
       } else {
         float v[32];
@@ -461,7 +463,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   constexpr uint32_t B_BOX_BYTES = (BN / 2) * KBOX * 2;
   constexpr uint32_t STAGE_BYTES = KSUB * (A_BOX_BYTES + B_BOX_BYTES);      // per CTA
   constexpr uint32_t TMEM_COLS = 2 * BN;
-  constexpr uint32_t IDESC = make_idesc(BN, 2 * BM);
+  const uint32_t IDESC = p.idesc;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -614,7 +616,7 @@ struct FixupParams {
 // with fp32 adds, the running sum kept at merge_dtype (an add whose result is rounded to bf16 when
 // the sum is kept at bf16); BALANCED is evaluated with a binary-counter stack, which visits
 // exactly the aligned pairs of the level-by-level definition.
-template <bool PART_BF16, bool MERGE_BF16>
+template <bool PART_16, bool MERGE_16>
 __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) {
   const int64_t ncol4 = (p.N + 3) / 4;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -627,16 +629,20 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
   const int64_t part_stride = (int64_t)p.M * p.ldw;
   const int64_t off = row * p.ldw + col0;
   auto load = [&](int s) -> float4 {
-    if (PART_BF16) {
+    if (PART_16) {
       const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.ws) + s * part_stride + off);
+      if (p.partial_dtype == RG_F16)
+        return make_float4(f16_bits_to_f32(w.x & 0xffffu), f16_bits_to_f32(w.x >> 16),
+                           f16_bits_to_f32(w.y & 0xffffu), f16_bits_to_f32(w.y >> 16));
       return make_float4(bf16_bits_to_f32(w.x & 0xffffu), bf16_bits_to_f32(w.x >> 16),
                          bf16_bits_to_f32(w.y & 0xffffu), bf16_bits_to_f32(w.y >> 16));
     }
     return *reinterpret_cast<const float4*>(static_cast<const float*>(p.ws) + s * part_stride + off);
   };
-  auto add1 = [](float a, float b) -> float {
+  const int merge_dtype = p.merge_dtype;
+  auto add1 = [merge_dtype](float a, float b) -> float {
     const float v = f_add(a, b);
-    return MERGE_BF16 ? __bfloat162float(__float2bfloat16_rn(v)) : v;
+    return MERGE_16 ? round_through(v, merge_dtype) : v;
   };
   auto add4 = [&](const float4& a, const float4& b) -> float4 {
     return make_float4(add1(a.x, b.x), add1(a.y, b.y), add1(a.z, b.z), add1(a.w, b.w));
@@ -665,9 +671,7 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     if (col0 + c < p.N) {
-      const float o = apply_epilogue(v[c], p.epi, row, col0 + c);
-      if (p.c_dtype == RG_BF16) static_cast<__nv_bfloat16*>(p.C)[row * p.ldc + col0 + c] = __float2bfloat16_rn(o);
-      else static_cast<float*>(p.C)[row * p.ldc + col0 + c] = o;
+      store_scalar(p.C, p.c_dtype, row * p.ldc + col0 + c, apply_epilogue(v[c], p.epi, row, col0 + c));
     }
   }
 }
@@ -691,16 +695,16 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// 2-D bf16 tensor map over a row-major [rows, cols] matrix: box = 64 columns x box_rows rows,
+// 2-D tensor map (bf16 or fp16 elements) over a row-major [rows, cols] matrix: box = 64 columns x box_rows rows,
 // 128-byte swizzle, zero fill outside the matrix (missing products are then exact zeros).
-bool make_tmap(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+bool make_tmap(CUtensorMap* map, const void* ptr, int dtype, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
   const cuuint32_t box[2] = {(cuuint32_t)KBOX, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+  return fn(map, dtype == RG_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -784,7 +788,8 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   const int tile_m = pair ? 2 * BM : BM;
   CUtensorMap ta, tb;
   const int a_rows = pair ? BM : a_box_rows_for(M);
-  if (!make_tmap(&ta, A->ptr, M, K, A->ld, a_rows) || !make_tmap(&tb, B->ptr, N, K, B->ld, pair ? plan.BN / 2 : plan.BN))
+  if (!make_tmap(&ta, A->ptr, A->dtype, M, K, A->ld, a_rows) ||
+      !make_tmap(&tb, B->ptr, B->dtype, N, K, B->ld, pair ? plan.BN / 2 : plan.BN))
     return RG_ERR_CUDA;
 
   GemmParams p;
@@ -797,7 +802,7 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   p.group_m = plan.group_m;
   p.a_box_bytes = (uint32_t)a_rows * KBOX * 2;
   p.bn = plan.BN;
-  p.idesc = make_idesc(plan.BN);
+  p.idesc = make_idesc(plan.BN, pair ? 2 * BM : BM, A->dtype == RG_F16 ? 0u : 1u);
   { uint32_t c = 32; while (c < 2u * (uint32_t)((plan.BN + 31) / 32 * 32)) c <<= 1; p.tmem_cols = c; }
   for (int s = 0; s < plan.n_parts; ++s) { p.part_begin[s] = plan.part_begin[s]; p.part_end[s] = plan.part_end[s]; }
   EpilogueArgs e{};
@@ -852,7 +857,7 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t fe;
-    if (plan.partial_dtype == RG_F32) fe = cudaLaunchKernelEx(&cfg, splitk_fixup_kernel<false, false>, f);
+    if (plan.partial_dtype == RG_F32) fe = cudaLaunchKernelEx(&cfg, splitk_fixup_kernel<false, false>, f);   // fp32 parts, fp32 sum
     else if (plan.merge_dtype == RG_F32) fe = cudaLaunchKernelEx(&cfg, splitk_fixup_kernel<true, false>, f);
     else fe = cudaLaunchKernelEx(&cfg, splitk_fixup_kernel<true, true>, f);
     if (fe != cudaSuccess) return RG_ERR_CUDA;

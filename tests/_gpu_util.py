@@ -15,11 +15,13 @@ def gpu_gemm(A, B, *, out_dtype=rgo.BF16, bias=None, act=0, residual=None, poiso
     At = A if torch.is_tensor(A) else synth.to_torch(A, DEV)
     Bt = B if torch.is_tensor(B) else synth.to_torch(B, DEV)
     M, N = At.shape[0], Bt.shape[0]
+    if At.dtype == torch.float16:
+        desc_kw.setdefault("in_dtype", rg.RG_F16)
     d = rg.rg_desc(**desc_kw)
-    tdt = torch.bfloat16 if out_dtype == rgo.BF16 else torch.float32
+    tdt = {rgo.BF16: torch.bfloat16, rgo.F32: torch.float32, rgo.F16: torch.float16}[out_dtype]
     Ct = torch.empty((M, N), dtype=tdt, device=DEV)
     if poison and Ct.numel():
-        Ct.view(torch.int16 if out_dtype == rgo.BF16 else torch.int32).fill_(-1)   # NaN pattern: unwritten elements show
+        Ct.view(torch.int32 if out_dtype == rgo.F32 else torch.int16).fill_(-1)   # NaN pattern: unwritten elements show
     nb = rg.rg_gemm_workspace_bytes(d, M, N)
     ws = None
     if nb:
@@ -48,7 +50,7 @@ def gpu_reduce(op, x, *, weight=None, eps=0.0, out_dtype=None, **desc_kw):
 
 
 def bits(a: np.ndarray) -> np.ndarray:
-    return a.view(np.uint32) if a.dtype == np.float32 else a.view(np.uint16)
+    return a.view(np.uint32) if a.dtype == np.float32 else a.view(np.uint16)   # uint16 and float16 alike
 
 
 def assert_bits_equal(got, want, what=""):

@@ -97,6 +97,8 @@ def test_argument_errors_are_reported_before_any_launch():
     assert call(d, A, _t(0x2000, K.RG_BF16, 8, 32), Cm) == 4                       # K disagrees
     assert call(d, A, B, _t(0x3000, K.RG_BF16, 4, 9)) == 4
     assert call(d, _t(0x1000, K.RG_F32, 4, 64), B, Cm) == 3                        # fp32 operands
+    assert call(d, _t(0x1000, K.RG_F16, 4, 64), _t(0x2000, K.RG_F16, 8, 64), Cm) == 4   # fp16 operands, bf16 descriptor
+    assert call(d, _t(0x1000, K.RG_F16, 4, 64), B, Cm) == 3                        # mixed operand types
     assert call(d, _t(0x1008, K.RG_BF16, 4, 64), B, Cm) == 5                       # 16-byte rule
     assert call(d, _t(0x1000, K.RG_BF16, 4, 60, 60), _t(0x2000, K.RG_BF16, 8, 60, 60), Cm) == 5   # ld % 8
     assert call(d, _t(0x1000, K.RG_BF16, 4, 0), _t(0x2000, K.RG_BF16, 8, 0), Cm) == 4            # K = 0

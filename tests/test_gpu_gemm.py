@@ -299,3 +299,45 @@ def test_partial_and_merge_dtypes_bit_exact(pd, md, tree):
     # the three combinations are three classes
     keys = {rg.rg_desc_class(rg.rg_desc(cuts=(256,), partial_dtype=p_, merge_dtype=m_)) for p_, m_ in ((1, 1), (0, 1), (0, 0))}
     assert len(keys) == 3
+
+
+# ------------------------------------------------------------------ fp16 operands
+def _f16_draws(M, N, K, seed):
+    g = np.random.default_rng(seed)
+    A = g.standard_normal((M, K)); B = g.standard_normal((N, K))
+    yield "ordinary", A.astype(np.float16), B.astype(np.float16)
+    yield "spread", (A * np.exp2(g.integers(-6, 7, A.shape))).astype(np.float16), (B * np.exp2(g.integers(-6, 7, B.shape))).astype(np.float16)
+
+
+def test_fp16_integer_inputs_exact_and_fp16_output():
+    g = np.random.default_rng(1)
+    for M, N, K in ((1, 8, 16), (129, 65, 80), (300, 520, 1000), (513, 260, 2048)):
+        A = g.integers(-8, 9, (M, K)).astype(np.float16); B = g.integers(-8, 9, (N, K)).astype(np.float16)
+        want = (A.astype(np.int64) @ B.astype(np.int64).T).astype(np.float32)
+        for knobs in (dict(), dict(cta_group=2, BN=128), dict(BN=48, cta_group=1)):
+            assert_bits_equal(gpu_gemm(A, B, out_dtype=rgo.F32, **knobs), want, f"fp16 ints {M}x{N}x{K} {knobs}")
+        assert_bits_equal(gpu_gemm(A, B, out_dtype=rgo.F16), rgo.gemm(A, B, atom_model=HW, out_dtype=rgo.F16), "fp16 output")
+
+
+@pytest.mark.parametrize("M,N,K,cuts", [(100, 96, 64, ()), (64, 128, 4096, ()), (40, 72, 2048, (512, 1024, 1536)), (300, 260, 1024, (256,))])
+def test_fp16_random_inputs_bit_exact_under_fitted_atom_model(M, N, K, cuts):
+    for name, A, B in _f16_draws(M, N, K, 70 + K):
+        want = rgo.gemm(A, B, cuts=cuts, atom_model=HW, out_dtype=rgo.F32)
+        for knobs in (dict(), dict(cta_group=2, BN=256), dict(BN=112, cta_group=1)):
+            assert_bits_equal(gpu_gemm(A, B, cuts=cuts, out_dtype=rgo.F32, **knobs), want, f"fp16 {M}x{N}x{K} {name} {knobs}")
+
+
+def test_fp16_split_partials_epilogue_and_class():
+    A, B = next(_f16_draws(70, 200, 1024, 5))[1:]
+    cuts = (256, 512, 768)
+    bias = np.random.default_rng(2).uniform(-0.1, 0.1, 200).astype(np.float16)
+    res = np.random.default_rng(3).standard_normal((70, 200)).astype(np.float16)
+    for pd, md in ((rgo.F32, rgo.F32), (rgo.F16, rgo.F32), (rgo.F16, rgo.F16), (rgo.BF16, rgo.BF16)):
+        for out in (rgo.F16, rgo.F32):
+            got = gpu_gemm(A, B, cuts=cuts, partial_dtype=pd, merge_dtype=md, bias=bias, act=1, residual=res, out_dtype=out)
+            want = rgo.gemm(A, B, cuts=cuts, atom_model=HW, partial_dtype=pd, merge_dtype=md, bias=bias, act=1, residual=res, out_dtype=out)
+            assert_bits_equal(got, want, f"fp16 split partial={pd} merge={md} out={out}")
+    assert rg.rg_desc_class(rg.rg_desc(in_dtype=rg.RG_F16)) != rg.rg_desc_class(rg.rg_desc())
+    # operands must be of the descriptor's input type
+    with pytest.raises(rg.RgError):
+        rg.rg_gemm(rg.rg_desc(), synth.to_torch(A, DEV), synth.to_torch(B, DEV), torch.empty((70, 200), dtype=torch.float16, device=DEV))

@@ -294,3 +294,39 @@ def test_partial_and_merge_dtypes():
     for pd, md in ((rgo.F32, rgo.F32), (rgo.BF16, rgo.F32), (rgo.BF16, rgo.BF16)):
         got = rgo.gemm(Ai, Bi, cuts=(16, 32, 48), out_dtype=rgo.F32, partial_dtype=pd, merge_dtype=md)
         assert np.array_equal(got, exact)
+
+
+# ---- fp16 operands (the paper's headline input type): same pins, another operand decode
+def _f16(x):
+    return np.asarray(x, np.float32).astype(np.float16)
+
+
+def test_fp16_integer_products_and_closed_forms():
+    g = np.random.default_rng(0)
+    for K, cuts in ((512, (256,)), (1000, ()), (72, (16, 48))):
+        A = _f16(g.integers(-8, 9, (5, K))); B = _f16(g.integers(-8, 9, (7, K)))
+        want = (A.astype(np.int64) @ B.astype(np.int64).T).astype(np.float32)
+        for name, m in MODELS.items():
+            got = rgo.gemm(A, B, cuts=cuts, atom_model=m, out_dtype=rgo.F32)
+            assert np.array_equal(got, want), (name, K)
+    ones = _f16(np.ones((3, 4096)))
+    assert np.all(rgo.gemm(ones, ones, atom_model=rgo.EXACT_RN, out_dtype=rgo.F32) == np.float32(4096))
+    # fp16 output: one rounding to binary16 (2049 is not representable: ties to even 2048)
+    assert np.all(rgo.gemm(_f16(np.ones((2, 2049))), _f16(np.ones((2, 2049))), out_dtype=rgo.F16) == np.float16(2048))
+
+
+@pytest.mark.parametrize("spread", [2, 8, 14])
+def test_fp16_exact_atom_against_rationals(spread):
+    g = np.random.default_rng(100 + spread)
+    for trial in range(300):
+        n = int(g.integers(1, 17))
+        a = _f16(g.standard_normal(n) * np.exp2(g.integers(-spread, spread + 1, n)))
+        b = _f16(g.standard_normal(n) * np.exp2(g.integers(-spread, spread + 1, n)))
+        acc = np.float32(g.standard_normal() * 2.0 ** int(g.integers(-spread, spread + 1)))
+        exact = Fraction(float(acc)) + sum(Fraction(float(x)) * Fraction(float(y)) for x, y in zip(a, b))
+        assert rgo.atom(rgo.EXACT_RN, acc, a, b) == _rn_f32(exact)
+        if n == 1:
+            assert rgo.atom(rgo.EXACT_RN, acc, a, b) == rgo.atom(rgo.SEQ_FMA, acc, a, b)
+    # fp16 subnormal operands take part exactly
+    a = np.array([2.0 ** -24, 2.0 ** -20], np.float16); b = np.array([1.0, 2.0 ** -4], np.float16)
+    assert rgo.atom(rgo.EXACT_RN, 0.0, a, b) == np.float32(2.0 ** -24 + 2.0 ** -24)

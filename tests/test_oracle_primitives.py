@@ -96,3 +96,29 @@ def test_silu():
         assert _ulp_err(float(rgo.silu(x)), want) <= 4.0
     assert rgo.silu(-200.0) == np.float32(-0.0)  # x / inf
     assert rgo.silu(200.0) == np.float32(200.0)
+
+
+def test_f16_widening_exhaustive():
+    allbits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    want = allbits.view(np.float16).astype(np.float32)
+    got = np.array([rgo.lib().rgo_f16_to_f32(int(h)) for h in allbits], dtype=np.float32)
+    nan = np.isnan(want)
+    assert np.array_equal(got[~nan].view(np.uint32), want[~nan].view(np.uint32)) and np.all(np.isnan(got[nan]))
+
+
+def test_f16_narrowing_matches_library_rne():
+    g = np.random.default_rng(2)
+    x = (g.standard_normal(200000) * np.exp2(g.integers(-30, 18, 200000))).astype(np.float32)
+    h = g.integers(0, 0x7bff, 30000).astype(np.uint16)                       # exact ties between neighbours
+    lo = h.view(np.float16).astype(np.float64); hi = (h + 1).astype(np.uint16).view(np.float16).astype(np.float64)
+    ties = ((lo + hi) / 2).astype(np.float32)
+    near = np.concatenate([np.nextafter(ties, np.float32(np.inf)), np.nextafter(ties, np.float32(-np.inf))])
+    edge = np.array([65504, 65519.99, 65520, 65536, 1e9, 2.0 ** -24, 2.0 ** -25, 2.0 ** -25 * 1.0001, 2.0 ** -26, 0.0, -0.0,
+                     6.1e-5, 6.097e-5, np.inf], dtype=np.float32)
+    x = np.concatenate([x, ties, -ties, near, edge, -edge])
+    with np.errstate(over="ignore"):
+        want = x.astype(np.float16).view(np.uint16)
+    got = np.array([rgo.f32_to_f16(v) for v in x], dtype=np.uint16)
+    assert np.array_equal(got, want)
+    for h16 in range(0, 0x7c00):                                            # round trip of every finite pattern
+        assert rgo.f32_to_f16(np.uint16(h16).view(np.float16).astype(np.float32)) == h16
