@@ -86,6 +86,16 @@ __device__ __forceinline__ float exp_nonpositive(float d) {
 // FULL: all V columns exist.  Otherwise `nvalid` leading ones do; the rest are -0.0f.
 template <int OP, int V, bool FULL>
 __device__ __forceinline__ float fold_block(const float (&x)[V], int nvalid, float shift, int fma) {
+  if (OP == OP_SOFTMAX) {
+    // exp(x - m) is exactly +0 below the library's underflow threshold.  When that holds for every
+    // leaf this warp is folding, the block's sum is a sum of zeros and the polynomial is skipped
+    // (a warp-uniform branch; called from warp-uniform control flow only).  Same bits, less work:
+    // with wide-ranged logits most of a row lies that far below its maximum.
+    bool live = false;
+#pragma unroll
+    for (int t = 0; t < V; ++t) live |= (FULL || t < nvalid) && !(f_add(x[t], -shift) < -87.33655f);
+    if (!__any_sync(0xffffffffu, live)) return (FULL || nvalid > 0) ? 0.0f : NEG_ZERO;
+  }
   float n[V / 2];
 #pragma unroll
   for (int t = 0; t < V / 2; ++t) {
