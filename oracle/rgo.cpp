@@ -433,6 +433,7 @@ struct GemmDesc {
   int32_t out_dtype;
   int32_t partial_dtype;   // type a finished part is written at (fp32 or bf16)
   int32_t merge_dtype;     // type the running sum of the parts is kept at
+  int64_t inner_span;      // second level of the cut nest: 0 = none, else an accumulator is closed every inner_span k
 };
 
 // One output element, Sec. 3.2.2.  `partials_out` (nullable) receives the
@@ -444,11 +445,24 @@ float gemm_element(const GemmDesc& d, const uint16_t* arow, const uint16_t* brow
   for (int s = 0; s < S; ++s) {
     int64_t k_lo = s == 0 ? 0 : d.cuts[s - 1];
     int64_t k_hi = s == S - 1 ? K : d.cuts[s];
-    float acc = 0.0f;                                   // every part starts from zero
     int ak = d.atom.model == ATOM_SEQ ? 1 : d.atom.atom_k;
-    for (int64_t k0 = k_lo; k0 < k_hi; k0 += ak) {      // ascending k, atoms relative to the part
-      int n = int(std::min<int64_t>(ak, k_hi - k0));
-      acc = atom_step(acc, arow + k0, brow + k0, n, d.atom);
+    // Sec. 3.2.2: "some kernels cut again inside a part, closing an accumulator every so many
+    // elements before the part is finished".  Each group of inner_span k runs its own chain from a
+    // zero accumulator; the closed groups are added at fp32, in ascending order, into the part's
+    // running sum (the first group starts it): one extra rounding per group (App. E, per-group
+    // accumulation).
+    const int64_t span = d.inner_span > 0 ? d.inner_span : (k_hi - k_lo);
+    float acc = 0.0f;
+    bool first_group = true;
+    for (int64_t g_lo = k_lo; g_lo < k_hi; g_lo += span) {
+      const int64_t g_hi = std::min(k_hi, g_lo + span);
+      float gacc = 0.0f;                                // every group starts from zero
+      for (int64_t k0 = g_lo; k0 < g_hi; k0 += ak) {    // ascending k, atoms relative to the group
+        int n = int(std::min<int64_t>(ak, g_hi - k0));
+        gacc = atom_step(gacc, arow + k0, brow + k0, n, d.atom);
+      }
+      acc = first_group ? gacc : acc + gacc;
+      first_group = false;
     }
     part[s] = round_to(acc, d.partial_dtype);           // the finished part, at partial_dtype
     if (partials_out) partials_out[s] = part[s];
@@ -500,8 +514,8 @@ void rgo_gemm(const AtomModel* atom, int tree, int n_cuts, const int64_t* cuts,
               const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
               void* C, int out_dtype, int64_t ldc,
               const void* bias, int bias_dtype, int act,
-              const void* residual, int residual_dtype, int64_t ldr, int partial_dtype, int merge_dtype) {
-  GemmDesc d{*atom, tree, n_cuts, cuts, bias, bias_dtype, act, residual, residual_dtype, ldr, out_dtype, partial_dtype, merge_dtype};
+              const void* residual, int residual_dtype, int64_t ldr, int partial_dtype, int merge_dtype, int64_t inner_span) {
+  GemmDesc d{*atom, tree, n_cuts, cuts, bias, bias_dtype, act, residual, residual_dtype, ldr, out_dtype, partial_dtype, merge_dtype, inner_span};
 #pragma omp parallel for collapse(2) schedule(static)
   for (int64_t i = 0; i < M; ++i)
     for (int64_t j = 0; j < N; ++j) {
@@ -518,8 +532,8 @@ void rgo_gemm_samples(const AtomModel* atom, int tree, int n_cuts, const int64_t
                       const void* bias, int bias_dtype, int act,
                       const void* residual, int residual_dtype, int64_t ldr,
                       int64_t n_samples, const int64_t* si, const int64_t* sj, float* out,
-                      int partial_dtype, int merge_dtype) {
-  GemmDesc d{*atom, tree, n_cuts, cuts, bias, bias_dtype, act, residual, residual_dtype, ldr, out_dtype, partial_dtype, merge_dtype};
+                      int partial_dtype, int merge_dtype, int64_t inner_span) {
+  GemmDesc d{*atom, tree, n_cuts, cuts, bias, bias_dtype, act, residual, residual_dtype, ldr, out_dtype, partial_dtype, merge_dtype, inner_span};
 #pragma omp parallel for schedule(static)
   for (int64_t t = 0; t < n_samples; ++t) {
     float v = gemm_element(d, A + si[t] * lda, B + sj[t] * ldb, K, si[t], sj[t], nullptr);
@@ -530,8 +544,8 @@ void rgo_gemm_samples(const AtomModel* atom, int tree, int n_cuts, const int64_t
 // Partials of every part, [S][M][N], before the merge (fp32 holding the value at partial_dtype).
 void rgo_gemm_partials(const AtomModel* atom, int n_cuts, const int64_t* cuts,
                        int64_t M, int64_t N, int64_t K,
-                       const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb, float* P, int partial_dtype) {
-  GemmDesc d{*atom, TREE_LEFT, n_cuts, cuts, nullptr, 0, 0, nullptr, 0, 0, DT_F32, partial_dtype, DT_F32};
+                       const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb, float* P, int partial_dtype, int64_t inner_span) {
+  GemmDesc d{*atom, TREE_LEFT, n_cuts, cuts, nullptr, 0, 0, nullptr, 0, 0, DT_F32, partial_dtype, DT_F32, inner_span};
   int S = n_cuts + 1;
 #pragma omp parallel for collapse(2) schedule(static)
   for (int64_t i = 0; i < M; ++i)

@@ -98,12 +98,12 @@ def lib():
         L.rgo_atom.restype = f32; L.rgo_atom.argtypes = [C.POINTER(_AtomStruct), f32, vp, vp, i32]
         L.rgo_gemm.restype = None
         L.rgo_gemm.argtypes = [C.POINTER(_AtomStruct), i32, i32, vp, i64, i64, i64, vp, i64, vp, i64,
-                               vp, i32, i64, vp, i32, i32, vp, i32, i64, i32, i32]
+                               vp, i32, i64, vp, i32, i32, vp, i32, i64, i32, i32, i64]
         L.rgo_gemm_samples.restype = None
         L.rgo_gemm_samples.argtypes = [C.POINTER(_AtomStruct), i32, i32, vp, i64, vp, i64, vp, i64,
-                                       i32, vp, i32, i32, vp, i32, i64, i64, vp, vp, vp, i32, i32]
+                                       i32, vp, i32, i32, vp, i32, i64, i64, vp, vp, vp, i32, i32, i64]
         L.rgo_gemm_partials.restype = None
-        L.rgo_gemm_partials.argtypes = [C.POINTER(_AtomStruct), i32, vp, i64, i64, i64, vp, i64, vp, i64, vp, i32]
+        L.rgo_gemm_partials.argtypes = [C.POINTER(_AtomStruct), i32, vp, i64, i64, i64, vp, i64, vp, i64, vp, i32, i64]
         L.rgo_reduce_rows.restype = None
         L.rgo_reduce_rows.argtypes = [i32, i32, i32, vp, i32, i64, i64, i64, vp, i32, i64, vp, i32, f32, vp]
         _lib = L
@@ -201,11 +201,12 @@ def _epi(bias, residual):
 
 
 def gemm(A, B, *, cuts=(), tree=TREE_BALANCED, atom_model: AtomModel = EXACT_RN, out_dtype=BF16,
-         bias=None, act=0, residual=None, partial_dtype=F32, merge_dtype=F32) -> np.ndarray:
+         bias=None, act=0, residual=None, partial_dtype=F32, merge_dtype=F32, inner_span=0) -> np.ndarray:
     """C = epilogue(A @ B.T) per the descriptor semantics (Sec. 3.2.2).
     A [M,K], B [N,K] are uint16 bf16 bit patterns.  Returns uint16 (bf16) or float32.
     partial_dtype / merge_dtype: the type a finished split-K part is written at and the type the
-    running sum of the parts is kept at."""
+    running sum of the parts is kept at.  inner_span: second level of the cut nest (0 = none): inside a
+    part an accumulator is closed every inner_span k and added at fp32 to the part's running sum."""
     A, B, atom_model = _operands(A, B, atom_model)
     M, K = A.shape; N, K2 = B.shape
     assert K == K2
@@ -214,12 +215,12 @@ def gemm(A, B, *, cuts=(), tree=TREE_BALANCED, atom_model: AtomModel = EXACT_RN,
     b, bd, r, rd, ldr = _epi(bias, residual)
     m = atom_model.c()
     lib().rgo_gemm(C.byref(m), tree, c.size, _ptr(c), M, N, K, _ptr(A), K, _ptr(B), K,
-                   _ptr(out), out_dtype, N, _ptr(b), bd, act, _ptr(r), rd, ldr, partial_dtype, merge_dtype)
+                   _ptr(out), out_dtype, N, _ptr(b), bd, act, _ptr(r), rd, ldr, partial_dtype, merge_dtype, inner_span)
     return out
 
 
 def gemm_samples(A, B, si, sj, *, cuts=(), tree=TREE_BALANCED, atom_model: AtomModel = EXACT_RN,
-                 out_dtype=BF16, bias=None, act=0, residual=None, partial_dtype=F32, merge_dtype=F32) -> np.ndarray:
+                 out_dtype=BF16, bias=None, act=0, residual=None, partial_dtype=F32, merge_dtype=F32, inner_span=0) -> np.ndarray:
     """Output elements (si[t], sj[t]) only; returned as float32 after the output rounding."""
     A, B, atom_model = _operands(A, B, atom_model)
     K = A.shape[1]
@@ -230,18 +231,18 @@ def gemm_samples(A, B, si, sj, *, cuts=(), tree=TREE_BALANCED, atom_model: AtomM
     m = atom_model.c()
     lib().rgo_gemm_samples(C.byref(m), tree, c.size, _ptr(c), K, _ptr(A), K, _ptr(B), K, out_dtype,
                            _ptr(b), bd, act, _ptr(r), rd, ldr, si.size, _ptr(si), _ptr(sj), _ptr(out),
-                           partial_dtype, merge_dtype)
+                           partial_dtype, merge_dtype, inner_span)
     return out
 
 
-def gemm_partials(A, B, *, cuts=(), atom_model: AtomModel = EXACT_RN, partial_dtype=F32) -> np.ndarray:
+def gemm_partials(A, B, *, cuts=(), atom_model: AtomModel = EXACT_RN, partial_dtype=F32, inner_span=0) -> np.ndarray:
     """The partial of every part, shape [S, M, N], as fp32 values at partial_dtype (Sec. 3.2.2, split-K)."""
     A, B, atom_model = _operands(A, B, atom_model)
     M, K = A.shape; N = B.shape[0]
     c = _cuts(cuts)
     P = np.empty((c.size + 1, M, N), dtype=np.float32)
     m = atom_model.c()
-    lib().rgo_gemm_partials(C.byref(m), c.size, _ptr(c), M, N, K, _ptr(A), K, _ptr(B), K, _ptr(P), partial_dtype)
+    lib().rgo_gemm_partials(C.byref(m), c.size, _ptr(c), M, N, K, _ptr(A), K, _ptr(B), K, _ptr(P), partial_dtype, inner_span)
     return P
 
 

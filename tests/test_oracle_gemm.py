@@ -330,3 +330,32 @@ def test_fp16_exact_atom_against_rationals(spread):
     # fp16 subnormal operands take part exactly
     a = np.array([2.0 ** -24, 2.0 ** -20], np.float16); b = np.array([1.0, 2.0 ** -4], np.float16)
     assert rgo.atom(rgo.EXACT_RN, 0.0, a, b) == np.float32(2.0 ** -24 + 2.0 ** -24)
+
+
+# ---- second level of the cut nest (Sec. 3.2.2 k_cuts; App. E per-group accumulation)
+def test_inner_span_worked_example_and_closed_forms():
+    """k=0: 1; k=32 and k=48: 2^-24 each (different 16-wide steps).  One chain: 1 + 2^-24 ties back to 1,
+    twice.  Closed every 32: the second group holds 2^-24 + 2^-24 = 2^-23 and 1 + 2^-23 is exact.
+    Closed every 16: each 2^-24 meets the running sum alone and is lost again."""
+    a = np.zeros((1, 96), np.float32); a[0, 0] = 1.0; a[0, 32] = 2.0 ** -24; a[0, 48] = 2.0 ** -24
+    ones = _bf(np.ones((1, 96), np.float32))
+    for m in (rgo.EXACT_RN, rgo.TCGEN05_BF16_B200):
+        assert rgo.gemm(_bf(a), ones, atom_model=m, out_dtype=rgo.F32)[0, 0] == np.float32(1.0)
+        assert rgo.gemm(_bf(a), ones, atom_model=m, out_dtype=rgo.F32, inner_span=32)[0, 0] == np.float32(1 + 2.0 ** -23)
+        assert rgo.gemm(_bf(a), ones, atom_model=m, out_dtype=rgo.F32, inner_span=16)[0, 0] == np.float32(1.0)
+        assert rgo.gemm(_bf(a), ones, atom_model=m, out_dtype=rgo.F32, inner_span=96)[0, 0] == np.float32(1.0)   # one group = no cut
+    # integers are exact under any nest; a span that does not divide the part leaves a short last group
+    A = synth.int_valued_bf16((4, 1000), -8, 8, 1); B = synth.int_valued_bf16((5, 1000), -8, 8, 2)
+    want = (synth.bf16_bits_to_f32(A).astype(np.int64) @ synth.bf16_bits_to_f32(B).astype(np.int64).T).astype(np.float32)
+    for span in (16, 64, 128, 448):
+        for cuts in ((), (512,)):
+            assert np.array_equal(rgo.gemm(A, B, cuts=cuts, inner_span=span, out_dtype=rgo.F32), want)
+    # the groups restart inside every part: a part equals the unsplit GEMM of its own K range under the same nest
+    A = synth.normal_bf16((3, 512), 1.0, 3); B = synth.normal_bf16((4, 512), 1.0, 4)
+    P = rgo.gemm_partials(A, B, cuts=(192,), inner_span=128)
+    assert np.array_equal(P[1], rgo.gemm(A[:, 192:], B[:, 192:], inner_span=128, out_dtype=rgo.F32))
+    # and the nest is visible on ordinary inputs
+    assert not np.array_equal(rgo.gemm(A, B, out_dtype=rgo.F32), rgo.gemm(A, B, inner_span=64, out_dtype=rgo.F32))
+    # group sums against the definition: chain of group results, each an unsplit GEMM of its own range
+    g = [rgo.gemm(A[:, k:k + 128], B[:, k:k + 128], out_dtype=rgo.F32) for k in range(0, 512, 128)]
+    assert np.array_equal(rgo.gemm(A, B, inner_span=128, out_dtype=rgo.F32), ((g[0] + g[1]) + g[2]) + g[3])
