@@ -79,6 +79,10 @@ typedef struct {
   uint8_t tree;           /* rg_tree_t */
   uint32_t n_cuts;        /* split-K: number of interior cut points (0 = plain GEMM) */
   uint32_t cuts[RG_MAX_CUTS]; /* 0 < cuts[0] < ... < cuts[n_cuts-1] < K; part s = [cuts[s-1], cuts[s]) */
+  uint32_t inner_span;    /* second level of the cut nest (Sec. 3.2.2; App. E per-group accumulation): 0 = none;
+                             else, inside every part, an accumulator is closed every inner_span k (a multiple
+                             of 64) and the closed groups are added at fp32, in ascending order, into the
+                             part's running sum.  Order-deciding: part of the class key. */
 } rg_desc_t;
 
 /* A row-major matrix in device memory. */

@@ -43,6 +43,13 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
   if (d->raster > 64) return RG_ERR_INVALID_DESC;
   for (uint32_t i = 0; i < d->n_cuts; ++i)
     if (d->cuts[i] % 16 != 0) return RG_ERR_UNSUPPORTED;   // a cut may not split a 16-wide step
+  if (d->inner_span) {
+    // groups are handed over per 64-wide K step by one CTA, with the running sum in registers
+    if (d->inner_span % 64 != 0) return RG_ERR_UNSUPPORTED;
+    if (d->cta_group == 2 || d->BM == 256 || d->BN > 128 || (d->BK != 0 && d->BK != 64)) return RG_ERR_UNSUPPORTED;
+    for (uint32_t i = 0; i < d->n_cuts; ++i)
+      if (d->cuts[i] % 64 != 0) return RG_ERR_UNSUPPORTED;
+  }
   return RG_OK;
 }
 
@@ -82,6 +89,7 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   plan->tree = d->tree;
   plan->partial_dtype = d->partial_dtype;
   plan->merge_dtype = d->merge_dtype;
+  plan->inner_span = (int)d->inner_span;
   for (int s = 0; s < plan->n_parts; ++s) {
     plan->part_begin[s] = s == 0 ? 0 : (int32_t)d->cuts[s - 1];
     plan->part_end[s] = s == plan->n_parts - 1 ? (int32_t)K : (int32_t)d->cuts[s];
@@ -107,15 +115,17 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
       if (tiles_m * ((N + bn - 1) / bn) * plan->n_parts >= sms) { plan->BN = bn; break; }
     }
   }
+  if (d->inner_span && plan->BN > 128) plan->BN = 128;
   // one CTA per 128-row tile, or a pair of CTAs (two SMs) per 256-row tile
-  if (d->cta_group) plan->cta_group = d->cta_group;
+  if (d->inner_span) plan->cta_group = 1;
+  else if (d->cta_group) plan->cta_group = d->cta_group;
   else if (d->BM == 256) plan->cta_group = 2;
   else if (d->BM == 128) plan->cta_group = 1;
   else plan->cta_group = (plan->BN >= 128 && M > 128 && ((M + 255) / 256) * ((N + plan->BN - 1) / plan->BN) * plan->n_parts >= sms / 2) ? 2 : 1;
   if (plan->cta_group == 2 && plan->BN < 128) plan->cta_group = 1;
   // a pair moves half the B bytes per CTA, so a 128-wide K step fits three times: fewer hand-offs per k
   // skinny problems read long runs of each weight row per stage (DRAM likes 512-byte bursts)
-  plan->BK = d->BK ? d->BK : ((plan->cta_group == 2 && plan->BN == 256) || skinny ? 128 : 64);
+  plan->BK = d->BK ? d->BK : (d->inner_span ? 64 : ((plan->cta_group == 2 && plan->BN == 256) || skinny ? 128 : 64));
   if (plan->cta_group == 2 && plan->BN != 128 && plan->BN != 256) return RG_ERR_UNSUPPORTED;
   const int smax = rg::max_stages_for(plan->BN, plan->BK, plan->cta_group, M);
   plan->stages = d->stages ? d->stages : smax;
@@ -148,7 +158,7 @@ rg_status_t rg_desc_validate(const rg_desc_t* d, int64_t M, int64_t N, int64_t K
 uint64_t rg_desc_class(const rg_desc_t* d) {
   if (check_desc_fields(d) != RG_OK) return 0;
   // canonical serialisation of the order-deciding fields only; "no cuts" has one spelling
-  uint8_t buf[12 + 4 * RG_MAX_CUTS];
+  uint8_t buf[16 + 4 * RG_MAX_CUTS];
   size_t n = 0;
   const uint8_t head[8] = {d->in_dtype, d->acc_dtype, d->partial_dtype, d->merge_dtype, d->atom, d->k_tail, d->fma, d->tree};
   memcpy(buf, head, 8); n = 8;
@@ -156,6 +166,7 @@ uint64_t rg_desc_class(const rg_desc_t* d) {
   for (int b = 0; b < 4; ++b) buf[n++] = (uint8_t)(nc >> (8 * b));
   for (uint32_t i = 0; i < nc; ++i)
     for (int b = 0; b < 4; ++b) buf[n++] = (uint8_t)(d->cuts[i] >> (8 * b));
+  for (int b = 0; b < 4; ++b) buf[n++] = (uint8_t)(d->inner_span >> (8 * b));
   uint64_t h = 0xcbf29ce484222325ull;                  // FNV-1a, 64 bit
   for (size_t i = 0; i < n; ++i) { h ^= buf[i]; h *= 0x100000001b3ull; }
   return h ? h : 1;

@@ -153,6 +153,7 @@ struct GemmParams {
   int32_t M, N, K;
   int32_t tiles_m, tiles_n, n_parts;
   int32_t num_stages, raster, group_m;
+  int32_t inner_span;     // second cut level: an accumulator is closed every inner_span k (0 = none; a multiple of the K step)
   int32_t bn;             // tile columns of the one-CTA kernel (any multiple of 16 up to 256)
   uint32_t idesc;         // instruction descriptor for N = bn
   uint32_t tmem_cols;     // tensor-memory columns allocated: two accumulators of tmem_cols / 2
@@ -239,9 +240,48 @@ __device__ __forceinline__ void store_row_segment(const GemmParams& p, int64_t r
   }
 }
 
+// One 32-column chunk of one output row, held as fp32 bit patterns in r: a split-K part goes to the
+// workspace rounded once to partial_dtype (untouched when that is fp32; Sec. 3.2.2); otherwise
+// bias / SiLU / residual and one rounding to the output type.
+__device__ __forceinline__ void epilogue_store_chunk(const GemmParams& p, int part, int64_t row, int col0, int ncols,
+                                                     const uint32_t (&r)[32]) {
+  if (p.ws && p.ws_dtype == RG_F32) {
+    float* dst = static_cast<float*>(p.ws) + ((int64_t)part * p.M + row) * p.ldw + col0;
+    if (ncols == 32) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        reinterpret_cast<uint4*>(dst)[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+    } else {
+#pragma unroll
+      for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __uint_as_float(r[c]);
+    }
+  } else if (p.ws) {
+    // the finished part written at a 16-bit type: one rounding of the fp32 accumulator
+    const int64_t off = ((int64_t)part * p.M + row) * p.ldw + col0;
+    uint16_t* dst = static_cast<uint16_t*>(p.ws) + off;
+    if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        reinterpret_cast<uint4*>(dst)[q] = make_uint4(
+            pack_16x2(__uint_as_float(r[8 * q]), __uint_as_float(r[8 * q + 1]), p.ws_dtype),
+            pack_16x2(__uint_as_float(r[8 * q + 2]), __uint_as_float(r[8 * q + 3]), p.ws_dtype),
+            pack_16x2(__uint_as_float(r[8 * q + 4]), __uint_as_float(r[8 * q + 5]), p.ws_dtype),
+            pack_16x2(__uint_as_float(r[8 * q + 6]), __uint_as_float(r[8 * q + 7]), p.ws_dtype));
+    } else {
+#pragma unroll
+      for (int c = 0; c < 32; ++c) if (c < ncols) store_scalar(p.ws, p.ws_dtype, off + c, __uint_as_float(r[c]));
+    }
+  } else {
+    float v[32];
+#pragma unroll
+    for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(r[c]);
+    epilogue_row_segment(v, p.epi, row, col0, ncols);
+    store_row_segment(p, row, col0, ncols, v);
+  }
+}
+
 // Epilogue of one accumulator tile for one warp: the warp's 32 TMEM lanes (one output row per
-// thread), 32-column chunks chunk0, chunk0+2, ...  Split-K parts go to the workspace at fp32,
-// untouched (Sec. 3.2.2); otherwise bias / SiLU / residual and one rounding to the output type.
+// thread), 32-column chunks chunk0, chunk0+2, ...
 __device__ __forceinline__ void epilogue_tile(const GemmParams& p, const int BN, int part, int64_t row, bool row_ok, int tn,
                                               uint32_t taddr, int chunk0) {
   const int col_end = min(p.N, (tn + 1) * BN);            // this tile's columns end here
@@ -252,42 +292,41 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, const int BN,
     uint32_t r[32];
     tmem_ld_32x32b_x32(taddr + c0, r);
     tmem_ld_wait();
-    const int ncols = min(32, col_end - col0);
-    if (row_ok) {
-      if (p.ws && p.ws_dtype == RG_F32) {
-        float* dst = static_cast<float*>(p.ws) + ((int64_t)part * p.M + row) * p.ldw + col0;
-        if (ncols == 32) {
+    if (row_ok) epilogue_store_chunk(p, part, row, col0, min(32, col_end - col0), r);
+  }
+}
+
+// Second cut level (Sec. 3.2.2 "some kernels cut again inside a part"; App. E per-group accumulation):
+// the MMA warp closes an accumulator every inner_span k; each epilogue warp adds every closed group,
+// at fp32 and in ascending order, into a running sum held in registers, then finishes the tile from
+// it.  Tiles are at most 128 columns wide in this mode, so a warp owns at most two 32-column chunks.
+struct GroupedAcc { uint32_t v[2][32]; };
+
+__device__ __forceinline__ void grouped_add(const GemmParams& p, const int BN, int tn, uint32_t taddr, int chunk0, bool first,
+                                            GroupedAcc& acc) {
+  const int col_end = min(p.N, (tn + 1) * BN);
 #pragma unroll
-          for (int q = 0; q < 8; ++q)
-            reinterpret_cast<uint4*>(dst)[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
-        } else {
+  for (int j = 0; j < 2; ++j) {
+    const int c0 = (chunk0 + 2 * j) * 32;
+    if (c0 < BN && tn * BN + c0 < col_end) {              // uniform across the warp
+      uint32_t r[32];
+      tmem_ld_32x32b_x32(taddr + c0, r);
+      tmem_ld_wait();
 #pragma unroll
-          for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __uint_as_float(r[c]);
-        }
-      } else if (p.ws) {
-        // the finished part written at a 16-bit type: one rounding of the fp32 accumulator
-        const int64_t off = ((int64_t)part * p.M + row) * p.ldw + col0;
-        uint16_t* dst = static_cast<uint16_t*>(p.ws) + off;
-        if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q)
-            reinterpret_cast<uint4*>(dst)[q] = make_uint4(
-                pack_16x2(__uint_as_float(r[8 * q]), __uint_as_float(r[8 * q + 1]), p.ws_dtype),
-                pack_16x2(__uint_as_float(r[8 * q + 2]), __uint_as_float(r[8 * q + 3]), p.ws_dtype),
-                pack_16x2(__uint_as_float(r[8 * q + 4]), __uint_as_float(r[8 * q + 5]), p.ws_dtype),
-                pack_16x2(__uint_as_float(r[8 * q + 6]), __uint_as_float(r[8 * q + 7]), p.ws_dtype));
-        } else {
-#pragma unroll
-          for (int c = 0; c < 32; ++c) if (c < ncols) store_scalar(p.ws, p.ws_dtype, off + c, __uint_as_float(r[c]));
-        }
-      } else {
-        float v[32];
-#pragma unroll
-        for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(r[c]);
-        epilogue_row_segment(v, p.epi, row, col0, ncols);
-        store_row_segment(p, row, col0, ncols, v);
-      }
+      for (int c = 0; c < 32; ++c)
+        acc.v[j][c] = first ? r[c] : __float_as_uint(f_add(__uint_as_float(acc.v[j][c]), __uint_as_float(r[c])));
     }
+  }
+}
+
+__device__ __forceinline__ void grouped_finish(const GemmParams& p, const int BN, int part, int64_t row, bool row_ok, int tn,
+                                               int chunk0, const GroupedAcc& acc) {
+  const int col_end = min(p.N, (tn + 1) * BN);
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int c0 = (chunk0 + 2 * j) * 32;
+    const int col0 = tn * BN + c0;
+    if (c0 < BN && col0 < col_end && row_ok) epilogue_store_chunk(p, part, row, col0, min(32, col_end - col0), acc.v[j]);
   }
 }
 
@@ -374,18 +413,26 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       bool alive = true;
-      int it = 0;
-      for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x, ++it) {
+      int gc = 0;                                         // accumulators handed to the epilogue so far
+      for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);
         const int k_begin = p.part_begin[part], k_end = p.part_end[part];
-        const int buf = it & 1;
-        const uint32_t acc_phase = (it >> 1) & 1;
-        if (!mbar_wait(bar_tempty + 8u * buf, acc_phase ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
-        tcgen05_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * ACC_STRIDE;
-        uint32_t accumulate = 0;                        // every part starts from a zero accumulator
+        // one accumulator per part, or one per group of inner_span k (a multiple of the K step)
+        const int span = p.inner_span > 0 ? p.inner_span : (k_end - k_begin);
+        int group_end = k_begin;
+        int buf = 0;
+        uint32_t d_tmem = 0, accumulate = 0;
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
+          if (k0 >= group_end) {
+            if (k0 > k_begin) { umma_commit(bar_tfull + 8u * buf); ++gc; }   // the previous group is complete
+            buf = gc & 1;
+            if (!mbar_wait(bar_tempty + 8u * buf, ((gc >> 1) & 1) ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
+            tcgen05_fence_after();
+            d_tmem = tmem_base + buf * ACC_STRIDE;
+            accumulate = 0;                              // every part and every group starts from zero
+            group_end = k0 + span;
+          }
           if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0x300u | stage)) { alive = false; break; }
           tcgen05_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
@@ -405,7 +452,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           umma_commit(bar_empty + 8u * stage);           // stage reusable once these steps have read it
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
-        if (alive) umma_commit(bar_tfull + 8u * buf);     // accumulator complete
+        if (alive) { umma_commit(bar_tfull + 8u * buf); ++gc; }   // last (or only) accumulator complete
       }
     }
   } else {
@@ -413,21 +460,38 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     const int quarter = warp & 3;                         // TMEM lanes [32*quarter, 32*quarter+32)
     const int chunk0 = (warp - 2) >> 2;                   // this warp takes chunks chunk0, chunk0+2, ...
     bool alive = true;
-    int it = 0;
-    for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x, ++it) {
+    int gc = 0;
+    for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
       int part, tm, tn;
       decode_work(p, w, part, tm, tn);
-      const int buf = it & 1;
-      const uint32_t acc_phase = (it >> 1) & 1;
-      if (!mbar_wait(bar_tfull + 8u * buf, acc_phase, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
-      tcgen05_fence_after();
       const int64_t row = (int64_t)tm * BM + quarter * 32 + lane;
       const bool row_ok = row < p.M;
-      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
-      epilogue_tile(p, BN, part, row, row_ok, tn, taddr, chunk0);
-      tcgen05_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
+      const int klen = p.part_end[part] - p.part_begin[part];
+      const int ngroups = p.inner_span > 0 ? (klen + p.inner_span - 1) / p.inner_span : 1;
+      if (ngroups == 1) {
+        const int buf = gc & 1;
+        if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
+        tcgen05_fence_after();
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
+        epilogue_tile(p, BN, part, row, row_ok, tn, taddr, chunk0);
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
+        ++gc;
+      } else {
+        GroupedAcc acc;
+        for (int g = 0; g < ngroups && alive; ++g, ++gc) {
+          const int buf = gc & 1;
+          if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
+          tcgen05_fence_after();
+          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
+          grouped_add(p, BN, tn, taddr, chunk0, g == 0, acc);
+          tcgen05_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
+        }
+        if (alive) grouped_finish(p, BN, part, row, row_ok, tn, chunk0, acc);
+      }
     }
   }
 
@@ -802,6 +866,7 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   p.group_m = plan.group_m;
   p.a_box_bytes = (uint32_t)a_rows * KBOX * 2;
   p.bn = plan.BN;
+  p.inner_span = plan.inner_span;
   p.idesc = make_idesc(plan.BN, pair ? 2 * BM : BM, A->dtype == RG_F16 ? 0u : 1u);
   { uint32_t c = 32; while (c < 2u * (uint32_t)((plan.BN + 31) / 32 * 32)) c <<= 1; p.tmem_cols = c; }
   for (int s = 0; s < plan.n_parts; ++s) { p.part_begin[s] = plan.part_begin[s]; p.part_end[s] = plan.part_end[s]; }

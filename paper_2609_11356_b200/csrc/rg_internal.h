@@ -12,6 +12,7 @@ struct GemmPlan {
   int BN, BK, stages, raster, group_m, cta_group;
   int n_parts, tree;
   int partial_dtype, merge_dtype;
+  int inner_span;
   int32_t part_begin[RG_MAX_CUTS + 1];
   int32_t part_end[RG_MAX_CUTS + 1];
 };

@@ -341,3 +341,29 @@ def test_fp16_split_partials_epilogue_and_class():
     # operands must be of the descriptor's input type
     with pytest.raises(rg.RgError):
         rg.rg_gemm(rg.rg_desc(), synth.to_torch(A, DEV), synth.to_torch(B, DEV), torch.empty((70, 200), dtype=torch.float16, device=DEV))
+
+
+# ------------------------------------------------------------------ second level of the cut nest
+def test_inner_span_groups_bit_exact():
+    """Sec. 3.2.2 / App. E: an accumulator closed every inner_span k, groups chained at fp32."""
+    a = np.zeros((1, 192), np.float32); a[0, 0] = 1.0; a[0, 64] = 2.0 ** -24; a[0, 80] = 2.0 ** -24
+    ones = synth.f32_to_bf16_bits(np.ones((8, 192), np.float32)); ab = synth.f32_to_bf16_bits(a)
+    assert gpu_gemm(ab, ones, out_dtype=rgo.F32)[0, 0] == np.float32(1.0)                       # one chain: both ties lost
+    assert gpu_gemm(ab, ones, out_dtype=rgo.F32, inner_span=64)[0, 0] == np.float32(1 + 2.0 ** -23)   # second group sums to 2^-23 first
+    for M, N, K, cuts in ((70, 200, 1024, ()), (300, 130, 1000, ()), (33, 260, 2048, (512, 1024, 1536)), (129, 64, 4096, (2048,))):
+        for name, A, B in _draws(M, N, K, 90 + K):
+            for span in (64, 128, 448):
+                for knobs in (dict(), dict(BN=64), dict(BN=112, stages=2)):
+                    got = gpu_gemm(A, B, cuts=cuts, inner_span=span, out_dtype=rgo.F32, **knobs)
+                    want = rgo.gemm(A, B, cuts=cuts, inner_span=span, atom_model=HW, out_dtype=rgo.F32)
+                    assert_bits_equal(got, want, f"{M}x{N}x{K} {name} span={span} {knobs}")
+    A = synth.int_valued_bf16((200, 1000), -8, 8, 1); B = synth.int_valued_bf16((300, 1000), -8, 8, 2)
+    assert_bits_equal(gpu_gemm(A, B, inner_span=128, out_dtype=rgo.F32), _exact_int(A, B), "ints under a nest")
+    bias = synth.uniform_bf16((300,), -0.1, 0.1, 3)
+    assert_bits_equal(gpu_gemm(A, B, inner_span=192, bias=bias, act=1), rgo.gemm(A, B, inner_span=192, atom_model=HW, bias=bias, act=1),
+                      "nest with fused epilogue")
+    k0 = rg.rg_desc_class(rg.rg_desc()); k1 = rg.rg_desc_class(rg.rg_desc(inner_span=64)); k2 = rg.rg_desc_class(rg.rg_desc(inner_span=128))
+    assert len({k0, k1, k2}) == 3
+    for bad in (dict(inner_span=48), dict(inner_span=64, cta_group=2), dict(inner_span=64, BN=256), dict(inner_span=64, BK=128)):
+        assert rg.rg_desc_validate(rg.rg_desc(**bad), 64, 256, 512) == 3
+    assert rg.rg_device_status() == 0
