@@ -83,9 +83,9 @@ __device__ __forceinline__ uint32_t pack_16x2(float lo, float hi, int dtype);
 // `n` (<= 32) consecutive elements starting at element index `idx` of a bf16 or fp32 array, widened
 // to fp32; entries past n are zero.  Uses 16-byte loads when the segment is full and aligned.
 __device__ __forceinline__ void load_row_segment(const void* base, int dtype, int64_t idx, int n, float (&out)[32]) {
-  if (dtype == RG_BF16 || dtype == RG_F16) {
+  // the type is tested once, outside the unrolled loops
+  if (dtype == RG_BF16) {
     const uint16_t* p = static_cast<const uint16_t*>(base) + idx;
-    const bool half = dtype == RG_F16;
     if (n == 32 && (reinterpret_cast<uintptr_t>(p) & 15) == 0) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
@@ -93,13 +93,30 @@ __device__ __forceinline__ void load_row_segment(const void* base, int dtype, in
         const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-          out[8 * q + 2 * t] = half ? f16_bits_to_f32(ww[t] & 0xffffu) : bf16_bits_to_f32(ww[t] & 0xffffu);
-          out[8 * q + 2 * t + 1] = half ? f16_bits_to_f32(ww[t] >> 16) : bf16_bits_to_f32(ww[t] >> 16);
+          out[8 * q + 2 * t] = bf16_bits_to_f32(ww[t] & 0xffffu);
+          out[8 * q + 2 * t + 1] = bf16_bits_to_f32(ww[t] >> 16);
         }
       }
     } else {
 #pragma unroll
-      for (int c = 0; c < 32; ++c) out[c] = c < n ? (half ? f16_bits_to_f32(p[c]) : bf16_bits_to_f32(p[c])) : 0.0f;
+      for (int c = 0; c < 32; ++c) out[c] = c < n ? bf16_bits_to_f32(p[c]) : 0.0f;
+    }
+  } else if (dtype == RG_F16) {
+    const uint16_t* p = static_cast<const uint16_t*>(base) + idx;
+    if (n == 32 && (reinterpret_cast<uintptr_t>(p) & 15) == 0) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 w = __ldg(reinterpret_cast<const uint4*>(p) + q);
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          out[8 * q + 2 * t] = f16_bits_to_f32(ww[t] & 0xffffu);
+          out[8 * q + 2 * t + 1] = f16_bits_to_f32(ww[t] >> 16);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < 32; ++c) out[c] = c < n ? f16_bits_to_f32(p[c]) : 0.0f;
     }
   } else {
     const float* p = static_cast<const float*>(base) + idx;

@@ -212,23 +212,11 @@ __device__ __forceinline__ void epilogue_row_segment(float (&v)[32], const Epilo
   }
 }
 
-// Store up to 32 consecutive columns of one output row, each value rounded once to the output type.
-__device__ __forceinline__ void store_row_segment(const GemmParams& p, int64_t row, int col0, int ncols, const float (&v)[32]) {
-  if (p.c_dtype == RG_BF16 || p.c_dtype == RG_F16) {
-    uint16_t* dst = static_cast<uint16_t*>(p.C) + row * p.ldc + col0;
-    if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint4 o = make_uint4(pack_16x2(v[8 * q], v[8 * q + 1], p.c_dtype), pack_16x2(v[8 * q + 2], v[8 * q + 3], p.c_dtype),
-                             pack_16x2(v[8 * q + 4], v[8 * q + 5], p.c_dtype), pack_16x2(v[8 * q + 6], v[8 * q + 7], p.c_dtype));
-        reinterpret_cast<uint4*>(dst)[q] = o;
-      }
-    } else {
-#pragma unroll
-      for (int c = 0; c < 32; ++c) if (c < ncols) store_scalar(p.C, p.c_dtype, row * p.ldc + col0 + c, v[c]);
-    }
-  } else {
-    float* dst = static_cast<float*>(p.C) + row * p.ldc + col0;
+// Store up to 32 consecutive columns of one row of a row-major matrix, each value rounded once to
+// `dtype`.  The type is tested once, outside the unrolled loops.
+__device__ __forceinline__ void store_row_values(void* base, int dtype, int64_t off, int ncols, const float (&v)[32]) {
+  if (dtype == RG_F32) {
+    float* dst = static_cast<float*>(base) + off;
     if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
 #pragma unroll
       for (int q = 0; q < 8; ++q)
@@ -236,6 +224,30 @@ __device__ __forceinline__ void store_row_segment(const GemmParams& p, int64_t r
     } else {
 #pragma unroll
       for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = v[c];
+    }
+    return;
+  }
+  uint16_t* dst = static_cast<uint16_t*>(base) + off;
+  const bool vec = ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0;
+  if (dtype == RG_BF16) {
+    if (vec) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        reinterpret_cast<uint4*>(dst)[q] = make_uint4(pack_bf16x2(v[8 * q], v[8 * q + 1]), pack_bf16x2(v[8 * q + 2], v[8 * q + 3]),
+                                                      pack_bf16x2(v[8 * q + 4], v[8 * q + 5]), pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
+    } else {
+#pragma unroll
+      for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __bfloat16_as_ushort(__float2bfloat16_rn(v[c]));
+    }
+  } else {
+    if (vec) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        reinterpret_cast<uint4*>(dst)[q] = make_uint4(pack_f16x2(v[8 * q], v[8 * q + 1]), pack_f16x2(v[8 * q + 2], v[8 * q + 3]),
+                                                      pack_f16x2(v[8 * q + 4], v[8 * q + 5]), pack_f16x2(v[8 * q + 6], v[8 * q + 7]));
+    } else {
+#pragma unroll
+      for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __half_as_ushort(__float2half_rn(v[c]));
     }
   }
 }
@@ -245,38 +257,14 @@ __device__ __forceinline__ void store_row_segment(const GemmParams& p, int64_t r
 // bias / SiLU / residual and one rounding to the output type.
 __device__ __forceinline__ void epilogue_store_chunk(const GemmParams& p, int part, int64_t row, int col0, int ncols,
                                                      const uint32_t (&r)[32]) {
-  if (p.ws && p.ws_dtype == RG_F32) {
-    float* dst = static_cast<float*>(p.ws) + ((int64_t)part * p.M + row) * p.ldw + col0;
-    if (ncols == 32) {
+  float v[32];
 #pragma unroll
-      for (int q = 0; q < 8; ++q)
-        reinterpret_cast<uint4*>(dst)[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
-    } else {
-#pragma unroll
-      for (int c = 0; c < 32; ++c) if (c < ncols) dst[c] = __uint_as_float(r[c]);
-    }
-  } else if (p.ws) {
-    // the finished part written at a 16-bit type: one rounding of the fp32 accumulator
-    const int64_t off = ((int64_t)part * p.M + row) * p.ldw + col0;
-    uint16_t* dst = static_cast<uint16_t*>(p.ws) + off;
-    if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        reinterpret_cast<uint4*>(dst)[q] = make_uint4(
-            pack_16x2(__uint_as_float(r[8 * q]), __uint_as_float(r[8 * q + 1]), p.ws_dtype),
-            pack_16x2(__uint_as_float(r[8 * q + 2]), __uint_as_float(r[8 * q + 3]), p.ws_dtype),
-            pack_16x2(__uint_as_float(r[8 * q + 4]), __uint_as_float(r[8 * q + 5]), p.ws_dtype),
-            pack_16x2(__uint_as_float(r[8 * q + 6]), __uint_as_float(r[8 * q + 7]), p.ws_dtype));
-    } else {
-#pragma unroll
-      for (int c = 0; c < 32; ++c) if (c < ncols) store_scalar(p.ws, p.ws_dtype, off + c, __uint_as_float(r[c]));
-    }
+  for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(r[c]);
+  if (p.ws) {
+    store_row_values(p.ws, p.ws_dtype, ((int64_t)part * p.M + row) * p.ldw + col0, ncols, v);
   } else {
-    float v[32];
-#pragma unroll
-    for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(r[c]);
     epilogue_row_segment(v, p.epi, row, col0, ncols);
-    store_row_segment(p, row, col0, ncols, v);
+    store_row_values(p.C, p.c_dtype, row * p.ldc + col0, ncols, v);
   }
 }
 
@@ -519,7 +507,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 //   empty[s]  in each CTA; tcgen05.commit arrives on both
 //   tfull[b]  in each CTA; tcgen05.commit arrives on both
 //   tempty[b] in the even CTA; the epilogue warps of both CTAs arrive on it
-template <int BN, int KSUB>
+template <int BN, int KSUB, bool F16>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                          const GemmParams p) {
@@ -527,7 +515,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   constexpr uint32_t B_BOX_BYTES = (BN / 2) * KBOX * 2;
   constexpr uint32_t STAGE_BYTES = KSUB * (A_BOX_BYTES + B_BOX_BYTES);      // per CTA
   constexpr uint32_t TMEM_COLS = 2 * BN;
-  const uint32_t IDESC = p.idesc;
+  constexpr uint32_t IDESC = make_idesc(BN, 2 * BM, F16 ? 0u : 1u);
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -788,12 +776,12 @@ size_t smem_bytes_for_pair(int bn, int ksub, int stages) {
   return 1024 + stages * stage + (2 * stages + 4) * 8 + 16;
 }
 
-template <int BN, int KSUB>
-cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
+template <int BN, int KSUB, bool F16>
+cudaError_t launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   const size_t smem = smem_bytes_for_pair(BN, KSUB, p.num_stages);
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_pair_kernel<BN, KSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_pair_kernel<BN, KSUB, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -807,7 +795,12 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const Gemm
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_pair_kernel<BN, KSUB>, ta, tb, p);
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_pair_kernel<BN, KSUB, F16>, ta, tb, p);
+}
+
+template <int BN, int KSUB>
+cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, bool f16, cudaStream_t st) {
+  return f16 ? launch_pair_t<BN, KSUB, true>(ta, tb, p, grid, st) : launch_pair_t<BN, KSUB, false>(ta, tb, p, grid, st);
 }
 
 template <int KSUB>
@@ -891,10 +884,10 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   if (pair) {
     const int64_t pairs = sms / 2;
     const int grid = 2 * (int)(total < pairs ? total : pairs);
-    if (plan.BN == 256 && ksub == 1) err = launch_pair<256, 1>(ta, tb, p, grid, st);
-    else if (plan.BN == 256 && ksub == 2) err = launch_pair<256, 2>(ta, tb, p, grid, st);
-    else if (plan.BN == 128 && ksub == 1) err = launch_pair<128, 1>(ta, tb, p, grid, st);
-    else if (plan.BN == 128 && ksub == 2) err = launch_pair<128, 2>(ta, tb, p, grid, st);
+    if (plan.BN == 256 && ksub == 1) err = launch_pair<256, 1>(ta, tb, p, grid, A->dtype == RG_F16, st);
+    else if (plan.BN == 256 && ksub == 2) err = launch_pair<256, 2>(ta, tb, p, grid, A->dtype == RG_F16, st);
+    else if (plan.BN == 128 && ksub == 1) err = launch_pair<128, 1>(ta, tb, p, grid, A->dtype == RG_F16, st);
+    else if (plan.BN == 128 && ksub == 2) err = launch_pair<128, 2>(ta, tb, p, grid, A->dtype == RG_F16, st);
     else return RG_ERR_UNSUPPORTED;
   } else {
     const int grid = (int)(total < sms ? total : sms);
