@@ -583,6 +583,8 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       int stage = 0; uint32_t phase = 0;
       bool alive = true;
       int it = 0;
+      const uint64_t desc_a0 = make_kmajor_sw128_desc(smem_base);
+      const uint64_t desc_b0 = make_kmajor_sw128_desc(smem_base + KSUB * A_BOX_BYTES);
       for (int w = pair_id; w < total_work && alive; w += num_pairs, ++it) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);
@@ -596,16 +598,30 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
           if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0xb00u | stage)) { alive = false; break; }
           tcgen05_fence_after();
-          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          // descriptors differ from the stage-0 ones only in the 16-byte-unit start address (low word)
+          const uint64_t adesc0 = desc_a0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
+          const uint64_t bdesc0 = desc_b0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
+          if (k0 + KBOX * KSUB <= k_end) {
+            // whole stage inside the part: 4*KSUB steps, ascending k, no per-step tests
 #pragma unroll
-          for (int sub = 0; sub < KSUB; ++sub) {
-            const uint64_t adesc = make_kmajor_sw128_desc(sa + sub * A_BOX_BYTES);
-            const uint64_t bdesc = make_kmajor_sw128_desc(sa + KSUB * A_BOX_BYTES + sub * B_BOX_BYTES);
+            for (int sub = 0; sub < KSUB; ++sub) {
 #pragma unroll
-            for (int a = 0; a < KBOX / UMMA_K; ++a) {
-              if (k0 + sub * KBOX + a * UMMA_K < k_end) {   // ascending k; nothing past the end of the part
-                umma_bf16_pair(d_tmem, adesc + 2u * a, bdesc + 2u * a, IDESC, accumulate);
-                accumulate = 1;
+              for (int a = 0; a < KBOX / UMMA_K; ++a) {
+                umma_bf16_pair(d_tmem, adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a,
+                               bdesc0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a, IDESC, (sub | a) ? 1u : accumulate);
+              }
+            }
+            accumulate = 1;
+          } else {
+#pragma unroll
+            for (int sub = 0; sub < KSUB; ++sub) {
+#pragma unroll
+              for (int a = 0; a < KBOX / UMMA_K; ++a) {
+                if (k0 + sub * KBOX + a * UMMA_K < k_end) {   // ascending k; nothing past the end of the part
+                  umma_bf16_pair(d_tmem, adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a,
+                                 bdesc0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a, IDESC, accumulate);
+                  accumulate = 1;
+                }
               }
             }
           }

@@ -40,8 +40,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait: gives up after WAIT_LIMIT_NS of wall time, or as soon as another role of the
 // CTA has raised `abort_flag`.  On its own timeout it raises the flag and records `code` in
 // *status (first writer wins).  Returns false if the wait was abandoned.
-static __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status,
-                                       uint32_t code) {
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status,
+                                            uint32_t code) {
   uint64_t t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -56,6 +56,12 @@ static __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, vol
       }
     }
   }
+}
+// Inline fast path: a barrier that is already complete costs one try_wait and no call.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status,
+                                          uint32_t code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status, code);
 }
 // 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier.  Both addresses
 // 16-byte aligned, size a multiple of 16.
