@@ -361,10 +361,10 @@ def cpu_baseline(budget_s: float):
     from oracle import rgo
     from paper_2609_11356_b200 import synth
     cores = rgo.num_threads()
-    t, fl = _oracle_gemm_sample(8, 256)                       # calibration
+    t, fl = _oracle_gemm_sample(16, 1024)                     # calibration (large enough to use every core)
     rate = fl / t
     cols = 2048
-    rows = int(max(8, min(256, budget_s * 0.7 * rate / (2.0 * cols * 8192))))
+    rows = int(max(8, min(1024, budget_s * 0.7 * rate / (2.0 * cols * 8192))))
     t, fl = _oracle_gemm_sample(rows, cols)
     x = synth.normal_f32((2048, RED_C), 100.0, 13)
     t0 = time.perf_counter()

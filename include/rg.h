@@ -71,7 +71,8 @@ typedef struct {
   /* ---- order-deciding fields: these ARE the class key ---- */
   uint8_t in_dtype;       /* rg_dtype_t of A and B: RG_BF16 or RG_F16 */
   uint8_t acc_dtype;      /* accumulator: RG_F32 */
-  uint8_t partial_dtype;  /* type a finished split-K part is written at: RG_F32, RG_BF16 or RG_F16 (Sec. 3.2.2) */
+  uint8_t partial_dtype;  /* type a finished split-K part is written at: RG_F32, RG_BF16 or RG_F16 (Sec. 3.2.2);
+                             without cuts no part is written and the field has no effect on the bits */
   uint8_t merge_dtype;    /* type the running sum of the parts is kept at: RG_F32, or the 16-bit type of the parts */
   uint8_t atom;           /* rg_atom_t */
   uint8_t k_tail;         /* 0 = the short K turn runs last, missing products are absent */

@@ -75,7 +75,7 @@ inline uint16_t f32_to_f16(float f) {
   const uint32_t u = f32_bits(f);
   const uint16_t sign = uint16_t((u >> 16) & 0x8000u);
   const uint32_t a = u & 0x7fffffffu;
-  if (a > 0x7f800000u) return uint16_t(sign | 0x7e00u);          // NaN
+  if (a > 0x7f800000u) return 0x7fffu;                           // NaN: canonical quiet NaN
   if (a >= 0x47800000u) return uint16_t(sign | 0x7c00u);         // >= 65536 (or inf): infinity
   const int e = int(a >> 23) - 127;                               // unbiased exponent
   uint32_t mant = (a & 0x7fffffu) | 0x800000u;                    // 24-bit significand
@@ -464,7 +464,9 @@ float gemm_element(const GemmDesc& d, const uint16_t* arow, const uint16_t* brow
       acc = first_group ? gacc : acc + gacc;
       first_group = false;
     }
-    part[s] = round_to(acc, d.partial_dtype);           // the finished part, at partial_dtype
+    // a finished part is written at partial_dtype only when the axis is split (Sec. 3.2.2, split-K:
+    // "a finished part is written at one type"); a plain GEMM writes no part and keeps fp32
+    part[s] = S > 1 ? round_to(acc, d.partial_dtype) : acc;
     if (partials_out) partials_out[s] = part[s];
   }
   float v = tree_reduce_at(part, d.tree, d.merge_dtype);  // merge in tree order, sum kept at merge_dtype

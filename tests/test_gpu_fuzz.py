@@ -1,0 +1,61 @@
+"""Descriptor-space fuzz (App. E: "a sweep of the plan-parameter space rather than of shapes"): random
+descriptors -- cuts, merge tree, part and merge types, inner span, operand type, tile knobs, epilogue --
+on small random shapes, every element against the oracle, ordinary and exponent-spread draws."""
+import numpy as np
+import pytest
+
+import paper_2609_11356_b200 as rg
+from oracle import rgo
+
+from _gpu_util import HW, assert_bits_equal, gpu_gemm
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(g):
+    M = int(g.choice([1, 7, 33, 128, 129, 200, 300]))
+    N = int(g.choice([8, 40, 64, 130, 256, 328]))
+    K = int(g.choice([64, 192, 576, 1000, 1024, 2048]))
+    f16 = bool(g.integers(0, 2))
+    nest = bool(g.integers(0, 3) == 0)
+    step = 64 if nest else 16
+    ncut = int(g.integers(0, 5))
+    pts = sorted(set(int(x) * step for x in g.integers(1, max(2, K // step), ncut) if 0 < int(x) * step < K))
+    desc = dict(cuts=tuple(pts), tree=int(g.integers(0, 2)))
+    pd, md = [(rgo.F32, rgo.F32), (rgo.BF16, rgo.F32), (rgo.BF16, rgo.BF16), (rgo.F16, rgo.F32), (rgo.F16, rgo.F16)][int(g.integers(0, 5))]
+    desc.update(partial_dtype=pd, merge_dtype=md)
+    knobs = {}
+    if nest:
+        desc["inner_span"] = int(g.choice([64, 128, 320]))
+        knobs = [dict(), dict(BN=64), dict(BN=96, stages=2)][int(g.integers(0, 3))]
+    else:
+        knobs = [dict(), dict(BN=64, BK=128), dict(cta_group=2, BN=128), dict(cta_group=2, BN=256, BK=64), dict(BN=48, cta_group=1),
+                 dict(BN=208, cta_group=1, raster=1), dict(BN=128, BK=256, cta_group=1, stages=1)][int(g.integers(0, 7))]
+    epi = {}
+    out = [rgo.BF16, rgo.F32, rgo.F16][int(g.integers(0, 3))]
+    return M, N, K, f16, desc, knobs, out
+
+
+@pytest.mark.parametrize("seed", range(150))
+def test_random_descriptor_matches_oracle(seed):
+    g = np.random.default_rng(1000 + seed)
+    M, N, K, f16, desc, knobs, out = _case(g)
+    spread = 6 if f16 else 10
+    A = g.standard_normal((M, K)); B = g.standard_normal((N, K))
+    if seed % 2:
+        A = A * np.exp2(g.integers(-spread, spread + 1, A.shape)); B = B * np.exp2(g.integers(-spread, spread + 1, B.shape))
+    if f16:
+        A, B = A.astype(np.float16), B.astype(np.float16)
+        conv = lambda x: np.asarray(x, np.float32).astype(np.float16)
+    else:
+        from paper_2609_11356_b200 import synth
+        A, B = synth.f32_to_bf16_bits(A.astype(np.float32)), synth.f32_to_bf16_bits(B.astype(np.float32))
+        conv = lambda x: synth.f32_to_bf16_bits(np.asarray(x, np.float32))
+    epi = {}
+    if g.integers(0, 2): epi["bias"] = conv(g.uniform(-0.5, 0.5, N))
+    if g.integers(0, 2): epi["act"] = 1
+    if g.integers(0, 2): epi["residual"] = g.standard_normal((M, N)).astype(np.float32)
+    got = gpu_gemm(A, B, out_dtype=out, **desc, **knobs, **epi)
+    want = rgo.gemm(A, B, atom_model=HW, out_dtype=out, **desc, **epi)
+    assert_bits_equal(got, want, f"seed {seed}: {M}x{N}x{K} f16={f16} {desc} {knobs} {list(epi)} out={out}")
+    assert rg.rg_device_status() == 0
