@@ -59,3 +59,40 @@ def test_random_descriptor_matches_oracle(seed):
     want = rgo.gemm(A, B, atom_model=HW, out_dtype=out, **desc, **epi)
     assert_bits_equal(got, want, f"seed {seed}: {M}x{N}x{K} f16={f16} {desc} {knobs} {list(epi)} out={out}")
     assert rg.rg_device_status() == 0
+
+
+@pytest.mark.parametrize("seed", range(100))
+def test_random_reduction_matches_oracle(seed):
+    """Row reductions over random widths, types, alignments and launch shapes, bit for bit."""
+    import torch
+    from _gpu_util import DEV, gpu_reduce
+    from paper_2609_11356_b200 import synth
+    g = np.random.default_rng(5000 + seed)
+    op = int(g.integers(0, 3))
+    bf = bool(g.integers(0, 2))
+    R = int(g.choice([1, 3, 37, 150, 400]))
+    Cc = int(g.choice([1, 5, 31, 128, 1000, 4096, 4100, 8192, 20000, 33001, 70000])) if R <= 37 else int(g.choice([7, 256, 1000, 4096, 9000]))
+    pad_l, pad_r = (int(g.integers(0, 9)), int(g.integers(0, 9))) if g.integers(0, 2) else (0, 0)
+    scale = float(g.choice([1.0, 100.0]))
+    full = synth.normal_f32((R, Cc + pad_l + pad_r), scale, 5000 + seed)
+    if seed % 3 == 0:
+        full = synth.spread_exponents_f32(full, seed, -8, 8)
+    if bf:
+        full = synth.f32_to_bf16_bits(full)
+    x = np.ascontiguousarray(full[:, pad_l:pad_l + Cc])
+    xt = synth.to_torch(full, DEV)[:, pad_l:pad_l + Cc]
+    knobs = {}
+    if g.integers(0, 2):
+        knobs = dict(BN=int(g.choice([32, 64, 128, 256, 512, 1024])), stages=int(g.choice([1, 2, 4, 8])))
+    kw = {}
+    if op == rg.RG_OP_RMSNORM:
+        kw = dict(eps=1e-5, fma=int(g.integers(0, 2)))
+        if g.integers(0, 2):
+            w = synth.normal_f32((Cc,), 0.05, seed, mean=1.0)
+            kw["weight"] = synth.f32_to_bf16_bits(w) if (bf and g.integers(0, 2)) else w
+    fma = kw.pop("fma", 0)
+    got, gaux = gpu_reduce(op, xt, **kw, fma=fma, **knobs)
+    want, waux = rgo.reduce_rows(op, x, fma=fma, **kw)
+    assert_bits_equal(got, want, f"seed {seed}: op={op} bf16={bf} {R}x{Cc} pad=({pad_l},{pad_r}) {knobs}")
+    if waux is not None:
+        assert_bits_equal(gaux, waux, f"seed {seed}: aux")
