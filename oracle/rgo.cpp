@@ -558,6 +558,60 @@ void rgo_gemm_partials(const AtomModel* atom, int n_cuts, const int64_t* cuts,
     }
 }
 
+// GEMV family (Sec. 3.2.2 "GEMV"): no matrix instruction; `lanes` lanes share one output element.
+// Each lane owns tiles of `tile` consecutive k and folds its elements in ascending k into one
+// accumulator with a scalar multiply-add (Sec. 3.2.1: one rounding per element with fma, two
+// without).  layout 0 (strided): lane l takes tiles l, l+lanes, l+2*lanes, ...; layout 1
+// (contiguous): lane l takes the l-th run of ceil(tiles/lanes) consecutive tiles.  The lane totals are
+// then folded by a butterfly: fold 0 counts the offsets up (1, 2, 4, ...), a balanced tree over the
+// lanes in index order; fold 1 counts them down (lanes/2, ..., 1), a balanced tree over the lanes
+// in bit-reversed order.  Then the same epilogue as the GEMM.
+void rgo_gemv(int in_dtype, int fma, int lanes, int tile, int layout, int fold,
+              int64_t M, int64_t N, int64_t K,
+              const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
+              void* C, int out_dtype, int64_t ldc,
+              const void* bias, int bias_dtype, int act,
+              const void* residual, int residual_dtype, int64_t ldr) {
+  const int64_t tiles = (K + tile - 1) / tile;
+  const int64_t run = (tiles + lanes - 1) / lanes;
+  int bits = 0;
+  while ((1 << bits) < lanes) ++bits;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int64_t i = 0; i < M; ++i)
+    for (int64_t j = 0; j < N; ++j) {
+      const uint16_t* a = A + i * lda;
+      const uint16_t* b = B + j * ldb;
+      std::vector<float> tot(lanes);
+      for (int l = 0; l < lanes; ++l) {
+        float acc = 0.0f;
+        for (int64_t t = 0; t < tiles; ++t) {
+          const bool mine = layout == 0 ? (t % lanes == l) : (t / run == l);
+          if (!mine) continue;
+          for (int64_t k = t * tile; k < std::min<int64_t>(K, (t + 1) * tile); ++k) {
+            const float x = in_to_f32(a[k], in_dtype), y = in_to_f32(b[k], in_dtype);
+            if (fma) acc = std::fmaf(x, y, acc);
+            else { const float p = x * y; acc = acc + p; }
+          }
+        }
+        tot[l] = acc;
+      }
+      std::vector<float> order(lanes);
+      for (int l = 0; l < lanes; ++l) {
+        int src = l;
+        if (fold == 1) {                                  // bit-reversed lane order
+          src = 0;
+          for (int q = 0; q < bits; ++q) src |= ((l >> q) & 1) << (bits - 1 - q);
+        }
+        order[l] = tot[src];
+      }
+      float v = tree_reduce(order, TREE_BALANCED);
+      if (bias) v = v + load_elem(bias, bias_dtype, j);
+      if (act == 1) v = silu(v);
+      if (residual) v = v + load_elem(residual, residual_dtype, i * ldr + j);
+      store_elem(C, out_dtype, i * ldc + j, v);
+    }
+}
+
 // Row reductions.  op: 0 sum, 1 RMSNorm, 2 softmax normaliser.
 //   sum:      out[r] = TREE(f32(x[r,:]))                                    (fp32 out)
 //   rmsnorm:  ss = TREE(x*x) (fma=1: level-0 nodes are fma(x1,x1,x0*x0));

@@ -104,6 +104,9 @@ def lib():
                                        i32, vp, i32, i32, vp, i32, i64, i64, vp, vp, vp, i32, i32, i64]
         L.rgo_gemm_partials.restype = None
         L.rgo_gemm_partials.argtypes = [C.POINTER(_AtomStruct), i32, vp, i64, i64, i64, vp, i64, vp, i64, vp, i32, i64]
+        L.rgo_gemv.restype = None
+        L.rgo_gemv.argtypes = [i32, i32, i32, i32, i32, i32, i64, i64, i64, vp, i64, vp, i64, vp, i32, i64,
+                               vp, i32, i32, vp, i32, i64]
         L.rgo_reduce_rows.restype = None
         L.rgo_reduce_rows.argtypes = [i32, i32, i32, vp, i32, i64, i64, i64, vp, i32, i64, vp, i32, f32, vp]
         _lib = L
@@ -244,6 +247,18 @@ def gemm_partials(A, B, *, cuts=(), atom_model: AtomModel = EXACT_RN, partial_dt
     m = atom_model.c()
     lib().rgo_gemm_partials(C.byref(m), c.size, _ptr(c), M, N, K, _ptr(A), K, _ptr(B), K, _ptr(P), partial_dtype, inner_span)
     return P
+
+
+def gemv(A, B, *, fma=1, lanes=32, tile=8, layout=0, fold=0, out_dtype=BF16, bias=None, act=0, residual=None) -> np.ndarray:
+    """C = epilogue(A @ B.T) in the GEMV family (Sec. 3.2.2): `lanes` lanes per output element, each folding
+    its tiles of `tile` k with scalar multiply-adds, then a butterfly over the lane totals."""
+    A, B, m = _operands(A, B, EXACT_RN)
+    M, K = A.shape; N = B.shape[0]
+    out = np.empty((M, N), dtype=_OUT_NP[out_dtype])
+    b, bd, r, rd, ldr = _epi(bias, residual)
+    lib().rgo_gemv(m.in_dtype, fma, lanes, tile, layout, fold, M, N, K, _ptr(A), K, _ptr(B), K, _ptr(out), out_dtype, N,
+                   _ptr(b), bd, act, _ptr(r), rd, ldr)
+    return out
 
 
 def reduce_rows(op: int, x, *, tree=TREE_BALANCED, fma=0, weight=None, eps=0.0, out_dtype=None):
