@@ -54,8 +54,11 @@ typedef enum { RG_TREE_LEFT = 0, RG_TREE_BALANCED = 1 } rg_tree_t;
 /* Which instruction folds products into the accumulator and how many per rounding step
  * (`instruction_k`, Sec. 3.2.1/3.2.2).  TC_BF16_K16: one tcgen05.mma kind::f16 step of 16
  * bf16 products, accumulator fp32 in tensor memory, steps chained in ascending k (App. E).
- * With RG_F16 operands the same step runs on fp16 products.  SCALAR names the fma-chain path; no kernel
- * here implements it. */
+ * With RG_F16 operands the same step runs on fp16 products.  SCALAR names the GEMV family: no matrix
+ * instruction; the 32 lanes of a warp share one output element, each folding its k tiles with scalar
+ * multiply-adds (fused when `fma` is set), then a shuffle butterfly over the lane totals (gemv_layout,
+ * gemv_fold below).  It is a different class of bits from the tensor-core path and is meant for a
+ * handful of rows (decode); it takes no cuts and no inner span. */
 typedef enum { RG_ATOM_TC_BF16_K16 = 0, RG_ATOM_SCALAR = 1 } rg_atom_t;
 
 #define RG_MAX_CUTS 63
@@ -84,6 +87,13 @@ typedef struct {
                              else, inside every part, an accumulator is closed every inner_span k (a multiple
                              of 64) and the closed groups are added at fp32, in ascending order, into the
                              part's running sum.  Order-deciding: part of the class key. */
+  uint8_t gemv_layout;    /* RG_ATOM_SCALAR only: how the 32 lanes of a warp deal the 8-wide k tiles of one output
+                             element (Sec. 3.2.2 "GEMV", `layout`): 0 = strided (lane l takes tiles l, l+32, ...),
+                             1 = contiguous (lane l takes the l-th run of ceil(tiles/32) tiles) */
+  uint8_t gemv_fold;      /* RG_ATOM_SCALAR only: the butterfly over the lane totals: 0 = offsets counted up
+                             (balanced tree over the lanes), 1 = counted down (balanced tree over the lanes in
+                             bit-reversed order: a different sum) */
+  uint8_t _pad1[2];
 } rg_desc_t;
 
 /* A row-major matrix in device memory. */

@@ -20,6 +20,7 @@ rg_status_t check_desc_fields(const rg_desc_t* d) {
     return RG_ERR_INVALID_DESC;
   if (d->atom > RG_ATOM_SCALAR || d->tree > RG_TREE_BALANCED || d->fma > 1 || d->k_tail > 1) return RG_ERR_INVALID_DESC;
   if (d->n_cuts > RG_MAX_CUTS) return RG_ERR_INVALID_DESC;
+  if (d->gemv_layout > 1 || d->gemv_fold > 1) return RG_ERR_INVALID_DESC;
   for (uint32_t i = 0; i < d->n_cuts; ++i) {
     if (d->cuts[i] == 0) return RG_ERR_INVALID_DESC;
     if (i > 0 && d->cuts[i] <= d->cuts[i - 1]) return RG_ERR_INVALID_DESC;
@@ -32,7 +33,13 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
   if ((d->in_dtype != RG_BF16 && d->in_dtype != RG_F16) || d->acc_dtype != RG_F32) return RG_ERR_UNSUPPORTED;
   // parts at fp32 summed at fp32, parts at a 16-bit type summed at fp32, or both at that type (Sec. 3.2.2)
   if (d->merge_dtype != RG_F32 && d->merge_dtype != d->partial_dtype) return RG_ERR_UNSUPPORTED;
-  if (d->atom != RG_ATOM_TC_BF16_K16 || d->k_tail != 0) return RG_ERR_UNSUPPORTED;
+  if (d->k_tail != 0) return RG_ERR_UNSUPPORTED;
+  if (d->atom == RG_ATOM_SCALAR) {
+    // GEMV family: one chain per lane, a balanced lane fold, nothing to split
+    if (d->n_cuts || d->inner_span || d->tree != RG_TREE_BALANCED) return RG_ERR_UNSUPPORTED;
+    return RG_OK;
+  }
+  if (d->gemv_layout || d->gemv_fold) return RG_ERR_INVALID_DESC;   // lane fields belong to the scalar family
   if (d->BM != 0 && d->BM != 128 && d->BM != 256) return RG_ERR_UNSUPPORTED;
   if (d->BN != 0 && (d->BN % 16 != 0 || d->BN < 16 || d->BN > 256)) return RG_ERR_UNSUPPORTED;
   if (d->BK != 0 && d->BK != 64 && d->BK != 128 && d->BK != 256) return RG_ERR_UNSUPPORTED;
@@ -158,7 +165,7 @@ rg_status_t rg_desc_validate(const rg_desc_t* d, int64_t M, int64_t N, int64_t K
 uint64_t rg_desc_class(const rg_desc_t* d) {
   if (check_desc_fields(d) != RG_OK) return 0;
   // canonical serialisation of the order-deciding fields only; "no cuts" has one spelling
-  uint8_t buf[16 + 4 * RG_MAX_CUTS];
+  uint8_t buf[20 + 4 * RG_MAX_CUTS];
   size_t n = 0;
   const uint8_t head[8] = {d->in_dtype, d->acc_dtype, d->partial_dtype, d->merge_dtype, d->atom, d->k_tail, d->fma, d->tree};
   memcpy(buf, head, 8); n = 8;
@@ -167,6 +174,7 @@ uint64_t rg_desc_class(const rg_desc_t* d) {
   for (uint32_t i = 0; i < nc; ++i)
     for (int b = 0; b < 4; ++b) buf[n++] = (uint8_t)(d->cuts[i] >> (8 * b));
   for (int b = 0; b < 4; ++b) buf[n++] = (uint8_t)(d->inner_span >> (8 * b));
+  buf[n++] = d->gemv_layout; buf[n++] = d->gemv_fold;
   uint64_t h = 0xcbf29ce484222325ull;                  // FNV-1a, 64 bit
   for (size_t i = 0; i < n; ++i) { h ^= buf[i]; h *= 0x100000001b3ull; }
   return h ? h : 1;
@@ -195,6 +203,7 @@ rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t*
     if (!ws || ws_bytes < rg_gemm_workspace_bytes(d, M, N)) return RG_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(ws) & 15) return RG_ERR_ALIGNMENT;
   }
+  if (d->atom == RG_ATOM_SCALAR) return rg::launch_gemv(d, A, B, C, epi, static_cast<cudaStream_t>(cuda_stream));
   rg::GemmPlan plan;
   if ((s = make_plan(d, M, N, K, &plan)) != RG_OK) return s;
   return rg::launch_gemm(plan, A, B, C, epi, ws, static_cast<cudaStream_t>(cuda_stream));

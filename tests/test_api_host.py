@@ -35,7 +35,11 @@ def test_validate_rules():
     assert rg.rg_desc_validate(rg.rg_desc(cuts=(512,)), 64, 256, 512) == 2          # cut at K
     assert rg.rg_desc_validate(rg.rg_desc(cuts=(0,)), 64, 256, 512) == 2
     assert rg.rg_desc_validate(rg.rg_desc(cuts=(40,)), 64, 256, 512) == 3           # splits a 16-wide step
-    assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_SCALAR), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_SCALAR), 64, 256, 512) == 0           # GEMV family
+    assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_SCALAR, cuts=(256,)), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_SCALAR, tree=K.RG_TREE_LEFT), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(gemv_fold=1), 64, 256, 512) == 2                      # lane fields without the scalar atom
+    assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_SCALAR, gemv_layout=2), 64, 256, 512) == 2
     assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16), 64, 256, 512) == 0
     assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16, merge_dtype=K.RG_BF16), 64, 256, 512) == 0
     assert rg.rg_desc_validate(rg.rg_desc(merge_dtype=K.RG_BF16), 64, 256, 512) == 3
@@ -64,7 +68,9 @@ def test_class_key_holds_order_fields_only():
     others = [rg.rg_desc(cuts=(1792,)), rg.rg_desc(cuts=(1792, 3600)), rg.rg_desc(),
               rg.rg_desc(cuts=(1792, 3584), tree=K.RG_TREE_LEFT), rg.rg_desc(cuts=(1792, 3584), fma=1),
               rg.rg_desc(cuts=(1792, 3584), partial_dtype=K.RG_BF16), rg.rg_desc(cuts=(1792, 3584), merge_dtype=K.RG_BF16),
-              rg.rg_desc(cuts=(1792, 3584), atom=K.RG_ATOM_SCALAR), rg.rg_desc(cuts=(1792, 3584), k_tail=1)]
+              rg.rg_desc(cuts=(1792, 3584), atom=K.RG_ATOM_SCALAR), rg.rg_desc(cuts=(1792, 3584), k_tail=1),
+              rg.rg_desc(cuts=(1792, 3584), inner_span=64), rg.rg_desc(cuts=(1792, 3584), atom=K.RG_ATOM_SCALAR, gemv_fold=1),
+              rg.rg_desc(cuts=(1792, 3584), atom=K.RG_ATOM_SCALAR, gemv_layout=1), rg.rg_desc(cuts=(1792, 3584), in_dtype=K.RG_F16)]
     keys = [rg.rg_desc_class(o) for o in others]
     assert len(set(keys + [k])) == len(keys) + 1
     # stale entries beyond n_cuts are not part of the record
