@@ -438,6 +438,19 @@ def run_only(args):
             it[0] += 1
             rg.rg_gemm(d, A, Ws[it[0] % 4], Cm, residual=R, ws=ws)
         work, unit = 2.0 * N * K / 1e9, "GB/s (weights)"
+    elif name == "gemv_decode":
+        # the lane-tree GEMV class on the decode weight shape, one to four rows
+        _, N, K = GEMMS["decode"]
+        M = args.gemv_rows
+        d = rg.rg_desc(atom=rg.RG_ATOM_SCALAR, fma=1)
+        A = synth.device_normal((M, K), 1.0, 4, bf, dev)
+        Ws = [synth.device_normal((N, K), 0.02, 3 + i, bf, dev) for i in range(4)]    # rotate: weights leave L2
+        Cm = torch.empty((M, N), dtype=bf, device=dev)
+        it = [0]
+        def fn():
+            it[0] += 1
+            rg.rg_gemm(d, A, Ws[it[0] % 4], Cm)
+        work, unit = 2.0 * N * K / 1e9, "GB/s (weights)"
     else:
         R_, C_ = (16384, RED_C) if name in ("row_sum", "softmax", "softmax_unit") else (RMS_R * 4, RMS_C)
         if name == "rmsnorm":
@@ -456,6 +469,12 @@ def run_only(args):
         fn()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if name in ("gemm_decode", "gemv_decode"):
+        # launches of tens of microseconds: keep the stream busy while the host queues them, so
+        # the events bracket device time and not the host's launch rate
+        filler = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+        for _ in range(8):
+            filler.fill_(1)
     e0.record()
     for _ in range(args.steps):
         fn()
@@ -471,8 +490,9 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_prefill", "gemm_decode", "row_sum", "softmax", "softmax_unit", "rmsnorm"],
+    ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_prefill", "gemm_decode", "gemv_decode", "row_sum", "softmax", "softmax_unit", "rmsnorm"],
                     help="run one kernel on a small case (used for the ncu captures)")
+    ap.add_argument("--gemv-rows", type=int, default=1, help="rows of A for --only gemv_decode")
     args = ap.parse_args()
     if args.only:
         run_only(args)

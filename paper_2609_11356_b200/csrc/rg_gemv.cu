@@ -56,8 +56,8 @@ __device__ __forceinline__ float mul_add(float a, float b, float acc) {
 constexpr int GEMV_THREADS = 128;
 // tiles of one lane per turn, and turns in the ring (one being folded, DEPTH-1 on their way):
 // the same ring bytes for every MR, fewer tiles per turn where the rows need the registers
-__host__ __device__ constexpr int gemv_unr(int mr) { return mr <= 2 ? 4 : 2; }
-__host__ __device__ constexpr int gemv_depth(int mr) { return mr <= 2 ? 3 : 6; }
+__host__ __device__ constexpr int gemv_unr(int mr) { return mr <= 2 ? 4 : mr <= 4 ? 2 : 1; }
+__host__ __device__ constexpr int gemv_depth(int mr) { return mr <= 2 ? 3 : mr <= 4 ? 6 : 12; }
 
 // 16 bytes global -> shared, asynchronously, past L1 (B is read once)
 __device__ __forceinline__ void copy16_async(void* smem_dst, const void* gsrc) {
@@ -114,20 +114,23 @@ __global__ void __launch_bounds__(GEMV_THREADS, 7) gemv_lane_tree_kernel(const G
         float w[UNR][8];
 #pragma unroll
         for (int u = 0; u < UNR; ++u) unpack8<F16>(my[(slot * UNR + u) * 32], w[u]);
+        // rows past M repeat the last row (their totals are not stored): no branch in the turn,
+        // so all MR * UNR loads of A go out together
+        uint4 araw[MR][UNR];
 #pragma unroll
         for (int r = 0; r < MR; ++r) {
-          if (m0 + r < p.M) {
-            const uint16_t* arow = p.A + (int64_t)(m0 + r) * p.lda;
-            uint4 araw[UNR];
+          const uint16_t* arow = p.A + (int64_t)min(m0 + r, p.M - 1) * p.lda;
 #pragma unroll
-            for (int u = 0; u < UNR; ++u) araw[u] = __ldg(reinterpret_cast<const uint4*>(arow + ((t + u * t_step) << 3)));
+          for (int u = 0; u < UNR; ++u) araw[r][u] = __ldg(reinterpret_cast<const uint4*>(arow + ((t + u * t_step) << 3)));
+        }
 #pragma unroll
-            for (int u = 0; u < UNR; ++u) {
-              float a[8];
-              unpack8<F16>(araw[u], a);
+        for (int u = 0; u < UNR; ++u) {
 #pragma unroll
-              for (int e = 0; e < 8; ++e) acc[r] = mul_add<FMA>(a[e], w[u][e], acc[r]);   // ascending k
-            }
+          for (int r = 0; r < MR; ++r) {
+            float a[8];
+            unpack8<F16>(araw[r][u], a);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[r] = mul_add<FMA>(a[e], w[u][e], acc[r]);   // ascending k
           }
         }
         slot = slot + 1 == DEPTH ? 0 : slot + 1;
