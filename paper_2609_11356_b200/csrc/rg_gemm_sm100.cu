@@ -149,6 +149,10 @@ __host__ __device__ constexpr uint32_t make_idesc(int bn, int m, uint32_t fmt) {
          (static_cast<uint32_t>(m >> 4) << 24);
 }
 
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
+}
+
 struct GemmParams {
   int32_t M, N, K;
   int32_t tiles_m, tiles_n, n_parts;
@@ -355,6 +359,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const int total_work = p.tiles_m * p.tiles_n * p.n_parts;
 
   if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmap_a);
+    prefetch_tensormap(&tmap_b);
     for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8u * s, 1); mbar_init(bar_empty + 8u * s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8u * b, 1); mbar_init(bar_tempty + 8u * b, NUM_EPI_WARPS); }
     *abort_flag = 0;
@@ -370,6 +376,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t tmem_base = *tmem_slot;
   // a split-K merge launched behind this kernel may be scheduled now; it still waits for this grid to finish
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // this kernel is itself launched with programmatic stream serialisation: everything above touched
+  // only this CTA's shared and tensor memory; global memory waits for the kernels before it
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -535,6 +544,8 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   const int total_work = p.tiles_m * p.tiles_n * p.n_parts;   // tiles_m counts 256-row tiles here
 
   if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmap_a);
+    prefetch_tensormap(&tmap_b);
     for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8u * s, 1); mbar_init(bar_empty + 8u * s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8u * b, 1); mbar_init(bar_tempty + 8u * b, 2 * NUM_EPI_WARPS); }
     *abort_flag = 0;
@@ -689,7 +700,9 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
   const int64_t ncol4 = (p.N + 3) / 4;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   // launched with programmatic stream serialisation: the grid may start while the GEMM kernel is
-  // still draining; nothing is read before that kernel has completed and flushed its stores
+  // still draining; nothing is read before that kernel has completed and flushed its stores.  A
+  // kernel launched the same way behind this one may set itself up meanwhile.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (idx >= (int64_t)p.M * ncol4) return;
   const int64_t row = idx / ncol4;
@@ -715,17 +728,32 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
   auto add4 = [&](const float4& a, const float4& b) -> float4 {
     return make_float4(add1(a.x, b.x), add1(a.y, b.y), add1(a.z, b.z), add1(a.w, b.w));
   };
+  // parts are fetched eight at a time (all eight loads in flight together), then folded in order
   float4 acc;
   if (p.tree == RG_TREE_LEFT) {
-    acc = load(0);
-    for (int s = 1; s < p.S; ++s) acc = add4(acc, load(s));
+    for (int s0 = 0; s0 < p.S; s0 += 8) {
+      float4 part[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) if (s0 + i < p.S) part[i] = load(s0 + i);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) if (s0 + i < p.S) acc = (s0 + i == 0) ? part[i] : add4(acc, part[i]);
+    }
   } else {
     float4 stack[7];
-    for (int s = 0; s < p.S; ++s) {
-      float4 v = load(s);
-      int b = 0;
-      for (; (s >> b) & 1; ++b) v = add4(stack[b], v);
-      stack[b] = v;
+    for (int s0 = 0; s0 < p.S; s0 += 8) {
+      float4 part[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) if (s0 + i < p.S) part[i] = load(s0 + i);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (s0 + i < p.S) {
+          const int s = s0 + i;
+          float4 v = part[i];
+          int b = 0;
+          for (; (s >> b) & 1; ++b) v = add4(stack[b], v);
+          stack[b] = v;
+        }
+      }
     }
     // leftovers: the lowest pending level moves up unchanged until it meets a sibling
     bool have = false;
@@ -828,8 +856,19 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmP
     if (e != cudaSuccess) return e;
     configured = SMEM_LIMIT;
   }
-  gemm_tcgen05_kernel<KSUB><<<grid, NUM_THREADS, smem, st>>>(ta, tb, p);
-  return cudaGetLastError();
+  // programmatic stream serialisation: the CTAs may set themselves up (barriers, tensor memory,
+  // descriptor prefetch) while the kernel before this one in the stream drains
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<KSUB>, ta, tb, p);
 }
 
 }  // namespace
