@@ -728,6 +728,15 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
   auto add4 = [&](const float4& a, const float4& b) -> float4 {
     return make_float4(add1(a.x, b.x), add1(a.y, b.y), add1(a.z, b.z), add1(a.w, b.w));
   };
+  // bias and residual are requested first so that their latency hides behind the parts'
+  float bias4[4] = {0.0f, 0.0f, 0.0f, 0.0f}, res4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    if (col0 + c < p.N) {
+      if (p.epi.bias) bias4[c] = load_scalar(p.epi.bias, p.epi.bias_dtype, col0 + c);
+      if (p.epi.residual) res4[c] = load_scalar(p.epi.residual, p.epi.residual_dtype, row * p.epi.ldr + col0 + c);
+    }
+  }
   // parts are fetched eight at a time (all eight loads in flight together), then folded in order
   float4 acc;
   if (p.tree == RG_TREE_LEFT) {
@@ -739,6 +748,7 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
       for (int i = 0; i < 8; ++i) if (s0 + i < p.S) acc = (s0 + i == 0) ? part[i] : add4(acc, part[i]);
     }
   } else {
+    // binary-counter stack with every index a compile-time constant, so it lives in registers
     float4 stack[7];
     for (int s0 = 0; s0 < p.S; s0 += 8) {
       float4 part[8];
@@ -749,26 +759,45 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
         if (s0 + i < p.S) {
           const int s = s0 + i;
           float4 v = part[i];
-          int b = 0;
-          for (; (s >> b) & 1; ++b) v = add4(stack[b], v);
-          stack[b] = v;
+          bool placed = false;
+#pragma unroll
+          for (int b = 0; b < 7; ++b) {
+            if (!placed) {
+              if ((s >> b) & 1) v = add4(stack[b], v);
+              else { stack[b] = v; placed = true; }
+            }
+          }
         }
       }
     }
     // leftovers: the lowest pending level moves up unchanged until it meets a sibling
     bool have = false;
+#pragma unroll
     for (int b = 0; b < 7; ++b) {
       if (!((p.S >> b) & 1)) continue;
       if (!have) { acc = stack[b]; have = true; }
       else acc = add4(stack[b], acc);
     }
   }
+  // bias -> SiLU -> residual -> one rounding, as in the GEMM kernels' epilogue
   float v[4] = {acc.x, acc.y, acc.z, acc.w};
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
-    if (col0 + c < p.N) {
-      store_scalar(p.C, p.c_dtype, row * p.ldc + col0 + c, apply_epilogue(v[c], p.epi, row, col0 + c));
-    }
+    if (p.epi.bias) v[c] = f_add(v[c], bias4[c]);
+    if (p.epi.act == 1) v[c] = rg_silu(v[c]);
+    if (p.epi.residual) v[c] = f_add(v[c], res4[c]);
+  }
+  uint16_t* const c16 = static_cast<uint16_t*>(p.C) + row * p.ldc + col0;
+  if (col0 + 4 <= p.N && p.c_dtype != RG_F32 && (reinterpret_cast<uintptr_t>(c16) & 7) == 0) {
+    // four 16-bit outputs as one 8-byte store
+    uint2 o;
+    o.x = pack_16x2(v[0], v[1], p.c_dtype);
+    o.y = pack_16x2(v[2], v[3], p.c_dtype);
+    *reinterpret_cast<uint2*>(c16) = o;
+  } else {
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      if (col0 + c < p.N) store_scalar(p.C, p.c_dtype, row * p.ldc + col0 + c, v[c]);
   }
 }
 
