@@ -376,9 +376,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t tmem_base = *tmem_slot;
   // a split-K merge launched behind this kernel may be scheduled now; it still waits for this grid to finish
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // this kernel is itself launched with programmatic stream serialisation: everything above touched
-  // only this CTA's shared and tensor memory; global memory waits for the kernels before it
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // This kernel is itself launched with programmatic stream serialisation, so it may be running
+  // before the kernels ahead of it in the stream have finished.  Each role that touches global
+  // memory waits for them (griddepcontrol.wait) immediately before its first access and not
+  // earlier: the instructions leading up to that access are then already fetched (the weight
+  // stream of the previous launch leaves no code in L2).  The MMA warp touches none.
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -391,6 +393,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       const uint32_t box_off = is_b ? KSUB * A_BOX_BYTES + sub * B_BOX_BYTES : sub * A_BOX_BYTES;
       int stage = 0; uint32_t phase = 0;
       bool alive = true;
+      bool deps_done = false;
       for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);
@@ -400,6 +403,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, &g_status_word, 0x100u | stage)) { alive = false; break; }
           const uint32_t full = bar_full + 8u * stage;
           if (lane == 0) mbar_expect_tx(full, STAGE_BYTES);
+          if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
           tma_load_2d(smem_base + stage * STAGE_BYTES + box_off, map, k0 + sub * KBOX, y, full);
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
@@ -457,6 +461,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     const int quarter = warp & 3;                         // TMEM lanes [32*quarter, 32*quarter+32)
     const int chunk0 = (warp - 2) >> 2;                   // this warp takes chunks chunk0, chunk0+2, ...
     bool alive = true;
+    bool deps_done = false;
     int gc = 0;
     for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
       int part, tm, tn;
@@ -469,6 +474,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         const int buf = gc & 1;
         if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
         tcgen05_fence_after();
+        if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
         epilogue_tile(p, BN, part, row, row_ok, tn, taddr, chunk0);
         tcgen05_fence_before();
@@ -481,6 +487,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           const int buf = gc & 1;
           if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
           tcgen05_fence_after();
+          if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
           grouped_add(p, BN, tn, taddr, chunk0, g == 0, acc);
           tcgen05_fence_before();
