@@ -88,6 +88,10 @@ __global__ void __launch_bounds__(GEMV_THREADS, 7) gemv_lane_tree_kernel(const G
   const int t_lim = min(t_end, p.K >> 3);
   const int n_full = t_lim > t_first ? (t_lim - t_first + t_step - 1) / t_step : 0;
   const int n_turns = n_full / UNR;
+  // launched with programmatic stream serialisation: a kernel queued behind this one may start
+  // its own set-up now, and this one reads nothing before the kernels ahead of it have finished
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   for (int64_t j = warp0; j < p.N; j += nwarps) {
     const uint16_t* brow = p.B + j * p.ldb;
     for (int m0 = 0; m0 < p.M; m0 += MR) {
@@ -185,9 +189,18 @@ __global__ void __launch_bounds__(GEMV_THREADS, 7) gemv_lane_tree_kernel(const G
 template <int MR, bool F16>
 cudaError_t launch_fma(const GemvParams& p, int grid, cudaStream_t st) {
   constexpr int smem = (GEMV_THREADS / 32) * gemv_depth(MR) * gemv_unr(MR) * 32 * 16;
-  if (p.fma) gemv_lane_tree_kernel<MR, F16, true><<<grid, GEMV_THREADS, smem, st>>>(p);
-  else gemv_lane_tree_kernel<MR, F16, false><<<grid, GEMV_THREADS, smem, st>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3(GEMV_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (p.fma) return cudaLaunchKernelEx(&cfg, gemv_lane_tree_kernel<MR, F16, true>, p);
+  return cudaLaunchKernelEx(&cfg, gemv_lane_tree_kernel<MR, F16, false>, p);
 }
 
 template <int MR>
