@@ -31,6 +31,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <limits>
 #include <vector>
 #ifdef _OPENMP
 #include <omp.h>
@@ -55,7 +56,7 @@ inline uint16_t f32_to_bf16(float f) {
   return uint16_t(u >> 16);
 }
 
-enum { DT_BF16 = 0, DT_F32 = 1, DT_F16 = 2 };
+enum { DT_BF16 = 0, DT_F32 = 1, DT_F16 = 2, DT_F8E4M3 = 3 };
 
 // IEEE binary16 (1-5-10): widening is exact.
 inline float f16_to_f32(uint16_t h) {
@@ -93,7 +94,22 @@ inline uint16_t f32_to_f16(float f) {
   return uint16_t(sign | r);                                      // 0x7c00 when it rounds up to infinity
 }
 
-inline float in_to_f32(uint16_t h, int dtype) { return dtype == DT_F16 ? f16_to_f32(h) : bf16_to_f32(h); }
+// 8-bit float 1-4-3, bias 7, no infinities, NaN = S.1111.111, largest finite 448 (the e4m3 input
+// type of Sec. 2's fp8 GEMMs).  Operands travel in 16-bit containers (value in the low byte).
+inline float f8e4m3_to_f32(uint16_t h) {
+  const int neg = (h >> 7) & 1;
+  const int e = (h >> 3) & 0xf;
+  const int m = h & 7;
+  float v;
+  if (e == 0xf && m == 7) v = std::numeric_limits<float>::quiet_NaN();
+  else if (e == 0) v = std::ldexp(float(m), -9);          // zero or subnormal: m * 2^-9
+  else v = std::ldexp(float(8 + m), e - 10);              // 1.m * 2^(e-7)
+  return neg ? -v : v;
+}
+
+inline float in_to_f32(uint16_t h, int dtype) {
+  return dtype == DT_F16 ? f16_to_f32(h) : dtype == DT_F8E4M3 ? f8e4m3_to_f32(h) : bf16_to_f32(h);
+}
 
 inline float load_elem(const void* p, int dtype, int64_t idx) {
   if (dtype == DT_BF16) return bf16_to_f32(static_cast<const uint16_t*>(p)[idx]);
@@ -270,7 +286,7 @@ struct AtomModel {
   int32_t acc_in_window;  // 1: the accumulator is aligned/truncated like a product
   int32_t addend_round;   // 0: truncate toward zero; 1: floor (toward -inf)
   int32_t final_round;    // 0: RZ; 1: RN-even
-  int32_t in_dtype;       // operand type of the products: DT_BF16 or DT_F16
+  int32_t in_dtype;       // operand type of the products: DT_BF16, DT_F16 or DT_F8E4M3
 };
 enum { ATOM_EXACT_RN = 0, ATOM_SEQ = 1, ATOM_ALIGN_TRUNC = 2 };
 
@@ -292,11 +308,22 @@ inline void f16_decode(uint16_t h, int& sign, uint32_t& mag, int& exp, int& e_le
   else { mag = m | 0x400; exp = e - 25; e_lead = e - 15; }
 }
 inline bool f16_finite(uint16_t h) { return ((h >> 10) & 0x1f) != 0x1f; }
-inline bool in_finite(uint16_t h, int dtype) { return dtype == DT_F16 ? f16_finite(h) : bf16_finite(h); }
+inline void f8e4m3_decode(uint16_t h, int& sign, uint32_t& mag, int& exp, int& e_lead) {
+  sign = ((h >> 7) & 1) ? -1 : 1;
+  int e = (h >> 3) & 0xf;
+  uint32_t m = h & 7;
+  if (e == 0) { mag = m; exp = -9; e_lead = -6; }
+  else { mag = m | 8; exp = e - 10; e_lead = e - 7; }
+}
+inline bool f8e4m3_finite(uint16_t h) { return (h & 0x7f) != 0x7f; }
+inline bool in_finite(uint16_t h, int dtype) {
+  return dtype == DT_F16 ? f16_finite(h) : dtype == DT_F8E4M3 ? f8e4m3_finite(h) : bf16_finite(h);
+}
 
 inline Prod make_prod(uint16_t a, uint16_t b, int dtype) {
   int sa, sb, ea, eb, la, lb; uint32_t ma, mb;
   if (dtype == DT_F16) { f16_decode(a, sa, ma, ea, la); f16_decode(b, sb, mb, eb, lb); }
+  else if (dtype == DT_F8E4M3) { f8e4m3_decode(a, sa, ma, ea, la); f8e4m3_decode(b, sb, mb, eb, lb); }
   else { bf16_decode(a, sa, ma, ea, la); bf16_decode(b, sb, mb, eb, lb); }
   Prod p; p.sign = sa * sb; p.mag = ma * mb; p.exp = ea + eb; p.e_op = la + lb;
   return p;
@@ -492,6 +519,7 @@ int rgo_num_threads() {
 float rgo_bf16_to_f32(uint16_t h) { return bf16_to_f32(h); }
 uint16_t rgo_f32_to_bf16(float f) { return f32_to_bf16(f); }
 float rgo_f16_to_f32(uint16_t h) { return f16_to_f32(h); }
+float rgo_f8e4m3_to_f32(uint8_t h) { return f8e4m3_to_f32(h); }
 uint16_t rgo_f32_to_f16(float f) { return f32_to_f16(f); }
 float rgo_add_f32(float a, float b) { return a + b; }
 float rgo_mul_f32(float a, float b) { return a * b; }

@@ -20,7 +20,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "rgo.cpp")
 _LIB = os.path.join(_HERE, "librgo.so")
 
-BF16, F32, F16 = 0, 1, 2
+BF16, F32, F16, F8E4M3 = 0, 1, 2, 3
 TREE_LEFT, TREE_BALANCED = 0, 1
 OP_SUM, OP_RMSNORM, OP_SOFTMAX_DENOM = 0, 1, 2
 ATOM_EXACT_RN, ATOM_SEQ, ATOM_ALIGN_TRUNC = 0, 1, 2
@@ -89,6 +89,7 @@ def lib():
         L.rgo_bf16_to_f32.restype = f32; L.rgo_bf16_to_f32.argtypes = [C.c_uint16]
         L.rgo_f32_to_bf16.restype = C.c_uint16; L.rgo_f32_to_bf16.argtypes = [f32]
         L.rgo_f16_to_f32.restype = f32; L.rgo_f16_to_f32.argtypes = [C.c_uint16]
+        L.rgo_f8e4m3_to_f32.restype = f32; L.rgo_f8e4m3_to_f32.argtypes = [C.c_uint8]
         L.rgo_f32_to_f16.restype = C.c_uint16; L.rgo_f32_to_f16.argtypes = [f32]
         for n in ("rgo_add_f32", "rgo_mul_f32"):
             getattr(L, n).restype = f32; getattr(L, n).argtypes = [f32, f32]
@@ -130,6 +131,10 @@ def f16_to_f32(h: int) -> float:
     return float(lib().rgo_f16_to_f32(int(h)))
 
 
+def f8e4m3_to_f32(h: int) -> float:
+    return float(lib().rgo_f8e4m3_to_f32(int(h)))
+
+
 def f32_to_f16(f) -> int:
     return int(lib().rgo_f32_to_f16(np.float32(f)))
 
@@ -165,8 +170,12 @@ def _dtype_code(a: np.ndarray) -> int:
 
 
 def _operands(A, B, atom_model):
-    """A, B as 16-bit patterns; float16 arrays select fp16 operands in the step model."""
+    """A, B as 16-bit patterns; float16 arrays select fp16 operands in the step model and uint8
+    arrays (e4m3 bit patterns, widened here to 16-bit containers) select fp8 operands."""
     A = np.ascontiguousarray(A); B = np.ascontiguousarray(B)
+    if A.dtype == np.uint8 or B.dtype == np.uint8:
+        assert A.dtype == np.uint8 and B.dtype == np.uint8
+        return A.astype(np.uint16), B.astype(np.uint16), atom_model.with_inputs(F8E4M3)
     if A.dtype == np.float16 or B.dtype == np.float16:
         assert A.dtype == np.float16 and B.dtype == np.float16
         return A.view(np.uint16), B.view(np.uint16), atom_model.with_inputs(F16)
@@ -182,7 +191,9 @@ def tree_sum(v, tree: int = TREE_BALANCED) -> np.float32:
 
 
 def atom(model: AtomModel, acc, a_bits, b_bits) -> np.float32:
-    if isinstance(a_bits, np.ndarray) and a_bits.dtype == np.float16:
+    if isinstance(a_bits, np.ndarray) and a_bits.dtype == np.uint8:
+        a_bits, b_bits, model = a_bits.astype(np.uint16), np.ascontiguousarray(b_bits, np.uint8).astype(np.uint16), model.with_inputs(F8E4M3)
+    elif isinstance(a_bits, np.ndarray) and a_bits.dtype == np.float16:
         a_bits, b_bits, model = a_bits.view(np.uint16), np.ascontiguousarray(b_bits, np.float16).view(np.uint16), model.with_inputs(F16)
     a = np.ascontiguousarray(a_bits, dtype=np.uint16)
     b = np.ascontiguousarray(b_bits, dtype=np.uint16)

@@ -29,6 +29,28 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
     return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32)
 
 
+def f32_to_f8e4m3_bits(x: np.ndarray) -> np.ndarray:
+    """Storage conversion binary32 -> 8-bit float e4m3 (torch's round to nearest even), as uint8 bits."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(torch.float8_e4m3fn)
+    return t.view(torch.uint8).numpy()
+
+
+def f8e4m3_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(b, dtype=np.uint8)).view(torch.float8_e4m3fn).to(torch.float32).numpy()
+
+
+def normal_f8e4m3(shape, std: float, seed: int, mean: float = 0.0) -> np.ndarray:
+    return f32_to_f8e4m3_bits(normal_f32(shape, std, seed, mean))
+
+
+def int_valued_f8e4m3(shape, lo: int, hi: int, seed: int) -> np.ndarray:
+    """Integers in [lo, hi] (|v| <= 16 are exact in e4m3)."""
+    v = _rng(seed).integers(lo, hi + 1, size=shape)
+    return f32_to_f8e4m3_bits(v.astype(np.float32))
+
+
 def normal_f32(shape, std: float, seed: int, mean: float = 0.0) -> np.ndarray:
     g = _rng(seed).standard_normal(size=shape, dtype=np.float64)
     return (g * std + mean).astype(np.float32)

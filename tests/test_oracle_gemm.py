@@ -332,6 +332,44 @@ def test_fp16_exact_atom_against_rationals(spread):
     assert rgo.atom(rgo.EXACT_RN, 0.0, a, b) == np.float32(2.0 ** -24 + 2.0 ** -24)
 
 
+# ---- fp8 e4m3 operands (Sec. 2: the fp8 GEMMs; a 32-wide step)
+def _with_k32(m):
+    import dataclasses
+    return dataclasses.replace(m, atom_k=32, group=(32 if m.group == 16 else m.group))
+
+
+def test_fp8_integer_products_and_closed_forms():
+    for K, cuts in ((512, (256,)), (1000, ()), (96, (32, 64))):
+        A = synth.int_valued_f8e4m3((5, K), -8, 8, 40 + K); B = synth.int_valued_f8e4m3((7, K), -8, 8, 41 + K)
+        Ai = synth.f8e4m3_bits_to_f32(A).astype(np.int64); Bi = synth.f8e4m3_bits_to_f32(B).astype(np.int64)
+        want = (Ai @ Bi.T).astype(np.float32)
+        for name, m in MODELS.items():
+            got = rgo.gemm(A, B, cuts=cuts, atom_model=_with_k32(m), out_dtype=rgo.F32)
+            assert np.array_equal(got, want), (name, K)
+    ones = synth.f32_to_f8e4m3_bits(np.ones((3, 4096), np.float32))
+    assert np.all(rgo.gemm(ones, ones, atom_model=_with_k32(rgo.EXACT_RN), out_dtype=rgo.F32) == np.float32(4096))
+    # rank one: every product alpha*beta, K of them
+    a = synth.f32_to_f8e4m3_bits(np.full((2, 640), 1.5, np.float32)); b = synth.f32_to_f8e4m3_bits(np.full((3, 640), -0.375, np.float32))
+    assert np.all(rgo.gemm(a, b, atom_model=_with_k32(rgo.EXACT_RN), out_dtype=rgo.F32) == np.float32(640 * 1.5 * -0.375))
+
+
+@pytest.mark.parametrize("spread", [1, 4, 7])
+def test_fp8_exact_atom_against_rationals(spread):
+    g = np.random.default_rng(300 + spread)
+    for trial in range(300):
+        n = int(g.integers(1, 33))
+        a = synth.f32_to_f8e4m3_bits((g.standard_normal(n) * np.exp2(g.integers(-spread, spread + 1, n))).astype(np.float32))
+        b = synth.f32_to_f8e4m3_bits((g.standard_normal(n) * np.exp2(g.integers(-spread, spread + 1, n))).astype(np.float32))
+        acc = np.float32(g.standard_normal() * 2.0 ** int(g.integers(-spread, spread + 1)))
+        af = synth.f8e4m3_bits_to_f32(a); bf = synth.f8e4m3_bits_to_f32(b)
+        exact = Fraction(float(acc)) + sum(Fraction(float(x)) * Fraction(float(y)) for x, y in zip(af, bf))
+        assert rgo.atom(_with_k32(rgo.EXACT_RN), acc, a, b) == _rn_f32(exact)
+    # subnormal operands take part exactly: 2^-9 * 1 + 2^-6 * 2^-3
+    a = np.array([0x01, 0x08], np.uint8); b = np.array([0x38, 0x20], np.uint8)
+    assert rgo.f8e4m3_to_f32(0x20) == 2.0 ** -3
+    assert rgo.atom(_with_k32(rgo.EXACT_RN), 0.0, a, b) == np.float32(2.0 ** -9 + 2.0 ** -9)
+
+
 # ---- second level of the cut nest (Sec. 3.2.2 k_cuts; App. E per-group accumulation)
 def test_inner_span_worked_example_and_closed_forms():
     """k=0: 1; k=32 and k=48: 2^-24 each (different 16-wide steps).  One chain: 1 + 2^-24 ties back to 1,

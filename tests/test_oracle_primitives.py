@@ -6,6 +6,7 @@ import pytest
 import torch
 
 from oracle import rgo
+from paper_2609_11356_b200 import synth
 
 
 def test_bf16_widening_exhaustive():
@@ -122,3 +123,17 @@ def test_f16_narrowing_matches_library_rne():
     assert np.array_equal(got, want)
     for h16 in range(0, 0x7c00):                                            # round trip of every finite pattern
         assert rgo.f32_to_f16(np.uint16(h16).view(np.float16).astype(np.float32)) == h16
+
+
+def test_f8e4m3_widening_exhaustive_and_landmarks():
+    allbits = np.arange(256, dtype=np.uint8)
+    want = synth.f8e4m3_bits_to_f32(allbits)                       # torch's conversion, an independent routine
+    got = np.array([rgo.f8e4m3_to_f32(int(h)) for h in allbits], dtype=np.float32)
+    nan = np.isnan(want)
+    assert list(np.nonzero(nan)[0]) == [0x7f, 0xff]                # the only NaN patterns; no infinities
+    assert np.array_equal(got[~nan].view(np.uint32), want[~nan].view(np.uint32)) and np.all(np.isnan(got[nan]))
+    # landmarks of the 1-4-3 format with bias 7
+    assert rgo.f8e4m3_to_f32(0x7e) == 448.0 and rgo.f8e4m3_to_f32(0xfe) == -448.0
+    assert rgo.f8e4m3_to_f32(0x01) == 2.0 ** -9 and rgo.f8e4m3_to_f32(0x07) == 7 * 2.0 ** -9
+    assert rgo.f8e4m3_to_f32(0x08) == 2.0 ** -6 and rgo.f8e4m3_to_f32(0x38) == 1.0 and rgo.f8e4m3_to_f32(0x3c) == 1.5
+    assert np.float32(rgo.f8e4m3_to_f32(0x80)).view(np.uint32) == 0x80000000
