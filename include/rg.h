@@ -42,7 +42,9 @@ typedef enum {
   RG_ERR_TIMEOUT = 8        /* a bounded device-side wait gave up (see rg_device_status) */
 } rg_status_t;
 
-typedef enum { RG_BF16 = 0, RG_F32 = 1, RG_F16 = 2 } rg_dtype_t;   /* RG_F16 = IEEE binary16 */
+/* RG_F16 = IEEE binary16.  RG_F8E4M3 = 8-bit float, 1-4-3, bias 7, no infinities, NaN = S.1111.111
+ * (the fp8 input type of Sec. 2); it is an operand type only (A and B of rg_gemm). */
+typedef enum { RG_BF16 = 0, RG_F32 = 1, RG_F16 = 2, RG_F8E4M3 = 3 } rg_dtype_t;
 
 /* The tree that combines values (split-K partials in rg_gemm, the leaves of a row in
  * rg_reduce_rows).  Sec. 3.1: a reduction order is a binary tree up to swapping an addition's
@@ -58,8 +60,12 @@ typedef enum { RG_TREE_LEFT = 0, RG_TREE_BALANCED = 1 } rg_tree_t;
  * instruction; the 32 lanes of a warp share one output element, each folding its k tiles with scalar
  * multiply-adds (fused when `fma` is set), then a shuffle butterfly over the lane totals (gemv_layout,
  * gemv_fold below).  It is a different class of bits from the tensor-core path and is meant for a
- * handful of rows (decode); it takes no cuts and no inner span. */
-typedef enum { RG_ATOM_TC_BF16_K16 = 0, RG_ATOM_SCALAR = 1 } rg_atom_t;
+ * handful of rows (decode); it takes no cuts and no inner span.  TC_F8_K32: one tcgen05.mma
+ * kind::f8f6f4 step of 32 e4m3 products (operands RG_F8E4M3, and only with them); cuts are multiples
+ * of 32, K is even (rows of A and B are whole byte pairs) and the leading dimensions are multiples
+ * of 16.  Its step has its own rounding behaviour (Sec. 3.2.1, footnote: fp8 steps differ between
+ * instruction families), so it is a class of its own. */
+typedef enum { RG_ATOM_TC_BF16_K16 = 0, RG_ATOM_SCALAR = 1, RG_ATOM_TC_F8_K32 = 2 } rg_atom_t;
 
 #define RG_MAX_CUTS 63
 
@@ -72,7 +78,7 @@ typedef struct {
   uint8_t raster;         /* tile walk: 0 = default grouped walk, 1 = row-major, n in 2..64 = groups of n tile rows */
   uint8_t _pad0;
   /* ---- order-deciding fields: these ARE the class key ---- */
-  uint8_t in_dtype;       /* rg_dtype_t of A and B: RG_BF16 or RG_F16 */
+  uint8_t in_dtype;       /* rg_dtype_t of A and B: RG_BF16, RG_F16, or RG_F8E4M3 (with atom = RG_ATOM_TC_F8_K32) */
   uint8_t acc_dtype;      /* accumulator: RG_F32 */
   uint8_t partial_dtype;  /* type a finished split-K part is written at: RG_F32, RG_BF16 or RG_F16 (Sec. 3.2.2);
                              without cuts no part is written and the field has no effect on the bits */

@@ -14,9 +14,9 @@ LIB_PATH = os.path.join(_HERE, "librg.so")
 RG_OK = 0
 STATUS_NAMES = {0: "RG_OK", 1: "RG_ERR_NULL", 2: "RG_ERR_INVALID_DESC", 3: "RG_ERR_UNSUPPORTED", 4: "RG_ERR_SHAPE",
                 5: "RG_ERR_ALIGNMENT", 6: "RG_ERR_WORKSPACE", 7: "RG_ERR_CUDA", 8: "RG_ERR_TIMEOUT"}
-RG_BF16, RG_F32, RG_F16 = 0, 1, 2
+RG_BF16, RG_F32, RG_F16, RG_F8E4M3 = 0, 1, 2, 3
 RG_TREE_LEFT, RG_TREE_BALANCED = 0, 1
-RG_ATOM_TC_BF16_K16, RG_ATOM_SCALAR = 0, 1
+RG_ATOM_TC_BF16_K16, RG_ATOM_SCALAR, RG_ATOM_TC_F8_K32 = 0, 1, 2
 RG_OP_SUM, RG_OP_RMSNORM, RG_OP_SOFTMAX_DENOM = 0, 1, 2
 RG_MAX_CUTS = 63
 RG_NOALLOC_WS_BYTES = 8 << 20

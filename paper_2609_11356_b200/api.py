@@ -30,6 +30,8 @@ def rg_desc(*, cuts: Sequence[int] = (), tree: int = K.RG_TREE_BALANCED, fma: in
         setattr(d, k, v)
     if "in_dtype" not in order_fields:
         d.in_dtype = K.RG_BF16
+    if d.in_dtype == K.RG_F8E4M3 and "atom" not in order_fields:
+        d.atom = K.RG_ATOM_TC_F8_K32           # the 8-bit operand type and the 32-wide step go together
     cuts = list(cuts)
     if len(cuts) > K.RG_MAX_CUTS:
         raise RgError(2, "rg_desc")
@@ -71,7 +73,9 @@ def _dtype_code(t) -> int:
         return K.RG_F32
     if t.dtype == torch.float16:
         return K.RG_F16
-    raise TypeError(f"rg tensors are bfloat16, float16 or float32, got {t.dtype}")
+    if t.dtype == torch.float8_e4m3fn:
+        return K.RG_F8E4M3
+    raise TypeError(f"rg tensors are bfloat16, float16, float32 or float8_e4m3fn, got {t.dtype}")
 
 
 def _tensor(t) -> K.rg_tensor_t:

@@ -8,17 +8,19 @@ namespace {
 
 constexpr int64_t DIM_LIMIT = (int64_t(1) << 31) - 1024;
 
-bool dtype_ok(int32_t t) { return t == RG_BF16 || t == RG_F32 || t == RG_F16; }
-size_t esize(int32_t t) { return t == RG_F32 ? 4 : 2; }
+bool dtype_ok(int32_t t) { return t == RG_BF16 || t == RG_F32 || t == RG_F16; }   // epilogue operands and outputs
+size_t esize(int32_t t) { return t == RG_F32 ? 4 : t == RG_F8E4M3 ? 1 : 2; }
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Structural checks that do not depend on a shape.
 rg_status_t check_desc_fields(const rg_desc_t* d) {
   if (!d) return RG_ERR_NULL;
   if (d->size != sizeof(rg_desc_t)) return RG_ERR_INVALID_DESC;
-  if (d->in_dtype > RG_F16 || d->acc_dtype > RG_F16 || d->partial_dtype > RG_F16 || d->merge_dtype > RG_F16)
+  if (d->in_dtype > RG_F8E4M3 || d->acc_dtype > RG_F8E4M3 || d->partial_dtype > RG_F8E4M3 || d->merge_dtype > RG_F8E4M3)
     return RG_ERR_INVALID_DESC;
-  if (d->atom > RG_ATOM_SCALAR || d->tree > RG_TREE_BALANCED || d->fma > 1 || d->k_tail > 1) return RG_ERR_INVALID_DESC;
+  // the 8-bit operand type and the 32-wide step name each other
+  if ((d->in_dtype == RG_F8E4M3) != (d->atom == RG_ATOM_TC_F8_K32)) return RG_ERR_INVALID_DESC;
+  if (d->atom > RG_ATOM_TC_F8_K32 || d->tree > RG_TREE_BALANCED || d->fma > 1 || d->k_tail > 1) return RG_ERR_INVALID_DESC;
   if (d->n_cuts > RG_MAX_CUTS) return RG_ERR_INVALID_DESC;
   if (d->gemv_layout > 1 || d->gemv_fold > 1) return RG_ERR_INVALID_DESC;
   for (uint32_t i = 0; i < d->n_cuts; ++i) {
@@ -30,7 +32,8 @@ rg_status_t check_desc_fields(const rg_desc_t* d) {
 
 // What the kernels of this library can honour.
 rg_status_t check_desc_supported(const rg_desc_t* d) {
-  if ((d->in_dtype != RG_BF16 && d->in_dtype != RG_F16) || d->acc_dtype != RG_F32) return RG_ERR_UNSUPPORTED;
+  if (d->in_dtype == RG_F32 || d->acc_dtype != RG_F32) return RG_ERR_UNSUPPORTED;
+  if (d->partial_dtype == RG_F8E4M3 || d->merge_dtype == RG_F8E4M3) return RG_ERR_UNSUPPORTED;
   // parts at fp32 summed at fp32, parts at a 16-bit type summed at fp32, or both at that type (Sec. 3.2.2)
   if (d->merge_dtype != RG_F32 && d->merge_dtype != d->partial_dtype) return RG_ERR_UNSUPPORTED;
   if (d->k_tail != 0) return RG_ERR_UNSUPPORTED;
@@ -48,21 +51,22 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
   if (d->cta_group == 2 && (d->BM == 128 || (d->BN != 0 && d->BN != 128 && d->BN != 256) || d->BK == 256)) return RG_ERR_UNSUPPORTED;   // a pair works on 256 rows, BN >= 128
   if (d->cta_group == 1 && d->BM == 256) return RG_ERR_UNSUPPORTED;
   if (d->raster > 64) return RG_ERR_INVALID_DESC;
+  const uint32_t step = d->atom == RG_ATOM_TC_F8_K32 ? 32 : 16;   // products per tensor-core step
   for (uint32_t i = 0; i < d->n_cuts; ++i)
-    if (d->cuts[i] % 16 != 0) return RG_ERR_UNSUPPORTED;   // a cut may not split a 16-wide step
+    if (d->cuts[i] % step != 0) return RG_ERR_UNSUPPORTED;   // a cut may not split a step
   if (d->inner_span) {
-    // groups are handed over per 64-wide K step by one CTA, with the running sum in registers
-    if (d->inner_span % 64 != 0) return RG_ERR_UNSUPPORTED;
+    // groups are handed over per pipeline stage (four steps) by one CTA, with the running sum in registers
+    if (d->inner_span % (4 * step) != 0) return RG_ERR_UNSUPPORTED;
     if (d->cta_group == 2 || d->BM == 256 || d->BN > 128 || (d->BK != 0 && d->BK != 64)) return RG_ERR_UNSUPPORTED;
     for (uint32_t i = 0; i < d->n_cuts; ++i)
-      if (d->cuts[i] % 64 != 0) return RG_ERR_UNSUPPORTED;
+      if (d->cuts[i] % (4 * step) != 0) return RG_ERR_UNSUPPORTED;
   }
   return RG_OK;
 }
 
-rg_status_t check_tensor(const rg_tensor_t* t) {
+rg_status_t check_tensor(const rg_tensor_t* t, bool operand = false) {
   if (!t) return RG_ERR_NULL;
-  if (!dtype_ok(t->dtype)) return RG_ERR_SHAPE;
+  if (!dtype_ok(t->dtype) && !(operand && t->dtype == RG_F8E4M3)) return RG_ERR_SHAPE;
   if (t->rows < 0 || t->cols < 0 || t->rows > DIM_LIMIT || t->cols > DIM_LIMIT) return RG_ERR_SHAPE;
   if (t->ld < t->cols) return RG_ERR_SHAPE;
   if (t->rows > 0 && t->cols > 0 && !t->ptr) return RG_ERR_NULL;
@@ -79,8 +83,8 @@ rg_status_t check_epilogue(const rg_epilogue_t* e, int64_t N) {
 
 rg_status_t check_gemm_shapes(const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C) {
   rg_status_t s;
-  if ((s = check_tensor(A)) != RG_OK || (s = check_tensor(B)) != RG_OK || (s = check_tensor(C)) != RG_OK) return s;
-  if ((A->dtype != RG_BF16 && A->dtype != RG_F16) || B->dtype != A->dtype) return RG_ERR_UNSUPPORTED;
+  if ((s = check_tensor(A, true)) != RG_OK || (s = check_tensor(B, true)) != RG_OK || (s = check_tensor(C)) != RG_OK) return s;
+  if (A->dtype == RG_F32 || B->dtype != A->dtype) return RG_ERR_UNSUPPORTED;
   if (A->cols != B->cols || C->rows != A->rows || C->cols != B->rows) return RG_ERR_SHAPE;
   return RG_OK;
 }
@@ -196,9 +200,11 @@ rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t*
   if (A->dtype != d->in_dtype) return RG_ERR_SHAPE;          // operands must be of the descriptor's input type
   if ((s = check_epilogue(epi, N)) != RG_OK) return s;
   if (M == 0 || N == 0) return RG_OK;
+  const int64_t ld_mult = 16 / (int64_t)esize(A->dtype);        // rows start on 16-byte boundaries
   if ((reinterpret_cast<uintptr_t>(A->ptr) & 15) || (reinterpret_cast<uintptr_t>(B->ptr) & 15) ||
-      (A->ld % 8) || (B->ld % 8))
+      (A->ld % ld_mult) || (B->ld % ld_mult))
     return RG_ERR_ALIGNMENT;
+  if (A->dtype == RG_F8E4M3 && (K & 1)) return RG_ERR_SHAPE;   // rows of 8-bit operands are whole byte pairs
   if (d->n_cuts) {
     if (!ws || ws_bytes < rg_gemm_workspace_bytes(d, M, N)) return RG_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(ws) & 15) return RG_ERR_ALIGNMENT;
@@ -237,10 +243,12 @@ rg_status_t rg_reduce_rows(const rg_desc_t* d, rg_reduce_op_t op, const rg_tenso
 size_t rg_gemm_host_scratch_bytes(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, int32_t c_dtype,
                                   const rg_epilogue_t* epi) {
   if (M <= 0 || N <= 0 || K <= 0) return 0;
-  const int64_t ldk = (K + 7) / 8 * 8;
+  const size_t ies = (d && d->in_dtype == RG_F8E4M3) ? 1 : 2;   // operand element size
+  const int64_t per16 = 16 / (int64_t)ies;
+  const int64_t ldk = (K + per16 - 1) / per16 * per16;
   size_t b = 0;
-  b += align_up((size_t)M * ldk * 2, 256);
-  b += align_up((size_t)N * ldk * 2, 256);
+  b += align_up((size_t)M * ldk * ies, 256);
+  b += align_up((size_t)N * ldk * ies, 256);
   b += align_up((size_t)M * N * esize(c_dtype), 256);
   if (epi && epi->bias) b += align_up((size_t)N * esize(epi->bias_dtype), 256);
   if (epi && epi->residual) b += align_up((size_t)M * N * esize(epi->residual_dtype), 256);
@@ -261,17 +269,20 @@ rg_status_t rg_gemm_host(const rg_desc_t* d, const rg_tensor_t* A, const rg_tens
   if (!dev_scratch || dev_scratch_bytes < rg_gemm_host_scratch_bytes(d, M, N, K, C->dtype, epi)) return RG_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(dev_scratch) & 255) return RG_ERR_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const int64_t ldk = (K + 7) / 8 * 8;
+  if (A->dtype != d->in_dtype) return RG_ERR_SHAPE;
+  const size_t ies = esize(A->dtype);
+  const int64_t per16 = 16 / (int64_t)ies;
+  const int64_t ldk = (K + per16 - 1) / per16 * per16;
   uint8_t* cur = static_cast<uint8_t*>(dev_scratch);
   auto take = [&](size_t bytes) { uint8_t* p = cur; cur += align_up(bytes, 256); return p; };
-  rg_tensor_t dA{take((size_t)M * ldk * 2), A->dtype, M, K, ldk};
-  rg_tensor_t dB{take((size_t)N * ldk * 2), B->dtype, N, K, ldk};
+  rg_tensor_t dA{take((size_t)M * ldk * ies), A->dtype, M, K, ldk};
+  rg_tensor_t dB{take((size_t)N * ldk * ies), B->dtype, N, K, ldk};
   rg_tensor_t dC{take((size_t)M * N * esize(C->dtype)), C->dtype, M, N, N};
   rg_epilogue_t de{};
   if (epi) de = *epi;
   bool ok = true;
-  ok &= cudaMemcpy2DAsync(dA.ptr, ldk * 2, A->ptr, A->ld * 2, K * 2, M, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpy2DAsync(dB.ptr, ldk * 2, B->ptr, B->ld * 2, K * 2, N, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpy2DAsync(dA.ptr, ldk * ies, A->ptr, A->ld * ies, K * ies, M, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpy2DAsync(dB.ptr, ldk * ies, B->ptr, B->ld * ies, K * ies, N, cudaMemcpyHostToDevice, st) == cudaSuccess;
   if (epi && epi->bias) {
     void* p = take((size_t)N * esize(epi->bias_dtype));
     ok &= cudaMemcpyAsync(p, epi->bias, (size_t)N * esize(epi->bias_dtype), cudaMemcpyHostToDevice, st) == cudaSuccess;

@@ -67,6 +67,15 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same step on 8-bit e4m3 operands: 32 products per step (32 bytes of K per operand row).
+__device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -144,6 +153,24 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
 }
 // Instruction descriptor: 16-bit x 16-bit -> fp32, both operands K-major.
 // operand format field: 0 = fp16, 1 = bf16
+__device__ __forceinline__ void umma_f8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// operand kinds of the kernels: what a 32-byte K step of an operand row holds
+enum { KIND_BF16 = 0, KIND_F16 = 1, KIND_F8E4M3 = 2 };
+// operand format field of the instruction descriptor: kind::f16 0 = fp16, 1 = bf16; kind::f8f6f4 0 = e4m3
+__host__ __device__ constexpr uint32_t idesc_format(int kind) { return kind == KIND_BF16 ? 1u : 0u; }
+template <int KIND>
+__device__ __forceinline__ void umma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  if (KIND == KIND_F8E4M3) umma_f8_pair(d_tmem, a_desc, b_desc, idesc, accumulate);
+  else umma_bf16_pair(d_tmem, a_desc, b_desc, idesc, accumulate);
+}
+
 __host__ __device__ constexpr uint32_t make_idesc(int bn, int m, uint32_t fmt) {
   return (1u << 4) | (fmt << 7) | (fmt << 10) | (static_cast<uint32_t>(bn >> 3) << 17) |
          (static_cast<uint32_t>(m >> 4) << 24);
@@ -160,6 +187,7 @@ struct GemmParams {
   int32_t inner_span;     // second cut level: an accumulator is closed every inner_span k (0 = none; a multiple of the K step)
   int32_t bn;             // tile columns of the one-CTA kernel (any multiple of 16 up to 256)
   uint32_t idesc;         // instruction descriptor for N = bn
+  int32_t f8;             // operands are e4m3 bytes: M, N as given, every K quantity counted in byte pairs
   uint32_t tmem_cols;     // tensor-memory columns allocated: two accumulators of tmem_cols / 2
   uint32_t a_box_bytes;   // bytes of one A box: 128 B per row actually loaded (rows past M are never fetched)
   void* C;
@@ -445,7 +473,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             for (int a = 0; a < KBOX / UMMA_K; ++a) {
               // ascending k; steps at or past the end of the part are not issued
               if (k0 + sub * KBOX + a * UMMA_K < k_end) {
-                umma_bf16(d_tmem, adesc + 2u * a, bdesc + 2u * a, IDESC, accumulate);
+                if (p.f8) umma_f8(d_tmem, adesc + 2u * a, bdesc + 2u * a, IDESC, accumulate);
+                else umma_bf16(d_tmem, adesc + 2u * a, bdesc + 2u * a, IDESC, accumulate);
                 accumulate = 1;
               }
             }
@@ -523,7 +552,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 //   empty[s]  in each CTA; tcgen05.commit arrives on both
 //   tfull[b]  in each CTA; tcgen05.commit arrives on both
 //   tempty[b] in the even CTA; the epilogue warps of both CTAs arrive on it
-template <int BN, int KSUB, bool F16>
+template <int BN, int KSUB, int KIND>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                          const GemmParams p) {
@@ -531,7 +560,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   constexpr uint32_t B_BOX_BYTES = (BN / 2) * KBOX * 2;
   constexpr uint32_t STAGE_BYTES = KSUB * (A_BOX_BYTES + B_BOX_BYTES);      // per CTA
   constexpr uint32_t TMEM_COLS = 2 * BN;
-  constexpr uint32_t IDESC = make_idesc(BN, 2 * BM, F16 ? 0u : 1u);
+  constexpr uint32_t IDESC = make_idesc(BN, 2 * BM, idesc_format(KIND));
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -625,7 +654,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
             for (int sub = 0; sub < KSUB; ++sub) {
 #pragma unroll
               for (int a = 0; a < KBOX / UMMA_K; ++a) {
-                umma_bf16_pair(d_tmem, adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a,
+                umma_pair<KIND>(d_tmem, adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a,
                                bdesc0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a, IDESC, (sub | a) ? 1u : accumulate);
               }
             }
@@ -636,7 +665,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 #pragma unroll
               for (int a = 0; a < KBOX / UMMA_K; ++a) {
                 if (k0 + sub * KBOX + a * UMMA_K < k_end) {   // ascending k; nothing past the end of the part
-                  umma_bf16_pair(d_tmem, adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a,
+                  umma_pair<KIND>(d_tmem, adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a,
                                  bdesc0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a, IDESC, accumulate);
                   accumulate = 1;
                 }
@@ -828,15 +857,19 @@ EncodeTiledFn get_encode_fn() {
 }
 
 // 2-D tensor map (bf16 or fp16 elements) over a row-major [rows, cols] matrix: box = 64 columns x box_rows rows,
-// 128-byte swizzle, zero fill outside the matrix (missing products are then exact zeros).
+// 128-byte swizzle, zero fill outside the matrix (missing products are then exact zeros).  An e4m3
+// matrix is described as byte pairs (cols and ld even, checked by the caller): the copy moves the
+// same bytes, a box is 128 of its columns, and a zero pair is two zero operands.
 bool make_tmap(CUtensorMap* map, const void* ptr, int dtype, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
+  if (dtype == RG_F8E4M3) { cols /= 2; ld /= 2; }
   const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
   const cuuint32_t box[2] = {(cuuint32_t)KBOX, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  return fn(map, dtype == RG_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+  const CUtensorMapDataType tdt = dtype == RG_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : dtype == RG_F8E4M3 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  return fn(map, tdt, 2, const_cast<void*>(ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -856,12 +889,12 @@ size_t smem_bytes_for_pair(int bn, int ksub, int stages) {
   return 1024 + stages * stage + (2 * stages + 4) * 8 + 16;
 }
 
-template <int BN, int KSUB, bool F16>
+template <int BN, int KSUB, int KIND>
 cudaError_t launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   const size_t smem = smem_bytes_for_pair(BN, KSUB, p.num_stages);
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_pair_kernel<BN, KSUB, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_pair_kernel<BN, KSUB, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -875,12 +908,14 @@ cudaError_t launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tb, const Ge
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_pair_kernel<BN, KSUB, F16>, ta, tb, p);
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_pair_kernel<BN, KSUB, KIND>, ta, tb, p);
 }
 
 template <int BN, int KSUB>
-cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, bool f16, cudaStream_t st) {
-  return f16 ? launch_pair_t<BN, KSUB, true>(ta, tb, p, grid, st) : launch_pair_t<BN, KSUB, false>(ta, tb, p, grid, st);
+cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, int kind, cudaStream_t st) {
+  if (kind == KIND_F16) return launch_pair_t<BN, KSUB, KIND_F16>(ta, tb, p, grid, st);
+  if (kind == KIND_F8E4M3) return launch_pair_t<BN, KSUB, KIND_F8E4M3>(ta, tb, p, grid, st);
+  return launch_pair_t<BN, KSUB, KIND_BF16>(ta, tb, p, grid, st);
 }
 
 template <int KSUB>
@@ -931,13 +966,17 @@ rg_status_t read_and_clear_status(uint32_t* code) {
 // Launch the GEMM (and the merge when there are cuts).  All arguments were validated by the caller.
 rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
                         const rg_epilogue_t* epi, void* ws, cudaStream_t st) {
-  const int64_t M = A->rows, K = A->cols, N = B->rows;
+  // e4m3 operands: every K quantity below (K, part bounds, inner span) counts byte pairs, so the
+  // kernels walk 32-byte steps of an operand row exactly as they do for 16-bit operands
+  const int kdiv = A->dtype == RG_F8E4M3 ? 2 : 1;
+  const int kind = A->dtype == RG_F16 ? KIND_F16 : A->dtype == RG_F8E4M3 ? KIND_F8E4M3 : KIND_BF16;
+  const int64_t M = A->rows, K = A->cols / kdiv, N = B->rows;
   const bool pair = plan.cta_group == 2;
   const int tile_m = pair ? 2 * BM : BM;
   CUtensorMap ta, tb;
   const int a_rows = pair ? BM : a_box_rows_for(M);
-  if (!make_tmap(&ta, A->ptr, A->dtype, M, K, A->ld, a_rows) ||
-      !make_tmap(&tb, B->ptr, B->dtype, N, K, B->ld, pair ? plan.BN / 2 : plan.BN))
+  if (!make_tmap(&ta, A->ptr, A->dtype, M, A->cols, A->ld, a_rows) ||
+      !make_tmap(&tb, B->ptr, B->dtype, N, B->cols, B->ld, pair ? plan.BN / 2 : plan.BN))
     return RG_ERR_CUDA;
 
   GemmParams p;
@@ -950,10 +989,11 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   p.group_m = plan.group_m;
   p.a_box_bytes = (uint32_t)a_rows * KBOX * 2;
   p.bn = plan.BN;
-  p.inner_span = plan.inner_span;
-  p.idesc = make_idesc(plan.BN, pair ? 2 * BM : BM, A->dtype == RG_F16 ? 0u : 1u);
+  p.inner_span = plan.inner_span / kdiv;
+  p.f8 = kind == KIND_F8E4M3;
+  p.idesc = make_idesc(plan.BN, pair ? 2 * BM : BM, idesc_format(kind));
   { uint32_t c = 32; while (c < 2u * (uint32_t)((plan.BN + 31) / 32 * 32)) c <<= 1; p.tmem_cols = c; }
-  for (int s = 0; s < plan.n_parts; ++s) { p.part_begin[s] = plan.part_begin[s]; p.part_end[s] = plan.part_end[s]; }
+  for (int s = 0; s < plan.n_parts; ++s) { p.part_begin[s] = plan.part_begin[s] / kdiv; p.part_end[s] = plan.part_end[s] / kdiv; }
   EpilogueArgs e{};
   if (epi) {
     e.bias = epi->bias; e.bias_dtype = epi->bias_dtype; e.act = epi->act;
@@ -975,10 +1015,10 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   if (pair) {
     const int64_t pairs = sms / 2;
     const int grid = 2 * (int)(total < pairs ? total : pairs);
-    if (plan.BN == 256 && ksub == 1) err = launch_pair<256, 1>(ta, tb, p, grid, A->dtype == RG_F16, st);
-    else if (plan.BN == 256 && ksub == 2) err = launch_pair<256, 2>(ta, tb, p, grid, A->dtype == RG_F16, st);
-    else if (plan.BN == 128 && ksub == 1) err = launch_pair<128, 1>(ta, tb, p, grid, A->dtype == RG_F16, st);
-    else if (plan.BN == 128 && ksub == 2) err = launch_pair<128, 2>(ta, tb, p, grid, A->dtype == RG_F16, st);
+    if (plan.BN == 256 && ksub == 1) err = launch_pair<256, 1>(ta, tb, p, grid, kind, st);
+    else if (plan.BN == 256 && ksub == 2) err = launch_pair<256, 2>(ta, tb, p, grid, kind, st);
+    else if (plan.BN == 128 && ksub == 1) err = launch_pair<128, 1>(ta, tb, p, grid, kind, st);
+    else if (plan.BN == 128 && ksub == 2) err = launch_pair<128, 2>(ta, tb, p, grid, kind, st);
     else return RG_ERR_UNSUPPORTED;
   } else {
     const int grid = (int)(total < sms ? total : sms);

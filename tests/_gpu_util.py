@@ -8,15 +8,25 @@ from paper_2609_11356_b200 import synth
 
 DEV = "cuda"
 HW = rgo.TCGEN05_BF16_B200   # the atom model the probes selected for this GPU
+HW8 = rgo.TCGEN05_F8E4M3_B200   # and for the 32-wide e4m3 step
 
 
 def gpu_gemm(A, B, *, out_dtype=rgo.BF16, bias=None, act=0, residual=None, poison=True, **desc_kw):
     """A, B: numpy uint16 (bf16 bits) or CUDA tensors.  Returns numpy (uint16 bits or float32)."""
     At = A if torch.is_tensor(A) else synth.to_torch(A, DEV)
     Bt = B if torch.is_tensor(B) else synth.to_torch(B, DEV)
+    if At.dtype == torch.uint8:                                   # numpy uint8 = e4m3 bit patterns
+        def rows16(t):                                            # rows start on 16-byte boundaries
+            Kp = (t.shape[1] + 15) // 16 * 16
+            buf = torch.full((t.shape[0], Kp), 0x7f, dtype=torch.uint8, device=DEV)   # padding is NaN: must never be read as data
+            buf[:, :t.shape[1]] = t
+            return buf.view(torch.float8_e4m3fn)[:, :t.shape[1]]
+        At, Bt = rows16(At), rows16(Bt)
     M, N = At.shape[0], Bt.shape[0]
     if At.dtype == torch.float16:
         desc_kw.setdefault("in_dtype", rg.RG_F16)
+    if At.dtype == torch.float8_e4m3fn:
+        desc_kw.setdefault("in_dtype", rg.RG_F8E4M3)
     d = rg.rg_desc(**desc_kw)
     tdt = {rgo.BF16: torch.bfloat16, rgo.F32: torch.float32, rgo.F16: torch.float16}[out_dtype]
     Ct = torch.empty((M, N), dtype=tdt, device=DEV)

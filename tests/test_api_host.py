@@ -40,6 +40,16 @@ def test_validate_rules():
     assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_SCALAR, tree=K.RG_TREE_LEFT), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(gemv_fold=1), 64, 256, 512) == 2                      # lane fields without the scalar atom
     assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_SCALAR, gemv_layout=2), 64, 256, 512) == 2
+    # 8-bit operands and the 32-wide step name each other; cuts fall on whole steps
+    assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, atom=K.RG_ATOM_TC_BF16_K16), 64, 256, 512) == 2
+    assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_TC_F8_K32), 64, 256, 512) == 2
+    assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, cuts=(48,)), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, cuts=(64,)), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, inner_span=64), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, inner_span=128), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, partial_dtype=K.RG_F8E4M3), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(in_dtype=4), 64, 256, 512) == 2
     assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16), 64, 256, 512) == 0
     assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16, merge_dtype=K.RG_BF16), 64, 256, 512) == 0
     assert rg.rg_desc_validate(rg.rg_desc(merge_dtype=K.RG_BF16), 64, 256, 512) == 3
@@ -108,6 +118,11 @@ def test_argument_errors_are_reported_before_any_launch():
     assert call(d, _t(0x1008, K.RG_BF16, 4, 64), B, Cm) == 5                       # 16-byte rule
     assert call(d, _t(0x1000, K.RG_BF16, 4, 60, 60), _t(0x2000, K.RG_BF16, 8, 60, 60), Cm) == 5   # ld % 8
     assert call(d, _t(0x1000, K.RG_BF16, 4, 0), _t(0x2000, K.RG_BF16, 8, 0), Cm) == 4            # K = 0
+    d8 = rg.rg_desc(in_dtype=K.RG_F8E4M3)
+    assert call(d8, _t(0x1000, K.RG_F8E4M3, 4, 63, 64), _t(0x2000, K.RG_F8E4M3, 8, 63, 64), Cm) == 4   # odd K: rows are whole byte pairs
+    assert call(d8, _t(0x1000, K.RG_F8E4M3, 4, 64, 72), _t(0x2000, K.RG_F8E4M3, 8, 64, 72), Cm) == 5   # ld % 16
+    assert call(d8, A, B, Cm) == 4                                                  # bf16 operands, e4m3 descriptor
+    assert call(d8, _t(0x1000, K.RG_F8E4M3, 4, 64), _t(0x2000, K.RG_F8E4M3, 8, 64), _t(0x3000, K.RG_F8E4M3, 4, 8)) == 4   # e4m3 is an operand type only
     ds = rg.rg_desc(cuts=(32,))
     assert call(ds, A, B, Cm) == 6                                                  # workspace missing
     assert call(ds, A, B, Cm, None, 0x4000, 16) == 6                                # too small
