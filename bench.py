@@ -426,6 +426,13 @@ def run_only(args):
         bias = synth.device_uniform((N,), -0.1, 0.1, 8, bf, dev) if name == "gemm_prefill" else None
         fn = lambda: rg.rg_gemm(d, A, B, Cm, bias=bias, act=1 if bias is not None else 0)
         work, unit = 2.0 * M * N * K / 1e12, "TFLOP/s"
+    elif name == "gemm_square_f8":
+        M, N, K = GEMMS["square"]
+        d = rg.rg_desc(in_dtype=rg.RG_F8E4M3)
+        A = synth.device_normal((M, K), 1.0, 11, torch.float8_e4m3fn, dev); B = synth.device_normal((N, K), 0.02, 12, torch.float8_e4m3fn, dev)
+        Cm = torch.empty((M, N), dtype=bf, device=dev)
+        fn = lambda: rg.rg_gemm(d, A, B, Cm)
+        work, unit = 2.0 * M * N * K / 1e12, "TFLOP/s"
     elif name == "gemm_decode":
         M, N, K = GEMMS["decode"]
         d = rg.rg_desc(cuts=tuple(1792 * t for t in range(1, 8)))
@@ -490,7 +497,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_prefill", "gemm_decode", "gemv_decode", "row_sum", "softmax", "softmax_unit", "rmsnorm"],
+    ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_square_f8", "gemm_prefill", "gemm_decode", "gemv_decode", "row_sum", "softmax", "softmax_unit", "rmsnorm"],
                     help="run one kernel on a small case (used for the ncu captures)")
     ap.add_argument("--gemv-rows", type=int, default=1, help="rows of A for --only gemv_decode")
     args = ap.parse_args()
