@@ -705,4 +705,38 @@ void rgo_reduce_rows(int op, int tree, int fma, const void* x, int x_dtype,
   }
 }
 
+// Reductions along the other axis (Sec. 6: "reductions on different dims/axes"; the column sum a
+// matrix-multiply epilogue emits; the LayerNorm weight-gradient reduction): out[c] = TREE over the
+// rows r = 0..R-1, in index order, of the leaf
+//   op 0 (sum):  x[r][c]
+//   op 1 (dot):  x[r][c] * y[r][c]   (one rounding per product; with fma and the balanced tree the
+//                second product of each level-0 pair is fused into that pair's add, as for RMSNorm)
+// The tree is the same "neighbours pair first" tree as along rows (Sec. 5.1).
+void rgo_reduce_cols(int op, int tree, int fma, const void* x, int x_dtype, const void* y, int y_dtype,
+                     int64_t R, int64_t C, int64_t ldx, int64_t ldy, float* out) {
+#pragma omp parallel for schedule(static)
+  for (int64_t c = 0; c < C; ++c) {
+    std::vector<float> leaf;
+    if (op == 0) {
+      leaf.resize(R);
+      for (int64_t r = 0; r < R; ++r) leaf[r] = load_elem(x, x_dtype, r * ldx + c);
+    } else if (fma && tree == TREE_BALANCED) {
+      leaf.resize((R + 1) / 2);
+      for (int64_t t = 0; 2 * t < R; ++t) {
+        float s = load_elem(x, x_dtype, 2 * t * ldx + c) * load_elem(y, y_dtype, 2 * t * ldy + c);
+        if (2 * t + 1 < R) s = std::fmaf(load_elem(x, x_dtype, (2 * t + 1) * ldx + c), load_elem(y, y_dtype, (2 * t + 1) * ldy + c), s);
+        leaf[t] = s;
+      }
+    } else if (fma) {
+      float acc = load_elem(x, x_dtype, c) * load_elem(y, y_dtype, c);
+      for (int64_t r = 1; r < R; ++r) acc = std::fmaf(load_elem(x, x_dtype, r * ldx + c), load_elem(y, y_dtype, r * ldy + c), acc);
+      leaf.assign(1, acc);
+    } else {
+      leaf.resize(R);
+      for (int64_t r = 0; r < R; ++r) leaf[r] = load_elem(x, x_dtype, r * ldx + c) * load_elem(y, y_dtype, r * ldy + c);
+    }
+    out[c] = tree_reduce(leaf, tree);
+  }
+}
+
 }  // extern "C"

@@ -115,6 +115,8 @@ def lib():
                                vp, i32, i32, vp, i32, i64]
         L.rgo_reduce_rows.restype = None
         L.rgo_reduce_rows.argtypes = [i32, i32, i32, vp, i32, i64, i64, i64, vp, i32, i64, vp, i32, f32, vp]
+        L.rgo_reduce_cols.restype = None
+        L.rgo_reduce_cols.argtypes = [i32, i32, i32, vp, i32, vp, i32, i64, i64, i64, i64, vp]
         _lib = L
     return _lib
 
@@ -297,3 +299,17 @@ def reduce_rows(op: int, x, *, tree=TREE_BALANCED, fma=0, weight=None, eps=0.0, 
     lib().rgo_reduce_rows(op, tree, fma, _ptr(x), xd, R, Cc, Cc, _ptr(out), od, ldo,
                           _ptr(w), wd, np.float32(eps), _ptr(aux))
     return out, (None if op == OP_SUM else aux)
+
+
+def reduce_cols(op: int, x, y=None, *, tree: int = TREE_BALANCED, fma: int = 0) -> np.ndarray:
+    """Reduction along axis 0 of x [R, C] (op 0: sum of x; op 1: sum of x*y), one tree per column
+    over the rows in index order.  Returns float32 [C]."""
+    x = np.ascontiguousarray(x)
+    R, Cc = x.shape
+    out = np.empty(Cc, dtype=np.float32)
+    if op == 1:
+        y = np.ascontiguousarray(y)
+        assert y.shape == x.shape
+    lib().rgo_reduce_cols(op, tree, fma, _ptr(x), _dtype_code(x), _ptr(y) if op == 1 else None,
+                          _dtype_code(y) if op == 1 else 0, R, Cc, Cc, Cc, _ptr(out))
+    return out

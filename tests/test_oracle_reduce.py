@@ -104,3 +104,68 @@ def test_softmax_normaliser():
     # a single column
     Z, m = rgo.reduce_rows(rgo.OP_SOFTMAX_DENOM, np.array([[5.0], [-2.0]], np.float32))
     assert np.all(Z == np.float32(1.0))
+
+
+# ---- reductions along the other axis (column sums; the LayerNorm weight-gradient shape)
+def test_col_sum_is_the_tree_per_column_over_rows_in_order():
+    x = synth.normal_f32((777, 6), 1.0, 5)
+    out = rgo.reduce_cols(0, x)
+    for c in range(6):
+        assert out[c] == _topdown(list(x[:, c]))                 # independent top-down restatement of the tree
+    # left fold spelled out
+    out_l = rgo.reduce_cols(0, x, tree=rgo.TREE_LEFT)
+    acc = x[0, 3]
+    for r in range(1, 777):
+        acc = np.float32(acc + x[r, 3])
+    assert out_l[3] == acc
+    # integer leaves: exact under any tree; all ones: R
+    xi = np.random.default_rng(1).integers(-100, 101, (1000, 9)).astype(np.float32)
+    assert np.array_equal(rgo.reduce_cols(0, xi), xi.astype(np.int64).sum(0).astype(np.float32))
+    assert np.all(rgo.reduce_cols(0, np.ones((4097, 3), np.float32)) == 4097)
+    # bf16 leaves widen exactly
+    xb = synth.int_valued_bf16((300, 4), -50, 50, 2)
+    assert np.array_equal(rgo.reduce_cols(0, xb), synth.bf16_bits_to_f32(xb).astype(np.int64).sum(0).astype(np.float32))
+
+
+def test_col_sum_probe_tells_the_tree_from_its_neighbours():
+    # +L, -L, r placed along the rows of one column: r survives exactly when +L and -L meet before r joins them
+    L, r = np.float32(1024.0), np.float32(2.0 ** -15)
+    def col(n, pos_r, pos_p, pos_m):
+        v = np.zeros((n, 1), np.float32); v[pos_r] = r; v[pos_p] = L; v[pos_m] = -L
+        return v
+    # rows 2,3 pair at level 0 in the balanced tree: +L and -L cancel before r (row 0) arrives
+    assert rgo.reduce_cols(0, col(8, 0, 2, 3))[0] == r
+    # rows 1,2 do not pair at level 0 (pairs are (0,1), (2,3)): r at row 0 is absorbed by +L
+    assert rgo.reduce_cols(0, col(8, 0, 1, 2))[0] == 0
+    # the left fold absorbs r at row 0 in both placements, and keeps it when it comes last
+    assert rgo.reduce_cols(0, col(8, 0, 2, 3), tree=rgo.TREE_LEFT)[0] == 0
+    assert rgo.reduce_cols(0, col(8, 7, 2, 3), tree=rgo.TREE_LEFT)[0] == r
+    # unpaired last row moves up unchanged: n = 5, rows (0,1), (2,3) pair, row 4 joins at the top
+    v = np.zeros((5, 1), np.float32); v[0] = L; v[1] = r; v[2] = -L; v[4] = r
+    assert rgo.reduce_cols(0, v)[0] == r                           # (L+r -> L) + (-L) = 0, then + r
+
+
+def test_col_dot_products_round_once_and_fma_flag():
+    g = np.random.default_rng(3)
+    x = g.standard_normal((513, 5)).astype(np.float32); y = g.standard_normal((513, 5)).astype(np.float32)
+    out = rgo.reduce_cols(1, x, y)
+    for c in range(5):
+        assert out[c] == _topdown([np.float32(a * b) for a, b in zip(x[:, c], y[:, c])])
+    # against double: 513 terms, a few ulp of the sum of magnitudes
+    ref = (x.astype(np.float64) * y.astype(np.float64)).sum(0)
+    assert np.all(np.abs(out - ref) <= 16 * 2.0 ** -24 * np.abs(x.astype(np.float64) * y).sum(0))
+    # integer-valued: exact; equals the sum path on the elementwise product
+    xi = g.integers(-30, 31, (400, 4)).astype(np.float32); yi = g.integers(-30, 31, (400, 4)).astype(np.float32)
+    assert np.array_equal(rgo.reduce_cols(1, xi, yi), (xi * yi).astype(np.int64).sum(0).astype(np.float32))
+    assert np.array_equal(rgo.reduce_cols(1, x, y), rgo.reduce_cols(0, (x * y).astype(np.float32)))
+    # fma: the second product of each level-0 pair is not rounded before the add.  a^2 = 1 + 2^-11 + 2^-24
+    # rounds to 1 + 2^-11; -RN(a^2) + a^2 is 0 with two roundings and the residual 2^-24 fused
+    a = np.float32(1 + 2.0 ** -12)
+    xx = np.array([[a], [a]], np.float32); yy = np.array([[-a], [a]], np.float32)
+    assert rgo.reduce_cols(1, xx, yy)[0] == 0
+    assert rgo.reduce_cols(1, xx, yy, fma=1)[0] == np.float32(2.0 ** -24)
+    assert rgo.reduce_cols(1, xx, yy, fma=1, tree=rgo.TREE_LEFT)[0] == np.float32(2.0 ** -24)
+    # the transpose relation: a column reduction is the row reduction of the transposed matrix
+    xt = np.ascontiguousarray(x.T)
+    rows, _ = rgo.reduce_rows(rgo.OP_SUM, xt)
+    assert np.array_equal(rgo.reduce_cols(0, x), rows)
