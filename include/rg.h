@@ -180,7 +180,24 @@ rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t*
 rg_status_t rg_reduce_rows(const rg_desc_t* d, rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out,
                            const rg_reduce_args_t* args, void* cuda_stream);
 
-/* Host-buffer forms of the two calls above, for callers whose data lives in host memory.
+/* Reductions along the other axis: one tree per column over the rows in index order (Sec. 6:
+ * "reductions on different dims/axes", the column sum a matrix-multiply epilogue emits, the
+ * LayerNorm weight-gradient reduction; the tree is the one of Sec. 5.1, `d->tree` BALANCED only).
+ *   RG_COLOP_SUM: out[c] = TREE_r f32(x[r,c])
+ *   RG_COLOP_DOT: out[c] = TREE_r f32(x[r,c]) * f32(y[r,c])   one rounding per product; with
+ *                 `d->fma` the second product of each level-0 pair is fused into that pair's add
+ * x (and y, same shape and type): bf16 or fp32, device pointers.  out: cols x 1 fp32.  More than
+ * 256 rows go through partial rows in `ws` (device, 16-byte aligned, at least
+ * rg_reduce_cols_workspace_bytes(rows, cols) bytes, caller-owned, contents arbitrary); the
+ * partials are totals of aligned blocks of 256 rows, i.e. subtrees of the same tree, so the result
+ * does not depend on the blocking.  cols == 0: RG_OK, nothing launched.  rows == 0: RG_ERR_SHAPE.
+ * Asynchronous on `cuda_stream`. */
+typedef enum { RG_COLOP_SUM = 0, RG_COLOP_DOT = 1 } rg_col_op_t;
+size_t rg_reduce_cols_workspace_bytes(int64_t rows, int64_t cols);
+rg_status_t rg_reduce_cols(const rg_desc_t* d, rg_col_op_t op, const rg_tensor_t* x, const rg_tensor_t* y,
+                           const rg_tensor_t* out, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Host-buffer forms of rg_gemm and rg_reduce_rows, for callers whose data lives in host memory.
  * Every tensor / epilogue / args pointer is a HOST pointer (pinned memory makes the copies
  * asynchronous).  `dev_scratch` is a caller-owned DEVICE buffer of at least
  * rg_*_host_scratch_bytes(...) bytes, 256-byte aligned, that the call uses for the device

@@ -17,6 +17,7 @@ STATUS_NAMES = {0: "RG_OK", 1: "RG_ERR_NULL", 2: "RG_ERR_INVALID_DESC", 3: "RG_E
 RG_BF16, RG_F32, RG_F16, RG_F8E4M3 = 0, 1, 2, 3
 RG_TREE_LEFT, RG_TREE_BALANCED = 0, 1
 RG_ATOM_TC_BF16_K16, RG_ATOM_SCALAR, RG_ATOM_TC_F8_K32 = 0, 1, 2
+RG_COLOP_SUM, RG_COLOP_DOT = 0, 1
 RG_OP_SUM, RG_OP_RMSNORM, RG_OP_SOFTMAX_DENOM = 0, 1, 2
 RG_MAX_CUTS = 63
 RG_NOALLOC_WS_BYTES = 8 << 20
@@ -24,7 +25,8 @@ RG_NOALLOC_WS_BYTES = 8 << 20
 # every symbol include/rg.h declares
 EXPORTS = ["rg_desc_init", "rg_desc_validate", "rg_desc_class", "rg_gemm_workspace_bytes", "rg_gemm",
            "rg_reduce_rows", "rg_gemm_host_scratch_bytes", "rg_gemm_host", "rg_reduce_rows_host_scratch_bytes",
-           "rg_reduce_rows_host", "rg_device_status", "rg_status_string", "rg_gemm_noalloc"]
+           "rg_reduce_rows_host", "rg_device_status", "rg_status_string", "rg_gemm_noalloc",
+           "rg_reduce_cols_workspace_bytes", "rg_reduce_cols"]
 
 
 class rg_desc_t(C.Structure):
@@ -75,6 +77,8 @@ def load():
     L.rg_gemm_host.restype = C.c_int; L.rg_gemm_host.argtypes = [D, T, T, T, E, vp, sz, vp]
     L.rg_reduce_rows_host_scratch_bytes.restype = sz; L.rg_reduce_rows_host_scratch_bytes.argtypes = [C.c_int, T, T]
     L.rg_reduce_rows_host.restype = C.c_int; L.rg_reduce_rows_host.argtypes = [D, C.c_int, T, T, A, vp, sz, vp]
+    L.rg_reduce_cols_workspace_bytes.restype = sz; L.rg_reduce_cols_workspace_bytes.argtypes = [i64, i64]
+    L.rg_reduce_cols.restype = C.c_int; L.rg_reduce_cols.argtypes = [D, C.c_int, T, T, T, vp, sz, vp]
     L.rg_gemm_noalloc.restype = C.c_int; L.rg_gemm_noalloc.argtypes = [D, T, T, T, E, vp]
     L.rg_device_status.restype = C.c_int; L.rg_device_status.argtypes = [C.POINTER(C.c_uint32)]
     L.rg_status_string.restype = C.c_char_p; L.rg_status_string.argtypes = [C.c_int]

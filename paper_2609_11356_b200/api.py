@@ -146,6 +146,25 @@ def rg_reduce_rows(d: K.rg_desc_t, op: int, x, out, *, weight=None, eps: float =
     return out
 
 
+def rg_reduce_cols_workspace_bytes(rows: int, cols: int) -> int:
+    return int(K.load().rg_reduce_cols_workspace_bytes(rows, cols))
+
+
+def rg_reduce_cols(d: K.rg_desc_t, op: int, x, out, *, y=None, ws=None):
+    """Reduction along axis 0 with the descriptor's tree: out[c] = TREE_r x[r, c] (RG_COLOP_SUM) or
+    TREE_r x[r, c] * y[r, c] (RG_COLOP_DOT).  `ws`: CUDA tensor of at least
+    rg_reduce_cols_workspace_bytes(rows, cols) bytes when x has more than 256 rows."""
+    L = K.load()
+    xt, ot = _tensor(x), _tensor(out)
+    yt = _tensor(y) if y is not None else None
+    ws_ptr = ws.data_ptr() if ws is not None else None
+    ws_bytes = ws.numel() * ws.element_size() if ws is not None else 0
+    st = L.rg_reduce_cols(C.byref(d), int(op), C.byref(xt), C.byref(yt) if yt is not None else None, C.byref(ot),
+                          ws_ptr, ws_bytes, _stream(x))
+    _check(st, "rg_reduce_cols")
+    return out
+
+
 def rg_gemm_host(d: K.rg_desc_t, A, B, C_out, dev_scratch, *, bias=None, act: int = 0, residual=None):
     """Host-buffer form: A, B, C_out, bias, residual are CPU tensors (pinned for async copies);
     `dev_scratch` is a CUDA tensor.  Enqueues copies + kernels on the current stream."""

@@ -239,6 +239,34 @@ rg_status_t rg_reduce_rows(const rg_desc_t* d, rg_reduce_op_t op, const rg_tenso
   return rg::launch_reduce_rows((int)op, d->fma, x, out, args, d->BN, d->stages, static_cast<cudaStream_t>(cuda_stream));
 }
 
+size_t rg_reduce_cols_workspace_bytes(int64_t rows, int64_t cols) {
+  if (rows <= 0 || cols <= 0) return 0;
+  return rg::reduce_cols_workspace_bytes(rows, cols);
+}
+
+rg_status_t rg_reduce_cols(const rg_desc_t* d, rg_col_op_t op, const rg_tensor_t* x, const rg_tensor_t* y,
+                           const rg_tensor_t* out, void* ws, size_t ws_bytes, void* cuda_stream) {
+  rg_status_t s = check_desc_fields(d);
+  if (s != RG_OK) return s;
+  if ((s = check_tensor(x)) != RG_OK || (s = check_tensor(out)) != RG_OK) return s;
+  if (op != RG_COLOP_SUM && op != RG_COLOP_DOT) return RG_ERR_UNSUPPORTED;
+  if (d->acc_dtype != RG_F32 || d->tree != RG_TREE_BALANCED) return RG_ERR_UNSUPPORTED;
+  if (x->dtype == RG_F16) return RG_ERR_UNSUPPORTED;                       // leaves are bf16 or fp32
+  if (op == RG_COLOP_DOT) {
+    if ((s = check_tensor(y)) != RG_OK) return s;
+    if (y->dtype != x->dtype || y->rows != x->rows || y->cols != x->cols) return RG_ERR_SHAPE;
+  }
+  if (x->rows < 1) return RG_ERR_SHAPE;
+  if (out->rows != x->cols || out->cols != 1 || out->dtype != RG_F32) return RG_ERR_SHAPE;
+  if (x->cols == 0) return RG_OK;
+  const size_t need = rg_reduce_cols_workspace_bytes(x->rows, x->cols);
+  if (need) {
+    if (!ws || ws_bytes < need) return RG_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(ws) & 15) return RG_ERR_ALIGNMENT;
+  }
+  return rg::launch_reduce_cols((int)op, d->fma, x, op == RG_COLOP_DOT ? y : nullptr, out, ws, static_cast<cudaStream_t>(cuda_stream));
+}
+
 // ------------------------------------------------------------ host-buffer forms
 size_t rg_gemm_host_scratch_bytes(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, int32_t c_dtype,
                                   const rg_epilogue_t* epi) {

@@ -24,6 +24,9 @@ rg_status_t launch_gemv(const rg_desc_t* d, const rg_tensor_t* A, const rg_tenso
                         const rg_epilogue_t* epi, cudaStream_t st);
 rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* out,
                                const rg_reduce_args_t* args, int threads_hint, int unroll_hint, cudaStream_t st);
+size_t reduce_cols_workspace_bytes(int64_t R, int64_t C);
+rg_status_t launch_reduce_cols(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* y, const rg_tensor_t* out,
+                               void* ws, cudaStream_t st);
 rg_status_t read_and_clear_status(uint32_t* code);
 rg_status_t read_and_clear_reduce_status(uint32_t* code);
 

@@ -138,6 +138,20 @@ def test_argument_errors_are_reported_before_any_launch():
     assert red(d, K.RG_OP_RMSNORM, x, o) == 4
     assert red(d, 9, x, o) == 3
     assert red(d, K.RG_OP_SUM, _t(None, K.RG_F32, 0, 64), _t(None, K.RG_F32, 0, 1)) == 0
+    col = lambda d_, op, x_, y_, o_, ws=None, wsb=0: L.rg_reduce_cols(C.byref(d_), op, C.byref(x_), C.byref(y_) if y_ is not None else None,
+                                                                   C.byref(o_), ws, wsb, None)
+    xc = _t(0x1000, K.RG_F32, 300, 64); oc = _t(0x2000, K.RG_F32, 64, 1)
+    assert col(d, K.RG_COLOP_SUM, xc, None, oc) == 6                                # more than 256 rows need the workspace
+    assert col(d, K.RG_COLOP_SUM, xc, None, oc, 0x4008, 1 << 20) == 5
+    assert col(d, K.RG_COLOP_DOT, xc, None, oc, 0x4000, 1 << 20) == 1               # y missing
+    assert col(d, K.RG_COLOP_DOT, xc, _t(0x5000, K.RG_BF16, 300, 64), oc, 0x4000, 1 << 20) == 4
+    assert col(d, K.RG_COLOP_SUM, xc, None, _t(0x2000, K.RG_F32, 63, 1), 0x4000, 1 << 20) == 4
+    assert col(d, K.RG_COLOP_SUM, _t(0x1000, K.RG_F32, 0, 64), None, oc) == 4       # no rows: nothing to fold
+    assert col(d, K.RG_COLOP_SUM, _t(None, K.RG_F32, 5, 0), None, _t(None, K.RG_F32, 0, 1)) == 0
+    assert col(rg.rg_desc(tree=K.RG_TREE_LEFT), K.RG_COLOP_SUM, xc, None, oc, 0x4000, 1 << 20) == 3
+    assert col(d, 7, xc, None, oc, 0x4000, 1 << 20) == 3
+    assert L.rg_reduce_cols_workspace_bytes(256, 1000) == 0 and L.rg_reduce_cols_workspace_bytes(257, 1000) == 2 * 1000 * 4
+    assert L.rg_reduce_cols_workspace_bytes(65537, 10) == (257 + 2) * 10 * 4
 
 
 def test_status_strings():
