@@ -458,6 +458,14 @@ def run_only(args):
             it[0] += 1
             rg.rg_gemm(d, A, Ws[it[0] % 4], Cm)
         work, unit = 2.0 * N * K / 1e9, "GB/s (weights)"
+    elif name in ("col_sum", "col_dot"):
+        R_, C_ = 65536, 8192
+        x = synth.device_normal((R_, C_), 100.0, 13, f32, dev)
+        y = synth.device_normal((R_, C_), 1.0, 14, f32, dev) if name == "col_dot" else None
+        out = torch.empty(C_, dtype=f32, device=dev)
+        ws = torch.empty(rg.rg_reduce_cols_workspace_bytes(R_, C_), dtype=torch.uint8, device=dev)
+        fn = lambda: rg.rg_reduce_cols(d, rg.RG_COLOP_DOT if y is not None else rg.RG_COLOP_SUM, x, out, y=y, ws=ws)
+        work, unit = (8.0 if y is not None else 4.0) * R_ * C_ / 1e9, "GB/s"
     else:
         R_, C_ = (16384, RED_C) if name in ("row_sum", "softmax", "softmax_unit") else (RMS_R * 4, RMS_C)
         if name == "rmsnorm":
@@ -497,7 +505,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_square_f8", "gemm_prefill", "gemm_decode", "gemv_decode", "row_sum", "softmax", "softmax_unit", "rmsnorm"],
+    ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_square_f8", "gemm_prefill", "gemm_decode", "gemv_decode", "col_sum", "col_dot", "row_sum", "softmax", "softmax_unit", "rmsnorm"],
                     help="run one kernel on a small case (used for the ncu captures)")
     ap.add_argument("--gemv-rows", type=int, default=1, help="rows of A for --only gemv_decode")
     args = ap.parse_args()
