@@ -224,7 +224,7 @@ def run_ours(args):
                          "frac_of_nominal_2250": round(sq_tflops / 2250.0, 4),
                          "peak_source": peaks["source"] + " (sustained: the kernel is timed inside a long step)",
                          "traffic": NCU_TRAFFIC_BYTES["gemm_8192"]},
-            "roofline_reduce": {"bound": "hbm", "kernel": "reduce_rows_warp_kernel<float,SUM> on 65536x32768",
+            "roofline_reduce": {"bound": "hbm", "kernel": "reduce_rows_cta_kernel<float,SUM> (one 1024-thread CTA per row) on 65536x32768",
                                 "achieved": round(sum_gbs, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                 "frac": round(sum_gbs / peaks["hbm_gbs"], 4), "frac_of_nominal_8000": round(sum_gbs / 8000.0, 4),
                                 "peak_source": peaks["source"], "traffic": NCU_TRAFFIC_BYTES["row_sum_65536x32768"]},
@@ -242,6 +242,52 @@ def run_ours(args):
         line["torch_cublas_square_tflops"] = round(2.0 * 8192 ** 3 / (e0.elapsed_time(e1) / 10 * 1e-3) / 1e12, 1)
         line["bitwise_equal_to_torch_cublas_square"] = bool(torch.equal(ref, T["sq_C"]))
         del ref
+
+    # ---- the rows built beyond the step above, timed alone (not part of `value`): fp8 operands, the
+    # decode GEMM and the GEMV family back to back on rotating weight copies, a column reduction
+    if rank == 0:
+        def timed(fn, n, filler=None):
+            for _ in range(3): fn()
+            torch.cuda.synchronize()
+            if filler is not None:
+                filler()                      # keeps the stream busy while the host queues short launches
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n): fn()
+            e1.record(); torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / n
+        busy = lambda: [rg.rg_reduce_rows(d_plain, rg.RG_OP_SUM, T["red_X"], T["red_sum"]) for _ in range(2)]
+        A8, B8 = T["sq_A"].to(torch.float8_e4m3fn), T["sq_B"].to(torch.float8_e4m3fn)
+        d8 = rg.rg_desc(in_dtype=rg.RG_F8E4M3)
+        c8 = torch.empty_like(T["sq_C"])        # own outputs: the step's results are checked further down
+        ms8 = timed(lambda: rg.rg_gemm(d8, A8, B8, c8), 10)
+        del A8, B8, c8
+        cd = torch.empty_like(T["dc_C"])
+        Ws = [T["dc_W"]] + [synth.device_normal((4096, 14336), 0.02, seed0 + 30 + i, bf, dev) for i in range(3)]
+        it = [0]
+        def decode():
+            it[0] += 1
+            rg.rg_gemm(d_split, T["dc_X"], Ws[it[0] % 4], cd, residual=T["dc_R"], ws=ws)
+        ms_dec = timed(decode, 40, busy)
+        dv = rg.rg_desc(atom=rg.RG_ATOM_SCALAR, fma=1)
+        x1 = T["dc_X"][:1]; c1 = cd[:1]
+        def gemv():
+            it[0] += 1
+            rg.rg_gemm(dv, x1, Ws[it[0] % 4], c1)
+        ms_gemv = timed(gemv, 40, busy)
+        del Ws
+        col_out = torch.empty(RED_C, dtype=f32, device=dev)
+        col_ws = torch.empty(rg.rg_reduce_cols_workspace_bytes(RED_R, RED_C), dtype=torch.uint8, device=dev)
+        ms_col = timed(lambda: rg.rg_reduce_cols(d_plain, rg.RG_COLOP_SUM, T["red_X"], col_out, ws=col_ws), 5)
+        wbytes = 2.0 * 4096 * 14336
+        line["widened"] = {
+            "note": "timed alone after the step loop; weights of the two decode paths rotate over four copies (above L2)",
+            "fp8_e4m3_square_tflops": round(2.0 * 8192 ** 3 / (ms8 * 1e-3) / 1e12, 1),
+            "decode_splitk8_back_to_back_us": round(ms_dec * 1e3, 2), "decode_splitk8_weight_gbs": round(wbytes / (ms_dec * 1e-3) / 1e9, 1),
+            "gemv_m1_back_to_back_us": round(ms_gemv * 1e3, 2), "gemv_m1_weight_gbs": round(wbytes / (ms_gemv * 1e-3) / 1e9, 1),
+            "col_sum_65536x32768_gbs": round(4.0 * RED_R * RED_C / (ms_col * 1e-3) / 1e9, 1),
+        }
+        del col_out, col_ws
 
     # ---- bit-match against the oracle on sampled outputs of this very run, and GPU-vs-GPU identity
     if rank == 0:
