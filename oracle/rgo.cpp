@@ -739,4 +739,57 @@ void rgo_reduce_cols(int op, int tree, int fma, const void* x, int x_dtype, cons
   }
 }
 
+// Attention with a fixed descriptor (App. F): one query row, keys cut into blocks of width w.
+// Per block j, with everything below in binary32 unless noted:
+//   s_t   = scale * (q . k_t)         the contraction is a chain of tensor-core steps over the head
+//                                     dimension from a zero accumulator (Sec. 3.2.1), then one multiply
+//   m_j   = max(m_{j-1}, max_t s_t)   a maximum rounds nothing
+//   alpha = exp(m_{j-1} - m_j),  p_t = exp(s_t - m_j)          (exp as fixed by this library)
+//   l_j   = alpha * l_{j-1} + TREE_t p_t                        (the block's row sum in the given tree)
+//   P_t   = p_t narrowed to p_dtype                             (the operand type of the second product)
+//   O_j   = alpha * O_{j-1} + (P . V)_block                     the block's product is a chain of steps
+//                                                               over its keys from a zero accumulator
+// and the answer is O_B / l_B, divided once at the end and rounded once to the output type.
+// Keys past Nk in the last block are absent: their scores are -inf, their probabilities exactly 0.
+// Vt is V transposed: [d, Nk], keys contiguous.
+void rgo_attention(const AtomModel* atom, int block_n, int sum_tree, int p_dtype, float scale,
+                   int64_t Nq, int64_t Nk, int64_t d, const uint16_t* Q, int64_t ldq, const uint16_t* K, int64_t ldk,
+                   const uint16_t* Vt, int64_t ldv, void* O, int o_dtype, int64_t ldo) {
+  const int ak = atom->atom_k;
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < Nq; ++i) {
+    const uint16_t* q = Q + i * ldq;
+    float m = -INFINITY, l = 0.0f;
+    std::vector<float> Oacc(d, 0.0f), s(block_n), pf(block_n);
+    std::vector<uint16_t> pn(block_n);
+    for (int64_t t0 = 0; t0 < Nk; t0 += block_n) {
+      const int n = (int)std::min<int64_t>(block_n, Nk - t0);
+      float mb = -INFINITY;
+      for (int t = 0; t < n; ++t) {
+        const uint16_t* k = K + (t0 + t) * ldk;
+        float acc = 0.0f;
+        for (int64_t c0 = 0; c0 < d; c0 += ak) acc = atom_step(acc, q + c0, k + c0, (int)std::min<int64_t>(ak, d - c0), *atom);
+        s[t] = acc * scale;
+        mb = std::max(mb, s[t]);
+      }
+      const float m_new = std::max(m, mb);
+      const float alpha = rg_expf(m - m_new);
+      std::vector<float> leaf(n);
+      for (int t = 0; t < n; ++t) { pf[t] = rg_expf(s[t] - m_new); leaf[t] = pf[t]; }
+      const float rowsum = tree_reduce(leaf, sum_tree);
+      l = alpha * l + rowsum;
+      for (int t = 0; t < n; ++t) pn[t] = p_dtype == DT_F16 ? f32_to_f16(pf[t]) : f32_to_bf16(pf[t]);
+      AtomModel pm = *atom; pm.in_dtype = p_dtype == DT_F16 ? DT_F16 : DT_BF16;
+      for (int64_t c = 0; c < d; ++c) {
+        const uint16_t* v = Vt + c * ldv + t0;
+        float acc = 0.0f;
+        for (int u0 = 0; u0 < n; u0 += ak) acc = atom_step(acc, pn.data() + u0, v + u0, std::min(ak, n - u0), pm);
+        Oacc[c] = alpha * Oacc[c] + acc;
+      }
+      m = m_new;
+    }
+    for (int64_t c = 0; c < d; ++c) store_elem(O, o_dtype, i * ldo + c, Oacc[c] / l);
+  }
+}
+
 }  // extern "C"

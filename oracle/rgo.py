@@ -115,6 +115,8 @@ def lib():
                                vp, i32, i32, vp, i32, i64]
         L.rgo_reduce_rows.restype = None
         L.rgo_reduce_rows.argtypes = [i32, i32, i32, vp, i32, i64, i64, i64, vp, i32, i64, vp, i32, f32, vp]
+        L.rgo_attention.restype = None
+        L.rgo_attention.argtypes = [C.POINTER(_AtomStruct), i32, i32, i32, f32, i64, i64, i64, vp, i64, vp, i64, vp, i64, vp, i32, i64]
         L.rgo_reduce_cols.restype = None
         L.rgo_reduce_cols.argtypes = [i32, i32, i32, vp, i32, vp, i32, i64, i64, i64, i64, vp]
         _lib = L
@@ -312,4 +314,20 @@ def reduce_cols(op: int, x, y=None, *, tree: int = TREE_BALANCED, fma: int = 0) 
         assert y.shape == x.shape
     lib().rgo_reduce_cols(op, tree, fma, _ptr(x), _dtype_code(x), _ptr(y) if op == 1 else None,
                           _dtype_code(y) if op == 1 else 0, R, Cc, Cc, Cc, _ptr(out))
+    return out
+
+
+def attention(Q, K, V, *, block_n: int, scale: float, atom_model: AtomModel = EXACT_RN, sum_tree: int = TREE_BALANCED,
+              p_dtype: int = BF16, out_dtype: int = BF16) -> np.ndarray:
+    """Attention of one head with a fixed descriptor (App. F): Q [Nq, d], K [Nk, d], V [Nk, d] as 16-bit
+    patterns (uint16 = bf16, float16 = fp16).  Returns [Nq, d] at out_dtype."""
+    Vt = np.ascontiguousarray(np.asarray(V).T)
+    Q, K, m = _operands(Q, K, atom_model)
+    Vt = Vt.view(np.uint16) if Vt.dtype == np.float16 else np.ascontiguousarray(Vt, dtype=np.uint16)
+    Nq, d = Q.shape; Nk = K.shape[0]
+    assert K.shape[1] == d and Vt.shape == (d, Nk)
+    out = np.empty((Nq, d), dtype=_OUT_NP[out_dtype])
+    mc = m.c()
+    lib().rgo_attention(C.byref(mc), block_n, sum_tree, p_dtype, np.float32(scale), Nq, Nk, d, _ptr(Q), d, _ptr(K), d,
+                        _ptr(Vt), Nk, _ptr(out), out_dtype, d)
     return out
