@@ -197,6 +197,34 @@ size_t rg_reduce_cols_workspace_bytes(int64_t rows, int64_t cols);
 rg_status_t rg_reduce_cols(const rg_desc_t* d, rg_col_op_t op, const rg_tensor_t* x, const rg_tensor_t* y,
                            const rg_tensor_t* out, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Attention of `heads` independent heads with a fixed reduction order (App. F).  Per query row the
+ * keys are walked in blocks of `block_n`; with s_t = scale * (q . k_t), everything fp32:
+ *   m_j = max(m_{j-1}, max_t s_t);  alpha = exp(m_{j-1} - m_j);  p_t = exp(s_t - m_j)
+ *   l_j = alpha * l_{j-1} + TREE_t p_t          (the block's row sum, keys in index order, `sum_tree`)
+ *   O_j = alpha * O_{j-1} + (P . V)_block       (P = p narrowed to `p_dtype`)
+ * and the answer is O_B / l_B: one division at the end, one rounding to O's type.  Both products are
+ * chains of tensor-core steps from a zero accumulator (RG_ATOM_TC_BF16_K16): over the head dimension
+ * for the scores, over the block's keys for P . V.  exp is the exponential this library fixes, base e.
+ * Every block boundary is a rounding of O and l, so block_n is part of the class of bits; the query
+ * tile is not (no masking here: `mask` must be 0).
+ *
+ * Q [heads*Nq, d], K [heads*Nk, d], Vt [heads*d, Nk] (V transposed: keys contiguous, what rg_gemm
+ * writes for W_v . X^T) and O [heads*Nq, d]: device pointers, heads stacked along the rows.  Q, K,
+ * Vt bf16, 16-byte aligned, leading dimensions multiples of 8; O bf16, fp16 or fp32.  d is 64 or 128,
+ * block_n 64 or 128.  Asynchronous on `cuda_stream`; no workspace. */
+typedef struct {
+  uint32_t size;          /* = sizeof(rg_attn_desc_t) */
+  uint32_t heads;         /* >= 1 */
+  uint32_t block_n;       /* key block width: 64 or 128 */
+  float scale;            /* scores are multiplied by this in fp32 */
+  uint8_t sum_tree;       /* rg_tree_t of the row sum inside a block: RG_TREE_BALANCED */
+  uint8_t p_dtype;        /* type the probabilities are narrowed to: RG_BF16 */
+  uint8_t mask;           /* 0 = none */
+  uint8_t div_place;      /* 0 = once, at the end */
+} rg_attn_desc_t;
+rg_status_t rg_attention(const rg_attn_desc_t* d, const rg_tensor_t* Q, const rg_tensor_t* K, const rg_tensor_t* Vt,
+                         const rg_tensor_t* O, void* cuda_stream);
+
 /* Host-buffer forms of rg_gemm and rg_reduce_rows, for callers whose data lives in host memory.
  * Every tensor / epilogue / args pointer is a HOST pointer (pinned memory makes the copies
  * asynchronous).  `dev_scratch` is a caller-owned DEVICE buffer of at least

@@ -146,6 +146,25 @@ def rg_reduce_rows(d: K.rg_desc_t, op: int, x, out, *, weight=None, eps: float =
     return out
 
 
+def rg_attn_desc(*, block_n: int, scale: float, heads: int = 1, sum_tree: int = K.RG_TREE_BALANCED, p_dtype: int = K.RG_BF16,
+                 mask: int = 0, div_place: int = 0) -> K.rg_attn_desc_t:
+    d = K.rg_attn_desc_t()
+    d.size = C.sizeof(K.rg_attn_desc_t)
+    d.heads, d.block_n, d.scale = heads, block_n, scale
+    d.sum_tree, d.p_dtype, d.mask, d.div_place = sum_tree, p_dtype, mask, div_place
+    return d
+
+
+def rg_attention(d: K.rg_attn_desc_t, Q, Kt, Vt, O):
+    """O = attention(Q, K, V) with the descriptor's key-block recurrence.  Q [heads*Nq, d],
+    Kt [heads*Nk, d], Vt [heads*d, Nk] (V transposed), O [heads*Nq, d]: CUDA tensors."""
+    L = K.load()
+    q, k, v, o = _tensor(Q), _tensor(Kt), _tensor(Vt), _tensor(O)
+    st = L.rg_attention(C.byref(d), C.byref(q), C.byref(k), C.byref(v), C.byref(o), _stream(Q))
+    _check(st, "rg_attention")
+    return O
+
+
 def rg_reduce_cols_workspace_bytes(rows: int, cols: int) -> int:
     return int(K.load().rg_reduce_cols_workspace_bytes(rows, cols))
 

@@ -267,6 +267,30 @@ rg_status_t rg_reduce_cols(const rg_desc_t* d, rg_col_op_t op, const rg_tensor_t
   return rg::launch_reduce_cols((int)op, d->fma, x, op == RG_COLOP_DOT ? y : nullptr, out, ws, static_cast<cudaStream_t>(cuda_stream));
 }
 
+rg_status_t rg_attention(const rg_attn_desc_t* d, const rg_tensor_t* Q, const rg_tensor_t* K, const rg_tensor_t* Vt,
+                         const rg_tensor_t* O, void* cuda_stream) {
+  if (!d) return RG_ERR_NULL;
+  if (d->size != sizeof(rg_attn_desc_t) || d->heads < 1 || d->sum_tree > RG_TREE_BALANCED || d->p_dtype > RG_F8E4M3)
+    return RG_ERR_INVALID_DESC;
+  rg_status_t s;
+  if ((s = check_tensor(Q)) != RG_OK || (s = check_tensor(K)) != RG_OK || (s = check_tensor(Vt)) != RG_OK || (s = check_tensor(O)) != RG_OK)
+    return s;
+  if (d->sum_tree != RG_TREE_BALANCED || d->p_dtype != RG_BF16 || d->mask != 0 || d->div_place != 0) return RG_ERR_UNSUPPORTED;
+  if (d->block_n != 64 && d->block_n != 128) return RG_ERR_UNSUPPORTED;
+  if (Q->dtype != RG_BF16 || K->dtype != RG_BF16 || Vt->dtype != RG_BF16) return RG_ERR_UNSUPPORTED;
+  const int64_t hd = Q->cols, H = d->heads;
+  if (hd != 64 && hd != 128) return RG_ERR_UNSUPPORTED;
+  if (Q->rows % H || K->rows % H || K->cols != hd || Vt->rows != H * hd) return RG_ERR_SHAPE;
+  const int64_t Nq = Q->rows / H, Nk = K->rows / H;
+  if (Nk < 1 || Vt->cols != Nk || O->rows != Q->rows || O->cols != hd) return RG_ERR_SHAPE;
+  if (Nq == 0) return RG_OK;
+  if ((reinterpret_cast<uintptr_t>(Q->ptr) & 15) || (reinterpret_cast<uintptr_t>(K->ptr) & 15) ||
+      (reinterpret_cast<uintptr_t>(Vt->ptr) & 15) || (reinterpret_cast<uintptr_t>(O->ptr) & 15) ||
+      (Q->ld % 8) || (K->ld % 8) || (Vt->ld % 8) || (O->ld % 8))
+    return RG_ERR_ALIGNMENT;
+  return rg::launch_attention_fixed((int)d->block_n, d->scale, (int)H, Q, K, Vt, O, static_cast<cudaStream_t>(cuda_stream));
+}
+
 // ------------------------------------------------------------ host-buffer forms
 size_t rg_gemm_host_scratch_bytes(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, int32_t c_dtype,
                                   const rg_epilogue_t* epi) {
@@ -382,13 +406,15 @@ rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_
 }
 
 rg_status_t rg_device_status(uint32_t* code) {
-  uint32_t a = 0, b = 0;
+  uint32_t a = 0, b = 0, c = 0;
   const rg_status_t s1 = rg::read_and_clear_status(&a);          // synchronises the device
   if (s1 == RG_ERR_CUDA) return s1;
   const rg_status_t s2 = rg::read_and_clear_reduce_status(&b);
   if (s2 == RG_ERR_CUDA) return s2;
-  if (code) *code = a ? a : b;
-  return (a || b) ? RG_ERR_TIMEOUT : RG_OK;
+  const rg_status_t s3 = rg::read_and_clear_attn_status(&c);
+  if (s3 == RG_ERR_CUDA) return s3;
+  if (code) *code = a ? a : (b ? b : c);
+  return (a || b || c) ? RG_ERR_TIMEOUT : RG_OK;
 }
 
 const char* rg_status_string(rg_status_t s) {

@@ -1,0 +1,380 @@
+// Attention with a fixed reduction order (App. F): per query row the keys are walked in blocks
+// of width w; each block contributes one rescale of the running output and denominator, so w,
+// the row-sum tree, the type the probabilities are narrowed to and the place of the division
+// are all part of the arithmetic and all come from the descriptor.
+//
+// One CTA owns 128 query rows of one head.  Per key block j:
+//   warp 0 (TMA)      K_j [w x d] and Vt_j [d x w] boxes into a two-stage ring (Q once)
+//   warp 1 (MMA)      S = Q K_j^T   d/16 tcgen05.mma steps from a zero accumulator, ascending k
+//                     PV = P Vt_j^T w/16 steps from a zero accumulator, ascending key
+//   warps 2-5         one query row per thread (its TMEM lane):
+//                     s_t = acc * scale; m_j = max(m_{j-1}, max_t s_t); alpha = exp(m_{j-1} - m_j);
+//                     p_t = exp(s_t - m_j); l_j = alpha*l_{j-1} + TREE_t p_t (balanced tree over the
+//                     block's keys in order); P = p narrowed to bf16, written to shared memory in the
+//                     swizzled K-major layout the tensor core reads; O_j = alpha*O_{j-1} + PV
+// and at the end O / l, one division, one rounding to the output type.  exp is the library's
+// specified exponential (rg_exp), not the hardware's base-two one.  Keys past Nk are masked to
+// -inf before the maximum, so their probabilities are exactly +0.
+//
+// Heads are stacked along the rows of Q [heads*Nq, d], K [heads*Nk, d], Vt [heads*d, Nk] and
+// O [heads*Nq, d]; blockIdx.y is the head.  Rows of another head that a box may pick up at a head
+// boundary are either masked (keys) or never stored (queries).
+#include <cuda.h>
+
+#include "rg_common.cuh"
+#include "rg_internal.h"
+#include "rg_ptx.cuh"
+
+namespace rg {
+
+__device__ unsigned int g_attn_status_word = 0;
+
+namespace {
+
+constexpr int QROWS = 128;          // query rows per CTA = TMEM lanes
+constexpr int ATT_THREADS = 192;    // warp 0 TMA, warp 1 MMA, warps 2-5 softmax
+constexpr int KV_STAGES = 2;
+
+// ---- PTX wrappers (tensor core side)
+__device__ __forceinline__ void att_tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void att_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void att_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void att_tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void att_tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void att_tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void att_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void att_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void att_tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void att_tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major tile with 128-byte rows and the 128-byte swizzle: 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t att_kmajor_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n
+__host__ __device__ constexpr uint32_t att_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(QROWS >> 4) << 24);
+}
+
+struct AttnParams {
+  int32_t Nq, Nk;        // per head
+  float scale;
+  void* O;
+  int64_t ldo;
+  int32_t o_dtype;
+};
+
+// balanced "neighbours pair first" tree over 32 values in index order
+__device__ __forceinline__ float tree32(const float (&p)[32]) {
+  float a[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) a[i] = f_add(p[2 * i], p[2 * i + 1]);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) a[i] = f_add(a[2 * i], a[2 * i + 1]);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) a[i] = f_add(a[2 * i], a[2 * i + 1]);
+  return f_add(f_add(a[0], a[1]), f_add(a[2], a[3]));
+}
+
+// W = key block width (64 or 128), HD = head dimension (64 or 128)
+template <int W, int HD>
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                 const __grid_constant__ CUtensorMap tmap_vt, const AttnParams p) {
+  constexpr uint32_t Q_BOX = QROWS * 128;                 // bytes of one [128 rows x 64 columns] box
+  constexpr uint32_t K_BOX = W * 128;                     // [W keys x 64 columns of d]
+  constexpr uint32_t V_BOX = HD * 128;                    // [HD rows of Vt x 64 keys]
+  constexpr uint32_t P_BOX = QROWS * 128;                 // [128 rows x 64 keys]
+  constexpr int DB = HD / 64, WB = W / 64;                // boxes along d and along the keys
+  constexpr uint32_t Q_BYTES = DB * Q_BOX, K_BYTES = DB * K_BOX, V_BYTES = WB * V_BOX, P_BYTES = WB * P_BOX;
+  constexpr uint32_t KV_BYTES = K_BYTES + V_BYTES;
+  constexpr uint32_t TMEM_COLS = 256;                     // S at columns [0, W), PV at [128, 128 + HD)
+  constexpr uint32_t IDESC_S = att_idesc(W), IDESC_PV = att_idesc(HD);
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t sQ = smem_base, sKV = sQ + Q_BYTES, sP = sKV + KV_STAGES * KV_BYTES;
+  uint8_t* sP_gen = smem_gen + Q_BYTES + KV_STAGES * KV_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + Q_BYTES + KV_STAGES * KV_BYTES + P_BYTES);
+  // barriers: q_full, kv_full[2], kv_empty[2], s_full, p_full, pv_full
+  const uint32_t bar_q = smem_u32(bars);
+  const uint32_t bar_kv_full = bar_q + 8u, bar_kv_empty = bar_kv_full + 8u * KV_STAGES;
+  const uint32_t bar_s = bar_kv_empty + 8u * KV_STAGES, bar_p = bar_s + 8u, bar_pv = bar_p + 8u;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int head = blockIdx.y;
+  const int q0 = blockIdx.x * QROWS;                      // first query row of this CTA within the head
+  const int nblocks = (p.Nk + W - 1) / W;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_q, 1);
+    for (int s = 0; s < KV_STAGES; ++s) { mbar_init(bar_kv_full + 8u * s, 1); mbar_init(bar_kv_empty + 8u * s, 1); }
+    mbar_init(bar_s, 1); mbar_init(bar_p, 4); mbar_init(bar_pv, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    att_tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+    att_tmem_relinquish();
+  }
+  att_fence_before();
+  __syncthreads();
+  att_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(bar_q, Q_BYTES);
+#pragma unroll
+      for (int b = 0; b < DB; ++b) att_tma_load_2d(sQ + b * Q_BOX, &tmap_q, b * 64, head * p.Nq + q0, bar_q);
+      int stage = 0; uint32_t phase = 0;
+      for (int j = 0; j < nblocks; ++j) {
+        if (!mbar_wait(bar_kv_empty + 8u * stage, phase ^ 1u, abort_flag, &g_attn_status_word, 0x1100u | stage)) break;
+        const uint32_t full = bar_kv_full + 8u * stage;
+        mbar_expect_tx(full, KV_BYTES);
+        const uint32_t dst = sKV + stage * KV_BYTES;
+#pragma unroll
+        for (int b = 0; b < DB; ++b) att_tma_load_2d(dst + b * K_BOX, &tmap_k, b * 64, head * p.Nk + j * W, full);
+#pragma unroll
+        for (int b = 0; b < WB; ++b) att_tma_load_2d(dst + K_BYTES + b * V_BOX, &tmap_vt, j * W + b * 64, head * HD, full);
+        if (++stage == KV_STAGES) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool alive = mbar_wait(bar_q, 0, abort_flag, &g_attn_status_word, 0x1200u);
+      int stage = 0; uint32_t phase = 0;
+      for (int j = 0; j < nblocks && alive; ++j) {
+        if (!mbar_wait(bar_kv_full + 8u * stage, phase, abort_flag, &g_attn_status_word, 0x1300u | stage)) break;
+        att_fence_after();
+        const uint32_t sK = sKV + stage * KV_BYTES, sV = sK + K_BYTES;
+        // S = Q K^T: ascending k over the head dimension, from zero
+#pragma unroll
+        for (int b = 0; b < DB; ++b) {
+          const uint64_t adesc = att_kmajor_desc(sQ + b * Q_BOX), bdesc = att_kmajor_desc(sK + b * K_BOX);
+#pragma unroll
+          for (int a = 0; a < 4; ++a) att_mma_bf16(tmem_base, adesc + 2u * a, bdesc + 2u * a, IDESC_S, (b | a) ? 1u : 0u);
+        }
+        att_commit(bar_s);
+        // PV = P Vt^T: ascending key over the block, from zero, once the probabilities are in shared memory
+        if (!mbar_wait(bar_p, j & 1, abort_flag, &g_attn_status_word, 0x1400u)) break;
+        att_fence_after();
+#pragma unroll
+        for (int b = 0; b < WB; ++b) {
+          const uint64_t adesc = att_kmajor_desc(sP + b * P_BOX), bdesc = att_kmajor_desc(sV + b * V_BOX);
+#pragma unroll
+          for (int a = 0; a < 4; ++a) att_mma_bf16(tmem_base + 128u, adesc + 2u * a, bdesc + 2u * a, IDESC_PV, (b | a) ? 1u : 0u);
+        }
+        att_commit(bar_pv);
+        att_commit(bar_kv_empty + 8u * stage);              // the stage may be refilled once these steps have read it
+        if (++stage == KV_STAGES) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ softmax and output rows
+    const int quarter = warp & 3;                           // TMEM lanes [32*quarter, 32*quarter + 32)
+    const int r = quarter * 32 + lane;                      // row of the tile
+    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    float m = -INFINITY, l = 0.0f;
+    float O[HD];
+#pragma unroll
+    for (int c = 0; c < HD; ++c) O[c] = 0.0f;
+    bool alive = true;
+    for (int j = 0; j < nblocks && alive; ++j) {
+      if (!mbar_wait(bar_s, j & 1, abort_flag, &g_attn_status_word, 0x1500u)) { alive = false; break; }
+      att_fence_after();
+      const int live = min(W, p.Nk - j * W);                // keys of this block that exist
+      // pass 1: the block's maximum
+      float mb = -INFINITY;
+#pragma unroll 1
+      for (int c0 = 0; c0 < W; c0 += 32) {
+        uint32_t raw[32];
+        att_tmem_ld32(t_row + c0, raw);
+        att_tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const float s = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
+          mb = fmaxf(mb, s);
+        }
+      }
+      const float m_new = fmaxf(m, mb);
+      const float alpha = rg_exp(f_add(m, -m_new));
+      // pass 2: probabilities, their row sum (balanced tree over the block's keys), narrowed copies
+      float chunk_sum[W / 32];
+#pragma unroll
+      for (int ci = 0; ci < W / 32; ++ci) {
+        const int c0 = ci * 32;
+        uint32_t raw[32];
+        att_tmem_ld32(t_row + c0, raw);
+        att_tmem_ld_wait();
+        float pr[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const float s = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
+          pr[c] = rg_exp(f_add(s, -m_new));
+        }
+        chunk_sum[ci] = tree32(pr);
+        // row r of the [128 x 64] box that holds keys c0..c0+31: four 16-byte pieces of 8 keys each
+        uint8_t* box = sP_gen + (c0 >> 6) * P_BOX + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int piece = ((c0 & 63) >> 3) + q;           // 16-byte piece of the 128-byte row
+          const uint4 v = make_uint4(pack_bf16x2(pr[8 * q], pr[8 * q + 1]), pack_bf16x2(pr[8 * q + 2], pr[8 * q + 3]),
+                                     pack_bf16x2(pr[8 * q + 4], pr[8 * q + 5]), pack_bf16x2(pr[8 * q + 6], pr[8 * q + 7]));
+          *reinterpret_cast<uint4*>(box + ((piece ^ (r & 7)) << 4)) = v;
+        }
+      }
+      float rowsum;
+      if (W == 128) rowsum = f_add(f_add(chunk_sum[0], chunk_sum[1]), f_add(chunk_sum[W / 32 - 2], chunk_sum[W / 32 - 1]));
+      else rowsum = f_add(chunk_sum[0], chunk_sum[1]);
+      l = f_add(f_mul(alpha, l), rowsum);
+      m = m_new;
+      // the tensor core reads shared memory through the async proxy
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      att_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_p);
+      // the block's P V product, then O = alpha * O + PV
+      if (!mbar_wait(bar_pv, j & 1, abort_flag, &g_attn_status_word, 0x1600u)) { alive = false; break; }
+      att_fence_after();
+#pragma unroll
+      for (int ci = 0; ci < HD / 32; ++ci) {
+        uint32_t raw[32];
+        att_tmem_ld32(t_row + 128u + ci * 32, raw);
+        att_tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) O[ci * 32 + c] = f_add(f_mul(alpha, O[ci * 32 + c]), __uint_as_float(raw[c]));
+      }
+      att_fence_before();
+    }
+    // one division at the end, one rounding to the output type
+    const int64_t row = (int64_t)q0 + r;
+    if (alive && row < p.Nq) {
+      const int64_t off = ((int64_t)head * p.Nq + row) * p.ldo;
+#pragma unroll
+      for (int ci = 0; ci < HD / 32; ++ci) {
+        float v[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) v[c] = __fdiv_rn(O[ci * 32 + c], l);
+        if (p.o_dtype == RG_F32) {
+          float* dst = static_cast<float*>(p.O) + off + ci * 32;
+#pragma unroll
+          for (int c = 0; c < 32; ++c) dst[c] = v[c];
+        } else {
+          uint16_t* dst = static_cast<uint16_t*>(p.O) + off + ci * 32;
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) *reinterpret_cast<uint32_t*>(dst + c) = pack_16x2(v[c], v[c + 1], p.o_dtype);
+        }
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  __syncthreads();
+  if (*abort_flag) {
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    att_fence_after();
+    att_tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+template <int W, int HD>
+size_t attn_smem_bytes() {
+  return 1024 + (HD / 64) * QROWS * 128 + KV_STAGES * ((HD / 64) * W * 128 + (W / 64) * HD * 128) + (W / 64) * QROWS * 128 + 8 * 8 + 16;
+}
+
+template <int W, int HD>
+cudaError_t launch_attention(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p, dim3 grid,
+                             cudaStream_t st) {
+  const size_t smem = attn_smem_bytes<W, HD>();
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel<W, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  attention_kernel<W, HD><<<grid, ATT_THREADS, smem, st>>>(tq, tk, tv, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// All arguments were validated by the caller: bf16 operands, d in {64, 128}, block_n in {64, 128},
+// 16-byte aligned pointers, leading dimensions multiples of 8.
+rg_status_t launch_attention_fixed(int block_n, float scale, int heads, const rg_tensor_t* Q, const rg_tensor_t* K,
+                                   const rg_tensor_t* Vt, const rg_tensor_t* O, cudaStream_t st) {
+  const int d = (int)Q->cols;
+  const int64_t Nq = Q->rows / heads, Nk = K->rows / heads;
+  CUtensorMap tq, tk, tv;
+  if (!make_operand_tmap(&tq, Q->ptr, Q->dtype, Q->rows, Q->cols, Q->ld, QROWS) ||
+      !make_operand_tmap(&tk, K->ptr, K->dtype, K->rows, K->cols, K->ld, block_n) ||
+      !make_operand_tmap(&tv, Vt->ptr, Vt->dtype, Vt->rows, Vt->cols, Vt->ld, d))
+    return RG_ERR_CUDA;
+  AttnParams p;
+  p.Nq = (int32_t)Nq; p.Nk = (int32_t)Nk; p.scale = scale;
+  p.O = O->ptr; p.ldo = O->ld; p.o_dtype = O->dtype;
+  const dim3 grid((unsigned)((Nq + QROWS - 1) / QROWS), (unsigned)heads, 1);
+  cudaError_t err;
+  if (block_n == 128 && d == 128) err = launch_attention<128, 128>(tq, tk, tv, p, grid, st);
+  else if (block_n == 64 && d == 128) err = launch_attention<64, 128>(tq, tk, tv, p, grid, st);
+  else if (block_n == 128 && d == 64) err = launch_attention<128, 64>(tq, tk, tv, p, grid, st);
+  else if (block_n == 64 && d == 64) err = launch_attention<64, 64>(tq, tk, tv, p, grid, st);
+  else return RG_ERR_UNSUPPORTED;
+  return err == cudaSuccess ? RG_OK : RG_ERR_CUDA;
+}
+
+rg_status_t read_and_clear_attn_status(uint32_t* code) {
+  unsigned int v = 0, zero = 0;
+  if (cudaMemcpyFromSymbol(&v, g_attn_status_word, sizeof(v)) != cudaSuccess) return RG_ERR_CUDA;
+  if (v != 0 && cudaMemcpyToSymbol(g_attn_status_word, &zero, sizeof(zero)) != cudaSuccess) return RG_ERR_CUDA;
+  if (code) *code = v;
+  return v ? RG_ERR_TIMEOUT : RG_OK;
+}
+
+}  // namespace rg

@@ -944,6 +944,11 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmP
 
 }  // namespace
 
+// The same tensor map for other kernels of the library (boxes of 64 columns x box_rows rows, 128-byte swizzle).
+bool make_operand_tmap(CUtensorMap_st* map, const void* ptr, int dtype, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+  return make_tmap(map, ptr, dtype, rows, cols, ld, box_rows);
+}
+
 int a_box_rows_for(int64_t M) { return M >= BM ? BM : (int)((M + 7) / 8 * 8); }
 
 int max_stages_for(int bn, int bk, int cta_group, int64_t M) {
