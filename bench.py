@@ -504,6 +504,13 @@ def run_only(args):
             it[0] += 1
             rg.rg_gemm(d, A, Ws[it[0] % 4], Cm)
         work, unit = 2.0 * N * K / 1e9, "GB/s (weights)"
+    elif name == "attention":
+        H, Nq, Nk, hd = 32, 4096, 4096, 128
+        Q = synth.device_normal((H * Nq, hd), 1.0, 21, bf, dev); Kt = synth.device_normal((H * Nk, hd), 1.0, 22, bf, dev)
+        Vt = synth.device_normal((H * hd, Nk), 1.0, 23, bf, dev); O = torch.empty((H * Nq, hd), dtype=bf, device=dev)
+        ad = rg.rg_attn_desc(block_n=args.attn_block, scale=hd ** -0.5, heads=H)
+        fn = lambda: rg.rg_attention(ad, Q, Kt, Vt, O)
+        work, unit = 4.0 * H * Nq * Nk * hd / 1e12, "TFLOP/s"
     elif name in ("col_sum", "col_dot"):
         R_, C_ = 65536, 8192
         x = synth.device_normal((R_, C_), 100.0, 13, f32, dev)
@@ -551,9 +558,10 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_square_f8", "gemm_prefill", "gemm_decode", "gemv_decode", "col_sum", "col_dot", "row_sum", "softmax", "softmax_unit", "rmsnorm"],
+    ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_square_f8", "gemm_prefill", "gemm_decode", "gemv_decode", "attention", "col_sum", "col_dot", "row_sum", "softmax", "softmax_unit", "rmsnorm"],
                     help="run one kernel on a small case (used for the ncu captures)")
     ap.add_argument("--gemv-rows", type=int, default=1, help="rows of A for --only gemv_decode")
+    ap.add_argument("--attn-block", type=int, default=128, help="key block width for --only attention")
     args = ap.parse_args()
     if args.only:
         run_only(args)
