@@ -7,7 +7,9 @@
 //   warp 0 (TMA)      K_j [w x d] and Vt_j [d x w] boxes into a two-stage ring (Q once)
 //   warp 1 (MMA)      S = Q K_j^T   d/16 tcgen05.mma steps from a zero accumulator, ascending k
 //                     PV = P Vt_j^T w/16 steps from a zero accumulator, ascending key
-//   warps 2-5         one query row per thread (its TMEM lane):
+//   warps 2-9         two threads per query row (its TMEM lane), each with half of the block's keys and
+//                     half of the output columns; partial maxima and partial row sums (subtrees of
+//                     the same tree) meet in shared memory:
 //                     s_t = acc * scale; m_j = max(m_{j-1}, max_t s_t); alpha = exp(m_{j-1} - m_j);
 //                     p_t = exp(s_t - m_j); l_j = alpha*l_{j-1} + TREE_t p_t (balanced tree over the
 //                     block's keys in order); P = p narrowed to bf16, written to shared memory in the
@@ -32,7 +34,8 @@ __device__ unsigned int g_attn_status_word = 0;
 namespace {
 
 constexpr int QROWS = 128;          // query rows per CTA = TMEM lanes
-constexpr int ATT_THREADS = 192;    // warp 0 TMA, warp 1 MMA, warps 2-5 softmax
+constexpr int ATT_THREADS = 320;    // warp 0 TMA, warp 1 MMA, warps 2-9 softmax (two threads per query row)
+constexpr int SOFTMAX_THREADS = 256;
 constexpr int KV_STAGES = 2;
 
 // ---- PTX wrappers (tensor core side)
@@ -140,6 +143,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   const uint32_t bar_s = bar_kv_empty + 8u * KV_STAGES, bar_p = bar_s + 8u, bar_pv = bar_p + 8u;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* xm = reinterpret_cast<float*>(bars + 10);        // [2][128] partial maxima of the two halves of a row
+  float* xs = xm + 2 * QROWS;                             // [2][128] partial row sums
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int head = blockIdx.y;
@@ -149,7 +154,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
     for (int s = 0; s < KV_STAGES; ++s) { mbar_init(bar_kv_full + 8u * s, 1); mbar_init(bar_kv_empty + 8u * s, 1); }
-    mbar_init(bar_s, 1); mbar_init(bar_p, 4); mbar_init(bar_pv, 1);
+    mbar_init(bar_s, 1); mbar_init(bar_p, SOFTMAX_THREADS / 32); mbar_init(bar_pv, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -215,86 +220,99 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   } else {
     // ------------------------------------------------------------ softmax and output rows
     const int quarter = warp & 3;                           // TMEM lanes [32*quarter, 32*quarter + 32)
+    const int half = (warp - 2) >> 2;                       // which half of the keys and of the output columns
     const int r = quarter * 32 + lane;                      // row of the tile
     const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    constexpr int KH = W / 2, OH = HD / 2;                  // keys and output columns per thread
+    const int kbase = half * KH, obase = half * OH;
     float m = -INFINITY, l = 0.0f;
-    float O[HD];
+    float O[OH];
 #pragma unroll
-    for (int c = 0; c < HD; ++c) O[c] = 0.0f;
+    for (int c = 0; c < OH; ++c) O[c] = 0.0f;
+    // A wait that gives up leaves this thread walking the loop without touching tensor memory, so
+    // that the 256-thread barriers below are still met by everyone.
     bool alive = true;
-    for (int j = 0; j < nblocks && alive; ++j) {
-      if (!mbar_wait(bar_s, j & 1, abort_flag, &g_attn_status_word, 0x1500u)) { alive = false; break; }
-      att_fence_after();
+    for (int j = 0; j < nblocks; ++j) {
+      if (alive) alive = mbar_wait(bar_s, j & 1, abort_flag, &g_attn_status_word, 0x1500u);
       const int live = min(W, p.Nk - j * W);                // keys of this block that exist
-      // pass 1: the block's maximum
+      // pass 1: the maximum over this thread's keys, then over the row
       float mb = -INFINITY;
-#pragma unroll 1
-      for (int c0 = 0; c0 < W; c0 += 32) {
-        uint32_t raw[32];
-        att_tmem_ld32(t_row + c0, raw);
-        att_tmem_ld_wait();
+      if (alive) {
+        att_fence_after();
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const float s = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
-          mb = fmaxf(mb, s);
+        for (int c0 = 0; c0 < KH; c0 += 32) {
+          uint32_t raw[32];
+          att_tmem_ld32(t_row + kbase + c0, raw);
+          att_tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            const float sc = kbase + c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
+            mb = fmaxf(mb, sc);
+          }
         }
       }
-      const float m_new = fmaxf(m, mb);
+      xm[half * QROWS + r] = mb;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      const float m_new = fmaxf(m, fmaxf(xm[r], xm[QROWS + r]));
       const float alpha = rg_exp(f_add(m, -m_new));
-      // pass 2: probabilities, their row sum (balanced tree over the block's keys), narrowed copies
-      float chunk_sum[W / 32];
+      // pass 2: probabilities, the subtree of the row sum over this thread's keys, narrowed copies
+      float part = 0.0f;
+      if (alive) {
+        float chunk_sum[KH / 32];
 #pragma unroll
-      for (int ci = 0; ci < W / 32; ++ci) {
-        const int c0 = ci * 32;
-        uint32_t raw[32];
-        att_tmem_ld32(t_row + c0, raw);
-        att_tmem_ld_wait();
-        float pr[32];
+        for (int ci = 0; ci < KH / 32; ++ci) {
+          const int c0 = kbase + ci * 32;
+          uint32_t raw[32];
+          att_tmem_ld32(t_row + c0, raw);
+          att_tmem_ld_wait();
+          float pr[32];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const float s = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
-          pr[c] = rg_exp(f_add(s, -m_new));
+          for (int c = 0; c < 32; ++c) {
+            const float sc = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
+            pr[c] = rg_exp(f_add(sc, -m_new));
+          }
+          chunk_sum[ci] = tree32(pr);
+          // row r of the [128 x 64] box that holds keys c0..c0+31: four 16-byte pieces of 8 keys each
+          uint8_t* box = sP_gen + (c0 >> 6) * P_BOX + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int piece = ((c0 & 63) >> 3) + q;         // 16-byte piece of the 128-byte row
+            const uint4 v = make_uint4(pack_bf16x2(pr[8 * q], pr[8 * q + 1]), pack_bf16x2(pr[8 * q + 2], pr[8 * q + 3]),
+                                       pack_bf16x2(pr[8 * q + 4], pr[8 * q + 5]), pack_bf16x2(pr[8 * q + 6], pr[8 * q + 7]));
+            *reinterpret_cast<uint4*>(box + ((piece ^ (r & 7)) << 4)) = v;
+          }
         }
-        chunk_sum[ci] = tree32(pr);
-        // row r of the [128 x 64] box that holds keys c0..c0+31: four 16-byte pieces of 8 keys each
-        uint8_t* box = sP_gen + (c0 >> 6) * P_BOX + (r >> 3) * 1024 + (r & 7) * 128;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int piece = ((c0 & 63) >> 3) + q;           // 16-byte piece of the 128-byte row
-          const uint4 v = make_uint4(pack_bf16x2(pr[8 * q], pr[8 * q + 1]), pack_bf16x2(pr[8 * q + 2], pr[8 * q + 3]),
-                                     pack_bf16x2(pr[8 * q + 4], pr[8 * q + 5]), pack_bf16x2(pr[8 * q + 6], pr[8 * q + 7]));
-          *reinterpret_cast<uint4*>(box + ((piece ^ (r & 7)) << 4)) = v;
-        }
+        part = KH == 64 ? f_add(chunk_sum[0], chunk_sum[KH / 32 - 1]) : chunk_sum[0];
       }
-      float rowsum;
-      if (W == 128) rowsum = f_add(f_add(chunk_sum[0], chunk_sum[1]), f_add(chunk_sum[W / 32 - 2], chunk_sum[W / 32 - 1]));
-      else rowsum = f_add(chunk_sum[0], chunk_sum[1]);
-      l = f_add(f_mul(alpha, l), rowsum);
-      m = m_new;
+      xs[half * QROWS + r] = part;
       // the tensor core reads shared memory through the async proxy
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       att_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_p);
-      // the block's P V product, then O = alpha * O + PV
-      if (!mbar_wait(bar_pv, j & 1, abort_flag, &g_attn_status_word, 0x1600u)) { alive = false; break; }
-      att_fence_after();
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (lane == 0 && alive) mbar_arrive(bar_p);
+      l = f_add(f_mul(alpha, l), f_add(xs[r], xs[QROWS + r]));
+      m = m_new;
+      // the block's P V product, then O = alpha * O + PV on this thread's output columns
+      if (alive) alive = mbar_wait(bar_pv, j & 1, abort_flag, &g_attn_status_word, 0x1600u);
+      if (alive) {
+        att_fence_after();
 #pragma unroll
-      for (int ci = 0; ci < HD / 32; ++ci) {
-        uint32_t raw[32];
-        att_tmem_ld32(t_row + 128u + ci * 32, raw);
-        att_tmem_ld_wait();
+        for (int ci = 0; ci < OH / 32; ++ci) {
+          uint32_t raw[32];
+          att_tmem_ld32(t_row + 128u + obase + ci * 32, raw);
+          att_tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < 32; ++c) O[ci * 32 + c] = f_add(f_mul(alpha, O[ci * 32 + c]), __uint_as_float(raw[c]));
+          for (int c = 0; c < 32; ++c) O[ci * 32 + c] = f_add(f_mul(alpha, O[ci * 32 + c]), __uint_as_float(raw[c]));
+        }
+        att_fence_before();
       }
-      att_fence_before();
     }
     // one division at the end, one rounding to the output type
     const int64_t row = (int64_t)q0 + r;
     if (alive && row < p.Nq) {
-      const int64_t off = ((int64_t)head * p.Nq + row) * p.ldo;
+      const int64_t off = ((int64_t)head * p.Nq + row) * p.ldo + obase;
 #pragma unroll
-      for (int ci = 0; ci < HD / 32; ++ci) {
+      for (int ci = 0; ci < OH / 32; ++ci) {
         float v[32];
 #pragma unroll
         for (int c = 0; c < 32; ++c) v[c] = __fdiv_rn(O[ci * 32 + c], l);
@@ -326,7 +344,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
 template <int W, int HD>
 size_t attn_smem_bytes() {
-  return 1024 + (HD / 64) * QROWS * 128 + KV_STAGES * ((HD / 64) * W * 128 + (W / 64) * HD * 128) + (W / 64) * QROWS * 128 + 8 * 8 + 16;
+  return 1024 + (HD / 64) * QROWS * 128 + KV_STAGES * ((HD / 64) * W * 128 + (W / 64) * HD * 128) + (W / 64) * QROWS * 128 + 10 * 8 + 4 * QROWS * 4;
 }
 
 template <int W, int HD>
