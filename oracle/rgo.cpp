@@ -445,6 +445,27 @@ float rg_expf(float x) {
   return (p * s1) * s2;
 }
 
+// Base-two exponential, fixed the same way (App. F: attention kernels fold log2 e into the score
+// scale and take a base-two exponential): n = rint(x); f = x - n (exact, |f| <= 1/2);
+// p = degree-7 Taylor polynomial of 2^f = exp(f ln 2) (Horner, fused); result = p * 2^n, an exact
+// scaling.  2^x for x < -126 is 0 and for x >= 128 is +inf; integers give exact powers of two.
+float rg_exp2f(float x) {
+  if (x != x) return x;
+  if (x >= 128.0f) return INFINITY;
+  if (x < -126.0f) return 0.0f;
+  float n = std::nearbyintf(x);
+  float f = x - n;
+  float p = 0x1.ffcbfcp-17f;              // (ln 2)^7 / 5040
+  p = std::fmaf(p, f, 0x1.430912p-13f);   // (ln 2)^6 / 720
+  p = std::fmaf(p, f, 0x1.5d87fep-10f);   // (ln 2)^5 / 120
+  p = std::fmaf(p, f, 0x1.3b2ab6p-7f);    // (ln 2)^4 / 24
+  p = std::fmaf(p, f, 0x1.c6b08ep-5f);    // (ln 2)^3 / 6
+  p = std::fmaf(p, f, 0x1.ebfbe0p-3f);    // (ln 2)^2 / 2
+  p = std::fmaf(p, f, 0x1.62e430p-1f);    // ln 2
+  p = std::fmaf(p, f, 1.0f);
+  return std::ldexp(p, int(n));           // exact: p in [0.70, 1.42], the result is a normal number
+}
+
 inline float silu(float v) { return v / (1.0f + rg_expf(-v)); }
 
 // ------------------------------------------------------------------- GEMM
@@ -524,6 +545,7 @@ uint16_t rgo_f32_to_f16(float f) { return f32_to_f16(f); }
 float rgo_add_f32(float a, float b) { return a + b; }
 float rgo_mul_f32(float a, float b) { return a * b; }
 float rgo_expf(float x) { return rg_expf(x); }
+float rgo_exp2f(float x) { return rg_exp2f(x); }
 float rgo_silu(float x) { return silu(x); }
 
 // Tree-reduce n fp32 values (input is not modified).
@@ -744,7 +766,8 @@ void rgo_reduce_cols(int op, int tree, int fma, const void* x, int x_dtype, cons
 //   s_t   = scale * (q . k_t)         the contraction is a chain of tensor-core steps over the head
 //                                     dimension from a zero accumulator (Sec. 3.2.1), then one multiply
 //   m_j   = max(m_{j-1}, max_t s_t)   a maximum rounds nothing
-//   alpha = exp(m_{j-1} - m_j),  p_t = exp(s_t - m_j)          (exp as fixed by this library)
+//   alpha = exp(m_{j-1} - m_j),  p_t = exp(s_t - m_j)          (exp as fixed by this library: base e,
+//                                     or base two with log2 e folded into `scale` by the caller)
 //   l_j   = alpha * l_{j-1} + TREE_t p_t                        (the block's row sum in the given tree)
 //   P_t   = p_t narrowed to p_dtype                             (the operand type of the second product)
 //   O_j   = alpha * O_{j-1} + (P . V)_block                     the block's product is a chain of steps
@@ -752,7 +775,7 @@ void rgo_reduce_cols(int op, int tree, int fma, const void* x, int x_dtype, cons
 // and the answer is O_B / l_B, divided once at the end and rounded once to the output type.
 // Keys past Nk in the last block are absent: their scores are -inf, their probabilities exactly 0.
 // Vt is V transposed: [d, Nk], keys contiguous.
-void rgo_attention(const AtomModel* atom, int block_n, int sum_tree, int p_dtype, float scale,
+void rgo_attention(const AtomModel* atom, int block_n, int sum_tree, int p_dtype, int exp_base, float scale,
                    int64_t Nq, int64_t Nk, int64_t d, const uint16_t* Q, int64_t ldq, const uint16_t* K, int64_t ldk,
                    const uint16_t* Vt, int64_t ldv, void* O, int o_dtype, int64_t ldo) {
   const int ak = atom->atom_k;
@@ -773,9 +796,9 @@ void rgo_attention(const AtomModel* atom, int block_n, int sum_tree, int p_dtype
         mb = std::max(mb, s[t]);
       }
       const float m_new = std::max(m, mb);
-      const float alpha = rg_expf(m - m_new);
+      const float alpha = exp_base == 2 ? rg_exp2f(m - m_new) : rg_expf(m - m_new);
       std::vector<float> leaf(n);
-      for (int t = 0; t < n; ++t) { pf[t] = rg_expf(s[t] - m_new); leaf[t] = pf[t]; }
+      for (int t = 0; t < n; ++t) { pf[t] = exp_base == 2 ? rg_exp2f(s[t] - m_new) : rg_expf(s[t] - m_new); leaf[t] = pf[t]; }
       const float rowsum = tree_reduce(leaf, sum_tree);
       l = alpha * l + rowsum;
       for (int t = 0; t < n; ++t) pn[t] = p_dtype == DT_F16 ? f32_to_f16(pf[t]) : f32_to_bf16(pf[t]);

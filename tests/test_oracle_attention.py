@@ -94,3 +94,19 @@ def test_ragged_last_block_and_row_independence():
     Kx = np.concatenate([K, _bf(np.full((42, d), -100.0) * np.sign(synth.bf16_bits_to_f32(Q[0]))[None, :])])
     far = rgo.attention(Q[:1], Kx, np.concatenate([V, V[:42]]), block_n=64, scale=0.2, atom_model=rgo.TCGEN05_BF16_B200)
     assert np.array_equal(far, full[:1])
+
+
+def test_base_two_exponential_variant():
+    g = np.random.default_rng(12)
+    d, Nk = 64, 300
+    Q, K, V = _bf(g.standard_normal((5, d))), _bf(g.standard_normal((Nk, d))), _bf(g.standard_normal((Nk, d)))
+    scale = d ** -0.5
+    e = rgo.attention(Q, K, V, block_n=128, scale=scale, atom_model=rgo.TCGEN05_BF16_B200, out_dtype=rgo.F32)
+    b2 = rgo.attention(Q, K, V, block_n=128, scale=np.float32(scale * np.log2(np.e)), atom_model=rgo.TCGEN05_BF16_B200, out_dtype=rgo.F32, exp_base=2)
+    ref = _ref64(Q, K, V, scale)
+    assert not np.array_equal(e, b2)                      # another class of bits
+    assert np.max(np.abs(b2 - ref)) <= 2.0 ** -8 * np.max(np.abs(_f(V))) + 1e-6
+    # uniform keys: probabilities 2^0 = 1 exactly, so the closed form holds in base two as well
+    Ku = _bf(np.tile(np.linspace(-1, 1, d, dtype=np.float32), (256, 1))); v = np.arange(d, dtype=np.float32) / 4
+    out = rgo.attention(_bf(np.ones((2, d))), Ku, _bf(np.tile(v, (256, 1))), block_n=64, scale=0.3, out_dtype=rgo.F32, exp_base=2)
+    assert np.array_equal(out, np.tile(v, (2, 1)))

@@ -137,3 +137,21 @@ def test_f8e4m3_widening_exhaustive_and_landmarks():
     assert rgo.f8e4m3_to_f32(0x01) == 2.0 ** -9 and rgo.f8e4m3_to_f32(0x07) == 7 * 2.0 ** -9
     assert rgo.f8e4m3_to_f32(0x08) == 2.0 ** -6 and rgo.f8e4m3_to_f32(0x38) == 1.0 and rgo.f8e4m3_to_f32(0x3c) == 1.5
     assert np.float32(rgo.f8e4m3_to_f32(0x80)).view(np.uint32) == 0x80000000
+
+
+def test_exp2f_accuracy_exact_powers_monotone_and_clamps():
+    g = np.random.default_rng(4)
+    x = np.concatenate([g.uniform(-126, 128, 200000), g.uniform(-2, 2, 100000), g.uniform(-40, 0, 100000)]).astype(np.float32)
+    got = np.array([rgo.exp2f(v) for v in x], dtype=np.float32)
+    ref = np.exp2(x.astype(np.float64))
+    ulp = np.spacing(ref.astype(np.float32)).astype(np.float64)
+    assert np.max(np.abs(got.astype(np.float64) - ref) / ulp) <= 2.0
+    for n in range(-126, 128):                                   # integers: exact powers of two
+        assert rgo.exp2f(n) == np.float32(2.0) ** n
+    assert rgo.exp2f(0.5) == np.float32(np.sqrt(2.0)) or abs(float(rgo.exp2f(0.5)) - 2 ** 0.5) < 2e-7
+    grid = np.linspace(-30, 30, 200001).astype(np.float32)
+    vals = np.array([rgo.exp2f(v) for v in grid], dtype=np.float32)
+    assert np.all(np.diff(vals) >= 0)
+    assert rgo.exp2f(-126.0) == np.float32(2.0 ** -126) and rgo.exp2f(np.float32(-126.00001)) == 0 and rgo.exp2f(-1e30) == 0
+    assert rgo.exp2f(-np.inf) == 0 and np.isinf(rgo.exp2f(128.0)) and np.isinf(rgo.exp2f(np.inf)) and np.isnan(rgo.exp2f(np.nan))
+    assert rgo.exp2f(np.float32(127.99999)) < np.inf
