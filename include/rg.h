@@ -204,7 +204,8 @@ rg_status_t rg_reduce_cols(const rg_desc_t* d, rg_col_op_t op, const rg_tensor_t
  *   O_j = alpha * O_{j-1} + (P . V)_block       (P = p narrowed to `p_dtype`)
  * and the answer is O_B / l_B: one division at the end, one rounding to O's type.  Both products are
  * chains of tensor-core steps from a zero accumulator (RG_ATOM_TC_BF16_K16): over the head dimension
- * for the scores, over the block's keys for P . V.  exp is the exponential this library fixes, base e.
+ * for the scores, over the block's keys for P . V.  exp is an exponential this library fixes from IEEE
+ * operations: base e, or base two (`exp_base`), a cheaper polynomial and another class of bits.
  * Every block boundary is a rounding of O and l, so block_n is part of the class of bits; the query
  * tile is not (no masking here: `mask` must be 0).
  *
@@ -221,6 +222,8 @@ typedef struct {
   uint8_t p_dtype;        /* type the probabilities are narrowed to: RG_BF16 */
   uint8_t mask;           /* 0 = none */
   uint8_t div_place;      /* 0 = once, at the end */
+  uint8_t exp_base;       /* 0 = base e; 2 = base two (the caller folds log2 e into `scale`, App. F) */
+  uint8_t _pad[3];
 } rg_attn_desc_t;
 rg_status_t rg_attention(const rg_attn_desc_t* d, const rg_tensor_t* Q, const rg_tensor_t* K, const rg_tensor_t* Vt,
                          const rg_tensor_t* O, void* cuda_stream);

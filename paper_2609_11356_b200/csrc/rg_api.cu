@@ -277,6 +277,7 @@ rg_status_t rg_attention(const rg_attn_desc_t* d, const rg_tensor_t* Q, const rg
     return s;
   if (d->sum_tree != RG_TREE_BALANCED || d->p_dtype != RG_BF16 || d->mask != 0 || d->div_place != 0) return RG_ERR_UNSUPPORTED;
   if (d->block_n != 64 && d->block_n != 128) return RG_ERR_UNSUPPORTED;
+  if (d->exp_base != 0 && d->exp_base != 2) return RG_ERR_INVALID_DESC;
   if (Q->dtype != RG_BF16 || K->dtype != RG_BF16 || Vt->dtype != RG_BF16) return RG_ERR_UNSUPPORTED;
   const int64_t hd = Q->cols, H = d->heads;
   if (hd != 64 && hd != 128) return RG_ERR_UNSUPPORTED;
@@ -288,7 +289,7 @@ rg_status_t rg_attention(const rg_attn_desc_t* d, const rg_tensor_t* Q, const rg
       (reinterpret_cast<uintptr_t>(Vt->ptr) & 15) || (reinterpret_cast<uintptr_t>(O->ptr) & 15) ||
       (Q->ld % 8) || (K->ld % 8) || (Vt->ld % 8) || (O->ld % 8))
     return RG_ERR_ALIGNMENT;
-  return rg::launch_attention_fixed((int)d->block_n, d->scale, (int)H, Q, K, Vt, O, static_cast<cudaStream_t>(cuda_stream));
+  return rg::launch_attention_fixed((int)d->block_n, (int)d->exp_base, d->scale, (int)H, Q, K, Vt, O, static_cast<cudaStream_t>(cuda_stream));
 }
 
 // ------------------------------------------------------------ host-buffer forms

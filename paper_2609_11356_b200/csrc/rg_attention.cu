@@ -14,8 +14,8 @@
 //                     p_t = exp(s_t - m_j); l_j = alpha*l_{j-1} + TREE_t p_t (balanced tree over the
 //                     block's keys in order); P = p narrowed to bf16, written to shared memory in the
 //                     swizzled K-major layout the tensor core reads; O_j = alpha*O_{j-1} + PV
-// and at the end O / l, one division, one rounding to the output type.  exp is the library's
-// specified exponential (rg_exp), not the hardware's base-two one.  Keys past Nk are masked to
+// and at the end O / l, one division, one rounding to the output type.  exp is one of the library's
+// specified exponentials (rg_exp, or rg_exp2 with log2 e folded into the scale), not the hardware's.  Keys past Nk are masked to
 // -inf before the maximum, so their probabilities are exactly +0.
 //
 // Heads are stacked along the rows of Q [heads*Nq, d], K [heads*Nk, d], Vt [heads*d, Nk] and
@@ -116,8 +116,8 @@ __device__ __forceinline__ float tree32(const float (&p)[32]) {
   return f_add(f_add(a[0], a[1]), f_add(a[2], a[3]));
 }
 
-// W = key block width (64 or 128), HD = head dimension (64 or 128)
-template <int W, int HD>
+// W = key block width (64 or 128), HD = head dimension (64 or 128), BASE2 = base-two exponential
+template <int W, int HD, bool BASE2>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                  const __grid_constant__ CUtensorMap tmap_vt, const AttnParams p) {
@@ -254,7 +254,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       xm[half * QROWS + r] = mb;
       asm volatile("bar.sync 1, 256;" ::: "memory");
       const float m_new = fmaxf(m, fmaxf(xm[r], xm[QROWS + r]));
-      const float alpha = rg_exp(f_add(m, -m_new));
+      const float alpha = BASE2 ? rg_exp2(f_add(m, -m_new)) : rg_exp(f_add(m, -m_new));
       // pass 2: probabilities, the subtree of the row sum over this thread's keys, narrowed copies
       float part = 0.0f;
       if (alive) {
@@ -269,7 +269,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 #pragma unroll
           for (int c = 0; c < 32; ++c) {
             const float sc = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
-            pr[c] = rg_exp(f_add(sc, -m_new));
+            pr[c] = BASE2 ? rg_exp2(f_add(sc, -m_new)) : rg_exp(f_add(sc, -m_new));
           }
           chunk_sum[ci] = tree32(pr);
           // row r of the [128 x 64] box that holds keys c0..c0+31: four 16-byte pieces of 8 keys each
@@ -347,17 +347,17 @@ size_t attn_smem_bytes() {
   return 1024 + (HD / 64) * QROWS * 128 + KV_STAGES * ((HD / 64) * W * 128 + (W / 64) * HD * 128) + (W / 64) * QROWS * 128 + 10 * 8 + 4 * QROWS * 4;
 }
 
-template <int W, int HD>
+template <int W, int HD, bool BASE2>
 cudaError_t launch_attention(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p, dim3 grid,
                              cudaStream_t st) {
   const size_t smem = attn_smem_bytes<W, HD>();
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attention_kernel<W, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel<W, HD, BASE2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  attention_kernel<W, HD><<<grid, ATT_THREADS, smem, st>>>(tq, tk, tv, p);
+  attention_kernel<W, HD, BASE2><<<grid, ATT_THREADS, smem, st>>>(tq, tk, tv, p);
   return cudaGetLastError();
 }
 
@@ -365,7 +365,7 @@ cudaError_t launch_attention(const CUtensorMap& tq, const CUtensorMap& tk, const
 
 // All arguments were validated by the caller: bf16 operands, d in {64, 128}, block_n in {64, 128},
 // 16-byte aligned pointers, leading dimensions multiples of 8.
-rg_status_t launch_attention_fixed(int block_n, float scale, int heads, const rg_tensor_t* Q, const rg_tensor_t* K,
+rg_status_t launch_attention_fixed(int block_n, int exp_base, float scale, int heads, const rg_tensor_t* Q, const rg_tensor_t* K,
                                    const rg_tensor_t* Vt, const rg_tensor_t* O, cudaStream_t st) {
   const int d = (int)Q->cols;
   const int64_t Nq = Q->rows / heads, Nk = K->rows / heads;
@@ -379,10 +379,11 @@ rg_status_t launch_attention_fixed(int block_n, float scale, int heads, const rg
   p.O = O->ptr; p.ldo = O->ld; p.o_dtype = O->dtype;
   const dim3 grid((unsigned)((Nq + QROWS - 1) / QROWS), (unsigned)heads, 1);
   cudaError_t err;
-  if (block_n == 128 && d == 128) err = launch_attention<128, 128>(tq, tk, tv, p, grid, st);
-  else if (block_n == 64 && d == 128) err = launch_attention<64, 128>(tq, tk, tv, p, grid, st);
-  else if (block_n == 128 && d == 64) err = launch_attention<128, 64>(tq, tk, tv, p, grid, st);
-  else if (block_n == 64 && d == 64) err = launch_attention<64, 64>(tq, tk, tv, p, grid, st);
+  const bool b2 = exp_base == 2;
+  if (block_n == 128 && d == 128) err = b2 ? launch_attention<128, 128, true>(tq, tk, tv, p, grid, st) : launch_attention<128, 128, false>(tq, tk, tv, p, grid, st);
+  else if (block_n == 64 && d == 128) err = b2 ? launch_attention<64, 128, true>(tq, tk, tv, p, grid, st) : launch_attention<64, 128, false>(tq, tk, tv, p, grid, st);
+  else if (block_n == 128 && d == 64) err = b2 ? launch_attention<128, 64, true>(tq, tk, tv, p, grid, st) : launch_attention<128, 64, false>(tq, tk, tv, p, grid, st);
+  else if (block_n == 64 && d == 64) err = b2 ? launch_attention<64, 64, true>(tq, tk, tv, p, grid, st) : launch_attention<64, 64, false>(tq, tk, tv, p, grid, st);
   else return RG_ERR_UNSUPPORTED;
   return err == cudaSuccess ? RG_OK : RG_ERR_CUDA;
 }

@@ -47,6 +47,29 @@ __device__ __forceinline__ float rg_exp(float x) {
   return x != x ? x : e;
 }
 
+// Base-two exponential fixed the same way (attention folds log2 e into the score scale, App. F):
+// n = rint(x), f = x - n (exact), degree-7 Taylor polynomial of 2^f in Horner form with fused
+// multiply-adds, and an exact scaling by 2^n done on the exponent field (the polynomial lies in
+// [0.70, 1.42] and n in [-126, 128], so the result is a normal number or overflows to the clamp).
+__device__ __forceinline__ float rg_exp2(float x) {
+  const float t = f_add(x, 12582912.0f);                // round to nearest-even integer
+  const float n = f_add(t, -12582912.0f);
+  const float f = f_add(x, -n);
+  float p = 0x1.ffcbfcp-17f;
+  p = f_fma(p, f, 0x1.430912p-13f);
+  p = f_fma(p, f, 0x1.5d87fep-10f);
+  p = f_fma(p, f, 0x1.3b2ab6p-7f);
+  p = f_fma(p, f, 0x1.c6b08ep-5f);
+  p = f_fma(p, f, 0x1.ebfbe0p-3f);
+  p = f_fma(p, f, 0x1.62e430p-1f);
+  p = f_fma(p, f, 1.0f);
+  const int ni = __float_as_int(t) - 0x4B400000;        // the integer n, read from t's mantissa
+  float e = __int_as_float(__float_as_int(p) + (ni << 23));
+  e = x < -126.0f ? 0.0f : e;
+  e = x >= 128.0f ? __int_as_float(0x7f800000) : e;
+  return x != x ? x : e;
+}
+
 __device__ __forceinline__ float rg_silu(float v) { return __fdiv_rn(v, f_add(1.0f, rg_exp(-v))); }
 
 // Epilogue operands, passed by value to kernels.

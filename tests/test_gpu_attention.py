@@ -12,7 +12,7 @@ from tests._gpu_util import DEV, HW, assert_bits_equal
 pytestmark = pytest.mark.gpu
 
 
-def gpu_attention(Q, K, V, *, block_n, scale, heads=1, out_dtype=rgo.BF16):
+def gpu_attention(Q, K, V, *, block_n, scale, heads=1, out_dtype=rgo.BF16, exp_base=0):
     """Q [heads*Nq, d], K [heads*Nk, d], V [heads*Nk, d] as bf16 bit patterns."""
     d = Q.shape[1]; Nk = K.shape[0] // heads
     Vt = np.ascontiguousarray(V.reshape(heads, Nk, d).transpose(0, 2, 1)).reshape(heads * d, Nk)
@@ -22,7 +22,7 @@ def gpu_attention(Q, K, V, *, block_n, scale, heads=1, out_dtype=rgo.BF16):
     tdt = {rgo.BF16: torch.bfloat16, rgo.F32: torch.float32, rgo.F16: torch.float16}[out_dtype]
     O = torch.empty((Q.shape[0], d), dtype=tdt, device=DEV)
     O.view(torch.int32 if out_dtype == rgo.F32 else torch.int16).fill_(-1)
-    rg.rg_attention(rg.rg_attn_desc(block_n=block_n, scale=scale, heads=heads), synth.to_torch(Q, DEV), synth.to_torch(K, DEV), vt[:, :Nk], O)
+    rg.rg_attention(rg.rg_attn_desc(block_n=block_n, scale=scale, heads=heads, exp_base=exp_base), synth.to_torch(Q, DEV), synth.to_torch(K, DEV), vt[:, :Nk], O)
     torch.cuda.synchronize()
     return synth.from_torch(O)
 
@@ -42,6 +42,15 @@ def test_single_head_bit_exact(Nq, Nk, d, w):
         got = gpu_attention(Q, K, V, block_n=w, scale=scale, out_dtype=out)
         want = rgo.attention(Q, K, V, block_n=w, scale=scale, atom_model=HW, out_dtype=out)
         assert_bits_equal(got, want, f"attention {Nq}x{Nk} d={d} w={w} out={out}")
+
+
+@pytest.mark.parametrize("Nq,Nk,d,w", [(128, 128, 128, 128), (5, 37, 128, 64), (257, 1000, 64, 128), (300, 520, 128, 64)])
+def test_base_two_variant_bit_exact(Nq, Nk, d, w):
+    Q, K, V = _draw(Nq, Nk, d, 17 + Nq + Nk)
+    scale = float(np.float32(d ** -0.5 * np.log2(np.e)))
+    got = gpu_attention(Q, K, V, block_n=w, scale=scale, out_dtype=rgo.F32, exp_base=2)
+    want = rgo.attention(Q, K, V, block_n=w, scale=scale, atom_model=HW, out_dtype=rgo.F32, exp_base=2)
+    assert_bits_equal(got, want, f"attention base two {Nq}x{Nk} d={d} w={w}")
 
 
 def test_heads_block_width_and_spread_inputs():
