@@ -244,10 +244,15 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
           uint32_t raw[32];
           att_tmem_ld32(t_row + kbase + c0, raw);
           att_tmem_ld_wait();
+          if (live == W) {                                  // every key exists: no masking (all blocks but the last)
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const float sc = kbase + c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
-            mb = fmaxf(mb, sc);
+            for (int c = 0; c < 32; ++c) mb = fmaxf(mb, f_mul(__uint_as_float(raw[c]), p.scale));
+          } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const float sc = kbase + c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
+              mb = fmaxf(mb, sc);
+            }
           }
         }
       }
@@ -266,10 +271,18 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
           att_tmem_ld32(t_row + c0, raw);
           att_tmem_ld_wait();
           float pr[32];
+          if (live == W) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const float sc = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
-            pr[c] = BASE2 ? rg_exp2(f_add(sc, -m_new)) : rg_exp(f_add(sc, -m_new));
+            for (int c = 0; c < 32; ++c) {
+              const float x = f_add(f_mul(__uint_as_float(raw[c]), p.scale), -m_new);
+              pr[c] = BASE2 ? rg_exp2(x) : rg_exp(x);
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const float sc = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
+              pr[c] = BASE2 ? rg_exp2(f_add(sc, -m_new)) : rg_exp(f_add(sc, -m_new));
+            }
           }
           chunk_sum[ci] = tree32(pr);
           // row r of the [128 x 64] box that holds keys c0..c0+31: four 16-byte pieces of 8 keys each
