@@ -4,8 +4,10 @@
 // are all part of the arithmetic and all come from the descriptor.
 //
 // One CTA owns 128 query rows of one head.  Per key block j:
-//   warp 0 (TMA)      K_j [w x d] and Vt_j [d x w] boxes into a two-stage ring (Q once)
-//   warp 1 (MMA)      S = Q K_j^T   d/16 tcgen05.mma steps from a zero accumulator, ascending k
+//   warp 0 (TMA)      K_j [w x d] and Vt_j [d x w] boxes, each into its own two-stage ring (Q once)
+//   warp 1 (MMA)      S = Q K_j^T   d/16 tcgen05.mma steps from a zero accumulator, ascending k; the
+//                     scores of block j+1 are issued before the P V product of block j (two score
+//                     accumulators in tensor memory), so the softmax threads never wait for scores
 //                     PV = P Vt_j^T w/16 steps from a zero accumulator, ascending key
 //   warps 2-9         two threads per query row (its TMEM lane), each with half of the block's keys and
 //                     half of the output columns; partial maxima and partial row sums (subtrees of
@@ -128,7 +130,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   constexpr int DB = HD / 64, WB = W / 64;                // boxes along d and along the keys
   constexpr uint32_t Q_BYTES = DB * Q_BOX, K_BYTES = DB * K_BOX, V_BYTES = WB * V_BOX, P_BYTES = WB * P_BOX;
   constexpr uint32_t KV_BYTES = K_BYTES + V_BYTES;
-  constexpr uint32_t TMEM_COLS = 256;                     // S at columns [0, W), PV at [128, 128 + HD)
+  constexpr uint32_t TMEM_COLS = 512;                     // S of block j at columns [128*(j&1), ... + W), PV at [256, 256 + HD)
   constexpr uint32_t IDESC_S = att_idesc(W), IDESC_PV = att_idesc(HD);
 
   extern __shared__ uint8_t smem_raw[];
@@ -137,13 +139,14 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   const uint32_t sQ = smem_base, sKV = sQ + Q_BYTES, sP = sKV + KV_STAGES * KV_BYTES;
   uint8_t* sP_gen = smem_gen + Q_BYTES + KV_STAGES * KV_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + Q_BYTES + KV_STAGES * KV_BYTES + P_BYTES);
-  // barriers: q_full, kv_full[2], kv_empty[2], s_full, p_full, pv_full
+  // barriers: q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full, pv_full
   const uint32_t bar_q = smem_u32(bars);
-  const uint32_t bar_kv_full = bar_q + 8u, bar_kv_empty = bar_kv_full + 8u * KV_STAGES;
-  const uint32_t bar_s = bar_kv_empty + 8u * KV_STAGES, bar_p = bar_s + 8u, bar_pv = bar_p + 8u;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  const uint32_t bar_k_full = bar_q + 8u, bar_k_empty = bar_k_full + 16u;
+  const uint32_t bar_v_full = bar_k_empty + 16u, bar_v_empty = bar_v_full + 16u;
+  const uint32_t bar_s = bar_v_empty + 16u, bar_p = bar_s + 16u, bar_pv = bar_p + 8u;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* xm = reinterpret_cast<float*>(bars + 10);        // [2][128] partial maxima of the two halves of a row
+  float* xm = reinterpret_cast<float*>(bars + 14);        // [2][128] partial maxima of the two halves of a row
   float* xs = xm + 2 * QROWS;                             // [2][128] partial row sums
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -153,8 +156,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
-    for (int s = 0; s < KV_STAGES; ++s) { mbar_init(bar_kv_full + 8u * s, 1); mbar_init(bar_kv_empty + 8u * s, 1); }
-    mbar_init(bar_s, 1); mbar_init(bar_p, SOFTMAX_THREADS / 32); mbar_init(bar_pv, 1);
+    for (int s = 0; s < KV_STAGES; ++s) {
+      mbar_init(bar_k_full + 8u * s, 1); mbar_init(bar_k_empty + 8u * s, 1);
+      mbar_init(bar_v_full + 8u * s, 1); mbar_init(bar_v_empty + 8u * s, 1);
+      mbar_init(bar_s + 8u * s, 1);
+    }
+    mbar_init(bar_p, SOFTMAX_THREADS / 32); mbar_init(bar_pv, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -173,48 +180,59 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       mbar_expect_tx(bar_q, Q_BYTES);
 #pragma unroll
       for (int b = 0; b < DB; ++b) att_tma_load_2d(sQ + b * Q_BOX, &tmap_q, b * 64, head * p.Nq + q0, bar_q);
-      int stage = 0; uint32_t phase = 0;
       for (int j = 0; j < nblocks; ++j) {
-        if (!mbar_wait(bar_kv_empty + 8u * stage, phase ^ 1u, abort_flag, &g_attn_status_word, 0x1100u | stage)) break;
-        const uint32_t full = bar_kv_full + 8u * stage;
-        mbar_expect_tx(full, KV_BYTES);
+        const int stage = j & 1; const uint32_t phase = (j >> 1) & 1;
         const uint32_t dst = sKV + stage * KV_BYTES;
+        if (!mbar_wait(bar_k_empty + 8u * stage, phase ^ 1u, abort_flag, &g_attn_status_word, 0x1100u | stage)) break;
+        mbar_expect_tx(bar_k_full + 8u * stage, K_BYTES);
 #pragma unroll
-        for (int b = 0; b < DB; ++b) att_tma_load_2d(dst + b * K_BOX, &tmap_k, b * 64, head * p.Nk + j * W, full);
+        for (int b = 0; b < DB; ++b) att_tma_load_2d(dst + b * K_BOX, &tmap_k, b * 64, head * p.Nk + j * W, bar_k_full + 8u * stage);
+        if (!mbar_wait(bar_v_empty + 8u * stage, phase ^ 1u, abort_flag, &g_attn_status_word, 0x1180u | stage)) break;
+        mbar_expect_tx(bar_v_full + 8u * stage, V_BYTES);
 #pragma unroll
-        for (int b = 0; b < WB; ++b) att_tma_load_2d(dst + K_BYTES + b * V_BOX, &tmap_vt, j * W + b * 64, head * HD, full);
-        if (++stage == KV_STAGES) { stage = 0; phase ^= 1u; }
+        for (int b = 0; b < WB; ++b) att_tma_load_2d(dst + K_BYTES + b * V_BOX, &tmap_vt, j * W + b * 64, head * HD, bar_v_full + 8u * stage);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       bool alive = mbar_wait(bar_q, 0, abort_flag, &g_attn_status_word, 0x1200u);
-      int stage = 0; uint32_t phase = 0;
-      for (int j = 0; j < nblocks && alive; ++j) {
-        if (!mbar_wait(bar_kv_full + 8u * stage, phase, abort_flag, &g_attn_status_word, 0x1300u | stage)) break;
+      // S_j = Q K_j^T into score accumulator j&1: ascending k over the head dimension, from zero
+      auto issue_scores = [&](int j) -> bool {
+        const int stage = j & 1; const uint32_t phase = (j >> 1) & 1;
+        if (!mbar_wait(bar_k_full + 8u * stage, phase, abort_flag, &g_attn_status_word, 0x1300u | stage)) return false;
         att_fence_after();
-        const uint32_t sK = sKV + stage * KV_BYTES, sV = sK + K_BYTES;
-        // S = Q K^T: ascending k over the head dimension, from zero
+        const uint32_t sK = sKV + stage * KV_BYTES;
 #pragma unroll
         for (int b = 0; b < DB; ++b) {
           const uint64_t adesc = att_kmajor_desc(sQ + b * Q_BOX), bdesc = att_kmajor_desc(sK + b * K_BOX);
 #pragma unroll
-          for (int a = 0; a < 4; ++a) att_mma_bf16(tmem_base, adesc + 2u * a, bdesc + 2u * a, IDESC_S, (b | a) ? 1u : 0u);
+          for (int a = 0; a < 4; ++a) att_mma_bf16(tmem_base + 128u * stage, adesc + 2u * a, bdesc + 2u * a, IDESC_S, (b | a) ? 1u : 0u);
         }
-        att_commit(bar_s);
+        att_commit(bar_s + 8u * stage);
+        att_commit(bar_k_empty + 8u * stage);
+        return true;
+      };
+      if (alive) alive = issue_scores(0);
+      for (int j = 0; j < nblocks && alive; ++j) {
+        // The next block's scores go first.  Their accumulator held block j-1's scores, which the
+        // softmax threads had finished reading before they released P_{j-1} (waited for below, one
+        // turn ago).
+        if (j + 1 < nblocks && !issue_scores(j + 1)) break;
         // PV = P Vt^T: ascending key over the block, from zero, once the probabilities are in shared memory
+        const int stage = j & 1; const uint32_t phase = (j >> 1) & 1;
         if (!mbar_wait(bar_p, j & 1, abort_flag, &g_attn_status_word, 0x1400u)) break;
+        if (!mbar_wait(bar_v_full + 8u * stage, phase, abort_flag, &g_attn_status_word, 0x1480u | stage)) break;
         att_fence_after();
+        const uint32_t sV = sKV + stage * KV_BYTES + K_BYTES;
 #pragma unroll
         for (int b = 0; b < WB; ++b) {
           const uint64_t adesc = att_kmajor_desc(sP + b * P_BOX), bdesc = att_kmajor_desc(sV + b * V_BOX);
 #pragma unroll
-          for (int a = 0; a < 4; ++a) att_mma_bf16(tmem_base + 128u, adesc + 2u * a, bdesc + 2u * a, IDESC_PV, (b | a) ? 1u : 0u);
+          for (int a = 0; a < 4; ++a) att_mma_bf16(tmem_base + 256u, adesc + 2u * a, bdesc + 2u * a, IDESC_PV, (b | a) ? 1u : 0u);
         }
         att_commit(bar_pv);
-        att_commit(bar_kv_empty + 8u * stage);              // the stage may be refilled once these steps have read it
-        if (++stage == KV_STAGES) { stage = 0; phase ^= 1u; }
+        att_commit(bar_v_empty + 8u * stage);               // the stage may be refilled once these steps have read it
       }
     }
   } else {
@@ -229,11 +247,26 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     float O[OH];
 #pragma unroll
     for (int c = 0; c < OH; ++c) O[c] = 0.0f;
+    // O = a * O + PV on this thread's output columns
+    auto fold_pv = [&](float a) {
+      att_fence_after();
+#pragma unroll
+      for (int ci = 0; ci < OH / 32; ++ci) {
+        uint32_t raw[32];
+        att_tmem_ld32(t_row + 256u + obase + ci * 32, raw);
+        att_tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) O[ci * 32 + c] = f_add(f_mul(a, O[ci * 32 + c]), __uint_as_float(raw[c]));
+      }
+      att_fence_before();
+    };
+    float alpha_prev = 0.0f;
     // A wait that gives up leaves this thread walking the loop without touching tensor memory, so
     // that the 256-thread barriers below are still met by everyone.
     bool alive = true;
     for (int j = 0; j < nblocks; ++j) {
-      if (alive) alive = mbar_wait(bar_s, j & 1, abort_flag, &g_attn_status_word, 0x1500u);
+      if (alive) alive = mbar_wait(bar_s + 8u * (j & 1), (j >> 1) & 1, abort_flag, &g_attn_status_word, 0x1500u);
+      const uint32_t t_s = t_row + 128u * (j & 1);          // this block's score accumulator
       const int live = min(W, p.Nk - j * W);                // keys of this block that exist
       // pass 1: the maximum over this thread's keys, then over the row
       float mb = -INFINITY;
@@ -242,7 +275,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 #pragma unroll
         for (int c0 = 0; c0 < KH; c0 += 32) {
           uint32_t raw[32];
-          att_tmem_ld32(t_row + kbase + c0, raw);
+          att_tmem_ld32(t_s + kbase + c0, raw);
           att_tmem_ld_wait();
           if (live == W) {                                  // every key exists: no masking (all blocks but the last)
 #pragma unroll
@@ -260,6 +293,14 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       asm volatile("bar.sync 1, 256;" ::: "memory");
       const float m_new = fmaxf(m, fmaxf(xm[r], xm[QROWS + r]));
       const float alpha = BASE2 ? rg_exp2(f_add(m, -m_new)) : rg_exp(f_add(m, -m_new));
+      // The previous block's P V product has had a whole first pass to finish: fold it into O now.
+      // This also orders the rewrite of P below after the tensor core's last read of it, and comes
+      // before this block's probabilities are released, so the barrier cannot run a phase ahead.
+      if (j > 0) {
+        if (alive) alive = mbar_wait(bar_pv, (j - 1) & 1, abort_flag, &g_attn_status_word, 0x1600u);
+        if (alive) fold_pv(alpha_prev);
+      }
+      alpha_prev = alpha;
       // pass 2: probabilities, the subtree of the row sum over this thread's keys, narrowed copies
       float part = 0.0f;
       if (alive) {
@@ -268,7 +309,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         for (int ci = 0; ci < KH / 32; ++ci) {
           const int c0 = kbase + ci * 32;
           uint32_t raw[32];
-          att_tmem_ld32(t_row + c0, raw);
+          att_tmem_ld32(t_s + c0, raw);
           att_tmem_ld_wait();
           float pr[32];
           if (live == W) {
@@ -305,21 +346,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       if (lane == 0 && alive) mbar_arrive(bar_p);
       l = f_add(f_mul(alpha, l), f_add(xs[r], xs[QROWS + r]));
       m = m_new;
-      // the block's P V product, then O = alpha * O + PV on this thread's output columns
-      if (alive) alive = mbar_wait(bar_pv, j & 1, abort_flag, &g_attn_status_word, 0x1600u);
-      if (alive) {
-        att_fence_after();
-#pragma unroll
-        for (int ci = 0; ci < OH / 32; ++ci) {
-          uint32_t raw[32];
-          att_tmem_ld32(t_row + 128u + obase + ci * 32, raw);
-          att_tmem_ld_wait();
-#pragma unroll
-          for (int c = 0; c < 32; ++c) O[ci * 32 + c] = f_add(f_mul(alpha, O[ci * 32 + c]), __uint_as_float(raw[c]));
-        }
-        att_fence_before();
-      }
     }
+    if (alive) alive = mbar_wait(bar_pv, (nblocks - 1) & 1, abort_flag, &g_attn_status_word, 0x1700u);
+    if (alive) fold_pv(alpha_prev);
     // one division at the end, one rounding to the output type
     const int64_t row = (int64_t)q0 + r;
     if (alive && row < p.Nq) {
@@ -357,7 +386,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
 template <int W, int HD>
 size_t attn_smem_bytes() {
-  return 1024 + (HD / 64) * QROWS * 128 + KV_STAGES * ((HD / 64) * W * 128 + (W / 64) * HD * 128) + (W / 64) * QROWS * 128 + 10 * 8 + 4 * QROWS * 4;
+  return 1024 + (HD / 64) * QROWS * 128 + KV_STAGES * ((HD / 64) * W * 128 + (W / 64) * HD * 128) + (W / 64) * QROWS * 128 + 14 * 8 + 4 * QROWS * 4;
 }
 
 template <int W, int HD, bool BASE2>
