@@ -279,6 +279,12 @@ def run_ours(args):
         col_out = torch.empty(RED_C, dtype=f32, device=dev)
         col_ws = torch.empty(rg.rg_reduce_cols_workspace_bytes(RED_R, RED_C), dtype=torch.uint8, device=dev)
         ms_col = timed(lambda: rg.rg_reduce_cols(d_plain, rg.RG_COLOP_SUM, T["red_X"], col_out, ws=col_ws), 5)
+        aH, aN, ad_ = 32, 4096, 128
+        aQ = synth.device_normal((aH * aN, ad_), 1.0, seed0 + 41, bf, dev); aK = synth.device_normal((aH * aN, ad_), 1.0, seed0 + 42, bf, dev)
+        aVt = synth.device_normal((aH * ad_, aN), 1.0, seed0 + 43, bf, dev); aO = torch.empty((aH * aN, ad_), dtype=bf, device=dev)
+        adesc = rg.rg_attn_desc(block_n=128, scale=ad_ ** -0.5 * 1.4426950408889634, heads=aH, exp_base=2)
+        ms_att = timed(lambda: rg.rg_attention(adesc, aQ, aK, aVt, aO), 5)
+        del aQ, aK, aVt, aO
         wbytes = 2.0 * 4096 * 14336
         line["widened"] = {
             "note": "timed alone after the step loop; weights of the two decode paths rotate over four copies (above L2)",
@@ -286,6 +292,7 @@ def run_ours(args):
             "decode_splitk8_back_to_back_us": round(ms_dec * 1e3, 2), "decode_splitk8_weight_gbs": round(wbytes / (ms_dec * 1e-3) / 1e9, 1),
             "gemv_m1_back_to_back_us": round(ms_gemv * 1e3, 2), "gemv_m1_weight_gbs": round(wbytes / (ms_gemv * 1e-3) / 1e9, 1),
             "col_sum_65536x32768_gbs": round(4.0 * RED_R * RED_C / (ms_col * 1e-3) / 1e9, 1),
+            "attention_32x4096x4096x128_base2_w128_tflops": round(4.0 * aH * aN * aN * ad_ / (ms_att * 1e-3) / 1e12, 1),
         }
         del col_out, col_ws
 

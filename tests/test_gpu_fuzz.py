@@ -174,3 +174,24 @@ def test_random_gemv_and_column_reduction_match_oracle(seed):
     want = rgo.reduce_cols(op, x[:, off:off + Cc], y[:, off:off + Cc] if op else None, fma=cfma)
     assert_bits_equal(o.cpu().numpy(), want, f"seed {seed}: cols op={op} {R}x{Cc} bf16={bf} fma={cfma} off={off}")
     assert rg.rg_device_status() == 0
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_attention_matches_oracle(seed):
+    """Attention descriptors (block width, base, head size, heads) on random ragged shapes, bit for bit."""
+    from test_gpu_attention import gpu_attention
+    from paper_2609_11356_b200 import synth
+    g = np.random.default_rng(20000 + seed)
+    H = int(g.choice([1, 2, 3])); Nq = int(g.choice([1, 17, 128, 130, 300])); Nk = int(g.choice([1, 40, 64, 129, 500, 1100]))
+    d = int(g.choice([64, 128])); w = int(g.choice([64, 128])); base = int(g.choice([0, 2]))
+    spread = int(g.choice([0, 2]))
+    mk = lambda n: synth.f32_to_bf16_bits((g.standard_normal((H * n, d)) * np.exp2(g.integers(-spread, spread + 1, (H * n, d)))).astype(np.float32))
+    Q, K, V = mk(Nq), mk(Nk), mk(Nk)
+    scale = float(np.float32(d ** -0.5 * (np.log2(np.e) if base == 2 else 1.0)))
+    out = [rgo.F32, rgo.BF16][int(g.integers(0, 2))]
+    got = gpu_attention(Q, K, V, block_n=w, scale=scale, heads=H, out_dtype=out, exp_base=base)
+    for h in range(H):
+        want = rgo.attention(Q[h * Nq:(h + 1) * Nq], K[h * Nk:(h + 1) * Nk], V[h * Nk:(h + 1) * Nk], block_n=w, scale=scale,
+                             atom_model=HW, out_dtype=out, exp_base=base)
+        assert_bits_equal(got[h * Nq:(h + 1) * Nq], want, f"seed {seed}: attention H={H} {Nq}x{Nk} d={d} w={w} base={base} head {h}")
+    assert rg.rg_device_status() == 0
