@@ -774,8 +774,12 @@ void rgo_reduce_cols(int op, int tree, int fma, const void* x, int x_dtype, cons
 //                                                               over its keys from a zero accumulator
 // and the answer is O_B / l_B, divided once at the end and rounded once to the output type.
 // Keys past Nk in the last block are absent: their scores are -inf, their probabilities exactly 0.
+// Causal masking (mask = 1, App. F "Masking puts the query block into the answer"): query row i sees
+// keys t <= i.  The walk of a row in query tile [q0, q0 + block_m) stops at key q0 + block_m; the blocks
+// from q0 on are the ones that straddle the diagonal, and there every score takes an offset before the
+// maximum: 0 where t <= i, -1e6 where t > i (so those probabilities underflow to exactly 0).
 // Vt is V transposed: [d, Nk], keys contiguous.
-void rgo_attention(const AtomModel* atom, int block_n, int sum_tree, int p_dtype, int exp_base, float scale,
+void rgo_attention(const AtomModel* atom, int block_n, int sum_tree, int p_dtype, int exp_base, int mask, int block_m, float scale,
                    int64_t Nq, int64_t Nk, int64_t d, const uint16_t* Q, int64_t ldq, const uint16_t* K, int64_t ldk,
                    const uint16_t* Vt, int64_t ldv, void* O, int o_dtype, int64_t ldo) {
   const int ak = atom->atom_k;
@@ -785,14 +789,18 @@ void rgo_attention(const AtomModel* atom, int block_n, int sum_tree, int p_dtype
     float m = -INFINITY, l = 0.0f;
     std::vector<float> Oacc(d, 0.0f), s(block_n), pf(block_n);
     std::vector<uint16_t> pn(block_n);
-    for (int64_t t0 = 0; t0 < Nk; t0 += block_n) {
-      const int n = (int)std::min<int64_t>(block_n, Nk - t0);
+    const int64_t tile0 = mask ? (i / block_m) * block_m : 0;
+    const int64_t kend = mask ? std::min<int64_t>(Nk, tile0 + block_m) : Nk;
+    for (int64_t t0 = 0; t0 < kend; t0 += block_n) {
+      const int n = (int)std::min<int64_t>(block_n, kend - t0);
+      const bool diagonal = mask && t0 >= tile0;
       float mb = -INFINITY;
       for (int t = 0; t < n; ++t) {
         const uint16_t* k = K + (t0 + t) * ldk;
         float acc = 0.0f;
         for (int64_t c0 = 0; c0 < d; c0 += ak) acc = atom_step(acc, q + c0, k + c0, (int)std::min<int64_t>(ak, d - c0), *atom);
         s[t] = acc * scale;
+        if (diagonal) s[t] = s[t] + ((t0 + t) <= i ? 0.0f : -1.0e6f);
         mb = std::max(mb, s[t]);
       }
       const float m_new = std::max(m, mb);

@@ -117,7 +117,7 @@ def lib():
         L.rgo_reduce_rows.argtypes = [i32, i32, i32, vp, i32, i64, i64, i64, vp, i32, i64, vp, i32, f32, vp]
         L.rgo_attention.restype = None
         L.rgo_exp2f.restype = f32; L.rgo_exp2f.argtypes = [f32]
-        L.rgo_attention.argtypes = [C.POINTER(_AtomStruct), i32, i32, i32, i32, f32, i64, i64, i64, vp, i64, vp, i64, vp, i64, vp, i32, i64]
+        L.rgo_attention.argtypes = [C.POINTER(_AtomStruct), i32, i32, i32, i32, i32, i32, f32, i64, i64, i64, vp, i64, vp, i64, vp, i64, vp, i32, i64]
         L.rgo_reduce_cols.restype = None
         L.rgo_reduce_cols.argtypes = [i32, i32, i32, vp, i32, vp, i32, i64, i64, i64, i64, vp]
         _lib = L
@@ -323,7 +323,7 @@ def reduce_cols(op: int, x, y=None, *, tree: int = TREE_BALANCED, fma: int = 0) 
 
 
 def attention(Q, K, V, *, block_n: int, scale: float, atom_model: AtomModel = EXACT_RN, sum_tree: int = TREE_BALANCED,
-              p_dtype: int = BF16, out_dtype: int = BF16, exp_base: int = 0) -> np.ndarray:
+              p_dtype: int = BF16, out_dtype: int = BF16, exp_base: int = 0, causal: bool = False, block_m: int = 128) -> np.ndarray:
     """Attention of one head with a fixed descriptor (App. F): Q [Nq, d], K [Nk, d], V [Nk, d] as 16-bit
     patterns (uint16 = bf16, float16 = fp16).  Returns [Nq, d] at out_dtype."""
     Vt = np.ascontiguousarray(np.asarray(V).T)
@@ -333,6 +333,6 @@ def attention(Q, K, V, *, block_n: int, scale: float, atom_model: AtomModel = EX
     assert K.shape[1] == d and Vt.shape == (d, Nk)
     out = np.empty((Nq, d), dtype=_OUT_NP[out_dtype])
     mc = m.c()
-    lib().rgo_attention(C.byref(mc), block_n, sum_tree, p_dtype, exp_base, np.float32(scale), Nq, Nk, d, _ptr(Q), d, _ptr(K), d,
+    lib().rgo_attention(C.byref(mc), block_n, sum_tree, p_dtype, exp_base, 1 if causal else 0, block_m, np.float32(scale), Nq, Nk, d, _ptr(Q), d, _ptr(K), d,
                         _ptr(Vt), Nk, _ptr(out), out_dtype, d)
     return out

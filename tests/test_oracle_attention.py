@@ -110,3 +110,29 @@ def test_base_two_exponential_variant():
     Ku = _bf(np.tile(np.linspace(-1, 1, d, dtype=np.float32), (256, 1))); v = np.arange(d, dtype=np.float32) / 4
     out = rgo.attention(_bf(np.ones((2, d))), Ku, _bf(np.tile(v, (256, 1))), block_n=64, scale=0.3, out_dtype=rgo.F32, exp_base=2)
     assert np.array_equal(out, np.tile(v, (2, 1)))
+
+
+def test_causal_masking():
+    g = np.random.default_rng(21)
+    d, N = 32, 300
+    Q, K, V = _bf(g.standard_normal((N, d))), _bf(g.standard_normal((N, d))), _bf(g.standard_normal((N, d)))
+    scale = d ** -0.5
+    out = rgo.attention(Q, K, V, block_n=64, scale=scale, atom_model=rgo.TCGEN05_BF16_B200, out_dtype=rgo.F32, causal=True)
+    # against double-precision causal softmax attention
+    S = (_f(Q) @ _f(K).T) * scale
+    S[np.triu_indices(N, 1)] = -np.inf
+    P = np.exp(S - S.max(1, keepdims=True)); ref = (P / P.sum(1, keepdims=True)) @ _f(V)
+    assert np.max(np.abs(out - ref)) <= 2.0 ** -8 * np.max(np.abs(_f(V))) + 1e-6
+    # the first query sees one key: its value row exactly; a row never depends on later keys or values
+    assert np.array_equal(out[0], synth.bf16_bits_to_f32(V[0]))
+    K2, V2 = K.copy(), V.copy(); K2[200:] = _bf(g.standard_normal((100, d))); V2[200:] = _bf(g.standard_normal((100, d)))
+    out2 = rgo.attention(Q, K2, V2, block_n=64, scale=scale, atom_model=rgo.TCGEN05_BF16_B200, out_dtype=rgo.F32, causal=True)
+    assert np.array_equal(out[:200], out2[:200]) and not np.array_equal(out[200:], out2[200:])
+    # rows of the first tile equal unmasked attention over their own prefix only when the prefix is a whole
+    # number of blocks and nothing above the diagonal is live: row 63 with 64-wide blocks
+    pref = rgo.attention(Q[63:64], K[:64], V[:64], block_n=64, scale=scale, atom_model=rgo.TCGEN05_BF16_B200, out_dtype=rgo.F32)
+    assert np.allclose(out[63], pref[0], atol=1e-6)
+    # with block_n dividing block_m and exp(0) = 1 exact, a fully masked block is an exact no-op
+    # (alpha = 1, every probability 0), so the query tile height moves no bit here
+    out256 = rgo.attention(Q, K, V, block_n=64, scale=scale, atom_model=rgo.TCGEN05_BF16_B200, out_dtype=rgo.F32, causal=True, block_m=256)
+    assert np.array_equal(out, out256)
