@@ -515,9 +515,9 @@ def run_only(args):
         H, Nq, Nk, hd = 32, 4096, 4096, 128
         Q = synth.device_normal((H * Nq, hd), 1.0, 21, bf, dev); Kt = synth.device_normal((H * Nk, hd), 1.0, 22, bf, dev)
         Vt = synth.device_normal((H * hd, Nk), 1.0, 23, bf, dev); O = torch.empty((H * Nq, hd), dtype=bf, device=dev)
-        ad = rg.rg_attn_desc(block_n=args.attn_block, scale=hd ** -0.5 * (1.4426950408889634 if args.attn_base == 2 else 1.0), heads=H, exp_base=args.attn_base)
+        ad = rg.rg_attn_desc(block_n=args.attn_block, scale=hd ** -0.5 * (1.4426950408889634 if args.attn_base == 2 else 1.0), heads=H, exp_base=args.attn_base, mask=args.attn_causal)
         fn = lambda: rg.rg_attention(ad, Q, Kt, Vt, O)
-        work, unit = 4.0 * H * Nq * Nk * hd / 1e12, "TFLOP/s"
+        work, unit = 4.0 * H * Nq * Nk * hd / 1e12 * (0.5 if args.attn_causal else 1.0), "TFLOP/s"
     elif name in ("col_sum", "col_dot"):
         R_, C_ = 65536, 8192
         x = synth.device_normal((R_, C_), 100.0, 13, f32, dev)
@@ -569,6 +569,7 @@ def main():
                     help="run one kernel on a small case (used for the ncu captures)")
     ap.add_argument("--gemv-rows", type=int, default=1, help="rows of A for --only gemv_decode")
     ap.add_argument("--attn-block", type=int, default=128, help="key block width for --only attention")
+    ap.add_argument("--attn-causal", type=int, default=0, help="1: causal masking, for --only attention (flops counted as half)")
     ap.add_argument("--attn-base", type=int, default=0, help="0: base-e exponential, 2: base-two, for --only attention")
     args = ap.parse_args()
     if args.only:

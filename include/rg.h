@@ -206,8 +206,11 @@ rg_status_t rg_reduce_cols(const rg_desc_t* d, rg_col_op_t op, const rg_tensor_t
  * chains of tensor-core steps from a zero accumulator (RG_ATOM_TC_BF16_K16): over the head dimension
  * for the scores, over the block's keys for P . V.  exp is an exponential this library fixes from IEEE
  * operations: base e, or base two (`exp_base`), a cheaper polynomial and another class of bits.
- * Every block boundary is a rounding of O and l, so block_n is part of the class of bits; the query
- * tile is not (no masking here: `mask` must be 0).
+ * Every block boundary is a rounding of O and l, so block_n is part of the class of bits.
+ * mask = 1 is causal masking (query row i sees keys t <= i, Nq rows against the first keys): the walk of
+ * the query tile [q0, q0 + block_m) stops at key q0 + block_m, and in the blocks from q0 on every score
+ * takes an offset before the maximum, 0 where t <= i and -1e6 where t > i.  block_m must be 128 (the
+ * kernel's query tile) and a multiple of block_n; it is 0 or 128 without masking.
  *
  * Q [heads*Nq, d], K [heads*Nk, d], Vt [heads*d, Nk] (V transposed: keys contiguous, what rg_gemm
  * writes for W_v . X^T) and O [heads*Nq, d]: device pointers, heads stacked along the rows.  Q, K,
@@ -217,10 +220,11 @@ typedef struct {
   uint32_t size;          /* = sizeof(rg_attn_desc_t) */
   uint32_t heads;         /* >= 1 */
   uint32_t block_n;       /* key block width: 64 or 128 */
+  uint32_t block_m;       /* query tile height, part of the descriptor when mask = 1 (App. F): 128; else 0 or 128 */
   float scale;            /* scores are multiplied by this in fp32 */
   uint8_t sum_tree;       /* rg_tree_t of the row sum inside a block: RG_TREE_BALANCED */
   uint8_t p_dtype;        /* type the probabilities are narrowed to: RG_BF16 */
-  uint8_t mask;           /* 0 = none */
+  uint8_t mask;           /* 0 = none, 1 = causal */
   uint8_t div_place;      /* 0 = once, at the end */
   uint8_t exp_base;       /* 0 = base e; 2 = base two (the caller folds log2 e into `scale`, App. F) */
   uint8_t _pad[3];

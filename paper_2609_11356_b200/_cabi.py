@@ -30,7 +30,7 @@ EXPORTS = ["rg_desc_init", "rg_desc_validate", "rg_desc_class", "rg_gemm_workspa
 
 
 class rg_attn_desc_t(C.Structure):
-    _fields_ = [("size", C.c_uint32), ("heads", C.c_uint32), ("block_n", C.c_uint32), ("scale", C.c_float),
+    _fields_ = [("size", C.c_uint32), ("heads", C.c_uint32), ("block_n", C.c_uint32), ("block_m", C.c_uint32), ("scale", C.c_float),
                 ("sum_tree", C.c_uint8), ("p_dtype", C.c_uint8), ("mask", C.c_uint8), ("div_place", C.c_uint8),
                 ("exp_base", C.c_uint8), ("_pad", C.c_uint8 * 3)]
 

@@ -147,10 +147,11 @@ def rg_reduce_rows(d: K.rg_desc_t, op: int, x, out, *, weight=None, eps: float =
 
 
 def rg_attn_desc(*, block_n: int, scale: float, heads: int = 1, sum_tree: int = K.RG_TREE_BALANCED, p_dtype: int = K.RG_BF16,
-                 mask: int = 0, div_place: int = 0, exp_base: int = 0) -> K.rg_attn_desc_t:
+                 mask: int = 0, div_place: int = 0, exp_base: int = 0, block_m: int = 0) -> K.rg_attn_desc_t:
     d = K.rg_attn_desc_t()
     d.size = C.sizeof(K.rg_attn_desc_t)
     d.heads, d.block_n, d.scale = heads, block_n, scale
+    d.block_m = block_m if block_m else (128 if mask else 0)
     d.sum_tree, d.p_dtype, d.mask, d.div_place, d.exp_base = sum_tree, p_dtype, mask, div_place, exp_base
     return d
 

@@ -275,7 +275,9 @@ rg_status_t rg_attention(const rg_attn_desc_t* d, const rg_tensor_t* Q, const rg
   rg_status_t s;
   if ((s = check_tensor(Q)) != RG_OK || (s = check_tensor(K)) != RG_OK || (s = check_tensor(Vt)) != RG_OK || (s = check_tensor(O)) != RG_OK)
     return s;
-  if (d->sum_tree != RG_TREE_BALANCED || d->p_dtype != RG_BF16 || d->mask != 0 || d->div_place != 0) return RG_ERR_UNSUPPORTED;
+  if (d->mask > 1) return RG_ERR_INVALID_DESC;
+  if (d->sum_tree != RG_TREE_BALANCED || d->p_dtype != RG_BF16 || d->div_place != 0) return RG_ERR_UNSUPPORTED;
+  if (d->mask ? d->block_m != 128 : (d->block_m != 0 && d->block_m != 128)) return RG_ERR_UNSUPPORTED;
   if (d->block_n != 64 && d->block_n != 128) return RG_ERR_UNSUPPORTED;
   if (d->exp_base != 0 && d->exp_base != 2) return RG_ERR_INVALID_DESC;
   if (Q->dtype != RG_BF16 || K->dtype != RG_BF16 || Vt->dtype != RG_BF16) return RG_ERR_UNSUPPORTED;
@@ -289,7 +291,7 @@ rg_status_t rg_attention(const rg_attn_desc_t* d, const rg_tensor_t* Q, const rg
       (reinterpret_cast<uintptr_t>(Vt->ptr) & 15) || (reinterpret_cast<uintptr_t>(O->ptr) & 15) ||
       (Q->ld % 8) || (K->ld % 8) || (Vt->ld % 8) || (O->ld % 8))
     return RG_ERR_ALIGNMENT;
-  return rg::launch_attention_fixed((int)d->block_n, (int)d->exp_base, d->scale, (int)H, Q, K, Vt, O, static_cast<cudaStream_t>(cuda_stream));
+  return rg::launch_attention_fixed((int)d->block_n, (int)d->exp_base, (int)d->mask, d->scale, (int)H, Q, K, Vt, O, static_cast<cudaStream_t>(cuda_stream));
 }
 
 // ------------------------------------------------------------ host-buffer forms

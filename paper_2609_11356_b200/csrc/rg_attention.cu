@@ -17,7 +17,9 @@
 //                     block's keys in order); P = p narrowed to bf16, written to shared memory in the
 //                     swizzled K-major layout the tensor core reads; O_j = alpha*O_{j-1} + PV
 // and at the end O / l, one division, one rounding to the output type.  exp is one of the library's
-// specified exponentials (rg_exp, or rg_exp2 with log2 e folded into the scale), not the hardware's.  Keys past Nk are masked to
+// specified exponentials (rg_exp, or rg_exp2 with log2 e folded into the scale), not the hardware's.
+// With causal masking the walk of a query tile stops at its own end, and the blocks from the tile's
+// first row on add 0 (key <= query) or -1e6 (key > query) to every score before the maximum.  Keys past Nk are masked to
 // -inf before the maximum, so their probabilities are exactly +0.
 //
 // Heads are stacked along the rows of Q [heads*Nq, d], K [heads*Nk, d], Vt [heads*d, Nk] and
@@ -100,6 +102,7 @@ __host__ __device__ constexpr uint32_t att_idesc(int n) {
 
 struct AttnParams {
   int32_t Nq, Nk;        // per head
+  int32_t causal;        // query row i sees keys t <= i; the query tile is this CTA's 128 rows
   float scale;
   void* O;
   int64_t ldo;
@@ -151,8 +154,11 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int head = blockIdx.y;
-  const int q0 = blockIdx.x * QROWS;                      // first query row of this CTA within the head
-  const int nblocks = (p.Nk + W - 1) / W;
+  // causal walks grow with the tile index: the long ones are scheduled first
+  const int q0 = (p.causal ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x) * QROWS;   // first query row of this CTA within the head
+  // causal: the walk stops at the end of the query tile; the blocks from q0 on straddle the diagonal
+  const int kend = p.causal ? min(p.Nk, q0 + QROWS) : p.Nk;
+  const int nblocks = (kend + W - 1) / W;
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
@@ -267,7 +273,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     for (int j = 0; j < nblocks; ++j) {
       if (alive) alive = mbar_wait(bar_s + 8u * (j & 1), (j >> 1) & 1, abort_flag, &g_attn_status_word, 0x1500u);
       const uint32_t t_s = t_row + 128u * (j & 1);          // this block's score accumulator
-      const int live = min(W, p.Nk - j * W);                // keys of this block that exist
+      const int live = min(W, kend - j * W);                // keys of this block that exist
+      const bool diagonal = p.causal && j * W >= q0;        // scores take the 0 / -1e6 offset (App. F)
+      const int qi = q0 + r;                                // this row's query index within the head
       // pass 1: the maximum over this thread's keys, then over the row
       float mb = -INFINITY;
       if (alive) {
@@ -277,7 +285,15 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
           uint32_t raw[32];
           att_tmem_ld32(t_s + kbase + c0, raw);
           att_tmem_ld_wait();
-          if (live == W) {                                  // every key exists: no masking (all blocks but the last)
+          if (diagonal) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const int t = kbase + c0 + c;
+              float sc = t < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
+              sc = f_add(sc, j * W + t <= qi ? 0.0f : -1.0e6f);
+              mb = fmaxf(mb, sc);
+            }
+          } else if (live == W) {                           // every key exists: no masking (all blocks but the last)
 #pragma unroll
             for (int c = 0; c < 32; ++c) mb = fmaxf(mb, f_mul(__uint_as_float(raw[c]), p.scale));
           } else {
@@ -312,7 +328,14 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
           att_tmem_ld32(t_s + c0, raw);
           att_tmem_ld_wait();
           float pr[32];
-          if (live == W) {
+          if (diagonal) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              float sc = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
+              sc = f_add(sc, j * W + c0 + c <= qi ? 0.0f : -1.0e6f);
+              pr[c] = BASE2 ? rg_exp2(f_add(sc, -m_new)) : rg_exp(f_add(sc, -m_new));
+            }
+          } else if (live == W) {
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
               const float x = f_add(f_mul(__uint_as_float(raw[c]), p.scale), -m_new);
@@ -407,7 +430,7 @@ cudaError_t launch_attention(const CUtensorMap& tq, const CUtensorMap& tk, const
 
 // All arguments were validated by the caller: bf16 operands, d in {64, 128}, block_n in {64, 128},
 // 16-byte aligned pointers, leading dimensions multiples of 8.
-rg_status_t launch_attention_fixed(int block_n, int exp_base, float scale, int heads, const rg_tensor_t* Q, const rg_tensor_t* K,
+rg_status_t launch_attention_fixed(int block_n, int exp_base, int causal, float scale, int heads, const rg_tensor_t* Q, const rg_tensor_t* K,
                                    const rg_tensor_t* Vt, const rg_tensor_t* O, cudaStream_t st) {
   const int d = (int)Q->cols;
   const int64_t Nq = Q->rows / heads, Nk = K->rows / heads;
@@ -417,7 +440,7 @@ rg_status_t launch_attention_fixed(int block_n, int exp_base, float scale, int h
       !make_operand_tmap(&tv, Vt->ptr, Vt->dtype, Vt->rows, Vt->cols, Vt->ld, d))
     return RG_ERR_CUDA;
   AttnParams p;
-  p.Nq = (int32_t)Nq; p.Nk = (int32_t)Nk; p.scale = scale;
+  p.Nq = (int32_t)Nq; p.Nk = (int32_t)Nk; p.scale = scale; p.causal = causal;
   p.O = O->ptr; p.ldo = O->ld; p.o_dtype = O->dtype;
   const dim3 grid((unsigned)((Nq + QROWS - 1) / QROWS), (unsigned)heads, 1);
   cudaError_t err;

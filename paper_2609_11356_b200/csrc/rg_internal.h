@@ -30,7 +30,7 @@ size_t reduce_cols_workspace_bytes(int64_t R, int64_t C);
 rg_status_t launch_reduce_cols(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* y, const rg_tensor_t* out,
                                void* ws, cudaStream_t st);
 bool make_operand_tmap(CUtensorMap_st* map, const void* ptr, int dtype, int64_t rows, int64_t cols, int64_t ld, int box_rows);
-rg_status_t launch_attention_fixed(int block_n, int exp_base, float scale, int heads, const rg_tensor_t* Q, const rg_tensor_t* K,
+rg_status_t launch_attention_fixed(int block_n, int exp_base, int causal, float scale, int heads, const rg_tensor_t* Q, const rg_tensor_t* K,
                                    const rg_tensor_t* Vt, const rg_tensor_t* O, cudaStream_t st);
 rg_status_t read_and_clear_attn_status(uint32_t* code);
 rg_status_t read_and_clear_status(uint32_t* code);

@@ -12,7 +12,7 @@ from tests._gpu_util import DEV, HW, assert_bits_equal
 pytestmark = pytest.mark.gpu
 
 
-def gpu_attention(Q, K, V, *, block_n, scale, heads=1, out_dtype=rgo.BF16, exp_base=0):
+def gpu_attention(Q, K, V, *, block_n, scale, heads=1, out_dtype=rgo.BF16, exp_base=0, causal=False):
     """Q [heads*Nq, d], K [heads*Nk, d], V [heads*Nk, d] as bf16 bit patterns."""
     d = Q.shape[1]; Nk = K.shape[0] // heads
     Vt = np.ascontiguousarray(V.reshape(heads, Nk, d).transpose(0, 2, 1)).reshape(heads * d, Nk)
@@ -22,7 +22,7 @@ def gpu_attention(Q, K, V, *, block_n, scale, heads=1, out_dtype=rgo.BF16, exp_b
     tdt = {rgo.BF16: torch.bfloat16, rgo.F32: torch.float32, rgo.F16: torch.float16}[out_dtype]
     O = torch.empty((Q.shape[0], d), dtype=tdt, device=DEV)
     O.view(torch.int32 if out_dtype == rgo.F32 else torch.int16).fill_(-1)
-    rg.rg_attention(rg.rg_attn_desc(block_n=block_n, scale=scale, heads=heads, exp_base=exp_base), synth.to_torch(Q, DEV), synth.to_torch(K, DEV), vt[:, :Nk], O)
+    rg.rg_attention(rg.rg_attn_desc(block_n=block_n, scale=scale, heads=heads, exp_base=exp_base, mask=1 if causal else 0), synth.to_torch(Q, DEV), synth.to_torch(K, DEV), vt[:, :Nk], O)
     torch.cuda.synchronize()
     return synth.from_torch(O)
 
@@ -51,6 +51,20 @@ def test_base_two_variant_bit_exact(Nq, Nk, d, w):
     got = gpu_attention(Q, K, V, block_n=w, scale=scale, out_dtype=rgo.F32, exp_base=2)
     want = rgo.attention(Q, K, V, block_n=w, scale=scale, atom_model=HW, out_dtype=rgo.F32, exp_base=2)
     assert_bits_equal(got, want, f"attention base two {Nq}x{Nk} d={d} w={w}")
+
+
+@pytest.mark.parametrize("N,d,w,base", [(128, 128, 128, 0), (300, 64, 64, 2), (1000, 128, 64, 0), (777, 128, 128, 2)])
+def test_causal_bit_exact(N, d, w, base):
+    H = 2
+    Q, K, V = _draw(N, N, d, 31 + N, heads=H)
+    scale = float(np.float32(d ** -0.5 * (np.log2(np.e) if base == 2 else 1.0)))
+    got = gpu_attention(Q, K, V, block_n=w, scale=scale, heads=H, out_dtype=rgo.F32, exp_base=base, causal=True)
+    for h in range(H):
+        want = rgo.attention(Q[h * N:(h + 1) * N], K[h * N:(h + 1) * N], V[h * N:(h + 1) * N], block_n=w, scale=scale,
+                             atom_model=HW, out_dtype=rgo.F32, exp_base=base, causal=True)
+        assert_bits_equal(got[h * N:(h + 1) * N], want, f"causal N={N} d={d} w={w} base={base} head {h}")
+    # the first query of every head sees one key
+    assert_bits_equal(got[0], synth.bf16_bits_to_f32(V[0]), "first row")
 
 
 def test_heads_block_width_and_spread_inputs():
@@ -90,7 +104,9 @@ def test_argument_errors():
     with pytest.raises(rg.RgError):
         rg.rg_attention(rg.rg_attn_desc(block_n=96, scale=1.0), q, k, vt, o)
     with pytest.raises(rg.RgError):
-        rg.rg_attention(rg.rg_attn_desc(block_n=64, scale=1.0, mask=1), q, k, vt, o)
+        rg.rg_attention(rg.rg_attn_desc(block_n=64, scale=1.0, mask=2), q, k, vt, o)
+    with pytest.raises(rg.RgError):
+        rg.rg_attention(rg.rg_attn_desc(block_n=64, scale=1.0, mask=1, block_m=256), q, k, vt, o)
     with pytest.raises(rg.RgError):
         rg.rg_attention(rg.rg_attn_desc(block_n=64, scale=1.0), q, k, vt[:, :200], o)
     with pytest.raises(rg.RgError):

@@ -185,13 +185,16 @@ def test_random_attention_matches_oracle(seed):
     H = int(g.choice([1, 2, 3])); Nq = int(g.choice([1, 17, 128, 130, 300])); Nk = int(g.choice([1, 40, 64, 129, 500, 1100]))
     d = int(g.choice([64, 128])); w = int(g.choice([64, 128])); base = int(g.choice([0, 2]))
     spread = int(g.choice([0, 2]))
+    causal = bool(g.integers(0, 2))
+    if causal:
+        Nk = Nq
     mk = lambda n: synth.f32_to_bf16_bits((g.standard_normal((H * n, d)) * np.exp2(g.integers(-spread, spread + 1, (H * n, d)))).astype(np.float32))
     Q, K, V = mk(Nq), mk(Nk), mk(Nk)
     scale = float(np.float32(d ** -0.5 * (np.log2(np.e) if base == 2 else 1.0)))
     out = [rgo.F32, rgo.BF16][int(g.integers(0, 2))]
-    got = gpu_attention(Q, K, V, block_n=w, scale=scale, heads=H, out_dtype=out, exp_base=base)
+    got = gpu_attention(Q, K, V, block_n=w, scale=scale, heads=H, out_dtype=out, exp_base=base, causal=causal)
     for h in range(H):
         want = rgo.attention(Q[h * Nq:(h + 1) * Nq], K[h * Nk:(h + 1) * Nk], V[h * Nk:(h + 1) * Nk], block_n=w, scale=scale,
-                             atom_model=HW, out_dtype=out, exp_base=base)
-        assert_bits_equal(got[h * Nq:(h + 1) * Nq], want, f"seed {seed}: attention H={H} {Nq}x{Nk} d={d} w={w} base={base} head {h}")
+                             atom_model=HW, out_dtype=out, exp_base=base, causal=causal)
+        assert_bits_equal(got[h * Nq:(h + 1) * Nq], want, f"seed {seed}: attention causal={causal} H={H} {Nq}x{Nk} d={d} w={w} base={base} head {h}")
     assert rg.rg_device_status() == 0
