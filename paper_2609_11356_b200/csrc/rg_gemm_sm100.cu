@@ -350,10 +350,10 @@ __device__ __forceinline__ void grouped_finish(const GemmParams& p, const int BN
   }
 }
 
-// KSUB: 64-wide boxes per pipeline stage (BK = 64 * KSUB).  The tile width p.bn is a run-time value:
+// KSUB: 64-wide boxes per pipeline stage (BK = 64 * KSUB); F8: e4m3 operands (kind::f8f6f4).  The tile width p.bn is a run-time value:
 // any multiple of 16 up to 256 is a legal step width, which lets the host size tiles so that the
 // work items fill whole waves.
-template <int KSUB>
+template <int KSUB, bool F8>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const GemmParams p) {
@@ -473,7 +473,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             for (int a = 0; a < KBOX / UMMA_K; ++a) {
               // ascending k; steps at or past the end of the part are not issued
               if (k0 + sub * KBOX + a * UMMA_K < k_end) {
-                if (p.f8) umma_f8(d_tmem, adesc + 2u * a, bdesc + 2u * a, IDESC, accumulate);
+                // the operand kind is a template parameter: a run-time test here slowed the issuing thread
+                // enough to cost the weight-streaming shapes 5 us per call
+                if (F8) umma_f8(d_tmem, adesc + 2u * a, bdesc + 2u * a, IDESC, accumulate);
                 else umma_bf16(d_tmem, adesc + 2u * a, bdesc + 2u * a, IDESC, accumulate);
                 accumulate = 1;
               }
@@ -918,12 +920,12 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const Gemm
   return launch_pair_t<BN, KSUB, KIND_BF16>(ta, tb, p, grid, st);
 }
 
-template <int KSUB>
-cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
+template <int KSUB, bool F8>
+cudaError_t launch_one_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   const size_t smem = smem_bytes_for(p.bn, KSUB, p.num_stages, (int)(p.a_box_bytes / (KBOX * 2)));
   static size_t configured = 0;
   if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<KSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<KSUB, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
     if (e != cudaSuccess) return e;
     configured = SMEM_LIMIT;
   }
@@ -939,7 +941,12 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmP
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<KSUB>, ta, tb, p);
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<KSUB, F8>, ta, tb, p);
+}
+
+template <int KSUB>
+cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
+  return p.f8 ? launch_one_t<KSUB, true>(ta, tb, p, grid, st) : launch_one_t<KSUB, false>(ta, tb, p, grid, st);
 }
 
 }  // namespace
