@@ -443,6 +443,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       int stage = 0; uint32_t phase = 0;
       bool alive = true;
       int gc = 0;                                         // accumulators handed to the epilogue so far
+      const uint64_t desc_a0 = make_kmajor_sw128_desc(smem_base);
+      const uint64_t desc_b0 = make_kmajor_sw128_desc(smem_base + KSUB * A_BOX_BYTES);
       for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);
@@ -464,20 +466,37 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           }
           if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0x300u | stage)) { alive = false; break; }
           tcgen05_fence_after();
-          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          // descriptors differ from the stage-0 ones only in the 16-byte-unit start address (low word).
+          // The operand kind is a template parameter: a run-time test in front of every step slowed
+          // this thread enough to cost the weight-streaming shapes 5 us per call.
+          const uint64_t adesc0 = desc_a0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
+          const uint64_t bdesc0 = desc_b0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
+          if (k0 + KBOX * KSUB <= k_end) {
+            // whole stage inside the part: 4*KSUB steps, ascending k, no per-step tests
 #pragma unroll
-          for (int sub = 0; sub < KSUB; ++sub) {
-            const uint64_t adesc = make_kmajor_sw128_desc(sa + sub * A_BOX_BYTES);
-            const uint64_t bdesc = make_kmajor_sw128_desc(sa + KSUB * A_BOX_BYTES + sub * B_BOX_BYTES);
+            for (int sub = 0; sub < KSUB; ++sub) {
 #pragma unroll
-            for (int a = 0; a < KBOX / UMMA_K; ++a) {
-              // ascending k; steps at or past the end of the part are not issued
-              if (k0 + sub * KBOX + a * UMMA_K < k_end) {
-                // the operand kind is a template parameter: a run-time test here slowed the issuing thread
-                // enough to cost the weight-streaming shapes 5 us per call
-                if (F8) umma_f8(d_tmem, adesc + 2u * a, bdesc + 2u * a, IDESC, accumulate);
-                else umma_bf16(d_tmem, adesc + 2u * a, bdesc + 2u * a, IDESC, accumulate);
-                accumulate = 1;
+              for (int a = 0; a < KBOX / UMMA_K; ++a) {
+                const uint64_t ad = adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a;
+                const uint64_t bd = bdesc0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a;
+                if (F8) umma_f8(d_tmem, ad, bd, IDESC, (sub | a) ? 1u : accumulate);
+                else umma_bf16(d_tmem, ad, bd, IDESC, (sub | a) ? 1u : accumulate);
+              }
+            }
+            accumulate = 1;
+          } else {
+#pragma unroll
+            for (int sub = 0; sub < KSUB; ++sub) {
+#pragma unroll
+              for (int a = 0; a < KBOX / UMMA_K; ++a) {
+                // ascending k; steps at or past the end of the part are not issued
+                if (k0 + sub * KBOX + a * UMMA_K < k_end) {
+                  const uint64_t ad = adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a;
+                  const uint64_t bd = bdesc0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a;
+                  if (F8) umma_f8(d_tmem, ad, bd, IDESC, accumulate);
+                  else umma_bf16(d_tmem, ad, bd, IDESC, accumulate);
+                  accumulate = 1;
+                }
               }
             }
           }
