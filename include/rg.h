@@ -167,20 +167,6 @@ size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N);
 rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
                     const rg_epilogue_t* epi, void* ws, size_t ws_bytes, void* cuda_stream);
 
-/* rg_gemm with the split-K merge inside the GEMM kernel (Sec. 7 "single launch across split-K
- * slices"): the same parts, the same tree, the same bits as rg_gemm, one kernel launch instead of two.
- * Every CTA counts the part it has written on its output tile's counter, and the CTA that counts a tile's
- * last part merges that tile; which CTA that is changes nothing, since it reads all parts back from the
- * workspace and folds them in the descriptor's order.  `counters`: device memory, 4-byte aligned, at
- * least rg_gemm_fused_merge_counters(d, M, N) entries, owned by the caller, which must be ZERO on entry;
- * the call leaves them zero, so one cudaMemset after allocation serves every later call.  Calls that
- * share counters or workspace must not overlap on the GPU.  Shapes that run on the two-SM kernel
- * (large M) ignore the counters and use the merge kernel.  Without cuts this is rg_gemm. */
-size_t rg_gemm_fused_merge_counters(const rg_desc_t* d, int64_t M, int64_t N);
-rg_status_t rg_gemm_fused_merge(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
-                                const rg_epilogue_t* epi, void* ws, size_t ws_bytes, uint32_t* counters, size_t n_counters,
-                                void* cuda_stream);
-
 /* Row reductions with a fixed tree over the columns (Sec. 3.1, Sec. 5.1; kernels named in
  * Sec. 7: row sums, softmax, rmsnorm).  `d->tree` (BALANCED only on the GPU), `d->acc_dtype`
  * (fp32) and `d->fma` apply; the leaves are the `x.cols` columns in index order.

@@ -26,8 +26,7 @@ RG_NOALLOC_WS_BYTES = 8 << 20
 EXPORTS = ["rg_desc_init", "rg_desc_validate", "rg_desc_class", "rg_gemm_workspace_bytes", "rg_gemm",
            "rg_reduce_rows", "rg_gemm_host_scratch_bytes", "rg_gemm_host", "rg_reduce_rows_host_scratch_bytes",
            "rg_reduce_rows_host", "rg_device_status", "rg_status_string", "rg_gemm_noalloc",
-           "rg_reduce_cols_workspace_bytes", "rg_reduce_cols", "rg_attention",
-           "rg_gemm_fused_merge_counters", "rg_gemm_fused_merge"]
+           "rg_reduce_cols_workspace_bytes", "rg_reduce_cols", "rg_attention"]
 
 
 class rg_attn_desc_t(C.Structure):
@@ -86,8 +85,6 @@ def load():
     L.rg_reduce_rows_host.restype = C.c_int; L.rg_reduce_rows_host.argtypes = [D, C.c_int, T, T, A, vp, sz, vp]
     L.rg_reduce_cols_workspace_bytes.restype = sz; L.rg_reduce_cols_workspace_bytes.argtypes = [i64, i64]
     L.rg_reduce_cols.restype = C.c_int; L.rg_reduce_cols.argtypes = [D, C.c_int, T, T, T, vp, sz, vp]
-    L.rg_gemm_fused_merge_counters.restype = sz; L.rg_gemm_fused_merge_counters.argtypes = [D, i64, i64]
-    L.rg_gemm_fused_merge.restype = C.c_int; L.rg_gemm_fused_merge.argtypes = [D, T, T, T, E, vp, sz, vp, sz, vp]
     L.rg_attention.restype = C.c_int; L.rg_attention.argtypes = [C.POINTER(rg_attn_desc_t), T, T, T, T, vp]
     L.rg_gemm_noalloc.restype = C.c_int; L.rg_gemm_noalloc.argtypes = [D, T, T, T, E, vp]
     L.rg_device_status.restype = C.c_int; L.rg_device_status.argtypes = [C.POINTER(C.c_uint32)]

@@ -118,26 +118,6 @@ def rg_gemm(d: K.rg_desc_t, A, B, C_out, *, bias=None, act: int = 0, residual=No
     return C_out
 
 
-def rg_gemm_fused_merge_counters(d: K.rg_desc_t, M: int, N: int) -> int:
-    return int(K.load().rg_gemm_fused_merge_counters(C.byref(d), M, N))
-
-
-def rg_gemm_fused_merge(d: K.rg_desc_t, A, B, C_out, counters, *, bias=None, act: int = 0, residual=None, ws=None):
-    """rg_gemm with the split-K merge inside the GEMM kernel (one launch).  `counters`: a CUDA int32
-    tensor of at least rg_gemm_fused_merge_counters(d, M, N) entries that is zero on entry (zero it once
-    after allocation; every call leaves it zero)."""
-    L = K.load()
-    a, b, c = _tensor(A), _tensor(B), _tensor(C_out)
-    e = _epilogue(bias, act, residual)
-    ws_ptr = ws.data_ptr() if ws is not None else None
-    ws_bytes = ws.numel() * ws.element_size() if ws is not None else 0
-    st = L.rg_gemm_fused_merge(C.byref(d), C.byref(a), C.byref(b), C.byref(c), C.byref(e) if e is not None else None,
-                               ws_ptr, ws_bytes, counters.data_ptr() if counters is not None else None,
-                               counters.numel() if counters is not None else 0, _stream(A))
-    _check(st, "rg_gemm_fused_merge")
-    return C_out
-
-
 def rg_gemm_noalloc(d: K.rg_desc_t, A, B, C_out, *, bias=None, act: int = 0, residual=None):
     """rg_gemm for callers that cannot allocate device memory: the split-K workspace is a fixed
     array inside the library (at most RG_NOALLOC_WS_BYTES; larger shapes raise RG_ERR_WORKSPACE).

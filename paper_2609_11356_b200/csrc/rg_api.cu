@@ -189,9 +189,8 @@ size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N) {
   return (size_t)(d->n_cuts + 1) * (size_t)M * (size_t)((N + 3) / 4 * 4) * (d->partial_dtype == RG_F32 ? 4 : 2);
 }
 
-static rg_status_t gemm_impl(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
-                             const rg_epilogue_t* epi, void* ws, size_t ws_bytes, unsigned int* counters, size_t n_counters,
-                             bool want_counters, void* cuda_stream) {
+rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
+                    const rg_epilogue_t* epi, void* ws, size_t ws_bytes, void* cuda_stream) {
   rg_status_t s = check_desc_fields(d);
   if (s != RG_OK) return s;
   if ((s = check_gemm_shapes(A, B, C)) != RG_OK) return s;
@@ -200,10 +199,6 @@ static rg_status_t gemm_impl(const rg_desc_t* d, const rg_tensor_t* A, const rg_
   if ((s = rg_desc_validate(d, M, N, K)) != RG_OK) return s;
   if (A->dtype != d->in_dtype) return RG_ERR_SHAPE;          // operands must be of the descriptor's input type
   if ((s = check_epilogue(epi, N)) != RG_OK) return s;
-  if (want_counters && d->n_cuts) {
-    if (!counters) return RG_ERR_NULL;
-    if ((reinterpret_cast<uintptr_t>(counters) & 3) || n_counters < rg_gemm_fused_merge_counters(d, M, N)) return RG_ERR_WORKSPACE;
-  }
   if (M == 0 || N == 0) return RG_OK;
   const int64_t ld_mult = 16 / (int64_t)esize(A->dtype);        // rows start on 16-byte boundaries
   if ((reinterpret_cast<uintptr_t>(A->ptr) & 15) || (reinterpret_cast<uintptr_t>(B->ptr) & 15) ||
@@ -217,23 +212,7 @@ static rg_status_t gemm_impl(const rg_desc_t* d, const rg_tensor_t* A, const rg_
   if (d->atom == RG_ATOM_SCALAR) return rg::launch_gemv(d, A, B, C, epi, static_cast<cudaStream_t>(cuda_stream));
   rg::GemmPlan plan;
   if ((s = make_plan(d, M, N, K, &plan)) != RG_OK) return s;
-  return rg::launch_gemm(plan, A, B, C, epi, ws, static_cast<cudaStream_t>(cuda_stream), d->n_cuts ? counters : nullptr);
-}
-
-size_t rg_gemm_fused_merge_counters(const rg_desc_t* d, int64_t M, int64_t N) {
-  if (!d || d->n_cuts == 0 || M <= 0 || N <= 0) return 0;
-  return (size_t)((M + 127) / 128) * (size_t)((N + 15) / 16);   // one per output tile of the narrowest tile width
-}
-
-rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
-                    const rg_epilogue_t* epi, void* ws, size_t ws_bytes, void* cuda_stream) {
-  return gemm_impl(d, A, B, C, epi, ws, ws_bytes, nullptr, 0, false, cuda_stream);
-}
-
-rg_status_t rg_gemm_fused_merge(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
-                                const rg_epilogue_t* epi, void* ws, size_t ws_bytes, uint32_t* counters, size_t n_counters,
-                                void* cuda_stream) {
-  return gemm_impl(d, A, B, C, epi, ws, ws_bytes, counters, n_counters, true, cuda_stream);
+  return rg::launch_gemm(plan, A, B, C, epi, ws, static_cast<cudaStream_t>(cuda_stream));
 }
 
 static rg_status_t check_reduce(const rg_desc_t* d, rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out) {

@@ -180,18 +180,6 @@ __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }
 
-// What the split-K merge needs: the parts, the tree, and the output with its epilogue.
-struct FixupParams {
-  const void* ws;
-  int64_t ldw;
-  int32_t M, N, S, tree;
-  int32_t partial_dtype, merge_dtype;
-  void* C;
-  int64_t ldc;
-  int32_t c_dtype;
-  EpilogueArgs epi;
-};
-
 struct GemmParams {
   int32_t M, N, K;
   int32_t tiles_m, tiles_n, n_parts;
@@ -209,16 +197,9 @@ struct GemmParams {
   int64_t ldw;
   int32_t ws_dtype;
   EpilogueArgs epi;
-  // single-launch split-K (one-CTA kernel): one counter per output tile, zero on entry and left zero;
-  // the CTA that delivers a tile's last part merges the tile.  Null: a merge kernel follows instead.
-  unsigned int* tile_counters;
-  FixupParams merge;
   int32_t part_begin[RG_MAX_CUTS + 1];
   int32_t part_end[RG_MAX_CUTS + 1];
 };
-
-template <bool PART_16, bool MERGE_16>
-__device__ __forceinline__ void merge_group(const FixupParams& p, const int64_t row, const int col0);
 
 __device__ __forceinline__ void decode_work(const GemmParams& p, int w, int& part, int& tm, int& tn) {
   const int tiles = p.tiles_m * p.tiles_n;
@@ -401,7 +382,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t bar_tempty = bar_tfull + 16u;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* merge_flag = abort_flag + 1;              // single-launch split-K: this CTA merges the tile it just finished
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int total_work = p.tiles_m * p.tiles_n * p.n_parts;
@@ -533,13 +513,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     bool alive = true;
     bool deps_done = false;
     int gc = 0;
-    const bool fused = p.tile_counters != nullptr;        // single launch: the last part's CTA merges the tile
-    const int etid = (warp - 2) * 32 + lane;              // 0..255 among the epilogue threads
-    for (int w = blockIdx.x; w < total_work; w += gridDim.x) {
-      // Without the in-kernel merge a role that gave up leaves the loop.  With it, the epilogue
-      // threads meet at two barriers per work item, so a thread that gave up keeps walking the
-      // loop (touching neither tensor memory nor global memory) until all items are done.
-      if (!alive && !fused) break;
+    for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
       int part, tm, tn;
       decode_work(p, w, part, tm, tn);
       const int64_t row = (int64_t)tm * BM + quarter * 32 + lane;
@@ -548,23 +522,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       const int ngroups = p.inner_span > 0 ? (klen + p.inner_span - 1) / p.inner_span : 1;
       if (ngroups == 1) {
         const int buf = gc & 1;
-        if (alive) alive = mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf);
-        if (alive) {
-          tcgen05_fence_after();
-          if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
-          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
-          epilogue_tile(p, BN, part, row, row_ok, tn, taddr, chunk0);
-          tcgen05_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
-        }
+        if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
+        tcgen05_fence_after();
+        if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
+        epilogue_tile(p, BN, part, row, row_ok, tn, taddr, chunk0);
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
         ++gc;
       } else {
         GroupedAcc acc;
-        for (int g = 0; g < ngroups; ++g, ++gc) {
+        for (int g = 0; g < ngroups && alive; ++g, ++gc) {
           const int buf = gc & 1;
-          if (alive) alive = mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf);
-          if (!alive) continue;
+          if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
           tcgen05_fence_after();
           if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
@@ -574,34 +545,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
         }
         if (alive) grouped_finish(p, BN, part, row, row_ok, tn, chunk0, acc);
-      }
-      if (fused) {
-        // This CTA's part of the tile is in the workspace.  Count it; whoever counts the last part
-        // merges the tile in the descriptor's tree (the same code the merge kernel runs, so the
-        // bits do not depend on which CTA comes last) and leaves the counter at zero.
-        __threadfence();                                   // the part is visible device-wide before it is counted
-        asm volatile("bar.sync 2, 256;" ::: "memory");
-        if (etid == 0) {
-          unsigned int last = 0;
-          if (alive) {
-            unsigned int* cnt = p.tile_counters + (tm * p.tiles_n + tn);
-            last = atomicAdd(cnt, 1u) == (unsigned int)(p.n_parts - 1);
-            if (last) *cnt = 0u;
-          }
-          *merge_flag = (int)last;
-        }
-        asm volatile("bar.sync 2, 256;" ::: "memory");
-        if (*merge_flag) {
-          __threadfence();                                 // the other CTAs' parts, counted before ours
-          const int row_lo = tm * BM, rows = min(BM, p.M - row_lo);
-          const int col_lo = tn * BN, groups = (min(BN, p.N - col_lo) + 3) >> 2;
-          for (int i = etid; i < rows * groups; i += NUM_EPI_WARPS * 32) {
-            const int r = i / groups, c4 = i - r * groups;
-            if (p.merge.partial_dtype == RG_F32) merge_group<false, false>(p.merge, row_lo + r, col_lo + 4 * c4);
-            else if (p.merge.merge_dtype == RG_F32) merge_group<true, false>(p.merge, row_lo + r, col_lo + 4 * c4);
-            else merge_group<true, true>(p.merge, row_lo + r, col_lo + 4 * c4);
-          }
-        }
       }
     }
   }
@@ -794,24 +737,45 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 }
 
 // -------------------------------------------------------------- split-K merge
+struct FixupParams {
+  const void* ws;
+  int64_t ldw;
+  int32_t M, N, S, tree;
+  int32_t partial_dtype, merge_dtype;
+  void* C;
+  int64_t ldc;
+  int32_t c_dtype;
+  EpilogueArgs epi;
+};
+
 // One thread per (row, 4 consecutive columns).  The parts are combined in the descriptor's tree
 // with fp32 adds, the running sum kept at merge_dtype (an add whose result is rounded to bf16 when
 // the sum is kept at bf16); BALANCED is evaluated with a binary-counter stack, which visits
 // exactly the aligned pairs of the level-by-level definition.
 template <bool PART_16, bool MERGE_16>
-__device__ __forceinline__ void merge_group(const FixupParams& p, const int64_t row, const int col0) {
+__global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) {
+  const int64_t ncol4 = (p.N + 3) / 4;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  // launched with programmatic stream serialisation: the grid may start while the GEMM kernel is
+  // still draining; nothing is read before that kernel has completed and flushed its stores.  A
+  // kernel launched the same way behind this one may set itself up meanwhile.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (idx >= (int64_t)p.M * ncol4) return;
+  const int64_t row = idx / ncol4;
+  const int col0 = (int)(idx - row * ncol4) * 4;
   const int64_t part_stride = (int64_t)p.M * p.ldw;
   const int64_t off = row * p.ldw + col0;
   auto load = [&](int s) -> float4 {
     if (PART_16) {
-      const uint2 w = __ldcg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.ws) + s * part_stride + off));
+      const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.ws) + s * part_stride + off);
       if (p.partial_dtype == RG_F16)
         return make_float4(f16_bits_to_f32(w.x & 0xffffu), f16_bits_to_f32(w.x >> 16),
                            f16_bits_to_f32(w.y & 0xffffu), f16_bits_to_f32(w.y >> 16));
       return make_float4(bf16_bits_to_f32(w.x & 0xffffu), bf16_bits_to_f32(w.x >> 16),
                          bf16_bits_to_f32(w.y & 0xffffu), bf16_bits_to_f32(w.y >> 16));
     }
-    return __ldcg(reinterpret_cast<const float4*>(static_cast<const float*>(p.ws) + s * part_stride + off));
+    return *reinterpret_cast<const float4*>(static_cast<const float*>(p.ws) + s * part_stride + off);
   };
   const int merge_dtype = p.merge_dtype;
   auto add1 = [merge_dtype](float a, float b) -> float {
@@ -892,21 +856,6 @@ __device__ __forceinline__ void merge_group(const FixupParams& p, const int64_t 
     for (int c = 0; c < 4; ++c)
       if (col0 + c < p.N) store_scalar(p.C, p.c_dtype, row * p.ldc + col0 + c, v[c]);
   }
-}
-
-// The merge as a kernel of its own: one thread per (row, 4 consecutive columns).
-template <bool PART_16, bool MERGE_16>
-__global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) {
-  const int64_t ncol4 = (p.N + 3) / 4;
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  // launched with programmatic stream serialisation: the grid may start while the GEMM kernel is
-  // still draining; nothing is read before that kernel has completed and flushed its stores.  A
-  // kernel launched the same way behind this one may set itself up meanwhile.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (idx >= (int64_t)p.M * ncol4) return;
-  const int64_t row = idx / ncol4;
-  merge_group<PART_16, MERGE_16>(p, row, (int)(idx - row * ncol4) * 4);
 }
 
 // ------------------------------------------------------------ host: tensor maps
@@ -1047,7 +996,7 @@ rg_status_t read_and_clear_status(uint32_t* code) {
 
 // Launch the GEMM (and the merge when there are cuts).  All arguments were validated by the caller.
 rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
-                        const rg_epilogue_t* epi, void* ws, cudaStream_t st, unsigned int* tile_counters) {
+                        const rg_epilogue_t* epi, void* ws, cudaStream_t st) {
   // e4m3 operands: every K quantity below (K, part bounds, inner span) counts byte pairs, so the
   // kernels walk 32-byte steps of an operand row exactly as they do for 16-bit operands
   const int kdiv = A->dtype == RG_F8E4M3 ? 2 : 1;
@@ -1088,15 +1037,6 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   p.ldw = (N + 3) / 4 * 4;
   p.epi = split ? EpilogueArgs{} : e;
 
-  // Single launch: the one-CTA kernel merges each tile itself when the caller supplied counters.
-  FixupParams f;
-  f.ws = ws; f.ldw = p.ldw; f.partial_dtype = plan.partial_dtype; f.merge_dtype = plan.merge_dtype;
-  f.M = p.M; f.N = p.N; f.S = plan.n_parts; f.tree = plan.tree;
-  f.C = C->ptr; f.ldc = C->ld; f.c_dtype = C->dtype; f.epi = e;
-  const bool fused = split && !pair && tile_counters != nullptr;
-  p.tile_counters = fused ? tile_counters : nullptr;
-  p.merge = f;
-
   const int64_t total = (int64_t)p.tiles_m * p.tiles_n * p.n_parts;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
@@ -1120,7 +1060,11 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   }
   if (err != cudaSuccess) return RG_ERR_CUDA;
 
-  if (split && !fused) {
+  if (split) {
+    FixupParams f;
+    f.ws = ws; f.ldw = p.ldw; f.partial_dtype = plan.partial_dtype; f.merge_dtype = plan.merge_dtype;
+    f.M = p.M; f.N = p.N; f.S = plan.n_parts; f.tree = plan.tree;
+    f.C = C->ptr; f.ldc = C->ld; f.c_dtype = C->dtype; f.epi = e;
     const int64_t items = M * ((N + 3) / 4);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)((items + 255) / 256), 1, 1);

@@ -21,7 +21,7 @@ struct GemmPlan {
 
 int max_stages_for(int bn, int bk, int cta_group, int64_t M);
 rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
-                        const rg_epilogue_t* epi, void* ws, cudaStream_t st, unsigned int* tile_counters = nullptr);
+                        const rg_epilogue_t* epi, void* ws, cudaStream_t st);
 rg_status_t launch_gemv(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
                         const rg_epilogue_t* epi, cudaStream_t st);
 rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* out,
