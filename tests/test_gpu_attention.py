@@ -98,6 +98,25 @@ def test_rows_are_independent_of_the_query_tile_and_runs_repeat():
     assert rg.rg_device_status() == 0
 
 
+def test_strided_operands_and_fp16_output():
+    H, Nq, Nk, d = 2, 150, 270, 64
+    Q, K, V = _draw(Nq, Nk, d, 41, heads=H)
+    scale = 0.125
+    pad = lambda a, extra: torch.cat([synth.to_torch(a, DEV), torch.full((a.shape[0], extra), float("nan"), dtype=torch.bfloat16, device=DEV)], 1)
+    Qp, Kp = pad(Q, 8), pad(K, 24)                          # leading dimensions 72 and 88: rows still 16-byte aligned
+    Vt = np.ascontiguousarray(V.reshape(H, Nk, d).transpose(0, 2, 1)).reshape(H * d, Nk)
+    vt = torch.full((H * d, 280), float("nan"), dtype=torch.bfloat16, device=DEV); vt[:, :Nk] = synth.to_torch(Vt, DEV)
+    Op = torch.full((H * Nq, d + 8), float("nan"), dtype=torch.float16, device=DEV)
+    rg.rg_attention(rg.rg_attn_desc(block_n=64, scale=scale, heads=H), Qp[:, :d], Kp[:, :d], vt[:, :Nk], Op[:, :d])
+    torch.cuda.synchronize()
+    got = Op[:, :d].cpu().numpy()
+    assert torch.isnan(Op[:, d:]).all()                     # nothing written past the output's columns
+    for h in range(H):
+        want = rgo.attention(Q[h * Nq:(h + 1) * Nq], K[h * Nk:(h + 1) * Nk], V[h * Nk:(h + 1) * Nk], block_n=64, scale=scale,
+                             atom_model=HW, out_dtype=rgo.F16)
+        assert_bits_equal(got[h * Nq:(h + 1) * Nq], want, f"strided, fp16 out, head {h}")
+
+
 def test_argument_errors():
     q = torch.zeros((128, 128), dtype=torch.bfloat16, device=DEV); k = torch.zeros((256, 128), dtype=torch.bfloat16, device=DEV)
     vt = torch.zeros((128, 256), dtype=torch.bfloat16, device=DEV); o = torch.zeros((128, 128), dtype=torch.bfloat16, device=DEV)
