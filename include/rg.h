@@ -1,4 +1,4 @@
-/* rg — reduction-order-fixed GEMM and row reductions for NVIDIA B200 (sm_100a).
+/* rg — reduction-order-fixed GEMM, reductions and attention for NVIDIA B200 (sm_100a).
  *
  * C ABI.  Every result's bits are decided by a reduction-order descriptor and by nothing
  * else: not by the tile shape, the batch size M, the launch, or the run.  The descriptor is
@@ -91,7 +91,7 @@ typedef struct {
   uint32_t cuts[RG_MAX_CUTS]; /* 0 < cuts[0] < ... < cuts[n_cuts-1] < K; part s = [cuts[s-1], cuts[s]) */
   uint32_t inner_span;    /* second level of the cut nest (Sec. 3.2.2; App. E per-group accumulation): 0 = none;
                              else, inside every part, an accumulator is closed every inner_span k (a multiple
-                             of 64) and the closed groups are added at fp32, in ascending order, into the
+                             of 64; of 128 with e4m3 operands) and the closed groups are added at fp32, in ascending order, into the
                              part's running sum.  Order-deciding: part of the class key. */
   uint8_t gemv_layout;    /* RG_ATOM_SCALAR only: how the 32 lanes of a warp deal the 8-wide k tiles of one output
                              element (Sec. 3.2.2 "GEMV", `layout`): 0 = strided (lane l takes tiles l, l+32, ...),
@@ -136,7 +136,8 @@ typedef struct {
 void rg_desc_init(rg_desc_t* d);
 
 /* Check a descriptor against a GEMM shape (Sec. 3.2.2: cuts are contiguous parts of the
- * contracted axis).  Host only.  Cuts must be strictly increasing multiples of 16 inside (0, K). */
+ * contracted axis).  Host only.  Cuts must be strictly increasing multiples of the step width (16; 32
+ * with e4m3 operands) inside (0, K). */
 rg_status_t rg_desc_validate(const rg_desc_t* d, int64_t M, int64_t N, int64_t K);
 
 /* Equivalence-class key (Sec. 4: a descriptor holds every order-deciding factor "and nothing
