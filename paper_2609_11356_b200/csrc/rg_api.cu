@@ -336,8 +336,14 @@ rg_status_t rg_gemm_host(const rg_desc_t* d, const rg_tensor_t* A, const rg_tens
   rg_epilogue_t de{};
   if (epi) de = *epi;
   bool ok = true;
-  ok &= cudaMemcpy2DAsync(dA.ptr, ldk * ies, A->ptr, A->ld * ies, K * ies, M, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpy2DAsync(dB.ptr, ldk * ies, B->ptr, B->ld * ies, K * ies, N, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  // rows that are already dense on both sides go as one flat copy
+  auto h2d_rows = [&](void* dst, int64_t dst_ld, const void* src, int64_t src_ld, int64_t cols, int64_t rows, size_t es) {
+    if (dst_ld == cols && src_ld == cols)
+      return cudaMemcpyAsync(dst, src, (size_t)rows * cols * es, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    return cudaMemcpy2DAsync(dst, dst_ld * es, src, src_ld * es, cols * es, rows, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  };
+  ok &= h2d_rows(dA.ptr, ldk, A->ptr, A->ld, K, M, ies);
+  ok &= h2d_rows(dB.ptr, ldk, B->ptr, B->ld, K, N, ies);
   if (epi && epi->bias) {
     void* p = take((size_t)N * esize(epi->bias_dtype));
     ok &= cudaMemcpyAsync(p, epi->bias, (size_t)N * esize(epi->bias_dtype), cudaMemcpyHostToDevice, st) == cudaSuccess;
@@ -354,8 +360,9 @@ rg_status_t rg_gemm_host(const rg_desc_t* d, const rg_tensor_t* A, const rg_tens
   void* ws = wsb ? take(wsb) : nullptr;
   if ((s = rg_gemm(d, &dA, &dB, &dC, epi ? &de : nullptr, ws, wsb, cuda_stream)) != RG_OK) return s;
   const size_t ces = esize(C->dtype);
-  if (cudaMemcpy2DAsync(C->ptr, C->ld * ces, dC.ptr, N * ces, N * ces, M, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-    return RG_ERR_CUDA;
+  const cudaError_t ce = C->ld == N ? cudaMemcpyAsync(C->ptr, dC.ptr, (size_t)M * N * ces, cudaMemcpyDeviceToHost, st)
+                                    : cudaMemcpy2DAsync(C->ptr, C->ld * ces, dC.ptr, N * ces, N * ces, M, cudaMemcpyDeviceToHost, st);
+  if (ce != cudaSuccess) return RG_ERR_CUDA;
   return RG_OK;
 }
 
