@@ -171,6 +171,24 @@ __device__ __forceinline__ void umma_pair(uint32_t d_tmem, uint64_t a_desc, uint
   else umma_bf16_pair(d_tmem, a_desc, b_desc, idesc, accumulate);
 }
 
+// The same step with the shared-memory descriptors given as (low word, high word): only the low word
+// (the 16-byte-unit start address) changes from step to step, so the issuing thread does 32-bit adds.
+// ACC: compile-time "accumulate onto D" (every step of a part but its first).
+template <int KIND, bool ACC>
+__device__ __forceinline__ void umma_pair_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
+  if (KIND == KIND_F8E4M3) {
+    if (ACC) asm volatile("{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.eq.b32 p, %0, %0;\n\t"
+                          "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc) : "memory");
+    else asm volatile("{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                      "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+  } else {
+    if (ACC) asm volatile("{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.eq.b32 p, %0, %0;\n\t"
+                          "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc) : "memory");
+    else asm volatile("{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+  }
+}
+
 __host__ __device__ constexpr uint32_t make_idesc(int bn, int m, uint32_t fmt) {
   return (1u << 4) | (fmt << 7) | (fmt << 10) | (static_cast<uint32_t>(bn >> 3) << 17) |
          (static_cast<uint32_t>(m >> 4) << 24);
@@ -670,13 +688,16 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
           const uint64_t adesc0 = desc_a0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
           const uint64_t bdesc0 = desc_b0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
           if (k0 + KBOX * KSUB <= k_end) {
-            // whole stage inside the part: 4*KSUB steps, ascending k, no per-step tests
+            // whole stage inside the part: 4*KSUB steps, ascending k, no per-step tests; the descriptors'
+            // high words are the same for every tile, and the low words never carry into them
+            const uint32_t a_lo = (uint32_t)adesc0, b_lo = (uint32_t)bdesc0, hi = (uint32_t)(desc_a0 >> 32);
 #pragma unroll
             for (int sub = 0; sub < KSUB; ++sub) {
 #pragma unroll
               for (int a = 0; a < KBOX / UMMA_K; ++a) {
-                umma_pair<KIND>(d_tmem, adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a,
-                               bdesc0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a, IDESC, (sub | a) ? 1u : accumulate);
+                const uint32_t al = a_lo + ((sub * A_BOX_BYTES) >> 4) + 2u * a, bl = b_lo + ((sub * B_BOX_BYTES) >> 4) + 2u * a;
+                if (sub | a) umma_pair_lo<KIND, true>(d_tmem, al, bl, hi, IDESC, 1u);
+                else umma_pair_lo<KIND, false>(d_tmem, al, bl, hi, IDESC, accumulate);
               }
             }
             accumulate = 1;
