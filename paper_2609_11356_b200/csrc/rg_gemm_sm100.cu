@@ -671,6 +671,20 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       int it = 0;
       const uint64_t desc_a0 = make_kmajor_sw128_desc(smem_base);
       const uint64_t desc_b0 = make_kmajor_sw128_desc(smem_base + KSUB * A_BOX_BYTES);
+      // With a ring of exactly three stages (the default of the widest tile) whole turns of the ring are
+      // issued from descriptor words computed once, with every barrier address a constant: this thread's
+      // instruction stream is on the critical path whenever the epilogue warps compete for issue slots.
+      constexpr int G = 3, STEPS = KSUB * (KBOX / UMMA_K);
+      const uint32_t desc_hi = (uint32_t)(desc_a0 >> 32);
+      uint32_t alo[G][STEPS], blo[G][STEPS];
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+#pragma unroll
+        for (int i = 0; i < STEPS; ++i) {
+          const uint32_t off = (uint32_t)((g * STAGE_BYTES) >> 4) + 2u * (i % (KBOX / UMMA_K));
+          alo[g][i] = (uint32_t)desc_a0 + off + (((i / (KBOX / UMMA_K)) * A_BOX_BYTES) >> 4);
+          blo[g][i] = (uint32_t)desc_b0 + off + (((i / (KBOX / UMMA_K)) * B_BOX_BYTES) >> 4);
+        }
       for (int w = pair_id; w < total_work && alive; w += num_pairs, ++it) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);
@@ -682,6 +696,27 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         const uint32_t d_tmem = tmem_base + buf * BN;
         uint32_t accumulate = 0;                        // every part starts from a zero accumulator
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
+          if (S == G && stage == 0 && k0 + G * KBOX * KSUB <= k_end) {
+            // one whole turn of the ring
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+              if (alive && !mbar_wait(bar_full + 8u * g, phase, abort_flag, &g_status_word, 0xb00u | g)) alive = false;
+              if (alive) {
+                tcgen05_fence_after();
+#pragma unroll
+                for (int i = 0; i < STEPS; ++i) {
+                  if (g | i) umma_pair_lo<KIND, true>(d_tmem, alo[g][i], blo[g][i], desc_hi, IDESC, 1u);
+                  else umma_pair_lo<KIND, false>(d_tmem, alo[0][0], blo[0][0], desc_hi, IDESC, accumulate);
+                }
+                umma_commit_pair(bar_empty + 8u * g);
+              }
+            }
+            if (!alive) break;
+            accumulate = 1;
+            phase ^= 1u;
+            k0 += (G - 1) * KBOX * KSUB;                  // the loop adds the last stage's width
+            continue;
+          }
           if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0xb00u | stage)) { alive = false; break; }
           tcgen05_fence_after();
           // descriptors differ from the stage-0 ones only in the 16-byte-unit start address (low word)
