@@ -217,7 +217,7 @@ def run_ours(args):
                        "row_sum_gbs": round(sum_gbs, 1),
                        "softmax_gbs": round((4.0 * RED_R * RED_C + 8.0 * RED_R) / (mean[5] * 1e-3) / 1e9, 1),
                        "rmsnorm_gbs": round((4.0 * RMS_R * RMS_C) / (mean[4] * 1e-3) / 1e9, 1)},
-            "roofline": {"bound": "tensor", "kernel": "gemm_tcgen05_pair_kernel<256,2> (two-SM tiles 256x256x128) on 8192^3",
+            "roofline": {"bound": "tensor", "kernel": "gemm_tcgen05_pair_kernel<256,1> (two-SM tiles 256x256x64, seven-stage ring) on 8192^3",
                          "achieved": round(sq_tflops, 1), "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                          "frac": round(sq_tflops / peaks["bf16_tflops_sustained"], 4),
                          "frac_of_burst_peak": round(sq_tflops / peaks["bf16_tflops"], 4),

@@ -134,9 +134,10 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   else if (d->BM == 128) plan->cta_group = 1;
   else plan->cta_group = (plan->BN >= 128 && M > 128 && ((M + 255) / 256) * ((N + plan->BN - 1) / plan->BN) * plan->n_parts >= sms / 2) ? 2 : 1;
   if (plan->cta_group == 2 && plan->BN < 128) plan->cta_group = 1;
-  // a pair moves half the B bytes per CTA, so a 128-wide K step fits three times: fewer hand-offs per k
+  // the widest two-SM tile runs a seven-stage ring of 64-wide K steps: more slack per byte of shared memory than
+  // three 128-wide stages, now that a whole turn of the ring is issued from precomputed descriptor words
   // skinny problems read long runs of each weight row per stage (DRAM likes 512-byte bursts)
-  plan->BK = d->BK ? d->BK : (d->inner_span ? 64 : ((plan->cta_group == 2 && plan->BN == 256) || skinny ? 128 : 64));
+  plan->BK = d->BK ? d->BK : (skinny && !d->inner_span ? 128 : 64);
   if (plan->cta_group == 2 && plan->BN != 128 && plan->BN != 256) return RG_ERR_UNSUPPORTED;
   const int smax = rg::max_stages_for(plan->BN, plan->BK, plan->cta_group, M);
   plan->stages = d->stages ? d->stages : smax;

@@ -674,7 +674,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       // With a ring of exactly three stages (the default of the widest tile) whole turns of the ring are
       // issued from descriptor words computed once, with every barrier address a constant: this thread's
       // instruction stream is on the critical path whenever the epilogue warps compete for issue slots.
-      constexpr int G = 3, STEPS = KSUB * (KBOX / UMMA_K);
+      constexpr int G = KSUB == 2 ? 3 : 7, STEPS = KSUB * (KBOX / UMMA_K);
       const uint32_t desc_hi = (uint32_t)(desc_a0 >> 32);
       uint32_t alo[G][STEPS], blo[G][STEPS];
 #pragma unroll
