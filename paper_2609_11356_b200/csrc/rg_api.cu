@@ -120,24 +120,51 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
     }
     plan->BN = best;
   } else {
-    // largest tile that still gives every SM a work item
-    plan->BN = 64;
-    for (int bn : {256, 128}) {
-      if (tiles_m * ((N + bn - 1) / bn) * plan->n_parts >= sms) { plan->BN = bn; break; }
+    plan->BN = 0;                                         // chosen together with the kernel below
+  }
+  // one CTA per 128-row tile, or a pair of CTAs (two SMs) per 256-row tile
+  int want_group = 0;
+  if (d->inner_span) want_group = 1;
+  else if (d->cta_group) want_group = d->cta_group;
+  else if (d->BM == 256) want_group = 2;
+  else if (d->BM == 128) want_group = 1;
+  if (plan->BN == 0 || (want_group == 0 && !skinny)) {
+    // Time ~ rounds of work items x (tile width + a fixed cost per tile).  Each CTA owns 128 rows either
+    // way; a pair halves the items per slot and the B bytes per CTA.  Fewest rounds of the widest tile
+    // wins, which for one to two rounds is often a narrower one-CTA tile (a 512 x 4096 problem is one
+    // round of 128 x 128 tiles), and for many rounds the 256-wide pair.
+    const int64_t tiles_m2 = (M + 255) / 256;
+    int best_bn = 0, best_group = 0; int64_t best_cost = -1;
+    for (int group = 1; group <= 2; ++group) {
+      if (want_group && group != want_group) continue;
+      if (group == 2 && M <= 128) continue;
+      for (int bn : {256, 128, 64}) {
+        if (d->BN && bn != d->BN) continue;
+        if (group == 2 && bn != 256) continue;
+        if (d->inner_span && bn > 128) continue;
+        const int64_t items = (group == 2 ? tiles_m2 : tiles_m) * ((N + bn - 1) / bn) * plan->n_parts;
+        const int64_t slots = group == 2 ? sms / 2 : sms;
+        const int64_t rounds = (items + slots - 1) / slots;
+        int64_t cost = rounds * (bn + 32) * 100;
+        if (group == 2 && rounds >= 2) cost = cost * 97 / 100;   // more than one round: the pair's lighter B traffic
+        if (group == 1 && rounds == 1) cost = cost * 99 / 100;   // a single round: no cluster set-up
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_bn = bn; best_group = group; }
+      }
     }
+    if (best_bn) {
+      if (plan->BN == 0) plan->BN = best_bn;
+      if (want_group == 0) want_group = best_group;
+    }
+    if (plan->BN == 0) plan->BN = 64;
   }
   if (d->inner_span && plan->BN > 128) plan->BN = 128;
-  // one CTA per 128-row tile, or a pair of CTAs (two SMs) per 256-row tile
-  if (d->inner_span) plan->cta_group = 1;
-  else if (d->cta_group) plan->cta_group = d->cta_group;
-  else if (d->BM == 256) plan->cta_group = 2;
-  else if (d->BM == 128) plan->cta_group = 1;
-  else plan->cta_group = (plan->BN >= 128 && M > 128 && ((M + 255) / 256) * ((N + plan->BN - 1) / plan->BN) * plan->n_parts >= sms / 2) ? 2 : 1;
+  plan->cta_group = want_group ? want_group : 1;
   if (plan->cta_group == 2 && plan->BN < 128) plan->cta_group = 1;
   // the widest two-SM tile runs a seven-stage ring of 64-wide K steps: more slack per byte of shared memory than
   // three 128-wide stages, now that a whole turn of the ring is issued from precomputed descriptor words
   // skinny problems read long runs of each weight row per stage (DRAM likes 512-byte bursts)
-  plan->BK = d->BK ? d->BK : (skinny && !d->inner_span ? 128 : 64);
+  // one-CTA tiles up to 128 columns take 128-wide K steps as well (half the hand-overs; the stage still fits four times)
+  plan->BK = d->BK ? d->BK : (!d->inner_span && (skinny || (plan->cta_group == 1 && plan->BN <= 128)) ? 128 : 64);
   if (plan->cta_group == 2 && plan->BN != 128 && plan->BN != 256) return RG_ERR_UNSUPPORTED;
   const int smax = rg::max_stages_for(plan->BN, plan->BK, plan->cta_group, M);
   plan->stages = d->stages ? d->stages : smax;
