@@ -189,6 +189,22 @@ __device__ __forceinline__ void umma_pair_lo(uint32_t d_tmem, uint32_t a_lo, uin
   }
 }
 
+// One-CTA form of the same: (low word, high word) descriptors, compile-time accumulate.
+template <bool F8, bool ACC>
+__device__ __forceinline__ void umma_one_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
+  if (F8) {
+    if (ACC) asm volatile("{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.eq.b32 p, %0, %0;\n\t"
+                          "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc) : "memory");
+    else asm volatile("{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+  } else {
+    if (ACC) asm volatile("{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.eq.b32 p, %0, %0;\n\t"
+                          "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc) : "memory");
+    else asm volatile("{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+  }
+}
+
 __host__ __device__ constexpr uint32_t make_idesc(int bn, int m, uint32_t fmt) {
   return (1u << 4) | (fmt << 7) | (fmt << 10) | (static_cast<uint32_t>(bn >> 3) << 17) |
          (static_cast<uint32_t>(m >> 4) << 24);
@@ -490,15 +506,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           const uint64_t adesc0 = desc_a0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
           const uint64_t bdesc0 = desc_b0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
           if (k0 + KBOX * KSUB <= k_end) {
-            // whole stage inside the part: 4*KSUB steps, ascending k, no per-step tests
+            // whole stage inside the part: 4*KSUB steps, ascending k, no per-step tests; 32-bit arithmetic on
+            // the descriptors' low words (the high words never change and nothing carries into them)
+            const uint32_t a_lo = (uint32_t)adesc0, b_lo = (uint32_t)bdesc0, hi = (uint32_t)(desc_a0 >> 32);
 #pragma unroll
             for (int sub = 0; sub < KSUB; ++sub) {
 #pragma unroll
               for (int a = 0; a < KBOX / UMMA_K; ++a) {
-                const uint64_t ad = adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a;
-                const uint64_t bd = bdesc0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a;
-                if (F8) umma_f8(d_tmem, ad, bd, IDESC, (sub | a) ? 1u : accumulate);
-                else umma_bf16(d_tmem, ad, bd, IDESC, (sub | a) ? 1u : accumulate);
+                const uint32_t al = a_lo + ((sub * A_BOX_BYTES) >> 4) + 2u * a, bl = b_lo + ((sub * B_BOX_BYTES) >> 4) + 2u * a;
+                if (sub | a) umma_one_lo<F8, true>(d_tmem, al, bl, hi, IDESC, 1u);
+                else umma_one_lo<F8, false>(d_tmem, al, bl, hi, IDESC, accumulate);
               }
             }
             accumulate = 1;
