@@ -110,6 +110,32 @@ struct AttnParams {
 };
 
 // balanced "neighbours pair first" tree over 32 values in index order
+// three-input maximum (one instruction on this architecture); NaN operands are ignored as in fmaxf
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
+// rg_exp2 for an argument that is <= 0 or NaN: the overflow select can never fire and is left out
+// (same bits as rg_exp2 on that domain).
+__device__ __forceinline__ float exp2_nonpositive(float x) {
+  const float t = f_add(x, 12582912.0f);
+  const float n = f_add(t, -12582912.0f);
+  const float f = f_add(x, -n);
+  float q = 0x1.ffcbfcp-17f;
+  q = f_fma(q, f, 0x1.430912p-13f);
+  q = f_fma(q, f, 0x1.5d87fep-10f);
+  q = f_fma(q, f, 0x1.3b2ab6p-7f);
+  q = f_fma(q, f, 0x1.c6b08ep-5f);
+  q = f_fma(q, f, 0x1.ebfbe0p-3f);
+  q = f_fma(q, f, 0x1.62e430p-1f);
+  q = f_fma(q, f, 1.0f);
+  float e = __int_as_float(__float_as_int(q) + (__float_as_int(t) << 23));   // t's low mantissa bits hold n
+  e = x < -126.0f ? 0.0f : e;
+  return x != x ? x : e;
+}
+
 __device__ __forceinline__ float tree32(const float (&p)[32]) {
   float a[16];
 #pragma unroll
@@ -295,7 +321,18 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             }
           } else if (live == W) {                           // every key exists: no masking (all blocks but the last)
 #pragma unroll
-            for (int c = 0; c < 32; ++c) mb = fmaxf(mb, f_mul(__uint_as_float(raw[c]), p.scale));
+            if (p.scale > 0.0f) {
+              // rounding a product by a positive scale is monotone, so the largest scaled score is the
+              // scaled largest score: one multiply per 32 keys instead of one per key
+              float rm = __uint_as_float(raw[0]);
+#pragma unroll
+              for (int c = 1; c + 1 < 32; c += 2) rm = max3f(rm, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
+              rm = fmaxf(rm, __uint_as_float(raw[31]));
+              mb = fmaxf(mb, f_mul(rm, p.scale));
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) mb = fmaxf(mb, f_mul(__uint_as_float(raw[c]), p.scale));
+            }
           } else {
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
@@ -339,7 +376,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
               const float x = f_add(f_mul(__uint_as_float(raw[c]), p.scale), -m_new);
-              pr[c] = BASE2 ? rg_exp2(x) : rg_exp(x);
+              pr[c] = BASE2 ? exp2_nonpositive(x) : rg_exp(x);      // x <= 0 here (or NaN): m_new bounds every score
             }
           } else {
 #pragma unroll
