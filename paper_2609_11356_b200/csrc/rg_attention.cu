@@ -38,8 +38,9 @@ __device__ unsigned int g_attn_status_word = 0;
 namespace {
 
 constexpr int QROWS = 128;          // query rows per CTA = TMEM lanes
-constexpr int ATT_THREADS = 320;    // warp 0 TMA, warp 1 MMA, warps 2-9 softmax (two threads per query row)
-constexpr int SOFTMAX_THREADS = 256;
+constexpr int SPLIT = 4;            // threads per query row: each owns W / SPLIT keys and HD / SPLIT output columns
+constexpr int SOFTMAX_THREADS = QROWS * SPLIT;
+constexpr int ATT_THREADS = 64 + SOFTMAX_THREADS;    // warp 0 TMA, warp 1 MMA, then the softmax warps
 constexpr int KV_STAGES = 2;
 
 // ---- PTX wrappers (tensor core side)
@@ -80,6 +81,15 @@ __device__ __forceinline__ void att_tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void att_tmem_ld32(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr)
       : "memory");
 }
@@ -136,6 +146,14 @@ __device__ __forceinline__ float exp2_nonpositive(float x) {
   return x != x ? x : e;
 }
 
+__device__ __forceinline__ float tree32(const float (&p)[16]) {
+  float a[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) a[i] = f_add(p[2 * i], p[2 * i + 1]);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) a[i] = f_add(a[2 * i], a[2 * i + 1]);
+  return f_add(f_add(a[0], a[1]), f_add(a[2], a[3]));
+}
 __device__ __forceinline__ float tree32(const float (&p)[32]) {
   float a[16];
 #pragma unroll
@@ -175,8 +193,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   const uint32_t bar_s = bar_v_empty + 16u, bar_p = bar_s + 16u, bar_pv = bar_p + 8u;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* xm = reinterpret_cast<float*>(bars + 14);        // [2][128] partial maxima of the two halves of a row
-  float* xs = xm + 2 * QROWS;                             // [2][128] partial row sums
+  float* xm = reinterpret_cast<float*>(bars + 14);        // [SPLIT][128] partial maxima of the parts of a row
+  float* xs = xm + SPLIT * QROWS;                         // [SPLIT][128] partial row sums
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int head = blockIdx.y;
@@ -270,11 +288,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   } else {
     // ------------------------------------------------------------ softmax and output rows
     const int quarter = warp & 3;                           // TMEM lanes [32*quarter, 32*quarter + 32)
-    const int half = (warp - 2) >> 2;                       // which half of the keys and of the output columns
+    const int part = (warp - 2) >> 2;                       // which part of the keys and of the output columns
     const int r = quarter * 32 + lane;                      // row of the tile
     const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-    constexpr int KH = W / 2, OH = HD / 2;                  // keys and output columns per thread
-    const int kbase = half * KH, obase = half * OH;
+    constexpr int KH = W / SPLIT, OH = HD / SPLIT;          // keys and output columns per thread
+    constexpr int CK = KH < 32 ? KH : 32, CO = OH < 32 ? OH : 32;   // widths of one tensor-memory load
+    const int kbase = part * KH, obase = part * OH;
     float m = -INFINITY, l = 0.0f;
     float O[OH];
 #pragma unroll
@@ -283,18 +302,29 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     auto fold_pv = [&](float a) {
       att_fence_after();
 #pragma unroll
-      for (int ci = 0; ci < OH / 32; ++ci) {
-        uint32_t raw[32];
-        att_tmem_ld32(t_row + 256u + obase + ci * 32, raw);
+      for (int ci = 0; ci < OH / CO; ++ci) {
+        uint32_t raw[CO];
+        att_tmem_ld32(t_row + 256u + obase + ci * CO, raw);
         att_tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < 32; ++c) O[ci * 32 + c] = f_add(f_mul(a, O[ci * 32 + c]), __uint_as_float(raw[c]));
+        for (int c = 0; c < CO; ++c) O[ci * CO + c] = f_add(f_mul(a, O[ci * CO + c]), __uint_as_float(raw[c]));
       }
       att_fence_before();
     };
+    // the row's value from the SPLIT parts, paired as the balanced tree pairs them
+    auto row_max = [&](const float* x) {
+      float v = fmaxf(x[r], x[QROWS + r]);
+#pragma unroll
+      for (int q = 2; q < SPLIT; q += 2) v = fmaxf(v, fmaxf(x[q * QROWS + r], x[(q + 1) * QROWS + r]));
+      return v;
+    };
+    auto row_sum = [&](const float* x) {
+      if (SPLIT == 2) return f_add(x[r], x[QROWS + r]);
+      return f_add(f_add(x[r], x[QROWS + r]), f_add(x[2 * QROWS + r], x[3 * QROWS + r]));
+    };
     float alpha_prev = 0.0f;
     // A wait that gives up leaves this thread walking the loop without touching tensor memory, so
-    // that the 256-thread barriers below are still met by everyone.
+    // that the barriers of all softmax threads below are still met by everyone.
     bool alive = true;
     for (int j = 0; j < nblocks; ++j) {
       if (alive) alive = mbar_wait(bar_s + 8u * (j & 1), (j >> 1) & 1, abort_flag, &g_attn_status_word, 0x1500u);
@@ -307,44 +337,43 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       if (alive) {
         att_fence_after();
 #pragma unroll
-        for (int c0 = 0; c0 < KH; c0 += 32) {
-          uint32_t raw[32];
+        for (int c0 = 0; c0 < KH; c0 += CK) {
+          uint32_t raw[CK];
           att_tmem_ld32(t_s + kbase + c0, raw);
           att_tmem_ld_wait();
           if (diagonal) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
+            for (int c = 0; c < CK; ++c) {
               const int t = kbase + c0 + c;
               float sc = t < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
               sc = f_add(sc, j * W + t <= qi ? 0.0f : -1.0e6f);
               mb = fmaxf(mb, sc);
             }
           } else if (live == W) {                           // every key exists: no masking (all blocks but the last)
-#pragma unroll
             if (p.scale > 0.0f) {
               // rounding a product by a positive scale is monotone, so the largest scaled score is the
-              // scaled largest score: one multiply per 32 keys instead of one per key
+              // scaled largest score: one multiply per load instead of one per key
               float rm = __uint_as_float(raw[0]);
 #pragma unroll
-              for (int c = 1; c + 1 < 32; c += 2) rm = max3f(rm, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
-              rm = fmaxf(rm, __uint_as_float(raw[31]));
+              for (int c = 1; c + 1 < CK; c += 2) rm = max3f(rm, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
+              rm = fmaxf(rm, __uint_as_float(raw[CK - 1]));
               mb = fmaxf(mb, f_mul(rm, p.scale));
             } else {
 #pragma unroll
-              for (int c = 0; c < 32; ++c) mb = fmaxf(mb, f_mul(__uint_as_float(raw[c]), p.scale));
+              for (int c = 0; c < CK; ++c) mb = fmaxf(mb, f_mul(__uint_as_float(raw[c]), p.scale));
             }
           } else {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
+            for (int c = 0; c < CK; ++c) {
               const float sc = kbase + c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
               mb = fmaxf(mb, sc);
             }
           }
         }
       }
-      xm[half * QROWS + r] = mb;
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      const float m_new = fmaxf(m, fmaxf(xm[r], xm[QROWS + r]));
+      xm[part * QROWS + r] = mb;
+      asm volatile("bar.sync 1, %0;" ::"n"(SOFTMAX_THREADS) : "memory");
+      const float m_new = fmaxf(m, row_max(xm));
       const float alpha = BASE2 ? rg_exp2(f_add(m, -m_new)) : rg_exp(f_add(m, -m_new));
       // The previous block's P V product has had a whole first pass to finish: fold it into O now.
       // This also orders the rewrite of P below after the tensor core's last read of it, and comes
@@ -355,56 +384,56 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       }
       alpha_prev = alpha;
       // pass 2: probabilities, the subtree of the row sum over this thread's keys, narrowed copies
-      float part = 0.0f;
+      float psum = 0.0f;
       if (alive) {
-        float chunk_sum[KH / 32];
+        float chunk_sum[KH / CK];
 #pragma unroll
-        for (int ci = 0; ci < KH / 32; ++ci) {
-          const int c0 = kbase + ci * 32;
-          uint32_t raw[32];
+        for (int ci = 0; ci < KH / CK; ++ci) {
+          const int c0 = kbase + ci * CK;
+          uint32_t raw[CK];
           att_tmem_ld32(t_s + c0, raw);
           att_tmem_ld_wait();
-          float pr[32];
+          float pr[CK];
           if (diagonal) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
+            for (int c = 0; c < CK; ++c) {
               float sc = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
               sc = f_add(sc, j * W + c0 + c <= qi ? 0.0f : -1.0e6f);
               pr[c] = BASE2 ? rg_exp2(f_add(sc, -m_new)) : rg_exp(f_add(sc, -m_new));
             }
           } else if (live == W) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
+            for (int c = 0; c < CK; ++c) {
               const float x = f_add(f_mul(__uint_as_float(raw[c]), p.scale), -m_new);
               pr[c] = BASE2 ? exp2_nonpositive(x) : rg_exp(x);      // x <= 0 here (or NaN): m_new bounds every score
             }
           } else {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
+            for (int c = 0; c < CK; ++c) {
               const float sc = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
               pr[c] = BASE2 ? rg_exp2(f_add(sc, -m_new)) : rg_exp(f_add(sc, -m_new));
             }
           }
           chunk_sum[ci] = tree32(pr);
-          // row r of the [128 x 64] box that holds keys c0..c0+31: four 16-byte pieces of 8 keys each
+          // row r of the [128 x 64] box that holds keys c0..c0+CK-1: 16-byte pieces of 8 keys each
           uint8_t* box = sP_gen + (c0 >> 6) * P_BOX + (r >> 3) * 1024 + (r & 7) * 128;
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
+          for (int q = 0; q < CK / 8; ++q) {
             const int piece = ((c0 & 63) >> 3) + q;         // 16-byte piece of the 128-byte row
             const uint4 v = make_uint4(pack_bf16x2(pr[8 * q], pr[8 * q + 1]), pack_bf16x2(pr[8 * q + 2], pr[8 * q + 3]),
                                        pack_bf16x2(pr[8 * q + 4], pr[8 * q + 5]), pack_bf16x2(pr[8 * q + 6], pr[8 * q + 7]));
             *reinterpret_cast<uint4*>(box + ((piece ^ (r & 7)) << 4)) = v;
           }
         }
-        part = KH == 64 ? f_add(chunk_sum[0], chunk_sum[KH / 32 - 1]) : chunk_sum[0];
+        psum = KH / CK == 2 ? f_add(chunk_sum[0], chunk_sum[KH / CK - 1]) : chunk_sum[0];
       }
-      xs[half * QROWS + r] = part;
+      xs[part * QROWS + r] = psum;
       // the tensor core reads shared memory through the async proxy
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       att_fence_before();
-      asm volatile("bar.sync 1, 256;" ::: "memory");
+      asm volatile("bar.sync 1, %0;" ::"n"(SOFTMAX_THREADS) : "memory");
       if (lane == 0 && alive) mbar_arrive(bar_p);
-      l = f_add(f_mul(alpha, l), f_add(xs[r], xs[QROWS + r]));
+      l = f_add(f_mul(alpha, l), row_sum(xs));
       m = m_new;
     }
     if (alive) alive = mbar_wait(bar_pv, (nblocks - 1) & 1, abort_flag, &g_attn_status_word, 0x1700u);
@@ -413,20 +442,17 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     const int64_t row = (int64_t)q0 + r;
     if (alive && row < p.Nq) {
       const int64_t off = ((int64_t)head * p.Nq + row) * p.ldo + obase;
+      float v[OH];
 #pragma unroll
-      for (int ci = 0; ci < OH / 32; ++ci) {
-        float v[32];
+      for (int c = 0; c < OH; ++c) v[c] = __fdiv_rn(O[c], l);
+      if (p.o_dtype == RG_F32) {
+        float* dst = static_cast<float*>(p.O) + off;
 #pragma unroll
-        for (int c = 0; c < 32; ++c) v[c] = __fdiv_rn(O[ci * 32 + c], l);
-        if (p.o_dtype == RG_F32) {
-          float* dst = static_cast<float*>(p.O) + off + ci * 32;
+        for (int c = 0; c < OH; ++c) dst[c] = v[c];
+      } else {
+        uint16_t* dst = static_cast<uint16_t*>(p.O) + off;
 #pragma unroll
-          for (int c = 0; c < 32; ++c) dst[c] = v[c];
-        } else {
-          uint16_t* dst = static_cast<uint16_t*>(p.O) + off + ci * 32;
-#pragma unroll
-          for (int c = 0; c < 32; c += 2) *reinterpret_cast<uint32_t*>(dst + c) = pack_16x2(v[c], v[c + 1], p.o_dtype);
-        }
+        for (int c = 0; c < OH; c += 2) *reinterpret_cast<uint32_t*>(dst + c) = pack_16x2(v[c], v[c + 1], p.o_dtype);
       }
     }
   }
@@ -446,7 +472,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
 template <int W, int HD>
 size_t attn_smem_bytes() {
-  return 1024 + (HD / 64) * QROWS * 128 + KV_STAGES * ((HD / 64) * W * 128 + (W / 64) * HD * 128) + (W / 64) * QROWS * 128 + 14 * 8 + 4 * QROWS * 4;
+  return 1024 + (HD / 64) * QROWS * 128 + KV_STAGES * ((HD / 64) * W * 128 + (W / 64) * HD * 128) + (W / 64) * QROWS * 128 + 14 * 8 + 2 * SPLIT * QROWS * 4;
 }
 
 template <int W, int HD, bool BASE2>
