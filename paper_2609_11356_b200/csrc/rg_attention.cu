@@ -127,6 +127,30 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
   return r;
 }
 
+// three-input minimum that returns NaN when any operand is NaN
+__device__ __forceinline__ float min3f_nan(float a, float b, float c) {
+  float r;
+  asm("min.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
+// rg_exp2 for an argument in [-126, 0]: none of the range selects can fire and none is evaluated
+// (same bits as rg_exp2 on that domain).
+__device__ __forceinline__ float exp2_core(float x) {
+  const float t = f_add(x, 12582912.0f);
+  const float n = f_add(t, -12582912.0f);
+  const float f = f_add(x, -n);
+  float q = 0x1.ffcbfcp-17f;
+  q = f_fma(q, f, 0x1.430912p-13f);
+  q = f_fma(q, f, 0x1.5d87fep-10f);
+  q = f_fma(q, f, 0x1.3b2ab6p-7f);
+  q = f_fma(q, f, 0x1.c6b08ep-5f);
+  q = f_fma(q, f, 0x1.ebfbe0p-3f);
+  q = f_fma(q, f, 0x1.62e430p-1f);
+  q = f_fma(q, f, 1.0f);
+  return __int_as_float(__float_as_int(q) + (__float_as_int(t) << 23));      // t's low mantissa bits hold n
+}
+
 // rg_exp2 for an argument that is <= 0 or NaN: the overflow select can never fire and is left out
 // (same bits as rg_exp2 on that domain).
 __device__ __forceinline__ float exp2_nonpositive(float x) {
@@ -402,10 +426,26 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
               pr[c] = BASE2 ? rg_exp2(f_add(sc, -m_new)) : rg_exp(f_add(sc, -m_new));
             }
           } else if (live == W) {
+            // x <= 0 here (or NaN): m_new bounds every score
 #pragma unroll
-            for (int c = 0; c < CK; ++c) {
-              const float x = f_add(f_mul(__uint_as_float(raw[c]), p.scale), -m_new);
-              pr[c] = BASE2 ? exp2_nonpositive(x) : rg_exp(x);      // x <= 0 here (or NaN): m_new bounds every score
+            for (int c = 0; c < CK; ++c) pr[c] = f_add(f_mul(__uint_as_float(raw[c]), p.scale), -m_new);
+            if (BASE2) {
+              // the smallest argument of the chunk, NaN if any argument is NaN: when it is at least -126
+              // no element needs the underflow or the NaN select of the specified exponential
+              float xmin = pr[0];
+#pragma unroll
+              for (int c = 1; c + 1 < CK; c += 2) xmin = min3f_nan(xmin, pr[c], pr[c + 1]);
+              xmin = min3f_nan(xmin, pr[CK - 1], pr[CK - 1]);
+              if (xmin >= -126.0f) {
+#pragma unroll
+                for (int c = 0; c < CK; ++c) pr[c] = exp2_core(pr[c]);
+              } else {
+#pragma unroll
+                for (int c = 0; c < CK; ++c) pr[c] = exp2_nonpositive(pr[c]);
+              }
+            } else {
+#pragma unroll
+              for (int c = 0; c < CK; ++c) pr[c] = rg_exp(pr[c]);
             }
           } else {
 #pragma unroll
