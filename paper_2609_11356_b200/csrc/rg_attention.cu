@@ -217,8 +217,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   const uint32_t bar_s = bar_v_empty + 16u, bar_p = bar_s + 16u, bar_pv = bar_p + 8u;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* xm = reinterpret_cast<float*>(bars + 14);        // [SPLIT][128] partial maxima of the parts of a row
-  float* xs = xm + SPLIT * QROWS;                         // [SPLIT][128] partial row sums
+  float* xm = reinterpret_cast<float*>(bars + 14);        // [2][SPLIT][128] partial maxima of the parts of a row, by block parity
+  float* xs = xm + 2 * SPLIT * QROWS;                     // [2][SPLIT][128] partial row sums, by block parity
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int head = blockIdx.y;
@@ -395,10 +395,15 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
           }
         }
       }
-      xm[part * QROWS + r] = mb;
+      float* xm_j = xm + (j & 1) * SPLIT * QROWS;
+      xm_j[part * QROWS + r] = mb;
+      // The only barrier of a block.  Behind it every thread of the row has also finished the block
+      // before, so that block's partial row sums are complete; the exchange buffers alternate with
+      // the block parity, and a thread can be at most one barrier ahead of another.
       asm volatile("bar.sync 1, %0;" ::"n"(SOFTMAX_THREADS) : "memory");
-      const float m_new = fmaxf(m, row_max(xm));
+      const float m_new = fmaxf(m, row_max(xm_j));
       const float alpha = BASE2 ? rg_exp2(f_add(m, -m_new)) : rg_exp(f_add(m, -m_new));
+      if (j > 0) l = f_add(f_mul(alpha_prev, l), row_sum(xs + ((j - 1) & 1) * SPLIT * QROWS));
       // The previous block's P V product has had a whole first pass to finish: fold it into O now.
       // This also orders the rewrite of P below after the tensor core's last read of it, and comes
       // before this block's probabilities are released, so the barrier cannot run a phase ahead.
@@ -467,15 +472,17 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         }
         psum = KH / CK == 2 ? f_add(chunk_sum[0], chunk_sum[KH / CK - 1]) : chunk_sum[0];
       }
-      xs[part * QROWS + r] = psum;
-      // the tensor core reads shared memory through the async proxy
+      xs[(j & 1) * SPLIT * QROWS + part * QROWS + r] = psum;
+      // the tensor core reads shared memory through the async proxy; one arrival per warp once all
+      // of its lanes have written and fenced their probabilities
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       att_fence_before();
-      asm volatile("bar.sync 1, %0;" ::"n"(SOFTMAX_THREADS) : "memory");
+      __syncwarp();
       if (lane == 0 && alive) mbar_arrive(bar_p);
-      l = f_add(f_mul(alpha, l), row_sum(xs));
       m = m_new;
     }
+    asm volatile("bar.sync 1, %0;" ::"n"(SOFTMAX_THREADS) : "memory");
+    l = f_add(f_mul(alpha_prev, l), row_sum(xs + ((nblocks - 1) & 1) * SPLIT * QROWS));
     if (alive) alive = mbar_wait(bar_pv, (nblocks - 1) & 1, abort_flag, &g_attn_status_word, 0x1700u);
     if (alive) fold_pv(alpha_prev);
     // one division at the end, one rounding to the output type
@@ -512,7 +519,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
 template <int W, int HD>
 size_t attn_smem_bytes() {
-  return 1024 + (HD / 64) * QROWS * 128 + KV_STAGES * ((HD / 64) * W * 128 + (W / 64) * HD * 128) + (W / 64) * QROWS * 128 + 14 * 8 + 2 * SPLIT * QROWS * 4;
+  return 1024 + (HD / 64) * QROWS * 128 + KV_STAGES * ((HD / 64) * W * 128 + (W / 64) * HD * 128) + (W / 64) * QROWS * 128 + 14 * 8 + 4 * SPLIT * QROWS * 4;
 }
 
 template <int W, int HD, bool BASE2>
