@@ -151,6 +151,26 @@ __device__ __forceinline__ float exp2_core(float x) {
   return __int_as_float(__float_as_int(q) + (__float_as_int(t) << 23));      // t's low mantissa bits hold n
 }
 
+// rg_exp for an argument in [-87.33655, 0]: no range select can fire, n lies in [-126, 0], so 2^n is
+// a normal number and the two-factor scaling of rg_exp equals one multiplication by it (scaling by
+// a power of two is exact until the single final rounding).  Same bits as rg_exp on that domain.
+__device__ __forceinline__ float exp_core(float x) {
+  const float y = f_mul(x, 0x1.715476p+0f);
+  const float t = f_add(y, 12582912.0f);
+  const float n = f_add(t, -12582912.0f);
+  float r = f_fma(n, -0x1.62e400p-1f, x);
+  r = f_fma(n, -0x1.7f7d1cp-20f, r);
+  float q = 0x1.a01a02p-13f;
+  q = f_fma(q, r, 0x1.6c16c2p-10f);
+  q = f_fma(q, r, 0x1.111112p-7f);
+  q = f_fma(q, r, 0x1.555556p-5f);
+  q = f_fma(q, r, 0x1.555556p-3f);
+  q = f_fma(q, r, 0.5f);
+  q = f_fma(q, r, 1.0f);
+  q = f_fma(q, r, 1.0f);
+  return f_mul(q, __int_as_float((__float_as_int(t) << 23) + 0x3f800000));   // t's low mantissa bits hold n
+}
+
 // rg_exp2 for an argument that is <= 0 or NaN: the overflow select can never fire and is left out
 // (same bits as rg_exp2 on that domain).
 __device__ __forceinline__ float exp2_nonpositive(float x) {
@@ -434,23 +454,18 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             // x <= 0 here (or NaN): m_new bounds every score
 #pragma unroll
             for (int c = 0; c < CK; ++c) pr[c] = f_add(f_mul(__uint_as_float(raw[c]), p.scale), -m_new);
-            if (BASE2) {
-              // the smallest argument of the chunk, NaN if any argument is NaN: when it is at least -126
-              // no element needs the underflow or the NaN select of the specified exponential
-              float xmin = pr[0];
+            // the smallest argument of the chunk, NaN if any argument is NaN: when it is above the
+            // underflow threshold no element needs a range or NaN select of the specified exponential
+            float xmin = pr[0];
 #pragma unroll
-              for (int c = 1; c + 1 < CK; c += 2) xmin = min3f_nan(xmin, pr[c], pr[c + 1]);
-              xmin = min3f_nan(xmin, pr[CK - 1], pr[CK - 1]);
-              if (xmin >= -126.0f) {
+            for (int c = 1; c + 1 < CK; c += 2) xmin = min3f_nan(xmin, pr[c], pr[c + 1]);
+            xmin = min3f_nan(xmin, pr[CK - 1], pr[CK - 1]);
+            if (xmin >= (BASE2 ? -126.0f : -87.33655f)) {
 #pragma unroll
-                for (int c = 0; c < CK; ++c) pr[c] = exp2_core(pr[c]);
-              } else {
-#pragma unroll
-                for (int c = 0; c < CK; ++c) pr[c] = exp2_nonpositive(pr[c]);
-              }
+              for (int c = 0; c < CK; ++c) pr[c] = BASE2 ? exp2_core(pr[c]) : exp_core(pr[c]);
             } else {
 #pragma unroll
-              for (int c = 0; c < CK; ++c) pr[c] = rg_exp(pr[c]);
+              for (int c = 0; c < CK; ++c) pr[c] = BASE2 ? exp2_nonpositive(pr[c]) : rg_exp(pr[c]);
             }
           } else {
 #pragma unroll

@@ -53,15 +53,16 @@ def test_base_two_variant_bit_exact(Nq, Nk, d, w):
     assert_bits_equal(got, want, f"attention base two {Nq}x{Nk} d={d} w={w}")
 
 
+@pytest.mark.parametrize("base", [2, 0])
 @pytest.mark.parametrize("Nq,Nk,d,w,scale", [(256, 512, 128, 128, 3.0), (130, 256, 64, 64, 6.0), (128, 384, 128, 128, 0.5)])
-def test_base_two_wide_scores_underflow(Nq, Nk, d, w, scale):
-    """Scores spread over more than 126 binades below the row maximum: full key blocks in which some
+def test_wide_scores_underflow(Nq, Nk, d, w, scale, base):
+    """Scores spread far past the underflow threshold below the row maximum: full key blocks in which some
     probabilities underflow to +0 and others do not (the chunk-level range test of the kernel must
     fall back to the per-element selects of the specified exponential)."""
     Q, K, V = _draw(Nq, Nk, d, 5 + Nq + Nk, spread=2)
-    got = gpu_attention(Q, K, V, block_n=w, scale=scale, out_dtype=rgo.F32, exp_base=2)
-    want = rgo.attention(Q, K, V, block_n=w, scale=scale, atom_model=HW, out_dtype=rgo.F32, exp_base=2)
-    assert_bits_equal(got, want, f"wide scores {Nq}x{Nk} d={d} w={w} scale={scale}")
+    got = gpu_attention(Q, K, V, block_n=w, scale=scale, out_dtype=rgo.F32, exp_base=base)
+    want = rgo.attention(Q, K, V, block_n=w, scale=scale, atom_model=HW, out_dtype=rgo.F32, exp_base=base)
+    assert_bits_equal(got, want, f"wide scores {Nq}x{Nk} d={d} w={w} scale={scale} base={base}")
 
 
 @pytest.mark.parametrize("N,d,w,base", [(128, 128, 128, 0), (300, 64, 64, 2), (1000, 128, 64, 0), (777, 128, 128, 2)])
