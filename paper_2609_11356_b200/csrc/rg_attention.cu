@@ -41,7 +41,7 @@ constexpr int QROWS = 128;          // query rows per CTA = TMEM lanes
 constexpr int SPLIT = 4;            // threads per query row: each owns W / SPLIT keys and HD / SPLIT output columns
 constexpr int SOFTMAX_THREADS = QROWS * SPLIT;
 constexpr int ATT_THREADS = 64 + SOFTMAX_THREADS;    // warp 0 TMA, warp 1 MMA, then the softmax warps
-constexpr int KV_STAGES = 2;
+constexpr int V_STAGES = 2;
 
 // ---- PTX wrappers (tensor core side)
 __device__ __forceinline__ void att_tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar) {
@@ -220,21 +220,23 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   constexpr uint32_t P_BOX = QROWS * 128;                 // [128 rows x 64 keys]
   constexpr int DB = HD / 64, WB = W / 64;                // boxes along d and along the keys
   constexpr uint32_t Q_BYTES = DB * Q_BOX, K_BYTES = DB * K_BOX, V_BYTES = WB * V_BOX, P_BYTES = WB * P_BOX;
-  constexpr uint32_t KV_BYTES = K_BYTES + V_BYTES;
-  constexpr uint32_t TMEM_COLS = 512;                     // S of block j at columns [128*(j&1), ... + W), PV at [256, 256 + HD)
+  constexpr uint32_t TMEM_COLS = 512;                     // S of block j at columns [128*(j&1), ... + W), P V of block j at [256 + 128*(j&1), ... + HD)
   constexpr uint32_t IDESC_S = att_idesc(W), IDESC_PV = att_idesc(HD);
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t sQ = smem_base, sKV = sQ + Q_BYTES, sP = sKV + KV_STAGES * KV_BYTES;
-  uint8_t* sP_gen = smem_gen + Q_BYTES + KV_STAGES * KV_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + Q_BYTES + KV_STAGES * KV_BYTES + P_BYTES);
-  // barriers: q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full, pv_full
+  // one K box set (the next block's keys are fetched as soon as the scores that read this one are
+  // done, a whole block before they are needed), two V stages, two P buffers
+  const uint32_t sQ = smem_base, sK = sQ + Q_BYTES, sV0 = sK + K_BYTES, sP = sV0 + V_STAGES * V_BYTES;
+  uint8_t* sP_gen = smem_gen + Q_BYTES + K_BYTES + V_STAGES * V_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + Q_BYTES + K_BYTES + V_STAGES * V_BYTES + 2 * P_BYTES);
+  // barriers: q_full, k_full, k_empty, pv_full[2], v_full[2], v_empty[2], s_full[2], p_full
   const uint32_t bar_q = smem_u32(bars);
-  const uint32_t bar_k_full = bar_q + 8u, bar_k_empty = bar_k_full + 16u;
-  const uint32_t bar_v_full = bar_k_empty + 16u, bar_v_empty = bar_v_full + 16u;
-  const uint32_t bar_s = bar_v_empty + 16u, bar_p = bar_s + 16u, bar_pv = bar_p + 8u;
+  const uint32_t bar_k_full = bar_q + 8u, bar_k_empty = bar_k_full + 8u;
+  const uint32_t bar_pv = bar_k_empty + 8u;
+  const uint32_t bar_v_full = bar_pv + 16u, bar_v_empty = bar_v_full + 16u;
+  const uint32_t bar_s = bar_v_empty + 16u, bar_p = bar_s + 16u;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* xm = reinterpret_cast<float*>(bars + 14);        // [2][SPLIT][128] partial maxima of the parts of a row, by block parity
@@ -250,12 +252,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
-    for (int s = 0; s < KV_STAGES; ++s) {
-      mbar_init(bar_k_full + 8u * s, 1); mbar_init(bar_k_empty + 8u * s, 1);
+    mbar_init(bar_k_full, 1); mbar_init(bar_k_empty, 1);
+    for (int s = 0; s < 2; ++s) {
       mbar_init(bar_v_full + 8u * s, 1); mbar_init(bar_v_empty + 8u * s, 1);
-      mbar_init(bar_s + 8u * s, 1);
+      mbar_init(bar_s + 8u * s, 1); mbar_init(bar_pv + 8u * s, 1);
     }
-    mbar_init(bar_p, SOFTMAX_THREADS / 32); mbar_init(bar_pv, 1);
+    mbar_init(bar_p, SOFTMAX_THREADS / 32);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -276,15 +278,14 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       for (int b = 0; b < DB; ++b) att_tma_load_2d(sQ + b * Q_BOX, &tmap_q, b * 64, head * p.Nq + q0, bar_q);
       for (int j = 0; j < nblocks; ++j) {
         const int stage = j & 1; const uint32_t phase = (j >> 1) & 1;
-        const uint32_t dst = sKV + stage * KV_BYTES;
-        if (!mbar_wait(bar_k_empty + 8u * stage, phase ^ 1u, abort_flag, &g_attn_status_word, 0x1100u | stage)) break;
-        mbar_expect_tx(bar_k_full + 8u * stage, K_BYTES);
+        if (!mbar_wait(bar_k_empty, (j & 1) ^ 1u, abort_flag, &g_attn_status_word, 0x1100u)) break;
+        mbar_expect_tx(bar_k_full, K_BYTES);
 #pragma unroll
-        for (int b = 0; b < DB; ++b) att_tma_load_2d(dst + b * K_BOX, &tmap_k, b * 64, head * p.Nk + j * W, bar_k_full + 8u * stage);
+        for (int b = 0; b < DB; ++b) att_tma_load_2d(sK + b * K_BOX, &tmap_k, b * 64, head * p.Nk + j * W, bar_k_full);
         if (!mbar_wait(bar_v_empty + 8u * stage, phase ^ 1u, abort_flag, &g_attn_status_word, 0x1180u | stage)) break;
         mbar_expect_tx(bar_v_full + 8u * stage, V_BYTES);
 #pragma unroll
-        for (int b = 0; b < WB; ++b) att_tma_load_2d(dst + K_BYTES + b * V_BOX, &tmap_vt, j * W + b * 64, head * HD, bar_v_full + 8u * stage);
+        for (int b = 0; b < WB; ++b) att_tma_load_2d(sV0 + stage * V_BYTES + b * V_BOX, &tmap_vt, j * W + b * 64, head * HD, bar_v_full + 8u * stage);
       }
     }
   } else if (warp == 1) {
@@ -293,10 +294,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       bool alive = mbar_wait(bar_q, 0, abort_flag, &g_attn_status_word, 0x1200u);
       // S_j = Q K_j^T into score accumulator j&1: ascending k over the head dimension, from zero
       auto issue_scores = [&](int j) -> bool {
-        const int stage = j & 1; const uint32_t phase = (j >> 1) & 1;
-        if (!mbar_wait(bar_k_full + 8u * stage, phase, abort_flag, &g_attn_status_word, 0x1300u | stage)) return false;
+        const int stage = j & 1;
+        if (!mbar_wait(bar_k_full, j & 1, abort_flag, &g_attn_status_word, 0x1300u)) return false;
         att_fence_after();
-        const uint32_t sK = sKV + stage * KV_BYTES;
 #pragma unroll
         for (int b = 0; b < DB; ++b) {
           const uint64_t adesc = att_kmajor_desc(sQ + b * Q_BOX), bdesc = att_kmajor_desc(sK + b * K_BOX);
@@ -304,7 +304,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
           for (int a = 0; a < 4; ++a) att_mma_bf16(tmem_base + 128u * stage, adesc + 2u * a, bdesc + 2u * a, IDESC_S, (b | a) ? 1u : 0u);
         }
         att_commit(bar_s + 8u * stage);
-        att_commit(bar_k_empty + 8u * stage);
+        att_commit(bar_k_empty);
         return true;
       };
       if (alive) alive = issue_scores(0);
@@ -313,19 +313,21 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         // softmax threads had finished reading before they released P_{j-1} (waited for below, one
         // turn ago).
         if (j + 1 < nblocks && !issue_scores(j + 1)) break;
-        // PV = P Vt^T: ascending key over the block, from zero, once the probabilities are in shared memory
+        // PV = P Vt^T: ascending key over the block, from zero, once the probabilities are in shared memory.
+        // Probabilities and product alternate between two buffers: the softmax threads folded the
+        // product of block j-2 and saw it complete before they wrote these probabilities.
         const int stage = j & 1; const uint32_t phase = (j >> 1) & 1;
         if (!mbar_wait(bar_p, j & 1, abort_flag, &g_attn_status_word, 0x1400u)) break;
         if (!mbar_wait(bar_v_full + 8u * stage, phase, abort_flag, &g_attn_status_word, 0x1480u | stage)) break;
         att_fence_after();
-        const uint32_t sV = sKV + stage * KV_BYTES + K_BYTES;
+        const uint32_t sV = sV0 + stage * V_BYTES, sPj = sP + stage * P_BYTES;
 #pragma unroll
         for (int b = 0; b < WB; ++b) {
-          const uint64_t adesc = att_kmajor_desc(sP + b * P_BOX), bdesc = att_kmajor_desc(sV + b * V_BOX);
+          const uint64_t adesc = att_kmajor_desc(sPj + b * P_BOX), bdesc = att_kmajor_desc(sV + b * V_BOX);
 #pragma unroll
-          for (int a = 0; a < 4; ++a) att_mma_bf16(tmem_base + 256u, adesc + 2u * a, bdesc + 2u * a, IDESC_PV, (b | a) ? 1u : 0u);
+          for (int a = 0; a < 4; ++a) att_mma_bf16(tmem_base + 256u + 128u * stage, adesc + 2u * a, bdesc + 2u * a, IDESC_PV, (b | a) ? 1u : 0u);
         }
-        att_commit(bar_pv);
+        att_commit(bar_pv + 8u * stage);
         att_commit(bar_v_empty + 8u * stage);               // the stage may be refilled once these steps have read it
       }
     }
@@ -343,12 +345,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 #pragma unroll
     for (int c = 0; c < OH; ++c) O[c] = 0.0f;
     // O = a * O + PV on this thread's output columns
-    auto fold_pv = [&](float a) {
+    auto fold_pv = [&](float a, int buf) {
       att_fence_after();
 #pragma unroll
       for (int ci = 0; ci < OH / CO; ++ci) {
         uint32_t raw[CO];
-        att_tmem_ld32(t_row + 256u + obase + ci * CO, raw);
+        att_tmem_ld32(t_row + 256u + 128u * buf + obase + ci * CO, raw);
         att_tmem_ld_wait();
 #pragma unroll
         for (int c = 0; c < CO; ++c) O[ci * CO + c] = f_add(f_mul(a, O[ci * CO + c]), __uint_as_float(raw[c]));
@@ -424,14 +426,6 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       const float m_new = fmaxf(m, row_max(xm_j));
       const float alpha = BASE2 ? rg_exp2(f_add(m, -m_new)) : rg_exp(f_add(m, -m_new));
       if (j > 0) l = f_add(f_mul(alpha_prev, l), row_sum(xs + ((j - 1) & 1) * SPLIT * QROWS));
-      // The previous block's P V product has had a whole first pass to finish: fold it into O now.
-      // This also orders the rewrite of P below after the tensor core's last read of it, and comes
-      // before this block's probabilities are released, so the barrier cannot run a phase ahead.
-      if (j > 0) {
-        if (alive) alive = mbar_wait(bar_pv, (j - 1) & 1, abort_flag, &g_attn_status_word, 0x1600u);
-        if (alive) fold_pv(alpha_prev);
-      }
-      alpha_prev = alpha;
       // pass 2: probabilities, the subtree of the row sum over this thread's keys, narrowed copies
       float psum = 0.0f;
       if (alive) {
@@ -476,7 +470,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
           }
           chunk_sum[ci] = tree32(pr);
           // row r of the [128 x 64] box that holds keys c0..c0+CK-1: 16-byte pieces of 8 keys each
-          uint8_t* box = sP_gen + (c0 >> 6) * P_BOX + (r >> 3) * 1024 + (r & 7) * 128;
+          uint8_t* box = sP_gen + (j & 1) * P_BYTES + (c0 >> 6) * P_BOX + (r >> 3) * 1024 + (r & 7) * 128;
 #pragma unroll
           for (int q = 0; q < CK / 8; ++q) {
             const int piece = ((c0 & 63) >> 3) + q;         // 16-byte piece of the 128-byte row
@@ -495,11 +489,19 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       __syncwarp();
       if (lane == 0 && alive) mbar_arrive(bar_p);
       m = m_new;
+      // The previous block's P V product has had this block's two passes to finish: fold it into O
+      // (O_{j-1} = alpha_{j-1} O_{j-2} + P_{j-1} V_{j-1}).  Seeing it complete also licenses the
+      // rewrite of its probability buffer two blocks after it was filled.
+      if (j > 0) {
+        if (alive) alive = mbar_wait(bar_pv + 8u * ((j - 1) & 1), ((j - 1) >> 1) & 1, abort_flag, &g_attn_status_word, 0x1600u);
+        if (alive) fold_pv(alpha_prev, (j - 1) & 1);
+      }
+      alpha_prev = alpha;
     }
     asm volatile("bar.sync 1, %0;" ::"n"(SOFTMAX_THREADS) : "memory");
     l = f_add(f_mul(alpha_prev, l), row_sum(xs + ((nblocks - 1) & 1) * SPLIT * QROWS));
-    if (alive) alive = mbar_wait(bar_pv, (nblocks - 1) & 1, abort_flag, &g_attn_status_word, 0x1700u);
-    if (alive) fold_pv(alpha_prev);
+    if (alive) alive = mbar_wait(bar_pv + 8u * ((nblocks - 1) & 1), ((nblocks - 1) >> 1) & 1, abort_flag, &g_attn_status_word, 0x1700u);
+    if (alive) fold_pv(alpha_prev, (nblocks - 1) & 1);
     // one division at the end, one rounding to the output type
     const int64_t row = (int64_t)q0 + r;
     if (alive && row < p.Nq) {
@@ -534,7 +536,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
 template <int W, int HD>
 size_t attn_smem_bytes() {
-  return 1024 + (HD / 64) * QROWS * 128 + KV_STAGES * ((HD / 64) * W * 128 + (W / 64) * HD * 128) + (W / 64) * QROWS * 128 + 14 * 8 + 4 * SPLIT * QROWS * 4;
+  return 1024 + (HD / 64) * QROWS * 128 + (HD / 64) * W * 128 + V_STAGES * (W / 64) * HD * 128 + 2 * (W / 64) * QROWS * 128 + 14 * 8 + 4 * SPLIT * QROWS * 4;
 }
 
 template <int W, int HD, bool BASE2>
