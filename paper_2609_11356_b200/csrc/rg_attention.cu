@@ -437,19 +437,28 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
           att_tmem_ld32(t_s + c0, raw);
           att_tmem_ld_wait();
           float pr[CK];
+          // the exponent x = s - m_new of every key: <= 0 (m_new bounds every score of the block), or NaN
           if (diagonal) {
 #pragma unroll
             for (int c = 0; c < CK; ++c) {
               float sc = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
               sc = f_add(sc, j * W + c0 + c <= qi ? 0.0f : -1.0e6f);
-              pr[c] = BASE2 ? rg_exp2(f_add(sc, -m_new)) : rg_exp(f_add(sc, -m_new));
+              pr[c] = f_add(sc, -m_new);
             }
           } else if (live == W) {
-            // x <= 0 here (or NaN): m_new bounds every score
 #pragma unroll
             for (int c = 0; c < CK; ++c) pr[c] = f_add(f_mul(__uint_as_float(raw[c]), p.scale), -m_new);
-            // the smallest argument of the chunk, NaN if any argument is NaN: when it is above the
-            // underflow threshold no element needs a range or NaN select of the specified exponential
+          } else {
+#pragma unroll
+            for (int c = 0; c < CK; ++c) {
+              const float sc = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
+              pr[c] = f_add(sc, -m_new);
+            }
+          }
+          {
+            // the smallest exponent of the chunk, NaN if any is NaN: when it is above the underflow
+            // threshold no element needs a range or NaN select of the specified exponential
+            // (masked keys have x = -inf and take the selects)
             float xmin = pr[0];
 #pragma unroll
             for (int c = 1; c + 1 < CK; c += 2) xmin = min3f_nan(xmin, pr[c], pr[c + 1]);
@@ -460,12 +469,6 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             } else {
 #pragma unroll
               for (int c = 0; c < CK; ++c) pr[c] = BASE2 ? exp2_nonpositive(pr[c]) : rg_exp(pr[c]);
-            }
-          } else {
-#pragma unroll
-            for (int c = 0; c < CK; ++c) {
-              const float sc = c0 + c < live ? f_mul(__uint_as_float(raw[c]), p.scale) : -INFINITY;
-              pr[c] = BASE2 ? rg_exp2(f_add(sc, -m_new)) : rg_exp(f_add(sc, -m_new));
             }
           }
           chunk_sum[ci] = tree32(pr);
