@@ -47,6 +47,33 @@ __device__ __forceinline__ float rg_exp(float x) {
   return x != x ? x : e;
 }
 
+// rg_exp for |x| <= 87 (and not NaN): no range select can fire, n lies in [-126, 126], so 2^n is a
+// normal number, the result is normal, and the two-factor scaling of rg_exp (two exact
+// multiplications there) equals one exact multiplication by 2^n.  Same bits as rg_exp on that domain.
+__device__ __forceinline__ float rg_exp_inrange(float x) {
+  const float y = f_mul(x, 0x1.715476p+0f);
+  const float t = f_add(y, 12582912.0f);
+  const float n = f_add(t, -12582912.0f);
+  float r = f_fma(n, -0x1.62e400p-1f, x);
+  r = f_fma(n, -0x1.7f7d1cp-20f, r);
+  float p = 0x1.a01a02p-13f;
+  p = f_fma(p, r, 0x1.6c16c2p-10f);
+  p = f_fma(p, r, 0x1.111112p-7f);
+  p = f_fma(p, r, 0x1.555556p-5f);
+  p = f_fma(p, r, 0x1.555556p-3f);
+  p = f_fma(p, r, 0.5f);
+  p = f_fma(p, r, 1.0f);
+  p = f_fma(p, r, 1.0f);
+  return f_mul(p, __int_as_float((__float_as_int(t) << 23) + 0x3f800000));   // t's low mantissa bits hold n
+}
+
+// largest magnitude of three values; NaN if any of them is NaN (one instruction on this architecture)
+__device__ __forceinline__ float absmax3_nan(float a, float b, float c) {
+  float r;
+  asm("max.NaN.abs.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
 // Base-two exponential fixed the same way (attention folds log2 e into the score scale, App. F):
 // n = rint(x), f = x - n (exact), degree-7 Taylor polynomial of 2^f in Horner form with fused
 // multiply-adds, and an exact scaling by 2^n done on the exponent field (the polynomial lies in

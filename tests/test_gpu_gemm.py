@@ -208,6 +208,23 @@ def test_fused_epilogue_small_every_element():
     assert_bits_equal(got, rgo.gemm(A, B, atom_model=HW, bias=b32, act=1, residual=r32, out_dtype=rgo.F32), "fp32 bias/residual")
 
 
+def test_silu_wide_range_every_element():
+    """Pre-activations from far below the exponential's underflow to far above its overflow, mixed
+    within rows: segments whose values all lie within +-87 take the select-free exponential, the
+    others the full one, and both must match the specified exponential bit for bit."""
+    for scale, seed in ((1.0, 40), (2.0, 41), (40.0, 42)):
+        A = synth.normal_bf16((150, 256), scale, seed); B = synth.normal_bf16((330, 256), 1.0, seed + 10)
+        bias = synth.uniform_bf16((330,), -0.1, 0.1, seed + 20)
+        for kw in (dict(act=1), dict(bias=bias, act=1), dict(act=1, cta_group=2), dict(act=1, cuts=(128,))):
+            got = gpu_gemm(A, B, out_dtype=rgo.F32, **kw)
+            okw = {k: v for k, v in kw.items() if k != "cta_group"}
+            want = rgo.gemm(A, B, atom_model=HW, out_dtype=rgo.F32, **okw)
+            assert_bits_equal(got, want, f"silu scale={scale} {list(kw)}")
+        if scale == 2.0:                                    # both kinds of 32-column segment occur
+            v = np.abs(gpu_gemm(A, B, out_dtype=rgo.F32))[:, :320].reshape(150, 10, 32).max(axis=2)
+            assert (v > 87).any() and (v <= 87).any()
+
+
 def test_fused_epilogue_prefill_full_size_sampled():
     M, N, K = 8192, 14336, 4096
     X = synth.device_normal((M, K), 1.0, 6, torch.bfloat16, DEV)
