@@ -126,17 +126,21 @@ template <typename T, int OP, bool VEC>
 __device__ __forceinline__ float load_fold(const T* __restrict__ xr, int64_t col, int64_t C, float shift, int fma) {
   constexpr int V = VecTraits<T>::V;
   float x[V];
+  int nvalid = V;
   if (VEC && col + V <= C) {
     unpack<T>(__ldg(reinterpret_cast<const uint4*>(xr + col)), x);
-    return fold_block<OP, V, true>(x, V, shift, fma);
-  }
-  int nvalid = 0;
+  } else {
+    nvalid = 0;
 #pragma unroll
-  for (int t = 0; t < V; ++t) {
-    const bool ok = (col + t) < C;
-    x[t] = ok ? elem_to_f32(xr[col + t]) : 0.0f;
-    nvalid += ok ? 1 : 0;
+    for (int t = 0; t < V; ++t) {
+      const bool ok = (col + t) < C;
+      x[t] = ok ? elem_to_f32(xr[col + t]) : 0.0f;
+      nvalid += ok ? 1 : 0;
+    }
   }
+  // The lanes of a warp may have taken different sides above (a ragged row end).  The fold votes
+  // across the warp, so every lane must reach it through this one call, converged.
+  __syncwarp();
   return fold_block<OP, V, false>(x, nvalid, shift, fma);
 }
 
