@@ -1065,7 +1065,7 @@ int max_stages_for(int bn, int bk, int cta_group, int64_t M) {
   const int ksub = bk / KBOX;
   int s = 1;
   if (cta_group == 2) { while (s < 8 && smem_bytes_for_pair(bn, ksub, s + 1) <= SMEM_LIMIT) ++s; }
-  else { while (s < 8 && smem_bytes_for(bn, ksub, s + 1, a_box_rows_for(M)) <= SMEM_LIMIT) ++s; }
+  else { while (s < 32 && smem_bytes_for(bn, ksub, s + 1, a_box_rows_for(M)) <= SMEM_LIMIT) ++s; }
   return s;
 }
 
