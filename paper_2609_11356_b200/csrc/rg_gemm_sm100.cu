@@ -189,6 +189,18 @@ __device__ __forceinline__ void umma_pair_lo(uint32_t d_tmem, uint32_t a_lo, uin
   }
 }
 
+// One lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+// A wait that the whole (converged) warp makes and leaves with one common answer.
+__device__ __forceinline__ bool warp_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status, uint32_t code) {
+  const bool ok = mbar_wait(bar, parity, abort_flag, status, code);
+  return __all_sync(0xffffffffu, ok);
+}
+
 // One-CTA form of the same: (low word, high word) descriptors, compile-time accumulate.
 template <bool F8, bool ACC>
 __device__ __forceinline__ void umma_one_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
@@ -484,7 +496,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp walks the loop with identical values and one elected lane issues: with every lane
+    // converged the descriptor arithmetic stays in the uniform datapath, where the tensor-core
+    // instruction takes its operands from (a single diverged thread pays a register-to-uniform move
+    // for each of them, which dominates when the tile is narrow and a step is short).
+    {
+      const bool leader = elect_one();
       int stage = 0; uint32_t phase = 0;
       bool alive = true;
       int gc = 0;                                         // accumulators handed to the epilogue so far
@@ -501,15 +518,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         uint32_t d_tmem = 0, accumulate = 0;
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
           if (k0 >= group_end) {
-            if (k0 > k_begin) { umma_commit(bar_tfull + 8u * buf); ++gc; }   // the previous group is complete
+            if (k0 > k_begin) { if (leader) umma_commit(bar_tfull + 8u * buf); ++gc; }   // the previous group is complete
             buf = gc & 1;
-            if (!mbar_wait(bar_tempty + 8u * buf, ((gc >> 1) & 1) ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
+            if (!warp_mbar_wait(bar_tempty + 8u * buf, ((gc >> 1) & 1) ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
             tcgen05_fence_after();
             d_tmem = tmem_base + buf * ACC_STRIDE;
             accumulate = 0;                              // every part and every group starts from zero
             group_end = k0 + span;
           }
-          if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0x300u | stage)) { alive = false; break; }
+          if (!warp_mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0x300u | stage)) { alive = false; break; }
           tcgen05_fence_after();
           // descriptors differ from the stage-0 ones only in the 16-byte-unit start address (low word).
           // The operand kind is a template parameter: a run-time test in front of every step slowed
@@ -525,8 +542,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 #pragma unroll
               for (int a = 0; a < KBOX / UMMA_K; ++a) {
                 const uint32_t al = a_lo + ((sub * A_BOX_BYTES) >> 4) + 2u * a, bl = b_lo + ((sub * B_BOX_BYTES) >> 4) + 2u * a;
-                if (sub | a) umma_one_lo<F8, true>(d_tmem, al, bl, hi, IDESC, 1u);
-                else umma_one_lo<F8, false>(d_tmem, al, bl, hi, IDESC, accumulate);
+                if (leader) {
+                  if (sub | a) umma_one_lo<F8, true>(d_tmem, al, bl, hi, IDESC, 1u);
+                  else umma_one_lo<F8, false>(d_tmem, al, bl, hi, IDESC, accumulate);
+                }
               }
             }
             accumulate = 1;
@@ -539,17 +558,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 if (k0 + sub * KBOX + a * UMMA_K < k_end) {
                   const uint64_t ad = adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a;
                   const uint64_t bd = bdesc0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a;
-                  if (F8) umma_f8(d_tmem, ad, bd, IDESC, accumulate);
-                  else umma_bf16(d_tmem, ad, bd, IDESC, accumulate);
+                  if (leader) {
+                    if (F8) umma_f8(d_tmem, ad, bd, IDESC, accumulate);
+                    else umma_bf16(d_tmem, ad, bd, IDESC, accumulate);
+                  }
                   accumulate = 1;
                 }
               }
             }
           }
-          umma_commit(bar_empty + 8u * stage);           // stage reusable once these steps have read it
+          if (leader) umma_commit(bar_empty + 8u * stage);   // stage reusable once these steps have read it
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
-        if (alive) { umma_commit(bar_tfull + 8u * buf); ++gc; }   // last (or only) accumulator complete
+        if (alive) { if (leader) umma_commit(bar_tfull + 8u * buf); ++gc; }   // last (or only) accumulator complete
       }
     }
   } else {
