@@ -113,7 +113,8 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
     // Weight streaming: time ~ (rounds of work items per SM) x (tile width).  Any multiple of 16 is a
     // legal tile width, so pick the one that wastes the least of the last round.
     int best = 128; int64_t best_cost = -1;
-    for (int bn = 64; bn <= 256; bn += 16) {
+    // Without cuts a tile is one long chain of steps and narrow tiles keep every SM busy: down to 32 columns.
+    for (int bn = plan->n_parts == 1 ? 32 : 64; bn <= 256; bn += 16) {
       const int64_t items = ((N + bn - 1) / bn) * plan->n_parts;
       const int64_t cost = ((items + sms - 1) / sms) * bn;
       if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
@@ -165,6 +166,11 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   // skinny problems read long runs of each weight row per stage (DRAM likes 512-byte bursts)
   // one-CTA tiles up to 128 columns take 128-wide K steps as well (half the hand-overs; the stage still fits four times)
   plan->BK = d->BK ? d->BK : (!d->inner_span && (skinny || (plan->cta_group == 1 && plan->BN <= 128)) ? 128 : 64);
+  // a skinny problem without cuts is bounded by the hand-overs along its one K chain: 256-wide stages halve them,
+  // as long as four of them still fit
+  if (!d->BK && skinny && plan->n_parts == 1 && !d->inner_span && plan->cta_group == 1 &&
+      rg::max_stages_for(plan->BN, 256, 1, M) >= 4)
+    plan->BK = 256;
   if (plan->cta_group == 2 && plan->BN != 128 && plan->BN != 256) return RG_ERR_UNSUPPORTED;
   const int smax = rg::max_stages_for(plan->BN, plan->BK, plan->cta_group, M);
   plan->stages = d->stages ? d->stages : smax;
