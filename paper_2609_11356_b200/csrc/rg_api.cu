@@ -130,25 +130,24 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   else if (d->BM == 256) want_group = 2;
   else if (d->BM == 128) want_group = 1;
   if (plan->BN == 0 || (want_group == 0 && !skinny)) {
-    // Time ~ rounds of work items x (tile width + a fixed cost per tile).  Each CTA owns 128 rows either
-    // way; a pair halves the items per slot and the B bytes per CTA.  Fewest rounds of the widest tile
-    // wins, which for one to two rounds is often a narrower one-CTA tile (a 512 x 4096 problem is one
-    // round of 128 x 128 tiles), and for many rounds the 256-wide pair.
+    // Time ~ rounds of work items x operand rows a tile loads (128 of A + its width of B): away from the
+    // largest problems the kernels are bound by the bytes a CTA pulls from L2, not by the tensor pipe.  A
+    // pair loads 128 + 128 rows per CTA for a 256-wide tile and measured 0.88 of that.  Any multiple of 16
+    // is a legal width for the one-CTA kernel, so the widest tile that still fits the fewest rounds wins:
+    // 640 x 4096 x 4096 is one round of 128 x 160 tiles, 1536 rows two rounds of 128 x 192.
     const int64_t tiles_m2 = (M + 255) / 256;
     int best_bn = 0, best_group = 0; int64_t best_cost = -1;
     for (int group = 1; group <= 2; ++group) {
       if (want_group && group != want_group) continue;
       if (group == 2 && M <= 128) continue;
-      for (int bn : {256, 128, 64}) {
+      for (int bn = 256; bn >= 32; bn -= 16) {
         if (d->BN && bn != d->BN) continue;
         if (group == 2 && bn != 256) continue;
         if (d->inner_span && bn > 128) continue;
         const int64_t items = (group == 2 ? tiles_m2 : tiles_m) * ((N + bn - 1) / bn) * plan->n_parts;
         const int64_t slots = group == 2 ? sms / 2 : sms;
         const int64_t rounds = (items + slots - 1) / slots;
-        int64_t cost = rounds * (bn + 32) * 100;
-        if (group == 2 && rounds >= 2) cost = cost * 97 / 100;   // more than one round: the pair's lighter B traffic
-        if (group == 1 && rounds == 1) cost = cost * 99 / 100;   // a single round: no cluster set-up
+        const int64_t cost = group == 2 ? rounds * 338 : rounds * (bn + 128);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_bn = bn; best_group = group; }
       }
     }
