@@ -290,21 +290,24 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      bool alive = mbar_wait(bar_q, 0, abort_flag, &g_attn_status_word, 0x1200u);
+    // the whole warp walks the loop converged and an elected lane issues, so that the descriptor
+    // arithmetic stays in the uniform datapath the tensor-core instruction reads its operands from
+    {
+      const bool leader = elect_one();
+      bool alive = warp_mbar_wait(bar_q, 0, abort_flag, &g_attn_status_word, 0x1200u);
       // S_j = Q K_j^T into score accumulator j&1: ascending k over the head dimension, from zero
       auto issue_scores = [&](int j) -> bool {
         const int stage = j & 1;
-        if (!mbar_wait(bar_k_full, j & 1, abort_flag, &g_attn_status_word, 0x1300u)) return false;
+        if (!warp_mbar_wait(bar_k_full, j & 1, abort_flag, &g_attn_status_word, 0x1300u)) return false;
         att_fence_after();
 #pragma unroll
         for (int b = 0; b < DB; ++b) {
           const uint64_t adesc = att_kmajor_desc(sQ + b * Q_BOX), bdesc = att_kmajor_desc(sK + b * K_BOX);
 #pragma unroll
-          for (int a = 0; a < 4; ++a) att_mma_bf16(tmem_base + 128u * stage, adesc + 2u * a, bdesc + 2u * a, IDESC_S, (b | a) ? 1u : 0u);
+          for (int a = 0; a < 4; ++a) if (leader) att_mma_bf16(tmem_base + 128u * stage, adesc + 2u * a, bdesc + 2u * a, IDESC_S, (b | a) ? 1u : 0u);
         }
-        att_commit(bar_s + 8u * stage);
-        att_commit(bar_k_empty);
+        if (leader) att_commit(bar_s + 8u * stage);
+        if (leader) att_commit(bar_k_empty);
         return true;
       };
       if (alive) alive = issue_scores(0);
@@ -317,18 +320,18 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         // Probabilities and product alternate between two buffers: the softmax threads folded the
         // product of block j-2 and saw it complete before they wrote these probabilities.
         const int stage = j & 1; const uint32_t phase = (j >> 1) & 1;
-        if (!mbar_wait(bar_p, j & 1, abort_flag, &g_attn_status_word, 0x1400u)) break;
-        if (!mbar_wait(bar_v_full + 8u * stage, phase, abort_flag, &g_attn_status_word, 0x1480u | stage)) break;
+        if (!warp_mbar_wait(bar_p, j & 1, abort_flag, &g_attn_status_word, 0x1400u)) break;
+        if (!warp_mbar_wait(bar_v_full + 8u * stage, phase, abort_flag, &g_attn_status_word, 0x1480u | stage)) break;
         att_fence_after();
         const uint32_t sV = sV0 + stage * V_BYTES, sPj = sP + stage * P_BYTES;
 #pragma unroll
         for (int b = 0; b < WB; ++b) {
           const uint64_t adesc = att_kmajor_desc(sPj + b * P_BOX), bdesc = att_kmajor_desc(sV + b * V_BOX);
 #pragma unroll
-          for (int a = 0; a < 4; ++a) att_mma_bf16(tmem_base + 256u + 128u * stage, adesc + 2u * a, bdesc + 2u * a, IDESC_PV, (b | a) ? 1u : 0u);
+          for (int a = 0; a < 4; ++a) if (leader) att_mma_bf16(tmem_base + 256u + 128u * stage, adesc + 2u * a, bdesc + 2u * a, IDESC_PV, (b | a) ? 1u : 0u);
         }
-        att_commit(bar_pv + 8u * stage);
-        att_commit(bar_v_empty + 8u * stage);               // the stage may be refilled once these steps have read it
+        if (leader) att_commit(bar_pv + 8u * stage);
+        if (leader) att_commit(bar_v_empty + 8u * stage);               // the stage may be refilled once these steps have read it
       }
     }
   } else {

@@ -189,18 +189,6 @@ __device__ __forceinline__ void umma_pair_lo(uint32_t d_tmem, uint32_t a_lo, uin
   }
 }
 
-// One lane of a converged warp.
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
-  return pred != 0;
-}
-// A wait that the whole (converged) warp makes and leaves with one common answer.
-__device__ __forceinline__ bool warp_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status, uint32_t code) {
-  const bool ok = mbar_wait(bar, parity, abort_flag, status, code);
-  return __all_sync(0xffffffffu, ok);
-}
-
 // One-CTA form of the same: (low word, high word) descriptors, compile-time accumulate.
 template <bool F8, bool ACC>
 __device__ __forceinline__ void umma_one_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
