@@ -702,7 +702,9 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (even CTA only)
-    if (lane == 0 && rank == 0) {
+    // the whole warp walks the loop converged, an elected lane issues (see the one-CTA kernel)
+    if (rank == 0) {
+      const bool leader = elect_one();
       int stage = 0; uint32_t phase = 0;
       bool alive = true;
       int it = 0;
@@ -728,7 +730,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         const int k_begin = p.part_begin[part], k_end = p.part_end[part];
         const int buf = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1;
-        if (!mbar_wait(bar_tempty + 8u * buf, acc_phase ^ 1u, abort_flag, &g_status_word, 0xa00u | buf)) { alive = false; break; }
+        if (!warp_mbar_wait(bar_tempty + 8u * buf, acc_phase ^ 1u, abort_flag, &g_status_word, 0xa00u | buf)) { alive = false; break; }
         tcgen05_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN;
         uint32_t accumulate = 0;                        // every part starts from a zero accumulator
@@ -737,15 +739,17 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
             // one whole turn of the ring
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-              if (alive && !mbar_wait(bar_full + 8u * g, phase, abort_flag, &g_status_word, 0xb00u | g)) alive = false;
+              if (alive && !warp_mbar_wait(bar_full + 8u * g, phase, abort_flag, &g_status_word, 0xb00u | g)) alive = false;
               if (alive) {
                 tcgen05_fence_after();
 #pragma unroll
                 for (int i = 0; i < STEPS; ++i) {
-                  if (g | i) umma_pair_lo<KIND, true>(d_tmem, alo[g][i], blo[g][i], desc_hi, IDESC, 1u);
-                  else umma_pair_lo<KIND, false>(d_tmem, alo[0][0], blo[0][0], desc_hi, IDESC, accumulate);
+                  if (leader) {
+                    if (g | i) umma_pair_lo<KIND, true>(d_tmem, alo[g][i], blo[g][i], desc_hi, IDESC, 1u);
+                    else umma_pair_lo<KIND, false>(d_tmem, alo[0][0], blo[0][0], desc_hi, IDESC, accumulate);
+                  }
                 }
-                umma_commit_pair(bar_empty + 8u * g);
+                if (leader) umma_commit_pair(bar_empty + 8u * g);
               }
             }
             if (!alive) break;
@@ -754,7 +758,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
             k0 += (G - 1) * KBOX * KSUB;                  // the loop adds the last stage's width
             continue;
           }
-          if (!mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0xb00u | stage)) { alive = false; break; }
+          if (!warp_mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0xb00u | stage)) { alive = false; break; }
           tcgen05_fence_after();
           // descriptors differ from the stage-0 ones only in the 16-byte-unit start address (low word)
           const uint64_t adesc0 = desc_a0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
@@ -768,8 +772,10 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 #pragma unroll
               for (int a = 0; a < KBOX / UMMA_K; ++a) {
                 const uint32_t al = a_lo + ((sub * A_BOX_BYTES) >> 4) + 2u * a, bl = b_lo + ((sub * B_BOX_BYTES) >> 4) + 2u * a;
-                if (sub | a) umma_pair_lo<KIND, true>(d_tmem, al, bl, hi, IDESC, 1u);
-                else umma_pair_lo<KIND, false>(d_tmem, al, bl, hi, IDESC, accumulate);
+                if (leader) {
+                  if (sub | a) umma_pair_lo<KIND, true>(d_tmem, al, bl, hi, IDESC, 1u);
+                  else umma_pair_lo<KIND, false>(d_tmem, al, bl, hi, IDESC, accumulate);
+                }
               }
             }
             accumulate = 1;
@@ -779,17 +785,17 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 #pragma unroll
               for (int a = 0; a < KBOX / UMMA_K; ++a) {
                 if (k0 + sub * KBOX + a * UMMA_K < k_end) {   // ascending k; nothing past the end of the part
-                  umma_pair<KIND>(d_tmem, adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a,
+                  if (leader) umma_pair<KIND>(d_tmem, adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a,
                                  bdesc0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a, IDESC, accumulate);
                   accumulate = 1;
                 }
               }
             }
           }
-          umma_commit_pair(bar_empty + 8u * stage);      // frees the stage in both CTAs
+          if (leader) umma_commit_pair(bar_empty + 8u * stage);   // frees the stage in both CTAs
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
-        if (alive) umma_commit_pair(bar_tfull + 8u * buf);   // accumulator complete, in both CTAs
+        if (alive && leader) umma_commit_pair(bar_tfull + 8u * buf);   // accumulator complete, in both CTAs
       }
     }
   } else {
