@@ -221,6 +221,7 @@ struct GemmParams {
   int32_t inner_span;     // second cut level: an accumulator is closed every inner_span k (0 = none; a multiple of the K step)
   int32_t bn;             // tile columns of the one-CTA kernel (any multiple of 16 up to 256)
   uint32_t idesc;         // instruction descriptor for N = bn
+  int32_t mma_m;          // rows of the tensor-core step: 128, or 64 when the problem has at most 64 rows
   int32_t f8;             // operands are e4m3 bytes: M, N as given, every K quantity counted in byte pairs
   uint32_t tmem_cols;     // tensor-memory columns allocated: two accumulators of tmem_cols / 2
   uint32_t a_box_bytes;   // bytes of one A box: 128 B per row actually loaded (rows past M are never fetched)
@@ -571,8 +572,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
       int part, tm, tn;
       decode_work(p, w, part, tm, tn);
-      const int64_t row = (int64_t)tm * BM + quarter * 32 + lane;
-      const bool row_ok = row < p.M;
+      // a 64-row step keeps rows 16q .. 16q+15 in the first 16 lanes of lane quarter q
+      const int64_t row = p.mma_m == 64 ? (int64_t)(quarter * 16 + lane) : (int64_t)tm * BM + quarter * 32 + lane;
+      const bool row_ok = row < p.M && (p.mma_m != 64 || lane < 16);
       const int klen = p.part_end[part] - p.part_begin[part];
       const int ngroups = p.inner_span > 0 ? (klen + p.inner_span - 1) / p.inner_span : 1;
       if (ngroups == 1) {
@@ -1121,7 +1123,10 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   p.bn = plan.BN;
   p.inner_span = plan.inner_span / kdiv;
   p.f8 = kind == KIND_F8E4M3;
-  p.idesc = make_idesc(plan.BN, pair ? 2 * BM : BM, idesc_format(kind));
+  // At most 64 rows: the 64-row step reads half the A rows from shared memory, which is what a narrow tile's
+  // step time is made of ((rows + width) x 32 bytes at 128 bytes per clock).  Same products, same order.
+  p.mma_m = (!pair && M <= 64) ? 64 : BM;
+  p.idesc = make_idesc(plan.BN, pair ? 2 * BM : p.mma_m, idesc_format(kind));
   { uint32_t c = 32; while (c < 2u * (uint32_t)((plan.BN + 31) / 32 * 32)) c <<= 1; p.tmem_cols = c; }
   for (int s = 0; s < plan.n_parts; ++s) { p.part_begin[s] = plan.part_begin[s] / kdiv; p.part_end[s] = plan.part_end[s] / kdiv; }
   EpilogueArgs e{};
