@@ -130,8 +130,8 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   else if (d->BM == 256) want_group = 2;
   else if (d->BM == 128) want_group = 1;
   if (plan->BN == 0 || (want_group == 0 && !skinny)) {
-    // Time ~ rounds of work items x operand rows a tile loads (128 of A + its width of B): away from the
-    // largest problems the kernels are bound by the bytes a CTA pulls from L2, not by the tensor pipe.  A
+    // Time ~ rounds of work items x operand rows of a tile (128 of A + its width of B): below 256 columns a
+    // step is bound by the rows it reads from shared memory (and the tile pulls from L2), not by arithmetic.  A
     // pair loads 128 + 128 rows per CTA for a 256-wide tile and measured 0.88 of that.  Any multiple of 16
     // is a legal width for the one-CTA kernel, so the widest tile that still fits the fewest rounds wins:
     // 640 x 4096 x 4096 is one round of 128 x 160 tiles, 1536 rows two rounds of 128 x 192.
