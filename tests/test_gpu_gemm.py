@@ -171,6 +171,28 @@ def test_batch_invariance_sweep():
     assert_bits_equal(synth.bf16_bits_to_f32(ref[si, sj]), want, "config 2 sampled oracle")
 
 
+def test_rows_up_to_64_take_the_narrow_step_and_keep_their_bits():
+    """Problems of at most 64 rows run the 64-row tensor-core step, larger ones the 128-row step
+    (another accumulator layout, the same products in the same order): a row's bits must not
+    depend on which one computed it, for ragged shapes, K tails, cuts, accumulator groups, a
+    narrowed partial type and the fused epilogue, and both must match the oracle."""
+    N, K = 300, 1000
+    W = synth.normal_bf16((N, K), 0.05, 71); X = synth.normal_bf16((200, K), 1.0, 72)
+    bias = synth.uniform_bf16((N,), -0.1, 0.1, 73); res = synth.normal_bf16((200, N), 1.0, 74)
+    variants = [dict(), dict(cuts=(256, 512)), dict(cuts=(320,), partial_dtype=rg.RG_BF16), dict(inner_span=256),
+                dict(BN=48, BK=64), dict(BN=96, BK=256, stages=2)]
+    for kw in variants:
+        okw = {k: v for k, v in kw.items() if k in ("cuts", "partial_dtype", "inner_span")}
+        big = gpu_gemm(X, W, out_dtype=rgo.F32, bias=bias, act=1, residual=res, **kw)          # 128-row step
+        want = rgo.gemm(X, W, atom_model=HW, out_dtype=rgo.F32, bias=bias, act=1, residual=res, **okw)
+        assert_bits_equal(big, want, f"200 rows {kw}")
+        for M in (1, 7, 16, 33, 64):
+            got = gpu_gemm(X[:M], W, out_dtype=rgo.F32, bias=bias, act=1, residual=res[:M], **kw)   # 64-row step
+            assert_bits_equal(got, big[:M], f"{M} rows against 200 rows {kw}")
+        got = gpu_gemm(X[:65], W, out_dtype=rgo.F32, bias=bias, act=1, residual=res[:65], **kw)     # back to 128
+        assert_bits_equal(got, big[:65], f"65 rows against 200 rows {kw}")
+
+
 # ------------------------------------------------------------------ config 3: decode split-K
 @pytest.mark.parametrize("M", [1, 8, 32])
 def test_decode_split_k_with_residual(M):
