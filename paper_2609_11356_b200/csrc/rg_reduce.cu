@@ -504,9 +504,10 @@ rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_t
   if (valid_hint) {
     warp_rows = (threads == 32) && op != RG_OP_SOFTMAX_DENOM;
   } else if (op == RG_OP_SOFTMAX_DENOM) {
-    // The second pass re-reads the row from L2.  Eight CTAs of 256 threads per SM measured best on
-    // 32768-column rows: enough CTAs in different phases to overlap the DRAM-bound maximum pass
-    // with the ALU-bound exp pass.
+    // The second pass re-reads the row from L2.  CTAs of 256 threads measured best on 32768-column
+    // rows (four are resident per SM at this kernel's register count): enough CTAs in different
+    // phases to overlap the DRAM-bound maximum pass with the ALU-bound exp pass, few enough rows in
+    // flight for the second pass to find its row in L2 (forcing more resident CTAs was slower).
     warp_rows = false;
     threads = 256;
     while (threads > 32 && nsb < threads / 32) threads /= 2;
