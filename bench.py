@@ -285,8 +285,26 @@ def run_ours(args):
         adesc = rg.rg_attn_desc(block_n=128, scale=ad_ ** -0.5 * 1.4426950408889634, heads=aH, exp_base=2)
         ms_att = timed(lambda: rg.rg_attention(adesc, aQ, aK, aVt, aO), 5)
         del aQ, aK, aVt, aO
+        # configs[1], the batch-invariance shape (N = K = 4096, no cuts), as latency per call: weights rotate
+        # over eight copies (256 MiB, above L2), torch/cuBLAS on the same tensors beside it
+        Wb = [synth.device_normal((4096, 4096), 0.02, seed0 + 50 + i, bf, dev) for i in range(8)]
+        Xb = synth.device_normal((1024, 4096), 1.0, seed0 + 60, bf, dev)
+        sweep_us, sweep_torch_us = {}, {}
+        for Mb in (1, 16, 64, 256, 1024):
+            cb = torch.empty((Mb, 4096), dtype=bf, device=dev)
+            xb = Xb[:Mb]
+            def ours():
+                it[0] += 1
+                rg.rg_gemm(d_plain, xb, Wb[it[0] % 8], cb)
+            def theirs():
+                it[0] += 1
+                torch.matmul(xb, Wb[it[0] % 8].T)
+            sweep_us[str(Mb)] = round(timed(ours, 40, busy) * 1e3, 2)
+            sweep_torch_us[str(Mb)] = round(timed(theirs, 40, busy) * 1e3, 2)
+        del Wb, Xb
         wbytes = 2.0 * 4096 * 14336
         line["widened"] = {
+            "batch_sweep_n4096_k4096_us_by_m": sweep_us, "batch_sweep_torch_cublas_us_by_m": sweep_torch_us,
             "note": "timed alone after the step loop; weights of the two decode paths rotate over four copies (above L2)",
             "fp8_e4m3_square_tflops": round(2.0 * 8192 ** 3 / (ms8 * 1e-3) / 1e12, 1),
             "decode_splitk8_back_to_back_us": round(ms_dec * 1e3, 2), "decode_splitk8_weight_gbs": round(wbytes / (ms_dec * 1e-3) / 1e9, 1),
