@@ -4,18 +4,22 @@
 // are all part of the arithmetic and all come from the descriptor.
 //
 // One CTA owns 128 query rows of one head.  Per key block j:
-//   warp 0 (TMA)      K_j [w x d] and Vt_j [d x w] boxes, each into its own two-stage ring (Q once)
-//   warp 1 (MMA)      S = Q K_j^T   d/16 tcgen05.mma steps from a zero accumulator, ascending k; the
+//   warp 0 (TMA)      K_j [w x d] into one stage (refilled as soon as the scores that read it are done, a
+//                     whole block before it is needed) and Vt_j [d x w] into a two-stage ring (Q once)
+//   warp 1 (MMA)      the whole warp walks the loop, an elected lane issues.
+//                     S = Q K_j^T   d/16 tcgen05.mma steps from a zero accumulator, ascending k; the
 //                     scores of block j+1 are issued before the P V product of block j (two score
 //                     accumulators in tensor memory), so the softmax threads never wait for scores
-//                     PV = P Vt_j^T w/16 steps from a zero accumulator, ascending key
-//   warps 2-9         two threads per query row (its TMEM lane), each with half of the block's keys and
-//                     half of the output columns; partial maxima and partial row sums (subtrees of
-//                     the same tree) meet in shared memory:
+//                     PV = P Vt_j^T w/16 steps from a zero accumulator, ascending key, into one of two
+//                     product accumulators (probabilities are double-buffered in shared memory too)
+//   warps 2-17        four threads per query row (its TMEM lane), each with a quarter of the block's keys
+//                     and a quarter of the output columns; partial maxima and partial row sums (subtrees
+//                     of the same tree) meet in shared memory, one barrier per block:
 //                     s_t = acc * scale; m_j = max(m_{j-1}, max_t s_t); alpha = exp(m_{j-1} - m_j);
 //                     p_t = exp(s_t - m_j); l_j = alpha*l_{j-1} + TREE_t p_t (balanced tree over the
 //                     block's keys in order); P = p narrowed to bf16, written to shared memory in the
-//                     swizzled K-major layout the tensor core reads; O_j = alpha*O_{j-1} + PV
+//                     swizzled K-major layout the tensor core reads; O_j = alpha*O_{j-1} + PV, folded
+//                     one block later so that the product has a whole block to finish
 // and at the end O / l, one division, one rounding to the output type.  exp is one of the library's
 // specified exponentials (rg_exp, or rg_exp2 with log2 e folded into the scale), not the hardware's.
 // With causal masking the walk of a query tile stops at its own end, and the blocks from the tile's
