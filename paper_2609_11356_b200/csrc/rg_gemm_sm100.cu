@@ -9,8 +9,10 @@
 //
 // CTA roles (320 threads):
 //   warp 0           TMA producer: A[BM x 64] and B[BN x 64] boxes (128-byte swizzle), one lane per box
-//   warp 1, lane 0   MMA issuer: 4 steps of K=16 per 64-wide box, ascending; tcgen05.commit
-//                    frees the stage; a final commit publishes the accumulator
+//   warp 1           MMA issuer: the warp walks the loop converged and an elected lane issues
+//                    4 steps of K=16 per 64-wide box, ascending; tcgen05.commit frees the stage; a
+//                    final commit publishes the accumulator.  The step is 128 rows, or 64 rows when
+//                    the problem has at most 64 (half the A rows read from shared memory per step)
 //   warps 2..9       epilogue: tcgen05.ld of their 32 TMEM lanes (warp % 4 picks the lane
 //                    quarter; the two warps of a quarter take alternate 32-column chunks),
 //                    epilogue math, global stores
