@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 
 def _case(g):
-    M = int(g.choice([1, 7, 33, 128, 129, 200, 300]))
+    M = int(g.choice([1, 7, 33, 64, 65, 128, 129, 200, 300]))      # up to 64 rows: the 64-row tensor-core step
     N = int(g.choice([8, 40, 64, 130, 256, 328]))
     K = int(g.choice([64, 192, 576, 1000, 1024, 2048]))
     f16 = bool(g.integers(0, 2))
@@ -104,7 +104,7 @@ def test_random_fp8_descriptor_matches_oracle(seed):
     from _gpu_util import HW8
     from paper_2609_11356_b200 import synth
     g = np.random.default_rng(9000 + seed)
-    M = int(g.choice([1, 7, 33, 129, 200, 300])); N = int(g.choice([8, 40, 130, 256, 328]))
+    M = int(g.choice([1, 7, 33, 64, 65, 129, 200, 300])); N = int(g.choice([8, 40, 130, 256, 328]))
     K = int(g.choice([64, 190, 576, 1000, 1024, 2048]))
     nest = bool(g.integers(0, 3) == 0)
     step = 128 if nest else 32
