@@ -146,7 +146,8 @@ rg_status_t rg_desc_validate(const rg_desc_t* d, int64_t M, int64_t N, int64_t K
  * the epilogue are excluded.  Returns 0 for a malformed descriptor.  Host only. */
 uint64_t rg_desc_class(const rg_desc_t* d);
 
-/* Bytes of workspace rg_gemm needs: 0 without cuts, else (n_cuts+1) * M * roundup(N,4) * sizeof(partial_dtype). */
+/* Bytes of workspace rg_gemm needs: 0 without cuts, else (n_cuts+1) * M * roundup(N,4) * sizeof(partial_dtype);
+ * SIZE_MAX if that product does not fit size_t (no buffer satisfies it, so the call is refused). */
 size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N);
 
 /* C[M,N] = epilogue( merge_s( sum_{k in part s} A[i,k] * B[j,k] ) )   (C = A * B^T).
@@ -244,6 +245,9 @@ size_t rg_gemm_host_scratch_bytes(const rg_desc_t* d, int64_t M, int64_t N, int6
                                   const rg_epilogue_t* epi);
 rg_status_t rg_gemm_host(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
                          const rg_epilogue_t* epi, void* dev_scratch, size_t dev_scratch_bytes, void* cuda_stream);
+/* rg_reduce_rows_host: args->weight is read by RG_OP_RMSNORM only; with another op a non-null weight is
+ * refused (RG_ERR_UNSUPPORTED) before anything is copied.  The scratch size covers the row copy, the
+ * result, the RMSNorm weight and the auxiliary output, whether or not a call uses them. */
 size_t rg_reduce_rows_host_scratch_bytes(rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out);
 rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out,
                                 const rg_reduce_args_t* args, void* dev_scratch, size_t dev_scratch_bytes,
@@ -269,6 +273,18 @@ rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_
 #define RG_NOALLOC_WS_BYTES (8u << 20)
 rg_status_t rg_gemm_noalloc(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
                             const rg_epilogue_t* epi, void* cuda_stream);
+
+/* Self-test of the bounded device-side wait (the paper has no counterpart: this is the library's
+ * failure-detection path, exercised on purpose).  Launches one small CTA that waits on a barrier
+ * nothing arrives on: one warp with the limit `limit_ns` (1 us .. 100 ms, else RG_ERR_SHAPE), which
+ * runs out, records RG_SELFTEST_WAIT_CODE in the health word and raises the CTA's abort flag; a second
+ * warp with the library's ordinary long limit, which must leave as soon as it sees the flag.  Each
+ * warp that abandoned its wait adds one to *dev_counter (a DEVICE pointer to 4 bytes the caller has
+ * set to zero), so a caller reads 2 there afterwards.  The kernel returns normally: nothing hangs,
+ * nothing faults and the context stays usable; rg_device_status then reports RG_ERR_TIMEOUT with
+ * that code, once.  Asynchronous on `cuda_stream`. */
+#define RG_SELFTEST_WAIT_CODE 0xE00u
+rg_status_t rg_selftest_bounded_wait(uint64_t limit_ns, uint32_t* dev_counter, void* cuda_stream);
 
 /* Device-side health word of the current device.  Every wait inside the kernels is bounded; a
  * wait that gives up records a code here, lets the kernel drain and return, and leaves the

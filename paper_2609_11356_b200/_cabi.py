@@ -21,12 +21,13 @@ RG_COLOP_SUM, RG_COLOP_DOT = 0, 1
 RG_OP_SUM, RG_OP_RMSNORM, RG_OP_SOFTMAX_DENOM = 0, 1, 2
 RG_MAX_CUTS = 63
 RG_NOALLOC_WS_BYTES = 8 << 20
+RG_SELFTEST_WAIT_CODE = 0xE00
 
 # every symbol include/rg.h declares
 EXPORTS = ["rg_desc_init", "rg_desc_validate", "rg_desc_class", "rg_gemm_workspace_bytes", "rg_gemm",
            "rg_reduce_rows", "rg_gemm_host_scratch_bytes", "rg_gemm_host", "rg_reduce_rows_host_scratch_bytes",
            "rg_reduce_rows_host", "rg_device_status", "rg_status_string", "rg_gemm_noalloc",
-           "rg_reduce_cols_workspace_bytes", "rg_reduce_cols", "rg_attention"]
+           "rg_reduce_cols_workspace_bytes", "rg_reduce_cols", "rg_attention", "rg_selftest_bounded_wait"]
 
 
 class rg_attn_desc_t(C.Structure):
@@ -87,6 +88,7 @@ def load():
     L.rg_reduce_cols.restype = C.c_int; L.rg_reduce_cols.argtypes = [D, C.c_int, T, T, T, vp, sz, vp]
     L.rg_attention.restype = C.c_int; L.rg_attention.argtypes = [C.POINTER(rg_attn_desc_t), T, T, T, T, vp]
     L.rg_gemm_noalloc.restype = C.c_int; L.rg_gemm_noalloc.argtypes = [D, T, T, T, E, vp]
+    L.rg_selftest_bounded_wait.restype = C.c_int; L.rg_selftest_bounded_wait.argtypes = [C.c_uint64, vp, vp]
     L.rg_device_status.restype = C.c_int; L.rg_device_status.argtypes = [C.POINTER(C.c_uint32)]
     L.rg_status_string.restype = C.c_char_p; L.rg_status_string.argtypes = [C.c_int]
     _lib = L

@@ -64,6 +64,13 @@ def rg_device_status() -> int:
     return int(code.value)
 
 
+def rg_selftest_bounded_wait(limit_ns: int, counter):
+    """Launch the bounded-wait self-test (see include/rg.h).  `counter`: a zeroed CUDA int32/uint32
+    tensor of one element; it holds 2 afterwards (both warps abandoned their wait)."""
+    st = K.load().rg_selftest_bounded_wait(int(limit_ns), counter.data_ptr(), _stream(counter))
+    _check(st, "rg_selftest_bounded_wait")
+
+
 # ---------------------------------------------------------------- marshalling
 def _dtype_code(t) -> int:
     import torch

@@ -89,11 +89,7 @@ rg_status_t check_gemm_shapes(const rg_tensor_t* A, const rg_tensor_t* B, const 
   return RG_OK;
 }
 
-int device_sms() {
-  int dev = 0, sms = 148;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  return sms > 0 ? sms : 148;
-}
+int device_sms() { return rg::current_device().sms; }
 
 rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::GemmPlan* plan) {
   plan->n_parts = (int)d->n_cuts + 1;
@@ -219,7 +215,13 @@ uint64_t rg_desc_class(const rg_desc_t* d) {
 
 size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N) {
   if (!d || d->n_cuts == 0 || d->n_cuts > RG_MAX_CUTS || M <= 0 || N <= 0) return 0;
-  return (size_t)(d->n_cuts + 1) * (size_t)M * (size_t)((N + 3) / 4 * 4) * (d->partial_dtype == RG_F32 ? 4 : 2);
+  // a product that does not fit size_t is reported as SIZE_MAX, which no buffer satisfies
+  if (N > INT64_MAX - 3) return SIZE_MAX;
+  size_t b = (size_t)(d->n_cuts + 1);
+  if (__builtin_mul_overflow(b, (size_t)M, &b) || __builtin_mul_overflow(b, (size_t)((N + 3) / 4 * 4), &b) ||
+      __builtin_mul_overflow(b, (size_t)(d->partial_dtype == RG_F32 ? 4 : 2), &b))
+    return SIZE_MAX;
+  return b;
 }
 
 rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
@@ -399,14 +401,28 @@ rg_status_t rg_gemm_host(const rg_desc_t* d, const rg_tensor_t* A, const rg_tens
   return RG_OK;
 }
 
+// Where each piece of a host-buffer reduction lives in the caller's device scratch.  The size
+// function and the call both go through this one routine, so they cannot disagree.  Every slot is
+// reserved whether or not this call uses it (the size function does not see `args`): the row copy,
+// the result, the RMSNorm weight (only that op reads one) and the per-row auxiliary output.
+struct ReduceHostLayout { size_t x, out, weight, aux, total; int64_t ldx; };
+
+static ReduceHostLayout reduce_host_layout(rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out) {
+  ReduceHostLayout L{};
+  L.ldx = (x->cols + 7) / 8 * 8;
+  size_t cur = 0;
+  auto take = [&](size_t bytes) { const size_t at = cur; cur += align_up(bytes, 256); return at; };
+  L.x = take((size_t)x->rows * L.ldx * esize(x->dtype));
+  L.out = take(op == RG_OP_RMSNORM ? (size_t)x->rows * L.ldx * esize(out->dtype) : (size_t)x->rows * 4);
+  L.weight = take(op == RG_OP_RMSNORM ? (size_t)x->cols * 4 : 0);
+  L.aux = take((size_t)x->rows * 4);
+  L.total = cur;
+  return L;
+}
+
 size_t rg_reduce_rows_host_scratch_bytes(rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out) {
   if (!x || !out || x->rows <= 0 || x->cols <= 0) return 0;
-  const int64_t ldx = (x->cols + 7) / 8 * 8;
-  size_t b = align_up((size_t)x->rows * ldx * esize(x->dtype), 256);
-  if (op == RG_OP_RMSNORM) b += align_up((size_t)x->rows * ldx * esize(out->dtype), 256) + align_up((size_t)x->cols * 4, 256);
-  else b += align_up((size_t)x->rows * 4, 256);
-  b += align_up((size_t)x->rows * 4, 256);   // aux
-  return b;
+  return reduce_host_layout(op, x, out).total;
 }
 
 rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_tensor_t* x, const rg_tensor_t* out,
@@ -415,28 +431,30 @@ rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_
   rg_status_t s = check_reduce(d, op, x, out);
   if (s != RG_OK) return s;
   if (args && args->weight && !dtype_ok(args->weight_dtype)) return RG_ERR_SHAPE;
+  // only RMSNorm reads a weight; a weight handed to another op has no slot in the scratch layout
+  if (args && args->weight && op != RG_OP_RMSNORM) return RG_ERR_UNSUPPORTED;
   if (x->rows == 0) return RG_OK;
-  if (!dev_scratch || dev_scratch_bytes < rg_reduce_rows_host_scratch_bytes(op, x, out)) return RG_ERR_WORKSPACE;
+  const ReduceHostLayout L = reduce_host_layout(op, x, out);
+  if (!dev_scratch || dev_scratch_bytes < L.total) return RG_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(dev_scratch) & 255) return RG_ERR_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const int64_t R = x->rows, Cc = x->cols, ldx = (Cc + 7) / 8 * 8;
+  const int64_t R = x->rows, Cc = x->cols, ldx = L.ldx;
   const size_t xes = esize(x->dtype), oes = esize(out->dtype);
-  uint8_t* cur = static_cast<uint8_t*>(dev_scratch);
-  auto take = [&](size_t bytes) { uint8_t* p = cur; cur += align_up(bytes, 256); return p; };
-  rg_tensor_t dx{take((size_t)R * ldx * xes), x->dtype, R, Cc, ldx};
+  uint8_t* base = static_cast<uint8_t*>(dev_scratch);
+  rg_tensor_t dx{base + L.x, x->dtype, R, Cc, ldx};
   rg_tensor_t dout;
-  if (op == RG_OP_RMSNORM) dout = rg_tensor_t{take((size_t)R * ldx * oes), out->dtype, R, Cc, ldx};
-  else dout = rg_tensor_t{take((size_t)R * 4), RG_F32, R, 1, 1};
+  if (op == RG_OP_RMSNORM) dout = rg_tensor_t{base + L.out, out->dtype, R, Cc, ldx};
+  else dout = rg_tensor_t{base + L.out, RG_F32, R, 1, 1};
   rg_reduce_args_t da{};
   if (args) da = *args;
   bool ok = cudaMemcpy2DAsync(dx.ptr, ldx * xes, x->ptr, x->ld * xes, Cc * xes, R, cudaMemcpyHostToDevice, st) == cudaSuccess;
   if (args && args->weight) {
     const size_t wes = esize(args->weight_dtype);
-    void* p = take((size_t)Cc * 4);
+    void* p = base + L.weight;
     ok &= cudaMemcpyAsync(p, args->weight, (size_t)Cc * wes, cudaMemcpyHostToDevice, st) == cudaSuccess;
     da.weight = p;
   }
-  void* daux = (args && args->aux_out) ? take((size_t)R * 4) : nullptr;
+  void* daux = (args && args->aux_out) ? base + L.aux : nullptr;
   da.aux_out = daux;
   if (!ok) return RG_ERR_CUDA;
   if ((s = rg_reduce_rows(d, op, &dx, &dout, &da, cuda_stream)) != RG_OK) return s;
@@ -446,6 +464,12 @@ rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_
     ok = cudaMemcpy2DAsync(out->ptr, out->ld * 4, dout.ptr, 4, 4, R, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   if (daux) ok &= cudaMemcpyAsync(args->aux_out, daux, (size_t)R * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   return ok ? RG_OK : RG_ERR_CUDA;
+}
+
+rg_status_t rg_selftest_bounded_wait(uint64_t limit_ns, uint32_t* dev_counter, void* cuda_stream) {
+  if (!dev_counter) return RG_ERR_NULL;
+  if (limit_ns < 1000ull || limit_ns > 100000000ull) return RG_ERR_SHAPE;     // 1 us .. 100 ms: never a long stall
+  return rg::launch_wait_selftest(limit_ns, RG_SELFTEST_WAIT_CODE, dev_counter, static_cast<cudaStream_t>(cuda_stream));
 }
 
 rg_status_t rg_device_status(uint32_t* code) {

@@ -553,11 +553,12 @@ template <int W, int HD, bool BASE2>
 cudaError_t launch_attention(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p, dim3 grid,
                              cudaStream_t st) {
   const size_t smem = attn_smem_bytes<W, HD>();
-  static bool configured = false;
-  if (!configured) {
+  static DeviceOnce configured;                          // the attribute is per device
+  const int dev = current_device().dev;
+  if (!configured.has(dev)) {
     cudaError_t e = cudaFuncSetAttribute(attention_kernel<W, HD, BASE2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured.set(dev);
   }
   attention_kernel<W, HD, BASE2><<<grid, ATT_THREADS, smem, st>>>(tq, tk, tv, p);
   return cudaGetLastError();

@@ -23,6 +23,8 @@
 // device status word, and all roles drain and return; tensor memory is always released.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "rg_common.cuh"
 #include "rg_internal.h"
 #include "rg_ptx.cuh"
@@ -961,6 +963,29 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
   }
 }
 
+// -------------------------------------------------------------- self-test of the bounded wait
+// One CTA, two warps, no copies and no tensor memory: a barrier that nothing ever arrives on.  Warp 0
+// waits on it with the caller's (short) limit, gives up, raises the CTA's abort flag and records
+// `code` in the status word; warp 1 waits on the same barrier with the library's long limit and must
+// leave as soon as it sees the flag.  The kernel then returns normally: this is the path a real kernel
+// takes when a copy or a tensor-core step it waits for never completes.
+__global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(uint64_t limit_ns, uint32_t code, unsigned int* left_early) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5;
+  bool ok;
+  if (warp == 0) ok = mbar_wait(smem_u32(&bar), 0, abort_flag, &g_status_word, code, limit_ns);
+  else ok = mbar_wait(smem_u32(&bar), 0, abort_flag, &g_status_word, code | 0x80u);      // 2 s limit: leaves through the flag
+  if (!ok && (threadIdx.x & 31) == 0) atomicAdd(left_early, 1u);
+}
+
 // ------------------------------------------------------------ host: tensor maps
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -998,6 +1023,43 @@ bool make_tmap(CUtensorMap* map, const void* ptr, int dtype, int64_t rows, int64
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Encoding a tensor map costs a driver call per operand, which shows on GEMMs of a few tens of
+// microseconds (App. E, last paragraph: the descriptor path's host cost is visible under ~100 us).  A
+// map depends only on (address, type, shape, pitch, box), never on the data, so the last few are kept:
+// a decode loop that calls with the same weights and activations buffers encodes nothing.
+struct TmapKey {
+  const void* ptr; int64_t rows, cols, ld; int32_t dtype, box_rows;
+  bool operator==(const TmapKey& o) const {
+    return ptr == o.ptr && rows == o.rows && cols == o.cols && ld == o.ld && dtype == o.dtype && box_rows == o.box_rows;
+  }
+};
+constexpr int TMAP_CACHE_ENTRIES = 64;
+struct TmapCache {
+  std::mutex mu;
+  TmapKey key[TMAP_CACHE_ENTRIES];
+  CUtensorMap map[TMAP_CACHE_ENTRIES];
+  uint64_t stamp[TMAP_CACHE_ENTRIES] = {};   // 0 = empty; otherwise the tick of the last use
+  uint64_t tick = 0;
+};
+TmapCache g_tmaps;
+
+bool cached_tmap(CUtensorMap* out, const void* ptr, int dtype, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+  const TmapKey k{ptr, rows, cols, ld, dtype, box_rows};
+  std::lock_guard<std::mutex> lock(g_tmaps.mu);
+  int victim = 0;
+  for (int i = 0; i < TMAP_CACHE_ENTRIES; ++i) {
+    if (g_tmaps.stamp[i] && g_tmaps.key[i] == k) {
+      g_tmaps.stamp[i] = ++g_tmaps.tick;
+      *out = g_tmaps.map[i];
+      return true;
+    }
+    if (g_tmaps.stamp[i] < g_tmaps.stamp[victim]) victim = i;      // least recently used (or empty)
+  }
+  if (!make_tmap(out, ptr, dtype, rows, cols, ld, box_rows)) return false;
+  g_tmaps.key[victim] = k; g_tmaps.map[victim] = *out; g_tmaps.stamp[victim] = ++g_tmaps.tick;
+  return true;
+}
+
 constexpr size_t SMEM_LIMIT = 232448;   // 227 KiB of dynamic shared memory per CTA
 
 size_t smem_bytes_for(int bn, int ksub, int stages, int a_rows) {
@@ -1016,11 +1078,12 @@ size_t smem_bytes_for_pair(int bn, int ksub, int stages) {
 template <int BN, int KSUB, int KIND>
 cudaError_t launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   const size_t smem = smem_bytes_for_pair(BN, KSUB, p.num_stages);
-  static bool configured = false;
-  if (!configured) {
+  static DeviceOnce configured;
+  const int dev = current_device().dev;
+  if (!configured.has(dev)) {
     cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_pair_kernel<BN, KSUB, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured.set(dev);
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid, 1, 1);
@@ -1045,11 +1108,12 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const Gemm
 template <int KSUB, bool F8>
 cudaError_t launch_one_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   const size_t smem = smem_bytes_for(p.bn, KSUB, p.num_stages, (int)(p.a_box_bytes / (KBOX * 2)));
-  static size_t configured = 0;
-  if (smem > configured) {
+  static DeviceOnce configured;
+  const int dev = current_device().dev;
+  if (!configured.has(dev)) {
     cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<KSUB, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
     if (e != cudaSuccess) return e;
-    configured = SMEM_LIMIT;
+    configured.set(dev);
   }
   // programmatic stream serialisation: the CTAs may set themselves up (barriers, tensor memory,
   // descriptor prefetch) while the kernel before this one in the stream drains
@@ -1075,7 +1139,7 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmP
 
 // The same tensor map for other kernels of the library (boxes of 64 columns x box_rows rows, 128-byte swizzle).
 bool make_operand_tmap(CUtensorMap_st* map, const void* ptr, int dtype, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
-  return make_tmap(map, ptr, dtype, rows, cols, ld, box_rows);
+  return cached_tmap(map, ptr, dtype, rows, cols, ld, box_rows);
 }
 
 int a_box_rows_for(int64_t M) { return M >= BM ? BM : (int)((M + 7) / 8 * 8); }
@@ -1097,6 +1161,11 @@ rg_status_t read_and_clear_status(uint32_t* code) {
   return v ? RG_ERR_TIMEOUT : RG_OK;
 }
 
+rg_status_t launch_wait_selftest(uint64_t limit_ns, uint32_t code, unsigned int* left_early, cudaStream_t st) {
+  bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(limit_ns, code, left_early);
+  return cudaGetLastError() == cudaSuccess ? RG_OK : RG_ERR_CUDA;
+}
+
 // Launch the GEMM (and the merge when there are cuts).  All arguments were validated by the caller.
 rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
                         const rg_epilogue_t* epi, void* ws, cudaStream_t st) {
@@ -1109,8 +1178,8 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   const int tile_m = pair ? 2 * BM : BM;
   CUtensorMap ta, tb;
   const int a_rows = pair ? BM : a_box_rows_for(M);
-  if (!make_tmap(&ta, A->ptr, A->dtype, M, A->cols, A->ld, a_rows) ||
-      !make_tmap(&tb, B->ptr, B->dtype, N, B->cols, B->ld, pair ? plan.BN / 2 : plan.BN))
+  if (!cached_tmap(&ta, A->ptr, A->dtype, M, A->cols, A->ld, a_rows) ||
+      !cached_tmap(&tb, B->ptr, B->dtype, N, B->cols, B->ld, pair ? plan.BN / 2 : plan.BN))
     return RG_ERR_CUDA;
 
   GemmParams p;
@@ -1144,9 +1213,7 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   p.epi = split ? EpilogueArgs{} : e;
 
   const int64_t total = (int64_t)p.tiles_m * p.tiles_n * p.n_parts;
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = current_device().sms;
   cudaError_t err;
   const int ksub = plan.BK / KBOX;
   if (pair) {

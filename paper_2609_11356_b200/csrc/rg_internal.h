@@ -3,11 +3,35 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/rg.h"
 
 struct CUtensorMap_st;
 
 namespace rg {
+
+// Function attributes are per device: one bit per device ordinal and kernel instantiation.
+struct DeviceOnce {
+  std::atomic<uint64_t> mask{0};
+  bool has(int dev) const { return dev >= 0 && dev < 64 && ((mask.load(std::memory_order_acquire) >> dev) & 1u); }
+  void set(int dev) { if (dev >= 0 && dev < 64) mask.fetch_or(uint64_t(1) << dev, std::memory_order_release); }
+};
+
+struct DeviceInfo { int dev, sms; };
+// The current device and its SM count (looked up once per device).
+inline DeviceInfo current_device() {
+  static std::atomic<int> sms_of[64];
+  DeviceInfo d{0, 148};
+  if (cudaGetDevice(&d.dev) != cudaSuccess) return d;
+  if (d.dev >= 0 && d.dev < 64 && sms_of[d.dev].load(std::memory_order_relaxed) > 0) { d.sms = sms_of[d.dev].load(std::memory_order_relaxed); return d; }
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, d.dev) == cudaSuccess && sms > 0) {
+    d.sms = sms;
+    if (d.dev >= 0 && d.dev < 64) sms_of[d.dev].store(sms, std::memory_order_relaxed);
+  }
+  return d;
+}
 
 // A validated launch plan: speed knobs resolved, parts laid out.
 struct GemmPlan {
@@ -34,6 +58,7 @@ rg_status_t launch_attention_fixed(int block_n, int exp_base, int causal, float 
                                    const rg_tensor_t* Vt, const rg_tensor_t* O, cudaStream_t st);
 rg_status_t read_and_clear_attn_status(uint32_t* code);
 rg_status_t read_and_clear_status(uint32_t* code);
+rg_status_t launch_wait_selftest(uint64_t limit_ns, uint32_t code, unsigned int* left_early, cudaStream_t st);
 rg_status_t read_and_clear_reduce_status(uint32_t* code);
 
 }  // namespace rg

@@ -7,6 +7,8 @@
 
 namespace rg {
 
+// How long a device-side wait may last before it gives up.  The kernels of the library use this
+// default; the limit is an argument of every wait so that a self-test can let a short one run out.
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -37,11 +39,11 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
-// Bounded wait: gives up after WAIT_LIMIT_NS of wall time, or as soon as another role of the
+// Bounded wait: gives up after `limit_ns` of wall time, or as soon as another role of the
 // CTA has raised `abort_flag`.  On its own timeout it raises the flag and records `code` in
 // *status (first writer wins).  Returns false if the wait was abandoned.
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status,
-                                            uint32_t code) {
+                                            uint32_t code, uint64_t limit_ns) {
   uint64_t t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -49,7 +51,7 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
       if (*abort_flag) return false;
       const uint64_t now = globaltimer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > WAIT_LIMIT_NS) {
+      else if (now - t0 > limit_ns) {
         *abort_flag = 1;
         atomicCAS(status, 0u, code);
         return false;
@@ -59,9 +61,9 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
 }
 // Inline fast path: a barrier that is already complete costs one try_wait and no call.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status,
-                                          uint32_t code) {
+                                          uint32_t code, uint64_t limit_ns = WAIT_LIMIT_NS) {
   if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, status, code);
+  return mbar_wait_slow(bar, parity, abort_flag, status, code, limit_ns);
 }
 // One lane of a converged warp.
 __device__ __forceinline__ bool elect_one() {

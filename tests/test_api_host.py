@@ -96,6 +96,62 @@ def test_workspace_bytes():
     assert rg.rg_gemm_workspace_bytes(rg.rg_desc(cuts=(16, 32, 48), partial_dtype=K.RG_BF16), 3, 5) == 4 * 3 * 8 * 2
 
 
+def test_workspace_bytes_do_not_wrap():
+    """Shapes at the dimension limit with many parts: the byte count is reported as unsatisfiable
+    rather than wrapped around, so neither rg_gemm nor rg_gemm_noalloc can accept a short buffer."""
+    L = K.load()
+    big = (1 << 31) - 1024
+    d = rg.rg_desc(cuts=tuple(16 * i for i in range(1, 64)))
+    exact = 64 * big * big * 4                                   # = 2^70: does not fit 64 bits
+    assert exact >= 1 << 64
+    assert rg.rg_gemm_workspace_bytes(d, big, big) == (1 << 64) - 1
+    assert rg.rg_gemm_workspace_bytes(rg.rg_desc(cuts=(16,)), big, 4096) == 2 * big * 4096 * 4   # large but representable
+    A = _t(0x1000, K.RG_BF16, big, 2048); B = _t(0x2000, K.RG_BF16, big, 2048); Cm = _t(0x3000, K.RG_BF16, big, big)
+    assert L.rg_gemm(C.byref(d), C.byref(A), C.byref(B), C.byref(Cm), None, 0x4000, 1 << 40, None) == 6
+    assert L.rg_gemm_noalloc(C.byref(d), C.byref(A), C.byref(B), C.byref(Cm), None, None) == 6
+
+
+def _align256(n):
+    return (n + 255) // 256 * 256
+
+
+@pytest.mark.parametrize("op", [K.RG_OP_SUM, K.RG_OP_RMSNORM, K.RG_OP_SOFTMAX_DENOM])
+@pytest.mark.parametrize("xdt,odt", [(K.RG_F32, K.RG_F32), (K.RG_BF16, K.RG_BF16), (K.RG_BF16, K.RG_F32)])
+def test_reduce_host_scratch_size_covers_every_slot(op, xdt, odt):
+    """The scratch a host-buffer reduction asks for holds the row copy, the result, the RMSNorm weight and
+    the auxiliary output, each on a 256-byte boundary, for every op; a weight handed to an op that does not
+    read one is refused before any copy."""
+    L = K.load()
+    R, Cc = 37, 1001
+    es = {K.RG_F32: 4, K.RG_BF16: 2}
+    if op != K.RG_OP_RMSNORM:
+        odt = K.RG_F32
+    x = _t(0x10000, xdt, R, Cc); o = _t(0x20000, odt, R, Cc if op == K.RG_OP_RMSNORM else 1)
+    ldx = (Cc + 7) // 8 * 8
+    want = _align256(R * ldx * es[xdt])
+    want += _align256(R * ldx * es[odt]) if op == K.RG_OP_RMSNORM else _align256(R * 4)
+    want += _align256(Cc * 4) if op == K.RG_OP_RMSNORM else 0
+    want += _align256(R * 4)
+    need = L.rg_reduce_rows_host_scratch_bytes(op, C.byref(x), C.byref(o))
+    assert need == want
+    d = rg.rg_desc()
+    args = K.rg_reduce_args_t(); args.weight = 0x30000; args.weight_dtype = K.RG_F32; args.aux_out = 0x40000
+    short = L.rg_reduce_rows_host(C.byref(d), op, C.byref(x), C.byref(o), C.byref(args), 0x100000, need - 1, None)
+    if op == K.RG_OP_RMSNORM:
+        assert short == 6                                        # one byte short: refused
+    else:
+        assert short == 3                                        # a weight with SUM / SOFTMAX_DENOM
+        args.weight = None
+        assert L.rg_reduce_rows_host(C.byref(d), op, C.byref(x), C.byref(o), C.byref(args), 0x100000, need - 1, None) == 6
+
+
+def test_selftest_arguments():
+    L = K.load()
+    assert L.rg_selftest_bounded_wait(1_000_000, None, None) == 1
+    assert L.rg_selftest_bounded_wait(10, 0x1000, None) == 4              # below 1 us
+    assert L.rg_selftest_bounded_wait(10**9, 0x1000, None) == 4           # above 100 ms: never a long stall
+
+
 def _t(ptr, dtype, rows, cols, ld=None):
     return K.rg_tensor_t(ptr, dtype, rows, cols, cols if ld is None else ld)
 

@@ -59,15 +59,15 @@ def test_rmsnorm_bit_exact(shape, dtype, fma):
 
 @pytest.mark.parametrize("shape", [(300, 8192), (200, 20000), (150, 32764), (160, 12292), (149, 32768), (700, 8196), (150, 49152)])
 @pytest.mark.parametrize("spread", [False, True])
-def test_softmax_normaliser_staged_rows_bit_exact(shape, spread):
-    """fp32 rows between 8192 and 32768 columns with at least one row per SM take the kernel that
-    stages whole rows in shared memory; ragged last chunks and exponent-spread draws included."""
+def test_softmax_normaliser_long_rows_bit_exact(shape, spread):
+    """fp32 rows of 8192 to 49152 columns, at least one row per SM: several steps of the two-pass kernel per
+    row; row lengths off the 16-byte and the warp-block grid, and exponent-spread draws included."""
     x = synth.normal_f32(shape, 100.0, 31)
     if spread:
         x = synth.spread_exponents_f32(synth.normal_f32(shape, 1.0, 32), 33, -6, 6)
     got, gmax = gpu_reduce(rg.RG_OP_SOFTMAX_DENOM, x)
     want, wmax = rgo.reduce_rows(rgo.OP_SOFTMAX_DENOM, x)
-    assert_bits_equal(got, want, f"staged softmax normaliser {shape}")
+    assert_bits_equal(got, want, f"long-row softmax normaliser {shape}")
     assert_bits_equal(gmax, wmax, "row max")
     # the generic kernel gives the same bits
     other, _ = gpu_reduce(rg.RG_OP_SOFTMAX_DENOM, x, BN=256)
@@ -185,3 +185,37 @@ def test_host_buffer_form_matches_device_form():
     torch.cuda.synchronize()
     want, _ = rgo.reduce_rows(rgo.OP_SUM, x)
     assert_bits_equal(oh.numpy(), want, "host-buffer row sum")
+
+
+@pytest.mark.parametrize("op", [rg.RG_OP_SUM, rg.RG_OP_RMSNORM, rg.RG_OP_SOFTMAX_DENOM])
+@pytest.mark.parametrize("with_weight,with_aux", [(False, False), (True, True), (False, True), (True, False)])
+def test_host_buffer_form_stays_inside_its_scratch(op, with_weight, with_aux):
+    """Scratch of exactly the size the library asks for, with canary bytes right behind it: every op and
+    every combination of optional arguments stays inside, and the results equal the oracle's."""
+    from paper_2609_11356_b200.api import rg_reduce_rows_host, rg_reduce_rows_host_scratch_bytes
+    R, Cc = 37, 1001
+    x = synth.normal_f32((R, Cc), 1.0, 40 + op)
+    w = synth.normal_f32((Cc,), 0.05, 41, mean=1.0)
+    xh = torch.from_numpy(x).pin_memory()
+    oh = (torch.empty((R, Cc), dtype=torch.float32) if op == rg.RG_OP_RMSNORM else torch.empty(R, dtype=torch.float32)).pin_memory()
+    auxh = torch.empty(R, dtype=torch.float32).pin_memory() if with_aux else None
+    need = rg_reduce_rows_host_scratch_bytes(op, xh, oh)
+    buf = torch.full((need + 4096,), 0xA5, dtype=torch.uint8, device=DEV)
+    kw = dict(aux_out=auxh)
+    if with_weight:
+        kw["weight"] = torch.from_numpy(w).pin_memory()
+    if with_weight and op != rg.RG_OP_RMSNORM:
+        with pytest.raises(rg.RgError) as ei:                    # only RMSNorm reads a weight
+            rg_reduce_rows_host(rg.rg_desc(), op, xh, oh, buf[:need], eps=1e-5, **kw)
+        assert ei.value.status == 3
+        torch.cuda.synchronize()
+        assert bool((buf == 0xA5).all())                         # refused before any copy
+        return
+    rg_reduce_rows_host(rg.rg_desc(), op, xh, oh, buf[:need], eps=1e-5, **kw)
+    torch.cuda.synchronize()
+    assert bool((buf[need:] == 0xA5).all()), "the call wrote past the scratch it asked for"
+    want, waux = rgo.reduce_rows({rg.RG_OP_SUM: rgo.OP_SUM, rg.RG_OP_RMSNORM: rgo.OP_RMSNORM, rg.RG_OP_SOFTMAX_DENOM: rgo.OP_SOFTMAX_DENOM}[op],
+                                 x, weight=w if with_weight else None, eps=1e-5)
+    assert_bits_equal(oh.numpy(), want, f"host-buffer reduction {op}")
+    if with_aux and op != rg.RG_OP_SUM:
+        assert_bits_equal(auxh.numpy(), waux, f"host-buffer reduction {op} aux")
