@@ -290,7 +290,6 @@ def test_k576_walk_of_the_paper():
 def test_position_independence(fmt):
     """P8: one K-vector pair gives the same bits at any row, column, tile width, kernel and M (Sec. 3.2.2:
     what tiles the output stays out of the order)."""
-    import torch
     from tests._gpu_util import gpu_gemm
     g = np.random.default_rng(8)
     K = 512
@@ -308,4 +307,3 @@ def test_position_independence(fmt):
         got = gpu_gemm(np.repeat(a1, M, 0), np.repeat(b1, N, 0), out_dtype=rgo.F32, **knobs)
         seen |= set(np.unique(got.view(np.uint32)).tolist())
     assert seen == {int(want.view(np.uint32)[0])}
-    del torch

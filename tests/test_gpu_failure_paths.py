@@ -3,7 +3,6 @@ with a short limit that runs out and returns.  Every device-side wait in the lib
 a wait that gives up raises the CTA's abort flag, records a code in the device health word, and the
 kernel drains and returns.  Here a tiny self-test kernel waits on a barrier nothing arrives on, with
 a limit of a few milliseconds; the real GEMM, attention and reduction kernels are never stalled."""
-import numpy as np
 import pytest
 import torch
 
@@ -46,4 +45,3 @@ def test_limits_outside_the_allowed_range_launch_nothing():
         assert ei.value.status == 4
     torch.cuda.synchronize()
     assert int(counter.item()) == 0 and rg.rg_device_status() == 0
-    del np
