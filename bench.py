@@ -189,7 +189,7 @@ def run_ours(args):
 
     d_plain = rg.rg_desc()
     dc_cuts = tuple(1792 * t for t in range(1, 8))
-    d_split = rg.rg_desc(cuts=dc_cuts)
+    d_split = rg.rg_desc(cuts=dc_cuts, b_static=1)          # the weights are not written by anything in flight (a speed knob)
     ws = torch.empty(rg.rg_gemm_workspace_bytes(d_split, 32, 4096), dtype=torch.uint8, device=dev)
 
     def step(ev=None):
@@ -553,7 +553,8 @@ def run_only(args):
         work, unit = 2.0 * M * N * K / 1e12, "TFLOP/s"
     elif name == "gemm_decode":
         M, N, K = GEMMS["decode"]
-        d = rg.rg_desc(cuts=tuple(1792 * t for t in range(1, 8)))
+        M = args.rows or M
+        d = rg.rg_desc(cuts=tuple(1792 * t for t in range(1, 8)), split_merge=args.split_merge, BN=args.bn, BK=args.bk, stages=args.stages, sm_share=args.sm_share, b_static=args.b_static)
         A = synth.device_normal((M, K), 1.0, 4, bf, dev)
         Ws = [synth.device_normal((N, K), 0.02, 3 + i, bf, dev) for i in range(4)]    # rotate: weights leave L2
         R = synth.device_normal((M, N), 1.0, 5, bf, dev); Cm = torch.empty((M, N), dtype=bf, device=dev)
@@ -592,11 +593,16 @@ def run_only(args):
         fn = lambda: rg.rg_reduce_cols(d, rg.RG_COLOP_DOT if y is not None else rg.RG_COLOP_SUM, x, out, y=y, ws=ws)
         work, unit = (8.0 if y is not None else 4.0) * R_ * C_ / 1e9, "GB/s"
     else:
-        R_, C_ = (16384, RED_C) if name in ("row_sum", "softmax", "softmax_unit") else (RMS_R * 4, RMS_C)
+        R_, C_ = (16384, RED_C) if name in ("row_sum", "softmax", "softmax_unit") else (args.rows or RMS_R * 4, RMS_C)
         if name == "rmsnorm":
-            x = synth.device_normal((R_, C_), 1.0, 9, bf, dev); w = synth.device_normal((C_,), 0.05, 10, bf, dev, mean=1.0)
-            y = torch.empty_like(x)
-            fn = lambda: rg.rg_reduce_rows(d, rg.RG_OP_RMSNORM, x, y, weight=w, eps=1e-5)
+            # four input/output pairs in rotation, so that a launch never finds its rows in L2
+            xs = [synth.device_normal((R_, C_), 1.0, 9 + i, bf, dev) for i in range(4)]
+            w = synth.device_normal((C_,), 0.05, 10, bf, dev, mean=1.0)
+            ys = [torch.empty_like(xs[0]) for _ in range(4)]
+            it = [0]
+            def fn():
+                it[0] += 1
+                rg.rg_reduce_rows(d, rg.RG_OP_RMSNORM, xs[it[0] % 4], ys[it[0] % 4], weight=w, eps=1e-5)
             work = 4.0 * R_ * C_ / 1e9
         else:
             x = synth.device_normal((R_, C_), 1.0 if name == "softmax_unit" else 100.0, 13, f32, dev)
@@ -633,6 +639,13 @@ def main():
     ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_square_f8", "gemm_prefill", "gemm_decode", "gemv_decode", "attention", "col_sum", "col_dot", "row_sum", "softmax", "softmax_unit", "rmsnorm"],
                     help="run one kernel on a small case (used for the ncu captures)")
     ap.add_argument("--gemv-rows", type=int, default=1, help="rows of A for --only gemv_decode")
+    ap.add_argument("--rows", type=int, default=0, help="rows of A for --only gemm_decode (default 32)")
+    ap.add_argument("--split-merge", type=int, default=0, help="--only gemm_decode: 0 library's choice, 1 second kernel through the workspace, 2 inside a cluster")
+    ap.add_argument("--bn", type=int, default=0, help="--only gemm_decode: tile width (0 = library's choice)")
+    ap.add_argument("--bk", type=int, default=0, help="--only gemm_decode: K per pipeline stage (0 = library's choice)")
+    ap.add_argument("--sm-share", type=int, default=0, help="--only gemm_decode: 0 library's choice, 1 one CTA per SM, 2 two CTAs per SM")
+    ap.add_argument("--b-static", type=int, default=0, help="--only gemm_decode: 1 = promise that the weights are not written by work in flight")
+    ap.add_argument("--stages", type=int, default=0, help="--only gemm_decode: ring depth (0 = as many as fit)")
     ap.add_argument("--attn-block", type=int, default=128, help="key block width for --only attention")
     ap.add_argument("--attn-causal", type=int, default=0, help="1: causal masking, for --only attention (flops counted as half)")
     ap.add_argument("--attn-base", type=int, default=0, help="0: base-e exponential, 2: base-two, for --only attention")

@@ -76,7 +76,10 @@ typedef struct {
   uint8_t stages;         /* shared-memory ring depth; 0 = as many as fit */
   uint8_t cta_group;      /* 1, or 2 (pair of SMs on one 256-row tile); 0 = default */
   uint8_t raster;         /* tile walk: 0 = default grouped walk, 1 = row-major, n in 2..64 = groups of n tile rows */
-  uint8_t _pad0;
+  uint8_t split_merge;    /* where split-K parts are added (same tree, same bits): 0 = the library chooses (today: 1);
+                             1 = by a second kernel, through the workspace; 2 = inside the GEMM kernel, by the CTAs
+                             of a thread-block cluster over distributed shared memory (one launch, no workspace;
+                             2..8 parts, one-CTA tiles; RG_ERR_UNSUPPORTED where it does not apply) */
   /* ---- order-deciding fields: these ARE the class key ---- */
   uint8_t in_dtype;       /* rg_dtype_t of A and B: RG_BF16, RG_F16, or RG_F8E4M3 (with atom = RG_ATOM_TC_F8_K32) */
   uint8_t acc_dtype;      /* accumulator: RG_F32 */
@@ -99,7 +102,13 @@ typedef struct {
   uint8_t gemv_fold;      /* RG_ATOM_SCALAR only: the butterfly over the lane totals: 0 = offsets counted up
                              (balanced tree over the lanes), 1 = counted down (balanced tree over the lanes in
                              bit-reversed order: a different sum) */
-  uint8_t _pad1[2];
+  /* ---- two more speed knobs (not part of the class key) ---- */
+  uint8_t sm_share;       /* one-CTA kernel: 0 = the library chooses (today: 1); 1 = a CTA takes a whole SM; 2 = a CTA takes
+                             half an SM's shared and tensor memory (four epilogue warps, tiles up to 128 columns), so the
+                             CTAs of the next launch become resident beside it while it finishes */
+  uint8_t b_static;       /* 1 = the caller promises that no work still in flight on the stream when this call is
+                             enqueued writes B (weights in an inference loop): the kernel may fetch its first B boxes
+                             before the kernels ahead of it have finished.  A is never read early.  0 = no promise */
 } rg_desc_t;
 
 /* A row-major matrix in device memory. */
@@ -157,13 +166,17 @@ size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N);
  * step per 16 consecutive k, in ascending k; a finished part is an fp32 value; the parts are
  * added in the descriptor's tree; then the epilogue.  Without cuts one kernel does everything;
  * with cuts the parts go to `ws` as [part][M][roundup(N,4)] at partial_dtype and a second kernel
- * merges them, the running sum kept at merge_dtype (no atomics anywhere).
+ * merges them, the running sum kept at merge_dtype (no atomics anywhere); or, on request and with 2..8
+ * parts (App. E: a single launch across the split-K slices), the parts stay in the shared memory of
+ * the CTAs of one thread-block cluster, which merge them in the same tree inside the GEMM kernel
+ * (`split_merge = 2`).
  *
  *   A: [M,K], B: [N,K] (both K-contiguous) at d->in_dtype (bf16 or fp16); C: [M,N] bf16, fp16 or fp32;
  *   bias and residual likewise bf16, fp16 or fp32.
  *   A.ptr, B.ptr 16-byte aligned; A.ld, B.ld multiples of 8.  C, bias, residual: any alignment.
  *   epi: nullable.  ws: device, 16-byte aligned, >= rg_gemm_workspace_bytes; contents undefined
- *   afterwards; may be NULL when there are no cuts.
+ *   afterwards (it may not be touched at all when the library merges in-cluster); may be NULL when
+ *   there are no cuts or when the descriptor sets split_merge = 2.
  *   M == 0 or N == 0: returns RG_OK and launches nothing.  K == 0: RG_ERR_SHAPE.
  * Asynchronous on `cuda_stream`. */
 rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,

@@ -39,11 +39,11 @@ class rg_attn_desc_t(C.Structure):
 class rg_desc_t(C.Structure):
     _fields_ = [("size", C.c_uint32),
                 ("BM", C.c_uint16), ("BN", C.c_uint16), ("BK", C.c_uint16),
-                ("stages", C.c_uint8), ("cta_group", C.c_uint8), ("raster", C.c_uint8), ("_pad0", C.c_uint8),
+                ("stages", C.c_uint8), ("cta_group", C.c_uint8), ("raster", C.c_uint8), ("split_merge", C.c_uint8),
                 ("in_dtype", C.c_uint8), ("acc_dtype", C.c_uint8), ("partial_dtype", C.c_uint8), ("merge_dtype", C.c_uint8),
                 ("atom", C.c_uint8), ("k_tail", C.c_uint8), ("fma", C.c_uint8), ("tree", C.c_uint8),
                 ("n_cuts", C.c_uint32), ("cuts", C.c_uint32 * RG_MAX_CUTS), ("inner_span", C.c_uint32),
-                ("gemv_layout", C.c_uint8), ("gemv_fold", C.c_uint8), ("_pad1", C.c_uint8 * 2)]
+                ("gemv_layout", C.c_uint8), ("gemv_fold", C.c_uint8), ("sm_share", C.c_uint8), ("b_static", C.c_uint8)]
 
 
 class rg_tensor_t(C.Structure):

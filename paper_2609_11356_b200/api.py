@@ -20,11 +20,11 @@ def _check(status: int, where: str):
 
 
 def rg_desc(*, cuts: Sequence[int] = (), tree: int = K.RG_TREE_BALANCED, fma: int = 0, BM: int = 0, BN: int = 0,
-            BK: int = 0, stages: int = 0, cta_group: int = 0, raster: int = 0, **order_fields) -> K.rg_desc_t:
+            BK: int = 0, stages: int = 0, cta_group: int = 0, raster: int = 0, split_merge: int = 0, **order_fields) -> K.rg_desc_t:
     """A descriptor with the library defaults (rg_desc_init), then the given fields."""
     d = K.rg_desc_t()
     K.load().rg_desc_init(C.byref(d))
-    d.BM, d.BN, d.BK, d.stages, d.cta_group, d.raster = BM, BN, BK, stages, cta_group, raster
+    d.BM, d.BN, d.BK, d.stages, d.cta_group, d.raster, d.split_merge = BM, BN, BK, stages, cta_group, raster, split_merge
     d.tree, d.fma = tree, fma
     for k, v in order_fields.items():
         setattr(d, k, v)

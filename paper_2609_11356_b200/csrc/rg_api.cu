@@ -51,6 +51,13 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
   if (d->cta_group == 2 && (d->BM == 128 || (d->BN != 0 && d->BN != 128 && d->BN != 256) || d->BK == 256)) return RG_ERR_UNSUPPORTED;   // a pair works on 256 rows, BN >= 128
   if (d->cta_group == 1 && d->BM == 256) return RG_ERR_UNSUPPORTED;
   if (d->raster > 64) return RG_ERR_INVALID_DESC;
+  if (d->split_merge > 2 || d->sm_share > 2 || d->b_static > 1) return RG_ERR_INVALID_DESC;
+  // two CTAs per SM: the one-CTA kernel with four epilogue warps, tiles up to 128 columns, no second cut level
+  if (d->sm_share == 2 && (d->cta_group == 2 || d->BM == 256 || d->BN > 128 || d->BK == 256 || d->inner_span || d->split_merge == 2))
+    return RG_ERR_UNSUPPORTED;
+  // the in-cluster merge: 2 to 8 parts (one CTA of a cluster per part), one-CTA tiles, no second cut level
+  if (d->split_merge == 2 && (d->n_cuts < 1 || d->n_cuts > 7 || d->inner_span || d->cta_group == 2 || d->BM == 256 || d->BK == 256))
+    return RG_ERR_UNSUPPORTED;
   const uint32_t step = d->atom == RG_ATOM_TC_F8_K32 ? 32 : 16;   // products per tensor-core step
   for (uint32_t i = 0; i < d->n_cuts; ++i)
     if (d->cuts[i] % step != 0) return RG_ERR_UNSUPPORTED;   // a cut may not split a step
@@ -91,8 +98,46 @@ rg_status_t check_gemm_shapes(const rg_tensor_t* A, const rg_tensor_t* B, const 
 
 int device_sms() { return rg::current_device().sms; }
 
+// Split-K in one launch: the parts of an output tile go to the CTAs of one thread-block cluster, which merge
+// them over distributed shared memory (no workspace, no second kernel).  Taken when the descriptor asks for it
+// (`split_merge = 2`); the default stays the two-kernel path, which is faster on this GPU: a cluster of eight
+// must sit in one GPC, so only 15 of them (120 of 148 SMs) stream at once, and the cluster-wide hand-over at the
+// end of a tile costs more than the second launch it saves (decode shape: 27.7 us against 26.2 us).
+// Returns false if it does not apply or fit.
+bool plan_cluster_merge(const rg_desc_t* d, int64_t M, int64_t N, rg::GemmPlan* plan) {
+  const int S = plan->n_parts;
+  if (S < 2 || S > 8 || d->inner_span || d->cta_group == 2 || d->BM == 256 || d->BK == 256 || d->split_merge == 1) return false;
+  if (d->split_merge != 2) return false;                    // on request only (see make_plan)
+  const bool f8 = d->in_dtype == RG_F8E4M3;
+  const int bk = d->BK ? d->BK : (M <= 64 ? 128 : 64);
+  const int avail = rg::max_active_clusters(S, bk, f8);
+  if (avail < 1) return false;
+  const int64_t tiles_m = (M + 127) / 128;
+  const int64_t rows = M < 128 ? M : 128;
+  int best = 0; int64_t best_cost = -1;
+  for (int bn = 32; bn <= 256; bn += 16) {
+    if (d->BN && bn != d->BN) continue;
+    const int smax = rg::max_stages_for(bn, bk, 1, M, true);
+    if (smax < (d->stages ? d->stages : 2)) continue;
+    // time ~ rounds of clusters x bytes a CTA streams per tile (its rows of A and its bn rows of B)
+    const int64_t tiles = tiles_m * ((N + bn - 1) / bn);
+    const int64_t cost = ((tiles + avail - 1) / avail) * (bn + rows);
+    if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
+  }
+  if (!best) return false;
+  plan->cluster_merge = 1;
+  plan->BN = best; plan->BK = bk; plan->cta_group = 1;
+  plan->stages = d->stages ? d->stages : rg::max_stages_for(best, bk, 1, M, true);
+  plan->raster = d->raster == 1 ? 1 : 0;
+  plan->group_m = d->raster >= 2 ? d->raster : 8;
+  return true;
+}
+
 rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::GemmPlan* plan) {
   plan->n_parts = (int)d->n_cuts + 1;
+  plan->cluster_merge = 0;
+  plan->half_sm = 0;
+  plan->b_static = d->b_static ? 1 : 0;
   plan->tree = d->tree;
   plan->partial_dtype = d->partial_dtype;
   plan->merge_dtype = d->merge_dtype;
@@ -101,18 +146,29 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
     plan->part_begin[s] = s == 0 ? 0 : (int32_t)d->cuts[s - 1];
     plan->part_end[s] = s == plan->n_parts - 1 ? (int32_t)K : (int32_t)d->cuts[s];
   }
+  if (plan_cluster_merge(d, M, N, plan)) return RG_OK;
+  if (d->split_merge == 2) return RG_ERR_UNSUPPORTED;       // asked for, but it does not fit this shape or device
   const int sms = device_sms();
   const int64_t tiles_m = (M + 127) / 128;
   const bool skinny = M <= 64;     // weight-streaming regime: HBM bound, one partial tile row
+  // On request (`sm_share = 2`) the one-CTA kernel runs at half an SM's shared and tensor memory, one CTA per SM:
+  // the CTAs of the next launch in the stream then become resident beside this launch's, set themselves up and,
+  // under `b_static`, fetch their first weight boxes before the kernels ahead have finished.  Not the default:
+  // on the decode shape the half-depth ring streams 8 % slower, which costs more than the overlap returns while
+  // the chain GEMM -> merge -> next GEMM (about 5 us of completion and launch hand-overs) paces a run of calls.
+  const bool half_ok = !d->inner_span && d->cta_group != 2 && d->BM != 256 && d->BN <= 128 && d->BK != 256;
+  const bool half = half_ok && d->sm_share == 2;
+  if (d->sm_share == 2 && !half) return RG_ERR_UNSUPPORTED;
+  const int slots = sms;
   if (d->BN) plan->BN = d->BN;
   else if (skinny) {
     // Weight streaming: time ~ (rounds of work items per SM) x (tile width).  Any multiple of 16 is a
     // legal tile width, so pick the one that wastes the least of the last round.
     int best = 128; int64_t best_cost = -1;
     // Without cuts a tile is one long chain of steps and narrow tiles keep every SM busy: down to 32 columns.
-    for (int bn = plan->n_parts == 1 ? 32 : 64; bn <= 256; bn += 16) {
+    for (int bn = plan->n_parts == 1 ? 32 : 64; bn <= (half ? 128 : 256); bn += 16) {
       const int64_t items = ((N + bn - 1) / bn) * plan->n_parts;
-      const int64_t cost = ((items + sms - 1) / sms) * bn;
+      const int64_t cost = ((items + slots - 1) / slots) * bn;
       if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
     }
     plan->BN = best;
@@ -154,20 +210,23 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
     if (plan->BN == 0) plan->BN = 64;
   }
   if (d->inner_span && plan->BN > 128) plan->BN = 128;
+  if (half && plan->BN > 128) plan->BN = 128;
   plan->cta_group = want_group ? want_group : 1;
   if (plan->cta_group == 2 && plan->BN < 128) plan->cta_group = 1;
   // the widest two-SM tile runs a seven-stage ring of 64-wide K steps: more slack per byte of shared memory than
   // three 128-wide stages, now that a whole turn of the ring is issued from precomputed descriptor words
   // skinny problems read long runs of each weight row per stage (DRAM likes 512-byte bursts)
   // one-CTA tiles up to 128 columns take 128-wide K steps as well (half the hand-overs; the stage still fits four times)
-  plan->BK = d->BK ? d->BK : (!d->inner_span && (skinny || (plan->cta_group == 1 && plan->BN <= 128)) ? 128 : 64);
+  plan->BK = d->BK ? d->BK : (!d->inner_span && (skinny || (plan->cta_group == 1 && plan->BN <= 128 && !half)) ? 128 : 64);
   // a skinny problem without cuts is bounded by the hand-overs along its one K chain: 256-wide stages halve them,
   // as long as four of them still fit
-  if (!d->BK && skinny && plan->n_parts == 1 && !d->inner_span && plan->cta_group == 1 &&
+  if (!d->BK && skinny && plan->n_parts == 1 && !d->inner_span && plan->cta_group == 1 && !half &&
       rg::max_stages_for(plan->BN, 256, 1, M) >= 4)
     plan->BK = 256;
   if (plan->cta_group == 2 && plan->BN != 128 && plan->BN != 256) return RG_ERR_UNSUPPORTED;
-  const int smax = rg::max_stages_for(plan->BN, plan->BK, plan->cta_group, M);
+  plan->half_sm = half && plan->cta_group == 1 && plan->BK <= 128 && rg::max_stages_for(plan->BN, plan->BK, 1, M, false, true) >= 2;
+  if (d->sm_share == 2 && !plan->half_sm) return RG_ERR_UNSUPPORTED;
+  const int smax = rg::max_stages_for(plan->BN, plan->BK, plan->cta_group, M, false, plan->half_sm != 0);
   plan->stages = d->stages ? d->stages : smax;
   if (plan->stages > smax) return RG_ERR_UNSUPPORTED;
   plan->raster = d->raster == 1 ? 1 : 0;
@@ -240,7 +299,7 @@ rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t*
       (A->ld % ld_mult) || (B->ld % ld_mult))
     return RG_ERR_ALIGNMENT;
   if (A->dtype == RG_F8E4M3 && (K & 1)) return RG_ERR_SHAPE;   // rows of 8-bit operands are whole byte pairs
-  if (d->n_cuts) {
+  if (d->n_cuts && d->split_merge != 2) {                    // the in-cluster merge keeps the parts in shared memory
     if (!ws || ws_bytes < rg_gemm_workspace_bytes(d, M, N)) return RG_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(ws) & 15) return RG_ERR_ALIGNMENT;
   }

@@ -23,6 +23,7 @@
 // device status word, and all roles drain and return; tensor memory is always released.
 #include <cuda.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "rg_common.cuh"
@@ -32,6 +33,15 @@
 namespace rg {
 
 __device__ unsigned int g_status_word = 0;
+
+// Optional wall-clock stamps of the one-CTA kernel's roles (compiled in with -DRG_TIMELINE only; the
+// library build has none of this): [launch % 8][CTA][what] in nanoseconds of the global timer.
+#ifdef RG_TIMELINE
+__device__ unsigned long long g_timeline[8][512][8];
+#define RG_STAMP(slot) do { if (blockIdx.x < 512) g_timeline[p.launch_seq & 7][blockIdx.x][slot] = globaltimer_ns(); } while (0)
+#else
+#define RG_STAMP(slot) do { } while (0)
+#endif
 
 namespace {
 
@@ -227,14 +237,21 @@ struct GemmParams {
   uint32_t idesc;         // instruction descriptor for N = bn
   int32_t mma_m;          // rows of the tensor-core step: 128, or 64 when the problem has at most 64 rows
   int32_t f8;             // operands are e4m3 bytes: M, N as given, every K quantity counted in byte pairs
+  int32_t launch_seq;     // host-side launch counter (used by the optional timeline stamps only)
+  int32_t b_static;       // the caller's promise that no work ahead in the stream writes B: its first boxes are fetched before the dependency wait
   uint32_t tmem_cols;     // tensor-memory columns allocated: two accumulators of tmem_cols / 2
   uint32_t a_box_bytes;   // bytes of one A box: 128 B per row actually loaded (rows past M are never fetched)
+  uint32_t slack_bytes;   // readable bytes kept behind the ring for the tensor-core step's surplus A rows
   void* C;
   int64_t ldc;
   int32_t c_dtype;
-  void* ws;             // split-K partials [part][M][ldw] at ws_dtype; null without cuts
+  void* ws;             // split-K partials [part][M][ldw] at ws_dtype; null without cuts and with the in-cluster merge
   int64_t ldw;
   int32_t ws_dtype;
+  // in-cluster merge (CLUSTER kernels): the n_parts CTAs of a cluster own the parts of one output tile
+  int32_t tree, merge_dtype;   // how the parts are added (descriptor's tree, type of the running sum)
+  int32_t part_rows;           // rows of a tile kept in a CTA's shared-memory partial buffer
+  int32_t part_ld;             // floats between its rows (tile width + 4: spreads the rows over the banks)
   EpilogueArgs epi;
   int32_t part_begin[RG_MAX_CUTS + 1];
   int32_t part_end[RG_MAX_CUTS + 1];
@@ -353,10 +370,10 @@ __device__ __forceinline__ void epilogue_store_chunk(const GemmParams& p, int pa
 // Epilogue of one accumulator tile for one warp: the warp's 32 TMEM lanes (one output row per
 // thread), 32-column chunks chunk0, chunk0+2, ...
 __device__ __forceinline__ void epilogue_tile(const GemmParams& p, const int BN, int part, int64_t row, bool row_ok, int tn,
-                                              uint32_t taddr, int chunk0) {
+                                              uint32_t taddr, int chunk0, int chunk_step = 64) {
   const int col_end = min(p.N, (tn + 1) * BN);            // this tile's columns end here
 #pragma unroll 1
-  for (int c0 = chunk0 * 32; c0 < BN; c0 += 64) {
+  for (int c0 = chunk0 * 32; c0 < BN; c0 += chunk_step) {
     const int col0 = tn * BN + c0;
     if (col0 >= col_end) break;                           // uniform across the warp
     uint32_t r[32];
@@ -400,11 +417,81 @@ __device__ __forceinline__ void grouped_finish(const GemmParams& p, const int BN
   }
 }
 
-// KSUB: 64-wide boxes per pipeline stage (BK = 64 * KSUB); F8: e4m3 operands (kind::f8f6f4).  The tile width p.bn is a run-time value:
+// ---- in-cluster split-K merge (App. E: "a single launch across the split-K slices"; Sec. 3.2.2 "Split-K")
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t cluster_addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr) : "memory");
+  return v;
+}
+
+// Up to eight parts added in the descriptor's tree, the running sum kept at merge_dtype.  BALANCED is
+// the level-by-level definition itself: neighbours pair, an unpaired last value moves up unchanged.
+template <bool MERGE_16>
+__device__ __forceinline__ float4 merge_upto8(float4 (&v)[8], int S, int tree, int merge_dtype) {
+  auto add1 = [merge_dtype](float a, float b) -> float {
+    const float r = f_add(a, b);
+    return MERGE_16 ? round_through(r, merge_dtype) : r;
+  };
+  auto add4 = [&](const float4& a, const float4& b) -> float4 {
+    return make_float4(add1(a.x, b.x), add1(a.y, b.y), add1(a.z, b.z), add1(a.w, b.w));
+  };
+  if (tree == RG_TREE_LEFT) {
+    float4 acc = v[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) if (i < S) acc = add4(acc, v[i]);
+    return acc;
+  }
+  int n = S;
+#pragma unroll
+  for (int half = 4; half >= 1; half >>= 1) {
+#pragma unroll
+    for (int t = 0; t < half; ++t) {
+      if (2 * t + 1 < n) v[t] = add4(v[2 * t], v[2 * t + 1]);
+      else if (2 * t < n) v[t] = v[2 * t];
+    }
+    n = (n + 1) >> 1;
+  }
+  return v[0];
+}
+
+// bias -> SiLU -> residual -> one rounding for four consecutive columns of one row, then the store.
+__device__ __forceinline__ void finish_and_store4(const EpilogueArgs& e, void* C, int64_t ldc, int c_dtype, int N, int64_t row, int col0, float4 acc) {
+  float v[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    if (col0 + c < N) {
+      if (e.bias) v[c] = f_add(v[c], load_scalar(e.bias, e.bias_dtype, col0 + c));
+      if (e.act == 1) v[c] = rg_silu(v[c]);
+      if (e.residual) v[c] = f_add(v[c], load_scalar(e.residual, e.residual_dtype, row * e.ldr + col0 + c));
+    }
+  }
+  uint16_t* const c16 = static_cast<uint16_t*>(C) + row * ldc + col0;
+  if (col0 + 4 <= N && c_dtype != RG_F32 && (reinterpret_cast<uintptr_t>(c16) & 7) == 0) {
+    uint2 o;
+    o.x = pack_16x2(v[0], v[1], c_dtype);
+    o.y = pack_16x2(v[2], v[3], c_dtype);
+    *reinterpret_cast<uint2*>(c16) = o;
+  } else {
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      if (col0 + c < N) store_scalar(C, c_dtype, row * ldc + col0 + c, v[c]);
+  }
+}
+
+// KSUB: 64-wide boxes per pipeline stage (BK = 64 * KSUB); F8: e4m3 operands (kind::f8f6f4).
+// CLUSTER: split-K in one launch.  The n_parts CTAs of a thread-block cluster own the parts of one output
+// tile (CTA rank = part); each walks its part exactly as the plain kernel does, leaves its fp32 part (rounded
+// once to partial_dtype) in its own shared memory, and after a cluster-wide hand-over every CTA merges one
+// slice of the tile, reading the parts of all CTAs over distributed shared memory in the descriptor's
+// tree, applies the epilogue and stores.  No workspace in global memory, no second launch, no atomics.  The tile width p.bn is a run-time value:
 // any multiple of 16 up to 256 is a legal step width, which lets the host size tiles so that the
 // work items fill whole waves.
-template <int KSUB, bool F8>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+// EPI_WARPS: 8 epilogue warps (320 threads, one CTA per SM), or 4 (192 threads, a warp takes every 32-column
+// chunk of its lane quarter): that form is launched with at most half an SM's shared memory and tensor memory, so
+// two CTAs share an SM, and the CTAs of the next launch in the stream can become resident, set themselves up and
+// fetch their first weight boxes while this launch's last CTAs finish (used for the weight-streaming shapes).
+template <int KSUB, bool F8, bool CLUSTER, int EPI_WARPS>
+__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, EPI_WARPS == 4 ? 3 : 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const GemmParams p) {
   // The A box holds only the rows that exist (a multiple of 8, so 1024-byte swizzle groups stay whole);
@@ -423,8 +510,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const int S = p.num_stages;
-  // barriers sit behind the ring and behind the span a short A box leaves readable (see smem_bytes_for)
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + (size_t)S * STAGE_BYTES + (BM * KBOX * 2 - A_BOX_BYTES));
+  // barriers sit behind the ring and behind the span a short A box leaves readable (see a_slack_bytes)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + (size_t)S * STAGE_BYTES + p.slack_bytes);
   // layout: full[S], empty[S], tmem_full[2], tmem_empty[2], then tmem base slot and abort flag
   const uint32_t bar_full = smem_u32(bars);
   const uint32_t bar_empty = bar_full + 8u * S;
@@ -432,15 +519,26 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t bar_tempty = bar_tfull + 16u;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  // CLUSTER: two more barriers (parts ready / parts read), then this CTA's partial tile
+  const uint32_t bar_ready = bar_tempty + 16u + 16u;
+  const uint32_t bar_free = bar_ready + 8u;
+  float* const part_buf = reinterpret_cast<float*>(bars + 2 * S + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_work = p.tiles_m * p.tiles_n * p.n_parts;
+  if (threadIdx.x == 0) RG_STAMP(0);                      // CTA entry
+  // Work items: (part, tile) for the plain kernel, walked by CTA; tiles for the CLUSTER kernel, walked by
+  // cluster, the CTA's rank in the cluster being its part.
+  const int crank = CLUSTER ? (int)cluster_ctarank() : 0;
+  const int total_work = CLUSTER ? p.tiles_m * p.tiles_n : p.tiles_m * p.tiles_n * p.n_parts;
+  const int work_first = CLUSTER ? (int)blockIdx.x / p.n_parts : (int)blockIdx.x;
+  const int work_step = CLUSTER ? (int)gridDim.x / p.n_parts : (int)gridDim.x;
 
   if (threadIdx.x == 0) {
     prefetch_tensormap(&tmap_a);
     prefetch_tensormap(&tmap_b);
     for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8u * s, 1); mbar_init(bar_empty + 8u * s, 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8u * b, 1); mbar_init(bar_tempty + 8u * b, NUM_EPI_WARPS); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8u * b, 1); mbar_init(bar_tempty + 8u * b, EPI_WARPS); }
+    if (CLUSTER) { mbar_init(bar_ready, EPI_WARPS * p.n_parts); mbar_init(bar_free, EPI_WARPS * p.n_parts); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -450,8 +548,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   }
   tcgen05_fence_before();
   __syncthreads();
+  if (CLUSTER) cluster_sync_all();                         // every CTA's barriers exist before any remote arrive
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) RG_STAMP(1);                      // set-up done
   // a split-K merge launched behind this kernel may be scheduled now; it still waits for this grid to finish
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // This kernel is itself launched with programmatic stream serialisation, so it may be running
@@ -472,17 +572,37 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       int stage = 0; uint32_t phase = 0;
       bool alive = true;
       bool deps_done = false;
-      for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
+      // Weights that nothing ahead in the stream writes (the caller's promise, `b_static`) need not wait for
+      // the kernels ahead: the B boxes of the first work item's first stages (the ring is empty, so at most
+      // S of them) go out at once, and only the A boxes of those stages wait for the dependency.
+      int prefetched = 0;
+      if (p.b_static && work_first < total_work) {
+        int part, tm, tn;
+        decode_work(p, work_first, part, tm, tn);
+        if (CLUSTER) part = crank;
+        const int k_begin = p.part_begin[part], k_end = p.part_end[part];
+        for (int k0 = k_begin; k0 < k_end && prefetched < S; k0 += KBOX * KSUB, ++prefetched) {
+          const uint32_t full = bar_full + 8u * prefetched;
+          if (lane == 0) mbar_expect_tx(full, STAGE_BYTES);
+          if (is_b) tma_load_2d(smem_base + prefetched * STAGE_BYTES + box_off, map, k0 + sub * KBOX, tn * BN, full);
+        }
+      }
+      int issued = 0;                                      // stages handed to the ring so far
+      for (int w = work_first; w < total_work && alive; w += work_step) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);
+        if (CLUSTER) part = crank;
         const int k_begin = p.part_begin[part], k_end = p.part_end[part];
         const int y = is_b ? tn * BN : tm * BM;
-        for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
-          if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, &g_status_word, 0x100u | stage)) { alive = false; break; }
+        for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB, ++issued) {
           const uint32_t full = bar_full + 8u * stage;
-          if (lane == 0) mbar_expect_tx(full, STAGE_BYTES);
-          if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
-          tma_load_2d(smem_base + stage * STAGE_BYTES + box_off, map, k0 + sub * KBOX, y, full);
+          const bool ahead = issued < prefetched;          // this stage's barrier is armed and its B boxes are on their way
+          if (!ahead) {
+            if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, &g_status_word, 0x100u | stage)) { alive = false; break; }
+            if (lane == 0) mbar_expect_tx(full, STAGE_BYTES);
+          }
+          if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; if (lane == 0) RG_STAMP(2); }
+          if (!ahead || !is_b) tma_load_2d(smem_base + stage * STAGE_BYTES + box_off, map, k0 + sub * KBOX, y, full);
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
       }
@@ -500,9 +620,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       int gc = 0;                                         // accumulators handed to the epilogue so far
       const uint64_t desc_a0 = make_kmajor_sw128_desc(smem_base);
       const uint64_t desc_b0 = make_kmajor_sw128_desc(smem_base + KSUB * A_BOX_BYTES);
-      for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
+      for (int w = work_first; w < total_work && alive; w += work_step) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);
+        if (CLUSTER) part = crank;
         const int k_begin = p.part_begin[part], k_end = p.part_end[part];
         // one accumulator per part, or one per group of inner_span k (a multiple of the K step)
         const int span = p.inner_span > 0 ? p.inner_span : (k_end - k_begin);
@@ -520,6 +641,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             group_end = k0 + span;
           }
           if (!warp_mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0x300u | stage)) { alive = false; break; }
+#ifdef RG_TIMELINE
+          if (leader && w == work_first && k0 == k_begin) RG_STAMP(3);   // first stage landed
+#endif
           tcgen05_fence_after();
           // descriptors differ from the stage-0 ones only in the 16-byte-unit start address (low word).
           // The operand kind is a template parameter: a run-time test in front of every step slowed
@@ -569,30 +693,90 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   } else {
     // ------------------------------------------------------------ epilogue warps
     const int quarter = warp & 3;                         // TMEM lanes [32*quarter, 32*quarter+32)
-    const int chunk0 = (warp - 2) >> 2;                   // this warp takes chunks chunk0, chunk0+2, ...
+    const int chunk0 = (warp - 2) >> 2;                   // this warp takes chunks chunk0, chunk0 + EPI_WARPS / 4, ...
+    constexpr int CHUNK_STEP = 32 * (EPI_WARPS / 4);
     bool alive = true;
     bool deps_done = false;
     int gc = 0;
-    for (int w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
+    for (int w = work_first; w < total_work && alive; w += work_step) {
       int part, tm, tn;
       decode_work(p, w, part, tm, tn);
+      if (CLUSTER) part = crank;
       // a 64-row step keeps rows 16q .. 16q+15 in the first 16 lanes of lane quarter q
       const int64_t row = p.mma_m == 64 ? (int64_t)(quarter * 16 + lane) : (int64_t)tm * BM + quarter * 32 + lane;
       const bool row_ok = row < p.M && (p.mma_m != 64 || lane < 16);
       const int klen = p.part_end[part] - p.part_begin[part];
       const int ngroups = p.inner_span > 0 ? (klen + p.inner_span - 1) / p.inner_span : 1;
-      if (ngroups == 1) {
+      if (CLUSTER) {
+        // ---- this CTA's part of the tile: tensor memory -> its shared-memory partial buffer
+        const int it = gc;                                  // tiles this cluster has finished
+        const int buf = gc & 1;
+        if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
+        tcgen05_fence_after();
+        if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
+        // the buffer still holds the previous tile's part until every CTA of the cluster has read its slice
+        if (it > 0 && !mbar_wait_cluster(bar_free, (uint32_t)(it - 1) & 1u, abort_flag, &g_status_word, 0x500u)) { alive = false; break; }
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
+        const int row_in_tile = p.mma_m == 64 ? quarter * 16 + lane : quarter * 32 + lane;
+        const int col_end = min(p.N, (tn + 1) * BN);
+#pragma unroll 1
+        for (int c0 = chunk0 * 32; c0 < BN; c0 += CHUNK_STEP) {
+          if (tn * BN + c0 >= col_end) break;               // uniform across the warp
+          uint32_t r[32];
+          tmem_ld_32x32b_x32(taddr + c0, r);
+          tmem_ld_wait();
+          if (row_ok) {
+            float4* dst = reinterpret_cast<float4*>(part_buf + (size_t)row_in_tile * p.part_ld + c0);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              if (c0 + 4 * q < BN)                          // the tile width is a multiple of 16, not of 32
+                dst[q] = make_float4(round_through(__uint_as_float(r[4 * q]), p.ws_dtype), round_through(__uint_as_float(r[4 * q + 1]), p.ws_dtype),
+                                     round_through(__uint_as_float(r[4 * q + 2]), p.ws_dtype), round_through(__uint_as_float(r[4 * q + 3]), p.ws_dtype));
+            }
+          }
+        }
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);  // the accumulator may be overwritten
+        ++gc;
+        // ---- tell every CTA of the cluster that this warp's share of the part is in place, wait for all shares
+        if (lane < p.n_parts) mbar_arrive_cluster(map_to_cta(bar_ready, (uint32_t)lane));
+        if (!mbar_wait_cluster(bar_ready, (uint32_t)it & 1u, abort_flag, &g_status_word, 0x600u)) { alive = false; break; }
+        // ---- merge this CTA's slice of the tile: groups of four columns, dealt to the CTAs in contiguous runs
+        {
+          const int tile_rows = min(p.part_rows, p.M - tm * BM);
+          const int c4s = BN >> 2;
+          const int units = tile_rows * c4s;
+          const int per = (units + p.n_parts - 1) / p.n_parts;
+          const int u_end = min(units, (crank + 1) * per);
+          const uint32_t part_local = smem_u32(part_buf);
+          for (int u = crank * per + (warp - 2) * 32 + lane; u < u_end; u += EPI_WARPS * 32) {
+            const int r_t = u / c4s, c4 = u - r_t * c4s;
+            const int col0 = tn * BN + 4 * c4;
+            if (col0 >= p.N) continue;
+            const uint32_t off = part_local + (uint32_t)(r_t * p.part_ld + 4 * c4) * 4u;
+            float4 v[8];
+#pragma unroll
+            for (int s2 = 0; s2 < 8; ++s2) if (s2 < p.n_parts) v[s2] = ld_cluster_f4(map_to_cta(off, (uint32_t)s2));
+            const float4 acc = p.merge_dtype == RG_F32 ? merge_upto8<false>(v, p.n_parts, p.tree, p.merge_dtype)
+                                                        : merge_upto8<true>(v, p.n_parts, p.tree, p.merge_dtype);
+            finish_and_store4(p.epi, p.C, p.ldc, p.c_dtype, p.N, (int64_t)tm * BM + r_t, col0, acc);
+          }
+        }
+        __syncwarp();
+        if (lane < p.n_parts) mbar_arrive_cluster(map_to_cta(bar_free, (uint32_t)lane));   // this warp no longer reads any CTA's part
+      } else if (ngroups == 1) {
         const int buf = gc & 1;
         if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
         tcgen05_fence_after();
         if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
-        epilogue_tile(p, BN, part, row, row_ok, tn, taddr, chunk0);
+        epilogue_tile(p, BN, part, row, row_ok, tn, taddr, chunk0, CHUNK_STEP);
         tcgen05_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
         ++gc;
-      } else {
+      } else if (EPI_WARPS == 8) {                          // the second cut level runs with eight epilogue warps only
         GroupedAcc acc;
         for (int g = 0; g < ngroups && alive; ++g, ++gc) {
           const int buf = gc & 1;
@@ -611,13 +795,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   }
 
   // ---------------------------------------------------------------- teardown
+  if (warp == 1 && lane == 0) RG_STAMP(4);                // last step issued
   __syncthreads();
+  if (threadIdx.x == 0) RG_STAMP(5);                      // all roles done
   if (*abort_flag) {
     // let copies and steps already in flight land before shared and tensor memory go away
     const uint64_t t0 = globaltimer_ns();
     while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
     __syncthreads();
   }
+  if (CLUSTER) cluster_sync_all();   // other CTAs may still be reading this CTA's part or arriving on its barriers
   if (warp == 1) {
     tcgen05_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
@@ -847,6 +1034,7 @@ struct FixupParams {
   int64_t ldw;
   int32_t M, N, S, tree;
   int32_t partial_dtype, merge_dtype;
+  int32_t launch_seq;     // the GEMM launch this merge belongs to (timeline stamps only)
   void* C;
   int64_t ldc;
   int32_t c_dtype;
@@ -865,7 +1053,13 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
   // still draining; nothing is read before that kernel has completed and flushed its stores.  A
   // kernel launched the same way behind this one may set itself up meanwhile.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#ifdef RG_TIMELINE
+  if (threadIdx.x == 0 && blockIdx.x < 512) g_timeline[p.launch_seq & 7][blockIdx.x][6] = globaltimer_ns();
+#endif
   asm volatile("griddepcontrol.wait;" ::: "memory");
+#ifdef RG_TIMELINE
+  if (threadIdx.x == 0 && blockIdx.x < 512) g_timeline[p.launch_seq & 7][blockIdx.x][7] = globaltimer_ns();
+#endif
   if (idx >= (int64_t)p.M * ncol4) return;
   const int64_t row = idx / ncol4;
   const int col0 = (int)(idx - row * ncol4) * 4;
@@ -1061,14 +1255,25 @@ bool cached_tmap(CUtensorMap* out, const void* ptr, int dtype, int64_t rows, int
 }
 
 constexpr size_t SMEM_LIMIT = 232448;   // 227 KiB of dynamic shared memory per CTA
+constexpr size_t SMEM_LIMIT_HALF = 115712;   // 113 KiB: two CTAs (and their 1 KiB system shares) fit the 228 KiB of an SM
+
+// The tensor-core step reads its full row count (128, or 64 for problems of at most 64 rows) from the start
+// of an A box even when the box holds fewer rows.  Inside a stage the surplus falls on the boxes behind it;
+// what the last A box of the last stage reads past the end of its stage must still lie inside the
+// allocation (those rows feed accumulator rows nobody stores).
+size_t a_slack_bytes(int bn, int ksub, int a_rows) {
+  const int span_rows = a_rows <= 64 ? 64 : BM;
+  const int64_t over = (int64_t)(span_rows - a_rows) * KBOX * 2 - (int64_t)ksub * bn * KBOX * 2;
+  return over > 0 ? (size_t)over : 0;
+}
 
 size_t smem_bytes_for(int bn, int ksub, int stages, int a_rows) {
   const size_t stage = (size_t)ksub * ((size_t)a_rows * KBOX * 2 + (size_t)bn * KBOX * 2);
-  // The tensor-core step reads 128 rows from the start of an A box even when the box holds fewer:
-  // keep that whole span inside the allocation (the extra rows feed accumulator rows nobody stores).
-  const size_t slack = (size_t)(BM - a_rows) * KBOX * 2;
-  return 1024 + stages * stage + slack + (2 * stages + 4) * 8 + 16;
+  return 1024 + stages * stage + a_slack_bytes(bn, ksub, a_rows) + (2 * stages + 4) * 8 + 16;
 }
+
+// CLUSTER kernels: two more barriers and the CTA's partial tile behind the plain kernel's layout
+size_t cluster_extra_bytes(int bn, int part_rows) { return 16 + (size_t)part_rows * (bn + 4) * 4; }
 
 size_t smem_bytes_for_pair(int bn, int ksub, int stages) {
   const size_t stage = (size_t)ksub * (BM * KBOX * 2 + (size_t)(bn / 2) * KBOX * 2);
@@ -1106,20 +1311,79 @@ cudaError_t launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const Gemm
 }
 
 template <int KSUB, bool F8>
+cudaError_t configure_cluster_kernel() {
+  static DeviceOnce configured;
+  const int dev = current_device().dev;
+  if (!configured.has(dev)) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<KSUB, F8, true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    if (e != cudaSuccess) return e;
+    configured.set(dev);
+  }
+  return cudaSuccess;
+}
+
+// The in-cluster split-K kernel: `clusters` clusters of p.n_parts CTAs, launched like the plain kernel
+// (programmatic stream serialisation: set-up overlaps the previous kernel's tail).
+template <int KSUB, bool F8>
+cudaError_t launch_cluster_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int clusters, cudaStream_t st) {
+  const size_t smem = smem_bytes_for(p.bn, KSUB, p.num_stages, (int)(p.a_box_bytes / (KBOX * 2))) + cluster_extra_bytes(p.bn, p.part_rows);
+  cudaError_t e = configure_cluster_kernel<KSUB, F8>();
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(clusters * p.n_parts), 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)p.n_parts; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<KSUB, F8, true, 8>, ta, tb, p);
+}
+
+// How many clusters of `csize` CTAs of the in-cluster kernel the device runs at once (each CTA takes a
+// whole SM, and a cluster must fit one GPC).  0 if such a cluster cannot be scheduled at all.
+template <int KSUB, bool F8>
+int query_clusters_t(int csize) {
+  if (configure_cluster_kernel<KSUB, F8>() != cudaSuccess) return 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(csize * 64), 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = SMEM_LIMIT;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<KSUB, F8, true, 8>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+  return n;
+}
+
+template <int KSUB, bool F8, int EPI_WARPS = 8>
 cudaError_t launch_one_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   const size_t smem = smem_bytes_for(p.bn, KSUB, p.num_stages, (int)(p.a_box_bytes / (KBOX * 2)));
   static DeviceOnce configured;
   const int dev = current_device().dev;
   if (!configured.has(dev)) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<KSUB, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<KSUB, F8, false, EPI_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(EPI_WARPS == 4 ? SMEM_LIMIT_HALF : SMEM_LIMIT));
     if (e != cudaSuccess) return e;
+    if (EPI_WARPS == 4) {
+      // two CTAs per SM: ask for the largest shared-memory carve-out
+      e = cudaFuncSetAttribute(gemm_tcgen05_kernel<KSUB, F8, false, EPI_WARPS>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+      if (e != cudaSuccess) return e;
+    }
     configured.set(dev);
   }
   // programmatic stream serialisation: the CTAs may set themselves up (barriers, tensor memory,
   // descriptor prefetch) while the kernel before this one in the stream drains
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid, 1, 1);
-  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.blockDim = dim3(64 + 32 * EPI_WARPS, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -1127,12 +1391,17 @@ cudaError_t launch_one_t(const CUtensorMap& ta, const CUtensorMap& tb, const Gem
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<KSUB, F8>, ta, tb, p);
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<KSUB, F8, false, EPI_WARPS>, ta, tb, p);
 }
 
 template <int KSUB>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   return p.f8 ? launch_one_t<KSUB, true>(ta, tb, p, grid, st) : launch_one_t<KSUB, false>(ta, tb, p, grid, st);
+}
+// the form that shares an SM between two CTAs (four epilogue warps, half the shared and tensor memory)
+template <int KSUB>
+cudaError_t launch_one_half(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
+  return p.f8 ? launch_one_t<KSUB, true, 4>(ta, tb, p, grid, st) : launch_one_t<KSUB, false, 4>(ta, tb, p, grid, st);
 }
 
 }  // namespace
@@ -1144,12 +1413,38 @@ bool make_operand_tmap(CUtensorMap_st* map, const void* ptr, int dtype, int64_t 
 
 int a_box_rows_for(int64_t M) { return M >= BM ? BM : (int)((M + 7) / 8 * 8); }
 
-int max_stages_for(int bn, int bk, int cta_group, int64_t M) {
+int cluster_part_rows(int64_t M) { return M >= BM ? BM : (int)M; }
+
+// cluster_merge: the in-cluster split-K kernel, whose partial tile shares the shared memory with the ring
+// (0 stages = it does not fit at all)
+int max_stages_for(int bn, int bk, int cta_group, int64_t M, bool cluster_merge, bool half_sm) {
   const int ksub = bk / KBOX;
   int s = 1;
   if (cta_group == 2) { while (s < 8 && smem_bytes_for_pair(bn, ksub, s + 1) <= SMEM_LIMIT) ++s; }
-  else { while (s < 32 && smem_bytes_for(bn, ksub, s + 1, a_box_rows_for(M)) <= SMEM_LIMIT) ++s; }
+  else {
+    const size_t limit = half_sm ? SMEM_LIMIT_HALF : SMEM_LIMIT;
+    const size_t extra = cluster_merge ? cluster_extra_bytes(bn, cluster_part_rows(M)) : 0;
+    if (smem_bytes_for(bn, ksub, 1, a_box_rows_for(M)) + extra > limit) return 0;
+    while (s < 32 && smem_bytes_for(bn, ksub, s + 1, a_box_rows_for(M)) + extra <= limit) ++s;
+  }
   return s;
+}
+
+// Clusters of `csize` CTAs of the in-cluster split-K kernel that run at once on the current device
+// (looked up once per device and cluster size).
+int max_active_clusters(int csize, int bk, bool f8) {
+  static std::mutex mu;
+  static int cache[64][9][2][2];                            // [device][csize][bk == 128][f8], value + 1
+  if (csize < 2 || csize > 8 || (bk != 64 && bk != 128)) return 0;
+  const int dev = current_device().dev;
+  std::lock_guard<std::mutex> lock(mu);
+  int* slot = (dev >= 0 && dev < 64) ? &cache[dev][csize][bk == 128][f8 ? 1 : 0] : nullptr;
+  if (slot && *slot) return *slot - 1;
+  int n;
+  if (bk == 128) n = f8 ? query_clusters_t<2, true>(csize) : query_clusters_t<2, false>(csize);
+  else n = f8 ? query_clusters_t<1, true>(csize) : query_clusters_t<1, false>(csize);
+  if (slot) *slot = n + 1;
+  return n;
 }
 
 rg_status_t read_and_clear_status(uint32_t* code) {
@@ -1165,6 +1460,12 @@ rg_status_t launch_wait_selftest(uint64_t limit_ns, uint32_t code, unsigned int*
   bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(limit_ns, code, left_early);
   return cudaGetLastError() == cudaSuccess ? RG_OK : RG_ERR_CUDA;
 }
+
+#ifdef RG_TIMELINE
+extern "C" int rg_debug_read_timeline(unsigned long long* host_out) {     // [8][512][8]
+  return cudaMemcpyFromSymbol(host_out, g_timeline, sizeof(g_timeline)) == cudaSuccess ? 0 : 1;
+}
+#endif
 
 // Launch the GEMM (and the merge when there are cuts).  All arguments were validated by the caller.
 rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
@@ -1191,9 +1492,12 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   p.raster = plan.raster;
   p.group_m = plan.group_m;
   p.a_box_bytes = (uint32_t)a_rows * KBOX * 2;
+  p.slack_bytes = pair ? 0u : (uint32_t)a_slack_bytes(plan.BN, plan.BK / KBOX, a_rows);
   p.bn = plan.BN;
   p.inner_span = plan.inner_span / kdiv;
   p.f8 = kind == KIND_F8E4M3;
+  p.b_static = plan.b_static;
+  { static std::atomic<int> seq{0}; p.launch_seq = seq.fetch_add(1, std::memory_order_relaxed); }
   // At most 64 rows: the 64-row step reads half the A rows from shared memory, which is what a narrow tile's
   // step time is made of ((rows + width) x 32 bytes at 128 bytes per clock).  Same products, same order.
   p.mma_m = (!pair && M <= 64) ? 64 : BM;
@@ -1205,12 +1509,15 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     e.bias = epi->bias; e.bias_dtype = epi->bias_dtype; e.act = epi->act;
     e.residual = epi->residual; e.residual_dtype = epi->residual_dtype; e.ldr = epi->ldr;
   }
-  const bool split = plan.n_parts > 1;
+  const bool in_cluster = plan.cluster_merge != 0;            // parts merged inside the GEMM kernel, no workspace
+  const bool split = plan.n_parts > 1 && !in_cluster;
   p.C = C->ptr; p.ldc = C->ld; p.c_dtype = C->dtype;
   p.ws = split ? ws : nullptr;
   p.ws_dtype = plan.partial_dtype;
   p.ldw = (N + 3) / 4 * 4;
   p.epi = split ? EpilogueArgs{} : e;
+  p.tree = plan.tree; p.merge_dtype = plan.merge_dtype;
+  p.part_rows = cluster_part_rows(M); p.part_ld = plan.BN + 4;
 
   const int64_t total = (int64_t)p.tiles_m * p.tiles_n * p.n_parts;
   const int sms = current_device().sms;
@@ -1224,6 +1531,20 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     else if (plan.BN == 128 && ksub == 1) err = launch_pair<128, 1>(ta, tb, p, grid, kind, st);
     else if (plan.BN == 128 && ksub == 2) err = launch_pair<128, 2>(ta, tb, p, grid, kind, st);
     else return RG_ERR_UNSUPPORTED;
+  } else if (in_cluster) {
+    const int avail = max_active_clusters(plan.n_parts, plan.BK, kind == KIND_F8E4M3);
+    if (avail < 1) return RG_ERR_UNSUPPORTED;
+    const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
+    const int clusters = (int)(tiles < avail ? tiles : avail);
+    if (ksub == 1) err = p.f8 ? launch_cluster_t<1, true>(ta, tb, p, clusters, st) : launch_cluster_t<1, false>(ta, tb, p, clusters, st);
+    else if (ksub == 2) err = p.f8 ? launch_cluster_t<2, true>(ta, tb, p, clusters, st) : launch_cluster_t<2, false>(ta, tb, p, clusters, st);
+    else return RG_ERR_UNSUPPORTED;
+  } else if (plan.half_sm) {
+    // one CTA per SM, each at half an SM's resources: the other half is where the next launch's CTAs set up
+    const int grid = (int)(total < sms ? total : sms);
+    if (ksub == 1) err = launch_one_half<1>(ta, tb, p, grid, st);
+    else if (ksub == 2) err = launch_one_half<2>(ta, tb, p, grid, st);
+    else return RG_ERR_UNSUPPORTED;
   } else {
     const int grid = (int)(total < sms ? total : sms);
     if (ksub == 1) err = launch_one<1>(ta, tb, p, grid, st);
@@ -1236,7 +1557,7 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   if (split) {
     FixupParams f;
     f.ws = ws; f.ldw = p.ldw; f.partial_dtype = plan.partial_dtype; f.merge_dtype = plan.merge_dtype;
-    f.M = p.M; f.N = p.N; f.S = plan.n_parts; f.tree = plan.tree;
+    f.M = p.M; f.N = p.N; f.S = plan.n_parts; f.tree = plan.tree; f.launch_seq = p.launch_seq;
     f.C = C->ptr; f.ldc = C->ld; f.c_dtype = C->dtype; f.epi = e;
     const int64_t items = M * ((N + 3) / 4);
     cudaLaunchConfig_t cfg = {};

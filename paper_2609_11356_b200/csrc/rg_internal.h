@@ -36,6 +36,9 @@ inline DeviceInfo current_device() {
 // A validated launch plan: speed knobs resolved, parts laid out.
 struct GemmPlan {
   int BN, BK, stages, raster, group_m, cta_group;
+  int b_static;             // caller's promise: nothing in flight on the stream writes B (its first boxes may be fetched early)
+  int half_sm;              // the one-CTA kernel in its half-SM form: two CTAs share an SM (weight-streaming shapes)
+  int cluster_merge;        // split-K parts merged inside the GEMM kernel by a thread-block cluster (no workspace, one launch)
   int n_parts, tree;
   int partial_dtype, merge_dtype;
   int inner_span;
@@ -43,7 +46,8 @@ struct GemmPlan {
   int32_t part_end[RG_MAX_CUTS + 1];
 };
 
-int max_stages_for(int bn, int bk, int cta_group, int64_t M);
+int max_stages_for(int bn, int bk, int cta_group, int64_t M, bool cluster_merge = false, bool half_sm = false);
+int max_active_clusters(int csize, int bk, bool f8);
 rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
                         const rg_epilogue_t* epi, void* ws, cudaStream_t st);
 rg_status_t launch_gemv(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,

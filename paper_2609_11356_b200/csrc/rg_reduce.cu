@@ -33,6 +33,14 @@ __device__ unsigned int g_reduce_status_word = 0;
 namespace {
 
 constexpr float NEG_ZERO = -0.0f;
+
+// Every kernel here is launched with programmatic stream serialisation: its CTAs may be scheduled while the
+// kernel ahead of it in the stream drains, and a kernel launched the same way behind it may be scheduled as
+// soon as all of this kernel's CTAs have started.  Nothing is read before the kernels ahead have completed.
+__device__ __forceinline__ void pdl_prologue() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
 constexpr int MAX_LEVELS = 13;          // super-blocks per row < 2^13
 
 enum : int { OP_SUM = 0, OP_RMS = 1, OP_SOFTMAX = 2 };
@@ -250,6 +258,7 @@ __global__ void __launch_bounds__(256) reduce_rows_warp_kernel(const ReduceParam
   const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   const int nsb = (int)((p.C + SBW - 1) / SBW);
+  pdl_prologue();
   for (int64_t row = warp0; row < p.R; row += nwarps) {
     const T* xr = static_cast<const T*>(p.x) + row * p.ldx;
     float stk[MAX_LEVELS];
@@ -298,6 +307,7 @@ __global__ void __launch_bounds__(1024) reduce_rows_cta_kernel(const ReduceParam
   constexpr int SBW = 32 * V * U;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int nsb = (int)((p.C + SBW - 1) / SBW);
+  pdl_prologue();
   for (int64_t row = blockIdx.x; row < p.R; row += gridDim.x) {
     const T* xr = static_cast<const T*>(p.x) + row * p.ldx;
     float shift = 0.0f;
@@ -364,21 +374,31 @@ __global__ void __launch_bounds__(1024) reduce_rows_cta_kernel(const ReduceParam
 // length is a multiple of V.
 template <typename T, int U>
 __global__ void __launch_bounds__(256) rmsnorm_keep_kernel(const ReduceParams p) {
-  __shared__ float sb[8];
+  __shared__ float sb[2][8];
   constexpr int V = VecTraits<T>::V;
   constexpr int WB = 32 * V;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const bool out_vec = rms_out_vec<T, true>(p);
-  for (int64_t row = blockIdx.x; row < p.R; row += gridDim.x) {
+  const int64_t base = (int64_t)warp * WB * U + lane * V;
+  const bool w_vec = p.weight && ((reinterpret_cast<uintptr_t>(p.weight) & 15) == 0) &&
+                     p.w_dtype == (sizeof(T) == 2 ? RG_BF16 : RG_F32);
+  pdl_prologue();
+  auto load_row = [&](int64_t row, uint4 (&raw)[U]) {
     const T* xr = static_cast<const T*>(p.x) + row * p.ldx;
-    const int64_t base = (int64_t)warp * WB * U + lane * V;
-    uint4 raw[U];
-    float bv[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int64_t c = base + (int64_t)u * WB;
       raw[u] = c + V <= p.C ? __ldg(reinterpret_cast<const uint4*>(xr + c)) : make_uint4(0, 0, 0, 0);
     }
+  };
+  uint4 raw[U], nxt[U];
+  if ((int64_t)blockIdx.x < p.R) load_row(blockIdx.x, raw);
+  int par = 0;
+  for (int64_t row = blockIdx.x; row < p.R; row += gridDim.x, par ^= 1) {
+    // the next row's vectors are requested now, so that they travel while this row is folded, scaled and stored
+    const bool more = row + gridDim.x < p.R;
+    if (more) load_row(row + gridDim.x, nxt);
+    float bv[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       float x[V];
@@ -393,13 +413,12 @@ __global__ void __launch_bounds__(256) rmsnorm_keep_kernel(const ReduceParams p)
     for (int s2 = 1; s2 < U; s2 <<= 1)
 #pragma unroll
       for (int u = 0; u < U; u += 2 * s2) bv[u] = f_add(bv[u], bv[u + s2]);
-    if (lane == 0) sb[warp] = bv[0];
-    __syncthreads();
-    float root = (lane < nwarps) ? sb[lane] : NEG_ZERO;   // nwarps <= 8 super-blocks, padded with the identity
+    if (lane == 0) sb[par][warp] = bv[0];
+    __syncthreads();                                      // one barrier per row: the totals alternate between two buffers
+    float root = (lane < nwarps) ? sb[par][lane] : NEG_ZERO;   // nwarps <= 8 super-blocks, padded with the identity
 #pragma unroll
     for (int off = 1; off < 8; off <<= 1) root = f_add(root, __shfl_xor_sync(0xffffffffu, root, off));
     root = __shfl_sync(0xffffffffu, root, 0);
-    __syncthreads();
     const float rinv = rms_rinv(root, p.C, p.eps);
     if (threadIdx.x == 0 && p.aux) p.aux[row] = rinv;
 #pragma unroll
@@ -408,8 +427,6 @@ __global__ void __launch_bounds__(256) rmsnorm_keep_kernel(const ReduceParams p)
       if (c + V > p.C) continue;
       float x[V], w[V], y[V];
       unpack<T>(raw[u], x);
-      const bool w_vec = p.weight && ((reinterpret_cast<uintptr_t>(p.weight) & 15) == 0) &&
-                         p.w_dtype == (sizeof(T) == 2 ? RG_BF16 : RG_F32);
       if (w_vec) unpack<T>(__ldg(reinterpret_cast<const uint4*>(static_cast<const T*>(p.weight) + c)), w);
       else {
 #pragma unroll
@@ -435,19 +452,35 @@ __global__ void __launch_bounds__(256) rmsnorm_keep_kernel(const ReduceParams p)
         }
       }
     }
+    if (more) {
+#pragma unroll
+      for (int u = 0; u < U; ++u) raw[u] = nxt[u];
+    }
   }
+}
+
+// Launch with programmatic stream serialisation (see pdl_prologue).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int threads, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3((unsigned)threads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 template <typename T, int OP, bool VEC, int U>
 cudaError_t launch_kernel(const ReduceParams& p, bool warp_rows, int threads, int grid, size_t smem, cudaStream_t st) {
   if constexpr (OP != OP_SOFTMAX) {
-    if (warp_rows) {
-      reduce_rows_warp_kernel<T, OP, VEC, U><<<grid, threads, 0, st>>>(p);
-      return cudaGetLastError();
-    }
+    if (warp_rows) return launch_pdl(reduce_rows_warp_kernel<T, OP, VEC, U>, grid, threads, 0, st, p);
   }
-  reduce_rows_cta_kernel<T, OP, VEC, U><<<grid, threads, smem, st>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(reduce_rows_cta_kernel<T, OP, VEC, U>, grid, threads, smem, st, p);
 }
 
 template <typename T, int OP, bool VEC>
@@ -494,9 +527,7 @@ rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_t
   }
   const int64_t nsb = (nblocks + U - 1) / U;
   if (nsb >= (1 << (MAX_LEVELS - 1))) return RG_ERR_UNSUPPORTED;   // rows beyond ~4M fp32 columns
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = current_device().sms;
 
   int threads = threads_hint;
   const bool valid_hint = threads == 32 || threads == 64 || threads == 128 || threads == 256 || threads == 512 || threads == 1024;
@@ -533,18 +564,17 @@ rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_t
   if (op == RG_OP_RMSNORM && !valid_hint && vec && C % V == 0 && nblocks <= 32) {
     const int Uk = nblocks >= 16 ? 4 : nblocks >= 4 ? 2 : 1;
     const int warps = (int)((nblocks + Uk - 1) / Uk);          // <= 8
-    const int64_t max_grid = (int64_t)sms * (2048 / (warps * 32));
-    const int grid = (int)(R < max_grid ? R : max_grid);
-    if (x->dtype == RG_BF16) {
-      if (Uk == 4) rmsnorm_keep_kernel<uint16_t, 4><<<grid, warps * 32, 0, st>>>(p);
-      else if (Uk == 2) rmsnorm_keep_kernel<uint16_t, 2><<<grid, warps * 32, 0, st>>>(p);
-      else rmsnorm_keep_kernel<uint16_t, 1><<<grid, warps * 32, 0, st>>>(p);
-    } else {
-      if (Uk == 4) rmsnorm_keep_kernel<float, 4><<<grid, warps * 32, 0, st>>>(p);
-      else if (Uk == 2) rmsnorm_keep_kernel<float, 2><<<grid, warps * 32, 0, st>>>(p);
-      else rmsnorm_keep_kernel<float, 1><<<grid, warps * 32, 0, st>>>(p);
-    }
-    return cudaGetLastError() == cudaSuccess ? RG_OK : RG_ERR_CUDA;
+    // every CTA takes the same number of rows (8192 rows on 2368 resident CTAs would leave a last round half
+    // empty: four rows each on 2048 CTAs instead)
+    void (*kern)(const ReduceParams);
+    if (x->dtype == RG_BF16) kern = Uk == 4 ? rmsnorm_keep_kernel<uint16_t, 4> : Uk == 2 ? rmsnorm_keep_kernel<uint16_t, 2> : rmsnorm_keep_kernel<uint16_t, 1>;
+    else kern = Uk == 4 ? rmsnorm_keep_kernel<float, 4> : Uk == 2 ? rmsnorm_keep_kernel<float, 2> : rmsnorm_keep_kernel<float, 1>;
+    int per_sm = 0;                                        // CTAs of this kernel an SM holds (registers decide)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, warps * 32, 0) != cudaSuccess || per_sm < 1) per_sm = 2048 / (warps * 32) / 2;
+    const int64_t max_grid = (int64_t)sms * per_sm;
+    const int64_t rows_per_cta = (R + max_grid - 1) / max_grid;
+    const int grid = (int)((R + rows_per_cta - 1) / rows_per_cta);
+    return launch_pdl(kern, grid, warps * 32, 0, st, p) == cudaSuccess ? RG_OK : RG_ERR_CUDA;
   }
   const int cap = (int)((nsb + 31) / 32 * 32);
   size_t smem = 0;
