@@ -93,9 +93,12 @@ typedef struct {
   uint32_t n_cuts;        /* split-K: number of interior cut points (0 = plain GEMM) */
   uint32_t cuts[RG_MAX_CUTS]; /* 0 < cuts[0] < ... < cuts[n_cuts-1] < K; part s = [cuts[s-1], cuts[s]) */
   uint32_t inner_span;    /* second level of the cut nest (Sec. 3.2.2; App. E per-group accumulation): 0 = none;
-                             else, inside every part, an accumulator is closed every inner_span k (a multiple
-                             of 64; of 128 with e4m3 operands) and the closed groups are added at fp32, in ascending order, into the
-                             part's running sum.  Order-deciding: part of the class key. */
+                             else, inside every part, an accumulator is closed every inner_span k (a multiple of the
+                             step width: 16, or 32 with e4m3 operands) and the closed groups are added at fp32, in
+                             ascending order, into the part's running sum.  inner_span = one step is the plan in
+                             which an instruction's result reaches the running sum in a rounding of its own
+                             (Sec. 3.2.2, `use_fast_accum` off; App. E, per-MMA accumulation).  Order-deciding:
+                             part of the class key. */
   uint8_t gemv_layout;    /* RG_ATOM_SCALAR only: how the 32 lanes of a warp deal the 8-wide k tiles of one output
                              element (Sec. 3.2.2 "GEMV", `layout`): 0 = strided (lane l takes tiles l, l+32, ...),
                              1 = contiguous (lane l takes the l-th run of ceil(tiles/32) tiles) */

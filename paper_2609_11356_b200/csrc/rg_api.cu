@@ -62,11 +62,10 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
   for (uint32_t i = 0; i < d->n_cuts; ++i)
     if (d->cuts[i] % step != 0) return RG_ERR_UNSUPPORTED;   // a cut may not split a step
   if (d->inner_span) {
-    // groups are handed over per pipeline stage (four steps) by one CTA, with the running sum in registers
-    if (d->inner_span % (4 * step) != 0) return RG_ERR_UNSUPPORTED;
-    if (d->cta_group == 2 || d->BM == 256 || d->BN > 128 || (d->BK != 0 && d->BK != 64)) return RG_ERR_UNSUPPORTED;
-    for (uint32_t i = 0; i < d->n_cuts; ++i)
-      if (d->cuts[i] % (4 * step) != 0) return RG_ERR_UNSUPPORTED;
+    // a group is a whole number of steps, down to a single one (an accumulator closed after every instruction:
+    // the two-rounding plan); groups are handed over by one CTA, the running sum lives in the epilogue warps' registers
+    if (d->inner_span % step != 0) return RG_ERR_UNSUPPORTED;
+    if (d->cta_group == 2 || d->BM == 256 || (d->BK != 0 && d->BK != 64)) return RG_ERR_UNSUPPORTED;
   }
   return RG_OK;
 }
@@ -195,7 +194,6 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
       for (int bn = 256; bn >= 32; bn -= 16) {
         if (d->BN && bn != d->BN) continue;
         if (group == 2 && bn != 256) continue;
-        if (d->inner_span && bn > 128) continue;
         const int64_t items = (group == 2 ? tiles_m2 : tiles_m) * ((N + bn - 1) / bn) * plan->n_parts;
         const int64_t slots = group == 2 ? sms / 2 : sms;
         const int64_t rounds = (items + slots - 1) / slots;
@@ -209,7 +207,6 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
     }
     if (plan->BN == 0) plan->BN = 64;
   }
-  if (d->inner_span && plan->BN > 128) plan->BN = 128;
   if (half && plan->BN > 128) plan->BN = 128;
   plan->cta_group = want_group ? want_group : 1;
   if (plan->cta_group == 2 && plan->BN < 128) plan->cta_group = 1;

@@ -386,14 +386,14 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, const int BN,
 // Second cut level (Sec. 3.2.2 "some kernels cut again inside a part"; App. E per-group accumulation):
 // the MMA warp closes an accumulator every inner_span k; each epilogue warp adds every closed group,
 // at fp32 and in ascending order, into a running sum held in registers, then finishes the tile from
-// it.  Tiles are at most 128 columns wide in this mode, so a warp owns at most two 32-column chunks.
-struct GroupedAcc { uint32_t v[2][32]; };
+// it.  A warp owns at most four 32-column chunks (tiles up to 256 columns wide).
+struct GroupedAcc { uint32_t v[4][32]; };
 
 __device__ __forceinline__ void grouped_add(const GemmParams& p, const int BN, int tn, uint32_t taddr, int chunk0, bool first,
                                             GroupedAcc& acc) {
   const int col_end = min(p.N, (tn + 1) * BN);
 #pragma unroll
-  for (int j = 0; j < 2; ++j) {
+  for (int j = 0; j < 4; ++j) {
     const int c0 = (chunk0 + 2 * j) * 32;
     if (c0 < BN && tn * BN + c0 < col_end) {              // uniform across the warp
       uint32_t r[32];
@@ -410,7 +410,7 @@ __device__ __forceinline__ void grouped_finish(const GemmParams& p, const int BN
                                                int chunk0, const GroupedAcc& acc) {
   const int col_end = min(p.N, (tn + 1) * BN);
 #pragma unroll
-  for (int j = 0; j < 2; ++j) {
+  for (int j = 0; j < 4; ++j) {
     const int c0 = (chunk0 + 2 * j) * 32;
     const int col0 = tn * BN + c0;
     if (c0 < BN && col0 < col_end && row_ok) epilogue_store_chunk(p, part, row, col0, min(32, col_end - col0), acc.v[j]);
@@ -490,7 +490,10 @@ __device__ __forceinline__ void finish_and_store4(const EpilogueArgs& e, void* C
 // chunk of its lane quarter): that form is launched with at most half an SM's shared memory and tensor memory, so
 // two CTAs share an SM, and the CTAs of the next launch in the stream can become resident, set themselves up and
 // fetch their first weight boxes while this launch's last CTAs finish (used for the weight-streaming shapes).
-template <int KSUB, bool F8, bool CLUSTER, int EPI_WARPS>
+// GROUPED: the second cut level (inner_span): accumulators closed inside a part and chained in the epilogue
+// warps' registers; an instantiation of its own, so that its 128 running-sum registers per thread are not
+// the plain kernel's problem.
+template <int KSUB, bool F8, bool CLUSTER, int EPI_WARPS, bool GROUPED = false>
 __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, EPI_WARPS == 4 ? 3 : 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const GemmParams p) {
@@ -626,12 +629,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         if (CLUSTER) part = crank;
         const int k_begin = p.part_begin[part], k_end = p.part_end[part];
         // one accumulator per part, or one per group of inner_span k (a multiple of the K step)
-        const int span = p.inner_span > 0 ? p.inner_span : (k_end - k_begin);
+        const int span = (GROUPED && p.inner_span > 0) ? p.inner_span : (k_end - k_begin);
         int group_end = k_begin;
         int buf = 0;
         uint32_t d_tmem = 0, accumulate = 0;
+        // groups that end inside a pipeline stage (a span that is not a multiple of the stage width, down to one
+        // instruction per accumulator: the two-rounding plan of Sec. 3.2.2 / App. E) take the step-by-step path below
+        const bool step_groups = GROUPED && p.inner_span > 0 && (p.inner_span % (KBOX * KSUB)) != 0;
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
-          if (k0 >= group_end) {
+          if (!step_groups && k0 >= group_end) {
             if (k0 > k_begin) { if (leader) umma_commit(bar_tfull + 8u * buf); ++gc; }   // the previous group is complete
             buf = gc & 1;
             if (!warp_mbar_wait(bar_tempty + 8u * buf, ((gc >> 1) & 1) ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
@@ -641,6 +647,37 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             group_end = k0 + span;
           }
           if (!warp_mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0x300u | stage)) { alive = false; break; }
+          if (step_groups) {
+            tcgen05_fence_after();
+            const uint64_t ad0 = desc_a0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
+            const uint64_t bd0 = desc_b0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
+#pragma unroll 1
+            for (int sa = 0; sa < KSUB * (KBOX / UMMA_K) && alive; ++sa) {
+              const int sub = sa / (KBOX / UMMA_K), a = sa % (KBOX / UMMA_K);
+              const int kk = k0 + sub * KBOX + a * UMMA_K;
+              if (kk >= k_end) break;                    // ascending k; nothing past the end of the part
+              if (kk >= group_end) {                     // this step opens a new accumulator
+                if (kk > k_begin) { if (leader) umma_commit(bar_tfull + 8u * buf); ++gc; }
+                buf = gc & 1;
+                if (!warp_mbar_wait(bar_tempty + 8u * buf, ((gc >> 1) & 1) ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
+                tcgen05_fence_after();
+                d_tmem = tmem_base + buf * ACC_STRIDE;
+                accumulate = 0;
+                group_end = kk + span;
+              }
+              const uint64_t ad = ad0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a;
+              const uint64_t bd = bd0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a;
+              if (leader) {
+                if (F8) umma_f8(d_tmem, ad, bd, IDESC, accumulate);
+                else umma_bf16(d_tmem, ad, bd, IDESC, accumulate);
+              }
+              accumulate = 1;
+            }
+            if (!alive) break;
+            if (leader) umma_commit(bar_empty + 8u * stage);
+            if (++stage == S) { stage = 0; phase ^= 1u; }
+            continue;
+          }
 #ifdef RG_TIMELINE
           if (leader && w == work_first && k0 == k_begin) RG_STAMP(3);   // first stage landed
 #endif
@@ -706,7 +743,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       const int64_t row = p.mma_m == 64 ? (int64_t)(quarter * 16 + lane) : (int64_t)tm * BM + quarter * 32 + lane;
       const bool row_ok = row < p.M && (p.mma_m != 64 || lane < 16);
       const int klen = p.part_end[part] - p.part_begin[part];
-      const int ngroups = p.inner_span > 0 ? (klen + p.inner_span - 1) / p.inner_span : 1;
+      const int ngroups = (GROUPED && p.inner_span > 0) ? (klen + p.inner_span - 1) / p.inner_span : 1;
       if (CLUSTER) {
         // ---- this CTA's part of the tile: tensor memory -> its shared-memory partial buffer
         const int it = gc;                                  // tiles this cluster has finished
@@ -765,7 +802,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         }
         __syncwarp();
         if (lane < p.n_parts) mbar_arrive_cluster(map_to_cta(bar_free, (uint32_t)lane));   // this warp no longer reads any CTA's part
-      } else if (ngroups == 1) {
+      } else if (!GROUPED) {
         const int buf = gc & 1;
         if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
         tcgen05_fence_after();
@@ -776,7 +813,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
         ++gc;
-      } else if (EPI_WARPS == 8) {                          // the second cut level runs with eight epilogue warps only
+      } else if (EPI_WARPS == 8) {                          // the second cut level runs with eight epilogue warps
         GroupedAcc acc;
         for (int g = 0; g < ngroups && alive; ++g, ++gc) {
           const int buf = gc & 1;
@@ -1394,6 +1431,30 @@ cudaError_t launch_one_t(const CUtensorMap& ta, const CUtensorMap& tb, const Gem
   return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<KSUB, F8, false, EPI_WARPS>, ta, tb, p);
 }
 
+// the second cut level: 64-wide stages, eight epilogue warps
+template <bool F8>
+cudaError_t launch_grouped_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
+  const size_t smem = smem_bytes_for(p.bn, 1, p.num_stages, (int)(p.a_box_bytes / (KBOX * 2)));
+  static DeviceOnce configured;
+  const int dev = current_device().dev;
+  if (!configured.has(dev)) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<1, F8, false, 8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    if (e != cudaSuccess) return e;
+    configured.set(dev);
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<1, F8, false, 8, true>, ta, tb, p);
+}
+
 template <int KSUB>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   return p.f8 ? launch_one_t<KSUB, true>(ta, tb, p, grid, st) : launch_one_t<KSUB, false>(ta, tb, p, grid, st);
@@ -1545,6 +1606,10 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     if (ksub == 1) err = launch_one_half<1>(ta, tb, p, grid, st);
     else if (ksub == 2) err = launch_one_half<2>(ta, tb, p, grid, st);
     else return RG_ERR_UNSUPPORTED;
+  } else if (plan.inner_span) {
+    if (ksub != 1) return RG_ERR_UNSUPPORTED;
+    const int grid = (int)(total < sms ? total : sms);
+    err = p.f8 ? launch_grouped_t<true>(ta, tb, p, grid, st) : launch_grouped_t<false>(ta, tb, p, grid, st);
   } else {
     const int grid = (int)(total < sms ? total : sms);
     if (ksub == 1) err = launch_one<1>(ta, tb, p, grid, st);

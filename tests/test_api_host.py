@@ -46,8 +46,20 @@ def test_validate_rules():
     assert rg.rg_desc_validate(rg.rg_desc(atom=K.RG_ATOM_TC_F8_K32), 64, 256, 512) == 2
     assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, cuts=(48,)), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, cuts=(64,)), 64, 256, 512) == 0
-    assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, inner_span=64), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, inner_span=48), 64, 256, 512) == 3     # not a whole number of 32-wide steps
+    assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, inner_span=32), 64, 256, 512) == 0     # one step per accumulator
     assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, inner_span=128), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(inner_span=16), 64, 256, 512) == 0                            # the two-rounding plan
+    assert rg.rg_desc_validate(rg.rg_desc(inner_span=8), 64, 256, 512) == 3                             # half a step
+    assert rg.rg_desc_validate(rg.rg_desc(inner_span=16, BK=128), 64, 256, 512) == 3
+    # speed knobs and promises that are not order fields
+    assert rg.rg_desc_validate(rg.rg_desc(cuts=(256,), split_merge=2), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(split_merge=2), 64, 256, 512) == 3                            # nothing to merge
+    assert rg.rg_desc_validate(rg.rg_desc(cuts=(256,), split_merge=3), 64, 256, 512) == 2
+    assert rg.rg_desc_validate(rg.rg_desc(sm_share=2), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(sm_share=2, BN=256), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(b_static=1), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(b_static=2), 64, 256, 512) == 2
     assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, partial_dtype=K.RG_F8E4M3), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(in_dtype=4), 64, 256, 512) == 2
     assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16), 64, 256, 512) == 0
@@ -72,7 +84,8 @@ def test_class_key_holds_order_fields_only():
     k = rg.rg_desc_class(base)
     assert k != 0
     # speed knobs do not move the class (Sec. 3.2.2)
-    for kw in (dict(BN=64), dict(BN=256, BK=128), dict(stages=2), dict(raster=1), dict(BM=128), dict(BM=256), dict(cta_group=2)):
+    for kw in (dict(BN=64), dict(BN=256, BK=128), dict(stages=2), dict(raster=1), dict(BM=128), dict(BM=256), dict(cta_group=2),
+               dict(split_merge=1), dict(split_merge=2), dict(sm_share=2), dict(b_static=1)):
         assert rg.rg_desc_class(rg.rg_desc(cuts=(1792, 3584), **kw)) == k
     # every order-deciding field does
     others = [rg.rg_desc(cuts=(1792,)), rg.rg_desc(cuts=(1792, 3600)), rg.rg_desc(),

@@ -18,7 +18,7 @@ def _case(g):
     K = int(g.choice([64, 192, 576, 1000, 1024, 2048]))
     f16 = bool(g.integers(0, 2))
     nest = bool(g.integers(0, 3) == 0)
-    step = 64 if nest else 16
+    step = 16
     ncut = int(g.integers(0, 5))
     pts = sorted(set(int(x) * step for x in g.integers(1, max(2, K // step), ncut) if 0 < int(x) * step < K))
     desc = dict(cuts=tuple(pts), tree=int(g.integers(0, 2)))
@@ -26,8 +26,8 @@ def _case(g):
     desc.update(partial_dtype=pd, merge_dtype=md)
     knobs = {}
     if nest:
-        desc["inner_span"] = int(g.choice([64, 128, 320]))
-        knobs = [dict(), dict(BN=64), dict(BN=96, stages=2)][int(g.integers(0, 3))]
+        desc["inner_span"] = int(g.choice([16, 48, 64, 128, 320]))
+        knobs = [dict(), dict(BN=64), dict(BN=96, stages=2), dict(BN=256)][int(g.integers(0, 4))]
     else:
         knobs = [dict(), dict(BN=64, BK=128), dict(cta_group=2, BN=128), dict(cta_group=2, BN=256, BK=64), dict(BN=48, cta_group=1),
                  dict(BN=208, cta_group=1, raster=1), dict(BN=128, BK=256, cta_group=1, stages=1)][int(g.integers(0, 7))]
@@ -107,14 +107,14 @@ def test_random_fp8_descriptor_matches_oracle(seed):
     M = int(g.choice([1, 7, 33, 64, 65, 129, 200, 300])); N = int(g.choice([8, 40, 130, 256, 328]))
     K = int(g.choice([64, 190, 576, 1000, 1024, 2048]))
     nest = bool(g.integers(0, 3) == 0)
-    step = 128 if nest else 32
+    step = 32
     pts = sorted(set(int(x) * step for x in g.integers(1, max(2, K // step), int(g.integers(0, 5))) if 0 < int(x) * step < K))
     desc = dict(cuts=tuple(pts), tree=int(g.integers(0, 2)))
     pd, md = [(rgo.F32, rgo.F32), (rgo.BF16, rgo.F32), (rgo.BF16, rgo.BF16), (rgo.F16, rgo.F16)][int(g.integers(0, 4))]
     desc.update(partial_dtype=pd, merge_dtype=md)
     if nest:
-        desc["inner_span"] = int(g.choice([128, 256, 640]))
-        knobs = [dict(), dict(BN=64), dict(BN=96, stages=2)][int(g.integers(0, 3))]
+        desc["inner_span"] = int(g.choice([32, 96, 128, 256, 640]))
+        knobs = [dict(), dict(BN=64), dict(BN=96, stages=2), dict(BN=256)][int(g.integers(0, 4))]
     else:
         knobs = [dict(), dict(BN=64, BK=128), dict(cta_group=2, BN=128), dict(cta_group=2, BN=256, BK=64), dict(BN=48, cta_group=1),
                  dict(BN=208, cta_group=1, raster=1)][int(g.integers(0, 6))]

@@ -391,8 +391,8 @@ def test_inner_span_groups_bit_exact():
     assert gpu_gemm(ab, ones, out_dtype=rgo.F32, inner_span=64)[0, 0] == np.float32(1 + 2.0 ** -23)   # second group sums to 2^-23 first
     for M, N, K, cuts in ((70, 200, 1024, ()), (300, 130, 1000, ()), (33, 260, 2048, (512, 1024, 1536)), (129, 64, 4096, (2048,))):
         for name, A, B in _draws(M, N, K, 90 + K):
-            for span in (64, 128, 448):
-                for knobs in (dict(), dict(BN=64), dict(BN=112, stages=2)):
+            for span in (16, 48, 64, 80, 128, 448):         # 16 = an accumulator per instruction (the two-rounding plan)
+                for knobs in (dict(), dict(BN=64), dict(BN=112, stages=2), dict(BN=256), dict(BN=208, raster=1)):
                     got = gpu_gemm(A, B, cuts=cuts, inner_span=span, out_dtype=rgo.F32, **knobs)
                     want = rgo.gemm(A, B, cuts=cuts, inner_span=span, atom_model=HW, out_dtype=rgo.F32)
                     assert_bits_equal(got, want, f"{M}x{N}x{K} {name} span={span} {knobs}")
@@ -403,6 +403,6 @@ def test_inner_span_groups_bit_exact():
                       "nest with fused epilogue")
     k0 = rg.rg_desc_class(rg.rg_desc()); k1 = rg.rg_desc_class(rg.rg_desc(inner_span=64)); k2 = rg.rg_desc_class(rg.rg_desc(inner_span=128))
     assert len({k0, k1, k2}) == 3
-    for bad in (dict(inner_span=48), dict(inner_span=64, cta_group=2), dict(inner_span=64, BN=256), dict(inner_span=64, BK=128)):
+    for bad in (dict(inner_span=40), dict(inner_span=8), dict(inner_span=64, cta_group=2), dict(inner_span=64, BK=128)):
         assert rg.rg_desc_validate(rg.rg_desc(**bad), 64, 256, 512) == 3
     assert rg.rg_device_status() == 0

@@ -60,7 +60,7 @@ def test_split_partials_epilogue_outputs_and_class():
 
 def test_inner_span_groups_bit_exact():
     A, B = list(_draws(50, 96, 1536, 9))[1][1:]
-    for cuts, span in (((), 128), ((512, 1024), 256), ((768,), 384)):
+    for cuts, span in (((), 128), ((512, 1024), 256), ((768,), 384), ((), 32), ((512, 1024), 96), ((), 160)):   # 32 = one step per accumulator
         want = rgo.gemm(A, B, cuts=cuts, inner_span=span, atom_model=HW8, out_dtype=rgo.F32)
         assert_bits_equal(gpu_gemm(A, B, cuts=cuts, inner_span=span, out_dtype=rgo.F32), want, f"fp8 inner_span {span} cuts {cuts}")
 

@@ -397,3 +397,29 @@ def test_inner_span_worked_example_and_closed_forms():
     # group sums against the definition: chain of group results, each an unsplit GEMM of its own range
     g = [rgo.gemm(A[:, k:k + 128], B[:, k:k + 128], out_dtype=rgo.F32) for k in range(0, 512, 128)]
     assert np.array_equal(rgo.gemm(A, B, inner_span=128, out_dtype=rgo.F32), ((g[0] + g[1]) + g[2]) + g[3])
+
+
+def test_one_step_groups_are_separately_rounded_steps_chained_at_fp32():
+    """inner_span = one step (Sec. 3.2.2, `use_fast_accum` off; App. E, per-instruction accumulation): every
+    instruction's result is formed from a zero accumulator and reaches the running sum in a rounding of its
+    own.  Spelled out from the pinned pieces: one step from zero (`rgo.atom`), then one fp32 add."""
+    g = np.random.default_rng(16)
+    for model, width, draw in ((rgo.TCGEN05_BF16_B200, 16, "bf16"), (rgo.EXACT_RN, 16, "bf16"), (_with_k32(rgo.TCGEN05_F8E4M3_B200), 32, "e4m3")):
+        K = 7 * width + width // 2                                     # a short last step
+        x = (g.standard_normal((3, K)) * np.exp2(g.integers(-5, 6, (3, K)))).astype(np.float32)
+        y = (g.standard_normal((2, K)) * np.exp2(g.integers(-5, 6, (2, K)))).astype(np.float32)
+        A, B = (_bf(x), _bf(y)) if draw == "bf16" else (synth.f32_to_f8e4m3_bits(np.clip(x, -448, 448)), synth.f32_to_f8e4m3_bits(np.clip(y, -448, 448)))
+        for span_steps in (1, 2, 3):
+            got = rgo.gemm(A, B, atom_model=model, out_dtype=rgo.F32, inner_span=span_steps * width)
+            for i in range(3):
+                for j in range(2):
+                    run = None
+                    for k0 in range(0, K, span_steps * width):
+                        acc = np.float32(0.0)
+                        for s0 in range(k0, min(K, k0 + span_steps * width), width):   # the steps of one group, chained in the accumulator
+                            acc = rgo.atom(model, acc, A[i, s0:s0 + width], B[j, s0:s0 + width])
+                        run = acc if run is None else rgo.add_f32(run, acc)           # the group reaches the running sum rounded
+                    assert got[i, j] == run, (draw, span_steps, i, j)
+        # and it is a different sum from the single chain
+        assert not np.array_equal(rgo.gemm(A, B, atom_model=model, out_dtype=rgo.F32, inner_span=width),
+                                  rgo.gemm(A, B, atom_model=model, out_dtype=rgo.F32))
