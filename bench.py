@@ -294,7 +294,14 @@ def run_ours(args):
         d8 = rg.rg_desc(in_dtype=rg.RG_F8E4M3)
         c8 = torch.empty_like(T["sq_C"])        # own outputs: the step's results are checked further down
         ms8 = timed(lambda: rg.rg_gemm(d8, A8, B8, c8), 10)
-        del A8, B8, c8
+        del A8, B8
+        # the second cut level on the square problem: an accumulator closed every 64 k, and after every instruction
+        span_tflops = {}
+        for span in (64, 16):
+            dn = rg.rg_desc(inner_span=span)
+            msn = timed(lambda: rg.rg_gemm(dn, T["sq_A"], T["sq_B"], c8), 3)
+            span_tflops[str(span)] = round(2.0 * 8192 ** 3 / (msn * 1e-3) / 1e12, 1)
+        del c8
         cd = torch.empty_like(T["dc_C"])
         Ws = [T["dc_W"]] + [synth.device_normal((4096, 14336), 0.02, seed0 + 30 + i, bf, dev) for i in range(3)]
         it = [0]
@@ -340,6 +347,7 @@ def run_ours(args):
             "batch_sweep_n4096_k4096_us_by_m": sweep_us, "batch_sweep_torch_cublas_us_by_m": sweep_torch_us,
             "note": "timed alone after the step loop; weights of the two decode paths rotate over four copies (above L2)",
             "fp8_e4m3_square_tflops": round(2.0 * 8192 ** 3 / (ms8 * 1e-3) / 1e12, 1),
+            "square_tflops_by_inner_span": span_tflops,
             "decode_splitk8_back_to_back_us": round(ms_dec * 1e3, 2), "decode_splitk8_weight_gbs": round(wbytes / (ms_dec * 1e-3) / 1e9, 1),
             "gemv_m1_back_to_back_us": round(ms_gemv * 1e3, 2), "gemv_m1_weight_gbs": round(wbytes / (ms_gemv * 1e-3) / 1e9, 1),
             "col_sum_65536x32768_gbs": round(4.0 * RED_R * RED_C / (ms_col * 1e-3) / 1e9, 1),

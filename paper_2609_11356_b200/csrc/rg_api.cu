@@ -63,9 +63,9 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
     if (d->cuts[i] % step != 0) return RG_ERR_UNSUPPORTED;   // a cut may not split a step
   if (d->inner_span) {
     // a group is a whole number of steps, down to a single one (an accumulator closed after every instruction:
-    // the two-rounding plan); groups are handed over by one CTA, the running sum lives in the epilogue warps' registers
+    // the two-rounding plan); the running sum lives in the epilogue warps' registers; 64-wide stages
     if (d->inner_span % step != 0) return RG_ERR_UNSUPPORTED;
-    if (d->cta_group == 2 || d->BM == 256 || (d->BK != 0 && d->BK != 64)) return RG_ERR_UNSUPPORTED;
+    if (d->BK != 0 && d->BK != 64) return RG_ERR_UNSUPPORTED;
   }
   return RG_OK;
 }
@@ -176,8 +176,7 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   }
   // one CTA per 128-row tile, or a pair of CTAs (two SMs) per 256-row tile
   int want_group = 0;
-  if (d->inner_span) want_group = 1;
-  else if (d->cta_group) want_group = d->cta_group;
+  if (d->cta_group) want_group = d->cta_group;
   else if (d->BM == 256) want_group = 2;
   else if (d->BM == 128) want_group = 1;
   if (plan->BN == 0 || (want_group == 0 && !skinny)) {

@@ -858,7 +858,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 //   empty[s]  in each CTA; tcgen05.commit arrives on both
 //   tfull[b]  in each CTA; tcgen05.commit arrives on both
 //   tempty[b] in the even CTA; the epilogue warps of both CTAs arrive on it
-template <int BN, int KSUB, int KIND>
+// GROUPED: the second cut level on the pair (see the one-CTA kernel): the issuing CTA closes an accumulator
+// every inner_span k, the epilogue warps of both CTAs chain the closed groups in registers.
+template <int BN, int KSUB, int KIND, bool GROUPED = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                          const GemmParams p) {
@@ -954,7 +956,47 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
           alo[g][i] = (uint32_t)desc_a0 + off + (((i / (KBOX / UMMA_K)) * A_BOX_BYTES) >> 4);
           blo[g][i] = (uint32_t)desc_b0 + off + (((i / (KBOX / UMMA_K)) * B_BOX_BYTES) >> 4);
         }
-      for (int w = pair_id; w < total_work && alive; w += num_pairs, ++it) {
+      if (GROUPED) {
+        // step by step: a step that reaches the end of its group closes the accumulator and opens the other one
+        int gc = 0;                                       // accumulators handed to the epilogue so far
+        for (int w = pair_id; w < total_work && alive; w += num_pairs) {
+          int part, tm, tn;
+          decode_work(p, w, part, tm, tn);
+          const int k_begin = p.part_begin[part], k_end = p.part_end[part];
+          const int span = p.inner_span > 0 ? p.inner_span : (k_end - k_begin);
+          int group_end = k_begin, buf = 0;
+          uint32_t d_tmem = 0, accumulate = 0;
+          for (int k0 = k_begin; k0 < k_end && alive; k0 += KBOX * KSUB) {
+            if (!warp_mbar_wait(bar_full + 8u * stage, phase, abort_flag, &g_status_word, 0xb00u | stage)) { alive = false; break; }
+            tcgen05_fence_after();
+            const uint64_t adesc0 = desc_a0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
+            const uint64_t bdesc0 = desc_b0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
+#pragma unroll 1
+            for (int sa = 0; sa < KSUB * (KBOX / UMMA_K); ++sa) {
+              const int sub = sa / (KBOX / UMMA_K), a = sa % (KBOX / UMMA_K);
+              const int kk = k0 + sub * KBOX + a * UMMA_K;
+              if (kk >= k_end) break;
+              if (kk >= group_end) {
+                if (kk > k_begin) { if (leader) umma_commit_pair(bar_tfull + 8u * buf); ++gc; }
+                buf = gc & 1;
+                if (!warp_mbar_wait(bar_tempty + 8u * buf, ((gc >> 1) & 1) ^ 1u, abort_flag, &g_status_word, 0xa00u | buf)) { alive = false; break; }
+                tcgen05_fence_after();
+                d_tmem = tmem_base + buf * BN;
+                accumulate = 0;                            // every part and every group starts from zero
+                group_end = kk + span;
+              }
+              if (leader) umma_pair<KIND>(d_tmem, adesc0 + (uint64_t)((sub * A_BOX_BYTES) >> 4) + 2u * a,
+                                          bdesc0 + (uint64_t)((sub * B_BOX_BYTES) >> 4) + 2u * a, IDESC, accumulate);
+              accumulate = 1;
+            }
+            if (!alive) break;
+            if (leader) umma_commit_pair(bar_empty + 8u * stage);
+            if (++stage == S) { stage = 0; phase ^= 1u; }
+          }
+          if (alive) { if (leader) umma_commit_pair(bar_tfull + 8u * buf); ++gc; }
+        }
+      }
+      for (int w = pair_id; !GROUPED && w < total_work && alive; w += num_pairs, ++it) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);
         const int k_begin = p.part_begin[part], k_end = p.part_end[part];
@@ -1035,7 +1077,29 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     const uint32_t tempty_leader = map_to_cta(bar_tempty, 0);
     bool alive = true;
     int it = 0;
-    for (int w = pair_id; w < total_work && alive; w += num_pairs, ++it) {
+    if (GROUPED) {
+      int gc = 0;
+      for (int w = pair_id; w < total_work && alive; w += num_pairs) {
+        int part, tm, tn;
+        decode_work(p, w, part, tm, tn);
+        const int klen = p.part_end[part] - p.part_begin[part];
+        const int ngroups = p.inner_span > 0 ? (klen + p.inner_span - 1) / p.inner_span : 1;
+        const int64_t row = (int64_t)tm * 2 * BM + (int64_t)rank * BM + quarter * 32 + lane;
+        GroupedAcc acc;
+        for (int g = 0; g < ngroups && alive; ++g, ++gc) {
+          const int buf = gc & 1;
+          if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0xc00u | buf)) { alive = false; break; }
+          tcgen05_fence_after();
+          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
+          grouped_add(p, BN, tn, taddr, chunk0, g == 0, acc);
+          tcgen05_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(tempty_leader + 8u * buf);
+        }
+        if (alive) grouped_finish(p, BN, part, row, row < p.M, tn, chunk0, acc);
+      }
+    }
+    for (int w = pair_id; !GROUPED && w < total_work && alive; w += num_pairs, ++it) {
       int part, tm, tn;
       decode_work(p, w, part, tm, tn);
       const int buf = it & 1;
@@ -1317,13 +1381,13 @@ size_t smem_bytes_for_pair(int bn, int ksub, int stages) {
   return 1024 + stages * stage + (2 * stages + 4) * 8 + 16;
 }
 
-template <int BN, int KSUB, int KIND>
+template <int BN, int KSUB, int KIND, bool GROUPED = false>
 cudaError_t launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   const size_t smem = smem_bytes_for_pair(BN, KSUB, p.num_stages);
   static DeviceOnce configured;
   const int dev = current_device().dev;
   if (!configured.has(dev)) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_pair_kernel<BN, KSUB, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_pair_kernel<BN, KSUB, KIND, GROUPED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
     if (e != cudaSuccess) return e;
     configured.set(dev);
   }
@@ -1337,7 +1401,15 @@ cudaError_t launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tb, const Ge
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_pair_kernel<BN, KSUB, KIND>, ta, tb, p);
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_pair_kernel<BN, KSUB, KIND, GROUPED>, ta, tb, p);
+}
+
+// the second cut level on the pair: 64-wide stages
+template <int BN>
+cudaError_t launch_pair_grouped(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, int kind, cudaStream_t st) {
+  if (kind == KIND_F16) return launch_pair_t<BN, 1, KIND_F16, true>(ta, tb, p, grid, st);
+  if (kind == KIND_F8E4M3) return launch_pair_t<BN, 1, KIND_F8E4M3, true>(ta, tb, p, grid, st);
+  return launch_pair_t<BN, 1, KIND_BF16, true>(ta, tb, p, grid, st);
 }
 
 template <int BN, int KSUB>
@@ -1587,7 +1659,13 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   if (pair) {
     const int64_t pairs = sms / 2;
     const int grid = 2 * (int)(total < pairs ? total : pairs);
-    if (plan.BN == 256 && ksub == 1) err = launch_pair<256, 1>(ta, tb, p, grid, kind, st);
+    if (plan.inner_span) {
+      if (ksub != 1) return RG_ERR_UNSUPPORTED;
+      if (plan.BN == 256) err = launch_pair_grouped<256>(ta, tb, p, grid, kind, st);
+      else if (plan.BN == 128) err = launch_pair_grouped<128>(ta, tb, p, grid, kind, st);
+      else return RG_ERR_UNSUPPORTED;
+    }
+    else if (plan.BN == 256 && ksub == 1) err = launch_pair<256, 1>(ta, tb, p, grid, kind, st);
     else if (plan.BN == 256 && ksub == 2) err = launch_pair<256, 2>(ta, tb, p, grid, kind, st);
     else if (plan.BN == 128 && ksub == 1) err = launch_pair<128, 1>(ta, tb, p, grid, kind, st);
     else if (plan.BN == 128 && ksub == 2) err = launch_pair<128, 2>(ta, tb, p, grid, kind, st);

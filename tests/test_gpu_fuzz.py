@@ -27,7 +27,7 @@ def _case(g):
     knobs = {}
     if nest:
         desc["inner_span"] = int(g.choice([16, 48, 64, 128, 320]))
-        knobs = [dict(), dict(BN=64), dict(BN=96, stages=2), dict(BN=256)][int(g.integers(0, 4))]
+        knobs = [dict(), dict(BN=64), dict(BN=96, stages=2), dict(BN=256), dict(cta_group=2, BN=128), dict(cta_group=2, BN=256)][int(g.integers(0, 6))]
     else:
         knobs = [dict(), dict(BN=64, BK=128), dict(cta_group=2, BN=128), dict(cta_group=2, BN=256, BK=64), dict(BN=48, cta_group=1),
                  dict(BN=208, cta_group=1, raster=1), dict(BN=128, BK=256, cta_group=1, stages=1)][int(g.integers(0, 7))]
@@ -114,7 +114,7 @@ def test_random_fp8_descriptor_matches_oracle(seed):
     desc.update(partial_dtype=pd, merge_dtype=md)
     if nest:
         desc["inner_span"] = int(g.choice([32, 96, 128, 256, 640]))
-        knobs = [dict(), dict(BN=64), dict(BN=96, stages=2), dict(BN=256)][int(g.integers(0, 4))]
+        knobs = [dict(), dict(BN=64), dict(BN=96, stages=2), dict(BN=256), dict(cta_group=2, BN=128), dict(cta_group=2, BN=256)][int(g.integers(0, 6))]
     else:
         knobs = [dict(), dict(BN=64, BK=128), dict(cta_group=2, BN=128), dict(cta_group=2, BN=256, BK=64), dict(BN=48, cta_group=1),
                  dict(BN=208, cta_group=1, raster=1)][int(g.integers(0, 6))]

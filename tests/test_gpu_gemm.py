@@ -392,7 +392,8 @@ def test_inner_span_groups_bit_exact():
     for M, N, K, cuts in ((70, 200, 1024, ()), (300, 130, 1000, ()), (33, 260, 2048, (512, 1024, 1536)), (129, 64, 4096, (2048,))):
         for name, A, B in _draws(M, N, K, 90 + K):
             for span in (16, 48, 64, 80, 128, 448):         # 16 = an accumulator per instruction (the two-rounding plan)
-                for knobs in (dict(), dict(BN=64), dict(BN=112, stages=2), dict(BN=256), dict(BN=208, raster=1)):
+                for knobs in (dict(), dict(BN=64), dict(BN=112, stages=2), dict(BN=256), dict(BN=208, raster=1),
+                              dict(cta_group=2, BN=256), dict(cta_group=2, BN=128, stages=3)):
                     got = gpu_gemm(A, B, cuts=cuts, inner_span=span, out_dtype=rgo.F32, **knobs)
                     want = rgo.gemm(A, B, cuts=cuts, inner_span=span, atom_model=HW, out_dtype=rgo.F32)
                     assert_bits_equal(got, want, f"{M}x{N}x{K} {name} span={span} {knobs}")
@@ -401,8 +402,16 @@ def test_inner_span_groups_bit_exact():
     bias = synth.uniform_bf16((300,), -0.1, 0.1, 3)
     assert_bits_equal(gpu_gemm(A, B, inner_span=192, bias=bias, act=1), rgo.gemm(A, B, inner_span=192, atom_model=HW, bias=bias, act=1),
                       "nest with fused epilogue")
+    # a problem large enough for the default plan to take the two-SM kernel, on sampled outputs
+    Ab = synth.normal_bf16((2304, 1024), 1.0, 5); Bb = synth.normal_bf16((2560, 1024), 1.0, 6)
+    gsi = np.random.default_rng(7)
+    si, sj = gsi.integers(0, 2304, 600), gsi.integers(0, 2560, 600)
+    for span in (16, 64, 192):
+        got = gpu_gemm(Ab, Bb, inner_span=span, out_dtype=rgo.F32)
+        assert_bits_equal(got[si, sj], rgo.gemm_samples(Ab, Bb, si, sj, inner_span=span, atom_model=HW, out_dtype=rgo.F32), f"large, span {span}")
+        assert_bits_equal(gpu_gemm(Ab, Bb, inner_span=span, out_dtype=rgo.F32, cta_group=1, BN=128), got, f"large, span {span}: one-CTA kernel agrees")
     k0 = rg.rg_desc_class(rg.rg_desc()); k1 = rg.rg_desc_class(rg.rg_desc(inner_span=64)); k2 = rg.rg_desc_class(rg.rg_desc(inner_span=128))
     assert len({k0, k1, k2}) == 3
-    for bad in (dict(inner_span=40), dict(inner_span=8), dict(inner_span=64, cta_group=2), dict(inner_span=64, BK=128)):
+    for bad in (dict(inner_span=40), dict(inner_span=8), dict(inner_span=64, BK=128), dict(inner_span=64, cta_group=2, BK=128)):
         assert rg.rg_desc_validate(rg.rg_desc(**bad), 64, 256, 512) == 3
     assert rg.rg_device_status() == 0
