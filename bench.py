@@ -355,6 +355,43 @@ def run_ours(args):
         }
         del col_out, col_ws
 
+    # ---- host time per call (App. E, last paragraph: the descriptor path's host cost shows on GEMMs of tens of
+    # microseconds): wall time of back-to-back calls while the stream is kept full by long kernels queued first, so
+    # that the host never waits for the device; through the C entry point with argument structs built once, and
+    # through the Python binding (which builds them on every call)
+    if rank == 0:
+        import ctypes as Ct
+        from paper_2609_11356_b200 import _cabi
+        from paper_2609_11356_b200.api import _tensor, _epilogue
+        Lc = _cabi.load()
+        host_us = {}
+        W1 = synth.device_normal((4096, 4096), 0.02, seed0 + 70, bf, dev)
+        shapes = {"decode_m32_splitk8": (d_split, T["dc_X"], T["dc_W"], T["dc_C"], dict(residual=T["dc_R"]), ws),
+                  "m1_n4096_k4096": (d_plain, T["dc_X"][:1, :4096], W1, T["dc_C"][:1], {}, None)}
+        for name, (dd, a_, b_, c_, ekw, ws_) in shapes.items():
+            ta_, tb_, tc_ = _tensor(a_), _tensor(b_), _tensor(c_)
+            ep_ = _epilogue(None, 0, ekw.get("residual"))
+            st_ = torch.cuda.current_stream(dev).cuda_stream
+            wsp, wsb = (ws_.data_ptr(), ws_.numel()) if ws_ is not None else (None, 0)
+            def c_call():
+                return Lc.rg_gemm(Ct.byref(dd), Ct.byref(ta_), Ct.byref(tb_), Ct.byref(tc_), Ct.byref(ep_) if ep_ is not None else None, wsp, wsb, st_)
+            def py_call():
+                rg.rg_gemm(dd, a_, b_, c_, ws=ws_, **ekw)
+            res = {}
+            for label, fn in (("c_abi", c_call), ("python_binding", py_call)):
+                for _ in range(20): fn()
+                torch.cuda.synchronize()
+                for _ in range(12): rg.rg_reduce_rows(d_plain, rg.RG_OP_SUM, T["red_X"], T["red_sum"])     # ~14 ms of queued device work
+                n_calls = 300
+                t0 = time.perf_counter()
+                for _ in range(n_calls): fn()
+                dt = time.perf_counter() - t0
+                torch.cuda.synchronize()
+                res[label] = round(dt / n_calls * 1e6, 2)
+            host_us[name] = res
+        line["host_us_per_call"] = host_us
+        del W1
+
     # ---- bit-match against the oracle on sampled outputs of this very run, and GPU-vs-GPU identity
     if rank == 0:
         from oracle import rgo
@@ -412,6 +449,16 @@ def run_ours(args):
         line["reduce"]["softmax_unit_normal_gbs"] = round(4.0 * 16384 * RED_C / t_unit / 1e9, 1)
         line["roofline_softmax"] = softmax_roofline(16384.0 * RED_C / t_unit, 4.0 * 16384 * RED_C / t_unit / 1e9, peaks, clocks)
         del xu, zu
+        # RMSNorm at its configured size, back to back on four rotating input/output pairs (above L2): what the
+        # kernel does when launches follow one another, beside the in-step figure that carries a whole launch
+        xs = [T["rms_X"]] + [synth.device_normal((RMS_R, RMS_C), 1.0, 90 + i, bf, dev) for i in range(3)]
+        ys = [torch.empty_like(T["rms_Y"]) for _ in range(4)]
+        for i in range(8): rg.rg_reduce_rows(d_plain, rg.RG_OP_RMSNORM, xs[i % 4], ys[i % 4], weight=T["rms_w"], eps=1e-5)
+        torch.cuda.synchronize(); e0.record()
+        for i in range(40): rg.rg_reduce_rows(d_plain, rg.RG_OP_RMSNORM, xs[i % 4], ys[i % 4], weight=T["rms_w"], eps=1e-5)
+        e1.record(); torch.cuda.synchronize()
+        line["reduce"]["rmsnorm_back_to_back_gbs"] = round(4.0 * RMS_R * RMS_C / (e0.elapsed_time(e1) / 40 * 1e-3) / 1e9, 1)
+        del xs, ys
 
     # ---- end to end through the host-buffer C entry points (GEMM metric): pinned host tensors,
     # H2D of the operands and D2H of the result inside the timed region, every step
@@ -462,6 +509,28 @@ def run_ours(args):
         if rank == 0:
             line["e2e"] = e2e
             line["e2e_matches_device_path"] = bool(torch.equal(host["sq_C"], T["sq_C"].cpu()))
+
+    # ---- the same for a reduction: fp32 row sum of 8192 x 32768 (1 GiB) from pinned host memory
+    if rank == 0:
+        e2e_rows = 8192
+        g_ = torch.Generator().manual_seed(5)
+        hx = torch.empty((e2e_rows, RED_C), dtype=f32).pin_memory()
+        hx.normal_(0.0, 100.0, generator=g_)
+        hsum = torch.empty(e2e_rows, dtype=f32).pin_memory()
+        scratch_r = torch.empty(rg_reduce_rows_host_scratch_bytes(rg.RG_OP_SUM, hx, hsum), dtype=torch.uint8, device=dev)
+        for _ in range(2): rg_reduce_rows_host(d_plain, rg.RG_OP_SUM, hx, hsum, scratch_r)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(3): rg_reduce_rows_host(d_plain, rg.RG_OP_SUM, hx, hsum, scratch_r)
+        e1.record(); torch.cuda.synchronize()
+        ms_r = e0.elapsed_time(e1) / 3
+        from oracle import rgo as _rgo
+        ok_r = bool(np.array_equal(hsum.numpy()[:16].view(np.uint32), _rgo.reduce_rows(_rgo.OP_SUM, hx.numpy()[:16])[0].view(np.uint32)))
+        line["e2e_reduce"] = {"value": round(hx.numel() * 4 / (ms_r * 1e-3) / 1e9, 2), "unit": "GB/s", "h2d_bytes_per_step": hx.numel() * 4,
+                              "d2h_bytes_per_step": e2e_rows * 4, "ms_per_step": round(ms_r, 3),
+                              "api": "rg_reduce_rows_host (row sum of 8192 x 32768 fp32 from pinned host memory)", "matches_oracle_on_16_rows": ok_r}
+        del hx, scratch_r
 
     if rank == 0:
         line["cpu_baseline"] = cpu_baseline(budget_s=12.0)
@@ -550,6 +619,8 @@ def run_only(args):
         A = synth.device_normal((M, K), 1.0, 11, bf, dev); B = synth.device_normal((N, K), 0.02, 12, bf, dev)
         Cm = torch.empty((M, N), dtype=bf, device=dev)
         bias = synth.device_uniform((N,), -0.1, 0.1, 8, bf, dev) if name == "gemm_prefill" else None
+        if args.inner_span:
+            d = rg.rg_desc(inner_span=args.inner_span, BN=args.bn, cta_group=args.cta_group)
         fn = lambda: rg.rg_gemm(d, A, B, Cm, bias=bias, act=1 if bias is not None else 0)
         work, unit = 2.0 * M * N * K / 1e12, "TFLOP/s"
     elif name == "gemm_square_f8":
@@ -653,6 +724,8 @@ def main():
     ap.add_argument("--bk", type=int, default=0, help="--only gemm_decode: K per pipeline stage (0 = library's choice)")
     ap.add_argument("--sm-share", type=int, default=0, help="--only gemm_decode: 0 library's choice, 1 one CTA per SM, 2 two CTAs per SM")
     ap.add_argument("--b-static", type=int, default=0, help="--only gemm_decode: 1 = promise that the weights are not written by work in flight")
+    ap.add_argument("--inner-span", type=int, default=0, help="--only gemm_square: second cut level (an accumulator closed every so many k)")
+    ap.add_argument("--cta-group", type=int, default=0, help="--only gemm_square with --inner-span: 1 one-CTA tiles, 2 two-SM tiles")
     ap.add_argument("--stages", type=int, default=0, help="--only gemm_decode: ring depth (0 = as many as fit)")
     ap.add_argument("--attn-block", type=int, default=128, help="key block width for --only attention")
     ap.add_argument("--attn-causal", type=int, default=0, help="1: causal masking, for --only attention (flops counted as half)")
