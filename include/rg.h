@@ -186,8 +186,10 @@ rg_status_t rg_gemm(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t*
                     const rg_epilogue_t* epi, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Row reductions with a fixed tree over the columns (Sec. 3.1, Sec. 5.1; kernels named in
- * Sec. 7: row sums, softmax, rmsnorm).  `d->tree` (BALANCED only on the GPU), `d->acc_dtype`
- * (fp32) and `d->fma` apply; the leaves are the `x.cols` columns in index order.
+ * Sec. 7: row sums, softmax, rmsnorm).  `d->tree`, `d->acc_dtype` (fp32) and `d->fma` apply; the leaves
+ * are the `x.cols` columns in index order.  RG_TREE_LEFT is the chain ((l0 + l1) + l2) + ... (Sec. 3.1:
+ * the other end of the work/depth range; with `fma` the sum of squares is acc = fma(x, x, acc)): the
+ * same class on every GPU as the balanced tree is, and far slower (C - 1 dependent adds per row).
  *   RG_OP_SUM:           out[r] = TREE(f32(x[r,:]));            out: rows x 1 fp32
  *   RG_OP_RMSNORM:       ss = TREE(x*x); rinv = 1/sqrt(ss/cols + eps);
  *                        y[r,c] = round((x*rinv)*w[c]);           out: rows x cols, bf16 or fp32
@@ -200,7 +202,8 @@ rg_status_t rg_reduce_rows(const rg_desc_t* d, rg_reduce_op_t op, const rg_tenso
 
 /* Reductions along the other axis: one tree per column over the rows in index order (Sec. 6:
  * "reductions on different dims/axes", the column sum a matrix-multiply epilogue emits, the
- * LayerNorm weight-gradient reduction; the tree is the one of Sec. 5.1, `d->tree` BALANCED only).
+ * LayerNorm weight-gradient reduction; the tree is the one of Sec. 5.1, or the left fold when
+ * `d->tree` is RG_TREE_LEFT, which needs no workspace).
  *   RG_COLOP_SUM: out[c] = TREE_r f32(x[r,c])
  *   RG_COLOP_DOT: out[c] = TREE_r f32(x[r,c]) * f32(y[r,c])   one rounding per product; with
  *                 `d->fma` the second product of each level-0 pair is fused into that pair's add

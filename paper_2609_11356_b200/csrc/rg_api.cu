@@ -310,7 +310,7 @@ static rg_status_t check_reduce(const rg_desc_t* d, rg_reduce_op_t op, const rg_
   if (s != RG_OK) return s;
   if ((s = check_tensor(x)) != RG_OK || (s = check_tensor(out)) != RG_OK) return s;
   if (op != RG_OP_SUM && op != RG_OP_RMSNORM && op != RG_OP_SOFTMAX_DENOM) return RG_ERR_UNSUPPORTED;
-  if (d->acc_dtype != RG_F32 || d->tree != RG_TREE_BALANCED) return RG_ERR_UNSUPPORTED;
+  if (d->acc_dtype != RG_F32) return RG_ERR_UNSUPPORTED;
   if (x->dtype == RG_F16 || out->dtype == RG_F16) return RG_ERR_UNSUPPORTED;   // reductions read bf16 or fp32 rows
   if (x->cols < 1) return RG_ERR_SHAPE;
   if (out->rows != x->rows) return RG_ERR_SHAPE;
@@ -326,7 +326,7 @@ rg_status_t rg_reduce_rows(const rg_desc_t* d, rg_reduce_op_t op, const rg_tenso
   if (args && args->weight && !dtype_ok(args->weight_dtype)) return RG_ERR_SHAPE;
   if (x->rows == 0) return RG_OK;
   // speed knobs reused for reductions: BN = threads per row, stages = warp-blocks per step
-  return rg::launch_reduce_rows((int)op, d->fma, x, out, args, d->BN, d->stages, static_cast<cudaStream_t>(cuda_stream));
+  return rg::launch_reduce_rows((int)op, d->tree, d->fma, x, out, args, d->BN, d->stages, static_cast<cudaStream_t>(cuda_stream));
 }
 
 size_t rg_reduce_cols_workspace_bytes(int64_t rows, int64_t cols) {
@@ -340,7 +340,7 @@ rg_status_t rg_reduce_cols(const rg_desc_t* d, rg_col_op_t op, const rg_tensor_t
   if (s != RG_OK) return s;
   if ((s = check_tensor(x)) != RG_OK || (s = check_tensor(out)) != RG_OK) return s;
   if (op != RG_COLOP_SUM && op != RG_COLOP_DOT) return RG_ERR_UNSUPPORTED;
-  if (d->acc_dtype != RG_F32 || d->tree != RG_TREE_BALANCED) return RG_ERR_UNSUPPORTED;
+  if (d->acc_dtype != RG_F32) return RG_ERR_UNSUPPORTED;
   if (x->dtype == RG_F16) return RG_ERR_UNSUPPORTED;                       // leaves are bf16 or fp32
   if (op == RG_COLOP_DOT) {
     if ((s = check_tensor(y)) != RG_OK) return s;
@@ -349,12 +349,12 @@ rg_status_t rg_reduce_cols(const rg_desc_t* d, rg_col_op_t op, const rg_tensor_t
   if (x->rows < 1) return RG_ERR_SHAPE;
   if (out->rows != x->cols || out->cols != 1 || out->dtype != RG_F32) return RG_ERR_SHAPE;
   if (x->cols == 0) return RG_OK;
-  const size_t need = rg_reduce_cols_workspace_bytes(x->rows, x->cols);
+  const size_t need = d->tree == RG_TREE_LEFT ? 0 : rg_reduce_cols_workspace_bytes(x->rows, x->cols);   // a chain has no partial rows
   if (need) {
     if (!ws || ws_bytes < need) return RG_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(ws) & 15) return RG_ERR_ALIGNMENT;
   }
-  return rg::launch_reduce_cols((int)op, d->fma, x, op == RG_COLOP_DOT ? y : nullptr, out, ws, static_cast<cudaStream_t>(cuda_stream));
+  return rg::launch_reduce_cols((int)op, d->tree, d->fma, x, op == RG_COLOP_DOT ? y : nullptr, out, ws, static_cast<cudaStream_t>(cuda_stream));
 }
 
 rg_status_t rg_attention(const rg_attn_desc_t* d, const rg_tensor_t* Q, const rg_tensor_t* K, const rg_tensor_t* Vt,

@@ -52,10 +52,10 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
                         const rg_epilogue_t* epi, void* ws, cudaStream_t st);
 rg_status_t launch_gemv(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
                         const rg_epilogue_t* epi, cudaStream_t st);
-rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* out,
+rg_status_t launch_reduce_rows(int op, int tree, int fma, const rg_tensor_t* x, const rg_tensor_t* out,
                                const rg_reduce_args_t* args, int threads_hint, int unroll_hint, cudaStream_t st);
 size_t reduce_cols_workspace_bytes(int64_t R, int64_t C);
-rg_status_t launch_reduce_cols(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* y, const rg_tensor_t* out,
+rg_status_t launch_reduce_cols(int op, int tree, int fma, const rg_tensor_t* x, const rg_tensor_t* y, const rg_tensor_t* out,
                                void* ws, cudaStream_t st);
 bool make_operand_tmap(CUtensorMap_st* map, const void* ptr, int dtype, int64_t rows, int64_t cols, int64_t ld, int box_rows);
 rg_status_t launch_attention_fixed(int block_n, int exp_base, int causal, float scale, int heads, const rg_tensor_t* Q, const rg_tensor_t* K,

@@ -459,6 +459,79 @@ __global__ void __launch_bounds__(256) rmsnorm_keep_kernel(const ReduceParams p)
   }
 }
 
+// ------------------------------------------------------------------ left fold (RG_TREE_LEFT)
+// The other end of the work/depth range (Sec. 3.1): ((l0 + l1) + l2) + ..., a chain of C - 1 dependent adds
+// per row.  A lane owns a row and walks it in column order; the warp moves 32 rows x 32 columns at a time
+// through shared memory so that global accesses stay coalesced (row-major input, one 128-byte run per row
+// and tile).  With `fma` the sum of squares is the chain acc = fma(x, x, acc) from acc = x0 * x0.
+template <typename T, int OP>
+__global__ void __launch_bounds__(256) reduce_rows_left_kernel(const ReduceParams p) {
+  __shared__ float tile[8][32][33];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float (*tw)[33] = tile[warp];
+  pdl_prologue();
+  auto load_tile = [&](int64_t rb, int64_t c0) {
+#pragma unroll 8
+    for (int i = 0; i < 32; ++i) {
+      const int64_t r = rb + i, c = c0 + lane;
+      tw[i][lane] = (r < p.R && c < p.C) ? elem_to_f32(static_cast<const T*>(p.x)[r * p.ldx + c]) : 0.0f;
+    }
+    __syncwarp();
+  };
+  for (int64_t rb = ((int64_t)blockIdx.x * 8 + warp) * 32; rb < p.R; rb += (int64_t)gridDim.x * 8 * 32) {
+    const int64_t row = rb + lane;
+    float shift = 0.0f;
+    if (OP == OP_SOFTMAX) {
+      float m = -INFINITY;                                // the maximum rounds nothing: any order (App. F)
+      for (int64_t c0 = 0; c0 < p.C; c0 += 32) {
+        load_tile(rb, c0);
+        const int n = (int)min((int64_t)32, p.C - c0);
+        for (int j = 0; j < n; ++j) m = fmaxf(m, tw[lane][j]);
+        __syncwarp();
+      }
+      shift = m;
+    }
+    float acc = 0.0f;
+    for (int64_t c0 = 0; c0 < p.C; c0 += 32) {
+      load_tile(rb, c0);
+      const int n = (int)min((int64_t)32, p.C - c0);
+      for (int j = 0; j < n; ++j) {
+        const float v = tw[lane][j];
+        const bool first = c0 == 0 && j == 0;
+        if (OP == OP_SUM) acc = first ? v : f_add(acc, v);
+        else if (OP == OP_RMS) acc = first ? f_mul(v, v) : (p.fma ? f_fma(v, v, acc) : f_add(acc, f_mul(v, v)));
+        else { const float e = exp_nonpositive(f_add(v, -shift)); acc = first ? e : f_add(acc, e); }
+      }
+      __syncwarp();
+    }
+    if (OP == OP_SUM) {
+      if (row < p.R) static_cast<float*>(p.out)[row * p.ldo] = acc;
+    } else if (OP == OP_SOFTMAX) {
+      if (row < p.R) { static_cast<float*>(p.out)[row * p.ldo] = acc; if (p.aux) p.aux[row] = shift; }
+    } else {
+      const float rinv = rms_rinv(acc, p.C, p.eps);
+      if (row < p.R && p.aux) p.aux[row] = rinv;
+      for (int64_t c0 = 0; c0 < p.C; c0 += 32) {
+        load_tile(rb, c0);
+        const int n = (int)min((int64_t)32, p.C - c0);
+        for (int j = 0; j < n; ++j) {
+          const float w = p.weight ? load_scalar(p.weight, p.w_dtype, c0 + j) : 1.0f;
+          tw[lane][j] = f_mul(f_mul(tw[lane][j], rinv), w);
+        }
+        __syncwarp();
+        for (int i = 0; i < 32; ++i) {
+          const int64_t r = rb + i, c = c0 + lane;
+          if (r < p.R && c < p.C) {
+            if (p.out_dtype == RG_BF16) static_cast<__nv_bfloat16*>(p.out)[r * p.ldo + c] = __float2bfloat16_rn(tw[i][lane]);
+            else static_cast<float*>(p.out)[r * p.ldo + c] = tw[i][lane];
+          }
+        }
+        __syncwarp();
+      }
+    }
+  }
+}
+
 // Launch with programmatic stream serialisation (see pdl_prologue).
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int threads, size_t smem, cudaStream_t st, Args... args) {
@@ -512,9 +585,30 @@ cudaError_t launch_op(int op, const ReduceParams& p, bool vec, bool wr, int U, i
 
 // Host launcher.  Speed knobs only (0 = choose): threads_hint = threads per row, where 32 selects
 // the warp-per-row kernel for sums and RMSNorm; unroll_hint = warp-blocks in flight per warp.
-rg_status_t launch_reduce_rows(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* out,
+rg_status_t launch_reduce_rows(int op, int tree, int fma, const rg_tensor_t* x, const rg_tensor_t* out,
                                const rg_reduce_args_t* args, int threads_hint, int unroll_hint,
                                cudaStream_t st) {
+  if (tree == RG_TREE_LEFT) {
+    ReduceParams p;
+    p.x = x->ptr; p.out = out->ptr;
+    p.weight = args ? args->weight : nullptr;
+    p.aux = args ? static_cast<float*>(args->aux_out) : nullptr;
+    p.R = x->rows; p.C = x->cols; p.ldx = x->ld; p.ldo = out->ld;
+    p.eps = args ? args->eps : 0.0f;
+    p.fma = fma; p.out_dtype = out->dtype; p.w_dtype = args ? args->weight_dtype : RG_F32; p.cap = 0;
+    const int64_t need = (x->rows + 255) / 256, max_grid = (int64_t)current_device().sms * 8;
+    const int grid = (int)(need < max_grid ? need : max_grid);
+    cudaError_t e;
+    if (x->dtype == RG_BF16)
+      e = op == RG_OP_SUM ? launch_pdl(reduce_rows_left_kernel<uint16_t, OP_SUM>, grid, 256, 0, st, p)
+        : op == RG_OP_RMSNORM ? launch_pdl(reduce_rows_left_kernel<uint16_t, OP_RMS>, grid, 256, 0, st, p)
+                              : launch_pdl(reduce_rows_left_kernel<uint16_t, OP_SOFTMAX>, grid, 256, 0, st, p);
+    else
+      e = op == RG_OP_SUM ? launch_pdl(reduce_rows_left_kernel<float, OP_SUM>, grid, 256, 0, st, p)
+        : op == RG_OP_RMSNORM ? launch_pdl(reduce_rows_left_kernel<float, OP_RMS>, grid, 256, 0, st, p)
+                              : launch_pdl(reduce_rows_left_kernel<float, OP_SOFTMAX>, grid, 256, 0, st, p);
+    return e == cudaSuccess ? RG_OK : RG_ERR_CUDA;
+  }
   const int V = x->dtype == RG_BF16 ? 8 : 4;
   const int64_t C = x->cols, R = x->rows;
   const size_t esz = x->dtype == RG_BF16 ? 2 : 4;

@@ -119,6 +119,38 @@ __global__ void __launch_bounds__(COL_THREADS) reduce_cols_kernel(const ColParam
   }
 }
 
+// Left fold (RG_TREE_LEFT): one thread per column walks the rows in index order, ((l0 + l1) + l2) + ...;
+// neighbouring threads read neighbouring columns, so every row is one coalesced run.  Eight rows are
+// requested ahead of the chain.  With `fma` the dot product is the chain acc = fma(x, y, acc) from x0 * y0.
+template <typename T, bool DOT>
+__global__ void __launch_bounds__(128) reduce_cols_left_kernel(const void* xv, const void* yv, int64_t ldx, int64_t ldy, int64_t R, int64_t C,
+                                                               int fma, float* out) {
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  const T* x = static_cast<const T*>(xv) + c;
+  const T* y = DOT ? static_cast<const T*>(yv) + c : nullptr;
+  auto widen = [](T v) -> float { if constexpr (sizeof(T) == 2) return bf16_bits_to_f32(v); else return v; };
+  float acc = 0.0f;
+  for (int64_t r0 = 0; r0 < R; r0 += 8) {
+    float a[8], b[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const bool ok = r0 + i < R;
+      a[i] = ok ? widen(x[(r0 + i) * ldx]) : 0.0f;
+      b[i] = (DOT && ok) ? widen(y[(r0 + i) * ldy]) : 0.0f;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (r0 + i < R) {
+        const bool first = r0 + i == 0;
+        if (!DOT) acc = first ? a[i] : f_add(acc, a[i]);
+        else acc = first ? f_mul(a[i], b[i]) : (fma ? f_fma(a[i], b[i], acc) : f_add(acc, f_mul(a[i], b[i])));
+      }
+    }
+  }
+  out[c] = acc;
+}
+
 template <int OP, bool IN16>
 cudaError_t launch_stage(const ColParams& p, bool fma, dim3 grid, cudaStream_t st) {
   if (OP == 1 && fma) reduce_cols_kernel<OP, IN16, true><<<grid, COL_THREADS, 0, st>>>(p);
@@ -135,9 +167,21 @@ size_t reduce_cols_workspace_bytes(int64_t R, int64_t C) {
 }
 
 // All arguments were validated by the caller.
-rg_status_t launch_reduce_cols(int op, int fma, const rg_tensor_t* x, const rg_tensor_t* y, const rg_tensor_t* out,
+rg_status_t launch_reduce_cols(int op, int tree, int fma, const rg_tensor_t* x, const rg_tensor_t* y, const rg_tensor_t* out,
                                void* ws, cudaStream_t st) {
   const int64_t C = x->cols;
+  if (tree == RG_TREE_LEFT) {
+    const unsigned grid = (unsigned)((C + 127) / 128);
+    const bool in16 = x->dtype == RG_BF16;
+    if (op == RG_COLOP_DOT) {
+      if (in16) reduce_cols_left_kernel<uint16_t, true><<<grid, 128, 0, st>>>(x->ptr, y->ptr, x->ld, y->ld, x->rows, C, fma, static_cast<float*>(out->ptr));
+      else reduce_cols_left_kernel<float, true><<<grid, 128, 0, st>>>(x->ptr, y->ptr, x->ld, y->ld, x->rows, C, fma, static_cast<float*>(out->ptr));
+    } else {
+      if (in16) reduce_cols_left_kernel<uint16_t, false><<<grid, 128, 0, st>>>(x->ptr, nullptr, x->ld, 0, x->rows, C, 0, static_cast<float*>(out->ptr));
+      else reduce_cols_left_kernel<float, false><<<grid, 128, 0, st>>>(x->ptr, nullptr, x->ld, 0, x->rows, C, 0, static_cast<float*>(out->ptr));
+    }
+    return cudaGetLastError() == cudaSuccess ? RG_OK : RG_ERR_CUDA;
+  }
   ColParams p;
   p.x = x->ptr; p.y = y ? y->ptr : nullptr; p.ldx = x->ld; p.ldy = y ? y->ld : 0;
   p.R = x->rows; p.C = C;

@@ -201,7 +201,7 @@ def test_argument_errors_are_reported_before_any_launch():
     assert call(d, _t(None, K.RG_BF16, 0, 64), B, _t(None, K.RG_BF16, 0, 8)) == 0
     x = _t(0x1000, K.RG_F32, 4, 64); o = _t(0x2000, K.RG_F32, 4, 1)
     red = lambda d_, op, x_, o_: L.rg_reduce_rows(C.byref(d_), op, C.byref(x_), C.byref(o_), None, None)
-    assert red(rg.rg_desc(tree=K.RG_TREE_LEFT), K.RG_OP_SUM, x, o) == 3
+    assert red(rg.rg_desc(tree=K.RG_TREE_LEFT), K.RG_OP_SUM, x, _t(0x2000, K.RG_F32, 5, 1)) == 4      # the left fold takes the same checks
     assert red(d, K.RG_OP_SUM, _t(0x1000, K.RG_F32, 4, 0), o) == 4
     assert red(d, K.RG_OP_SUM, x, _t(0x2000, K.RG_F32, 5, 1)) == 4
     assert red(d, K.RG_OP_RMSNORM, x, o) == 4
@@ -217,7 +217,7 @@ def test_argument_errors_are_reported_before_any_launch():
     assert col(d, K.RG_COLOP_SUM, xc, None, _t(0x2000, K.RG_F32, 63, 1), 0x4000, 1 << 20) == 4
     assert col(d, K.RG_COLOP_SUM, _t(0x1000, K.RG_F32, 0, 64), None, oc) == 4       # no rows: nothing to fold
     assert col(d, K.RG_COLOP_SUM, _t(None, K.RG_F32, 5, 0), None, _t(None, K.RG_F32, 0, 1)) == 0
-    assert col(rg.rg_desc(tree=K.RG_TREE_LEFT), K.RG_COLOP_SUM, xc, None, oc, 0x4000, 1 << 20) == 3
+    assert col(rg.rg_desc(tree=K.RG_TREE_LEFT), K.RG_COLOP_SUM, xc, None, _t(0x2000, K.RG_F32, 63, 1)) == 4   # shape errors come first
     assert col(d, 7, xc, None, oc, 0x4000, 1 << 20) == 3
     assert L.rg_reduce_cols_workspace_bytes(256, 1000) == 0 and L.rg_reduce_cols_workspace_bytes(257, 1000) == 2 * 1000 * 4
     assert L.rg_reduce_cols_workspace_bytes(65537, 10) == (257 + 2) * 10 * 4

@@ -219,3 +219,27 @@ def test_host_buffer_form_stays_inside_its_scratch(op, with_weight, with_aux):
     assert_bits_equal(oh.numpy(), want, f"host-buffer reduction {op}")
     if with_aux and op != rg.RG_OP_SUM:
         assert_bits_equal(auxh.numpy(), waux, f"host-buffer reduction {op} aux")
+
+
+@pytest.mark.parametrize("shape", [(1, 1), (3, 7), (33, 31), (40, 32), (64, 4096), (300, 1001), (70, 20000)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_left_fold_bit_exact(shape, dtype):
+    """RG_TREE_LEFT (Sec. 3.1: the chain, the other end of the work/depth range): all three operations, both
+    input types, with and without the fused square; a different class of bits from the balanced tree."""
+    if dtype == "f32":
+        x = synth.add_cancellation_pairs(synth.normal_f32(shape, 100.0, 51 + shape[1]), 52, pairs=min(4, shape[1] // 2)) if shape[1] > 1 else synth.normal_f32(shape, 100.0, 51)
+        w = synth.normal_f32((shape[1],), 0.05, 53, mean=1.0)
+    else:
+        x = synth.normal_bf16(shape, 1.0, 54 + shape[1]); w = synth.normal_bf16((shape[1],), 0.05, 55, mean=1.0)
+    got, _ = gpu_reduce(rg.RG_OP_SUM, x, tree=rg.RG_TREE_LEFT)
+    assert_bits_equal(got, rgo.reduce_rows(rgo.OP_SUM, x, tree=rgo.TREE_LEFT)[0], f"left row sum {shape} {dtype}")
+    got, gmax = gpu_reduce(rg.RG_OP_SOFTMAX_DENOM, x, tree=rg.RG_TREE_LEFT)
+    want, wmax = rgo.reduce_rows(rgo.OP_SOFTMAX_DENOM, x, tree=rgo.TREE_LEFT)
+    assert_bits_equal(got, want, f"left softmax normaliser {shape} {dtype}")
+    assert_bits_equal(gmax, wmax, "row maxima")
+    for fma in (0, 1):
+        got, grinv = gpu_reduce(rg.RG_OP_RMSNORM, x, weight=w, eps=1e-5, tree=rg.RG_TREE_LEFT, fma=fma)
+        want, wrinv = rgo.reduce_rows(rgo.OP_RMSNORM, x, weight=w, eps=1e-5, tree=rgo.TREE_LEFT, fma=fma)
+        assert_bits_equal(got, want, f"left rmsnorm {shape} {dtype} fma={fma}")
+        assert_bits_equal(grinv, wrinv, "1/rms")
+    assert rg.rg_desc_class(rg.rg_desc(tree=rg.RG_TREE_LEFT)) != rg.rg_desc_class(rg.rg_desc())

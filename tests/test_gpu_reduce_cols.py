@@ -91,6 +91,23 @@ def test_argument_errors():
     with pytest.raises(rg.RgError):
         rg.rg_reduce_cols(rg.rg_desc(), rg.RG_COLOP_DOT, x[:200], out)               # y missing
     with pytest.raises(rg.RgError):
-        rg.rg_reduce_cols(rg.rg_desc(tree=rg.RG_TREE_LEFT), rg.RG_COLOP_SUM, x[:200], out)
-    with pytest.raises(rg.RgError):
         rg.rg_reduce_cols(rg.rg_desc(), rg.RG_COLOP_SUM, x[:200], torch.zeros(9, dtype=torch.float32, device=DEV))
+
+
+@pytest.mark.parametrize("R,C", [(1, 9), (2, 5), (33, 257), (300, 131), (5000, 260), (70000, 40)])
+@pytest.mark.parametrize("in16", [False, True])
+def test_left_fold_bit_exact(R, C, in16):
+    """RG_TREE_LEFT: the chain over the rows in index order (Sec. 3.1), no workspace."""
+    x = synth.normal_bf16((R, C), 1.0, 5 + R) if in16 else synth.add_cancellation_pairs(synth.normal_f32((R, C), 100.0, 3 + R + C).T.copy(), 7, pairs=min(2, R // 2)).T.copy()
+    y = synth.normal_bf16((R, C), 1.0, 6 + R) if in16 else synth.normal_f32((R, C), 1.0, 4 + R)
+    xt, yt = synth.to_torch(x, DEV), synth.to_torch(y, DEV)
+    out = torch.full((C,), float("nan"), dtype=torch.float32, device=DEV)
+    rg.rg_reduce_cols(rg.rg_desc(tree=rg.RG_TREE_LEFT), rg.RG_COLOP_SUM, xt, out)           # no workspace at any row count
+    torch.cuda.synchronize()
+    assert_bits_equal(out.cpu().numpy(), rgo.reduce_cols(0, x, tree=rgo.TREE_LEFT), f"left col sum {R}x{C}")
+    for fma in (0, 1):
+        rg.rg_reduce_cols(rg.rg_desc(tree=rg.RG_TREE_LEFT, fma=fma), rg.RG_COLOP_DOT, xt, out, y=yt)
+        torch.cuda.synchronize()
+        assert_bits_equal(out.cpu().numpy(), rgo.reduce_cols(1, x, y, tree=rgo.TREE_LEFT, fma=fma), f"left col dot {R}x{C} fma={fma}")
+    if R >= 33 and not in16:                                      # and it is a different sum from the balanced tree
+        assert not np.array_equal(rgo.reduce_cols(0, x, tree=rgo.TREE_LEFT), rgo.reduce_cols(0, x))
