@@ -190,9 +190,14 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
     for (int group = 1; group <= 2; ++group) {
       if (want_group && group != want_group) continue;
       if (group == 2 && M <= 128) continue;
+      // the second cut level keeps a running sum per thread: up to 128 columns it stays in registers, and the
+      // one-CTA kernel's hand-over is the shorter one (8192^3, a group every 64 k: 539 TFLOP/s on 128 x 128 tiles,
+      // 274 on two-SM 256 x 128, 171 on 256-wide tiles of either kernel)
+      if (d->inner_span && !want_group && group == 2) continue;
       for (int bn = 256; bn >= 32; bn -= 16) {
         if (d->BN && bn != d->BN) continue;
-        if (group == 2 && bn != 256) continue;
+        if (d->inner_span && !d->BN && bn > 128) continue;
+        if (group == 2 && bn != 256 && !(d->inner_span && bn == 128)) continue;
         const int64_t items = (group == 2 ? tiles_m2 : tiles_m) * ((N + bn - 1) / bn) * plan->n_parts;
         const int64_t slots = group == 2 ? sms / 2 : sms;
         const int64_t rounds = (items + slots - 1) / slots;

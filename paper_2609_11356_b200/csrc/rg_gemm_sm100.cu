@@ -239,7 +239,7 @@ struct GemmParams {
   int32_t f8;             // operands are e4m3 bytes: M, N as given, every K quantity counted in byte pairs
   int32_t launch_seq;     // host-side launch counter (used by the optional timeline stamps only)
   int32_t b_static;       // the caller's promise that no work ahead in the stream writes B: its first boxes are fetched before the dependency wait
-  uint32_t tmem_cols;     // tensor-memory columns allocated: two accumulators of tmem_cols / 2
+  uint32_t tmem_cols;     // tensor-memory columns allocated: two (or four) accumulators of equal width
   uint32_t a_box_bytes;   // bytes of one A box: 128 B per row actually loaded (rows past M are never fetched)
   uint32_t slack_bytes;   // readable bytes kept behind the ring for the tensor-core step's surplus A rows
   void* C;
@@ -386,14 +386,16 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, const int BN,
 // Second cut level (Sec. 3.2.2 "some kernels cut again inside a part"; App. E per-group accumulation):
 // the MMA warp closes an accumulator every inner_span k; each epilogue warp adds every closed group,
 // at fp32 and in ascending order, into a running sum held in registers, then finishes the tile from
-// it.  A warp owns at most four 32-column chunks (tiles up to 256 columns wide).
-struct GroupedAcc { uint32_t v[4][32]; };
+// it.  A warp owns two 32-column chunks (tiles up to 128 columns, the running sum stays in registers) or four
+// (tiles up to 256 columns: 128 running-sum registers, part of which the compiler keeps in local memory).
+template <int NCH> struct GroupedAcc { uint32_t v[NCH][32]; };
 
+template <int NCH>
 __device__ __forceinline__ void grouped_add(const GemmParams& p, const int BN, int tn, uint32_t taddr, int chunk0, bool first,
-                                            GroupedAcc& acc) {
+                                            GroupedAcc<NCH>& acc) {
   const int col_end = min(p.N, (tn + 1) * BN);
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
+  for (int j = 0; j < NCH; ++j) {
     const int c0 = (chunk0 + 2 * j) * 32;
     if (c0 < BN && tn * BN + c0 < col_end) {              // uniform across the warp
       uint32_t r[32];
@@ -406,11 +408,12 @@ __device__ __forceinline__ void grouped_add(const GemmParams& p, const int BN, i
   }
 }
 
+template <int NCH>
 __device__ __forceinline__ void grouped_finish(const GemmParams& p, const int BN, int part, int64_t row, bool row_ok, int tn,
-                                               int chunk0, const GroupedAcc& acc) {
+                                               int chunk0, const GroupedAcc<NCH>& acc) {
   const int col_end = min(p.N, (tn + 1) * BN);
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
+  for (int j = 0; j < NCH; ++j) {
     const int c0 = (chunk0 + 2 * j) * 32;
     const int col0 = tn * BN + c0;
     if (c0 < BN && col0 < col_end && row_ok) epilogue_store_chunk(p, part, row, col0, min(32, col_end - col0), acc.v[j]);
@@ -493,7 +496,7 @@ __device__ __forceinline__ void finish_and_store4(const EpilogueArgs& e, void* C
 // GROUPED: the second cut level (inner_span): accumulators closed inside a part and chained in the epilogue
 // warps' registers; an instantiation of its own, so that its 128 running-sum registers per thread are not
 // the plain kernel's problem.
-template <int KSUB, bool F8, bool CLUSTER, int EPI_WARPS, bool GROUPED = false>
+template <int KSUB, bool F8, bool CLUSTER, int EPI_WARPS, bool GROUPED = false, int NCH = 2>
 __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, EPI_WARPS == 4 ? 3 : 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const GemmParams p) {
@@ -504,8 +507,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const int BN = p.bn;
   const uint32_t B_BOX_BYTES = (uint32_t)BN * KBOX * 2;
   const uint32_t STAGE_BYTES = KSUB * (A_BOX_BYTES + B_BOX_BYTES);
-  const uint32_t TMEM_COLS = p.tmem_cols;                // a power of two >= 32; accumulator b starts at column b * TMEM_COLS / 2
-  const uint32_t ACC_STRIDE = TMEM_COLS >> 1;
+  // Accumulators in tensor memory: two, or four for the second cut level on tiles up to 128 columns (its
+  // groups are short, and more of them in flight hide the hand-over between the issuing warp and the epilogue)
+  constexpr int NB = (GROUPED && NCH == 2) ? 4 : 2;
+  const uint32_t TMEM_COLS = p.tmem_cols;                // a power of two >= 32; accumulator b starts at column b * TMEM_COLS / NB
+  const uint32_t ACC_STRIDE = TMEM_COLS / NB;
   const uint32_t IDESC = p.idesc;
 
   extern __shared__ uint8_t smem_raw[];
@@ -515,17 +521,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const int S = p.num_stages;
   // barriers sit behind the ring and behind the span a short A box leaves readable (see a_slack_bytes)
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + (size_t)S * STAGE_BYTES + p.slack_bytes);
-  // layout: full[S], empty[S], tmem_full[2], tmem_empty[2], then tmem base slot and abort flag
+  // layout: full[S], empty[S], tmem_full[NB], tmem_empty[NB], then tmem base slot and abort flag
   const uint32_t bar_full = smem_u32(bars);
   const uint32_t bar_empty = bar_full + 8u * S;
   const uint32_t bar_tfull = bar_empty + 8u * S;
-  const uint32_t bar_tempty = bar_tfull + 16u;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+  const uint32_t bar_tempty = bar_tfull + 8u * NB;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2 * NB);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   // CLUSTER: two more barriers (parts ready / parts read), then this CTA's partial tile
-  const uint32_t bar_ready = bar_tempty + 16u + 16u;
+  const uint32_t bar_ready = bar_tempty + 8u * NB + 16u;
   const uint32_t bar_free = bar_ready + 8u;
-  float* const part_buf = reinterpret_cast<float*>(bars + 2 * S + 8);
+  float* const part_buf = reinterpret_cast<float*>(bars + 2 * S + 2 * NB + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) RG_STAMP(0);                      // CTA entry
@@ -540,7 +546,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     prefetch_tensormap(&tmap_a);
     prefetch_tensormap(&tmap_b);
     for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8u * s, 1); mbar_init(bar_empty + 8u * s, 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8u * b, 1); mbar_init(bar_tempty + 8u * b, EPI_WARPS); }
+    for (int b = 0; b < NB; ++b) { mbar_init(bar_tfull + 8u * b, 1); mbar_init(bar_tempty + 8u * b, EPI_WARPS); }
     if (CLUSTER) { mbar_init(bar_ready, EPI_WARPS * p.n_parts); mbar_init(bar_free, EPI_WARPS * p.n_parts); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -639,8 +645,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
           if (!step_groups && k0 >= group_end) {
             if (k0 > k_begin) { if (leader) umma_commit(bar_tfull + 8u * buf); ++gc; }   // the previous group is complete
-            buf = gc & 1;
-            if (!warp_mbar_wait(bar_tempty + 8u * buf, ((gc >> 1) & 1) ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
+            buf = gc % NB;
+            if (!warp_mbar_wait(bar_tempty + 8u * buf, ((gc / NB) & 1) ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
             tcgen05_fence_after();
             d_tmem = tmem_base + buf * ACC_STRIDE;
             accumulate = 0;                              // every part and every group starts from zero
@@ -658,8 +664,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
               if (kk >= k_end) break;                    // ascending k; nothing past the end of the part
               if (kk >= group_end) {                     // this step opens a new accumulator
                 if (kk > k_begin) { if (leader) umma_commit(bar_tfull + 8u * buf); ++gc; }
-                buf = gc & 1;
-                if (!warp_mbar_wait(bar_tempty + 8u * buf, ((gc >> 1) & 1) ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
+                buf = gc % NB;
+                if (!warp_mbar_wait(bar_tempty + 8u * buf, ((gc / NB) & 1) ^ 1u, abort_flag, &g_status_word, 0x200u | buf)) { alive = false; break; }
                 tcgen05_fence_after();
                 d_tmem = tmem_base + buf * ACC_STRIDE;
                 accumulate = 0;
@@ -747,8 +753,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       if (CLUSTER) {
         // ---- this CTA's part of the tile: tensor memory -> its shared-memory partial buffer
         const int it = gc;                                  // tiles this cluster has finished
-        const int buf = gc & 1;
-        if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
+        const int buf = gc % NB;
+        if (!mbar_wait(bar_tfull + 8u * buf, (gc / NB) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
         tcgen05_fence_after();
         if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
         // the buffer still holds the previous tile's part until every CTA of the cluster has read its slice
@@ -803,8 +809,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         __syncwarp();
         if (lane < p.n_parts) mbar_arrive_cluster(map_to_cta(bar_free, (uint32_t)lane));   // this warp no longer reads any CTA's part
       } else if (!GROUPED) {
-        const int buf = gc & 1;
-        if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
+        const int buf = gc % NB;
+        if (!mbar_wait(bar_tfull + 8u * buf, (gc / NB) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
         tcgen05_fence_after();
         if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
@@ -814,10 +820,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
         ++gc;
       } else if (EPI_WARPS == 8) {                          // the second cut level runs with eight epilogue warps
-        GroupedAcc acc;
+        GroupedAcc<NCH> acc;
         for (int g = 0; g < ngroups && alive; ++g, ++gc) {
-          const int buf = gc & 1;
-          if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
+          const int buf = gc % NB;
+          if (!mbar_wait(bar_tfull + 8u * buf, (gc / NB) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
           tcgen05_fence_after();
           if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
@@ -1085,7 +1091,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         const int klen = p.part_end[part] - p.part_begin[part];
         const int ngroups = p.inner_span > 0 ? (klen + p.inner_span - 1) / p.inner_span : 1;
         const int64_t row = (int64_t)tm * 2 * BM + (int64_t)rank * BM + quarter * 32 + lane;
-        GroupedAcc acc;
+        GroupedAcc<BN / 64> acc;
         for (int g = 0; g < ngroups && alive; ++g, ++gc) {
           const int buf = gc & 1;
           if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0xc00u | buf)) { alive = false; break; }
@@ -1370,7 +1376,7 @@ size_t a_slack_bytes(int bn, int ksub, int a_rows) {
 
 size_t smem_bytes_for(int bn, int ksub, int stages, int a_rows) {
   const size_t stage = (size_t)ksub * ((size_t)a_rows * KBOX * 2 + (size_t)bn * KBOX * 2);
-  return 1024 + stages * stage + a_slack_bytes(bn, ksub, a_rows) + (2 * stages + 4) * 8 + 16;
+  return 1024 + stages * stage + a_slack_bytes(bn, ksub, a_rows) + (2 * stages + 8) * 8 + 16;   // room for four accumulator barrier pairs
 }
 
 // CLUSTER kernels: two more barriers and the CTA's partial tile behind the plain kernel's layout
@@ -1503,14 +1509,14 @@ cudaError_t launch_one_t(const CUtensorMap& ta, const CUtensorMap& tb, const Gem
   return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<KSUB, F8, false, EPI_WARPS>, ta, tb, p);
 }
 
-// the second cut level: 64-wide stages, eight epilogue warps
-template <bool F8>
+// the second cut level: 64-wide stages, eight epilogue warps; NCH = 32-column chunks a warp keeps a running sum of
+template <bool F8, int NCH>
 cudaError_t launch_grouped_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   const size_t smem = smem_bytes_for(p.bn, 1, p.num_stages, (int)(p.a_box_bytes / (KBOX * 2)));
   static DeviceOnce configured;
   const int dev = current_device().dev;
   if (!configured.has(dev)) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<1, F8, false, 8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<1, F8, false, 8, true, NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
     if (e != cudaSuccess) return e;
     configured.set(dev);
   }
@@ -1524,7 +1530,7 @@ cudaError_t launch_grouped_t(const CUtensorMap& ta, const CUtensorMap& tb, const
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<1, F8, false, 8, true>, ta, tb, p);
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<1, F8, false, 8, true, NCH>, ta, tb, p);
 }
 
 template <int KSUB>
@@ -1635,7 +1641,12 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   // step time is made of ((rows + width) x 32 bytes at 128 bytes per clock).  Same products, same order.
   p.mma_m = (!pair && M <= 64) ? 64 : BM;
   p.idesc = make_idesc(plan.BN, pair ? 2 * BM : p.mma_m, idesc_format(kind));
-  { uint32_t c = 32; while (c < 2u * (uint32_t)((plan.BN + 31) / 32 * 32)) c <<= 1; p.tmem_cols = c; }
+  {
+    const uint32_t accumulators = (plan.inner_span && !pair && plan.BN <= 128) ? 4u : 2u;   // see NB in the one-CTA kernel
+    uint32_t c = 32;
+    while (c < accumulators * (uint32_t)((plan.BN + 31) / 32 * 32)) c <<= 1;
+    p.tmem_cols = c;
+  }
   for (int s = 0; s < plan.n_parts; ++s) { p.part_begin[s] = plan.part_begin[s] / kdiv; p.part_end[s] = plan.part_end[s] / kdiv; }
   EpilogueArgs e{};
   if (epi) {
@@ -1687,7 +1698,8 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   } else if (plan.inner_span) {
     if (ksub != 1) return RG_ERR_UNSUPPORTED;
     const int grid = (int)(total < sms ? total : sms);
-    err = p.f8 ? launch_grouped_t<true>(ta, tb, p, grid, st) : launch_grouped_t<false>(ta, tb, p, grid, st);
+    if (plan.BN <= 128) err = p.f8 ? launch_grouped_t<true, 2>(ta, tb, p, grid, st) : launch_grouped_t<false, 2>(ta, tb, p, grid, st);
+    else err = p.f8 ? launch_grouped_t<true, 4>(ta, tb, p, grid, st) : launch_grouped_t<false, 4>(ta, tb, p, grid, st);
   } else {
     const int grid = (int)(total < sms ? total : sms);
     if (ksub == 1) err = launch_one<1>(ta, tb, p, grid, st);
