@@ -175,6 +175,31 @@ __device__ __forceinline__ float exp_core(float x) {
   return f_mul(q, __int_as_float((__float_as_int(t) << 23) + 0x3f800000));   // t's low mantissa bits hold n
 }
 
+// exp_core on two arguments at once, with the packed fp32x2 instructions of this architecture
+// (each half is one IEEE round-to-nearest operation, so every intermediate has the bits of the scalar form;
+// x - n is written as fma(n, -1, x): the product is exact, so it is the same single rounding).  A thread then
+// issues half as many floating-point instructions per key in the polynomial.  Only chains of fused multiply-adds
+// are packed: a packed multiply feeding a packed add is contracted into one packed fma by the assembler even
+// when both carry an explicit rounding mode (measured: 1 % of such pairs change their last bit), so the
+// score scaling (multiply, then subtract the maximum) and the fold O = a * O + PV stay scalar.
+__device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
+__device__ __forceinline__ float2 exp_core2(float2 x) {
+  const float2 y = __fmul2_rn(x, splat2(0x1.715476p+0f));
+  const float2 t = __fadd2_rn(y, splat2(12582912.0f));
+  const float2 n = __fadd2_rn(t, splat2(-12582912.0f));
+  float2 r = __ffma2_rn(n, splat2(-0x1.62e400p-1f), x);
+  r = __ffma2_rn(n, splat2(-0x1.7f7d1cp-20f), r);
+  float2 q = splat2(0x1.a01a02p-13f);
+  q = __ffma2_rn(q, r, splat2(0x1.6c16c2p-10f));
+  q = __ffma2_rn(q, r, splat2(0x1.111112p-7f));
+  q = __ffma2_rn(q, r, splat2(0x1.555556p-5f));
+  q = __ffma2_rn(q, r, splat2(0x1.555556p-3f));
+  q = __ffma2_rn(q, r, splat2(0.5f));
+  q = __ffma2_rn(q, r, splat2(1.0f));
+  q = __ffma2_rn(q, r, splat2(1.0f));
+  return __fmul2_rn(q, make_float2(__int_as_float((__float_as_int(t.x) << 23) + 0x3f800000), __int_as_float((__float_as_int(t.y) << 23) + 0x3f800000)));
+}
+
 // rg_exp2 for an argument that is <= 0 or NaN: the overflow select can never fire and is left out
 // (same bits as rg_exp2 on that domain).
 __device__ __forceinline__ float exp2_nonpositive(float x) {
@@ -472,7 +497,18 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             xmin = min3f_nan(xmin, pr[CK - 1], pr[CK - 1]);
             if (xmin >= (BASE2 ? -126.0f : -87.33655f)) {
 #pragma unroll
-              for (int c = 0; c < CK; ++c) pr[c] = BASE2 ? exp2_core(pr[c]) : exp_core(pr[c]);
+              if (BASE2) {
+#pragma unroll
+                for (int c = 0; c < CK; ++c) pr[c] = exp2_core(pr[c]);
+              } else {
+                // base e has three more floating-point operations per key than base two: packed, it gains 3 %
+                // (452 against 437 TFLOP/s); base two does not (the threads wait on dependent results, not on issue slots)
+#pragma unroll
+                for (int c = 0; c < CK; c += 2) {
+                  const float2 e2 = exp_core2(make_float2(pr[c], pr[c + 1]));
+                  pr[c] = e2.x; pr[c + 1] = e2.y;
+                }
+              }
             } else {
 #pragma unroll
               for (int c = 0; c < CK; ++c) pr[c] = BASE2 ? exp2_nonpositive(pr[c]) : rg_exp(pr[c]);
