@@ -637,7 +637,7 @@ def run_only(args):
         A = synth.device_normal((M, K), 1.0, 4, bf, dev)
         Ws = [synth.device_normal((N, K), 0.02, 3 + i, bf, dev) for i in range(4)]    # rotate: weights leave L2
         R = synth.device_normal((M, N), 1.0, 5, bf, dev); Cm = torch.empty((M, N), dtype=bf, device=dev)
-        ws = torch.empty(rg.rg_gemm_workspace_bytes(d, M, N), dtype=torch.uint8, device=dev)
+        ws = torch.zeros(rg.rg_gemm_workspace_bytes(d, M, N), dtype=torch.uint8, device=dev)   # zero-filled once (split_merge = 3 needs it)
         it = [0]
         def fn():
             it[0] += 1

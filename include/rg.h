@@ -79,7 +79,13 @@ typedef struct {
   uint8_t split_merge;    /* where split-K parts are added (same tree, same bits): 0 = the library chooses (today: 1);
                              1 = by a second kernel, through the workspace; 2 = inside the GEMM kernel, by the CTAs
                              of a thread-block cluster over distributed shared memory (one launch, no workspace;
-                             2..8 parts, one-CTA tiles; RG_ERR_UNSUPPORTED where it does not apply) */
+                             2..8 parts, one-CTA tiles; RG_ERR_UNSUPPORTED where it does not apply);
+                             3 = inside the GEMM kernel, by the CTA that stores a tile's last part: the parts go
+                             through the workspace, whose first bytes hold one ticket per tile (2..8 parts, one-CTA
+                             tiles).  The caller's PROMISE with 3: the workspace was zero-filled once (e.g. a
+                             cudaMemset when it was allocated) and only calls of this library with split_merge = 3
+                             have written it since; every such call leaves the tickets zero again.  After an
+                             RG_ERR_TIMEOUT from rg_device_status, zero it again */
   /* ---- order-deciding fields: these ARE the class key ---- */
   uint8_t in_dtype;       /* rg_dtype_t of A and B: RG_BF16, RG_F16, or RG_F8E4M3 (with atom = RG_ATOM_TC_F8_K32) */
   uint8_t acc_dtype;      /* accumulator: RG_F32 */
@@ -158,8 +164,10 @@ rg_status_t rg_desc_validate(const rg_desc_t* d, int64_t M, int64_t N, int64_t K
  * the epilogue are excluded.  Returns 0 for a malformed descriptor.  Host only. */
 uint64_t rg_desc_class(const rg_desc_t* d);
 
-/* Bytes of workspace rg_gemm needs: 0 without cuts, else (n_cuts+1) * M * roundup(N,4) * sizeof(partial_dtype);
- * SIZE_MAX if that product does not fit size_t (no buffer satisfies it, so the call is refused). */
+/* Bytes of workspace rg_gemm needs: 0 without cuts, else (n_cuts+1) * M * roundup(N,4) * sizeof(partial_dtype),
+ * plus, with split_merge = 3, 64 KiB of tickets in front of the parts (the same place for every shape, so one
+ * zero-filled workspace serves calls of different shapes; at most 16384 output tiles);
+ * SIZE_MAX if that does not fit size_t (no buffer satisfies it, so the call is refused). */
 size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N);
 
 /* C[M,N] = epilogue( merge_s( sum_{k in part s} A[i,k] * B[j,k] ) )   (C = A * B^T).

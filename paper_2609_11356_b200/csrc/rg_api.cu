@@ -51,7 +51,10 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
   if (d->cta_group == 2 && (d->BM == 128 || (d->BN != 0 && d->BN != 128 && d->BN != 256) || d->BK == 256)) return RG_ERR_UNSUPPORTED;   // a pair works on 256 rows, BN >= 128
   if (d->cta_group == 1 && d->BM == 256) return RG_ERR_UNSUPPORTED;
   if (d->raster > 64) return RG_ERR_INVALID_DESC;
-  if (d->split_merge > 2 || d->sm_share > 2 || d->b_static > 1) return RG_ERR_INVALID_DESC;
+  if (d->split_merge > 3 || d->sm_share > 2 || d->b_static > 1) return RG_ERR_INVALID_DESC;
+  // the last-arriver merge: 2 to 8 parts, one-CTA tiles at a whole SM each, no second cut level
+  if (d->split_merge == 3 && (d->n_cuts < 1 || d->n_cuts > 7 || d->inner_span || d->cta_group == 2 || d->BM == 256 || d->BK == 256 || d->sm_share == 2))
+    return RG_ERR_UNSUPPORTED;
   // two CTAs per SM: the one-CTA kernel with four epilogue warps, tiles up to 128 columns, no second cut level
   if (d->sm_share == 2 && (d->cta_group == 2 || d->BM == 256 || d->BN > 128 || d->BK == 256 || d->inner_span || d->split_merge == 2))
     return RG_ERR_UNSUPPORTED;
@@ -135,6 +138,7 @@ bool plan_cluster_merge(const rg_desc_t* d, int64_t M, int64_t N, rg::GemmPlan* 
 rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::GemmPlan* plan) {
   plan->n_parts = (int)d->n_cuts + 1;
   plan->cluster_merge = 0;
+  plan->ticket_merge = d->split_merge == 3 ? 1 : 0;
   plan->half_sm = 0;
   plan->b_static = d->b_static ? 1 : 0;
   plan->tree = d->tree;
@@ -176,7 +180,8 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   }
   // one CTA per 128-row tile, or a pair of CTAs (two SMs) per 256-row tile
   int want_group = 0;
-  if (d->cta_group) want_group = d->cta_group;
+  if (plan->ticket_merge) want_group = 1;
+  else if (d->cta_group) want_group = d->cta_group;
   else if (d->BM == 256) want_group = 2;
   else if (d->BM == 128) want_group = 1;
   if (plan->BN == 0 || (want_group == 0 && !skinny)) {
@@ -224,6 +229,7 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   if (!d->BK && skinny && plan->n_parts == 1 && !d->inner_span && plan->cta_group == 1 && !half &&
       rg::max_stages_for(plan->BN, 256, 1, M) >= 4)
     plan->BK = 256;
+  if (plan->ticket_merge && plan->BK > 128) plan->BK = 128;
   if (plan->cta_group == 2 && plan->BN != 128 && plan->BN != 256) return RG_ERR_UNSUPPORTED;
   plan->half_sm = half && plan->cta_group == 1 && plan->BK <= 128 && rg::max_stages_for(plan->BN, plan->BK, 1, M, false, true) >= 2;
   if (d->sm_share == 2 && !plan->half_sm) return RG_ERR_UNSUPPORTED;
@@ -281,6 +287,7 @@ size_t rg_gemm_workspace_bytes(const rg_desc_t* d, int64_t M, int64_t N) {
   if (__builtin_mul_overflow(b, (size_t)M, &b) || __builtin_mul_overflow(b, (size_t)((N + 3) / 4 * 4), &b) ||
       __builtin_mul_overflow(b, (size_t)(d->partial_dtype == RG_F32 ? 4 : 2), &b))
     return SIZE_MAX;
+  if (d->split_merge == 3 && __builtin_add_overflow(b, rg::ticket_bytes(), &b)) return SIZE_MAX;   // the tickets in front of the parts
   return b;
 }
 

@@ -248,6 +248,7 @@ struct GemmParams {
   void* ws;             // split-K partials [part][M][ldw] at ws_dtype; null without cuts and with the in-cluster merge
   int64_t ldw;
   int32_t ws_dtype;
+  unsigned int* tickets;  // TICKET kernels: one counter per output tile (zero on entry, zero again on exit), else null
   // in-cluster merge (CLUSTER kernels): the n_parts CTAs of a cluster own the parts of one output tile
   int32_t tree, merge_dtype;   // how the parts are added (descriptor's tree, type of the running sum)
   int32_t part_rows;           // rows of a tile kept in a CTA's shared-memory partial buffer
@@ -496,7 +497,14 @@ __device__ __forceinline__ void finish_and_store4(const EpilogueArgs& e, void* C
 // GROUPED: the second cut level (inner_span): accumulators closed inside a part and chained in the epilogue
 // warps' registers; an instantiation of its own, so that its 128 running-sum registers per thread are not
 // the plain kernel's problem.
-template <int KSUB, bool F8, bool CLUSTER, int EPI_WARPS, bool GROUPED = false, int NCH = 2>
+// TICKET: split-K in one launch without clusters.  Work items are (part, tile) as in the plain kernel and the parts go to
+// the workspace; the CTA that stores a tile's LAST part (an integer ticket per tile, taken after a device-wide fence)
+// merges the tile from the workspace in the descriptor's tree, applies the epilogue and stores.  Nobody waits for
+// anybody: which CTA merges depends on timing, what it computes does not (Sec. 3.1: the tree, not the schedule).
+// Measured on the decode shape it does not pay: equal to the two-kernel path at 1 and 8 rows (24.7-26 us), 6 us
+// slower at 32 rows, where every CTA pays a device-wide fence and two barriers per item and the tiles' merges
+// (37 CTAs, one tile each, alone with their L2 latency) all fall at the end of the launch.  Kept as an option.
+template <int KSUB, bool F8, bool CLUSTER, int EPI_WARPS, bool GROUPED = false, int NCH = 2, bool TICKET = false>
 __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, EPI_WARPS == 4 ? 3 : 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const GemmParams p) {
@@ -528,6 +536,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t bar_tempty = bar_tfull + 8u * NB;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2 * NB);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* ticket_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);   // TICKET: "this CTA merges the tile"
   // CLUSTER: two more barriers (parts ready / parts read), then this CTA's partial tile
   const uint32_t bar_ready = bar_tempty + 8u * NB + 16u;
   const uint32_t bar_free = bar_ready + 8u;
@@ -741,7 +750,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     bool alive = true;
     bool deps_done = false;
     int gc = 0;
-    for (int w = work_first; w < total_work && alive; w += work_step) {
+    for (int w = work_first; w < total_work && (alive || TICKET); w += work_step) {
       int part, tm, tn;
       decode_work(p, w, part, tm, tn);
       if (CLUSTER) part = crank;
@@ -808,6 +817,63 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         }
         __syncwarp();
         if (lane < p.n_parts) mbar_arrive_cluster(map_to_cta(bar_free, (uint32_t)lane));   // this warp no longer reads any CTA's part
+      } else if (TICKET) {
+        // A wait that gives up leaves this warp walking the loop without touching memory, so that the two
+        // barriers of the epilogue warps below are still met by all of them.
+        const int buf = gc % NB;
+        if (alive) alive = mbar_wait(bar_tfull + 8u * buf, (gc / NB) & 1, abort_flag, &g_status_word, 0x400u | buf);
+        if (alive) {
+          tcgen05_fence_after();
+          if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
+          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
+          epilogue_tile(p, BN, part, row, row_ok, tn, taddr, chunk0, CHUNK_STEP);      // this part of the tile -> workspace
+          tcgen05_fence_before();
+        }
+        __syncwarp();
+        if (lane == 0 && alive) mbar_arrive(bar_tempty + 8u * buf);
+        ++gc;
+        // ---- ticket: the part is in the workspace for every CTA to see before the tile's counter moves
+        __threadfence();
+        asm volatile("bar.sync 1, %0;" ::"n"(EPI_WARPS * 32) : "memory");
+        const int tile = tm * p.tiles_n + tn;
+        if (warp == 2 && lane == 0) {
+          const unsigned int old = atomicAdd(p.tickets + tile, 1u);
+          const bool last = old == (unsigned int)(p.n_parts - 1);
+          if (last) p.tickets[tile] = 0u;                  // nobody touches it again before the next call
+          *ticket_flag = last ? 1 : 0;
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(EPI_WARPS * 32) : "memory");
+        if (*ticket_flag && alive) {
+          // ---- this CTA stored the tile's last part: merge all of them (read at L2: other SMs wrote them)
+          __threadfence();
+          const int tile_rows = min(BM, p.M - tm * BM);
+          const int c4s = BN >> 2;
+          const int units = tile_rows * c4s;
+          const int64_t part_stride = (int64_t)p.M * p.ldw;
+          for (int u = (warp - 2) * 32 + lane; u < units; u += EPI_WARPS * 32) {
+            const int r_t = u / c4s, c4 = u - r_t * c4s;
+            const int col0 = tn * BN + 4 * c4;
+            if (col0 >= p.N) continue;
+            const int64_t grow = (int64_t)tm * BM + r_t;
+            const int64_t off = grow * p.ldw + col0;
+            float4 v[8];
+#pragma unroll
+            for (int s2 = 0; s2 < 8; ++s2) {
+              if (s2 < p.n_parts) {
+                if (p.ws_dtype == RG_F32) {
+                  v[s2] = __ldcg(reinterpret_cast<const float4*>(static_cast<const float*>(p.ws) + s2 * part_stride + off));
+                } else {
+                  const uint2 w = __ldcg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.ws) + s2 * part_stride + off));
+                  v[s2] = p.ws_dtype == RG_F16 ? make_float4(f16_bits_to_f32(w.x & 0xffffu), f16_bits_to_f32(w.x >> 16), f16_bits_to_f32(w.y & 0xffffu), f16_bits_to_f32(w.y >> 16))
+                                               : make_float4(bf16_bits_to_f32(w.x & 0xffffu), bf16_bits_to_f32(w.x >> 16), bf16_bits_to_f32(w.y & 0xffffu), bf16_bits_to_f32(w.y >> 16));
+                }
+              }
+            }
+            const float4 acc = p.merge_dtype == RG_F32 ? merge_upto8<false>(v, p.n_parts, p.tree, p.merge_dtype)
+                                                        : merge_upto8<true>(v, p.n_parts, p.tree, p.merge_dtype);
+            finish_and_store4(p.epi, p.C, p.ldc, p.c_dtype, p.N, grow, col0, acc);
+          }
+        }
       } else if (!GROUPED) {
         const int buf = gc % NB;
         if (!mbar_wait(bar_tfull + 8u * buf, (gc / NB) & 1, abort_flag, &g_status_word, 0x400u | buf)) { alive = false; break; }
@@ -1509,6 +1575,30 @@ cudaError_t launch_one_t(const CUtensorMap& ta, const CUtensorMap& tb, const Gem
   return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<KSUB, F8, false, EPI_WARPS>, ta, tb, p);
 }
 
+// split-K in one launch, the tile's last-arriving CTA merging (TICKET instantiations)
+template <int KSUB, bool F8>
+cudaError_t launch_ticket_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
+  const size_t smem = smem_bytes_for(p.bn, KSUB, p.num_stages, (int)(p.a_box_bytes / (KBOX * 2)));
+  static DeviceOnce configured;
+  const int dev = current_device().dev;
+  if (!configured.has(dev)) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<KSUB, F8, false, 8, false, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    if (e != cudaSuccess) return e;
+    configured.set(dev);
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<KSUB, F8, false, 8, false, 2, true>, ta, tb, p);
+}
+
 // the second cut level: 64-wide stages, eight epilogue warps; NCH = 32-column chunks a warp keeps a running sum of
 template <bool F8, int NCH>
 cudaError_t launch_grouped_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
@@ -1553,6 +1643,13 @@ bool make_operand_tmap(CUtensorMap_st* map, const void* ptr, int dtype, int64_t 
 int a_box_rows_for(int64_t M) { return M >= BM ? BM : (int)((M + 7) / 8 * 8); }
 
 int cluster_part_rows(int64_t M) { return M >= BM ? BM : (int)M; }
+
+constexpr size_t TICKET_TILES_MAX = 16384;
+
+// Bytes in front of the parts that hold the per-tile tickets of the TICKET kernels.  The size does not depend
+// on the shape, so a workspace that serves calls of different shapes keeps its tickets where no call's parts
+// ever land: 16384 tiles at most.
+size_t ticket_bytes() { return TICKET_TILES_MAX * sizeof(unsigned int); }
 
 // cluster_merge: the in-cluster split-K kernel, whose partial tile shares the shared memory with the ring
 // (0 stages = it does not fit at all)
@@ -1654,12 +1751,15 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     e.residual = epi->residual; e.residual_dtype = epi->residual_dtype; e.ldr = epi->ldr;
   }
   const bool in_cluster = plan.cluster_merge != 0;            // parts merged inside the GEMM kernel, no workspace
+  const bool ticket = plan.ticket_merge != 0;                 // parts through the workspace, merged by the tile's last CTA
   const bool split = plan.n_parts > 1 && !in_cluster;
   p.C = C->ptr; p.ldc = C->ld; p.c_dtype = C->dtype;
-  p.ws = split ? ws : nullptr;
+  // ticket mode: the tickets sit in front of the parts (see ticket_bytes)
+  p.tickets = ticket ? static_cast<unsigned int*>(ws) : nullptr;
+  p.ws = split ? (ticket ? static_cast<void*>(static_cast<uint8_t*>(ws) + ticket_bytes()) : ws) : nullptr;
   p.ws_dtype = plan.partial_dtype;
   p.ldw = (N + 3) / 4 * 4;
-  p.epi = split ? EpilogueArgs{} : e;
+  p.epi = (split && !ticket) ? EpilogueArgs{} : e;
   p.tree = plan.tree; p.merge_dtype = plan.merge_dtype;
   p.part_rows = cluster_part_rows(M); p.part_ld = plan.BN + 4;
 
@@ -1695,6 +1795,12 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     if (ksub == 1) err = launch_one_half<1>(ta, tb, p, grid, st);
     else if (ksub == 2) err = launch_one_half<2>(ta, tb, p, grid, st);
     else return RG_ERR_UNSUPPORTED;
+  } else if (ticket) {
+    if ((size_t)p.tiles_m * (size_t)p.tiles_n > TICKET_TILES_MAX) return RG_ERR_UNSUPPORTED;   // more tiles than tickets
+    const int grid = (int)(total < sms ? total : sms);
+    if (ksub == 1) err = p.f8 ? launch_ticket_t<1, true>(ta, tb, p, grid, st) : launch_ticket_t<1, false>(ta, tb, p, grid, st);
+    else if (ksub == 2) err = p.f8 ? launch_ticket_t<2, true>(ta, tb, p, grid, st) : launch_ticket_t<2, false>(ta, tb, p, grid, st);
+    else return RG_ERR_UNSUPPORTED;
   } else if (plan.inner_span) {
     if (ksub != 1) return RG_ERR_UNSUPPORTED;
     const int grid = (int)(total < sms ? total : sms);
@@ -1709,7 +1815,7 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   }
   if (err != cudaSuccess) return RG_ERR_CUDA;
 
-  if (split) {
+  if (split && !ticket) {
     FixupParams f;
     f.ws = ws; f.ldw = p.ldw; f.partial_dtype = plan.partial_dtype; f.merge_dtype = plan.merge_dtype;
     f.M = p.M; f.N = p.N; f.S = plan.n_parts; f.tree = plan.tree; f.launch_seq = p.launch_seq;

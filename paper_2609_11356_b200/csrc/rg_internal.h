@@ -38,6 +38,7 @@ struct GemmPlan {
   int BN, BK, stages, raster, group_m, cta_group;
   int b_static;             // caller's promise: nothing in flight on the stream writes B (its first boxes may be fetched early)
   int half_sm;              // the one-CTA kernel in its half-SM form: two CTAs share an SM (weight-streaming shapes)
+  int ticket_merge;         // split-K parts through the workspace, merged inside the GEMM kernel by the CTA that stores a tile's last part
   int cluster_merge;        // split-K parts merged inside the GEMM kernel by a thread-block cluster (no workspace, one launch)
   int n_parts, tree;
   int partial_dtype, merge_dtype;
@@ -48,6 +49,7 @@ struct GemmPlan {
 
 int max_stages_for(int bn, int bk, int cta_group, int64_t M, bool cluster_merge = false, bool half_sm = false);
 int max_active_clusters(int csize, int bk, bool f8);
+size_t ticket_bytes();
 rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,
                         const rg_epilogue_t* epi, void* ws, cudaStream_t st);
 rg_status_t launch_gemv(const rg_desc_t* d, const rg_tensor_t* A, const rg_tensor_t* B, const rg_tensor_t* C,

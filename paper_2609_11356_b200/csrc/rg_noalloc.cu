@@ -44,6 +44,9 @@ extern "C" rg_status_t rg_gemm_noalloc(const rg_desc_t* d, const rg_tensor_t* A,
   if (!d || !A || !B || !C) return RG_ERR_NULL;
   if (d->n_cuts > RG_MAX_CUTS) return RG_ERR_INVALID_DESC;
   if (d->n_cuts == 0) return rg_gemm(d, A, B, C, epi, nullptr, 0, cuda_stream);   // no parts, no scratch
+  // split_merge = 3 keeps tickets in the workspace that must be zero between calls; the shared array is also
+  // written by calls that keep parts there, so that promise cannot be made for it
+  if (d->split_merge == 3) return RG_ERR_UNSUPPORTED;
   // the size check comes first: a request beyond the fixed array is refused, never truncated
   const size_t need = rg_gemm_workspace_bytes(d, A->rows, B->rows);
   if (need > (size_t)RG_NOALLOC_WS_BYTES) return RG_ERR_WORKSPACE;

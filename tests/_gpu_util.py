@@ -37,6 +37,10 @@ def gpu_gemm(A, B, *, out_dtype=rgo.BF16, bias=None, act=0, residual=None, poiso
     if nb:
         ws = torch.empty(nb, dtype=torch.uint8, device=DEV)
         ws.fill_(0xFF)
+        if d.split_merge == 3:
+            # the tickets in front of the parts start at zero (the caller's promise); the parts stay poisoned
+            d1 = rg.rg_desc(**{**desc_kw, "split_merge": 1})
+            ws[:nb - rg.rg_gemm_workspace_bytes(d1, M, N)].zero_()
     bt = None if bias is None else (bias if torch.is_tensor(bias) else synth.to_torch(bias, DEV))
     rt = None if residual is None else (residual if torch.is_tensor(residual) else synth.to_torch(residual, DEV))
     rg.rg_gemm(d, At, Bt, Ct, bias=bt, act=act, residual=rt, ws=ws)

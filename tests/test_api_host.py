@@ -55,7 +55,12 @@ def test_validate_rules():
     # speed knobs and promises that are not order fields
     assert rg.rg_desc_validate(rg.rg_desc(cuts=(256,), split_merge=2), 64, 256, 512) == 0
     assert rg.rg_desc_validate(rg.rg_desc(split_merge=2), 64, 256, 512) == 3                            # nothing to merge
-    assert rg.rg_desc_validate(rg.rg_desc(cuts=(256,), split_merge=3), 64, 256, 512) == 2
+    assert rg.rg_desc_validate(rg.rg_desc(cuts=(256,), split_merge=3), 64, 256, 512) == 0                # the last-arriver merge
+    assert rg.rg_desc_validate(rg.rg_desc(cuts=(256,), split_merge=3, cta_group=2), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(cuts=(256,), split_merge=4), 64, 256, 512) == 2
+    # its tickets sit in front of the parts, 64 KiB for every shape
+    assert rg.rg_gemm_workspace_bytes(rg.rg_desc(cuts=(256,), split_merge=3), 64, 256) == 2 * 64 * 256 * 4 + 65536
+    assert rg.rg_gemm_workspace_bytes(rg.rg_desc(cuts=(256,), split_merge=3), 300, 4096) == 2 * 300 * 4096 * 4 + 65536
     assert rg.rg_desc_validate(rg.rg_desc(sm_share=2), 64, 256, 512) == 0
     assert rg.rg_desc_validate(rg.rg_desc(sm_share=2, BN=256), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(b_static=1), 64, 256, 512) == 0
@@ -85,7 +90,7 @@ def test_class_key_holds_order_fields_only():
     assert k != 0
     # speed knobs do not move the class (Sec. 3.2.2)
     for kw in (dict(BN=64), dict(BN=256, BK=128), dict(stages=2), dict(raster=1), dict(BM=128), dict(BM=256), dict(cta_group=2),
-               dict(split_merge=1), dict(split_merge=2), dict(sm_share=2), dict(b_static=1)):
+               dict(split_merge=1), dict(split_merge=2), dict(split_merge=3), dict(sm_share=2), dict(b_static=1)):
         assert rg.rg_desc_class(rg.rg_desc(cuts=(1792, 3584), **kw)) == k
     # every order-deciding field does
     others = [rg.rg_desc(cuts=(1792,)), rg.rg_desc(cuts=(1792, 3600)), rg.rg_desc(),

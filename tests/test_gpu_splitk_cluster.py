@@ -14,7 +14,7 @@ from tests._gpu_util import DEV, HW, HW8, assert_bits_equal, gpu_gemm
 
 pytestmark = pytest.mark.gpu
 
-IN_CLUSTER, TWO_KERNELS = 2, 1
+IN_CLUSTER, TWO_KERNELS, LAST_ARRIVER = 2, 1, 3
 
 
 def _inputs(M, N, K, seed, spread=True):
@@ -43,6 +43,7 @@ def test_in_cluster_merge_matches_oracle_and_two_kernel_path(M, parts):
                           f"two kernels M={M} parts={parts} tree={tree} vs oracle")
         assert_bits_equal(gpu_gemm(A, B, cuts=cuts, tree=tree, residual=res), want, f"default path M={M} parts={parts}")
         assert_bits_equal(gpu_gemm(A, B, cuts=cuts, tree=tree, residual=res, b_static=1), want, f"static weights M={M} parts={parts}")
+        assert_bits_equal(gpu_gemm(A, B, cuts=cuts, tree=tree, residual=res, split_merge=LAST_ARRIVER), want, f"last-arriver merge M={M} parts={parts}")
 
 
 @pytest.mark.parametrize("M,N,K,cuts", [(32, 4096, 14336, tuple(1792 * t for t in range(1, 8))),
@@ -158,3 +159,48 @@ def test_two_ctas_per_sm_form_is_the_same_class(M, N, K, cuts):
     for bad in (dict(BN=256), dict(cta_group=2), dict(BK=256)):
         with pytest.raises(rg.RgError):
             gpu_gemm(A, B, cuts=cuts, sm_share=2, **bad)
+
+
+def test_last_arriver_merge_reuses_its_workspace_and_leaves_the_tickets_zero():
+    """split_merge = 3: the parts go through the workspace and the CTA that stores a tile's last part merges it.  The
+    tickets in front of the parts are zero before the first call (the caller's promise) and zero again after every
+    call, so the same workspace serves call after call, for shapes and tilings that change from call to call."""
+    cuts8 = tuple(1792 * t for t in range(1, 8))
+    A, B = _inputs(32, 4096, 14336, 4, spread=False)
+    res = synth.normal_bf16((32, 4096), 1.0, 5)
+    d = rg.rg_desc(cuts=cuts8, split_merge=LAST_ARRIVER, b_static=1)
+    nb = rg.rg_gemm_workspace_bytes(d, 32, 4096)
+    tickets = nb - rg.rg_gemm_workspace_bytes(rg.rg_desc(cuts=cuts8), 32, 4096)
+    assert tickets == 65536                                          # the same place for every shape
+    ws = torch.zeros(nb, dtype=torch.uint8, device=DEV)              # zero-filled once
+    At, Bt, Rt = synth.to_torch(A, DEV), synth.to_torch(B, DEV), synth.to_torch(res, DEV)
+    two = gpu_gemm(A, B, cuts=cuts8, residual=res, split_merge=TWO_KERNELS)
+    for call in range(4):
+        out = torch.empty((32, 4096), dtype=torch.bfloat16, device=DEV); out.view(torch.int16).fill_(-1)
+        rg.rg_gemm(d, At, Bt, out, residual=Rt, ws=ws)
+        torch.cuda.synchronize()
+        assert_bits_equal(synth.from_torch(out), two, f"decode shape, call {call}")
+        assert int(ws[:tickets].max().item()) == 0, "tickets not back at zero"
+    # other shapes, tilings and part counts on the same (never re-zeroed) workspace
+    for M, N, K, cuts, knobs in ((8, 1003, 1000, (256, 512, 768), dict(BN=48)), (37, 520, 2304, (768, 1536), dict(BN=112, BK=64)),
+                                 (128, 260, 1024, (512,), dict(BN=64)), (300, 200, 2048, (512, 1024, 1536), dict(BN=128))):
+        A2, B2 = _inputs(M, N, K, 60 + M)
+        bias = synth.uniform_bf16((N,), -0.1, 0.1, 8)
+        d2 = rg.rg_desc(cuts=cuts, split_merge=LAST_ARRIVER, **knobs)
+        assert rg.rg_gemm_workspace_bytes(d2, M, N) <= nb
+        out = torch.empty((M, N), dtype=torch.float32, device=DEV); out.view(torch.int32).fill_(-1)
+        rg.rg_gemm(d2, synth.to_torch(A2, DEV), synth.to_torch(B2, DEV), out, bias=synth.to_torch(bias, DEV), act=1, ws=ws)
+        torch.cuda.synchronize()
+        assert_bits_equal(out.cpu().numpy(), rgo.gemm(A2, B2, cuts=cuts, atom_model=HW, bias=bias, act=1, out_dtype=rgo.F32), f"{M}x{N}x{K} {knobs}")
+        assert int(ws[:tickets].max().item()) == 0
+    for pd, md in ((rgo.BF16, rgo.F32), (rgo.F16, rgo.F16)):
+        for tree in (rg.RG_TREE_LEFT, rg.RG_TREE_BALANCED):
+            got = gpu_gemm(A[:, :2048], B[:300, :2048], cuts=(512, 1024, 1536), tree=tree, partial_dtype=pd, merge_dtype=md, split_merge=LAST_ARRIVER, out_dtype=rgo.F16)
+            want = rgo.gemm(A[:, :2048], B[:300, :2048], cuts=(512, 1024, 1536), tree=tree, atom_model=HW, partial_dtype=pd, merge_dtype=md, out_dtype=rgo.F16)
+            assert_bits_equal(got, want, f"last-arriver partial={pd} merge={md} tree={tree}")
+    assert rg.rg_desc_class(d) == rg.rg_desc_class(rg.rg_desc(cuts=cuts8))
+    with pytest.raises(rg.RgError):
+        rg.rg_gemm(rg.rg_desc(cuts=tuple(64 * t for t in range(1, 10)), split_merge=LAST_ARRIVER), At, Bt, out, ws=ws)   # nine cuts: ten parts
+    with pytest.raises(rg.RgError):
+        rg.rg_gemm_noalloc(rg.rg_desc(cuts=cuts8, split_merge=LAST_ARRIVER), At, Bt, torch.empty((32, 4096), dtype=torch.bfloat16, device=DEV))
+    assert rg.rg_device_status() == 0
