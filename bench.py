@@ -366,8 +366,9 @@ def run_ours(args):
         Lc = _cabi.load()
         host_us = {}
         W1 = synth.device_normal((4096, 4096), 0.02, seed0 + 70, bf, dev)
-        shapes = {"decode_m32_splitk8": (d_split, T["dc_X"], T["dc_W"], T["dc_C"], dict(residual=T["dc_R"]), ws),
-                  "m1_n4096_k4096": (d_plain, T["dc_X"][:1, :4096], W1, T["dc_C"][:1], {}, None)}
+        c_host = torch.empty_like(T["dc_C"])          # own output: the step's results are compared with the oracle further down
+        shapes = {"decode_m32_splitk8": (d_split, T["dc_X"], T["dc_W"], c_host, dict(residual=T["dc_R"]), ws),
+                  "m1_n4096_k4096": (d_plain, T["dc_X"][:1, :4096], W1, c_host[:1], {}, None)}
         for name, (dd, a_, b_, c_, ekw, ws_) in shapes.items():
             ta_, tb_, tc_ = _tensor(a_), _tensor(b_), _tensor(c_)
             ep_ = _epilogue(None, 0, ekw.get("residual"))
@@ -390,7 +391,7 @@ def run_ours(args):
                 res[label] = round(dt / n_calls * 1e6, 2)
             host_us[name] = res
         line["host_us_per_call"] = host_us
-        del W1
+        del W1, c_host
 
     # ---- bit-match against the oracle on sampled outputs of this very run, and GPU-vs-GPU identity
     if rank == 0:
