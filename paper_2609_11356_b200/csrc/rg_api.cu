@@ -187,7 +187,7 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   if (plan->BN == 0 || (want_group == 0 && !skinny)) {
     // Time ~ rounds of work items x operand rows of a tile (128 of A + its width of B): below 256 columns a
     // step is bound by the rows it reads from shared memory (and the tile pulls from L2), not by arithmetic.  A
-    // pair loads 128 + 128 rows per CTA for a 256-wide tile and measured 0.88 of that.  Any multiple of 16
+    // pair loads 128 + 128 rows per CTA for a 256-wide tile and is charged 0.82 of that.  Any multiple of 16
     // is a legal width for the one-CTA kernel, so the widest tile that still fits the fewest rounds wins:
     // 640 x 4096 x 4096 is one round of 128 x 160 tiles, 1536 rows two rounds of 128 x 192.
     const int64_t tiles_m2 = (M + 255) / 256;
@@ -206,7 +206,9 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
         const int64_t items = (group == 2 ? tiles_m2 : tiles_m) * ((N + bn - 1) / bn) * plan->n_parts;
         const int64_t slots = group == 2 ? sms / 2 : sms;
         const int64_t rounds = (items + slots - 1) / slots;
-        const int64_t cost = group == 2 ? rounds * 338 : rounds * (bn + 128);
+        // the pair's factor: 0.82 of the 384 rows it stands for (measured on 14336 x 4096 weights at 512, 768 and
+        // 1024 rows: the 256 x 256 pair 53 / 75 / 95 us, the best one-CTA tile 57 / 81 / 104 us, which 0.88 ranked the other way)
+        const int64_t cost = group == 2 ? rounds * 315 : rounds * (bn + 128);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_bn = bn; best_group = group; }
       }
     }
