@@ -74,7 +74,7 @@ typedef struct {
   /* ---- speed knobs: validated, NOT part of the class key (Sec. 3.2.2) ---- */
   uint16_t BM, BN, BK;    /* output tile and K step per pipeline stage; 0 = library default */
   uint8_t stages;         /* shared-memory ring depth; 0 = as many as fit */
-  uint8_t cta_group;      /* 1, or 2 (pair of SMs on one 256-row tile); 0 = default */
+  uint8_t cta_group;      /* 1, or 2 (pair of SMs on one 256-row tile: BN from 32, BK 64 or 128; with inner_span BN 128 or 256); 0 = default */
   uint8_t raster;         /* tile walk: 0 = default grouped walk, 1 = row-major, n in 2..64 = groups of n tile rows */
   uint8_t split_merge;    /* where split-K parts are added (same tree, same bits): 0 = the library chooses (today: 1);
                              1 = by a second kernel, through the workspace; 2 = inside the GEMM kernel, by the CTAs

@@ -1,5 +1,6 @@
 // The C boundary: argument validation, descriptor canonicalisation and class key, plan
 // selection, and the host-buffer forms.  Nothing here does arithmetic on data.
+#include <algorithm>
 #include <string.h>
 
 #include "rg_internal.h"
@@ -48,7 +49,9 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
   if (d->BK != 0 && d->BK != 64 && d->BK != 128 && d->BK != 256) return RG_ERR_UNSUPPORTED;
 
   if (d->cta_group > 2) return RG_ERR_INVALID_DESC;
-  if (d->cta_group == 2 && (d->BM == 128 || (d->BN != 0 && d->BN != 128 && d->BN != 256) || d->BK == 256)) return RG_ERR_UNSUPPORTED;   // a pair works on 256 rows, BN >= 128
+  // a pair works on 256 rows and at least 32 columns; with a second cut level on 128 or 256 columns
+  if (d->cta_group == 2 && (d->BM == 128 || (d->BN != 0 && (d->BN < 32 || (d->inner_span && d->BN != 128 && d->BN != 256))) || d->BK == 256))
+    return RG_ERR_UNSUPPORTED;
   if (d->cta_group == 1 && d->BM == 256) return RG_ERR_UNSUPPORTED;
   if (d->raster > 64) return RG_ERR_INVALID_DESC;
   if (d->split_merge > 3 || d->sm_share > 2 || d->b_static > 1) return RG_ERR_INVALID_DESC;
@@ -185,16 +188,23 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   else if (d->BM == 256) want_group = 2;
   else if (d->BM == 128) want_group = 1;
   if (plan->BN == 0 || (want_group == 0 && !skinny)) {
-    // Time ~ rounds of work items x operand rows of a tile (128 of A + its width of B): below 256 columns a
-    // step is bound by the rows it reads from shared memory (and the tile pulls from L2), not by arithmetic.  A
-    // pair loads 128 + 128 rows per CTA for a 256-wide tile and is charged 0.82 of that.  Any multiple of 16
-    // is a legal width for the one-CTA kernel, so the widest tile that still fits the fewest rounds wins:
-    // 640 x 4096 x 4096 is one round of 128 x 160 tiles, 1536 rows two rounds of 128 x 192.
+    // Time per k of a round of work items, in operand rows pulled from L2 (2 bytes per row and k), is the largest of
+    //   the round's CTAs x rows of one CTA / 121   L2 feeds the SMs about 15 TB/s in total, 121 SMs' worth of the next line
+    //   rows of one CTA                            an SM takes in 64 bytes per clock
+    //   1.3 x width (1.4 for a pair)               the arithmetic of a 128-row step, at the clock the power cap leaves
+    // where a CTA of the one-CTA kernel pulls 128 rows of A and the tile's width of B, a CTA of a pair 128 and half
+    // the width (charged 1.17 of that: the two CTAs' boxes meet on one barrier), and a pair's launch costs about
+    // 1.4 us more (88000 row-k), which counts on short K.  Fitted on 4096- and 14336-column problems of 256-2048
+    // rows (K = 512 ... 14336): 512 x 4096 x 4096 is one round of 256 x 128 pairs (19 us; 128 x 112 tiles 24),
+    // 768 rows one round of 256 x 192 pairs, 384 rows 128 x 96 tiles.  Any multiple of 16 is a legal width; the
+    // pair is offered multiples of 32 (a pair's step on an odd multiple of 16 measured 10-15 % slower than on its
+    // neighbours).
     const int64_t tiles_m2 = (M + 255) / 256;
-    int best_bn = 0, best_group = 0; int64_t best_cost = -1;
+    const int64_t klen = plan->n_parts > 1 ? (K + plan->n_parts - 1) / plan->n_parts : K;
+    int best_bn = 0, best_group = 0; double best_cost = -1;
     for (int group = 1; group <= 2; ++group) {
       if (want_group && group != want_group) continue;
-      if (group == 2 && M <= 128) continue;
+      if (group == 2 && (M <= 128 || d->BK == 256)) continue;        // a pair's stage is 64 or 128 k
       // the second cut level keeps a running sum per thread: up to 128 columns it stays in registers, and the
       // one-CTA kernel's hand-over is the shorter one (8192^3, a group every 64 k: 539 TFLOP/s on 128 x 128 tiles,
       // 274 on two-SM 256 x 128, 171 on 256-wide tiles of either kernel)
@@ -202,13 +212,17 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
       for (int bn = 256; bn >= 32; bn -= 16) {
         if (d->BN && bn != d->BN) continue;
         if (d->inner_span && !d->BN && bn > 128) continue;
-        if (group == 2 && bn != 256 && !(d->inner_span && bn == 128)) continue;
+        if (group == 2 && d->inner_span && bn != 256 && bn != 128) continue;
+        if (group == 2 && !d->BN && bn % 32 != 0) continue;
         const int64_t items = (group == 2 ? tiles_m2 : tiles_m) * ((N + bn - 1) / bn) * plan->n_parts;
         const int64_t slots = group == 2 ? sms / 2 : sms;
-        const int64_t rounds = (items + slots - 1) / slots;
-        // the pair's factor: 0.82 of the 384 rows it stands for (measured on 14336 x 4096 weights at 512, 768 and
-        // 1024 rows: the 256 x 256 pair 53 / 75 / 95 us, the best one-CTA tile 57 / 81 / 104 us, which 0.88 ranked the other way)
-        const int64_t cost = group == 2 ? rounds * 315 : rounds * (bn + 128);
+        const double rows = group == 2 ? 128 + bn / 2 : 128 + bn;
+        const double one_cta = std::max(rows * (group == 2 ? 1.17 : 1.0), (group == 2 ? 1.4 : 1.3) * bn);
+        const int64_t last = items % slots;                               // work items of the last, partial round
+        double cost = (double)(items / slots) * std::max((double)(slots * group) * rows / 121.0, one_cta);
+        if (last) cost += std::max((double)(last * group) * rows / 121.0, one_cta);
+        if (group == 2) cost += 88000.0 / (double)(klen > 0 ? klen : 1);
+        if (group == 2 && bn != 256 && bn != 128) cost *= 1.03;       // 256 and 128 columns are compile-time forms of the pair kernel
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_bn = bn; best_group = group; }
       }
     }
@@ -220,19 +234,19 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   }
   if (half && plan->BN > 128) plan->BN = 128;
   plan->cta_group = want_group ? want_group : 1;
-  if (plan->cta_group == 2 && plan->BN < 128) plan->cta_group = 1;
+  if (plan->cta_group == 2 && plan->BN < 32) plan->cta_group = 1;
   // the widest two-SM tile runs a seven-stage ring of 64-wide K steps: more slack per byte of shared memory than
   // three 128-wide stages, now that a whole turn of the ring is issued from precomputed descriptor words
   // skinny problems read long runs of each weight row per stage (DRAM likes 512-byte bursts)
-  // one-CTA tiles up to 128 columns take 128-wide K steps as well (half the hand-overs; the stage still fits four times)
-  plan->BK = d->BK ? d->BK : (!d->inner_span && (skinny || (plan->cta_group == 1 && plan->BN <= 128 && !half)) ? 128 : 64);
+  // tiles up to 128 columns (pairs up to 192) take 128-wide K steps as well (half the hand-overs; the stage still fits four times)
+  plan->BK = d->BK ? d->BK : (!d->inner_span && (skinny || ((plan->BN <= 128 || (plan->cta_group == 2 && plan->BN <= 192)) && !half)) ? 128 : 64);
   // a skinny problem without cuts is bounded by the hand-overs along its one K chain: 256-wide stages halve them,
   // as long as four of them still fit
   if (!d->BK && skinny && plan->n_parts == 1 && !d->inner_span && plan->cta_group == 1 && !half &&
       rg::max_stages_for(plan->BN, 256, 1, M) >= 4)
     plan->BK = 256;
   if (plan->ticket_merge && plan->BK > 128) plan->BK = 128;
-  if (plan->cta_group == 2 && plan->BN != 128 && plan->BN != 256) return RG_ERR_UNSUPPORTED;
+  if (plan->cta_group == 2 && ((d->inner_span && plan->BN != 128 && plan->BN != 256) || plan->BK == 256)) return RG_ERR_UNSUPPORTED;
   plan->half_sm = half && plan->cta_group == 1 && plan->BK <= 128 && rg::max_stages_for(plan->BN, plan->BK, 1, M, false, true) >= 2;
   if (d->sm_share == 2 && !plan->half_sm) return RG_ERR_UNSUPPORTED;
   const int smax = rg::max_stages_for(plan->BN, plan->BK, plan->cta_group, M, false, plan->half_sm != 0);

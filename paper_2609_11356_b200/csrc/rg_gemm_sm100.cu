@@ -932,15 +932,22 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 //   tempty[b] in the even CTA; the epilogue warps of both CTAs arrive on it
 // GROUPED: the second cut level on the pair (see the one-CTA kernel): the issuing CTA closes an accumulator
 // every inner_span k, the epilogue warps of both CTAs chain the closed groups in registers.
-template <int BN, int KSUB, int KIND, bool GROUPED = false>
+// BN_T = 0: the tile width is a launch parameter (any multiple of 16 from 32 to 256): a CTA then reads
+// 128 + width/2 operand rows per step where the one-CTA kernel reads 128 + width, which is what a step's time is
+// made of below 256 columns.  The widths that large problems use (256, 128) keep their compile-time forms.
+template <int BN_T, int KSUB, int KIND, bool GROUPED = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                          const GemmParams p) {
+  constexpr bool RT = BN_T == 0;
+  static_assert(!(RT && GROUPED), "the second cut level on the pair is built for 128 and 256 columns");
+  const int BN = RT ? p.bn : BN_T;
+  const int ACC = RT ? 256 : BN_T;                                          // tensor-memory columns between the two accumulators
   constexpr uint32_t A_BOX_BYTES = BM * KBOX * 2;
-  constexpr uint32_t B_BOX_BYTES = (BN / 2) * KBOX * 2;
-  constexpr uint32_t STAGE_BYTES = KSUB * (A_BOX_BYTES + B_BOX_BYTES);      // per CTA
-  constexpr uint32_t TMEM_COLS = 2 * BN;
-  constexpr uint32_t IDESC = make_idesc(BN, 2 * BM, idesc_format(KIND));
+  const uint32_t B_BOX_BYTES = (uint32_t)(BN / 2) * KBOX * 2;
+  const uint32_t STAGE_BYTES = KSUB * (A_BOX_BYTES + B_BOX_BYTES);          // per CTA
+  constexpr uint32_t TMEM_COLS = RT ? 512u : 2u * BN_T;
+  const uint32_t IDESC = RT ? p.idesc : make_idesc(BN_T, 2 * BM, idesc_format(KIND));
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -989,6 +996,9 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       const uint32_t box_off = is_b ? KSUB * A_BOX_BYTES + sub * B_BOX_BYTES : sub * A_BOX_BYTES;
       int stage = 0; uint32_t phase = 0;
       bool alive = true;
+      // launched with programmatic stream serialisation like the one-CTA kernel: the kernels ahead in the stream
+      // are waited for immediately before this role's first access to global memory
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int w = pair_id; w < total_work && alive; w += num_pairs) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);
@@ -1053,7 +1063,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                 buf = gc & 1;
                 if (!warp_mbar_wait(bar_tempty + 8u * buf, ((gc >> 1) & 1) ^ 1u, abort_flag, &g_status_word, 0xa00u | buf)) { alive = false; break; }
                 tcgen05_fence_after();
-                d_tmem = tmem_base + buf * BN;
+                d_tmem = tmem_base + buf * ACC;
                 accumulate = 0;                            // every part and every group starts from zero
                 group_end = kk + span;
               }
@@ -1076,7 +1086,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         const uint32_t acc_phase = (it >> 1) & 1;
         if (!warp_mbar_wait(bar_tempty + 8u * buf, acc_phase ^ 1u, abort_flag, &g_status_word, 0xa00u | buf)) { alive = false; break; }
         tcgen05_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * BN;
+        const uint32_t d_tmem = tmem_base + buf * ACC;
         uint32_t accumulate = 0;                        // every part starts from a zero accumulator
         for (int k0 = k_begin; k0 < k_end; k0 += KBOX * KSUB) {
           if (S == G && stage == 0 && k0 + G * KBOX * KSUB <= k_end) {
@@ -1149,6 +1159,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     const uint32_t tempty_leader = map_to_cta(bar_tempty, 0);
     bool alive = true;
     int it = 0;
+    bool deps_done = false;
     if (GROUPED) {
       int gc = 0;
       for (int w = pair_id; w < total_work && alive; w += num_pairs) {
@@ -1157,12 +1168,13 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         const int klen = p.part_end[part] - p.part_begin[part];
         const int ngroups = p.inner_span > 0 ? (klen + p.inner_span - 1) / p.inner_span : 1;
         const int64_t row = (int64_t)tm * 2 * BM + (int64_t)rank * BM + quarter * 32 + lane;
-        GroupedAcc<BN / 64> acc;
+        GroupedAcc<(RT ? 64 : BN_T) / 64> acc;
         for (int g = 0; g < ngroups && alive; ++g, ++gc) {
           const int buf = gc & 1;
           if (!mbar_wait(bar_tfull + 8u * buf, (gc >> 1) & 1, abort_flag, &g_status_word, 0xc00u | buf)) { alive = false; break; }
           tcgen05_fence_after();
-          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
+          if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
+          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC;
           grouped_add(p, BN, tn, taddr, chunk0, g == 0, acc);
           tcgen05_fence_before();
           __syncwarp();
@@ -1178,8 +1190,9 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       const uint32_t acc_phase = (it >> 1) & 1;
       if (!mbar_wait(bar_tfull + 8u * buf, acc_phase, abort_flag, &g_status_word, 0xc00u | buf)) { alive = false; break; }
       tcgen05_fence_after();
+      if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
       const int64_t row = (int64_t)tm * 2 * BM + (int64_t)rank * BM + quarter * 32 + lane;
-      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC;
       epilogue_tile(p, BN, part, row, row < p.M, tn, taddr, chunk0);
       tcgen05_fence_before();
       __syncwarp();
@@ -1455,7 +1468,7 @@ size_t smem_bytes_for_pair(int bn, int ksub, int stages) {
 
 template <int BN, int KSUB, int KIND, bool GROUPED = false>
 cudaError_t launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
-  const size_t smem = smem_bytes_for_pair(BN, KSUB, p.num_stages);
+  const size_t smem = smem_bytes_for_pair(BN ? BN : p.bn, KSUB, p.num_stages);
   static DeviceOnce configured;
   const int dev = current_device().dev;
   if (!configured.has(dev)) {
@@ -1468,11 +1481,13 @@ cudaError_t launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tb, const Ge
   cfg.blockDim = dim3(NUM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // set-up runs under the tail of the kernel ahead
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, gemm_tcgen05_pair_kernel<BN, KSUB, KIND, GROUPED>, ta, tb, p);
 }
 
@@ -1780,6 +1795,9 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     else if (plan.BN == 256 && ksub == 2) err = launch_pair<256, 2>(ta, tb, p, grid, kind, st);
     else if (plan.BN == 128 && ksub == 1) err = launch_pair<128, 1>(ta, tb, p, grid, kind, st);
     else if (plan.BN == 128 && ksub == 2) err = launch_pair<128, 2>(ta, tb, p, grid, kind, st);
+    else if (plan.BN % 16 != 0 || plan.BN < 32 || plan.BN > 256) return RG_ERR_UNSUPPORTED;
+    else if (ksub == 1) err = launch_pair<0, 1>(ta, tb, p, grid, kind, st);
+    else if (ksub == 2) err = launch_pair<0, 2>(ta, tb, p, grid, kind, st);
     else return RG_ERR_UNSUPPORTED;
   } else if (in_cluster) {
     const int avail = max_active_clusters(plan.n_parts, plan.BK, kind == KIND_F8E4M3);

@@ -72,10 +72,12 @@ def test_validate_rules():
     assert rg.rg_desc_validate(rg.rg_desc(merge_dtype=K.RG_BF16), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(BN=100), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(BN=112, BK=256), 64, 256, 512) == 0
-    assert rg.rg_desc_validate(rg.rg_desc(BN=112, cta_group=2), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(BN=112, cta_group=2), 64, 256, 512) == 0     # a pair takes any width from 32 columns
+    assert rg.rg_desc_validate(rg.rg_desc(BN=112, cta_group=2, inner_span=64), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(cta_group=2), 64, 256, 512) == 0
     assert rg.rg_desc_validate(rg.rg_desc(cta_group=3), 64, 256, 512) == 2
-    assert rg.rg_desc_validate(rg.rg_desc(cta_group=2, BN=64), 64, 256, 512) == 3
+    assert rg.rg_desc_validate(rg.rg_desc(cta_group=2, BN=64), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(cta_group=2, BN=16), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(cta_group=1, BM=256), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(tree=7), 64, 256, 512) == 2
     assert rg.rg_desc_validate(ok, 64, 256, 0) == 4

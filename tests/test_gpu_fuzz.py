@@ -30,7 +30,8 @@ def _case(g):
         knobs = [dict(), dict(BN=64), dict(BN=96, stages=2), dict(BN=256), dict(cta_group=2, BN=128), dict(cta_group=2, BN=256)][int(g.integers(0, 6))]
     else:
         knobs = [dict(), dict(BN=64, BK=128), dict(cta_group=2, BN=128), dict(cta_group=2, BN=256, BK=64), dict(BN=48, cta_group=1),
-                 dict(BN=208, cta_group=1, raster=1), dict(BN=128, BK=256, cta_group=1, stages=1)][int(g.integers(0, 7))]
+                 dict(BN=208, cta_group=1, raster=1), dict(BN=128, BK=256, cta_group=1, stages=1), dict(cta_group=2, BN=80),
+                 dict(cta_group=2, BN=192, BK=128)][int(g.integers(0, 9))]
     epi = {}
     out = [rgo.BF16, rgo.F32, rgo.F16][int(g.integers(0, 3))]
     return M, N, K, f16, desc, knobs, out

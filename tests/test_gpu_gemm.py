@@ -43,7 +43,9 @@ def test_tiny_descriptor_check_full_oracle_compare():
                                    (7, 4096, 1024), (2000, 3000, 2048), (64, 100, 72)])
 @pytest.mark.parametrize("knobs", [dict(), dict(BN=64), dict(BN=128, BK=128), dict(BN=256, stages=2, raster=1),
                                    dict(cta_group=1, BN=256), dict(cta_group=2, BN=256, BK=64), dict(BM=256, BN=128, BK=128, raster=4),
-                                   dict(BN=112, BK=128), dict(BN=48, BK=256, cta_group=1), dict(BN=240, cta_group=1), dict(BN=16, cta_group=1)])
+                                   dict(BN=112, BK=128), dict(BN=48, BK=256, cta_group=1), dict(BN=240, cta_group=1), dict(BN=16, cta_group=1),
+                                   dict(cta_group=2, BN=32), dict(cta_group=2, BN=48, BK=128), dict(cta_group=2, BN=64, stages=2),
+                                   dict(cta_group=2, BN=112, BK=128, raster=1), dict(cta_group=2, BN=240)])
 def test_integer_inputs_exact(M, N, K, knobs):
     A = synth.int_valued_bf16((M, K), -8, 8, K + M); B = synth.int_valued_bf16((N, K), -8, 8, K + N + 1)
     assert_bits_equal(gpu_gemm(A, B, out_dtype=rgo.F32, **knobs), _exact_int(A, B), f"ints {M}x{N}x{K} {knobs}")
@@ -122,7 +124,7 @@ def test_position_independence_of_one_k_vector():
     A = np.repeat(a, 300, 0); B = np.repeat(b, 600, 0)
     vals = set()
     for knobs in (dict(BN=64), dict(BN=128), dict(BN=256), dict(BN=256, BK=128), dict(cta_group=2, BN=256), dict(cta_group=2, BN=128),
-                  dict(cta_group=1, BN=112, BK=256), dict(cta_group=1, BN=208)):
+                  dict(cta_group=1, BN=112, BK=256), dict(cta_group=1, BN=208), dict(cta_group=2, BN=48), dict(cta_group=2, BN=176, BK=128)):
         got = gpu_gemm(A, B, out_dtype=rgo.F32, **knobs)
         vals |= set(np.unique(got.view(np.uint32)).tolist())
     vals |= set(np.unique(gpu_gemm(A[:1], B[:5], out_dtype=rgo.F32).view(np.uint32)).tolist())
@@ -271,6 +273,7 @@ def test_large_square_all_tile_configs_agree_bitwise():
     configs += [dict(cta_group=2, BN=bn, BK=bk, stages=st, raster=ra) for bn in (128, 256) for bk in (64, 128)
                 for st in (0, 2) for ra in (0, 1, 16)]
     configs += [dict(cta_group=1, BN=bn, BK=bk) for bn in (112, 176, 240) for bk in (64, 256)]
+    configs += [dict(cta_group=2, BN=bn, BK=bk) for bn in (32, 64, 80, 160, 240) for bk in (64, 128)]
     keys = {rg.rg_desc_class(rg.rg_desc(**c)) for c in configs}
     assert len(keys) == 1
     ref = gpu_gemm(A, B, **configs[0])

@@ -21,7 +21,8 @@ def _draws(M, N, K, seed):
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 1, 32), (1, 8, 16), (3, 5, 48), (129, 65, 160), (300, 520, 1000), (513, 260, 2048)])
-@pytest.mark.parametrize("knobs", [dict(), dict(BN=64), dict(cta_group=2, BN=128), dict(BN=48, cta_group=1), dict(BN=256, BK=128, stages=2)])
+@pytest.mark.parametrize("knobs", [dict(), dict(BN=64), dict(cta_group=2, BN=128), dict(BN=48, cta_group=1), dict(BN=256, BK=128, stages=2),
+                                   dict(cta_group=2, BN=64), dict(cta_group=2, BN=208, BK=128)])
 def test_integer_inputs_exact(M, N, K, knobs):
     A = synth.int_valued_f8e4m3((M, K), -8, 8, 1 + K); B = synth.int_valued_f8e4m3((N, K), -8, 8, 2 + K)
     want = (synth.f8e4m3_bits_to_f32(A).astype(np.int64) @ synth.f8e4m3_bits_to_f32(B).astype(np.int64).T).astype(np.float32)
