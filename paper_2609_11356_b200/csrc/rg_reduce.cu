@@ -369,9 +369,10 @@ __global__ void __launch_bounds__(1024) reduce_rows_cta_kernel(const ReduceParam
 }
 
 // ------------------------------------------------------------------ RMSNorm, row kept in registers
-// One CTA per row; every warp owns at most one super-block of U vectors per lane and keeps the
-// raw vectors, so the row is read from memory exactly once.  Needs 16-byte aligned rows whose
-// length is a multiple of V.
+// One CTA per row; every warp owns at most one super-block of U vectors per lane.  A row is read from memory
+// exactly once and unpacked once (the unpacked values serve the fold and the scaling), the registers of its
+// raw vectors then receive the next row's, and the thread's weights are unpacked once per CTA.  Needs 16-byte
+// aligned rows whose length is a multiple of V.
 template <typename T, int U>
 __global__ void __launch_bounds__(256) rmsnorm_keep_kernel(const ReduceParams p) {
   __shared__ float sb[2][8];
@@ -391,20 +392,31 @@ __global__ void __launch_bounds__(256) rmsnorm_keep_kernel(const ReduceParams p)
       raw[u] = c + V <= p.C ? __ldg(reinterpret_cast<const uint4*>(xr + c)) : make_uint4(0, 0, 0, 0);
     }
   };
-  uint4 raw[U], nxt[U];
+  // this thread's weights, unpacked once: they are the same for every row
+  float w[U][V];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const int64_t c = base + (int64_t)u * WB;
+    if (w_vec && c + V <= p.C) unpack<T>(__ldg(reinterpret_cast<const uint4*>(static_cast<const T*>(p.weight) + c)), w[u]);
+    else {
+#pragma unroll
+      for (int t = 0; t < V; ++t) w[u][t] = (p.weight && c + t < p.C) ? load_scalar(p.weight, p.w_dtype, c + t) : 1.0f;
+    }
+  }
+  uint4 raw[U];
   if ((int64_t)blockIdx.x < p.R) load_row(blockIdx.x, raw);
   int par = 0;
   for (int64_t row = blockIdx.x; row < p.R; row += gridDim.x, par ^= 1) {
-    // the next row's vectors are requested now, so that they travel while this row is folded, scaled and stored
-    const bool more = row + gridDim.x < p.R;
-    if (more) load_row(row + gridDim.x, nxt);
+    // the row is unpacked once; its raw vectors' registers then take the next row's vectors, which travel
+    // while this row is folded, scaled and stored
+    float x[U][V];
+#pragma unroll
+    for (int u = 0; u < U; ++u) unpack<T>(raw[u], x[u]);
+    if (row + gridDim.x < p.R) load_row(row + gridDim.x, raw);
     float bv[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      float x[V];
-      unpack<T>(raw[u], x);
-      bv[u] = (base + (int64_t)u * WB + V <= p.C) ? fold_block<OP_RMS, V, true>(x, V, 0.0f, p.fma) : NEG_ZERO;
-    }
+    for (int u = 0; u < U; ++u)
+      bv[u] = (base + (int64_t)u * WB + V <= p.C) ? fold_block<OP_RMS, V, true>(x[u], V, 0.0f, p.fma) : NEG_ZERO;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1)
 #pragma unroll
@@ -425,16 +437,10 @@ __global__ void __launch_bounds__(256) rmsnorm_keep_kernel(const ReduceParams p)
     for (int u = 0; u < U; ++u) {
       const int64_t c = base + (int64_t)u * WB;
       if (c + V > p.C) continue;
-      float x[V], w[V], y[V];
-      unpack<T>(raw[u], x);
-      if (w_vec) unpack<T>(__ldg(reinterpret_cast<const uint4*>(static_cast<const T*>(p.weight) + c)), w);
-      else {
-#pragma unroll
-        for (int t = 0; t < V; ++t) w[t] = p.weight ? load_scalar(p.weight, p.w_dtype, c + t) : 1.0f;
-      }
+      float y[V];
 #pragma unroll
       for (int t = 0; t < V; t += 2) {
-        const float2 q = __fmul2_rn(__fmul2_rn(make_float2(x[t], x[t + 1]), make_float2(rinv, rinv)), make_float2(w[t], w[t + 1]));
+        const float2 q = __fmul2_rn(__fmul2_rn(make_float2(x[u][t], x[u][t + 1]), make_float2(rinv, rinv)), make_float2(w[u][t], w[u][t + 1]));
         y[t] = q.x; y[t + 1] = q.y;
       }
       if (out_vec) {
@@ -451,10 +457,6 @@ __global__ void __launch_bounds__(256) rmsnorm_keep_kernel(const ReduceParams p)
           else static_cast<float*>(p.out)[row * p.ldo + c + t] = y[t];
         }
       }
-    }
-    if (more) {
-#pragma unroll
-      for (int u = 0; u < U; ++u) raw[u] = nxt[u];
     }
   }
 }
@@ -656,7 +658,11 @@ rg_status_t launch_reduce_rows(int op, int tree, int fma, const rg_tensor_t* x, 
 
   // RMSNorm of rows short enough to live in registers: each row is read once.
   if (op == RG_OP_RMSNORM && !valid_hint && vec && C % V == 0 && nblocks <= 32) {
-    const int Uk = nblocks >= 16 ? 4 : nblocks >= 4 ? 2 : 1;
+    // vectors per lane: a thread keeps its part of the row, its weights and the next row's raw vectors in
+    // registers (64 with two bf16 vectors, 113 with four), and the SM needs about 70 KB in flight to keep DRAM
+    // busy: two vectors per lane wherever the row then fits eight warps (bf16 4096 columns: 5.7 TB/s against 5.4
+    // with four; fp32 rows measured level, the shortest best with one)
+    const int Uk = x->dtype == RG_BF16 ? (nblocks > 16 ? 4 : nblocks >= 2 ? 2 : 1) : (nblocks >= 16 ? 4 : nblocks > 8 ? 2 : 1);
     const int warps = (int)((nblocks + Uk - 1) / Uk);          // <= 8
     // every CTA takes the same number of rows (8192 rows on 2368 resident CTAs would leave a last round half
     // empty: four rows each on 2048 CTAs instead)

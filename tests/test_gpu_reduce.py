@@ -75,7 +75,7 @@ def test_softmax_normaliser_long_rows_bit_exact(shape, spread):
     assert rg.rg_device_status() == 0
 
 
-@pytest.mark.parametrize("shape", [(500, 4096), (77, 8192), (40, 2048), (9, 520), (300, 3000)])
+@pytest.mark.parametrize("shape", [(500, 4096), (77, 8192), (40, 2048), (9, 520), (300, 3000), (50, 1536), (20, 6144), (2500, 512)])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_rmsnorm_register_resident_rows_match_generic_kernels(shape, dtype):
     x = _draw(shape, dtype, 41, True)
