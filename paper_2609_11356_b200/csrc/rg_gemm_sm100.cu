@@ -391,31 +391,47 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, const int BN,
 // (tiles up to 256 columns: 128 running-sum registers, part of which the compiler keeps in local memory).
 template <int NCH> struct GroupedAcc { uint32_t v[NCH][32]; };
 
-template <int NCH>
-__device__ __forceinline__ void grouped_add(const GemmParams& p, const int BN, int tn, uint32_t taddr, int chunk0, bool first,
-                                            GroupedAcc<NCH>& acc) {
+// FIRST: the group that opens the running sum (a copy); the other groups are one add per element and nothing else.
+template <int NCH, bool FIRST, int CSTEP>
+__device__ __forceinline__ void grouped_add_t(const GemmParams& p, const int BN, int tn, uint32_t taddr, int chunk0, GroupedAcc<NCH>& acc) {
   const int col_end = min(p.N, (tn + 1) * BN);
 #pragma unroll
   for (int j = 0; j < NCH; ++j) {
-    const int c0 = (chunk0 + 2 * j) * 32;
+    const int c0 = (chunk0 + CSTEP * j) * 32;
     if (c0 < BN && tn * BN + c0 < col_end) {              // uniform across the warp
-      uint32_t r[32];
-      tmem_ld_32x32b_x32(taddr + c0, r);
-      tmem_ld_wait();
+      if (FIRST) {
+        tmem_ld_32x32b_x32(taddr + c0, acc.v[j]);
+        tmem_ld_wait();
+      } else {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(taddr + c0, r);
+        tmem_ld_wait();
+        // two adds per instruction (a packed add rounds each half like the scalar add; it feeds no multiply here)
 #pragma unroll
-      for (int c = 0; c < 32; ++c)
-        acc.v[j][c] = first ? r[c] : __float_as_uint(f_add(__uint_as_float(acc.v[j][c]), __uint_as_float(r[c])));
+        for (int c = 0; c < 32; c += 2) {
+          const float2 q = __fadd2_rn(make_float2(__uint_as_float(acc.v[j][c]), __uint_as_float(acc.v[j][c + 1])),
+                                      make_float2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])));
+          acc.v[j][c] = __float_as_uint(q.x); acc.v[j][c + 1] = __float_as_uint(q.y);
+        }
+      }
     }
   }
 }
+// CSTEP: the warp's chunks are chunk0, chunk0 + CSTEP, ... (CSTEP = epilogue warps per lane quarter)
+template <int NCH, int CSTEP = 2>
+__device__ __forceinline__ void grouped_add(const GemmParams& p, const int BN, int tn, uint32_t taddr, int chunk0, bool first,
+                                            GroupedAcc<NCH>& acc) {
+  if (first) grouped_add_t<NCH, true, CSTEP>(p, BN, tn, taddr, chunk0, acc);      // uniform across the warp
+  else grouped_add_t<NCH, false, CSTEP>(p, BN, tn, taddr, chunk0, acc);
+}
 
-template <int NCH>
+template <int NCH, int CSTEP = 2>
 __device__ __forceinline__ void grouped_finish(const GemmParams& p, const int BN, int part, int64_t row, bool row_ok, int tn,
                                                int chunk0, const GroupedAcc<NCH>& acc) {
   const int col_end = min(p.N, (tn + 1) * BN);
 #pragma unroll
   for (int j = 0; j < NCH; ++j) {
-    const int c0 = (chunk0 + 2 * j) * 32;
+    const int c0 = (chunk0 + CSTEP * j) * 32;
     const int col0 = tn * BN + c0;
     if (c0 < BN && col0 < col_end && row_ok) epilogue_store_chunk(p, part, row, col0, min(32, col_end - col0), acc.v[j]);
   }
@@ -517,7 +533,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t STAGE_BYTES = KSUB * (A_BOX_BYTES + B_BOX_BYTES);
   // Accumulators in tensor memory: two, or four for the second cut level on tiles up to 128 columns (its
   // groups are short, and more of them in flight hide the hand-over between the issuing warp and the epilogue)
-  constexpr int NB = (GROUPED && NCH == 2) ? 4 : 2;
+  constexpr int NB = (GROUPED && NCH <= 2) ? 4 : 2;
   const uint32_t TMEM_COLS = p.tmem_cols;                // a power of two >= 32; accumulator b starts at column b * TMEM_COLS / NB
   const uint32_t ACC_STRIDE = TMEM_COLS / NB;
   const uint32_t IDESC = p.idesc;
@@ -736,7 +752,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
               }
             }
           }
-          if (leader) umma_commit(bar_empty + 8u * stage);   // stage reusable once these steps have read it
+          // stage reusable once these steps have read it (with the second cut level a group's last stage could be
+          // released by the epilogue when it sees the group's accumulator complete, which saves this thread one of
+          // its two commits per group: built and measured, 739 against 763 TFLOP/s at a group every 64 k; dropped)
+          if (leader) umma_commit(bar_empty + 8u * stage);
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
         if (alive) { if (leader) umma_commit(bar_tfull + 8u * buf); ++gc; }   // last (or only) accumulator complete
@@ -885,7 +904,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
         ++gc;
-      } else if (EPI_WARPS == 8) {                          // the second cut level runs with eight epilogue warps
+      } else if (EPI_WARPS >= 8) {                          // the second cut level runs with eight or sixteen epilogue warps
         GroupedAcc<NCH> acc;
         for (int g = 0; g < ngroups && alive; ++g, ++gc) {
           const int buf = gc % NB;
@@ -893,12 +912,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           tcgen05_fence_after();
           if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * ACC_STRIDE;
-          grouped_add(p, BN, tn, taddr, chunk0, g == 0, acc);
+          grouped_add<NCH, EPI_WARPS / 4>(p, BN, tn, taddr, chunk0, g == 0, acc);
           tcgen05_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
         }
-        if (alive) grouped_finish(p, BN, part, row, row_ok, tn, chunk0, acc);
+        if (alive) grouped_finish<NCH, EPI_WARPS / 4>(p, BN, part, row, row_ok, tn, chunk0, acc);
       }
     }
   }
@@ -1614,20 +1633,22 @@ cudaError_t launch_ticket_t(const CUtensorMap& ta, const CUtensorMap& tb, const 
   return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<KSUB, F8, false, 8, false, 2, true>, ta, tb, p);
 }
 
-// the second cut level: 64-wide stages, eight epilogue warps; NCH = 32-column chunks a warp keeps a running sum of
-template <bool F8, int NCH>
+// the second cut level: 64-wide stages; NCH = 32-column chunks a warp keeps a running sum of.  Eight epilogue warps:
+// sixteen with one chunk each measured 8 % slower (702 against 763 TFLOP/s at a group every 64 k): the issuing
+// thread paces this mode, and more polling warps take its issue slots.
+template <bool F8, int NCH, int EPI = 8>
 cudaError_t launch_grouped_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
   const size_t smem = smem_bytes_for(p.bn, 1, p.num_stages, (int)(p.a_box_bytes / (KBOX * 2)));
   static DeviceOnce configured;
   const int dev = current_device().dev;
   if (!configured.has(dev)) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<1, F8, false, 8, true, NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<1, F8, false, EPI, true, NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
     if (e != cudaSuccess) return e;
     configured.set(dev);
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid, 1, 1);
-  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.blockDim = dim3(64 + 32 * EPI, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -1635,7 +1656,7 @@ cudaError_t launch_grouped_t(const CUtensorMap& ta, const CUtensorMap& tb, const
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<1, F8, false, 8, true, NCH>, ta, tb, p);
+  return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<1, F8, false, EPI, true, NCH>, ta, tb, p);
 }
 
 template <int KSUB>
