@@ -313,6 +313,19 @@ rg_status_t rg_gemm_noalloc(const rg_desc_t* d, const rg_tensor_t* A, const rg_t
 #define RG_SELFTEST_WAIT_CODE 0xE00u
 rg_status_t rg_selftest_bounded_wait(uint64_t limit_ns, uint32_t* dev_counter, void* cuda_stream);
 
+/* Self-test of the exponentials.  The paper's attention kernel calls the hardware's base-two exponential
+ * (App. F), whose bits are not defined off the GPU; this library fixes exp and exp2 as sequences of IEEE
+ * operations instead (rg_exp, rg_exp2), and its kernels use forms of them with the range selects removed where an
+ * argument's range is known.  y[i] = FORM(x[i]), computed on the device by the very functions the kernels call,
+ * so that every form can be compared with the CPU oracle directly rather than through a reduction:
+ *   0 rg_exp            1 rg_exp2            2 the GEMM epilogue's form of rg_exp for |x| <= 87
+ *   3 the attention kernel's packed (fp32x2) form of rg_exp for -87.33655 <= x <= 0
+ *   4 the attention kernel's form of rg_exp2 for -126 <= x <= 0      5 its form of rg_exp2 for x <= 0 or NaN
+ *   6 the softmax normaliser's form of rg_exp for x <= 0 or NaN
+ * Outside a form's stated range its result is unspecified.  x, y: DEVICE pointers to n floats (n >= 0, may
+ * alias).  RG_ERR_SHAPE for another form or n < 0.  Asynchronous on `cuda_stream`. */
+rg_status_t rg_selftest_exp(int32_t form, const float* x, float* y, int64_t n, void* cuda_stream);
+
 /* Device-side health word of the current device.  Every wait inside the kernels is bounded; a
  * wait that gives up records a code here, lets the kernel drain and return, and leaves the
  * context usable.  Copies the word to *code (0 = healthy) and clears it.  Synchronises the

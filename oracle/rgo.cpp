@@ -547,6 +547,10 @@ float rgo_mul_f32(float a, float b) { return a * b; }
 float rgo_expf(float x) { return rg_expf(x); }
 float rgo_exp2f(float x) { return rg_exp2f(x); }
 float rgo_silu(float x) { return silu(x); }
+// the same two functions over an array (a loop around the scalar definitions, for the tests' sake)
+void rgo_exp_array(const float* x, float* y, int64_t n, int base2) {
+  for (int64_t i = 0; i < n; ++i) y[i] = base2 ? rg_exp2f(x[i]) : rg_expf(x[i]);
+}
 
 // Tree-reduce n fp32 values (input is not modified).
 float rgo_tree_sum(const float* v, int64_t n, int tree) {

@@ -117,6 +117,7 @@ def lib():
         L.rgo_reduce_rows.argtypes = [i32, i32, i32, vp, i32, i64, i64, i64, vp, i32, i64, vp, i32, f32, vp]
         L.rgo_attention.restype = None
         L.rgo_exp2f.restype = f32; L.rgo_exp2f.argtypes = [f32]
+        L.rgo_exp_array.restype = None; L.rgo_exp_array.argtypes = [vp, vp, i64, i32]
         L.rgo_attention.argtypes = [C.POINTER(_AtomStruct), i32, i32, i32, i32, i32, i32, f32, i64, i64, i64, vp, i64, vp, i64, vp, i64, vp, i32, i64]
         L.rgo_reduce_cols.restype = None
         L.rgo_reduce_cols.argtypes = [i32, i32, i32, vp, i32, vp, i32, i64, i64, i64, i64, vp]
@@ -159,6 +160,14 @@ def add_f32(a, b) -> np.float32:
 
 def mul_f32(a, b) -> np.float32:
     return np.float32(lib().rgo_mul_f32(np.float32(a), np.float32(b)))
+
+
+def exp_array(x: np.ndarray, base2: bool = False) -> np.ndarray:
+    """The specified exponential (base e, or base two) of every element: a loop around `expf` / `exp2f`."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    y = np.empty_like(x)
+    lib().rgo_exp_array(_ptr(x), _ptr(y), x.size, 1 if base2 else 0)
+    return y
 
 
 def expf(x) -> np.float32:

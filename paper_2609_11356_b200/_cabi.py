@@ -27,7 +27,7 @@ RG_SELFTEST_WAIT_CODE = 0xE00
 EXPORTS = ["rg_desc_init", "rg_desc_validate", "rg_desc_class", "rg_gemm_workspace_bytes", "rg_gemm",
            "rg_reduce_rows", "rg_gemm_host_scratch_bytes", "rg_gemm_host", "rg_reduce_rows_host_scratch_bytes",
            "rg_reduce_rows_host", "rg_device_status", "rg_status_string", "rg_gemm_noalloc",
-           "rg_reduce_cols_workspace_bytes", "rg_reduce_cols", "rg_attention", "rg_selftest_bounded_wait"]
+           "rg_reduce_cols_workspace_bytes", "rg_reduce_cols", "rg_attention", "rg_selftest_bounded_wait", "rg_selftest_exp"]
 
 
 class rg_attn_desc_t(C.Structure):
@@ -89,6 +89,7 @@ def load():
     L.rg_attention.restype = C.c_int; L.rg_attention.argtypes = [C.POINTER(rg_attn_desc_t), T, T, T, T, vp]
     L.rg_gemm_noalloc.restype = C.c_int; L.rg_gemm_noalloc.argtypes = [D, T, T, T, E, vp]
     L.rg_selftest_bounded_wait.restype = C.c_int; L.rg_selftest_bounded_wait.argtypes = [C.c_uint64, vp, vp]
+    L.rg_selftest_exp.restype = C.c_int; L.rg_selftest_exp.argtypes = [C.c_int32, vp, vp, C.c_int64, vp]
     L.rg_device_status.restype = C.c_int; L.rg_device_status.argtypes = [C.POINTER(C.c_uint32)]
     L.rg_status_string.restype = C.c_char_p; L.rg_status_string.argtypes = [C.c_int]
     _lib = L

@@ -64,6 +64,13 @@ def rg_device_status() -> int:
     return int(code.value)
 
 
+def rg_selftest_exp(form: int, x, y):
+    """y[i] = FORM(x[i]) by the device functions the kernels use (forms: see include/rg.h).  x, y: float32 CUDA tensors."""
+    st = K.load().rg_selftest_exp(int(form), x.data_ptr(), y.data_ptr(), int(x.numel()), _stream(x))
+    _check(st, "rg_selftest_exp")
+    return y
+
+
 def rg_selftest_bounded_wait(limit_ns: int, counter):
     """Launch the bounded-wait self-test (see include/rg.h).  `counter`: a zeroed CUDA int32/uint32
     tensor of one element; it holds 2 afterwards (both warps abandoned their wait)."""

@@ -549,6 +549,14 @@ rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_
   return ok ? RG_OK : RG_ERR_CUDA;
 }
 
+rg_status_t rg_selftest_exp(int32_t form, const float* x, float* y, int64_t n, void* cuda_stream) {
+  if (form < 0 || form > 6 || n < 0) return RG_ERR_SHAPE;
+  if (n == 0) return RG_OK;
+  if (!x || !y) return RG_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  return (form >= 3 && form <= 5) ? rg::launch_exp_selftest_attention(form, x, y, n, st) : rg::launch_exp_selftest(form, x, y, n, st);
+}
+
 rg_status_t rg_selftest_bounded_wait(uint64_t limit_ns, uint32_t* dev_counter, void* cuda_stream) {
   if (!dev_counter) return RG_ERR_NULL;
   if (limit_ns < 1000ull || limit_ns > 100000000ull) return RG_ERR_SHAPE;     // 1 us .. 100 ms: never a long stall

@@ -181,10 +181,13 @@ __device__ __forceinline__ float exp_core(float x) {
 // issues half as many floating-point instructions per key in the polynomial.  Only chains of fused multiply-adds
 // are packed: a packed multiply feeding a packed add is contracted into one packed fma by the assembler even
 // when both carry an explicit rounding mode (measured: 1 % of such pairs change their last bit), so the
-// score scaling (multiply, then subtract the maximum) and the fold O = a * O + PV stay scalar.
+// score scaling (multiply, then subtract the maximum) and the fold O = a * O + PV stay scalar, and so does the
+// first multiply here: with y = x * log2(e) packed in front of the packed add that rounds it to an integer, 12 of
+// the 1,118,743,633 arguments of this form's domain came out with another n and other bits (an exhaustive
+// comparison with the scalar form; with the scalar multiply: none).  rg_selftest_exp exposes this function.
 __device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
 __device__ __forceinline__ float2 exp_core2(float2 x) {
-  const float2 y = __fmul2_rn(x, splat2(0x1.715476p+0f));
+  const float2 y = make_float2(f_mul(x.x, 0x1.715476p+0f), f_mul(x.y, 0x1.715476p+0f));
   const float2 t = __fadd2_rn(y, splat2(12582912.0f));
   const float2 n = __fadd2_rn(t, splat2(-12582912.0f));
   float2 r = __ffma2_rn(n, splat2(-0x1.62e400p-1f), x);
@@ -600,7 +603,27 @@ cudaError_t launch_attention(const CUtensorMap& tq, const CUtensorMap& tk, const
   return cudaGetLastError();
 }
 
+// y[i] = one of this file's range-restricted exponentials on x[i] (see rg_selftest_exp)
+__global__ void __launch_bounds__(256) exp_selftest_attention_kernel(int form, const float* __restrict__ x, float* __restrict__ y, int64_t n) {
+  for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 2; i < n; i += (int64_t)gridDim.x * blockDim.x * 2) {
+    const bool two = i + 1 < n;
+    const float a = x[i], b = two ? x[i + 1] : x[i];
+    float ra, rb;
+    if (form == 3) { const float2 e = exp_core2(make_float2(a, b)); ra = e.x; rb = e.y; }
+    else if (form == 4) { ra = exp2_core(a); rb = exp2_core(b); }
+    else { ra = exp2_nonpositive(a); rb = exp2_nonpositive(b); }
+    y[i] = ra;
+    if (two) y[i + 1] = rb;
+  }
+}
+
 }  // namespace
+
+rg_status_t launch_exp_selftest_attention(int form, const float* x, float* y, int64_t n, cudaStream_t st) {
+  const int64_t need = (n / 2 + 255) / 256 + 1;
+  exp_selftest_attention_kernel<<<(unsigned)(need < 148 * 8 ? need : 148 * 8), 256, 0, st>>>(form, x, y, n);
+  return cudaGetLastError() == cudaSuccess ? RG_OK : RG_ERR_CUDA;
+}
 
 // All arguments were validated by the caller: bf16 operands, d in {64, 128}, block_n in {64, 128},
 // 16-byte aligned pointers, leading dimensions multiples of 8.

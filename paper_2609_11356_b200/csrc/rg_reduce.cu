@@ -583,7 +583,21 @@ cudaError_t launch_op(int op, const ReduceParams& p, bool vec, bool wr, int U, i
   }
 }
 
+// y[i] = one of the specified exponentials on x[i] (see rg_selftest_exp)
+__global__ void __launch_bounds__(256) exp_selftest_kernel(int form, const float* __restrict__ x, float* __restrict__ y, int64_t n) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const float v = x[i];
+    y[i] = form == 0 ? rg_exp(v) : form == 1 ? rg_exp2(v) : form == 2 ? rg_exp_inrange(v) : exp_nonpositive(v);
+  }
+}
+
 }  // namespace
+
+rg_status_t launch_exp_selftest(int form, const float* x, float* y, int64_t n, cudaStream_t st) {
+  const int64_t need = (n + 255) / 256;
+  exp_selftest_kernel<<<(unsigned)(need < 148 * 8 ? need : 148 * 8), 256, 0, st>>>(form, x, y, n);
+  return cudaGetLastError() == cudaSuccess ? RG_OK : RG_ERR_CUDA;
+}
 
 // Host launcher.  Speed knobs only (0 = choose): threads_hint = threads per row, where 32 selects
 // the warp-per-row kernel for sums and RMSNorm; unroll_hint = warp-blocks in flight per warp.

@@ -155,3 +155,13 @@ def test_exp2f_accuracy_exact_powers_monotone_and_clamps():
     assert rgo.exp2f(-126.0) == np.float32(2.0 ** -126) and rgo.exp2f(np.float32(-126.00001)) == 0 and rgo.exp2f(-1e30) == 0
     assert rgo.exp2f(-np.inf) == 0 and np.isinf(rgo.exp2f(128.0)) and np.isinf(rgo.exp2f(np.inf)) and np.isnan(rgo.exp2f(np.nan))
     assert rgo.exp2f(np.float32(127.99999)) < np.inf
+
+
+def test_exp_array_is_the_scalar_functions_in_a_loop():
+    g = np.random.default_rng(9)
+    x = np.concatenate([g.uniform(-100, 100, 500), [0.0, -0.0, np.inf, -np.inf, np.nan, 88.8, -87.4, 128.0, -126.5]]).astype(np.float32)
+    for base2 in (False, True):
+        y = rgo.exp_array(x, base2)
+        for xi, yi in zip(x, y):
+            want = rgo.exp2f(xi) if base2 else rgo.expf(xi)
+            assert (np.isnan(yi) and np.isnan(want)) or np.float32(yi).view(np.uint32) == np.float32(want).view(np.uint32)
