@@ -322,8 +322,11 @@ rg_status_t rg_selftest_bounded_wait(uint64_t limit_ns, uint32_t* dev_counter, v
  *   3 the attention kernel's packed (fp32x2) form of rg_exp for -87.33655 <= x <= 0
  *   4 the attention kernel's form of rg_exp2 for -126 <= x <= 0      5 its form of rg_exp2 for x <= 0 or NaN
  *   6 the softmax normaliser's form of rg_exp for x <= 0 or NaN
+ *   7 the GEMM epilogue's SiLU, v / (1 + e^-v) with the specified exponential, applied as the kernels apply it: to segments of 32
+ *     consecutive values, with the range-free exponential when no magnitude of a segment exceeds 87 (n % 32 == 0)
  * Outside a form's stated range its result is unspecified.  x, y: DEVICE pointers to n floats (n >= 0, may
- * alias).  RG_ERR_SHAPE for another form or n < 0.  Asynchronous on `cuda_stream`. */
+ * alias).  RG_ERR_SHAPE for another form, n < 0, or form 7 with n not a multiple of 32.  Asynchronous on
+ * `cuda_stream`. */
 rg_status_t rg_selftest_exp(int32_t form, const float* x, float* y, int64_t n, void* cuda_stream);
 
 /* Device-side health word of the current device.  Every wait inside the kernels is bounded; a

@@ -551,6 +551,9 @@ float rgo_silu(float x) { return silu(x); }
 void rgo_exp_array(const float* x, float* y, int64_t n, int base2) {
   for (int64_t i = 0; i < n; ++i) y[i] = base2 ? rg_exp2f(x[i]) : rg_expf(x[i]);
 }
+void rgo_silu_array(const float* x, float* y, int64_t n) {
+  for (int64_t i = 0; i < n; ++i) y[i] = silu(x[i]);
+}
 
 // Tree-reduce n fp32 values (input is not modified).
 float rgo_tree_sum(const float* v, int64_t n, int tree) {

@@ -118,6 +118,7 @@ def lib():
         L.rgo_attention.restype = None
         L.rgo_exp2f.restype = f32; L.rgo_exp2f.argtypes = [f32]
         L.rgo_exp_array.restype = None; L.rgo_exp_array.argtypes = [vp, vp, i64, i32]
+        L.rgo_silu_array.restype = None; L.rgo_silu_array.argtypes = [vp, vp, i64]
         L.rgo_attention.argtypes = [C.POINTER(_AtomStruct), i32, i32, i32, i32, i32, i32, f32, i64, i64, i64, vp, i64, vp, i64, vp, i64, vp, i32, i64]
         L.rgo_reduce_cols.restype = None
         L.rgo_reduce_cols.argtypes = [i32, i32, i32, vp, i32, vp, i32, i64, i64, i64, i64, vp]
@@ -167,6 +168,14 @@ def exp_array(x: np.ndarray, base2: bool = False) -> np.ndarray:
     x = np.ascontiguousarray(x, dtype=np.float32)
     y = np.empty_like(x)
     lib().rgo_exp_array(_ptr(x), _ptr(y), x.size, 1 if base2 else 0)
+    return y
+
+
+def silu_array(x: np.ndarray) -> np.ndarray:
+    """The epilogue's activation v / (1 + exp(-v)) of every element: a loop around `silu`."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    y = np.empty_like(x)
+    lib().rgo_silu_array(_ptr(x), _ptr(y), x.size)
     return y
 
 

@@ -550,10 +550,11 @@ rg_status_t rg_reduce_rows_host(const rg_desc_t* d, rg_reduce_op_t op, const rg_
 }
 
 rg_status_t rg_selftest_exp(int32_t form, const float* x, float* y, int64_t n, void* cuda_stream) {
-  if (form < 0 || form > 6 || n < 0) return RG_ERR_SHAPE;
+  if (form < 0 || form > 7 || n < 0 || (form == 7 && n % 32 != 0)) return RG_ERR_SHAPE;
   if (n == 0) return RG_OK;
   if (!x || !y) return RG_ERR_NULL;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (form == 7) return rg::launch_silu_selftest(x, y, n, st);
   return (form >= 3 && form <= 5) ? rg::launch_exp_selftest_attention(form, x, y, n, st) : rg::launch_exp_selftest(form, x, y, n, st);
 }
 

@@ -1669,7 +1669,29 @@ cudaError_t launch_one_half(const CUtensorMap& ta, const CUtensorMap& tb, const 
   return p.f8 ? launch_one_t<KSUB, true, 4>(ta, tb, p, grid, st) : launch_one_t<KSUB, false, 4>(ta, tb, p, grid, st);
 }
 
+// The epilogue's SiLU as the kernels apply it: a thread takes 32 consecutive values (one accumulator chunk of one
+// row) through epilogue_row_segment, which picks the range-free exponential when no magnitude of the segment
+// exceeds 87 and the general one otherwise (see rg_selftest_exp, form 7).  n is a multiple of 32.
+__global__ void __launch_bounds__(128) silu_selftest_kernel(const float* __restrict__ x, float* __restrict__ y, int64_t n) {
+  EpilogueArgs e{};
+  e.act = 1;
+  for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s * 32 < n; s += (int64_t)gridDim.x * blockDim.x) {
+    float v[32];
+#pragma unroll
+    for (int c = 0; c < 32; ++c) v[c] = x[s * 32 + c];
+    epilogue_row_segment(v, e, 0, 0, 32);
+#pragma unroll
+    for (int c = 0; c < 32; ++c) y[s * 32 + c] = v[c];
+  }
+}
+
 }  // namespace
+
+rg_status_t launch_silu_selftest(const float* x, float* y, int64_t n, cudaStream_t st) {
+  const int64_t need = (n / 32 + 127) / 128;
+  silu_selftest_kernel<<<(unsigned)(need < 148 * 8 ? (need < 1 ? 1 : need) : 148 * 8), 128, 0, st>>>(x, y, n);
+  return cudaGetLastError() == cudaSuccess ? RG_OK : RG_ERR_CUDA;
+}
 
 // The same tensor map for other kernels of the library (boxes of 64 columns x box_rows rows, 128-byte swizzle).
 bool make_operand_tmap(CUtensorMap_st* map, const void* ptr, int dtype, int64_t rows, int64_t cols, int64_t ld, int box_rows) {

@@ -68,6 +68,7 @@ rg_status_t launch_wait_selftest(uint64_t limit_ns, uint32_t code, unsigned int*
 // y[i] = FORM(x[i]) by the device functions the kernels use (forms 0-2 and 6; the attention kernel's forms 3-5)
 rg_status_t launch_exp_selftest(int form, const float* x, float* y, int64_t n, cudaStream_t st);
 rg_status_t launch_exp_selftest_attention(int form, const float* x, float* y, int64_t n, cudaStream_t st);
+rg_status_t launch_silu_selftest(const float* x, float* y, int64_t n, cudaStream_t st);   // form 7: the epilogue's SiLU on segments of 32
 rg_status_t read_and_clear_reduce_status(uint32_t* code);
 
 }  // namespace rg

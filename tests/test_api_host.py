@@ -170,7 +170,8 @@ def test_selftest_arguments():
     assert L.rg_selftest_bounded_wait(1_000_000, None, None) == 1
     assert L.rg_selftest_bounded_wait(10, 0x1000, None) == 4              # below 1 us
     assert L.rg_selftest_bounded_wait(10**9, 0x1000, None) == 4           # above 100 ms: never a long stall
-    assert L.rg_selftest_exp(7, 0x1000, 0x2000, 4, None) == 4             # no such form
+    assert L.rg_selftest_exp(8, 0x1000, 0x2000, 4, None) == 4             # no such form
+    assert L.rg_selftest_exp(7, 0x1000, 0x2000, 33, None) == 4            # SiLU segments are 32 wide
     assert L.rg_selftest_exp(-1, 0x1000, 0x2000, 4, None) == 4
     assert L.rg_selftest_exp(0, 0x1000, 0x2000, -1, None) == 4
     assert L.rg_selftest_exp(0, None, 0x2000, 4, None) == 1

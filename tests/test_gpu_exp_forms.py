@@ -90,10 +90,29 @@ def test_softmax_normaliser_form():
     assert_bits_equal(_run(6, neg), rgo.exp_array(neg.view(np.float32)), "base-e form for x <= 0 or NaN")
 
 
+def test_epilogue_silu_on_segments_of_32():
+    g = np.random.default_rng(8)
+    seg = []
+    seg.append(g.standard_normal((20000, 32)).astype(np.float32) * 3)                  # every magnitude small: range-free form
+    big = g.standard_normal((20000, 32)).astype(np.float32) * 3
+    big[np.arange(20000), g.integers(0, 32, 20000)] = (g.uniform(87.0, 200.0, 20000) * g.choice([-1, 1], 20000)).astype(np.float32)
+    seg.append(big)                                                                    # one magnitude above 87: general form
+    seg.append(_bits_between(0, 0xffffffff, 9)[: 32 * 20000].view(np.float32).reshape(-1, 32))   # anything, NaN and inf included
+    edge = np.zeros((8, 32), np.float32)
+    edge[0, :8] = [87.0, -87.0, 87.00001, -87.00001, 88.72284, -88.72284, 0.0, -0.0]
+    edge[1, :6] = [np.inf, -np.inf, np.nan, 1e-45, -1e-45, 3.4e38]
+    edge[2, :] = np.linspace(-20, 20, 32, dtype=np.float32)
+    seg.append(edge)
+    x = np.concatenate(seg).reshape(-1)
+    assert_bits_equal(_run(7, x.view(np.uint32)), rgo.silu_array(x), "epilogue SiLU")
+
+
 def test_arguments():
     x = torch.zeros(4, device=DEV)
     with pytest.raises(RgError):
-        rg_selftest_exp(7, x, x)
+        rg_selftest_exp(8, x, x)
+    with pytest.raises(RgError):
+        rg_selftest_exp(7, x, x)                  # SiLU segments are 32 wide
     rg_selftest_exp(0, x[:0], x[:0])              # nothing to do
     y = torch.empty_like(x)
     rg_selftest_exp(0, x, y); torch.cuda.synchronize()

@@ -165,3 +165,6 @@ def test_exp_array_is_the_scalar_functions_in_a_loop():
         for xi, yi in zip(x, y):
             want = rgo.exp2f(xi) if base2 else rgo.expf(xi)
             assert (np.isnan(yi) and np.isnan(want)) or np.float32(yi).view(np.uint32) == np.float32(want).view(np.uint32)
+    for xi, yi in zip(x, rgo.silu_array(x)):
+        want = rgo.silu(xi)
+        assert (np.isnan(yi) and np.isnan(want)) or np.float32(yi).view(np.uint32) == np.float32(want).view(np.uint32)
