@@ -67,6 +67,30 @@ __device__ __forceinline__ float rg_exp_inrange(float x) {
   return f_mul(p, __int_as_float((__float_as_int(t) << 23) + 0x3f800000));   // t's low mantissa bits hold n
 }
 
+// rg_exp_inrange(-v) for a pair of values with |v| <= 87, computed from v itself with packed fp32x2 instructions
+// where that is safe.  Rounding to nearest is symmetric in sign, so with n' = rint(v * log2 e) = -n and
+// r' = v - n' ln2 = -r every intermediate of rg_exp_inrange(-v) appears here with its sign flipped or not at
+// all changed: the Horner steps in r' take the coefficients with alternating signs, and 2^n is 2^-n'.  Same
+// bits as the scalar form.  The first multiply stays scalar: a packed multiply in front of the packed add that
+// rounds to an integer is fused with it by the assembler (another n on a few arguments in a billion).
+__device__ __forceinline__ float2 rg_exp_neg_inrange2(float2 v) {
+  const float2 y = make_float2(f_mul(v.x, 0x1.715476p+0f), f_mul(v.y, 0x1.715476p+0f));
+  const float2 t = __fadd2_rn(y, make_float2(12582912.0f, 12582912.0f));
+  const float2 n = __fadd2_rn(t, make_float2(-12582912.0f, -12582912.0f));
+  float2 r = __ffma2_rn(n, make_float2(-0x1.62e400p-1f, -0x1.62e400p-1f), v);
+  r = __ffma2_rn(n, make_float2(-0x1.7f7d1cp-20f, -0x1.7f7d1cp-20f), r);
+  float2 q = make_float2(-0x1.a01a02p-13f, -0x1.a01a02p-13f);                       // degree 7: odd, sign flipped
+  q = __ffma2_rn(q, r, make_float2(0x1.6c16c2p-10f, 0x1.6c16c2p-10f));
+  q = __ffma2_rn(q, r, make_float2(-0x1.111112p-7f, -0x1.111112p-7f));
+  q = __ffma2_rn(q, r, make_float2(0x1.555556p-5f, 0x1.555556p-5f));
+  q = __ffma2_rn(q, r, make_float2(-0x1.555556p-3f, -0x1.555556p-3f));
+  q = __ffma2_rn(q, r, make_float2(0.5f, 0.5f));
+  q = __ffma2_rn(q, r, make_float2(-1.0f, -1.0f));
+  q = __ffma2_rn(q, r, make_float2(1.0f, 1.0f));
+  // t's low mantissa bits hold n'; the scale is 2^-n'
+  return __fmul2_rn(q, make_float2(__int_as_float(0x3f800000 - (__float_as_int(t.x) << 23)), __int_as_float(0x3f800000 - (__float_as_int(t.y) << 23))));
+}
+
 // largest magnitude of three values; NaN if any of them is NaN (one instruction on this architecture)
 __device__ __forceinline__ float absmax3_nan(float a, float b, float c) {
   float r;

@@ -296,7 +296,10 @@ __device__ __forceinline__ void epilogue_row_segment(float (&v)[32], const Epilo
     amax = absmax3_nan(amax, v[31], v[31]);
     if (amax <= 87.0f) {
 #pragma unroll
-      for (int c = 0; c < 32; ++c) ex[c] = f_add(1.0f, rg_exp_inrange(-v[c]));
+      for (int c = 0; c < 32; c += 2) {
+        const float2 e2 = rg_exp_neg_inrange2(make_float2(v[c], v[c + 1]));
+        ex[c] = f_add(1.0f, e2.x); ex[c + 1] = f_add(1.0f, e2.y);
+      }
     } else {
 #pragma unroll
       for (int c = 0; c < 32; ++c) ex[c] = f_add(1.0f, rg_exp(-v[c]));
