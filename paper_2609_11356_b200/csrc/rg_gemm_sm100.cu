@@ -38,7 +38,16 @@ __device__ unsigned int g_status_word = 0;
 // library build has none of this): [launch % 8][CTA][what] in nanoseconds of the global timer.
 #ifdef RG_TIMELINE
 __device__ unsigned long long g_timeline[8][512][8];
-#define RG_STAMP(slot) do { if (blockIdx.x < 512) g_timeline[p.launch_seq & 7][blockIdx.x][slot] = globaltimer_ns(); } while (0)
+// a call, not inline code: the stamps must not change the kernels' register counts (what fits beside what on an
+// SM decides when the launch behind a kernel becomes resident, which is what the stamps are there to show)
+static __device__ __noinline__ void rg_stamp(int seq, int slot) {
+  if (blockIdx.x < 512) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    g_timeline[seq & 7][blockIdx.x][slot] = t;
+  }
+}
+#define RG_STAMP(slot) rg_stamp(p.launch_seq, slot)
 #else
 #define RG_STAMP(slot) do { } while (0)
 #endif

@@ -224,9 +224,7 @@ rg_status_t launch_gemv(const rg_desc_t* d, const rg_tensor_t* A, const rg_tenso
     e.residual = epi->residual; e.residual_dtype = epi->residual_dtype; e.ldr = epi->ldr;
   }
   p.epi = e;
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = current_device().sms;                     // looked up once per device
   constexpr int WARPS = GEMV_THREADS / 32;
   const int64_t need = ((int64_t)p.N + WARPS - 1) / WARPS, cap = (int64_t)sms * (2048 / GEMV_THREADS);
   const int grid = (int)(need < cap ? need : cap);
