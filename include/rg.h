@@ -80,9 +80,10 @@ typedef struct {
                              1 = by a second kernel, through the workspace; 2 = inside the GEMM kernel, by the CTAs
                              of a thread-block cluster over distributed shared memory (one launch, no workspace;
                              2..8 parts, one-CTA tiles; RG_ERR_UNSUPPORTED where it does not apply);
-                             3 = inside the GEMM kernel, by the CTA that stores a tile's last part: the parts go
-                             through the workspace, whose first bytes hold one ticket per tile (2..8 parts, one-CTA
-                             tiles).  The caller's PROMISE with 3: the workspace was zero-filled once (e.g. a
+                             3 = inside the GEMM kernel, through the workspace, whose first bytes hold one ticket per
+                             tile (2..8 parts, one-CTA tiles): by the tile's CTAs together when every part has a
+                             resident CTA of its own (no more work items than SMs: they wait for each other, with the
+                             library's bounded wait), else by the CTA that stores the tile's last part.  The caller's PROMISE with 3: the workspace was zero-filled once (e.g. a
                              cudaMemset when it was allocated) and only calls of this library with split_merge = 3
                              have written it since; every such call leaves the tickets zero again.  After an
                              RG_ERR_TIMEOUT from rg_device_status, zero it again */

@@ -172,10 +172,16 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
     // legal tile width, so pick the one that wastes the least of the last round.
     int best = 128; int64_t best_cost = -1;
     // Without cuts a tile is one long chain of steps and narrow tiles keep every SM busy: down to 32 columns.
-    for (int bn = plan->n_parts == 1 ? 32 : 64; bn <= (half ? 128 : 256); bn += 16) {
-      const int64_t items = ((N + bn - 1) / bn) * plan->n_parts;
-      const int64_t cost = ((items + slots - 1) / slots) * bn;
-      if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
+    // The merge by the tile's own CTAs (split_merge = 3) wants one round: every part of a tile on a resident CTA of its
+    // own, so that the tile's CTAs can wait for each other and share the merge.  Widths that need a second round
+    // are considered for it only if none fits one.
+    for (int pass = plan->ticket_merge ? 0 : 1; pass < 2 && best_cost < 0; ++pass) {
+      for (int bn = plan->n_parts == 1 ? 32 : 64; bn <= (half ? 128 : 256); bn += 16) {
+        const int64_t items = ((N + bn - 1) / bn) * plan->n_parts;
+        if (pass == 0 && items > slots) continue;
+        const int64_t cost = ((items + slots - 1) / slots) * bn;
+        if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
+      }
     }
     plan->BN = best;
   } else {

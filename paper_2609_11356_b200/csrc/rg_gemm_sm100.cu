@@ -258,6 +258,7 @@ struct GemmParams {
   int64_t ldw;
   int32_t ws_dtype;
   unsigned int* tickets;  // TICKET kernels: one counter per output tile (zero on entry, zero again on exit), else null
+  int32_t ticket_all;     // TICKET kernels: every work item has a CTA of its own (one round), so the CTAs of a tile may wait for each other
   // in-cluster merge (CLUSTER kernels): the n_parts CTAs of a cluster own the parts of one output tile
   int32_t tree, merge_dtype;   // how the parts are added (descriptor's tree, type of the running sum)
   int32_t part_rows;           // rows of a tile kept in a CTA's shared-memory partial buffer
@@ -529,9 +530,10 @@ __device__ __forceinline__ void finish_and_store4(const EpilogueArgs& e, void* C
 // the workspace; the CTA that stores a tile's LAST part (an integer ticket per tile, taken after a device-wide fence)
 // merges the tile from the workspace in the descriptor's tree, applies the epilogue and stores.  Nobody waits for
 // anybody: which CTA merges depends on timing, what it computes does not (Sec. 3.1: the tree, not the schedule).
-// Measured on the decode shape it does not pay: equal to the two-kernel path at 1 and 8 rows (24.7-26 us), 6 us
-// slower at 32 rows, where every CTA pays a device-wide fence and two barriers per item and the tiles' merges
-// (37 CTAs, one tile each, alone with their L2 latency) all fall at the end of the launch.  Kept as an option.
+// When the work items fit one round (p.ticket_all) the tile's CTAs wait for each other instead (bounded) and each
+// merges a slice of the tile.  Measured on the decode shape it does not pay: within 3 % of the two-kernel path at 1
+// and 8 rows, 2 us slower at 32 rows (27.7 against 25.6 us): part store, device-wide fence, ticket, the spread of the
+// tile's eight CTAs and one L2 round trip cost what the second launch costs.  Kept as an option.
 template <int KSUB, bool F8, bool CLUSTER, int EPI_WARPS, bool GROUPED = false, int NCH = 2, bool TICKET = false>
 __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, EPI_WARPS == 4 ? 3 : 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -867,6 +869,67 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         __threadfence();
         asm volatile("bar.sync 1, %0;" ::"n"(EPI_WARPS * 32) : "memory");
         const int tile = tm * p.tiles_n + tn;
+        if (p.ticket_all) {
+          // ---- one round of work items, each on a CTA of its own (all resident: one CTA per SM, no more items than
+          // SMs): the tile's CTAs wait until all of its parts are in the workspace, and each merges one slice of
+          // the tile, so that the merge after the last part is one L2 round trip of 256 threads per CTA, not the
+          // whole tile on the last arriver.  The counter goes up once per CTA on arrival and once on leaving; the
+          // CTA that brings it to twice the number of parts sets it back to zero (all have left their wait by then).
+          if (warp == 2 && lane == 0) {
+            volatile unsigned int* t = p.tickets + tile;
+            atomicAdd(p.tickets + tile, 1u);
+            bool ok = true;
+            uint64_t t0 = 0;
+            for (uint32_t it = 0; *t < (unsigned int)p.n_parts; ++it) {
+              __nanosleep(40);
+              if ((it & 63u) == 63u) {
+                if (*abort_flag) { ok = false; break; }
+                const uint64_t now = globaltimer_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; atomicCAS(&g_status_word, 0u, 0x700u); ok = false; break; }
+              }
+            }
+            if (ok) {
+              const unsigned int old = atomicAdd(p.tickets + tile, 1u);
+              if (old == (unsigned int)(2 * p.n_parts - 1)) *t = 0u;
+            }
+            *ticket_flag = ok ? 1 : 0;
+          }
+          asm volatile("bar.sync 1, %0;" ::"n"(EPI_WARPS * 32) : "memory");
+          if (*ticket_flag && alive) {
+            __threadfence();
+            const int tile_rows = min(BM, p.M - tm * BM);
+            const int c4s = BN >> 2;
+            const int units = tile_rows * c4s;
+            const int per = (units + p.n_parts - 1) / p.n_parts;
+            const int u_end = min(units, (part + 1) * per);
+            const int64_t part_stride = (int64_t)p.M * p.ldw;
+            for (int u = part * per + (warp - 2) * 32 + lane; u < u_end; u += EPI_WARPS * 32) {
+              const int r_t = u / c4s, c4 = u - r_t * c4s;
+              const int col0 = tn * BN + 4 * c4;
+              if (col0 >= p.N) continue;
+              const int64_t grow = (int64_t)tm * BM + r_t;
+              const int64_t off = grow * p.ldw + col0;
+              float4 v[8];
+#pragma unroll
+              for (int s2 = 0; s2 < 8; ++s2) {
+                if (s2 < p.n_parts) {
+                  if (p.ws_dtype == RG_F32) {
+                    v[s2] = __ldcg(reinterpret_cast<const float4*>(static_cast<const float*>(p.ws) + s2 * part_stride + off));
+                  } else {
+                    const uint2 w = __ldcg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.ws) + s2 * part_stride + off));
+                    v[s2] = p.ws_dtype == RG_F16 ? make_float4(f16_bits_to_f32(w.x & 0xffffu), f16_bits_to_f32(w.x >> 16), f16_bits_to_f32(w.y & 0xffffu), f16_bits_to_f32(w.y >> 16))
+                                                 : make_float4(bf16_bits_to_f32(w.x & 0xffffu), bf16_bits_to_f32(w.x >> 16), bf16_bits_to_f32(w.y & 0xffffu), bf16_bits_to_f32(w.y >> 16));
+                  }
+                }
+              }
+              const float4 acc = p.merge_dtype == RG_F32 ? merge_upto8<false>(v, p.n_parts, p.tree, p.merge_dtype)
+                                                          : merge_upto8<true>(v, p.n_parts, p.tree, p.merge_dtype);
+              finish_and_store4(p.epi, p.C, p.ldc, p.c_dtype, p.N, grow, col0, acc);
+            }
+          }
+          continue;
+        }
         if (warp == 2 && lane == 0) {
           const unsigned int old = atomicAdd(p.tickets + tile, 1u);
           const bool last = old == (unsigned int)(p.n_parts - 1);
@@ -1826,6 +1889,7 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   p.C = C->ptr; p.ldc = C->ld; p.c_dtype = C->dtype;
   // ticket mode: the tickets sit in front of the parts (see ticket_bytes)
   p.tickets = ticket ? static_cast<unsigned int*>(ws) : nullptr;
+  p.ticket_all = 0;                                           // set below, once the number of work items is known
   p.ws = split ? (ticket ? static_cast<void*>(static_cast<uint8_t*>(ws) + ticket_bytes()) : ws) : nullptr;
   p.ws_dtype = plan.partial_dtype;
   p.ldw = (N + 3) / 4 * 4;
@@ -1871,6 +1935,7 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
   } else if (ticket) {
     if ((size_t)p.tiles_m * (size_t)p.tiles_n > TICKET_TILES_MAX) return RG_ERR_UNSUPPORTED;   // more tiles than tickets
     const int grid = (int)(total < sms ? total : sms);
+    p.ticket_all = total <= sms ? 1 : 0;                     // one round: every part of a tile has a resident CTA
     if (ksub == 1) err = p.f8 ? launch_ticket_t<1, true>(ta, tb, p, grid, st) : launch_ticket_t<1, false>(ta, tb, p, grid, st);
     else if (ksub == 2) err = p.f8 ? launch_ticket_t<2, true>(ta, tb, p, grid, st) : launch_ticket_t<2, false>(ta, tb, p, grid, st);
     else return RG_ERR_UNSUPPORTED;

@@ -181,9 +181,19 @@ def test_last_arriver_merge_reuses_its_workspace_and_leaves_the_tickets_zero():
         torch.cuda.synchronize()
         assert_bits_equal(synth.from_torch(out), two, f"decode shape, call {call}")
         assert int(ws[:tickets].max().item()) == 0, "tickets not back at zero"
+    # the same problem on narrow tiles: 512 work items, more than one round, so nobody may wait for anybody and the
+    # CTA that stores a tile's last part merges it alone (the default width above is one round: the tile's CTAs share it)
+    d64 = rg.rg_desc(cuts=cuts8, split_merge=LAST_ARRIVER, BN=64)
+    for call in range(2):
+        out = torch.empty((32, 4096), dtype=torch.bfloat16, device=DEV); out.view(torch.int16).fill_(-1)
+        rg.rg_gemm(d64, At, Bt, out, residual=Rt, ws=ws)
+        torch.cuda.synchronize()
+        assert_bits_equal(synth.from_torch(out), two, f"decode shape on 64-wide tiles, call {call}")
+        assert int(ws[:tickets].max().item()) == 0, "tickets not back at zero"
     # other shapes, tilings and part counts on the same (never re-zeroed) workspace
     for M, N, K, cuts, knobs in ((8, 1003, 1000, (256, 512, 768), dict(BN=48)), (37, 520, 2304, (768, 1536), dict(BN=112, BK=64)),
-                                 (128, 260, 1024, (512,), dict(BN=64)), (300, 200, 2048, (512, 1024, 1536), dict(BN=128))):
+                                 (128, 260, 1024, (512,), dict(BN=64)), (300, 200, 2048, (512, 1024, 1536), dict(BN=128)),
+                                 (70, 2100, 1024, (256, 512, 768), dict(BN=32))):     # 264 work items: two rounds
         A2, B2 = _inputs(M, N, K, 60 + M)
         bias = synth.uniform_bf16((N,), -0.1, 0.1, 8)
         d2 = rg.rg_desc(cuts=cuts, split_merge=LAST_ARRIVER, **knobs)
