@@ -34,7 +34,7 @@ WORKLOAD = ("configs[4] large square 8192^3 + reduction stress 65536x32768 fp32,
 # summarised in profiles/kernels_ncu_full.md.  The GEMM figure is a capture of the full 8192^3 launch
 # (algorithmic minimum 0.403 GB: the excess is B re-streamed once per group of tile rows; 1.21-1.35 GB from capture to capture).  The row-sum
 # figure is the 16384-row capture scaled by 4 to the bench's 65536 rows (traffic is proportional to rows).
-NCU_TRAFFIC_BYTES = {"gemm_8192": 1.0914e9 + 0.1277e9, "row_sum_65536x32768": 4 * (2.1475e9 + 0.0038e9)}
+NCU_TRAFFIC_BYTES = {"gemm_8192": 1.0865e9 + 0.1276e9, "row_sum_65536x32768": 4 * (2.1475e9 + 0.0038e9)}
 
 GEMMS = {  # name: (M, N, K)
     "square": (8192, 8192, 8192),
