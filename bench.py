@@ -622,6 +622,8 @@ def run_only(args):
         bias = synth.device_uniform((N,), -0.1, 0.1, 8, bf, dev) if name == "gemm_prefill" else None
         if args.inner_span:
             d = rg.rg_desc(inner_span=args.inner_span, BN=args.bn, cta_group=args.cta_group)
+        elif args.raster:
+            d = rg.rg_desc(raster=args.raster)
         fn = lambda: rg.rg_gemm(d, A, B, Cm, bias=bias, act=1 if bias is not None else 0)
         work, unit = 2.0 * M * N * K / 1e12, "TFLOP/s"
     elif name == "gemm_square_f8":
@@ -727,6 +729,7 @@ def main():
     ap.add_argument("--b-static", type=int, default=0, help="--only gemm_decode: 1 = promise that the weights are not written by work in flight")
     ap.add_argument("--inner-span", type=int, default=0, help="--only gemm_square: second cut level (an accumulator closed every so many k)")
     ap.add_argument("--cta-group", type=int, default=0, help="--only gemm_square with --inner-span: 1 one-CTA tiles, 2 two-SM tiles")
+    ap.add_argument("--raster", type=int, default=0, help="--only gemm_square / gemm_prefill: tile walk (0 library's choice, 1 row-major, n = groups of n tile rows)")
     ap.add_argument("--stages", type=int, default=0, help="--only gemm_decode: ring depth (0 = as many as fit)")
     ap.add_argument("--attn-block", type=int, default=128, help="key block width for --only attention")
     ap.add_argument("--attn-causal", type=int, default=0, help="1: causal masking, for --only attention (flops counted as half)")
