@@ -418,3 +418,26 @@ def test_inner_span_groups_bit_exact():
     for bad in (dict(inner_span=40), dict(inner_span=8), dict(inner_span=64, BK=128), dict(inner_span=64, cta_group=2, BK=128)):
         assert rg.rg_desc_validate(rg.rg_desc(**bad), 64, 256, 512) == 3
     assert rg.rg_device_status() == 0
+
+
+# ------------------------------------------------------------------ the planner's choices are speed knobs
+@pytest.mark.parametrize("seed", range(48))
+def test_library_chosen_tiles_on_random_shapes_equal_a_fixed_tile(seed):
+    """Whatever kernel, tile width and stage width the planner picks for a shape (one-CTA tiles of any multiple of
+    16 columns, two-SM tiles of any width from 32, 64- to 256-wide K stages), the bits are those of one fixed
+    configuration of the same class, and sampled elements are the oracle's."""
+    g = np.random.default_rng(7000 + seed)
+    M = int(g.choice([g.integers(1, 130), g.integers(129, 600), g.integers(600, 2600)]))
+    N = int(g.choice([g.integers(8, 300), g.integers(300, 2100), g.integers(2100, 6200)]))
+    K = int(g.choice([64, 80, 256, 520, 1000, 1024, 2048, 4096]))
+    A = synth.device_normal((M, K), 1.0, 100 + seed, torch.bfloat16, DEV)
+    B = synth.device_normal((N, K), 1.0, 200 + seed, torch.bfloat16, DEV)
+    ref = gpu_gemm(A, B, out_dtype=rgo.F32, cta_group=1, BN=128, BK=64)
+    assert_bits_equal(gpu_gemm(A, B, out_dtype=rgo.F32), ref, f"library's choice for {M}x{N}x{K}")
+    if M > 128:
+        bn = int(g.choice(np.arange(32, 257, 16)))
+        assert_bits_equal(gpu_gemm(A, B, out_dtype=rgo.F32, cta_group=2, BN=bn, BK=int(g.choice([64, 128]))), ref, f"two-SM tiles of {bn} columns, {M}x{N}x{K}")
+    si, sj = g.integers(0, M, 24), g.integers(0, N, 24)
+    want = rgo.gemm_samples(synth.from_torch(A), synth.from_torch(B), si, sj, atom_model=HW, out_dtype=rgo.F32)
+    assert_bits_equal(ref[si, sj], want, f"sampled oracle {M}x{N}x{K}")
+    assert rg.rg_device_status() == 0
