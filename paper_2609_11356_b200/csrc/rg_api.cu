@@ -259,7 +259,16 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   plan->stages = d->stages ? d->stages : smax;
   if (plan->stages > smax) return RG_ERR_UNSUPPORTED;
   plan->raster = d->raster == 1 ? 1 : 0;
-  plan->group_m = d->raster >= 2 ? d->raster : 8;
+  // Tile walk: groups of group_m tile rows, column by column inside a group.  A B tile is then fetched once per group
+  // (the group's tiles of that column run together) and the group's A rows are read again for every column, which
+  // costs nothing while they stay in L2: the tallest group whose A rows take no more than about 56 MiB of it, as a
+  // power of two from 4 to 32 (8192^3 and K = 14336: 8; K = 4096 or e4m3 operands at K = 8192: 16, +2 %; K = 2048: 32, +2 %).
+  {
+    const int64_t row_bytes = (int64_t)(plan->cta_group == 2 ? 256 : 128) * K * (d->in_dtype == RG_F8E4M3 ? 1 : 2);
+    int g = 32;
+    while (g > 4 && (int64_t)g * row_bytes > ((int64_t)56 << 20)) g >>= 1;
+    plan->group_m = d->raster >= 2 ? d->raster : g;
+  }
   return RG_OK;
 }
 
