@@ -646,6 +646,19 @@ def run_only(args):
             it[0] += 1
             rg.rg_gemm(d, A, Ws[it[0] % 4], Cm, residual=R, ws=ws)
         work, unit = 2.0 * N * K / 1e9, "GB/s (weights)"
+    elif name == "gemm_mid":
+        # the batch-invariance shape in the regime between weight streaming and tensor bound: N = K = 4096 weights in
+        # rotation (above L2), --rows rows (default 768), the library's choice of kernel and tile or --cta-group / --bn / --bk
+        M, N, K = args.rows or 768, 4096, 4096
+        d = rg.rg_desc(cta_group=args.cta_group, BN=args.bn, BK=args.bk)
+        A = synth.device_normal((M, K), 1.0, 4, bf, dev)
+        Ws = [synth.device_normal((N, K), 0.02, 3 + i, bf, dev) for i in range(10)]
+        Cm = torch.empty((M, N), dtype=bf, device=dev)
+        it = [0]
+        def fn():
+            it[0] += 1
+            rg.rg_gemm(d, A, Ws[it[0] % 10], Cm)
+        work, unit = 2.0 * M * N * K / 1e12, "TFLOP/s"
     elif name == "gemv_decode":
         # the lane-tree GEMV class on the decode weight shape, one to four rows
         _, N, K = GEMMS["decode"]
@@ -697,7 +710,7 @@ def run_only(args):
         fn()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if name in ("gemm_decode", "gemv_decode"):
+    if name in ("gemm_decode", "gemv_decode", "gemm_mid"):
         # launches of tens of microseconds: keep the stream busy while the host queues them, so
         # the events bracket device time and not the host's launch rate
         filler = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
@@ -718,7 +731,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_square_f8", "gemm_prefill", "gemm_decode", "gemv_decode", "attention", "col_sum", "col_dot", "row_sum", "softmax", "softmax_unit", "rmsnorm"],
+    ap.add_argument("--only", default=None, choices=["gemm_square", "gemm_square_f8", "gemm_prefill", "gemm_decode", "gemm_mid", "gemv_decode", "attention", "col_sum", "col_dot", "row_sum", "softmax", "softmax_unit", "rmsnorm"],
                     help="run one kernel on a small case (used for the ncu captures)")
     ap.add_argument("--gemv-rows", type=int, default=1, help="rows of A for --only gemv_decode")
     ap.add_argument("--rows", type=int, default=0, help="rows of A for --only gemm_decode (default 32)")
