@@ -118,7 +118,10 @@ typedef struct {
                              CTAs of the next launch become resident beside it while it finishes */
   uint8_t b_static;       /* 1 = the caller promises that no work still in flight on the stream when this call is
                              enqueued writes B (weights in an inference loop): the kernel may fetch its first B boxes
-                             before the kernels ahead of it have finished.  A is never read early.  0 = no promise */
+                             before the kernels ahead of it have finished (A is not read early).  2 = the same
+                             promise for A and B (calls that share an input, or whose input was complete before the work
+                             now in flight was enqueued): no load of the call waits for the kernels ahead; its stores to
+                             C and to the workspace still do.  0 = no promise */
 } rg_desc_t;
 
 /* A row-major matrix in device memory. */

@@ -54,7 +54,7 @@ rg_status_t check_desc_supported(const rg_desc_t* d) {
     return RG_ERR_UNSUPPORTED;
   if (d->cta_group == 1 && d->BM == 256) return RG_ERR_UNSUPPORTED;
   if (d->raster > 64) return RG_ERR_INVALID_DESC;
-  if (d->split_merge > 3 || d->sm_share > 2 || d->b_static > 1) return RG_ERR_INVALID_DESC;
+  if (d->split_merge > 3 || d->sm_share > 2 || d->b_static > 2) return RG_ERR_INVALID_DESC;
   // the last-arriver merge: 2 to 8 parts, one-CTA tiles at a whole SM each, no second cut level
   if (d->split_merge == 3 && (d->n_cuts < 1 || d->n_cuts > 7 || d->inner_span || d->cta_group == 2 || d->BM == 256 || d->BK == 256 || d->sm_share == 2))
     return RG_ERR_UNSUPPORTED;
@@ -143,7 +143,7 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   plan->cluster_merge = 0;
   plan->ticket_merge = d->split_merge == 3 ? 1 : 0;
   plan->half_sm = 0;
-  plan->b_static = d->b_static ? 1 : 0;
+  plan->b_static = d->b_static;
   plan->tree = d->tree;
   plan->partial_dtype = d->partial_dtype;
   plan->merge_dtype = d->merge_dtype;

@@ -649,7 +649,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             if (!mbar_wait(bar_empty + 8u * stage, phase ^ 1u, abort_flag, &g_status_word, 0x100u | stage)) { alive = false; break; }
             if (lane == 0) mbar_expect_tx(full, STAGE_BYTES);
           }
-          if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; if (lane == 0) RG_STAMP(2); }
+          // (b_static = 2: A is not written by work in flight either, so no load of this launch waits; its stores do)
+          if (!deps_done && p.b_static < 2) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; if (lane == 0) RG_STAMP(2); }
           if (!ahead || !is_b) tma_load_2d(smem_base + stage * STAGE_BYTES + box_off, map, k0 + sub * KBOX, y, full);
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
@@ -1091,8 +1092,9 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       int stage = 0; uint32_t phase = 0;
       bool alive = true;
       // launched with programmatic stream serialisation like the one-CTA kernel: the kernels ahead in the stream
-      // are waited for immediately before this role's first access to global memory
-      asm volatile("griddepcontrol.wait;" ::: "memory");
+      // are waited for immediately before this role's first access to global memory (not at all when neither operand
+      // is written by work in flight, b_static = 2: the epilogue still waits before its first store)
+      if (p.b_static < 2) asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int w = pair_id; w < total_work && alive; w += num_pairs) {
         int part, tm, tn;
         decode_work(p, w, part, tm, tn);

@@ -64,7 +64,8 @@ def test_validate_rules():
     assert rg.rg_desc_validate(rg.rg_desc(sm_share=2), 64, 256, 512) == 0
     assert rg.rg_desc_validate(rg.rg_desc(sm_share=2, BN=256), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(b_static=1), 64, 256, 512) == 0
-    assert rg.rg_desc_validate(rg.rg_desc(b_static=2), 64, 256, 512) == 2
+    assert rg.rg_desc_validate(rg.rg_desc(b_static=2), 64, 256, 512) == 0
+    assert rg.rg_desc_validate(rg.rg_desc(b_static=3), 64, 256, 512) == 2
     assert rg.rg_desc_validate(rg.rg_desc(in_dtype=K.RG_F8E4M3, partial_dtype=K.RG_F8E4M3), 64, 256, 512) == 3
     assert rg.rg_desc_validate(rg.rg_desc(in_dtype=4), 64, 256, 512) == 2
     assert rg.rg_desc_validate(rg.rg_desc(partial_dtype=K.RG_BF16), 64, 256, 512) == 0

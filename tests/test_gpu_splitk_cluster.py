@@ -43,6 +43,7 @@ def test_in_cluster_merge_matches_oracle_and_two_kernel_path(M, parts):
                           f"two kernels M={M} parts={parts} tree={tree} vs oracle")
         assert_bits_equal(gpu_gemm(A, B, cuts=cuts, tree=tree, residual=res), want, f"default path M={M} parts={parts}")
         assert_bits_equal(gpu_gemm(A, B, cuts=cuts, tree=tree, residual=res, b_static=1), want, f"static weights M={M} parts={parts}")
+        assert_bits_equal(gpu_gemm(A, B, cuts=cuts, tree=tree, residual=res, b_static=2), want, f"static operands M={M} parts={parts}")
         assert_bits_equal(gpu_gemm(A, B, cuts=cuts, tree=tree, residual=res, split_merge=LAST_ARRIVER), want, f"last-arriver merge M={M} parts={parts}")
 
 
@@ -213,4 +214,39 @@ def test_last_arriver_merge_reuses_its_workspace_and_leaves_the_tickets_zero():
         rg.rg_gemm(rg.rg_desc(cuts=tuple(64 * t for t in range(1, 10)), split_merge=LAST_ARRIVER), At, Bt, out, ws=ws)   # nine cuts: ten parts
     with pytest.raises(rg.RgError):
         rg.rg_gemm_noalloc(rg.rg_desc(cuts=cuts8, split_merge=LAST_ARRIVER), At, Bt, torch.empty((32, 4096), dtype=torch.bfloat16, device=DEV))
+    assert rg.rg_device_status() == 0
+
+
+def test_static_operands_in_a_run_of_independent_calls():
+    """b_static = 2 (neither operand is written by work in flight): the loads of a call start while the merge of the
+    call before it is still running; its stores wait.  A run of calls that share the workspace, back to back on one
+    stream, with and without cuts and on both kernels, gives the bits of the same calls made one at a time."""
+    cuts8 = tuple(1792 * t for t in range(1, 8))
+    A, _ = _inputs(32, 8, 14336, 21, spread=False)
+    At = synth.to_torch(A, DEV)
+    Ws = [synth.device_normal((4096, 14336), 0.02, 30 + i, torch.bfloat16, DEV) for i in range(3)]
+    res = synth.device_normal((32, 4096), 1.0, 40, torch.bfloat16, DEV)
+    d = rg.rg_desc(cuts=cuts8, b_static=2)
+    ws = torch.empty(rg.rg_gemm_workspace_bytes(d, 32, 4096), dtype=torch.uint8, device=DEV)
+    alone = [gpu_gemm(At, W, cuts=cuts8, residual=res) for W in Ws]
+    outs = [torch.empty((32, 4096), dtype=torch.bfloat16, device=DEV) for _ in range(12)]
+    for o in outs: o.view(torch.int16).fill_(-1)
+    torch.cuda.synchronize()
+    for i, o in enumerate(outs):
+        rg.rg_gemm(d, At, Ws[i % 3], o, residual=res, ws=ws)
+    torch.cuda.synchronize()
+    for i, o in enumerate(outs):
+        assert_bits_equal(synth.from_torch(o), alone[i % 3], f"call {i} of the run")
+    # large tiles without cuts (the two-SM kernel), alternating with the split-K calls above on the same stream
+    X = synth.device_normal((600, 2048), 1.0, 50, torch.bfloat16, DEV); Wb = synth.device_normal((1500, 2048), 0.05, 51, torch.bfloat16, DEV)
+    ref = gpu_gemm(X, Wb)
+    d2 = rg.rg_desc(b_static=2)
+    big = [torch.empty((600, 1500), dtype=torch.bfloat16, device=DEV) for _ in range(4)]
+    for i, o in enumerate(big):
+        rg.rg_gemm(d2, X, Wb, o)
+        rg.rg_gemm(d, At, Ws[i % 3], outs[i], residual=res, ws=ws)
+    torch.cuda.synchronize()
+    for i, o in enumerate(big):
+        assert_bits_equal(synth.from_torch(o), ref, f"two-SM call {i}")
+        assert_bits_equal(synth.from_torch(outs[i]), alone[i % 3], f"split-K call {i} between them")
     assert rg.rg_device_status() == 0
