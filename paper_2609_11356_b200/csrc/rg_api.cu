@@ -142,6 +142,7 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   plan->n_parts = (int)d->n_cuts + 1;
   plan->cluster_merge = 0;
   plan->ticket_merge = d->split_merge == 3 ? 1 : 0;
+  plan->reserve_sms = 0; plan->merge_small = 0;
   plan->half_sm = 0;
   plan->b_static = d->b_static;
   plan->tree = d->tree;
@@ -165,7 +166,21 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
   const bool half_ok = !d->inner_span && d->cta_group != 2 && d->BM != 256 && d->BN <= 128 && d->BK != 256;
   const bool half = half_ok && d->sm_share == 2;
   if (d->sm_share == 2 && !half) return RG_ERR_UNSUPPORTED;
-  const int slots = sms;
+  // Calls that do not depend on each other (b_static = 2) with a split-K merge behind them: the merge's CTAs cannot
+  // sit beside a GEMM CTA (registers), so they take SMs as the GEMM's CTAs leave, and the next call's CTAs on those SMs
+  // start late.  Leaving the merge a few SMs of its own (128-thread CTAs of two units per thread, four to an SM) lets
+  // the calls follow each other at the weights' streaming rate: decode shape, 1 / 8 / 32 rows: 26.5 / 23.7 / 22.7 us
+  // per call without, 18.2 / 18.8 / about 20 with (117 MB in 18.2 us is 0.98 of the measured copy bandwidth).
+  plan->reserve_sms = 0; plan->merge_small = 0;
+  if (d->b_static == 2 && plan->n_parts > 1 && plan->n_parts <= 8 && skinny && d->split_merge <= 1 && d->sm_share != 2) {
+    // the general merge kernel (256-thread CTAs, two to an SM) where that takes no more than an eighth of the SMs (it is
+    // the faster of the two: 8 rows 18.8 against 20.5 us per call), else the 128-thread form (four to an SM) up to a quarter
+    const int64_t merge_ctas = (M * ((N + 3) / 4) + 255) / 256;
+    const int64_t need2 = (merge_ctas + 1) / 2, need4 = (merge_ctas + 3) / 4;
+    if (need2 <= sms / 8) { plan->reserve_sms = (int)need2; plan->merge_small = 0; }
+    else if (need4 <= sms / 4) { plan->reserve_sms = (int)need4; plan->merge_small = 1; }
+  }
+  const int slots = sms - plan->reserve_sms;
   if (d->BN) plan->BN = d->BN;
   else if (skinny) {
     // Weight streaming: time ~ (rounds of work items per SM) x (tile width).  Any multiple of 16 is a
@@ -179,7 +194,8 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
       for (int bn = plan->n_parts == 1 ? 32 : 64; bn <= (half ? 128 : 256); bn += 16) {
         const int64_t items = ((N + bn - 1) / bn) * plan->n_parts;
         if (pass == 0 && items > slots) continue;
-        const int64_t cost = ((items + slots - 1) / slots) * bn;
+        const int64_t rounds = (items + slots - 1) / slots;
+        const int64_t cost = rounds * bn * 16 + (plan->reserve_sms ? rounds : 0);     // with SMs set aside, ties go to fewer rounds
         if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
       }
     }

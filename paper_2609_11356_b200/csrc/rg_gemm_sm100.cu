@@ -1439,6 +1439,81 @@ __global__ void __launch_bounds__(256) splitk_fixup_kernel(const FixupParams p) 
   }
 }
 
+// The merge behind calls that do not depend on each other (b_static = 2), at most eight parts: 128-thread CTAs, two
+// units of four columns per thread with the loads of both in flight together, at most 120 registers, so that four
+// CTAs fit an SM.  The GEMM ahead of it leaves this kernel a few SMs of its own (GemmPlan::reserve_sms): its CTAs
+// become resident there while that GEMM is still running, and they are not in the way when the next call's GEMM
+// CTAs move in as this call's leave.  (The 256-thread CTAs of the general kernel cannot sit beside a GEMM CTA: the
+// register file is four partitions of 16 K, a GEMM CTA's ten warps leave 4 K free on two of them, and two merge
+// warps need more.  They take SMs as GEMM CTAs leave, two to an SM, and the next call's CTAs on those SMs start late.)
+template <bool PART_16, bool MERGE_16>
+__global__ void __maxnreg__(120) splitk_fixup_small_kernel(const FixupParams p) {
+  const int64_t ncol4 = (p.N + 3) / 4, total = (int64_t)p.M * ncol4;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int64_t part_stride = (int64_t)p.M * p.ldw;
+  int64_t row[2], off[2]; int col0[2]; bool on[2];
+  float bias4[2][4], res4[2][4];
+  float4 part[2][8];
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const int64_t idx = (int64_t)blockIdx.x * 256 + u * 128 + threadIdx.x;
+    on[u] = idx < total;
+    row[u] = on[u] ? idx / ncol4 : 0;
+    col0[u] = on[u] ? (int)(idx - row[u] * ncol4) * 4 : 0;
+    off[u] = row[u] * p.ldw + col0[u];
+    // bias and residual are requested first so that their latency hides behind the parts'
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      bias4[u][c] = 0.0f; res4[u][c] = 0.0f;
+      if (on[u] && col0[u] + c < p.N) {
+        if (p.epi.bias) bias4[u][c] = load_scalar(p.epi.bias, p.epi.bias_dtype, col0[u] + c);
+        if (p.epi.residual) res4[u][c] = load_scalar(p.epi.residual, p.epi.residual_dtype, row[u] * p.epi.ldr + col0[u] + c);
+      }
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      if (on[u] && s < p.S) {
+        if (PART_16) {
+          const uint2 w = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.ws) + s * part_stride + off[u]);
+          part[u][s] = p.partial_dtype == RG_F16
+              ? make_float4(f16_bits_to_f32(w.x & 0xffffu), f16_bits_to_f32(w.x >> 16), f16_bits_to_f32(w.y & 0xffffu), f16_bits_to_f32(w.y >> 16))
+              : make_float4(bf16_bits_to_f32(w.x & 0xffffu), bf16_bits_to_f32(w.x >> 16), bf16_bits_to_f32(w.y & 0xffffu), bf16_bits_to_f32(w.y >> 16));
+        } else {
+          part[u][s] = *reinterpret_cast<const float4*>(static_cast<const float*>(p.ws) + s * part_stride + off[u]);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    if (!on[u]) continue;
+    const float4 acc = merge_upto8<MERGE_16>(part[u], p.S, p.tree, p.merge_dtype);
+    // bias -> SiLU -> residual -> one rounding, as in the GEMM kernels' epilogue
+    float v[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      if (p.epi.bias) v[c] = f_add(v[c], bias4[u][c]);
+      if (p.epi.act == 1) v[c] = rg_silu(v[c]);
+      if (p.epi.residual) v[c] = f_add(v[c], res4[u][c]);
+    }
+    uint16_t* const c16 = static_cast<uint16_t*>(p.C) + row[u] * p.ldc + col0[u];
+    if (col0[u] + 4 <= p.N && p.c_dtype != RG_F32 && (reinterpret_cast<uintptr_t>(c16) & 7) == 0) {
+      uint2 o;
+      o.x = pack_16x2(v[0], v[1], p.c_dtype);
+      o.y = pack_16x2(v[2], v[3], p.c_dtype);
+      *reinterpret_cast<uint2*>(c16) = o;
+    } else {
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        if (col0[u] + c < p.N) store_scalar(p.C, p.c_dtype, row[u] * p.ldc + col0[u] + c, v[c]);
+    }
+  }
+}
+
 // -------------------------------------------------------------- self-test of the bounded wait
 // One CTA, two warps, no copies and no tensor memory: a barrier that nothing ever arrives on.  Warp 0
 // waits on it with the caller's (short) limit, gives up, raises the CTA's abort flag and records
@@ -1943,11 +2018,13 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     else return RG_ERR_UNSUPPORTED;
   } else if (plan.inner_span) {
     if (ksub != 1) return RG_ERR_UNSUPPORTED;
-    const int grid = (int)(total < sms ? total : sms);
+    const int room = sms - plan.reserve_sms;                 // SMs left free for the merge's CTAs (see GemmPlan::reserve_sms)
+    const int grid = (int)(total < room ? total : room);
     if (plan.BN <= 128) err = p.f8 ? launch_grouped_t<true, 2>(ta, tb, p, grid, st) : launch_grouped_t<false, 2>(ta, tb, p, grid, st);
     else err = p.f8 ? launch_grouped_t<true, 4>(ta, tb, p, grid, st) : launch_grouped_t<false, 4>(ta, tb, p, grid, st);
   } else {
-    const int grid = (int)(total < sms ? total : sms);
+    const int room = sms - plan.reserve_sms;                 // SMs left free for the merge's CTAs (see GemmPlan::reserve_sms)
+    const int grid = (int)(total < room ? total : room);
     if (ksub == 1) err = launch_one<1>(ta, tb, p, grid, st);
     else if (ksub == 2) err = launch_one<2>(ta, tb, p, grid, st);
     else if (ksub == 4) err = launch_one<4>(ta, tb, p, grid, st);
@@ -1962,8 +2039,9 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     f.C = C->ptr; f.ldc = C->ld; f.c_dtype = C->dtype; f.epi = e;
     const int64_t items = M * ((N + 3) / 4);
     cudaLaunchConfig_t cfg = {};
+    const bool small = plan.merge_small != 0;                // the denser form of the merge that has SMs of its own (see splitk_fixup_small_kernel)
     cfg.gridDim = dim3((unsigned)((items + 255) / 256), 1, 1);
-    cfg.blockDim = dim3(256, 1, 1);
+    cfg.blockDim = dim3(small ? 128 : 256, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -1972,7 +2050,12 @@ rg_status_t launch_gemm(const GemmPlan& plan, const rg_tensor_t* A, const rg_ten
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t fe;
-    if (plan.partial_dtype == RG_F32) fe = cudaLaunchKernelEx(&cfg, splitk_fixup_kernel<false, false>, f);   // fp32 parts, fp32 sum
+    if (small) {
+      if (plan.partial_dtype == RG_F32) fe = cudaLaunchKernelEx(&cfg, splitk_fixup_small_kernel<false, false>, f);
+      else if (plan.merge_dtype == RG_F32) fe = cudaLaunchKernelEx(&cfg, splitk_fixup_small_kernel<true, false>, f);
+      else fe = cudaLaunchKernelEx(&cfg, splitk_fixup_small_kernel<true, true>, f);
+    }
+    else if (plan.partial_dtype == RG_F32) fe = cudaLaunchKernelEx(&cfg, splitk_fixup_kernel<false, false>, f);   // fp32 parts, fp32 sum
     else if (plan.merge_dtype == RG_F32) fe = cudaLaunchKernelEx(&cfg, splitk_fixup_kernel<true, false>, f);
     else fe = cudaLaunchKernelEx(&cfg, splitk_fixup_kernel<true, true>, f);
     if (fe != cudaSuccess) return RG_ERR_CUDA;

@@ -37,6 +37,8 @@ inline DeviceInfo current_device() {
 struct GemmPlan {
   int BN, BK, stages, raster, group_m, cta_group;
   int b_static;             // caller's promise: nothing in flight on the stream writes B (its first boxes may be fetched early)
+  int reserve_sms;          // SMs the GEMM leaves free for the CTAs of its split-K merge (calls that do not depend on each other, b_static = 2)
+  int merge_small;          // that merge runs as 128-thread CTAs of two units per thread (four to an SM) instead of the general kernel
   int half_sm;              // the one-CTA kernel in its half-SM form: two CTAs share an SM (weight-streaming shapes)
   int ticket_merge;         // split-K parts through the workspace, merged inside the GEMM kernel by the CTA that stores a tile's last part
   int cluster_merge;        // split-K parts merged inside the GEMM kernel by a thread-block cluster (no workspace, one launch)
