@@ -195,7 +195,9 @@ rg_status_t make_plan(const rg_desc_t* d, int64_t M, int64_t N, int64_t K, rg::G
         const int64_t items = ((N + bn - 1) / bn) * plan->n_parts;
         if (pass == 0 && items > slots) continue;
         const int64_t rounds = (items + slots - 1) / slots;
-        const int64_t cost = rounds * bn * 16 + (plan->reserve_sms ? rounds : 0);     // with SMs set aside, ties go to fewer rounds
+        // with SMs set aside for the merge a round costs about 24 columns' worth beside its width (4 rows: three rounds of
+        // 80-wide tiles 22 us per call, one round of 256-wide tiles 19)
+        const int64_t cost = rounds * (bn + (plan->reserve_sms ? 24 : 0));
         if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
       }
     }
