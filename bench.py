@@ -316,6 +316,12 @@ def run_ours(args):
             it[0] += 1
             rg.rg_gemm(d_indep, T["dc_X"], Ws[it[0] % 4], cd, residual=T["dc_R"], ws=ws)
         ms_dec_indep = timed(decode_indep, 40, busy)
+        d_gemv_indep = rg.rg_desc(atom=rg.RG_ATOM_SCALAR, fma=1, b_static=2)
+        cg1 = torch.empty((1, 4096), dtype=bf, device=dev)
+        def gemv_indep():
+            it[0] += 1
+            rg.rg_gemm(d_gemv_indep, T["dc_X"][:1], Ws[it[0] % 4], cg1)
+        ms_gemv_indep = timed(gemv_indep, 40, busy)
         dv = rg.rg_desc(atom=rg.RG_ATOM_SCALAR, fma=1)
         x1 = T["dc_X"][:1]; c1 = cd[:1]
         def gemv():
@@ -356,7 +362,7 @@ def run_ours(args):
             "fp8_e4m3_square_tflops": round(2.0 * 8192 ** 3 / (ms8 * 1e-3) / 1e12, 1),
             "square_tflops_by_inner_span": span_tflops,
             "decode_splitk8_back_to_back_us": round(ms_dec * 1e3, 2), "decode_splitk8_weight_gbs": round(wbytes / (ms_dec * 1e-3) / 1e9, 1),
-            "decode_splitk8_independent_calls_us": round(ms_dec_indep * 1e3, 2),
+            "decode_splitk8_independent_calls_us": round(ms_dec_indep * 1e3, 2), "gemv_m1_independent_calls_us": round(ms_gemv_indep * 1e3, 2),
             "gemv_m1_back_to_back_us": round(ms_gemv * 1e3, 2), "gemv_m1_weight_gbs": round(wbytes / (ms_gemv * 1e-3) / 1e9, 1),
             "col_sum_65536x32768_gbs": round(4.0 * RED_R * RED_C / (ms_col * 1e-3) / 1e9, 1),
             "attention_32x4096x4096x128_base2_w128_tflops": round(4.0 * aH * aN * aN * ad_ / (ms_att * 1e-3) / 1e12, 1),

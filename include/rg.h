@@ -121,7 +121,9 @@ typedef struct {
                              before the kernels ahead of it have finished (A is not read early).  2 = the same
                              promise for A and B (calls that share an input, or whose input was complete before the work
                              now in flight was enqueued): no load of the call waits for the kernels ahead; its stores to
-                             C and to the workspace still do.  0 = no promise */
+                             C and to the workspace still do, and a split-K call leaves its merge a few SMs of its own so
+                             that such calls follow each other at the weights' streaming rate.  Honoured by the
+                             tensor-core kernels and the GEMV family.  0 = no promise */
 } rg_desc_t;
 
 /* A row-major matrix in device memory. */

@@ -30,6 +30,7 @@ struct GemvParams {
   int64_t lda, ldb, ldc;
   int32_t M, N, K;
   int32_t fma, layout, fold, c_dtype;
+  int32_t b_static;       // 2: the caller's promise that neither operand is written by work in flight (loads do not wait for it)
   EpilogueArgs epi;
 };
 
@@ -91,7 +92,10 @@ __global__ void __launch_bounds__(GEMV_THREADS, 7) gemv_lane_tree_kernel(const G
   // launched with programmatic stream serialisation: a kernel queued behind this one may start
   // its own set-up now, and this one reads nothing before the kernels ahead of it have finished
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // (with the promise that neither operand is written by work in flight, b_static = 2, only the epilogue's reads and
+  // the stores wait for the kernels ahead)
+  bool deps_done = p.b_static < 2;
+  if (deps_done) asm volatile("griddepcontrol.wait;" ::: "memory");
   for (int64_t j = warp0; j < p.N; j += nwarps) {
     const uint16_t* brow = p.B + j * p.ldb;
     for (int m0 = 0; m0 < p.M; m0 += MR) {
@@ -174,6 +178,7 @@ __global__ void __launch_bounds__(GEMV_THREADS, 7) gemv_lane_tree_kernel(const G
         for (int r = 0; r < MR; ++r) acc[r] = f_add(acc[r], __shfl_xor_sync(0xffffffffu, acc[r], off));
       }
       if (lane == 0) {
+        if (!deps_done) { asm volatile("griddepcontrol.wait;" ::: "memory"); deps_done = true; }
 #pragma unroll
         for (int r = 0; r < MR; ++r) {
           if (m0 + r < p.M) {
@@ -217,7 +222,7 @@ rg_status_t launch_gemv(const rg_desc_t* d, const rg_tensor_t* A, const rg_tenso
   p.A = static_cast<const uint16_t*>(A->ptr); p.B = static_cast<const uint16_t*>(B->ptr); p.C = C->ptr;
   p.lda = A->ld; p.ldb = B->ld; p.ldc = C->ld;
   p.M = (int32_t)A->rows; p.N = (int32_t)B->rows; p.K = (int32_t)A->cols;
-  p.fma = d->fma; p.layout = d->gemv_layout; p.fold = d->gemv_fold; p.c_dtype = C->dtype;
+  p.fma = d->fma; p.layout = d->gemv_layout; p.fold = d->gemv_fold; p.c_dtype = C->dtype; p.b_static = d->b_static;
   EpilogueArgs e{};
   if (epi) {
     e.bias = epi->bias; e.bias_dtype = epi->bias_dtype; e.act = epi->act;

@@ -249,4 +249,15 @@ def test_static_operands_in_a_run_of_independent_calls():
     for i, o in enumerate(big):
         assert_bits_equal(synth.from_torch(o), ref, f"two-SM call {i}")
         assert_bits_equal(synth.from_torch(outs[i]), alone[i % 3], f"split-K call {i} between them")
+    # the GEMV family under the same promise: its loads do not wait either, its epilogue reads and stores do
+    dv = rg.rg_desc(atom=rg.RG_ATOM_SCALAR, fma=1, b_static=2)
+    alone_v = [gpu_gemm(At[:2], W, atom=rg.RG_ATOM_SCALAR, fma=1, residual=res[:2]) for W in Ws]
+    outs_v = [torch.empty((2, 4096), dtype=torch.bfloat16, device=DEV) for _ in range(9)]
+    for o in outs_v: o.view(torch.int16).fill_(-1)
+    torch.cuda.synchronize()
+    for i, o in enumerate(outs_v):
+        rg.rg_gemm(dv, At[:2], Ws[i % 3], o, residual=res[:2])
+    torch.cuda.synchronize()
+    for i, o in enumerate(outs_v):
+        assert_bits_equal(synth.from_torch(o), alone_v[i % 3], f"GEMV call {i} of the run")
     assert rg.rg_device_status() == 0
