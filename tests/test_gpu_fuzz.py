@@ -34,6 +34,7 @@ def _case(g):
                  dict(cta_group=2, BN=192, BK=128)][int(g.integers(0, 9))]
     epi = {}
     out = [rgo.BF16, rgo.F32, rgo.F16][int(g.integers(0, 3))]
+    knobs = dict(knobs, b_static=int(g.integers(0, 3)))       # a promise about in-flight work: never moves a bit (with cuts and few rows it also changes the grid)
     return M, N, K, f16, desc, knobs, out
 
 
